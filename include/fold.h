@@ -1,0 +1,194 @@
+/*
+ * fold.h -- C ABI of the declared-reference ("fold") softmax-attention decode library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The library computes single-token decode attention over a BF16 key/value cache.  A
+ * finite per-row reference Z_i is fixed before the cache is scanned (Section 3, Eq. 2),
+ * so every weight 2^(s_ij - Z_i) is final when computed and the per-range pairs
+ * (A, L) = (sum_j 2^(s_ij - Z_i) v_j, sum_j 2^(s_ij - Z_i)) add across key ranges with no
+ * maximum compared and nothing rescaled (Prop. 1).  A per-call depth T cuts keys whose
+ * weight is below 2^-T: they keep their weight in L, add nothing to A, and their value
+ * rows are not read (Section 4, "Depth as a dial", Algorithm 1).
+ *
+ * Units.  Scores are base 2: s_ij = log2(e) * softmax_scale * <q_i, k_j> (Section 2).
+ * z, lse and depth_T are all in binades; natural-log lse = ln(2) * lse.
+ *
+ * Pointers.  Unless a comment says HOST, every pointer is a DEVICE pointer owned by the
+ * caller.  The library allocates, frees and retains nothing.  Every call enqueues work
+ * on `stream` and returns without synchronising the host.  Calls that share a workspace
+ * must be ordered by the caller (same stream, or events).
+ *
+ * Errors.  Functions return a fold_status.  Only host-detectable conditions are
+ * returned (bad arguments, unsupported shapes, workspace too small, a CUDA launch
+ * error).  Conditions found on the device are reported in `row_status` bits and in the
+ * workspace header (see fold_ws_header); no kernel traps, asserts or waits unboundedly.
+ */
+#ifndef FOLD_H_
+#define FOLD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *fold_stream;            /* a cudaStream_t; NULL is the legacy default stream */
+
+typedef enum fold_status {
+  FOLD_OK = 0,
+  FOLD_EINVAL = 1,        /* null / misaligned pointer, inconsistent sizes, T < 0 or NaN */
+  FOLD_EUNSUPPORTED = 2,  /* head_dim not in {64,128}, page_size not a power of two >= 16, ... */
+  FOLD_EWORKSPACE = 3,    /* workspace_bytes < fold_workspace_bytes(args) */
+  FOLD_ECUDA = 4          /* a CUDA runtime / driver call failed (launch error, no sm_100 device) */
+} fold_status;
+
+/* How the per-row reference Z_i (Section 3, "Choosing the reference") is obtained. */
+typedef enum fold_zmode {
+  FOLD_Z_ESTIMATE = 0,  /* the 192-key estimate: sink + 63 most recent keys exactly, plus a
+                           trimmed stratified estimate from 128 stratum centres; written to z[] */
+  FOLD_Z_GIVEN = 1,     /* caller supplies z[] (e.g. the lse of a previous step, or a cascade's
+                           flat estimate shared by all its levels) */
+  FOLD_Z_EXACT_MAX = 2, /* test mode: an extra full pass sets z = max_j s_ij; written to z[] */
+  FOLD_Z_ZERO = 3       /* z = 0 for every row; written to z[] */
+} fold_zmode;
+
+/* Bits of row_status[b * num_q_heads + h]. */
+enum {
+  FOLD_ROW_RANGE = 1,     /* L outside [2^-1, 2^100]: the range certificate of Section 3 failed;
+                             decode the row again with z = the returned lse */
+  FOLD_ROW_NONFINITE = 2, /* an output element or L is not finite */
+  FOLD_ROW_EMPTY = 4      /* the row has no keys: out = 0, lse = -inf */
+};
+
+/* A key/value cache view.  Elements are BF16; the head_dim elements of one (token, head)
+ * row are contiguous and every row starts on a 16-byte boundary (all strides, in
+ * elements, are multiples of 8).
+ *
+ * Contiguous (page_table == NULL): row (seq, tok, head) is at
+ *     k + seq*stride_seq + tok*stride_tok + head*stride_head,   tok < capacity.
+ * Paged (page_table != NULL): logical token j of sequence `seq` is row
+ *     (page = page_table[seq*max_pages_per_seq + j / page_size], j % page_size, head) at
+ *     k + page*stride_seq + (j % page_size)*stride_tok + head*stride_head.
+ * Rows at or beyond seqlens[seq] (and unused page tails) are never used, whatever they hold. */
+typedef struct fold_kv {
+  const void *k, *v;
+  int64_t stride_seq, stride_tok, stride_head;   /* elements */
+  const int32_t *page_table;                     /* [num_seqs, max_pages_per_seq] or NULL */
+  int32_t page_size;                             /* tokens per page, power of two >= 16; 0 if contiguous */
+  int32_t max_pages_per_seq;
+  int32_t num_pages;                             /* pages in the pool (paged) */
+  int32_t capacity;                              /* tokens allocated per sequence (contiguous) */
+  int32_t num_seqs;                              /* KV sequences */
+  const int32_t *seqlens;                        /* [num_seqs] keys per sequence */
+  int32_t max_seqlen;                            /* HOST upper bound on seqlens[]; sizes grids and slots */
+} fold_kv;
+
+/* One decode call.  `batch` requests with one query token each; request b reads KV
+ * sequence b / stack (stack consecutive requests share a sequence: stack = 1 for plain
+ * decode; a cascade's shared-prefix level stacks the query rows of all requests that hold
+ * the prefix, Section 4 "Value product" last sentence).  batch == kv.num_seqs * stack.
+ * Query head h reads KV head h / (num_q_heads / num_kv_heads). */
+typedef struct fold_args {
+  int32_t batch, num_q_heads, num_kv_heads, head_dim;  /* head_dim in {64, 128} */
+  int32_t stack;
+  const void *q;                       /* BF16 [batch, num_q_heads, head_dim], head_dim contiguous */
+  int64_t q_stride_b, q_stride_h;      /* elements, multiples of 8 */
+  fold_kv kv;
+  float softmax_scale;                 /* c; > 0, finite */
+  int32_t z_mode;                      /* fold_zmode */
+  float *z;                            /* [batch, num_q_heads] fp32, binades; read (GIVEN) or written */
+  float depth_T;                       /* binades, >= 0; INFINITY = dense decode */
+  int32_t num_splits;                  /* CTAs per (sequence, kv head); 0 = choose.  A scheduling
+                                          hint only: it never changes a bit of the result */
+  void *workspace;                     /* 256-byte aligned */
+  size_t workspace_bytes;              /* >= fold_workspace_bytes(args) */
+  void *out;                           /* BF16 [batch, num_q_heads, head_dim], contiguous */
+  float *lse;                          /* [batch, num_q_heads] base-2 log-sum-exp, or NULL */
+  int32_t *row_status;                 /* [batch, num_q_heads] bit flags, or NULL */
+} fold_args;
+
+/* First 64 bytes of every workspace, zeroed at the start of each scan. */
+typedef struct fold_ws_header {
+  uint32_t wait_timeouts;      /* != 0: a bounded on-chip wait gave up; the results are invalid */
+  uint32_t reserved;
+  uint64_t v_rows_fetched;     /* value rows actually requested from memory, all (seq, kv head) */
+  uint64_t v_rows_total;       /* value rows a dense decode would read (= keys scanned) */
+  uint64_t v_slices_skipped;   /* 16-key slices of a tile whose value work was skipped entirely */
+  uint64_t pad[4];
+} fold_ws_header;
+
+/* The (A, L) partial pairs one scan leaves in its workspace (Algorithm 1, last line).
+ * The key axis of every sequence is cut into canonical chunks of fold_chunk_keys(n) keys,
+ * aligned to absolute key index; chunk c of (seq, kv head) owns slot c:
+ *     slot = slots + ((seq*num_kv_heads + kvh)*max_slots + c) * slot_stride   (floats)
+ *     A[r][d] = slot[r*head_dim + d],  L[r] = slot[rows*head_dim + r],
+ *     r = (request % stack) * group + (q head % group),  rows = stack * group.
+ * Slots 0 .. fold_num_chunks(seqlens[seq])-1 are valid; the rest are never read.  A slot's
+ * content depends only on (q rows, that chunk's keys/values, z, T): not on num_splits,
+ * batch composition or cache layout.  Partial sets can be added only if they were
+ * scanned under the same z. */
+typedef struct fold_partials {
+  float *slots;
+  const int32_t *seqlens;      /* [num_seqs], the scanned sequence lengths */
+  const float *z;              /* [batch, num_q_heads] the reference the partials were formed under */
+  int32_t batch, num_q_heads, num_kv_heads, head_dim, stack;
+  int32_t num_seqs, max_slots, rows;
+  int32_t max_seqlen;          /* the HOST bound the slots were sized for */
+  int64_t slot_stride;         /* floats */
+} fold_partials;
+
+/* Keys per canonical chunk for a sequence of n keys, and the number of chunks.  Pure
+ * host functions of n (and of nothing else), so results cannot depend on the batch. */
+int32_t fold_chunk_keys(int32_t n);
+int32_t fold_num_chunks(int32_t n);
+
+/* Bytes of workspace fold_decode / fold_decode_split need for `args` (header + slots).
+ * Depends only on shapes and kv.max_seqlen.  Returns 0 if args is invalid. */
+size_t fold_workspace_bytes(const fold_args *args);
+
+/* Reference estimate (Section 3): writes levels[0]->z for every (request, q head).
+ * The logical key sequence of request b is the concatenation of its sequences in
+ * levels[0], levels[1], ... (a cascade's prefix then suffix; Appendix "Cascades and
+ * drafts": the cascade takes its references from the flat estimate).  q, z and the head
+ * counts are taken from levels[0]; each level contributes its kv and stack.  n_levels
+ * in 1..4.  `levels` is a HOST array of HOST pointers. */
+int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream stream);
+
+/* Scan only (Algorithm 1 with a BF16 cache): obtains z per args->z_mode, scores every key
+ * against it, accumulates FP32 (A, L) per canonical chunk into args->workspace and fills
+ * *dst (HOST struct) describing them.  out / lse / row_status are not touched. */
+int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream stream);
+
+/* Order-free partial add (Prop. 1(i); summation on a declared integer grid, Eq. 3 /
+ * Prop. 2, so that the result is a function of the SET of partials): for every
+ * (request, q head) adds all valid slots of all levels, writes out = A / L (BF16, round
+ * to nearest even), lse = z + log2 L and row_status.  Used for the split-KV merge
+ * (n_levels = 1) and the shared-prefix cascade (prefix level + suffix level).  All levels
+ * must describe the same batch / heads / head_dim and the same z.  `levels` is a HOST
+ * array of HOST pointers to HOST structs; n_levels in 1..4. */
+int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *out, float *lse,
+                       int32_t *row_status, fold_stream stream);
+
+/* Whole decode: reference (per z_mode) -> scan -> partial add.  Equivalent to
+ * fold_decode_split followed by fold_cascade_merge over its one level. */
+int fold_decode(const fold_args *args, fold_stream stream);
+
+/* The same decode for callers whose tensors live in HOST memory (pinned for the copies to
+ * be asynchronous): q, kv.k, kv.v, kv.page_table, kv.seqlens, z (if GIVEN), out, lse and
+ * row_status of *host_args are HOST pointers laid out as described above (the cache is
+ * copied as the single span its strides cover).  `staging` is DEVICE memory of at least
+ * fold_host_staging_bytes(host_args) bytes, 256-byte aligned, which receives the copies,
+ * the workspace and the results before they are copied back.  Everything is enqueued on
+ * `stream`; the host buffers are valid after the caller synchronises the stream. */
+size_t fold_host_staging_bytes(const fold_args *host_args);
+int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_bytes, fold_stream stream);
+
+const char *fold_status_string(int status);
+/* Library version as major*10000 + minor*100 + patch. */
+int fold_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FOLD_H_ */

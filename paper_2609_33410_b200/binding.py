@@ -1,0 +1,260 @@
+"""ctypes binding of the fold decode C ABI (include/fold.h).
+
+Argument marshalling only: every step of the decode path runs in the CUDA library.  The
+library is loaded from the in-tree shared object; if it is missing it is built with nvcc,
+and if that fails the import fails -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+# ------------------------------------------------------------------ C structs (mirror include/fold.h)
+FOLD_OK, FOLD_EINVAL, FOLD_EUNSUPPORTED, FOLD_EWORKSPACE, FOLD_ECUDA = range(5)
+Z_ESTIMATE, Z_GIVEN, Z_EXACT_MAX, Z_ZERO = range(4)
+ROW_RANGE, ROW_NONFINITE, ROW_EMPTY = 1, 2, 4
+
+
+class FoldKV(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p),
+                ("stride_seq", C.c_int64), ("stride_tok", C.c_int64), ("stride_head", C.c_int64),
+                ("page_table", C.c_void_p), ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32),
+                ("num_pages", C.c_int32), ("capacity", C.c_int32), ("num_seqs", C.c_int32),
+                ("seqlens", C.c_void_p), ("max_seqlen", C.c_int32)]
+
+
+class FoldArgs(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("stack", C.c_int32),
+                ("q", C.c_void_p), ("q_stride_b", C.c_int64), ("q_stride_h", C.c_int64),
+                ("kv", FoldKV),
+                ("softmax_scale", C.c_float), ("z_mode", C.c_int32), ("z", C.c_void_p),
+                ("depth_T", C.c_float), ("num_splits", C.c_int32),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("out", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p)]
+
+
+class FoldPartials(C.Structure):
+    _fields_ = [("slots", C.c_void_p), ("seqlens", C.c_void_p), ("z", C.c_void_p),
+                ("batch", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("stack", C.c_int32),
+                ("num_seqs", C.c_int32), ("max_slots", C.c_int32), ("rows", C.c_int32),
+                ("max_seqlen", C.c_int32), ("slot_stride", C.c_int64)]
+
+
+class FoldWsHeader(C.Structure):
+    _fields_ = [("wait_timeouts", C.c_uint32), ("reserved", C.c_uint32),
+                ("v_rows_fetched", C.c_uint64), ("v_rows_total", C.c_uint64),
+                ("v_slices_skipped", C.c_uint64), ("pad", C.c_uint64 * 4)]
+
+
+EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
+           "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_host_staging_bytes",
+           "fold_decode_host", "fold_status_string", "fold_version"]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded CUDA library.  Raises if it cannot be built or loaded."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        L.fold_chunk_keys.restype = C.c_int32; L.fold_chunk_keys.argtypes = [C.c_int32]
+        L.fold_num_chunks.restype = C.c_int32; L.fold_num_chunks.argtypes = [C.c_int32]
+        L.fold_workspace_bytes.restype = C.c_size_t; L.fold_workspace_bytes.argtypes = [C.POINTER(FoldArgs)]
+        L.fold_estimate_z.restype = C.c_int
+        L.fold_estimate_z.argtypes = [C.POINTER(C.POINTER(FoldArgs)), C.c_int, C.c_void_p]
+        L.fold_decode_split.restype = C.c_int
+        L.fold_decode_split.argtypes = [C.POINTER(FoldArgs), C.POINTER(FoldPartials), C.c_void_p]
+        L.fold_cascade_merge.restype = C.c_int
+        L.fold_cascade_merge.argtypes = [C.POINTER(C.POINTER(FoldPartials)), C.c_int, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_void_p]
+        L.fold_decode.restype = C.c_int; L.fold_decode.argtypes = [C.POINTER(FoldArgs), C.c_void_p]
+        L.fold_host_staging_bytes.restype = C.c_size_t; L.fold_host_staging_bytes.argtypes = [C.POINTER(FoldArgs)]
+        L.fold_decode_host.restype = C.c_int
+        L.fold_decode_host.argtypes = [C.POINTER(FoldArgs), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.fold_status_string.restype = C.c_char_p; L.fold_status_string.argtypes = [C.c_int]
+        L.fold_version.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+class FoldError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib().fold_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != FOLD_OK:
+        raise FoldError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream=None) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+# ------------------------------------------------------------------ argument building
+@dataclass
+class KVCache:
+    """A BF16 cache view.  Contiguous: k, v [num_seqs, capacity, Hkv, D] (any strides with D
+    contiguous).  Paged: k, v [num_pages, page_size, Hkv, D] and page_table [num_seqs, max_pages]."""
+    k: torch.Tensor
+    v: torch.Tensor
+    seqlens: torch.Tensor
+    max_seqlen: int
+    page_table: Optional[torch.Tensor] = None
+
+    def to_c(self) -> FoldKV:
+        k, v = self.k, self.v
+        assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.dim() == 4
+        assert k.stride() == v.stride() and k.shape == v.shape and k.stride(3) == 1
+        assert self.seqlens.dtype == torch.int32 and self.seqlens.is_contiguous()
+        kv = FoldKV()
+        kv.k, kv.v = k.data_ptr(), v.data_ptr()
+        kv.stride_seq, kv.stride_tok, kv.stride_head = k.stride(0), k.stride(1), k.stride(2)
+        kv.seqlens = self.seqlens.data_ptr()
+        kv.num_seqs = self.seqlens.shape[0]
+        kv.max_seqlen = int(self.max_seqlen)
+        if self.page_table is not None:
+            pt = self.page_table
+            assert pt.dtype == torch.int32 and pt.is_contiguous() and pt.dim() == 2
+            kv.page_table = pt.data_ptr()
+            kv.page_size = k.shape[1]
+            kv.max_pages_per_seq = pt.shape[1]
+            kv.num_pages = k.shape[0]
+            kv.capacity = 0
+        else:
+            kv.page_table = None
+            kv.page_size = 0
+            kv.max_pages_per_seq = 0
+            kv.num_pages = 0
+            kv.capacity = k.shape[1]
+        return kv
+
+
+def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None, z_mode: int = Z_ESTIMATE,
+              z: Optional[torch.Tensor] = None, depth_T: float = math.inf, num_splits: int = 0, stack: int = 1,
+              workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+              lse: Optional[torch.Tensor] = None, row_status: Optional[torch.Tensor] = None) -> FoldArgs:
+    assert q.dtype == torch.bfloat16 and q.dim() == 3 and q.stride(2) == 1
+    B, Hq, D = q.shape
+    a = FoldArgs()
+    a.batch, a.num_q_heads, a.num_kv_heads, a.head_dim = B, Hq, cache.k.shape[2], D
+    a.stack = stack
+    a.q, a.q_stride_b, a.q_stride_h = q.data_ptr(), q.stride(0), q.stride(1)
+    a.kv = cache.to_c()
+    a.softmax_scale = float(scale if scale is not None else 1.0 / math.sqrt(D))
+    a.z_mode = z_mode
+    a.z = _ptr(z)
+    a.depth_T = float(depth_T)
+    a.num_splits = int(num_splits)
+    a.workspace = _ptr(workspace)
+    a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    a.out, a.lse, a.row_status = _ptr(out), _ptr(lse), _ptr(row_status)
+    return a
+
+
+def fold_workspace_bytes(args: FoldArgs) -> int:
+    return int(lib().fold_workspace_bytes(C.byref(args)))
+
+
+def fold_chunk_keys(n: int) -> int:
+    return int(lib().fold_chunk_keys(n))
+
+
+def fold_num_chunks(n: int) -> int:
+    return int(lib().fold_num_chunks(n))
+
+
+# ------------------------------------------------------------------ entry points (same names as the C ABI)
+def fold_estimate_z(levels: Sequence[FoldArgs], stream=None) -> None:
+    arr = (C.POINTER(FoldArgs) * len(levels))(*[C.pointer(a) for a in levels])
+    _check(lib().fold_estimate_z(arr, len(levels), _stream(stream)), "fold_estimate_z")
+
+
+def fold_decode_split(args: FoldArgs, stream=None) -> FoldPartials:
+    part = FoldPartials()
+    _check(lib().fold_decode_split(C.byref(args), C.byref(part), _stream(stream)), "fold_decode_split")
+    return part
+
+
+def fold_cascade_merge(levels: Sequence[FoldPartials], out: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                       row_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    arr = (C.POINTER(FoldPartials) * len(levels))(*[C.pointer(p) for p in levels])
+    _check(lib().fold_cascade_merge(arr, len(levels), out.data_ptr(), _ptr(lse), _ptr(row_status), _stream(stream)),
+           "fold_cascade_merge")
+
+
+def fold_decode(args: FoldArgs, stream=None) -> None:
+    _check(lib().fold_decode(C.byref(args), _stream(stream)), "fold_decode")
+
+
+def fold_host_staging_bytes(args: FoldArgs) -> int:
+    return int(lib().fold_host_staging_bytes(C.byref(args)))
+
+
+def fold_decode_host(host_args: FoldArgs, staging: torch.Tensor, stream=None) -> None:
+    _check(lib().fold_decode_host(C.byref(host_args), staging.data_ptr(), staging.numel() * staging.element_size(),
+                                  _stream(stream)), "fold_decode_host")
+
+
+# ------------------------------------------------------------------ small conveniences for tests and the benchmark
+@dataclass
+class DecodeBuffers:
+    out: torch.Tensor
+    lse: torch.Tensor
+    z: torch.Tensor
+    row_status: torch.Tensor
+    workspace: torch.Tensor
+
+    def header(self) -> FoldWsHeader:
+        raw = self.workspace[:64].cpu().numpy().tobytes()
+        return FoldWsHeader.from_buffer_copy(raw)
+
+
+def alloc_buffers(q: torch.Tensor, cache: KVCache, stack: int = 1) -> DecodeBuffers:
+    """Device buffers one decode call needs (torch is used for memory only)."""
+    B, Hq, D = q.shape
+    dev = q.device
+    probe = make_args(q, cache, stack=stack)
+    nbytes = fold_workspace_bytes(probe)
+    if nbytes == 0:
+        raise FoldError(FOLD_EINVAL, "fold_workspace_bytes")
+    return DecodeBuffers(out=torch.empty(B, Hq, D, dtype=torch.bfloat16, device=dev),
+                         lse=torch.empty(B, Hq, dtype=torch.float32, device=dev),
+                         z=torch.zeros(B, Hq, dtype=torch.float32, device=dev),
+                         row_status=torch.zeros(B, Hq, dtype=torch.int32, device=dev),
+                         workspace=torch.empty(nbytes, dtype=torch.uint8, device=dev))
+
+
+def decode(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, depth_T: float = math.inf,
+           z_mode: int = Z_ESTIMATE, num_splits: int = 0, scale: Optional[float] = None, stack: int = 1,
+           stream=None) -> FoldArgs:
+    args = make_args(q, cache, scale=scale, z_mode=z_mode, z=bufs.z, depth_T=depth_T, num_splits=num_splits,
+                     stack=stack, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status)
+    fold_decode(args, stream)
+    return args
+
+
+def slots_view(part: FoldPartials, workspace: torch.Tensor) -> torch.Tensor:
+    """FP32 view [num_seqs, Hkv, max_slots, slot_stride] of the partial slots inside `workspace`."""
+    off = part.slots - workspace.data_ptr()
+    n = part.num_seqs * part.num_kv_heads * part.max_slots * part.slot_stride
+    flat = workspace[off: off + 4 * n].view(torch.float32)
+    return flat.view(part.num_seqs, part.num_kv_heads, part.max_slots, part.slot_stride)

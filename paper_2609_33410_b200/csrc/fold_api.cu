@@ -1,0 +1,470 @@
+// C ABI of the fold decode library: argument checks, tensor-map creation, workspace
+// carving and kernel launches.  Nothing here allocates device memory or synchronises.
+#include <math.h>
+#include <string.h>
+
+#include "fold_common.cuh"
+#include "fold_estimate.cuh"
+#include "fold_merge.cuh"
+#include "fold_scan.cuh"
+
+using namespace fold;
+
+namespace {
+
+constexpr size_t kHeaderBytes = 256;
+constexpr int kSmemPerSm = 233472;       // 228 KB per SM
+constexpr int kSmemPerCtaMax = 232448;   // 227 KB opt-in per CTA
+constexpr int kSmemCtaReserve = 1024;
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
+
+struct Geometry {
+  int B, Hq, Hkv, G, D, stack, R, num_seqs, max_slots;
+  long long slot_stride;
+  size_t slot_bytes;
+};
+
+int check_kv(const fold_kv &kv, int D) {
+  if (!kv.k || !kv.v || !kv.seqlens) return FOLD_EINVAL;
+  if (!aligned(kv.k, 16) || !aligned(kv.v, 16)) return FOLD_EINVAL;
+  if (kv.num_seqs < 1 || kv.max_seqlen < 0) return FOLD_EINVAL;
+  if (kv.stride_tok < D || kv.stride_head < 0 || kv.stride_seq < 0) return FOLD_EINVAL;
+  if (kv.stride_tok % 8 || kv.stride_head % 8 || kv.stride_seq % 8) return FOLD_EINVAL;
+  if (kv.page_table) {
+    if (kv.page_size < 16 || (kv.page_size & (kv.page_size - 1))) return FOLD_EUNSUPPORTED;
+    if (kv.num_pages < 1 || kv.max_pages_per_seq < 1) return FOLD_EINVAL;
+    if ((long long)kv.max_pages_per_seq * kv.page_size < kv.max_seqlen) return FOLD_EINVAL;
+  } else {
+    if (kv.capacity < kv.max_seqlen || kv.capacity < 1) return FOLD_EINVAL;
+  }
+  return FOLD_OK;
+}
+
+int check_args(const fold_args *a, Geometry *g, bool need_out) {
+  if (!a) return FOLD_EINVAL;
+  if (a->head_dim != 64 && a->head_dim != 128) return FOLD_EUNSUPPORTED;
+  if (a->batch < 1 || a->num_q_heads < 1 || a->num_kv_heads < 1 || a->stack < 1) return FOLD_EINVAL;
+  if (a->num_q_heads % a->num_kv_heads) return FOLD_EINVAL;
+  if (a->batch % a->stack || a->batch / a->stack != a->kv.num_seqs) return FOLD_EINVAL;
+  if (!a->q || !aligned(a->q, 16) || a->q_stride_b % 8 || a->q_stride_h % 8) return FOLD_EINVAL;
+  if (a->q_stride_h < a->head_dim && a->num_q_heads > 1) return FOLD_EINVAL;
+  if (int rc = check_kv(a->kv, a->head_dim)) return rc;
+  if (!(a->softmax_scale > 0.f) || isinf(a->softmax_scale)) return FOLD_EINVAL;
+  if (a->z_mode < FOLD_Z_ESTIMATE || a->z_mode > FOLD_Z_ZERO) return FOLD_EINVAL;
+  if (!a->z || !aligned(a->z, 4)) return FOLD_EINVAL;
+  if (isnan(a->depth_T) || a->depth_T < 0.f) return FOLD_EINVAL;
+  if (a->num_splits < 0) return FOLD_EINVAL;
+  if (need_out && (!a->out || !aligned(a->out, 2))) return FOLD_EINVAL;
+  const int G = a->num_q_heads / a->num_kv_heads;
+  const long long R = (long long)a->stack * G;
+  if (R > kMaxRows) return FOLD_EUNSUPPORTED;
+  g->B = a->batch; g->Hq = a->num_q_heads; g->Hkv = a->num_kv_heads; g->G = G; g->D = a->head_dim;
+  g->stack = a->stack; g->R = (int)R; g->num_seqs = a->kv.num_seqs;
+  g->max_slots = max_chunks_upto(a->kv.max_seqlen);
+  if (g->max_slots < 1) g->max_slots = 1;
+  g->slot_stride = (long long)g->R * g->D + ((g->R + 3) / 4) * 4;
+  g->slot_bytes = (size_t)g->num_seqs * g->Hkv * g->max_slots * g->slot_stride * sizeof(float);
+  return FOLD_OK;
+}
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// 4-D view of a cache tensor: axis 0 is the channel, the token / head / sequence-or-page axes
+// follow in order of increasing stride (pos[] returns where each landed).  Box = 64 channels
+// x box_tok tokens, 128-byte swizzle, out-of-range elements read as zero.
+struct MapAxes { int pos_tok, pos_head, pos_seq; };
+
+int make_map(CUtensorMap *map, MapAxes *axes, const void *ptr, const fold_kv &kv, int D, int Hkv, int box_tok) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return FOLD_ECUDA;
+  const bool paged = kv.page_table != nullptr;
+  struct Axis { cuuint64_t extent, stride; cuuint32_t box; int id; };
+  Axis ax[3] = {{(cuuint64_t)(paged ? kv.page_size : kv.capacity), (cuuint64_t)kv.stride_tok * 2, (cuuint32_t)box_tok, 0},
+                {(cuuint64_t)Hkv, (cuuint64_t)kv.stride_head * 2, 1u, 1},
+                {(cuuint64_t)(paged ? kv.num_pages : kv.num_seqs), (cuuint64_t)kv.stride_seq * 2, 1u, 2}};
+  // extent-1 axes carry no information: sort them last, the rest by stride
+  for (int i = 0; i < 3; ++i)
+    for (int j = i + 1; j < 3; ++j) {
+      const bool i_one = ax[i].extent == 1, j_one = ax[j].extent == 1;
+      if ((i_one && !j_one) || (i_one == j_one && ax[j].stride < ax[i].stride)) { Axis t = ax[i]; ax[i] = ax[j]; ax[j] = t; }
+    }
+  cuuint64_t prev_stride = (cuuint64_t)D * 2, prev_extent = 1;
+  for (int i = 0; i < 3; ++i) {
+    if (ax[i].extent == 1 || ax[i].stride == 0) ax[i].stride = prev_stride * prev_extent;
+    prev_stride = ax[i].stride; prev_extent = ax[i].extent;
+  }
+  cuuint64_t dims[4] = {(cuuint64_t)D, ax[0].extent, ax[1].extent, ax[2].extent};
+  cuuint64_t strides[3] = {ax[0].stride, ax[1].stride, ax[2].stride};
+  cuuint32_t box[4] = {64u, ax[0].box, ax[1].box, ax[2].box};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  for (int i = 0; i < 3; ++i) {
+    if (ax[i].id == 0) axes->pos_tok = i + 1;
+    if (ax[i].id == 1) axes->pos_head = i + 1;
+    if (ax[i].id == 2) axes->pos_seq = i + 1;
+  }
+  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   D == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? FOLD_OK : FOLD_ECUDA;
+}
+
+// ------------------------------------------------------------------ launches
+KvLevel kv_level(const fold_kv &kv, int stack) {
+  KvLevel L;
+  L.k = static_cast<const __nv_bfloat16 *>(kv.k);
+  L.stride_seq = kv.stride_seq; L.stride_tok = kv.stride_tok; L.stride_head = kv.stride_head;
+  L.page_table = kv.page_table;
+  L.seqlens = kv.seqlens;
+  L.paged = kv.page_table != nullptr;
+  L.page_shift = L.paged ? ilog2(kv.page_size) : 0;
+  L.max_pages = kv.max_pages_per_seq;
+  L.num_pages = kv.num_pages > 0 ? kv.num_pages : 1;
+  L.stack = stack;
+  L.max_seqlen = kv.max_seqlen;
+  return L;
+}
+
+EstParams est_params(const fold_args *a, const Geometry &g) {
+  EstParams p;
+  memset(&p, 0, sizeof(p));
+  p.q = static_cast<const __nv_bfloat16 *>(a->q);
+  p.q_stride_b = a->q_stride_b; p.q_stride_h = a->q_stride_h;
+  p.z = a->z;
+  p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
+  p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
+  return p;
+}
+
+int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st) {
+  if (a->z_mode == FOLD_Z_GIVEN) return FOLD_OK;
+  const int rows = g.B * g.Hq;
+  if (a->z_mode == FOLD_Z_ZERO) {
+    fold_fill_kernel<<<(rows + 255) / 256, 256, 0, st>>>(a->z, rows, 0.f);
+  } else {
+    if (g.G > kMaxRows) return FOLD_EUNSUPPORTED;
+    EstParams p = est_params(a, g);
+    p.n_levels = 1;
+    p.lv[0] = kv_level(a->kv, a->stack);
+    const dim3 grid(g.Hkv, g.B);
+    if (a->z_mode == FOLD_Z_ESTIMATE) {
+      if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
+      else fold_estimate_kernel<64><<<grid, kEstThreads, 0, st>>>(p);
+    } else {
+      if (g.D == 128) fold_exact_max_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
+      else fold_exact_max_kernel<64><<<grid, kEstThreads, 0, st>>>(p);
+    }
+  }
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+template <int D, bool GATHER>
+int launch_scan_t(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LO = ScanLayout<D, GATHER>;
+  // two CTAs per SM when a useful ring fits, else one with a deeper ring
+  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  int stages, vr = GATHER ? 3 : 1;
+  const int fixed2 = LO::total(0, vr, p.R);
+  stages = (per_cta2 - fixed2) / (LO::kStage + 16);
+  if (stages < 3) {
+    const int fixed1 = LO::total(0, vr, p.R);
+    stages = (kSmemPerCtaMax - fixed1) / (LO::kStage + 16);
+  }
+  if (stages > 8) stages = 8;
+  if (stages < 2) return FOLD_EUNSUPPORTED;
+  p.stages = stages;
+  p.vr = vr;
+  const int smem = LO::total(stages, vr, p.R);
+  static int configured[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FOLD_ECUDA;
+  if (dev < 0 || dev >= 64 || configured[dev] < smem) {
+    if (cudaFuncSetAttribute(fold_scan_kernel<D, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSmemPerCtaMax) != cudaSuccess)
+      return FOLD_ECUDA;
+    if (dev >= 0 && dev < 64) configured[dev] = kSmemPerCtaMax;
+  }
+  fold_scan_kernel<D, GATHER><<<grid, kScanThreads, smem, st>>>(mk, mv, p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+int choose_splits(const fold_args *a, const Geometry &g) {
+  const int max_chunks = num_chunks_of(a->kv.max_seqlen) > 0 ? num_chunks_of(a->kv.max_seqlen) : 1;
+  if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
+  const long long units = (long long)g.num_seqs * g.Hkv;
+  const long long target = 8LL * 296;
+  long long per_cta = units * max_chunks / target;
+  if (per_cta < 1) per_cta = 1;
+  return (int)((max_chunks + per_cta - 1) / per_cta);
+}
+
+int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
+  const fold_kv &kv = a->kv;
+  const bool paged = kv.page_table != nullptr;
+  const int box_tok = paged ? (kv.page_size < kTileKeys ? kv.page_size : kTileKeys) : kTileKeys;
+  CUtensorMap mk, mv;
+  MapAxes axes;
+  if (int rc = make_map(&mk, &axes, kv.k, kv, g.D, g.Hkv, box_tok)) return rc;
+  if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, box_tok)) return rc;
+
+  ScanParams p;
+  memset(&p, 0, sizeof(p));
+  p.q = static_cast<const __nv_bfloat16 *>(a->q);
+  p.q_stride_b = a->q_stride_b; p.q_stride_h = a->q_stride_h;
+  p.z = a->z;
+  p.seqlens = kv.seqlens;
+  p.page_table = kv.page_table;
+  p.v = static_cast<const __nv_bfloat16 *>(kv.v);
+  p.v_stride_seq = kv.stride_seq; p.v_stride_tok = kv.stride_tok; p.v_stride_head = kv.stride_head;
+  p.slots = reinterpret_cast<float *>(static_cast<uint8_t *>(a->workspace) + kHeaderBytes);
+  p.slot_stride = g.slot_stride;
+  p.hdr = static_cast<fold_ws_header *>(a->workspace);
+  p.max_slots = g.max_slots; p.max_seqlen = kv.max_seqlen;
+  p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.stack = g.stack; p.R = g.R;
+  p.paged = paged; p.page_shift = paged ? ilog2(kv.page_size) : 0;
+  p.max_pages = kv.max_pages_per_seq; p.num_pages = kv.num_pages > 0 ? kv.num_pages : 1;
+  p.box_tok = box_tok;
+  p.pos_tok = axes.pos_tok; p.pos_head = axes.pos_head; p.pos_seq = axes.pos_seq;
+  p.num_splits = choose_splits(a, g);
+  p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
+  p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
+
+  if (cudaMemsetAsync(a->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
+  const dim3 grid(p.num_splits, g.Hkv, g.num_seqs);
+  const bool gather = !isinf(a->depth_T);
+  if (g.D == 128) return gather ? launch_scan_t<128, true>(mk, mv, p, grid, st) : launch_scan_t<128, false>(mk, mv, p, grid, st);
+  return gather ? launch_scan_t<64, true>(mk, mv, p, grid, st) : launch_scan_t<64, false>(mk, mv, p, grid, st);
+}
+
+void fill_partials(const fold_args *a, const Geometry &g, fold_partials *dst) {
+  dst->slots = reinterpret_cast<float *>(static_cast<uint8_t *>(a->workspace) + kHeaderBytes);
+  dst->seqlens = a->kv.seqlens;
+  dst->z = a->z;
+  dst->batch = g.B; dst->num_q_heads = g.Hq; dst->num_kv_heads = g.Hkv; dst->head_dim = g.D; dst->stack = g.stack;
+  dst->num_seqs = g.num_seqs; dst->max_slots = g.max_slots; dst->rows = g.R;
+  dst->slot_stride = g.slot_stride;
+  dst->max_seqlen = a->kv.max_seqlen;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t fold_chunk_keys(int32_t n) { return chunk_keys_of(n); }
+int32_t fold_num_chunks(int32_t n) { return n <= 0 ? 0 : num_chunks_of(n); }
+
+size_t fold_workspace_bytes(const fold_args *args) {
+  Geometry g;
+  fold_args tmp;
+  if (!args) return 0;
+  tmp = *args;
+  // sizing must not depend on pointers the caller has not allocated yet
+  if (tmp.head_dim != 64 && tmp.head_dim != 128) return 0;
+  if (tmp.batch < 1 || tmp.num_q_heads < 1 || tmp.num_kv_heads < 1 || tmp.stack < 1) return 0;
+  if (tmp.num_q_heads % tmp.num_kv_heads || tmp.batch % tmp.stack) return 0;
+  const int G = tmp.num_q_heads / tmp.num_kv_heads;
+  const long long R = (long long)tmp.stack * G;
+  if (R > kMaxRows || tmp.kv.max_seqlen < 0) return 0;
+  g.max_slots = max_chunks_upto(tmp.kv.max_seqlen);
+  if (g.max_slots < 1) g.max_slots = 1;
+  g.slot_stride = R * tmp.head_dim + ((R + 3) / 4) * 4;
+  return kHeaderBytes + (size_t)(tmp.batch / tmp.stack) * tmp.num_kv_heads * g.max_slots * g.slot_stride * sizeof(float);
+}
+
+int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream stream) {
+  if (!levels || n_levels < 1 || n_levels > kMaxLevels) return FOLD_EINVAL;
+  const fold_args *a0 = levels[0];
+  if (!a0) return FOLD_EINVAL;
+  if (a0->head_dim != 64 && a0->head_dim != 128) return FOLD_EUNSUPPORTED;
+  if (a0->batch < 1 || a0->num_q_heads < 1 || a0->num_kv_heads < 1 || a0->num_q_heads % a0->num_kv_heads)
+    return FOLD_EINVAL;
+  if (!a0->q || !a0->z || !aligned(a0->q, 16) || a0->q_stride_b % 8 || a0->q_stride_h % 8) return FOLD_EINVAL;
+  if (!(a0->softmax_scale > 0.f) || isinf(a0->softmax_scale)) return FOLD_EINVAL;
+  const int G = a0->num_q_heads / a0->num_kv_heads;
+  if (G > kMaxRows) return FOLD_EUNSUPPORTED;
+  Geometry g;
+  g.B = a0->batch; g.Hq = a0->num_q_heads; g.Hkv = a0->num_kv_heads; g.G = G; g.D = a0->head_dim;
+  EstParams p = est_params(a0, g);
+  p.n_levels = n_levels;
+  for (int l = 0; l < n_levels; ++l) {
+    const fold_args *a = levels[l];
+    if (!a || a->head_dim != a0->head_dim || a->num_kv_heads != a0->num_kv_heads || a->batch != a0->batch)
+      return FOLD_EINVAL;
+    if (a->stack < 1 || a->batch % a->stack || a->batch / a->stack != a->kv.num_seqs) return FOLD_EINVAL;
+    if (int rc = check_kv(a->kv, a->head_dim)) return rc;
+    p.lv[l] = kv_level(a->kv, a->stack);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const dim3 grid(g.Hkv, g.B);
+  if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
+  else fold_estimate_kernel<64><<<grid, kEstThreads, 0, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream stream) {
+  Geometry g;
+  if (int rc = check_args(args, &g, false)) return rc;
+  if (!dst) return FOLD_EINVAL;
+  if (!args->workspace || !aligned(args->workspace, 256)) return FOLD_EINVAL;
+  if (args->workspace_bytes < kHeaderBytes + g.slot_bytes) return FOLD_EWORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (int rc = launch_reference(args, g, st)) return rc;
+  if (int rc = launch_scan(args, g, st)) return rc;
+  fill_partials(args, g, dst);
+  return FOLD_OK;
+}
+
+int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *out, float *lse, int32_t *row_status,
+                       fold_stream stream) {
+  if (!levels || n_levels < 1 || n_levels > kMaxLevels || !out) return FOLD_EINVAL;
+  const fold_partials *p0 = levels[0];
+  if (!p0) return FOLD_EINVAL;
+  if (p0->head_dim != 64 && p0->head_dim != 128) return FOLD_EUNSUPPORTED;
+  MergeParams p;
+  memset(&p, 0, sizeof(p));
+  for (int l = 0; l < n_levels; ++l) {
+    const fold_partials *q = levels[l];
+    if (!q || !q->slots || !q->seqlens || !q->z) return FOLD_EINVAL;
+    if (q->batch != p0->batch || q->num_q_heads != p0->num_q_heads || q->num_kv_heads != p0->num_kv_heads ||
+        q->head_dim != p0->head_dim || q->z != p0->z)
+      return FOLD_EINVAL;
+    if (q->stack < 1 || q->batch % q->stack || q->num_seqs != q->batch / q->stack) return FOLD_EINVAL;
+    if (q->rows != q->stack * (q->num_q_heads / q->num_kv_heads) || q->max_slots < 1) return FOLD_EINVAL;
+    p.lv[l].slots = q->slots; p.lv[l].seqlens = q->seqlens; p.lv[l].slot_stride = q->slot_stride;
+    p.lv[l].stack = q->stack; p.lv[l].max_slots = q->max_slots; p.lv[l].rows = q->rows;
+    p.lv[l].max_seqlen = q->max_seqlen;
+  }
+  p.z = p0->z;
+  p.out = static_cast<__nv_bfloat16 *>(out);
+  p.lse = lse; p.row_status = row_status;
+  p.n_levels = n_levels; p.Hq = p0->num_q_heads; p.Hkv = p0->num_kv_heads;
+  p.G = p0->num_q_heads / p0->num_kv_heads; p.D = p0->head_dim;
+  const dim3 grid(p.Hq, p0->batch), block(p.D, kMergeSlices);
+  fold_merge_kernel<<<grid, block, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+int fold_decode(const fold_args *args, fold_stream stream) {
+  Geometry g;
+  if (int rc = check_args(args, &g, true)) return rc;
+  fold_partials part;
+  if (int rc = fold_decode_split(args, &part, stream)) return rc;
+  const fold_partials *lv[1] = {&part};
+  return fold_cascade_merge(lv, 1, args->out, args->lse, args->row_status, stream);
+}
+
+// ------------------------------------------------------------------ host-buffer variant
+namespace {
+struct HostPlan {
+  size_t q, k, v, table, lens, z, out, lse, status, ws, total;
+  size_t q_bytes, kv_bytes, table_bytes, lens_bytes, rows;
+};
+size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+bool plan_host(const fold_args *a, HostPlan *h) {
+  const fold_kv &kv = a->kv;
+  const bool paged = kv.page_table != nullptr;
+  const long long outer = paged ? kv.num_pages : kv.num_seqs;
+  const long long toks = paged ? kv.page_size : kv.capacity;
+  if (outer < 1 || toks < 1) return false;
+  const long long span = (outer - 1) * kv.stride_seq + (toks - 1) * kv.stride_tok +
+                         (long long)(a->num_kv_heads - 1) * kv.stride_head + a->head_dim;
+  h->rows = (size_t)a->batch * a->num_q_heads;
+  h->q_bytes = ((size_t)(a->batch - 1) * a->q_stride_b + (size_t)(a->num_q_heads - 1) * a->q_stride_h + a->head_dim) * 2;
+  h->kv_bytes = (size_t)span * 2;
+  h->table_bytes = paged ? (size_t)kv.num_seqs * kv.max_pages_per_seq * 4 : 0;
+  h->lens_bytes = (size_t)kv.num_seqs * 4;
+  size_t o = 0;
+  h->q = o; o += up256(h->q_bytes);
+  h->k = o; o += up256(h->kv_bytes);
+  h->v = o; o += up256(h->kv_bytes);
+  h->table = o; o += up256(h->table_bytes);
+  h->lens = o; o += up256(h->lens_bytes);
+  h->z = o; o += up256(h->rows * 4);
+  h->out = o; o += up256(h->rows * a->head_dim * 2);
+  h->lse = o; o += up256(h->rows * 4);
+  h->status = o; o += up256(h->rows * 4);
+  h->ws = o; o += up256(fold_workspace_bytes(a));
+  h->total = o;
+  return true;
+}
+}  // namespace
+
+size_t fold_host_staging_bytes(const fold_args *host_args) {
+  HostPlan h;
+  if (!host_args || fold_workspace_bytes(host_args) == 0 || !plan_host(host_args, &h)) return 0;
+  return h.total;
+}
+
+int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, fold_stream stream) {
+  if (!ha || !staging || !aligned(staging, 256)) return FOLD_EINVAL;
+  if (!ha->q || !ha->kv.k || !ha->kv.v || !ha->kv.seqlens || !ha->out) return FOLD_EINVAL;
+  if (ha->z_mode == FOLD_Z_GIVEN && !ha->z) return FOLD_EINVAL;
+  HostPlan h;
+  if (fold_workspace_bytes(ha) == 0 || !plan_host(ha, &h)) return FOLD_EINVAL;
+  if (staging_bytes < h.total) return FOLD_EWORKSPACE;
+  uint8_t *d = static_cast<uint8_t *>(staging);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  fold_args da = *ha;
+  da.q = d + h.q; da.kv.k = d + h.k; da.kv.v = d + h.v;
+  da.kv.page_table = ha->kv.page_table ? reinterpret_cast<const int32_t *>(d + h.table) : nullptr;
+  da.kv.seqlens = reinterpret_cast<const int32_t *>(d + h.lens);
+  da.z = reinterpret_cast<float *>(d + h.z);
+  da.out = d + h.out;
+  da.lse = reinterpret_cast<float *>(d + h.lse);
+  da.row_status = reinterpret_cast<int32_t *>(d + h.status);
+  da.workspace = d + h.ws;
+  da.workspace_bytes = fold_workspace_bytes(ha);
+  Geometry g;
+  if (int rc = check_args(&da, &g, true)) return rc;
+  bool ok = true;
+  ok &= cudaMemcpyAsync(d + h.q, ha->q, h.q_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d + h.k, ha->kv.k, h.kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d + h.v, ha->kv.v, h.kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (h.table_bytes)
+    ok &= cudaMemcpyAsync(d + h.table, ha->kv.page_table, h.table_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d + h.lens, ha->kv.seqlens, h.lens_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (ha->z_mode == FOLD_Z_GIVEN)
+    ok &= cudaMemcpyAsync(d + h.z, ha->z, h.rows * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) return FOLD_ECUDA;
+  if (int rc = fold_decode(&da, stream)) return rc;
+  ok &= cudaMemcpyAsync(ha->out, d + h.out, h.rows * ha->head_dim * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (ha->lse) ok &= cudaMemcpyAsync(ha->lse, d + h.lse, h.rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (ha->row_status)
+    ok &= cudaMemcpyAsync(ha->row_status, d + h.status, h.rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (ha->z && ha->z_mode != FOLD_Z_GIVEN)
+    ok &= cudaMemcpyAsync(ha->z, d + h.z, h.rows * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  return ok ? FOLD_OK : FOLD_ECUDA;
+}
+
+const char *fold_status_string(int status) {
+  switch (status) {
+    case FOLD_OK: return "ok";
+    case FOLD_EINVAL: return "invalid argument";
+    case FOLD_EUNSUPPORTED: return "unsupported shape or layout";
+    case FOLD_EWORKSPACE: return "workspace too small";
+    case FOLD_ECUDA: return "CUDA call failed";
+    default: return "unknown status";
+  }
+}
+
+int fold_version(void) { return 100; }
+
+}  // extern "C"

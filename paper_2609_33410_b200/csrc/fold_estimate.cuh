@@ -1,0 +1,193 @@
+// Reference kernels: the 192-key estimate of Z (Section 3, "Choosing the reference") and
+// the exact-maximum test mode.
+//
+// Estimate, per (request, q head), over the request's logical key sequence (the
+// concatenation of up to four cache levels): rows of at most 192 keys use their exact
+// base-2 log-sum-exp; longer rows score key 0 (the sink) and the last 63 keys exactly and
+// take the mass of the n-64 keys between them as (n-64) * mean of the 128 stratum-centre
+// weights with the 8 largest dropped.
+#pragma once
+
+#include "fold_common.cuh"
+
+namespace fold {
+
+constexpr int kEstSamples = 192;
+constexpr int kEstRecent = 63;
+constexpr int kEstStrata = 128;
+constexpr int kEstTrim = 8;
+constexpr int kEstThreads = 256;
+
+struct KvLevel {
+  const __nv_bfloat16 *k;
+  long long stride_seq, stride_tok, stride_head;
+  const int *page_table;
+  const int *seqlens;
+  int paged, page_shift, max_pages, num_pages, stack, max_seqlen;
+};
+
+struct EstParams {
+  const __nv_bfloat16 *q;
+  long long q_stride_b, q_stride_h;
+  float *z;
+  KvLevel lv[kMaxLevels];
+  int n_levels, Hq, Hkv, G;
+  float scale_log2;
+};
+
+__device__ __forceinline__ int level_len(const KvLevel &L, int req) {
+  int n = L.seqlens[req / L.stack];
+  return n < 0 ? 0 : (n > L.max_seqlen ? L.max_seqlen : n);
+}
+
+// Address of key row `tok` of sequence `seq` (caller guarantees tok < that sequence's length).
+__device__ __forceinline__ const __nv_bfloat16 *key_row(const KvLevel &L, int seq, int tok, int kvh) {
+  long long s = seq, t = tok;
+  if (L.paged) {
+    int pg = L.page_table[(long long)seq * L.max_pages + (tok >> L.page_shift)];
+    pg = min(max(pg, 0), L.num_pages - 1);
+    s = pg;
+    t = tok & ((1 << L.page_shift) - 1);
+  }
+  return L.k + s * L.stride_seq + t * L.stride_tok + (long long)kvh * L.stride_head;
+}
+
+// Which logical key the i-th sample of a row of n keys is.
+__device__ __forceinline__ int est_sample_key(int i, int n) {
+  if (n <= kEstSamples) return i;
+  if (i == 0) return 0;
+  if (i <= kEstRecent) return n - kEstRecent + (i - 1);
+  const int k = i - 1 - kEstRecent;
+  const long long n_mid = n - 1 - kEstRecent;
+  const int e0 = 1 + (int)((k * n_mid) / kEstStrata);
+  const int e1 = 1 + (int)(((k + 1) * n_mid) / kEstStrata);
+  return (e0 + e1) >> 1;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kEstThreads) fold_estimate_kernel(const EstParams p) {
+  constexpr int EPL = D / 32;                       // elements per lane
+  __shared__ float qs[kMaxRows][D];
+  __shared__ float sc[kMaxRows][kEstSamples];
+  const int kvh = blockIdx.x, req = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = p.G;
+
+  int lens[kMaxLevels];
+  int n = 0;
+  for (int l = 0; l < p.n_levels; ++l) {
+    lens[l] = level_len(p.lv[l], req);
+    n += lens[l];
+  }
+  for (int i = threadIdx.x; i < G * D; i += kEstThreads) {
+    const int g = i / D, d = i % D;
+    qs[g][d] = __bfloat162float(p.q[(long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + d]);
+  }
+  __syncthreads();
+
+  const int n_samples = n < kEstSamples ? n : kEstSamples;
+  for (int i = warp; i < n_samples; i += kEstThreads / 32) {
+    int j = est_sample_key(i, n), l = 0;
+    while (l < p.n_levels - 1 && j >= lens[l]) { j -= lens[l]; ++l; }
+    const __nv_bfloat16 *row = key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + lane * EPL;
+    float kf[EPL];
+    if (EPL == 4) {
+      const uint2 w = *reinterpret_cast<const uint2 *>(row);
+      const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&w.x);
+      const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&w.y);
+      kf[0] = __low2float(a); kf[1] = __high2float(a); kf[EPL - 2] = __low2float(b); kf[EPL - 1] = __high2float(b);
+    } else {
+      const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(row);
+      kf[0] = __low2float(a); kf[1] = __high2float(a);
+    }
+    for (int g = 0; g < G; ++g) {
+      float acc = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc = fmaf(kf[e], qs[g][lane * EPL + e], acc);
+#pragma unroll
+      for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+      if (lane == 0) sc[g][i] = acc * p.scale_log2;
+    }
+  }
+  __syncthreads();
+
+  for (int g = warp; g < G; g += kEstThreads / 32) {
+    float zval = 0.f;
+    if (n_samples > 0) {
+      float m = -INFINITY;
+      for (int i = lane; i < n_samples; i += 32) m = fmaxf(m, sc[g][i]);
+#pragma unroll
+      for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+      float total = 0.f;
+      if (n <= kEstSamples) {
+        for (int i = lane; i < n_samples; i += 32) total += exp2f(sc[g][i] - m);
+      } else {
+        for (int i = lane; i <= kEstRecent; i += 32) total += exp2f(sc[g][i] - m);      // sink + 63 recent
+        // trimmed mean of the 128 centre weights: drop the 8 largest (ties broken by index)
+        float kept = 0.f;
+        for (int k = lane; k < kEstStrata; k += 32) {
+          const float wk = sc[g][1 + kEstRecent + k];
+          int rank = 0;
+          for (int j = 0; j < kEstStrata; ++j) {
+            const float wj = sc[g][1 + kEstRecent + j];
+            rank += (wj > wk || (wj == wk && j < k)) ? 1 : 0;
+          }
+          if (rank >= kEstTrim) kept += exp2f(wk - m);
+        }
+        total += kept * ((float)(n - 1 - kEstRecent) / (float)(kEstStrata - kEstTrim));
+      }
+#pragma unroll
+      for (int k = 16; k > 0; k >>= 1) total += __shfl_xor_sync(0xffffffffu, total, k);
+      zval = m + log2f(total);
+    }
+    if (lane == 0) p.z[(long long)req * p.Hq + kvh * G + g] = zval;
+  }
+}
+
+// Test mode: z = max_j s_ij over every key of a single level.
+template <int D>
+__global__ void __launch_bounds__(kEstThreads) fold_exact_max_kernel(const EstParams p) {
+  constexpr int EPL = D / 32;
+  __shared__ float qs[kMaxRows][D];
+  __shared__ float wm[kEstThreads / 32][kMaxRows];
+  const int kvh = blockIdx.x, req = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = p.G;
+  const int n = level_len(p.lv[0], req);
+  for (int i = threadIdx.x; i < G * D; i += kEstThreads) {
+    const int g = i / D, d = i % D;
+    qs[g][d] = __bfloat162float(p.q[(long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + d]);
+  }
+  __syncthreads();
+  float best[kMaxRows];
+  for (int g = 0; g < kMaxRows; ++g) best[g] = -INFINITY;
+  for (int j = warp; j < n; j += kEstThreads / 32) {
+    const __nv_bfloat16 *row = key_row(p.lv[0], req / p.lv[0].stack, j, kvh) + lane * EPL;
+    float kf[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) kf[e] = __bfloat162float(row[e]);
+    for (int g = 0; g < G; ++g) {
+      float acc = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc = fmaf(kf[e], qs[g][lane * EPL + e], acc);
+#pragma unroll
+      for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+      best[g] = fmaxf(best[g], acc * p.scale_log2);
+    }
+  }
+  if (lane == 0)
+    for (int g = 0; g < G; ++g) wm[warp][g] = best[g];
+  __syncthreads();
+  if (threadIdx.x < G) {
+    float m = -INFINITY;
+    for (int w = 0; w < kEstThreads / 32; ++w) m = fmaxf(m, wm[w][threadIdx.x]);
+    p.z[(long long)req * p.Hq + kvh * G + threadIdx.x] = n > 0 ? m : 0.f;
+  }
+}
+
+__global__ void fold_fill_kernel(float *z, int count, float value) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) z[i] = value;
+}
+
+}  // namespace fold
