@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the fold decode hot path on B200.
+
+A step is one whole decode over one synthetic batch: reference estimate -> split-KV scan
+-> order-free partial add, through the C ABI.  Default workload: the GQA configuration the
+headline metric is quoted on (32 q / 8 kv heads, D=128, batch 16, 32768 keys, peaked keys,
+T=16).  Prints ONE JSON line.  `--impl reference` times the float64 CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "decode attn effective HBM GB/s (full-cache bytes / time) at T=16; us/call and T=inf alongside"
+UNIT = "GB/s"
+
+WORKLOADS = {
+    # name: generator kwargs, depth, split hint
+    "c2": dict(gen=dict(batch=16, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=32768, seed=1), T=16.0),
+    "c3": dict(gen=dict(batch=4, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=131072, seed=2, paged=True,
+                        page_size=64), T=16.0),
+    "c1": dict(gen=dict(batch=1, num_q_heads=8, num_kv_heads=8, head_dim=128, seqlens=4096, seed=0, peak_frac=0.0),
+               T=16.0),
+    "c2_small": dict(gen=dict(batch=4, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=16384, seed=1), T=16.0),
+}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                pass
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w, T, units, z=None):
+    """Time the float64 oracle, as it stands, on `units` (sequence, kv head) units of workload w.
+    Returns (seconds, bytes of cache those units hold, threads used)."""
+    import numpy as np
+    from oracle import fold_oracle as O
+    from paper_2609_33410_b200.workloads import bf16_bits
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    G = w.num_q_heads // w.num_kv_heads
+    data = []
+    for (seq, kvh) in units:
+        K = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh)))
+        V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
+        qs = [O.widen_bf16(bf16_bits(w.q[seq * w.stack + r // G, kvh * G + r % G])) for r in range(w.stack * G)]
+        data.append((K, V, qs))
+    t0 = time.perf_counter()
+    nbytes = 0
+    for (K, V, qs) in data:
+        for q in qs:
+            s = O.scores(q, K, w.scale)
+            zz = O.estimate_z(lambda i: s[i], len(s))
+            O.fold_row(s, V, zz, T)
+        nbytes += K.shape[0] * 4 * w.head_dim
+    return time.perf_counter() - t0, nbytes, threads
+
+
+def bounded_oracle(w, T, budget_s=12.0):
+    units_all = [(s, h) for s in range(w.num_seqs) for h in range(w.num_kv_heads)]
+    t1, b1, threads = oracle_sample(w, T, units_all[:1])
+    k = int(max(1, min(len(units_all) - 1, budget_s / max(t1, 1e-3))))
+    t, b, threads = oracle_sample(w, T, units_all[1:1 + k]) if k >= 1 and len(units_all) > 1 else (t1, b1, threads)
+    return dict(seconds=t, bytes=b, units=k, threads=threads)
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the float64 oracle on the host cores, bounded sample per step."""
+    if rank != 0:
+        return
+    from paper_2609_33410_b200.workloads import make_decode_workload
+    spec = WORKLOADS[args.workload]
+    gen = dict(spec["gen"])
+    gen["batch"] = min(gen["batch"], 2)                 # the sample never needs more than two requests
+    w = make_decode_workload(device="cpu", **gen)
+    units = [(s, h) for s in range(w.num_seqs) for h in range(w.num_kv_heads)]
+    per_step = units[: max(1, min(len(units), args.ref_units))]
+    for _ in range(args.warmup):
+        oracle_sample(w, spec["T"], per_step[:1])
+    tot_t = tot_b = 0.0
+    threads = 1
+    for _ in range(args.steps):
+        t, b, threads = oracle_sample(w, spec["T"], per_step)
+        tot_t += t; tot_b += b
+    val = tot_b / tot_t / 1e9
+    sample = f"{len(per_step)} (sequence, kv head) units x {w.num_q_heads // w.num_kv_heads} rows of {args.workload} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "depth_T": spec["T"]},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def shard_note(world: int) -> str:
+    return "replicas: every rank decodes its own batch of the same shape; no data-path collective"
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    if world <= 1:
+        return ms
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="fold", choices=["fold", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--num-splits", type=int, default=0)
+    ap.add_argument("--ref-units", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import paper_2609_33410_b200 as F
+    from paper_2609_33410_b200.workloads import make_decode_workload
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    spec = WORKLOADS[args.workload]
+    gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
+    w = make_decode_workload(device=dev, **gen)
+    T = spec["T"]
+    cache = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table)
+    bufs = F.alloc_buffers(w.q, cache)
+    cache_bytes = w.cache_bytes()
+    stream = torch.cuda.current_stream()
+
+    def make(depth):
+        return F.make_args(w.q, cache, scale=w.scale, z_mode=F.Z_GIVEN, z=bufs.z, depth_T=depth,
+                           num_splits=args.num_splits, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse,
+                           row_status=bufs.row_status)
+
+    def step(a, evs=None):
+        # the three launches of fold_decode, issued one by one so the scan can be timed on its own
+        if evs: evs[0].record(stream)
+        F.fold_estimate_z([a], stream)
+        if evs: evs[1].record(stream)
+        part = F.fold_decode_split(a, stream)
+        if evs: evs[2].record(stream)
+        F.fold_cascade_merge([part], bufs.out, bufs.lse, bufs.row_status, stream)
+        if evs: evs[3].record(stream)
+
+    def timed(depth, steps, warmup, sample_clocks):
+        a = make(depth)
+        for _ in range(warmup):
+            step(a)
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local)
+        ctx = sampler if sample_clocks else None
+        if ctx: ctx.__enter__()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for i in range(steps):
+            step(a, evs[i])
+        t1.record(stream)
+        torch.cuda.synchronize()
+        if ctx: ctx.__exit__()
+        if world > 1:
+            torch.distributed.barrier()
+        total_ms = t0.elapsed_time(t1)
+        scan_ms = [e[1].elapsed_time(e[2]) for e in evs]
+        est_ms = [e[0].elapsed_time(e[1]) for e in evs]
+        mrg_ms = [e[2].elapsed_time(e[3]) for e in evs]
+        hdr = bufs.header()
+        return dict(ms_per_step=max_over_ranks(total_ms / steps, world, dev), scan_ms=statistics.mean(scan_ms),
+                    scan_ms_min=min(scan_ms), est_ms=statistics.mean(est_ms), merge_ms=statistics.mean(mrg_ms),
+                    fetched=hdr.v_rows_fetched, total=hdr.v_rows_total, timeouts=hdr.wait_timeouts,
+                    clocks=sampler.summary() if sample_clocks else None)
+
+    warm = max(args.warmup, 3)
+    r16 = timed(T, args.steps, warm, True)
+    rinf = timed(math.inf, args.steps, warm, False)
+    if r16["timeouts"] or rinf["timeouts"]:
+        raise SystemExit("a bounded wait timed out inside the scan kernel: results invalid")
+
+    D = w.head_dim
+    slot_bytes = F.fold_workspace_bytes(make(T)) - 256
+
+    def actual_bytes(r):                                  # K in full + fetched V rows + slots written
+        return r["total"] * 2 * D + r["fetched"] * 2 * D + slot_bytes
+
+    peak, peak_src = load_peaks()
+    value = world * cache_bytes / (r16["ms_per_step"] * 1e-3) / 1e9
+    ach16 = actual_bytes(r16) / (r16["scan_ms"] * 1e-3) / 1e9
+    achinf = actual_bytes(rinf) / (rinf["scan_ms"] * 1e-3) / 1e9
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+        "ms_per_step": r16["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 in, fp32 accumulate", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: " + json.dumps(spec["gen"], sort_keys=True), "depth_T": T,
+                   "num_splits": args.num_splits or "auto", "l2": "inputs (cache) larger than L2, no flush needed"
+                   if cache_bytes > 4 * 126e6 else "cache smaller than 4x L2: partly L2-resident",
+                   "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes},
+        "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
+        "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},
+        "kernel_ms": {"estimate": r16["est_ms"], "scan_T16": r16["scan_ms"], "scan_Tinf": rinf["scan_ms"],
+                      "merge": r16["merge_ms"]},
+        "v_rows_fetched_frac": {"T16": r16["fetched"] / max(r16["total"], 1), "Tinf": rinf["fetched"] / max(rinf["total"], 1)},
+        "roofline": {"bound": "hbm", "kernel": "fold_scan_kernel (T=16, gather path)", "achieved": ach16, "peak": peak,
+                     "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src, "traffic": None,
+                     "algorithmic_bytes_per_launch": actual_bytes(r16),
+                     "dense": {"kernel": "fold_scan_kernel (T=inf, TMA path)", "achieved": achinf, "frac": achinf / peak,
+                               "frac_of_nominal_8TBs": achinf / 8000.0,
+                               "algorithmic_bytes_per_launch": actual_bytes(rinf)}},
+        "gpu_launches": 3 * args.steps,
+        "clocks": r16["clocks"],
+    }
+
+    if rank == 0 and not args.no_e2e:
+        # end to end through the C ABI with HOST buffers: every step copies q and the whole cache
+        # host -> device, decodes, and copies out / lse / status back
+        hq, hk, hv = w.q.cpu().pin_memory(), w.k.cpu().pin_memory(), w.v.cpu().pin_memory()
+        hlen = w.seqlens.cpu().pin_memory()
+        htab = w.page_table.cpu().pin_memory() if w.paged else None
+        hout = torch.empty(w.q.shape, dtype=torch.bfloat16).pin_memory()
+        hlse = torch.empty(w.q.shape[:2], dtype=torch.float32).pin_memory()
+        hz = torch.empty(w.q.shape[:2], dtype=torch.float32).pin_memory()
+        hst = torch.empty(w.q.shape[:2], dtype=torch.int32).pin_memory()
+        hcache = F.KVCache(hk, hv, hlen, w.max_seqlen, htab)
+        ha = F.make_args(hq, hcache, scale=w.scale, depth_T=T, num_splits=args.num_splits, z=hz, out=hout, lse=hlse,
+                         row_status=hst)
+        staging = torch.empty(F.fold_host_staging_bytes(ha), dtype=torch.uint8, device=dev)
+        e2e_steps = max(1, min(args.steps, 5))
+        F.fold_decode_host(ha, staging, stream); torch.cuda.synchronize()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(e2e_steps):
+            F.fold_decode_host(ha, staging, stream)
+        t1.record(stream); torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / e2e_steps
+        h2d = hq.numel() * 2 + 2 * hk.numel() * 2 + hlen.numel() * 4 + (htab.numel() * 4 if htab is not None else 0)
+        d2h = hout.numel() * 2 + 3 * hlse.numel() * 4
+        out["e2e"] = {"value": cache_bytes / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": e2e_steps,
+                      "note": "fold_decode_host: whole cache copied from pinned host memory every step"}
+        del staging, hk, hv
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        wc = make_decode_workload(device="cpu", **dict(spec["gen"], batch=min(spec["gen"]["batch"], 2)))
+        ob = bounded_oracle(wc, T)
+        out["cpu_baseline"] = {"value": ob["bytes"] / ob["seconds"] / 1e9, "unit": UNIT, "cores": ob["threads"],
+                               "kind": "oracle",
+                               "sample": f"{ob['units']} (sequence, kv head) units of {args.workload} "
+                                         f"({ob['seconds']:.1f} s of float64 numpy; estimate + declared-Z row per q head)"}
+
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

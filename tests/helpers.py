@@ -1,0 +1,107 @@
+"""Shared pieces of the GPU parity tests: run the CUDA path through the C ABI binding, run
+the float64 oracle on the same seeded inputs, and compare with the stated tolerances."""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+import torch
+
+import paper_2609_33410_b200 as F
+from oracle import fold_oracle as O
+from paper_2609_33410_b200.workloads import DecodeWorkload, bf16_bits
+
+# Tolerances of the build target, written out:
+#   dense (T = inf): max abs error <= 1e-2 * max|V| and mean row-relative l2 error <= 5e-3
+#                    against the float64 result;
+#   finite T:        global relative l2 error against the float64 declared-reference result
+#                    at the same Z and T  <=  1.5 x the error of a plain BF16 online-softmax
+#                    kernel (emulated) against float64 softmax attention, plus the mass of keys
+#                    within 2^-10 binades of the threshold (fp32 vs fp64 scores may flip them).
+DENSE_MAX_ABS = 1e-2
+DENSE_MEAN_REL = 5e-3
+FINITE_T_FACTOR = 1.5
+Z_TOL = 1e-3
+LSE_TOL = 2e-3
+
+
+def cache_of(w: DecodeWorkload) -> F.KVCache:
+    return F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table)
+
+
+def run_gpu(w: DecodeWorkload, T=math.inf, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, bufs=None):
+    cache = cache_of(w)
+    if bufs is None:
+        bufs = F.alloc_buffers(w.q, cache, w.stack)
+    if z is not None:
+        bufs.z.copy_(z)
+    F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale)
+    torch.cuda.synchronize()
+    assert bufs.header().wait_timeouts == 0
+    return bufs
+
+
+def row_inputs(w: DecodeWorkload, b: int, h: int):
+    G = w.num_q_heads // w.num_kv_heads
+    seq, kvh = b // w.stack, h // G
+    K = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh)))
+    V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
+    q = O.widen_bf16(bf16_bits(w.q[b, h]))
+    return q, K, V
+
+
+def all_rows(w: DecodeWorkload):
+    return [(b, h) for b in range(w.batch) for h in range(w.num_q_heads)]
+
+
+def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False, yardstick=True):
+    """Element-by-element comparison of the CUDA outputs with the oracle run at the GPU's own
+    references.  Returns a dict of the measured errors; asserts the tolerances."""
+    out = bufs.out.float().cpu().numpy().astype(np.float64)
+    lse = bufs.lse.cpu().numpy().astype(np.float64)
+    z = bufs.z.cpu().numpy().astype(np.float64)
+    status = bufs.row_status.cpu().numpy()
+    rows = rows if rows is not None else all_rows(w)
+    num = den = ynum = 0.0
+    max_abs = 0.0
+    vmax = 0.0
+    rel_rows, slack_sum, dz = [], 0.0, 0.0
+    for (b, h) in rows:
+        q, K, V = row_inputs(w, b, h)
+        n = K.shape[0]
+        if n == 0:
+            assert not out[b, h].any() and lse[b, h] == -np.inf and status[b, h] == F.ROW_EMPTY
+            continue
+        s = O.scores(q, K, w.scale)
+        o_ref, lse_ref, _, L = O.fold_row(s, V, z[b, h], T)
+        d = out[b, h] - o_ref
+        num += float(d @ d); den += float(o_ref @ o_ref)
+        max_abs = max(max_abs, float(np.abs(d).max())); vmax = max(vmax, float(np.abs(V).max()))
+        rel_rows.append(np.linalg.norm(d) / max(np.linalg.norm(o_ref), 1e-300))
+        assert abs(lse[b, h] - lse_ref) <= LSE_TOL, (b, h, lse[b, h], lse_ref)
+        if 0.5 <= L <= 2.0 ** 100:
+            assert status[b, h] == 0, (b, h, status[b, h], L)
+        if check_estimate:
+            dz = max(dz, abs(O.estimate_z(lambda i: s[i], n) - z[b, h]))
+        if not math.isinf(T):
+            slack_sum += O.cut_report(s, V, z[b, h], T)["slack"] ** 2 * V.shape[1]
+            if yardstick:
+                o_dense, _ = O.dense_row(s, V)
+                y = O.online_softmax_bf16(q, K, V, w.scale) - o_dense
+                ynum += float(y @ y)
+    res = dict(rel_l2=math.sqrt(num / max(den, 1e-300)), max_abs=max_abs, vmax=vmax,
+               mean_rel=float(np.mean(rel_rows)) if rel_rows else 0.0, dz=dz)
+    if math.isinf(T):
+        assert max_abs <= DENSE_MAX_ABS * vmax, res
+        assert res["mean_rel"] <= DENSE_MEAN_REL, res
+    elif yardstick:
+        res["yard"] = math.sqrt(ynum / max(den, 1e-300))
+        res["slack"] = math.sqrt(slack_sum / max(den, 1e-300))
+        assert res["rel_l2"] <= FINITE_T_FACTOR * res["yard"] + res["slack"], res
+    if check_estimate:
+        assert dz <= Z_TOL, res
+    return res
+
+
+def same_bits(a: torch.Tensor, b: torch.Tensor) -> bool:
+    return torch.equal(a.contiguous().view(torch.uint8), b.contiguous().view(torch.uint8))

@@ -1,0 +1,126 @@
+"""The C-ABI library without a GPU: it builds, loads, exports every symbol the header
+declares, the Python structs mirror the C ones byte for byte, and host-side argument
+checks answer with status codes before any CUDA call is made."""
+import ctypes as C
+import os
+import re
+import subprocess
+import sys
+import tempfile
+
+import pytest
+import torch
+
+import paper_2609_33410_b200 as F
+from paper_2609_33410_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "fold.h")
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(fold_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert set(names) == set(binding.EXPORTS), (names, binding.EXPORTS)
+    L = F.lib()
+    for n in names:
+        assert getattr(L, n) is not None
+    assert L.fold_version() >= 100
+    assert L.fold_status_string(F.FOLD_EWORKSPACE) == b"workspace too small"
+
+
+def test_python_structs_mirror_the_header():
+    prog = r"""
+#include <stdio.h>
+#include <stddef.h>
+#include "fold.h"
+int main(void) {
+  printf("%zu %zu %zu %zu\n", sizeof(fold_kv), sizeof(fold_args), sizeof(fold_partials), sizeof(fold_ws_header));
+  printf("%zu %zu %zu %zu %zu\n", offsetof(fold_kv, seqlens), offsetof(fold_kv, max_seqlen), offsetof(fold_args, kv),
+         offsetof(fold_args, depth_T), offsetof(fold_args, row_status));
+  printf("%zu %zu %zu\n", offsetof(fold_partials, rows), offsetof(fold_partials, slot_stride),
+         offsetof(fold_ws_header, v_rows_total));
+  return 0;
+}
+"""
+    with tempfile.TemporaryDirectory() as d:
+        src = os.path.join(d, "t.c"); exe = os.path.join(d, "t")
+        open(src, "w").write(prog)
+        subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), src, "-o", exe],
+                       check=True)
+        out = subprocess.run([exe], check=True, capture_output=True, text=True).stdout.split()
+    got = [int(x) for x in out]
+    want = [C.sizeof(F.FoldKV), C.sizeof(F.FoldArgs), C.sizeof(F.FoldPartials), C.sizeof(F.FoldWsHeader),
+            F.FoldKV.seqlens.offset, F.FoldKV.max_seqlen.offset, F.FoldArgs.kv.offset, F.FoldArgs.depth_T.offset,
+            F.FoldArgs.row_status.offset, F.FoldPartials.rows.offset, F.FoldPartials.slot_stride.offset,
+            F.FoldWsHeader.v_rows_total.offset]
+    assert got == want
+
+
+def test_chunk_rule_depends_on_length_only():
+    assert F.fold_chunk_keys(1) == 256 and F.fold_chunk_keys(8192) == 256 and F.fold_chunk_keys(8193) == 1024
+    assert [F.fold_num_chunks(n) for n in (0, 1, 256, 257, 8192, 8193, 131072)] == [0, 1, 1, 2, 32, 9, 128]
+
+
+def _cpu_args(B=2, Hq=8, Hkv=2, D=128, n=1000, **kw):
+    q = torch.zeros(B, Hq, D, dtype=torch.bfloat16)
+    k = torch.zeros(B, n, Hkv, D, dtype=torch.bfloat16)
+    v = torch.zeros_like(k)
+    lens = torch.full((B,), n, dtype=torch.int32)
+    z = torch.zeros(B, Hq)
+    out = torch.zeros(B, Hq, D, dtype=torch.bfloat16)
+    cache = F.KVCache(k, v, lens, n)
+    a = F.make_args(q, cache, z=z, out=out, **kw)
+    keep = (q, k, v, lens, z, out)
+    return a, keep
+
+
+def test_workspace_size_formula():
+    a, _ = _cpu_args()
+    G, R = 4, 4
+    slots = (1000 + 255) // 256
+    assert F.fold_workspace_bytes(a) == 256 + 2 * 2 * slots * (R * 128 + 4) * 4
+    a, _ = _cpu_args(n=40000)
+    assert F.fold_workspace_bytes(a) == 256 + 2 * 2 * 40 * (R * 128 + 4) * 4
+    a.head_dim = 80
+    assert F.fold_workspace_bytes(a) == 0
+
+
+def test_host_checks_answer_before_any_cuda_call():
+    L = F.lib()
+    a, keep = _cpu_args()
+    ws = torch.zeros(F.fold_workspace_bytes(a) + 256, dtype=torch.uint8)
+    off = (-ws.data_ptr()) % 256
+    a.workspace = ws.data_ptr() + off
+    a.workspace_bytes = ws.numel() - 256
+    for field, value, want in [("depth_T", -0.5, F.FOLD_EINVAL), ("depth_T", float("nan"), F.FOLD_EINVAL),
+                               ("head_dim", 96, F.FOLD_EUNSUPPORTED), ("softmax_scale", 0.0, F.FOLD_EINVAL),
+                               ("z_mode", 7, F.FOLD_EINVAL), ("num_splits", -1, F.FOLD_EINVAL),
+                               ("workspace_bytes", 100, F.FOLD_EWORKSPACE), ("stack", 3, F.FOLD_EINVAL),
+                               ("num_kv_heads", 3, F.FOLD_EINVAL), ("out", None, F.FOLD_EINVAL)]:
+        old = getattr(a, field)
+        setattr(a, field, value)
+        assert L.fold_decode(a, None) == want, field
+        setattr(a, field, old)
+    a.kv.page_table = keep[3].data_ptr(); a.kv.page_size = 24; a.kv.num_pages = 4; a.kv.max_pages_per_seq = 100
+    assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED          # page size not a power of two
+    a.kv.page_size = 64; a.kv.max_pages_per_seq = 2
+    assert L.fold_decode(a, None) == F.FOLD_EINVAL                # table cannot hold max_seqlen
+    assert L.fold_cascade_merge(None, 1, None, None, None, None) == F.FOLD_EINVAL
+    assert L.fold_estimate_z(None, 0, None) == F.FOLD_EINVAL
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="only meaningful without a device")
+def test_no_device_means_a_loud_error_not_a_fallback():
+    a, keep = _cpu_args()
+    ws = torch.zeros(F.fold_workspace_bytes(a) + 256, dtype=torch.uint8)
+    a.workspace = ws.data_ptr() + ((-ws.data_ptr()) % 256)
+    a.workspace_bytes = ws.numel() - 256
+    with pytest.raises(F.FoldError) as e:
+        F.fold_decode(a, stream=0)
+    assert e.value.status == F.FOLD_ECUDA

@@ -1,0 +1,148 @@
+"""Bit-identity of the CUDA path under everything that only regroups the same sum
+(Prop. 1(i) made exact by canonical chunks + the integer-grid partial add), and the
+shared-prefix cascade."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_33410_b200 as F
+from oracle import fold_oracle as O
+from paper_2609_33410_b200.workloads import make_decode_workload, DecodeWorkload
+from helpers import run_gpu, compare, cache_of, same_bits, row_inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("T", [math.inf, 16.0])
+def test_split_count_never_changes_a_bit(T):
+    w = make_decode_workload(2, 8, 2, 128, [40000, 9000], seed=41, device=DEV)
+    ref = run_gpu(w, T=T, num_splits=1)
+    o, l = ref.out.clone(), ref.lse.clone()
+    for s in (2, 3, 4, 8, 16, 32, 0):
+        b = run_gpu(w, T=T, num_splits=s)
+        assert same_bits(b.out, o) and same_bits(b.lse, l), s
+
+
+@pytest.mark.parametrize("T", [math.inf, 16.0])
+def test_alone_equals_in_batch(T):
+    w = make_decode_workload(4, 8, 2, 128, [5000, 333, 12000, 64], seed=43, device=DEV)
+    full = run_gpu(w, T=T)
+    for b in range(4):
+        n = int(w.seqlens[b])
+        solo = DecodeWorkload(w.q[b:b + 1].contiguous(), w.k[b:b + 1, :max(n, 1)].contiguous(),
+                              w.v[b:b + 1, :max(n, 1)].contiguous(), w.seqlens[b:b + 1].contiguous(), n,
+                              w.num_q_heads, w.num_kv_heads, w.head_dim, scale=w.scale)
+        r = run_gpu(solo, T=T)
+        assert same_bits(r.out[0], full.out[b]) and same_bits(r.lse[0], full.lse[b]), b
+
+
+@pytest.mark.parametrize("T", [math.inf, 16.0])
+@pytest.mark.parametrize("page_size", [16, 64])
+def test_paged_equals_contiguous(T, page_size):
+    w = make_decode_workload(2, 8, 2, 128, [3000, 10000], seed=47, device=DEV)
+    ref = run_gpu(w, T=T)
+    # scatter the same logical rows into a randomly permuted page pool
+    g = torch.Generator(device=DEV); g.manual_seed(5)
+    lens = [3000, 10000]
+    npg = [(n + page_size - 1) // page_size for n in lens]
+    perm = torch.randperm(sum(npg) + 3, generator=g, device=DEV)
+    kp = torch.full((sum(npg) + 3, page_size, 2, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+    vp = torch.full_like(kp, float("nan"))
+    table = torch.zeros(2, max(npg), dtype=torch.int32, device=DEV)
+    cur = 0
+    for s, n in enumerate(lens):
+        ids = perm[cur:cur + npg[s]]; cur += npg[s]
+        table[s, :npg[s]] = ids.to(torch.int32)
+        pad = npg[s] * page_size - n
+        kk = torch.cat([w.k[s, :n], torch.full((pad, 2, 128), float("nan"), dtype=torch.bfloat16, device=DEV)])
+        vv = torch.cat([w.v[s, :n], torch.full((pad, 2, 128), float("nan"), dtype=torch.bfloat16, device=DEV)])
+        kp[ids] = kk.view(npg[s], page_size, 2, 128); vp[ids] = vv.view(npg[s], page_size, 2, 128)
+    wp = DecodeWorkload(w.q, kp, vp, w.seqlens, w.max_seqlen, 8, 2, 128, 1, table, page_size, w.scale)
+    r = run_gpu(wp, T=T)
+    assert same_bits(r.out, ref.out) and same_bits(r.lse, ref.lse) and same_bits(r.z, ref.z)
+
+
+def _split_then_merge(w, T, z, order=None, perm_seed=None):
+    cache = cache_of(w)
+    bufs = F.alloc_buffers(w.q, cache, w.stack)
+    bufs.z.copy_(z)
+    args = F.make_args(w.q, cache, scale=w.scale, z_mode=F.Z_GIVEN, z=bufs.z, depth_T=T, stack=w.stack,
+                       workspace=bufs.workspace)
+    part = F.fold_decode_split(args)
+    torch.cuda.synchronize()
+    if perm_seed is not None:                     # permute the valid slots of every (sequence, kv head)
+        sv = F.slots_view(part, bufs.workspace)
+        g = torch.Generator(device=DEV); g.manual_seed(perm_seed)
+        for s in range(part.num_seqs):
+            c = F.fold_num_chunks(int(w.seqlens[s]))
+            for h in range(part.num_kv_heads):
+                sv[s, h, :c] = sv[s, h, :c][torch.randperm(c, generator=g, device=DEV)]
+    return part, bufs
+
+
+@pytest.mark.parametrize("T", [math.inf, 16.0])
+def test_slot_order_never_changes_a_bit(T):
+    w = make_decode_workload(2, 8, 2, 128, [30000, 7000], seed=53, device=DEV)
+    z = run_gpu(w, T=T).z.clone()
+    part, bufs = _split_then_merge(w, T, z)
+    F.fold_cascade_merge([part], bufs.out, bufs.lse, bufs.row_status)
+    torch.cuda.synchronize()
+    o, l = bufs.out.clone(), bufs.lse.clone()
+    ref = run_gpu(w, T=T, z_mode=F.Z_GIVEN, z=z)
+    assert same_bits(o, ref.out) and same_bits(l, ref.lse)
+    for seed in (1, 2, 3):
+        part2, bufs2 = _split_then_merge(w, T, z, perm_seed=seed)
+        F.fold_cascade_merge([part2], bufs2.out, bufs2.lse, bufs2.row_status)
+        torch.cuda.synchronize()
+        assert same_bits(bufs2.out, o) and same_bits(bufs2.lse, l)
+
+
+def _cascade(B, Hq, Hkv, D, n_prefix, suffix_lens, seed, T):
+    """Requests share one prefix and own private suffixes.  Returns (out, lse, z, flat workload)."""
+    g = torch.Generator(device=DEV); g.manual_seed(seed)
+    q = torch.randn(B, Hq, D, generator=g, device=DEV).to(torch.bfloat16)
+    pre = make_decode_workload(B, Hq, Hkv, D, n_prefix, seed=seed + 1, device=DEV, stack=B, q=q)
+    suf = make_decode_workload(B, Hq, Hkv, D, suffix_lens, seed=seed + 2, device=DEV, q=q, sink_gain=1.0)
+    cp, cs = cache_of(pre), cache_of(suf)
+    bp, bs = F.alloc_buffers(q, cp, stack=B), F.alloc_buffers(q, cs)
+    z = bs.z
+    ap = F.make_args(q, cp, z_mode=F.Z_GIVEN, z=z, depth_T=T, stack=B, workspace=bp.workspace)
+    as_ = F.make_args(q, cs, z_mode=F.Z_GIVEN, z=z, depth_T=T, workspace=bs.workspace)
+    F.fold_estimate_z([ap, as_])                  # one estimate over prefix ++ suffix, used by both levels
+    pp, ps = F.fold_decode_split(ap), F.fold_decode_split(as_)
+    F.fold_cascade_merge([pp, ps], bs.out, bs.lse, bs.row_status)
+    torch.cuda.synchronize()
+    out, lse = bs.out.clone(), bs.lse.clone()
+    F.fold_cascade_merge([ps, pp], bp.out, bp.lse, bp.row_status)       # level order swapped
+    torch.cuda.synchronize()
+    assert same_bits(bp.out, out) and same_bits(bp.lse, lse)
+    # the same requests as a flat batch over the concatenated sequences
+    lens = [n_prefix + s for s in suffix_lens]
+    cap = max(lens)
+    kf = torch.zeros(B, cap, Hkv, D, dtype=torch.bfloat16, device=DEV); vf = torch.zeros_like(kf)
+    for b in range(B):
+        kf[b, :n_prefix] = pre.k[0, :n_prefix]; vf[b, :n_prefix] = pre.v[0, :n_prefix]
+        kf[b, n_prefix:lens[b]] = suf.k[b, :suffix_lens[b]]; vf[b, n_prefix:lens[b]] = suf.v[b, :suffix_lens[b]]
+    flat = DecodeWorkload(q, kf, vf, torch.tensor(lens, dtype=torch.int32, device=DEV), cap, Hq, Hkv, D,
+                          scale=1.0 / math.sqrt(D))
+    return bs, flat
+
+
+@pytest.mark.parametrize("T", [math.inf, 16.0])
+def test_shared_prefix_cascade_matches_oracle_and_flat_decode(T):
+    B, Hq, Hkv, D = 4, 8, 2, 128                  # 4 requests x group 4 = 16 stacked rows on the prefix
+    bs, flat = _cascade(B, Hq, Hkv, D, 3000, [500, 1, 0, 257], seed=61, T=T)
+    # oracle on the concatenated sequence at the cascade's references
+    r = compare(flat, bs, T=T, check_estimate=True)
+    # flat decode of the same requests under the same references: same values within tolerance
+    fb = run_gpu(flat, T=T, z_mode=F.Z_GIVEN, z=bs.z.clone())
+    assert same_bits(fb.z, bs.z)
+    a, b = fb.out.float(), bs.out.float()
+    assert (a - b).norm() / a.norm() < 3e-3
+    assert torch.allclose(fb.lse, bs.lse, atol=1e-4)
+    # and the flat estimate equals the cascade's two-level estimate bit for bit
+    fe = run_gpu(flat, T=T)
+    assert same_bits(fe.z, bs.z)
