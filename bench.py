@@ -33,6 +33,8 @@ WORKLOADS = {
                         page_size=64), T=16.0),
     "c1": dict(gen=dict(batch=1, num_q_heads=8, num_kv_heads=8, head_dim=128, seqlens=4096, seed=0, peak_frac=0.0),
                T=16.0),
+    "c3_small": dict(gen=dict(batch=1, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=131072, seed=2, paged=True,
+                              page_size=64), T=16.0),
     "c2_small": dict(gen=dict(batch=4, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=16384, seed=1), T=16.0),
 }
 

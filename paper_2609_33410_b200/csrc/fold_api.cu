@@ -1,6 +1,7 @@
 // C ABI of the fold decode library: argument checks, tensor-map creation, workspace
 // carving and kernel launches.  Nothing here allocates device memory or synchronises.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "fold_common.cuh"
@@ -166,8 +167,8 @@ int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st) {
     p.lv[0] = kv_level(a->kv, a->stack);
     const dim3 grid(g.Hkv, g.B);
     if (a->z_mode == FOLD_Z_ESTIMATE) {
-      if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
-      else fold_estimate_kernel<64><<<grid, kEstThreads, 0, st>>>(p);
+      if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstSampleThreads, 0, st>>>(p);
+      else fold_estimate_kernel<64><<<grid, kEstSampleThreads, 0, st>>>(p);
     } else {
       if (g.D == 128) fold_exact_max_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
       else fold_exact_max_kernel<64><<<grid, kEstThreads, 0, st>>>(p);
@@ -176,33 +177,62 @@ int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
-template <int D, bool GATHER>
-int launch_scan_t(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
-  using LO = ScanLayout<D, GATHER>;
-  // two CTAs per SM when a useful ring fits, else one with a deeper ring
-  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
-  int stages, vr = GATHER ? 3 : 1;
-  const int fixed2 = LO::total(0, vr, p.R);
-  stages = (per_cta2 - fixed2) / (LO::kStage + 16);
-  if (stages < 3) {
-    const int fixed1 = LO::total(0, vr, p.R);
-    stages = (kSmemPerCtaMax - fixed1) / (LO::kStage + 16);
-  }
-  if (stages > 8) stages = 8;
-  if (stages < 2) return FOLD_EUNSUPPORTED;
-  p.stages = stages;
-  p.vr = vr;
-  const int smem = LO::total(stages, vr, p.R);
-  static int configured[64] = {0};
+template <typename Kernel>
+int opt_in_smem(Kernel k, int *configured) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return FOLD_ECUDA;
-  if (dev < 0 || dev >= 64 || configured[dev] < smem) {
-    if (cudaFuncSetAttribute(fold_scan_kernel<D, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kSmemPerCtaMax) != cudaSuccess)
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax) != cudaSuccess)
       return FOLD_ECUDA;
-    if (dev >= 0 && dev < 64) configured[dev] = kSmemPerCtaMax;
+    if (dev >= 0 && dev < 64) configured[dev] = 1;
   }
-  fold_scan_kernel<D, GATHER><<<grid, kScanThreads, smem, st>>>(mk, mv, p);
+  return FOLD_OK;
+}
+
+// Ring depths: two CTAs per SM when a useful ring fits, else one CTA with a deeper ring.
+template <int D>
+int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LO = DenseLayout<D>;
+  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  int stages = (per_cta2 - LO::total(0, p.R)) / (LO::kStage + 16);
+  if (stages < 3) stages = (kSmemPerCtaMax - LO::total(0, p.R)) / (LO::kStage + 16);
+  if (stages > 8) stages = 8;
+#ifdef FOLD_TUNING
+  if (const char *e = getenv("FOLD_TUNE_STAGES")) stages = atoi(e);
+#endif
+  if (stages < 2) return FOLD_EUNSUPPORTED;
+  p.stages = stages;
+  p.vr = 0;
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_dense_kernel<D>, configured)) return rc;
+  fold_scan_dense_kernel<D><<<grid, kDenseThreads, LO::total(stages, p.R), st>>>(mk, mv, p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+// Gated scan: value slots hold rows whose requests can only be issued after scoring, so shared
+// memory is split between the key ring and the value slots of each slice.
+template <int D>
+int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LO = GatedLayout<D>;
+  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  int vr = 2;
+  int stages = (per_cta2 - LO::total(0, vr, p.R)) / (LO::kKTile + 16);
+  if (stages < 2) {
+    vr = 3;
+    stages = (kSmemPerCtaMax - LO::total(0, vr, p.R)) / (LO::kKTile + 16);
+  }
+  if (stages > 8) stages = 8;
+#ifdef FOLD_TUNING
+  if (const char *e = getenv("FOLD_TUNE_STAGES")) stages = atoi(e);
+  if (const char *e = getenv("FOLD_TUNE_VR")) vr = atoi(e);
+  if (const char *e = getenv("FOLD_TUNE_BOXMIN")) p.box_min = atoi(e);
+#endif
+  if (stages < 2 || vr < 1 || LO::total(stages, vr, p.R) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
+  p.stages = stages;
+  p.vr = vr;
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_gated_kernel<D>, configured)) return rc;
+  fold_scan_gated_kernel<D><<<grid, kGatedThreads, LO::total(stages, vr, p.R), st>>>(mk, mvs, p);
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
@@ -220,10 +250,12 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const fold_kv &kv = a->kv;
   const bool paged = kv.page_table != nullptr;
   const int box_tok = paged ? (kv.page_size < kTileKeys ? kv.page_size : kTileKeys) : kTileKeys;
+  const bool gated = !isinf(a->depth_T);
   CUtensorMap mk, mv;
   MapAxes axes;
   if (int rc = make_map(&mk, &axes, kv.k, kv, g.D, g.Hkv, box_tok)) return rc;
-  if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, box_tok)) return rc;
+  // dense: value tiles like key tiles; gated: a box of one 16-key slice
+  if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, gated ? 16 : box_tok)) return rc;
 
   ScanParams p;
   memset(&p, 0, sizeof(p));
@@ -249,9 +281,9 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
 
   if (cudaMemsetAsync(a->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
   const dim3 grid(p.num_splits, g.Hkv, g.num_seqs);
-  const bool gather = !isinf(a->depth_T);
-  if (g.D == 128) return gather ? launch_scan_t<128, true>(mk, mv, p, grid, st) : launch_scan_t<128, false>(mk, mv, p, grid, st);
-  return gather ? launch_scan_t<64, true>(mk, mv, p, grid, st) : launch_scan_t<64, false>(mk, mv, p, grid, st);
+  p.box_min = 13;
+  if (g.D == 128) return gated ? launch_gated<128>(mk, mv, p, grid, st) : launch_dense<128>(mk, mv, p, grid, st);
+  return gated ? launch_gated<64>(mk, mv, p, grid, st) : launch_dense<64>(mk, mv, p, grid, st);
 }
 
 void fill_partials(const fold_args *a, const Geometry &g, fold_partials *dst) {
@@ -314,8 +346,8 @@ int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream st
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(g.Hkv, g.B);
-  if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
-  else fold_estimate_kernel<64><<<grid, kEstThreads, 0, st>>>(p);
+  if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstSampleThreads, 0, st>>>(p);
+  else fold_estimate_kernel<64><<<grid, kEstSampleThreads, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 

@@ -64,10 +64,15 @@ __device__ __forceinline__ int est_sample_key(int i, int n) {
   return (e0 + e1) >> 1;
 }
 
+// One CTA per (kv head, request).  Four threads share a sampled key row (a quarter of its
+// channels each), so all 192 rows are requested at once and the kernel pays one memory
+// latency; warp g then reduces row g of the group.
+constexpr int kEstSampleThreads = 4 * kEstSamples;       // 768
+
 template <int D>
-__global__ void __launch_bounds__(kEstThreads) fold_estimate_kernel(const EstParams p) {
-  constexpr int EPL = D / 32;                       // elements per lane
-  __shared__ float qs[kMaxRows][D];
+__global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const EstParams p) {
+  constexpr int QD = D / 4;                         // channels per thread
+  __shared__ float qs[kMaxRows][D + 4];             // quarter q padded by one float: no bank conflicts
   __shared__ float sc[kMaxRows][kEstSamples];
   const int kvh = blockIdx.x, req = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -79,55 +84,65 @@ __global__ void __launch_bounds__(kEstThreads) fold_estimate_kernel(const EstPar
     lens[l] = level_len(p.lv[l], req);
     n += lens[l];
   }
-  for (int i = threadIdx.x; i < G * D; i += kEstThreads) {
-    const int g = i / D, d = i % D;
-    qs[g][d] = __bfloat162float(p.q[(long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + d]);
-  }
-  __syncthreads();
-
   const int n_samples = n < kEstSamples ? n : kEstSamples;
-  for (int i = warp; i < n_samples; i += kEstThreads / 32) {
+  const int i = threadIdx.x >> 2, part = threadIdx.x & 3;
+
+  // request this thread's quarter row first, then stage q while it is in flight
+  uint4 raw[QD / 8];
+#pragma unroll
+  for (int c = 0; c < QD / 8; ++c) raw[c] = make_uint4(0, 0, 0, 0);
+  if (i < n_samples) {
     int j = est_sample_key(i, n), l = 0;
     while (l < p.n_levels - 1 && j >= lens[l]) { j -= lens[l]; ++l; }
-    const __nv_bfloat16 *row = key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + lane * EPL;
-    float kf[EPL];
-    if (EPL == 4) {
-      const uint2 w = *reinterpret_cast<const uint2 *>(row);
-      const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&w.x);
-      const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&w.y);
-      kf[0] = __low2float(a); kf[1] = __high2float(a); kf[EPL - 2] = __low2float(b); kf[EPL - 1] = __high2float(b);
-    } else {
-      const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(row);
-      kf[0] = __low2float(a); kf[1] = __high2float(a);
-    }
-    for (int g = 0; g < G; ++g) {
-      float acc = 0.f;
+    const uint4 *row = reinterpret_cast<const uint4 *>(key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + part * QD);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) acc = fmaf(kf[e], qs[g][lane * EPL + e], acc);
-#pragma unroll
-      for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
-      if (lane == 0) sc[g][i] = acc * p.scale_log2;
-    }
+    for (int c = 0; c < QD / 8; ++c) raw[c] = row[c];
+  }
+  for (int e = threadIdx.x; e < G * D; e += kEstSampleThreads) {
+    const int g = e / D, d = e % D;
+    qs[g][(d / QD) * (QD + 1) + d % QD] =
+        __bfloat162float(p.q[(long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + d]);
   }
   __syncthreads();
 
-  for (int g = warp; g < G; g += kEstThreads / 32) {
+  float kf[QD];
+#pragma unroll
+  for (int c = 0; c < QD / 8; ++c) {
+    const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      kf[c * 8 + 2 * e] = __uint_as_float(w[e] << 16);
+      kf[c * 8 + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+    }
+  }
+  for (int g = 0; g < G; ++g) {
+    float acc = 0.f;
+#pragma unroll
+    for (int e = 0; e < QD; ++e) acc = fmaf(kf[e], qs[g][part * (QD + 1) + e], acc);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+    if (part == 0 && i < n_samples) sc[g][i] = acc * p.scale_log2;
+  }
+  __syncthreads();
+
+  for (int g = warp; g < G; g += kEstSampleThreads / 32) {
     float zval = 0.f;
     if (n_samples > 0) {
       float m = -INFINITY;
-      for (int i = lane; i < n_samples; i += 32) m = fmaxf(m, sc[g][i]);
+      for (int k = lane; k < n_samples; k += 32) m = fmaxf(m, sc[g][k]);
 #pragma unroll
       for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
       float total = 0.f;
       if (n <= kEstSamples) {
-        for (int i = lane; i < n_samples; i += 32) total += exp2f(sc[g][i] - m);
+        for (int k = lane; k < n_samples; k += 32) total += exp2f(sc[g][k] - m);
       } else {
-        for (int i = lane; i <= kEstRecent; i += 32) total += exp2f(sc[g][i] - m);      // sink + 63 recent
+        for (int k = lane; k <= kEstRecent; k += 32) total += exp2f(sc[g][k] - m);      // sink + 63 recent
         // trimmed mean of the 128 centre weights: drop the 8 largest (ties broken by index)
         float kept = 0.f;
         for (int k = lane; k < kEstStrata; k += 32) {
           const float wk = sc[g][1 + kEstRecent + k];
           int rank = 0;
+#pragma unroll 8
           for (int j = 0; j < kEstStrata; ++j) {
             const float wj = sc[g][1 + kEstRecent + j];
             rank += (wj > wk || (wj == wk && j < k)) ? 1 : 0;

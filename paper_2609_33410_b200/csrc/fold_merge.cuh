@@ -11,7 +11,8 @@
 
 namespace fold {
 
-constexpr int kMergeSlices = 8;
+constexpr int kMergeSlices = 4;
+constexpr int kMergeCache = 8;
 
 struct MergeLevel {
   const float *slots;
@@ -42,8 +43,10 @@ __device__ __forceinline__ double pow2_double(int e) {       // 2^e, e in the no
 }
 
 // grid (Hq, batch); block (D, kMergeSlices).  Thread (x, y): element x of A (and, for
-// x == 0, L as well) over the slots k = y, y + kMergeSlices, ...
-__global__ void __launch_bounds__(1024) fold_merge_kernel(const MergeParams p) {
+// x == 0, L as well) over the slots k = y, y + kMergeSlices, ... of the flattened slot list
+// of all levels.  The first kMergeCache terms of a thread stay in registers between the two
+// passes; longer lists are read again.
+__global__ void __launch_bounds__(128 * kMergeSlices) fold_merge_kernel(const MergeParams p) {
   __shared__ unsigned s_max[129];
   __shared__ unsigned long long s_sum[129];
   __shared__ float s_l;
@@ -58,51 +61,85 @@ __global__ void __launch_bounds__(1024) fold_merge_kernel(const MergeParams p) {
 
   const float *lbase[kMaxLevels];
   const float *llbase[kMaxLevels];
+  long long lstride[kMaxLevels];
   int cnt[kMaxLevels];
   unsigned C = 0;
-  for (int l = 0; l < p.n_levels; ++l) {
-    const MergeLevel &L = p.lv[l];
-    const int seq = b / L.stack;
-    int n = L.seqlens[seq];
-    n = n < 0 ? 0 : (n > L.max_seqlen ? L.max_seqlen : n);
-    cnt[l] = num_chunks_of(n);
-    C += cnt[l];
-    const int r = (b % L.stack) * G + (h % G);
-    const float *s0 = L.slots + ((long long)seq * p.Hkv + kvh) * L.max_slots * L.slot_stride;
-    lbase[l] = s0 + (long long)r * D + x;
-    llbase[l] = s0 + (long long)L.rows * D + r;
-  }
-  __syncthreads();
-
-  // pass 1: order-free maximum of |g| through the bit patterns
-  unsigned mx = 0u, mxl = 0u;
-  for (int l = 0; l < p.n_levels; ++l) {
-    const long long st = p.lv[l].slot_stride;
-    for (int k = y; k < cnt[l]; k += kMergeSlices) {
-      mx = max(mx, __float_as_uint(lbase[l][k * st]) & 0x7fffffffu);
-      if (x == 0) mxl = max(mxl, __float_as_uint(llbase[l][k * st]) & 0x7fffffffu);
+#pragma unroll
+  for (int l = 0; l < kMaxLevels; ++l) {
+    cnt[l] = 0; lbase[l] = nullptr; llbase[l] = nullptr; lstride[l] = 0;
+    if (l < p.n_levels) {
+      const MergeLevel &L = p.lv[l];
+      const int seq = b / L.stack;
+      int n = L.seqlens[seq];
+      n = n < 0 ? 0 : (n > L.max_seqlen ? L.max_seqlen : n);
+      cnt[l] = num_chunks_of(n);
+      C += cnt[l];
+      const int r = (b % L.stack) * G + (h % G);
+      const float *s0 = L.slots + ((long long)seq * p.Hkv + kvh) * L.max_slots * L.slot_stride;
+      lbase[l] = s0 + (long long)r * D + x;
+      llbase[l] = s0 + (long long)L.rows * D + r;
+      lstride[l] = L.slot_stride;
     }
   }
-  atomicMax(&s_max[x], mx);
-  if (x == 0) atomicMax(&s_max[D], mxl);
+  // term t of this thread is flattened slot y + t * kMergeSlices
+  auto locate = [&](int k, const float *&pa, const float *&pl) {
+    int l = 0;
+#pragma unroll
+    for (int i = 0; i < kMaxLevels - 1; ++i)
+      if (l == i && k >= cnt[i]) { k -= cnt[i]; l = i + 1; }
+    pa = lbase[l] + k * lstride[l];
+    pl = llbase[l] + k * lstride[l];
+  };
+  const int my_terms = ((int)C > y) ? ((int)C - y + kMergeSlices - 1) / kMergeSlices : 0;
+
+  // pass 1: order-free maximum of |g| through the bit patterns
+  float ca[kMergeCache], cl[kMergeCache];
+  unsigned mx = 0u, mxl = 0u;
+#pragma unroll
+  for (int t = 0; t < kMergeCache; ++t) {
+    ca[t] = 0.f; cl[t] = 0.f;
+    if (t < my_terms) {
+      const float *pa, *pl;
+      locate(y + t * kMergeSlices, pa, pl);
+      ca[t] = *pa;
+      if (x == 0) cl[t] = *pl;
+    }
+  }
+#pragma unroll
+  for (int t = 0; t < kMergeCache; ++t) {
+    mx = max(mx, __float_as_uint(ca[t]) & 0x7fffffffu);
+    mxl = max(mxl, __float_as_uint(cl[t]) & 0x7fffffffu);
+  }
+  for (int t = kMergeCache; t < my_terms; ++t) {
+    const float *pa, *pl;
+    locate(y + t * kMergeSlices, pa, pl);
+    mx = max(mx, __float_as_uint(*pa) & 0x7fffffffu);
+    if (x == 0) mxl = max(mxl, __float_as_uint(*pl) & 0x7fffffffu);
+  }
+  __syncthreads();                                   // s_max / s_sum are zeroed
+  if (mx) atomicMax(&s_max[x], mx);
+  if (x == 0 && mxl) atomicMax(&s_max[D], mxl);
   __syncthreads();
 
   // pass 2: integer sums on the declared grid
   {
     const unsigned ma = s_max[x], ml = s_max[D];
-    const int sh_a = grid_shift(ma, C), sh_l = grid_shift(ml, C);
-    const double mul_a = pow2_double(sh_a), mul_l = pow2_double(sh_l);
+    const double mul_a = pow2_double(grid_shift(ma, C)), mul_l = pow2_double(grid_shift(ml, C));
     const bool fin_a = (ma >> 23) != 255u, fin_l = (ml >> 23) != 255u;
     long long acc = 0, accl = 0;
-    for (int l = 0; l < p.n_levels; ++l) {
-      const long long st = p.lv[l].slot_stride;
-      for (int k = y; k < cnt[l]; k += kMergeSlices) {
-        if (fin_a) acc += __double2ll_rn((double)lbase[l][k * st] * mul_a);
-        if (x == 0 && fin_l) accl += __double2ll_rn((double)llbase[l][k * st] * mul_l);
-      }
+#pragma unroll
+    for (int t = 0; t < kMergeCache; ++t) {
+      if (fin_a) acc += __double2ll_rn((double)ca[t] * mul_a);
+      if (x == 0 && fin_l) accl += __double2ll_rn((double)cl[t] * mul_l);
     }
-    atomicAdd(&s_sum[x], (unsigned long long)acc);
-    if (x == 0) atomicAdd(&s_sum[D], (unsigned long long)accl);
+    for (int t = kMergeCache; t < my_terms; ++t) {
+      const float *pa, *pl;
+      locate(y + t * kMergeSlices, pa, pl);
+      if (fin_a) acc += __double2ll_rn((double)*pa * mul_a);
+      if (x == 0 && fin_l) accl += __double2ll_rn((double)*pl * mul_l);
+    }
+    if (acc) atomicAdd(&s_sum[x], (unsigned long long)acc);
+    if (x == 0 && accl) atomicAdd(&s_sum[D], (unsigned long long)accl);
   }
   __syncthreads();
 
@@ -115,7 +152,7 @@ __global__ void __launch_bounds__(1024) fold_merge_kernel(const MergeParams p) {
     else Lf = (float)((double)(long long)s_sum[D] * pow2_double(-grid_shift(ml, C)));
     s_l = Lf;
   }
-  // every y == 0 thread passes the same barrier count: use a named barrier over D threads
+  // only the y == 0 threads are left: a named barrier over those D threads
   asm volatile("bar.sync 2, %0;" ::"r"(D) : "memory");
   const float Lf = s_l;
   const unsigned ma = s_max[x];

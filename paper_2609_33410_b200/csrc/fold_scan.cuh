@@ -1,20 +1,39 @@
 // Split-KV scan (Algorithm 1, rebuilt for a BF16 cache on sm_100a).
 //
-// One CTA = 4 consumer warps + 1 producer warp, walking the 64-key tiles of its canonical
-// chunks for one (KV sequence, kv head).  The producer thread stages K (and, for dense
-// decode, V) tiles HBM -> shared memory with TMA through a ring of mbarriers.  Each
-// consumer warp owns 16 keys of every tile: BF16 mma.sync scores them against the row
-// block (query rows on M, keys on N), forms the final FP32 weights 2^(s - Z), gates them
-// by the depth T, and multiplies the two-term BF16 weights into its FP32 A accumulator
-// (rows on M, channels on N, its 16 keys on K).  With a finite depth, value rows are
-// fetched only after scoring, row by row, by zero-filling 16-byte async copies, so cut
-// rows cost no memory traffic.  At the end of a chunk the four warps' partials are added
-// in a fixed order and the chunk's (A, L) goes to its own slot.
+// A CTA walks the 64-key tiles of its canonical chunks for one (KV sequence, kv head).  A
+// producer thread stages tiles HBM -> shared memory with TMA through a ring of mbarriers.
+// Every tile is cut into four 16-key slices; slice w of every tile belongs to warp w of a
+// role, which keeps the instruction sequence that forms a chunk's (A, L) independent of the
+// grid, the batch and the split count.
+//
+//   scores   BF16 mma.sync, query rows on M (padded to 16), the slice's 16 keys on N
+//   weights  p = 2^(s - Z) in FP32, final when computed; the depth gate s - Z >= -T decides
+//            per row whether a key's value is used; L sums every key's weight
+//   values   two-term BF16 weights (P_hi + P_lo) times V, rows on M, channels on N, the
+//            slice's 16 keys on K, FP32 accumulate
+//
+// Two kernels share that arithmetic:
+//   fold_scan_dense_kernel (T = inf): K and V tiles arrive together by TMA; four consumer
+//     warps score and multiply in place.
+//   fold_scan_gated_kernel (finite T): only K is prefetched.  Four scorer warps score a
+//     slice, publish its weights and request just the value rows some row of the group
+//     keeps (one bulk async copy per row); four multiplier warps wait for those rows and
+//     accumulate A.  Scoring never waits for values and values never wait for keys, so both
+//     memory latencies are covered by ring depth, and cut rows cost no traffic.
+// At the end of a chunk the four warps of a role add their partials in a fixed order and
+// write the chunk's slot.
 #pragma once
 
 #include "fold_common.cuh"
 
 namespace fold {
+
+#ifndef FOLD_QK_CHAINS_DENSE
+#define FOLD_QK_CHAINS_DENSE 1
+#endif
+#ifndef FOLD_QK_CHAINS_GATED
+#define FOLD_QK_CHAINS_GATED 1
+#endif
 
 struct ScanParams {
   const __nv_bfloat16 *q;
@@ -22,7 +41,7 @@ struct ScanParams {
   const float *z;
   const int *seqlens;
   const int *page_table;
-  const __nv_bfloat16 *v;                         // gather path reads value rows directly
+  const __nv_bfloat16 *v;                         // gated path reads value rows directly
   long long v_stride_seq, v_stride_tok, v_stride_head;
   float *slots;
   long long slot_stride;
@@ -31,48 +50,291 @@ struct ScanParams {
   int paged, page_shift, max_pages, num_pages, box_tok;
   int num_splits, stages, vr;
   int pos_tok, pos_head, pos_seq;                 // which tensor-map coordinate (1..3) each axis is
+  int box_min;                                    // gated: fetch a whole slice by one TMA box from this many live rows on
   float scale_log2, neg_T;
 };
 
-template <int D, bool GATHER>
-struct ScanLayout {
-  static constexpr int kHalves = D / 64;
+constexpr int kDenseThreads = (kConsumerWarps + 1) * 32;        // 4 consumers + producer
+constexpr int kGatedThreads = (2 * kConsumerWarps + 1) * 32;    // 4 scorers + 4 multipliers + producer
+
+// Shared-memory carve-up.  All offsets are from a 1 KB-aligned base.
+template <int D>
+struct DenseLayout {
   static constexpr int kKTile = kTileKeys * D * 2;
-  static constexpr int kStage = GATHER ? kKTile : 2 * kKTile;
-  static constexpr int kVWarp = 16 * D * 2;
-  __host__ __device__ static int pentry(int R) { return R > 8 ? 1024 : 512; }
-  __host__ __device__ static int off_vring(int stages) { return stages * kStage; }
-  __host__ __device__ static int off_pring(int stages, int vr) {
-    return off_vring(stages) + (GATHER ? kConsumerWarps * vr * kVWarp : 0);
-  }
-  __host__ __device__ static int off_flags(int stages, int vr, int R) {
-    return off_pring(stages, vr) + (GATHER ? kConsumerWarps * vr * pentry(R) : 0);
-  }
-  __host__ __device__ static int off_red(int stages, int vr, int R) {
-    return off_flags(stages, vr, R) + (GATHER ? 64 : 0);
-  }
-  __host__ __device__ static int off_redl(int stages, int vr, int R) {
-    return off_red(stages, vr, R) + kConsumerWarps * R * D * 4;
-  }
-  __host__ __device__ static int off_bar(int stages, int vr, int R) {
-    return off_redl(stages, vr, R) + kConsumerWarps * kMaxRows * 4;
-  }
+  static constexpr int kStage = 2 * kKTile;                                    // K tile then V tile
+  __host__ __device__ static int off_red(int stages) { return stages * kStage; }
+  __host__ __device__ static int off_redl(int stages, int R) { return off_red(stages) + kConsumerWarps * R * D * 4; }
+  __host__ __device__ static int off_bar(int stages, int R) { return off_redl(stages, R) + kConsumerWarps * kMaxRows * 4; }
+  __host__ __device__ static int total(int stages, int R) { return off_bar(stages, R) + 2 * stages * 8 + 1024; }
+};
+
+template <int D>
+struct GatedLayout {
+  static constexpr int kKTile = kTileKeys * D * 2;
+  static constexpr int kVRow = D * 2 + 16;          // value row + 16 B pad: conflict-free ldmatrix
+  // one slice's 16 value rows: padded rows (row-by-row fetch) or a swizzled TMA box (whole slice),
+  // so the slot is 1 KB aligned
+  static constexpr int kVSlice = ((16 * kVRow + 1023) / 1024) * 1024;
+  // a slice's weights as A-operand registers (hi and lo terms; rows 8..15 only when present) + its fetch mask
+  __host__ __device__ static int pentry(int R) { return (R > 8 ? 1024 : 512) + 32; }
+  __host__ __device__ static int off_vring(int stages) { return stages * kKTile; }
+  __host__ __device__ static int off_pring(int stages, int vr) { return off_vring(stages) + kConsumerWarps * vr * kVSlice; }
+  __host__ __device__ static int off_red(int stages, int vr, int R) { return off_pring(stages, vr) + kConsumerWarps * vr * pentry(R); }
+  __host__ __device__ static int off_redl(int stages, int vr, int R) { return off_red(stages, vr, R) + kConsumerWarps * R * D * 4; }
+  __host__ __device__ static int off_bar(int stages, int vr, int R) { return off_redl(stages, vr, R) + kConsumerWarps * kMaxRows * 4; }
+  // barriers: K full / empty per stage, then value full / empty per (slice, slot)
   __host__ __device__ static int total(int stages, int vr, int R) {
-    return off_bar(stages, vr, R) + 2 * stages * 8 + 1024;   // + slack to align the base to 1 KB
+    return off_bar(stages, vr, R) + 2 * stages * 8 + 2 * kConsumerWarps * vr * 8 + 1024;
   }
 };
 
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
-template <int D, bool GATHER>
-__global__ void __launch_bounds__(kScanThreads, 2)
-fold_scan_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                 const ScanParams p) {
-  using LO = ScanLayout<D, GATHER>;
-  constexpr int KSTEPS = D / 16;      // k-steps of the score product; also channel pairs of the value product
-  constexpr int NT = D / 8;           // 8-channel n-tiles of the A accumulator
-  constexpr int C16 = D / 8;          // 16-byte chunks per row
+// ------------------------------------------------------------------------------------------------
+// Geometry of the CTA's work: sequence length, tiles, chunks.
+struct SeqWork {
+  int n, n_tiles, ctiles, n_chunks;
+};
+__device__ __forceinline__ SeqWork seq_work(const ScanParams &p, int seq) {
+  SeqWork w;
+  int n = p.seqlens[seq];
+  w.n = n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
+  w.n_tiles = (w.n + kTileKeys - 1) / kTileKeys;
+  w.ctiles = chunk_keys_of(w.n) / kTileKeys;
+  w.n_chunks = num_chunks_of(w.n);
+  return w;
+}
 
+struct TileCursor {            // walks the tiles of chunks split, split + num_splits, ... in order
+  int c, t, t_end;
+};
+__device__ __forceinline__ TileCursor cursor_begin(const SeqWork &w, int split) {
+  TileCursor k;
+  k.c = split;
+  k.t = split * w.ctiles;
+  k.t_end = min((split + 1) * w.ctiles, w.n_tiles);
+  return k;
+}
+__device__ __forceinline__ bool cursor_valid(const TileCursor &k, const SeqWork &w) { return k.c < w.n_chunks; }
+// returns true if the tile just left was the last of its chunk
+__device__ __forceinline__ bool cursor_next(TileCursor &k, const SeqWork &w, int num_splits) {
+  if (++k.t < k.t_end) return false;
+  k.c += num_splits;
+  k.t = k.c * w.ctiles;
+  k.t_end = min((k.c + 1) * w.ctiles, w.n_tiles);
+  return true;
+}
+
+// Producer thread: TMA-stage the tiles of chunks split, split + num_splits, ... in order.
+template <int D, bool WITH_V, int STAGE_BYTES>
+__device__ __forceinline__ void produce_tiles(const CUtensorMap *tmK, const CUtensorMap *tmV, const ScanParams &p,
+                                              const SeqWork &w, int split, int kvh, int seq, uint32_t ring,
+                                              uint32_t full0, uint32_t empty0) {
+  constexpr int HALVES = D / 64;
+  constexpr int KTILE = kTileKeys * D * 2;
+  tma_prefetch_desc(tmK);
+  if (WITH_V) tma_prefetch_desc(tmV);
+  const uint64_t pol = policy_evict_first();
+  bool dead = false;
+  int stage = 0;
+  uint32_t wrapped = 0, phase = 0;                 // phase = parity of the ring round being refilled
+  const int boxes_per_tile = kTileKeys / p.box_tok;
+  const int page_mask = (1 << p.page_shift) - 1;
+  for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w); cursor_next(k, w, p.num_splits)) {
+    if (wrapped && !mbar_wait(empty0 + 8u * stage, phase ^ 1u, dead)) break;
+    const int tok0 = k.t * kTileKeys;
+    const int nbox = min(boxes_per_tile, (w.n - tok0 + p.box_tok - 1) / p.box_tok);
+    const uint32_t full = full0 + 8u * stage;
+    mbar_expect_tx(full, nbox * p.box_tok * D * 2 * (WITH_V ? 2 : 1));
+    const uint32_t kdst = ring + stage * STAGE_BYTES;
+    const uint32_t vdst = kdst + KTILE;
+    for (int bx = 0; bx < nbox; ++bx) {
+      const int j0 = tok0 + bx * p.box_tok;
+      int c_seq = seq, c_tok = j0;
+      if (p.paged) {
+        c_seq = p.page_table[(long long)seq * p.max_pages + (j0 >> p.page_shift)];
+        c_tok = j0 & page_mask;
+      }
+      // the map's axes are ordered by stride; place each coordinate where its axis sits
+      const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
+      const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
+      const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
+#pragma unroll
+      for (int h = 0; h < HALVES; ++h) {
+        const uint32_t o = (h * kTileKeys + bx * p.box_tok) * 128;
+        tma_load_4d(kdst + o, tmK, full, h * 64, c1, c2, c3, pol);
+        if (WITH_V) tma_load_4d(vdst + o, tmV, full, h * 64, c1, c2, c3, pol);
+      }
+    }
+    if (++stage == p.stages) { stage = 0; wrapped = 1u; phase ^= 1u; }
+  }
+  if (dead) atomicOr(&p.hdr->wait_timeouts, 1u);
+}
+
+// Query rows of the block as A-operand fragments, and their references.
+template <int D>
+struct RowBlock {
+  uint32_t qf[D / 16][4];
+  float z_lo, z_hi;
+  bool rv_lo, rv_hi, two_blocks;
+};
+template <int D>
+__device__ __forceinline__ void load_rows(RowBlock<D> &rb, const ScanParams &p, int seq, int kvh, int lane) {
+  const int row_lo = lane >> 2, row_hi = row_lo + 8, qcol = (lane & 3) * 2;
+  rb.rv_lo = row_lo < p.R;
+  rb.rv_hi = row_hi < p.R;
+  rb.two_blocks = p.R > 8;
+  const int req_lo = seq * p.stack + row_lo / p.G, head_lo = kvh * p.G + row_lo % p.G;
+  const int req_hi = seq * p.stack + row_hi / p.G, head_hi = kvh * p.G + row_hi % p.G;
+  const __nv_bfloat16 *ql = p.q + (long long)req_lo * p.q_stride_b + (long long)head_lo * p.q_stride_h;
+  const __nv_bfloat16 *qh = p.q + (long long)req_hi * p.q_stride_b + (long long)head_hi * p.q_stride_h;
+#pragma unroll
+  for (int kk = 0; kk < D / 16; ++kk) {
+    const int col = kk * 16 + qcol;
+    rb.qf[kk][0] = rb.rv_lo ? *reinterpret_cast<const uint32_t *>(ql + col) : 0u;
+    rb.qf[kk][1] = rb.rv_hi ? *reinterpret_cast<const uint32_t *>(qh + col) : 0u;
+    rb.qf[kk][2] = rb.rv_lo ? *reinterpret_cast<const uint32_t *>(ql + col + 8) : 0u;
+    rb.qf[kk][3] = rb.rv_hi ? *reinterpret_cast<const uint32_t *>(qh + col + 8) : 0u;
+  }
+  rb.z_lo = rb.rv_lo ? p.z[(long long)req_lo * p.Hq + head_lo] : 0.f;
+  rb.z_hi = rb.rv_hi ? p.z[(long long)req_hi * p.Hq + head_hi] : 0.f;
+}
+
+// Score one 16-key slice of the K tile at `kt` against the row block and form the weights.
+// Returns the slice's fetch mask (bit k: key k is live for some row); ah / al receive the
+// two-term BF16 weights as A-operand fragments of the value product; l_lo / l_hi accumulate
+// this thread's share of L.
+template <int D, bool GATED, int QK_CHAINS>
+__device__ __forceinline__ uint32_t score_slice(const RowBlock<D> &rb, uint32_t kt, int warp, int lane, int key0,
+                                                int n, float scale_log2, float neg_T, uint32_t (&ah)[4],
+                                                uint32_t (&al)[4], float &l_lo, float &l_hi) {
+  // S[rows, 16 keys] = Q K^T.  Lane l addresses key row (l>>4)*8 + (l&7), 16-byte chunk 2*kk + ((l>>3)&1)
+  // of the tile laid out [half][key][128 B] with the 128-byte swizzle.
+  const int k_key = warp * 16 + ((lane >> 4) << 3) + (lane & 7);
+  const uint32_t k_row = k_key * 128, k_x = ((lane >> 3) & 1) ^ (k_key & 7);
+  // QK_CHAINS independent accumulator chains keep the dependent-MMA depth short; they are added
+  // in a fixed order afterwards.
+  float acc[QK_CHAINS][2][4];
+#pragma unroll
+  for (int j = 0; j < QK_CHAINS; ++j)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[j][0][i] = acc[j][1][i] = 0.f;
+#pragma unroll
+  for (int kk = 0; kk < D / 16; ++kk) {
+    uint32_t b0, b1, b2, b3;
+    ldsm_x4(kt + (kk >> 2) * (kTileKeys * 128) + k_row + ((((2 * kk) & 7) ^ k_x) << 4), b0, b1, b2, b3);
+    mma_bf16(acc[kk % QK_CHAINS][0], rb.qf[kk], b0, b1);
+    mma_bf16(acc[kk % QK_CHAINS][1], rb.qf[kk], b2, b3);
+  }
+  float s[2][4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float v = acc[0][nt][i];
+#pragma unroll
+      for (int j = 1; j < QK_CHAINS; ++j) v += acc[j][nt][i];
+      s[nt][i] = v;
+    }
+  const int qcol = (lane & 3) * 2;
+  uint32_t livemask = 0;
+  ah[0] = ah[1] = ah[2] = ah[3] = 0u;
+  al[0] = al[1] = al[2] = al[3] = 0u;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+      if (blk == 1 && !rb.two_blocks) continue;
+      float pw[2], pm[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int kk16 = nt * 8 + qcol + e;
+        const bool ok = ((key0 + kk16) < n) && (blk ? rb.rv_hi : rb.rv_lo);
+        const float x = ok ? fmaf(s[nt][2 * blk + e], scale_log2, blk ? -rb.z_hi : -rb.z_lo) : -INFINITY;
+        const bool live = GATED ? (x >= neg_T) : ok;         // dense: every valid key is live
+        pw[e] = ex2_approx(x);                               // 2^-inf = 0 for masked keys
+        pm[e] = live ? pw[e] : 0.f;
+        if (live) livemask |= 1u << kk16;
+      }
+      // two-term BF16 split of the live weights; L sums the weights the products use, cut keys add p
+      const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
+      const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
+      const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
+      const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
+      const float add = ((h0 + g0) + (pw[0] - pm[0])) + ((h1 + g1) + (pw[1] - pm[1]));
+      if (blk) l_hi += add; else l_lo += add;
+      ah[nt * 2 + blk] = hi2;
+      al[nt * 2 + blk] = lo2;
+    }
+  }
+  return __reduce_or_sync(0xffffffffu, livemask);            // verdicts ORed over the row block
+}
+
+// A += P_hi V + P_lo V for one slice.  SWIZZLED: V rows sit in a TMA tile ([half][key][128 B], swizzled)
+// of HALF_ROWS rows per half, starting at row `row0`; otherwise in padded rows of ROW_BYTES.
+template <int D, bool SWIZZLED, int ROW_BYTES, int HALF_ROWS = kTileKeys>
+__device__ __forceinline__ void value_product(float (&o)[D / 8][4], uint32_t vbase, int row0, int lane,
+                                              const uint32_t (&ah)[4], const uint32_t (&al)[4]) {
+  const int v_key = ((lane >> 3) & 1) * 8 + (lane & 7);      // key row this lane addresses (ldmatrix.trans)
+  const uint32_t sw_row = (row0 + v_key) * 128, sw_x = (lane >> 4) ^ (v_key & 7);
+  const uint32_t pad_off = v_key * ROW_BYTES + (lane >> 4) * 16;
+#pragma unroll
+  for (int pr = 0; pr < D / 16; ++pr) {
+    uint32_t b0, b1, b2, b3;
+    if (SWIZZLED) ldsm_x4_trans(vbase + (pr >> 2) * (HALF_ROWS * 128) + sw_row + ((((2 * pr) & 7) ^ sw_x) << 4), b0, b1, b2, b3);
+    else ldsm_x4_trans(vbase + pad_off + pr * 32, b0, b1, b2, b3);
+    mma_bf16(o[2 * pr], ah, b0, b1);
+    mma_bf16(o[2 * pr], al, b0, b1);
+    mma_bf16(o[2 * pr + 1], ah, b2, b3);
+    mma_bf16(o[2 * pr + 1], al, b2, b3);
+  }
+}
+
+// Chunk end, A part: the four warps of a role park their partials, then 128 threads add them in
+// warp order and store the chunk slot's A.  `bar_id` is the role's named barrier.
+template <int D>
+__device__ __forceinline__ void reduce_store_A(float (&o)[D / 8][4], float *red, float *slot, int R, int warp,
+                                               int lane, int tid128, int bar_id) {
+  const int row_lo = lane >> 2, row_hi = row_lo + 8, qcol = (lane & 3) * 2;
+  float *mine = red + warp * R * D;
+#pragma unroll
+  for (int nt = 0; nt < D / 8; ++nt) {
+    if (row_lo < R) *reinterpret_cast<float2 *>(mine + row_lo * D + nt * 8 + qcol) = make_float2(o[nt][0], o[nt][1]);
+    if (row_hi < R) *reinterpret_cast<float2 *>(mine + row_hi * D + nt * 8 + qcol) = make_float2(o[nt][2], o[nt][3]);
+    o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+  }
+  named_bar(bar_id);
+  const int RD = R * D;
+  for (int i = tid128; i < RD; i += 128) slot[i] = ((red[i] + red[RD + i]) + red[2 * RD + i]) + red[3 * RD + i];
+  named_bar(bar_id);
+}
+// Chunk end, L part.
+__device__ __forceinline__ void reduce_store_L(float &l_lo, float &l_hi, float *redl, float *slot_l, int R, int warp,
+                                               int lane, int tid128, int bar_id) {
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  const int row_lo = lane >> 2, row_hi = row_lo + 8;
+  if ((lane & 3) == 0) {
+    if (row_lo < R) redl[warp * kMaxRows + row_lo] = l_lo;
+    if (row_hi < R) redl[warp * kMaxRows + row_hi] = l_hi;
+  }
+  l_lo = l_hi = 0.f;
+  named_bar(bar_id);
+  if (tid128 < R)
+    slot_l[tid128] = ((redl[tid128] + redl[kMaxRows + tid128]) + redl[2 * kMaxRows + tid128]) + redl[3 * kMaxRows + tid128];
+  named_bar(bar_id);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Dense decode (T = inf)
+template <int D>
+__global__ void __launch_bounds__(kDenseThreads, 2)
+fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                       const ScanParams p) {
+  using LO = DenseLayout<D>;
+  constexpr int C16 = D / 8;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -80,323 +342,267 @@ fold_scan_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
-  int n = p.seqlens[seq];
-  n = n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
-  const int n_tiles = (n + kTileKeys - 1) / kTileKeys;
-  const int ctiles = chunk_keys_of(n) / kTileKeys;
-  const int n_chunks = num_chunks_of(n);
-  if (split >= n_chunks) return;
-
-  const int stages = p.stages, vr = p.vr, R = p.R;
-  const uint32_t bar0 = base + LO::off_bar(stages, vr, R);
-  auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (stages + s); };
+  const SeqWork w = seq_work(p, seq);
+  if (split >= w.n_chunks) return;
+  const int stages = p.stages, R = p.R, n = w.n;
+  const uint32_t full0 = base + LO::off_bar(stages, R), empty0 = full0 + 8u * stages;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), kConsumerWarps);
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, kConsumerWarps);
     }
     mbar_fence_init();
   }
   __syncthreads();
 
-  // ------------------------------------------------------------------ producer
   if (warp == kConsumerWarps) {
-    if (lane == 0) {
-      tma_prefetch_desc(&tmK);
-      if (!GATHER) tma_prefetch_desc(&tmV);
-      const uint64_t pol = policy_evict_first();
-      bool dead = false;
-      int it = 0;
-      const int boxes_per_tile = kTileKeys / p.box_tok;
-      const int page_mask = (1 << p.page_shift) - 1;
-      for (int c = split; c < n_chunks && !dead; c += p.num_splits) {
-        const int t_end = min((c + 1) * ctiles, n_tiles);
-        for (int t = c * ctiles; t < t_end; ++t, ++it) {
-          const int stage = it % stages, round = it / stages;
-          if (round > 0 && !mbar_wait(empty_bar(stage), (round - 1) & 1, dead)) break;
-          const int tok0 = t * kTileKeys;
-          const int nbox = min(boxes_per_tile, (n - tok0 + p.box_tok - 1) / p.box_tok);
-          mbar_expect_tx(full_bar(stage), nbox * p.box_tok * D * 2 * (GATHER ? 1 : 2));
-          const uint32_t kdst = base + stage * LO::kStage;
-          const uint32_t vdst = kdst + LO::kKTile;
-          for (int bx = 0; bx < nbox; ++bx) {
-            const int j0 = tok0 + bx * p.box_tok;
-            int c_seq = seq, c_tok = j0;
-            if (p.paged) {
-              c_seq = p.page_table[(long long)seq * p.max_pages + (j0 >> p.page_shift)];
-              c_tok = j0 & page_mask;
-            }
-            // the map's axes are ordered by stride; place each coordinate where its axis sits
-            const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
-            const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
-            const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
-#pragma unroll
-            for (int h = 0; h < LO::kHalves; ++h) {
-              const uint32_t o = (h * kTileKeys + bx * p.box_tok) * 128;
-              tma_load_4d(kdst + o, &tmK, full_bar(stage), h * 64, c1, c2, c3, pol);
-              if (!GATHER) tma_load_4d(vdst + o, &tmV, full_bar(stage), h * 64, c1, c2, c3, pol);
-            }
-          }
-        }
-      }
-      if (dead) atomicOr(&p.hdr->wait_timeouts, 1u);
-    }
+    if (lane == 0) produce_tiles<D, true, LO::kStage>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
     return;
   }
 
-  // ------------------------------------------------------------------ consumers
-  const int row_lo = lane >> 2, row_hi = row_lo + 8;
-  const bool rv_lo = row_lo < R, rv_hi = row_hi < R;
-  const bool two_blocks = R > 8;                       // warp-uniform
-  const int qcol = (lane & 3) * 2;
-
-  uint32_t qf[KSTEPS][4];
-  float z_lo = 0.f, z_hi = 0.f;
-  {
-    const int req_lo = seq * p.stack + row_lo / p.G, head_lo = kvh * p.G + row_lo % p.G;
-    const int req_hi = seq * p.stack + row_hi / p.G, head_hi = kvh * p.G + row_hi % p.G;
-    const __nv_bfloat16 *ql = p.q + (long long)req_lo * p.q_stride_b + (long long)head_lo * p.q_stride_h;
-    const __nv_bfloat16 *qh = p.q + (long long)req_hi * p.q_stride_b + (long long)head_hi * p.q_stride_h;
+  RowBlock<D> rb;
+  load_rows<D>(rb, p, seq, kvh, lane);
+  float o[D / 8][4];
 #pragma unroll
-    for (int kk = 0; kk < KSTEPS; ++kk) {
-      const int col = kk * 16 + qcol;
-      qf[kk][0] = rv_lo ? *reinterpret_cast<const uint32_t *>(ql + col) : 0u;
-      qf[kk][1] = rv_hi ? *reinterpret_cast<const uint32_t *>(qh + col) : 0u;
-      qf[kk][2] = rv_lo ? *reinterpret_cast<const uint32_t *>(ql + col + 8) : 0u;
-      qf[kk][3] = rv_hi ? *reinterpret_cast<const uint32_t *>(qh + col + 8) : 0u;
-    }
-    if (rv_lo) z_lo = p.z[(long long)req_lo * p.Hq + head_lo];
-    if (rv_hi) z_hi = p.z[(long long)req_hi * p.Hq + head_hi];
-  }
-
-  float o[NT][4];
-#pragma unroll
-  for (int i = 0; i < NT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
   float l_lo = 0.f, l_hi = 0.f;
-
-  float *red = reinterpret_cast<float *>(gen + LO::off_red(stages, vr, R));
-  float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, vr, R));
-  const uint32_t vring = base + LO::off_vring(stages) + warp * vr * LO::kVWarp;
-  const int pentry = LO::pentry(R);
-  uint32_t *pring = reinterpret_cast<uint32_t *>(gen + LO::off_pring(stages, vr) + warp * vr * pentry);
-  const int page_mask = (1 << p.page_shift) - 1;
+  float *red = reinterpret_cast<float *>(gen + LO::off_red(stages));
+  float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, R));
 
   bool dead = false;
-  int it = 0;
-  unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
+  int stage = 0;
+  uint32_t phase = 0;
+  unsigned long long st_total = 0;
 
-  // value product of one 16-key slice: A += P_hi V + P_lo V
-  auto value_product = [&](uint32_t vbase, int rows_per_half, int key0, const uint32_t (&ah)[4],
-                           const uint32_t (&al)[4]) {
-    const int key = key0 + (((lane >> 3) & 1) << 3) + (lane & 7);
-#pragma unroll
-    for (int pr = 0; pr < KSTEPS; ++pr) {
-      uint32_t b0, b1, b2, b3;
-      ldsm_x4_trans(vbase + tile_off(key, pr * 2 + (lane >> 4), rows_per_half), b0, b1, b2, b3);
-      mma_bf16(o[2 * pr], ah, b0, b1);
-      mma_bf16(o[2 * pr], al, b0, b1);
-      mma_bf16(o[2 * pr + 1], ah, b2, b3);
-      mma_bf16(o[2 * pr + 1], al, b2, b3);
-    }
-  };
-
-  for (int c = split; c < n_chunks; c += p.num_splits) {
-    const int t_end = min((c + 1) * ctiles, n_tiles);
-    int pend = 0, vslot = 0;                                  // gather pipeline state (per chunk)
-    uint32_t pend_fetch = 0;                                  // bit i: pending tile (vslot-1-i) has rows to multiply
-    for (int t = c * ctiles; t < t_end; ++t, ++it) {
-      const int stage = it % stages, round = it / stages;
-      if (!mbar_wait(full_bar(stage), round & 1, dead)) continue;
-      const uint32_t kt = base + stage * LO::kStage;
-
-      // ---- scores: S[rows, 16 keys] = Q K^T
-      float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-      {
-        const int key = warp * 16 + ((lane >> 4) << 3) + (lane & 7);
-#pragma unroll
-        for (int kk = 0; kk < KSTEPS; ++kk) {
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(kt + tile_off(key, kk * 2 + ((lane >> 3) & 1), kTileKeys), b0, b1, b2, b3);
-          mma_bf16(s[0], qf[kk], b0, b1);
-          mma_bf16(s[1], qf[kk], b2, b3);
-        }
-      }
-      if (GATHER) {                                            // K is in registers: release the stage early
+  for (int c = split; c < w.n_chunks; c += p.num_splits) {
+    const int t_end = min((c + 1) * w.ctiles, w.n_tiles);
+    for (int t = c * w.ctiles; t < t_end; ++t) {
+      const int my_stage = stage;
+      const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+      if (!ready) continue;
+      const uint32_t kt = base + my_stage * LO::kStage;
+      const int key0 = t * kTileKeys + warp * 16;
+      uint32_t ah[4], al[4];
+      const uint32_t fetch16 = score_slice<D, false, FOLD_QK_CHAINS_DENSE>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+      st_total += min(16, max(0, n - key0));
+      if (key0 + 16 > n) {                                   // ragged tail: value rows past n may hold anything
+        for (int r = 0; r < 16; ++r)
+          if (key0 + r >= n && lane < C16)
+            *reinterpret_cast<uint4 *>(gen + my_stage * LO::kStage + LO::kKTile +
+                                       tile_off(warp * 16 + r, lane, kTileKeys)) = make_uint4(0, 0, 0, 0);
         __syncwarp();
-        if (lane == 0) mbar_arrive(empty_bar(stage));
       }
-
-      // ---- final weights against the declared reference, depth gate, mass
-      const int kwarp0 = t * kTileKeys + warp * 16;
-      uint32_t ah[4] = {0u, 0u, 0u, 0u}, al[4] = {0u, 0u, 0u, 0u};
-      uint32_t livemask = 0;
-#pragma unroll
-      for (int nt = 0; nt < 2; ++nt) {
-        float h0[2], l0[2], h1[2] = {0.f, 0.f}, l1[2] = {0.f, 0.f};
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int kk16 = nt * 8 + qcol + e;
-          const bool valid = (kwarp0 + kk16) < n;
-          {
-            const float x = fmaf(s[nt][e], p.scale_log2, -z_lo);
-            const bool ok = valid && rv_lo;
-            const bool live = ok && (x >= p.neg_T);
-            const float pw = ok ? ex2_approx(x) : 0.f;
-            float hi, lo;
-            split_bf16(pw, hi, lo);
-            l_lo += live ? (hi + lo) : pw;
-            h0[e] = live ? hi : 0.f;
-            l0[e] = live ? lo : 0.f;
-            if (live) livemask |= 1u << kk16;
-          }
-          if (two_blocks) {
-            const float x = fmaf(s[nt][2 + e], p.scale_log2, -z_hi);
-            const bool ok = valid && rv_hi;
-            const bool live = ok && (x >= p.neg_T);
-            const float pw = ok ? ex2_approx(x) : 0.f;
-            float hi, lo;
-            split_bf16(pw, hi, lo);
-            l_hi += live ? (hi + lo) : pw;
-            h1[e] = live ? hi : 0.f;
-            l1[e] = live ? lo : 0.f;
-            if (live) livemask |= 1u << kk16;
-          }
-        }
-        ah[nt * 2] = pack_bf16(h0[0], h0[1]);
-        al[nt * 2] = pack_bf16(l0[0], l0[1]);
-        ah[nt * 2 + 1] = pack_bf16(h1[0], h1[1]);
-        al[nt * 2 + 1] = pack_bf16(l1[0], l1[1]);
-      }
-      const uint32_t fetch16 = __reduce_or_sync(0xffffffffu, livemask);   // verdicts ORed over the row block
-      {
-        const int nvalid = min(16, max(0, n - kwarp0));
-        st_total += nvalid;
-        st_fetched += __popc(fetch16);
-        st_skipped += (fetch16 == 0 && nvalid > 0) ? 1 : 0;
-      }
-
-      if (!GATHER) {
-        const uint32_t vt = kt + LO::kKTile;
-        if (kwarp0 + 16 > n) {                                 // ragged tail: rows past n may hold anything
-          for (int r = 0; r < 16; ++r)
-            if (kwarp0 + r >= n && lane < C16)
-              *reinterpret_cast<uint4 *>(gen + stage * LO::kStage + LO::kKTile +
-                                         tile_off(warp * 16 + r, lane, kTileKeys)) = make_uint4(0, 0, 0, 0);
-          __syncwarp();
-        }
-        if (fetch16 != 0) value_product(vt, kTileKeys, warp * 16, ah, al);
-        if (kwarp0 + 16 > n) fence_proxy_async_smem();         // generic writes before the next TMA fill
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_bar(stage));
-      } else {
-        // ---- request the live value rows (zero-fill the rest), defer the product
-        const int slot = vslot % vr;
-        __syncwarp();                                          // earlier ldmatrix reads of this slot are done
-        if (fetch16 != 0) {
-          int c_seq = seq, c_tok = kwarp0;
-          if (p.paged) {
-            const int pg = kwarp0 < n ? p.page_table[(long long)seq * p.max_pages + (kwarp0 >> p.page_shift)] : 0;
-            c_seq = min(max(pg, 0), p.num_pages - 1);
-            c_tok = kwarp0 & page_mask;
-          }
-          const __nv_bfloat16 *vsrc = p.v + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
-                                      (long long)kvh * p.v_stride_head;
-          const uint32_t vdst = vring + slot * LO::kVWarp;
-#pragma unroll
-          for (int i = 0; i < (16 * C16) / 32; ++i) {
-            const int id = i * 32 + lane;
-            const int r = id / C16, c16 = id % C16;
-            const bool f = (fetch16 >> r) & 1u;
-            const __nv_bfloat16 *src = f ? vsrc + (long long)r * p.v_stride_tok + c16 * 8 : p.v;
-            cp_async_16(vdst + tile_off(r, c16, 16), src, f ? 16u : 0u);
-          }
-        }
-        cp_async_commit();
-        {
-          uint32_t *pe = pring + slot * (pentry / 4);
-          if (two_blocks) {
-            *reinterpret_cast<uint4 *>(pe + lane * 4) = make_uint4(ah[0], ah[1], ah[2], ah[3]);
-            *reinterpret_cast<uint4 *>(pe + 128 + lane * 4) = make_uint4(al[0], al[1], al[2], al[3]);
-          } else {
-            *reinterpret_cast<uint4 *>(pe + lane * 4) = make_uint4(ah[0], ah[2], al[0], al[2]);
-          }
-        }
-        pend_fetch = (pend_fetch << 1) | (fetch16 != 0 ? 1u : 0u);
-        ++vslot;
-        ++pend;
-      }
-
-      if (GATHER) {
-        // multiply the oldest pending tile once the ring is full, or drain at the chunk's end
-        const bool last = (t + 1 == t_end);
-        while (pend > 0 && (pend == vr || last)) {
-          switch (pend - 1) {
-            case 0: cp_async_wait<0>(); break;
-            case 1: cp_async_wait<1>(); break;
-            case 2: cp_async_wait<2>(); break;
-            default: cp_async_wait<3>(); break;
-          }
-          __syncwarp();
-          const int old = vslot - pend;
-          if ((pend_fetch >> (pend - 1)) & 1u) {
-            const uint32_t *pe = pring + (old % vr) * (pentry / 4);
-            uint32_t bh[4], bl[4];
-            if (two_blocks) {
-              const uint4 a = *reinterpret_cast<const uint4 *>(pe + lane * 4);
-              const uint4 b = *reinterpret_cast<const uint4 *>(pe + 128 + lane * 4);
-              bh[0] = a.x; bh[1] = a.y; bh[2] = a.z; bh[3] = a.w;
-              bl[0] = b.x; bl[1] = b.y; bl[2] = b.z; bl[3] = b.w;
-            } else {
-              const uint4 a = *reinterpret_cast<const uint4 *>(pe + lane * 4);
-              bh[0] = a.x; bh[1] = 0u; bh[2] = a.y; bh[3] = 0u;
-              bl[0] = a.z; bl[1] = 0u; bl[2] = a.w; bl[3] = 0u;
-            }
-            value_product(vring + (old % vr) * LO::kVWarp, 16, 0, bh, bl);
-          }
-          --pend;
-        }
-      }
+      if (fetch16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, ah, al);
+      if (key0 + 16 > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);
     }
-
-    // ---- chunk end: add the four warps' partials in a fixed order, store the slot
-    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
-    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
-    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-    {
-      float *mine = red + warp * R * D;
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        if (rv_lo) *reinterpret_cast<float2 *>(mine + row_lo * D + nt * 8 + qcol) = make_float2(o[nt][0], o[nt][1]);
-        if (rv_hi) *reinterpret_cast<float2 *>(mine + row_hi * D + nt * 8 + qcol) = make_float2(o[nt][2], o[nt][3]);
-        o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-      }
-      if ((lane & 3) == 0) {
-        if (rv_lo) redl[warp * kMaxRows + row_lo] = l_lo;
-        if (rv_hi) redl[warp * kMaxRows + row_hi] = l_hi;
-      }
-      l_lo = l_hi = 0.f;
-    }
-    consumer_bar();
-    {
-      float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
-      const int RD = R * D;
-      for (int i = threadIdx.x; i < RD; i += kConsumerWarps * 32)
-        slot[i] = ((red[i] + red[RD + i]) + red[2 * RD + i]) + red[3 * RD + i];
-      if (threadIdx.x < R)
-        slot[RD + threadIdx.x] = ((redl[threadIdx.x] + redl[kMaxRows + threadIdx.x]) +
-                                  redl[2 * kMaxRows + threadIdx.x]) + redl[3 * kMaxRows + threadIdx.x];
-    }
-    consumer_bar();
+    float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
+    reduce_store_L(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
+    reduce_store_A<D>(o, red, slot, R, warp, lane, threadIdx.x, 1);
   }
 
   if (lane == 0) {
     if (dead) atomicOr(&p.hdr->wait_timeouts, 2u);
-    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_fetched);
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_total);
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
-    if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Depth-gated decode (finite T)
+//
+// Roles.  Scorer warp w: waits for a K tile, scores slice w, releases the tile, publishes the
+// slice's weights and verdict and requests the value rows the verdict asks for into a slot of
+// its slice's value ring -- the whole slice by TMA when most rows are live, else row by row
+// with zero-filling 16-byte async copies (cut rows are not read and become zero rows).
+// Multiplier warp w: waits for a slot to land, multiplies, hands the slot back.
+template <int D>
+__global__ void __launch_bounds__(kGatedThreads, 2)
+fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
+                       const ScanParams p) {
+  using LO = GatedLayout<D>;
+  constexpr int C16 = D / 8;                                 // 16-byte chunks per value row
+  constexpr int RPI = 32 / C16;                              // rows one warp-wide async copy covers
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
+  const SeqWork w = seq_work(p, seq);
+  if (split >= w.n_chunks) return;
+  const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
+  // barriers: K full / empty per stage; value full / empty per (slice, slot)
+  const uint32_t full0 = base + LO::off_bar(stages, vr, R), empty0 = full0 + 8u * stages;
+  const uint32_t vfull0 = empty0 + 8u * stages, vempty0 = vfull0 + 8u * kConsumerWarps * vr;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, kConsumerWarps);
+    }
+    for (int s = 0; s < kConsumerWarps * vr; ++s) {
+      mbar_init(vfull0 + 8u * s, 1);
+      mbar_init(vempty0 + 8u * s, 1);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  if (warp == 2 * kConsumerWarps) {
+    if (lane == 0) produce_tiles<D, false, LO::kKTile>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
+    return;
+  }
+
+  const bool scorer = warp < kConsumerWarps;
+  const int sl = warp & 3;                                   // the slice of every tile this warp owns
+  const int pentry = LO::pentry(R), pmask = pentry - 32;
+  uint8_t *pring = gen + LO::off_pring(stages, vr) + sl * vr * pentry;
+  const uint32_t vring = base + LO::off_vring(stages) + sl * vr * LO::kVSlice;
+  const uint32_t vfull = vfull0 + 8u * sl * vr, vempty = vempty0 + 8u * sl * vr;
+  bool dead = false;
+  int vs = 0;
+  uint32_t vphase = 0, vwrapped = 0;
+
+  if (scorer) {
+    RowBlock<D> rb;
+    load_rows<D>(rb, p, seq, kvh, lane);
+    float l_lo = 0.f, l_hi = 0.f;
+    float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, vr, R));
+    const int page_mask = (1 << p.page_shift) - 1;
+    const uint64_t vpol = policy_evict_first();
+    // row-by-row fetch: lane covers 16-byte chunk (lane % C16) of rows (lane / C16) + RPI * i
+    const uint32_t rdst0 = (lane / C16) * LO::kVRow + (lane % C16) * 16;
+    const long long rsrc0 = (long long)(lane / C16) * p.v_stride_tok + (lane % C16) * 8;
+    int stage = 0;
+    uint32_t phase = 0;
+    unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
+
+    for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
+      const int my_stage = stage;
+      const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+      const int key0 = k.t * kTileKeys + sl * 16;
+      uint32_t ah[4] = {0u, 0u, 0u, 0u}, al[4] = {0u, 0u, 0u, 0u};
+      uint32_t fetch16 = 0;
+      if (ready) {
+        fetch16 = score_slice<D, true, FOLD_QK_CHAINS_GATED>(rb, base + my_stage * LO::kKTile, sl, lane, key0, n,
+                                                            p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);   // the K tile is in registers: release it
+      }
+      // a mostly-live slice is cheaper to fetch whole (two TMA boxes) than row by row; rows nobody keeps
+      // then ride along under a zero weight.  Never past the sequence end: those rows may hold anything.
+      const bool whole = (key0 + 16 <= n) && (__popc(fetch16) >= p.box_min);
+      {
+        const int nvalid = min(16, max(0, n - key0));
+        st_total += nvalid;
+        st_fetched += whole ? 16 : __popc(fetch16);
+        st_skipped += (fetch16 == 0 && nvalid > 0) ? 1 : 0;
+      }
+      if (!vwrapped || mbar_wait(vempty + 8u * vs, vphase ^ 1u, dead)) {
+        // publish the slice: weights as the value product's A-operand registers, and the verdict
+        uint8_t *pe = pring + vs * pentry;
+        if (rb.two_blocks) {
+          *reinterpret_cast<uint4 *>(pe + lane * 16) = make_uint4(ah[0], ah[1], ah[2], ah[3]);
+          *reinterpret_cast<uint4 *>(pe + 512 + lane * 16) = make_uint4(al[0], al[1], al[2], al[3]);
+        } else {
+          *reinterpret_cast<uint4 *>(pe + lane * 16) = make_uint4(ah[0], ah[2], al[0], al[2]);
+        }
+        if (lane == 0) *reinterpret_cast<uint32_t *>(pe + pmask) = fetch16 | (whole ? 0x10000u : 0u);
+        const uint32_t bar = vfull + 8u * vs;
+        if (fetch16 != 0u) {
+          int c_seq = seq, c_tok = key0;
+          if (p.paged) {
+            const int pg = p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)];
+            c_seq = min(max(pg, 0), p.num_pages - 1);
+            c_tok = key0 & page_mask;
+          }
+          const uint32_t vdst = vring + vs * LO::kVSlice;
+          if (whole) {
+            fence_proxy_async_smem();                        // the slot's earlier generic-proxy traffic, then TMA writes
+            __syncwarp();
+            if (lane == 0) {
+              mbar_expect_tx(bar, 16 * D * 2);
+              const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
+              const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
+              const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
+#pragma unroll
+              for (int h = 0; h < D / 64; ++h) tma_load_4d(vdst + h * (16 * 128), &tmVs, bar, h * 64, c1, c2, c3, vpol);
+            }
+          } else {
+            const __nv_bfloat16 *src = p.v + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
+                                       (long long)kvh * p.v_stride_head + rsrc0;
+            uint32_t dst = vdst + rdst0;
+#pragma unroll
+            for (int i = 0; i < 16 / RPI; ++i) {
+              const bool f = (fetch16 >> (i * RPI + lane / C16)) & 1u;
+              cp_async_16(dst, f ? src : p.v, f ? 16u : 0u);
+              dst += RPI * LO::kVRow;
+              src += (long long)RPI * p.v_stride_tok;
+            }
+            cp_async_mbar_arrive(bar);                       // this lane's copies hold the phase open
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar);
+          }
+        } else {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar);
+        }
+      }
+      if (++vs == vr) { vs = 0; vwrapped = 1u; vphase ^= 1u; }
+      const int c_done = k.c;
+      if (cursor_next(k, w, p.num_splits)) {
+        float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
+        reduce_store_L(l_lo, l_hi, redl, slot + R * D, R, sl, lane, threadIdx.x, 1);
+      }
+    }
+    if (lane == 0) {
+      if (dead) atomicOr(&p.hdr->wait_timeouts, 2u);
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_fetched);
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
+      if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
+    }
+  } else {
+    float o[D / 8][4];
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float *red = reinterpret_cast<float *>(gen + LO::off_red(stages, vr, R));
+    for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
+      const int my = vs;
+      const bool landed = mbar_wait(vfull + 8u * my, vphase, dead);
+      if (++vs == vr) { vs = 0; vphase ^= 1u; }
+      if (landed) {
+        const uint8_t *pe = pring + my * pentry;
+        const uint32_t verdict = *reinterpret_cast<const uint32_t *>(pe + pmask);
+        if (verdict != 0u) {
+          uint32_t ah[4], al[4];
+          const uint4 a = *reinterpret_cast<const uint4 *>(pe + lane * 16);
+          if (R > 8) {
+            const uint4 b = *reinterpret_cast<const uint4 *>(pe + 512 + lane * 16);
+            ah[0] = a.x; ah[1] = a.y; ah[2] = a.z; ah[3] = a.w;
+            al[0] = b.x; al[1] = b.y; al[2] = b.z; al[3] = b.w;
+          } else {
+            ah[0] = a.x; ah[1] = 0u; ah[2] = a.y; ah[3] = 0u;
+            al[0] = a.z; al[1] = 0u; al[2] = a.w; al[3] = 0u;
+          }
+          if (verdict & 0x10000u) value_product<D, true, 0, 16>(o, vring + my * LO::kVSlice, 0, lane, ah, al);
+          else value_product<D, false, LO::kVRow>(o, vring + my * LO::kVSlice, 0, lane, ah, al);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(vempty + 8u * my);
+      }
+      const int c_done = k.c;
+      if (cursor_next(k, w, p.num_splits)) {
+        float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
+        reduce_store_A<D>(o, red, slot, R, sl, lane, threadIdx.x - 128, 2);
+      }
+    }
+    if (lane == 0 && dead) atomicOr(&p.hdr->wait_timeouts, 4u);
   }
 }
 
