@@ -129,6 +129,20 @@ int make_map(CUtensorMap *map, MapAxes *axes, const void *ptr, const fold_kv &kv
 }
 
 // ------------------------------------------------------------------ launches
+// Launch with programmatic stream serialization: the kernel may begin (its prologue, up to its
+// griddepcontrol.wait) while the kernel before it in the stream drains.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 KvLevel kv_level(const fold_kv &kv, int stack) {
   KvLevel L;
   L.k = static_cast<const __nv_bfloat16 *>(kv.k);
@@ -205,7 +219,8 @@ int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, di
   p.vr = 0;
   static int configured[64] = {0};
   if (int rc = opt_in_smem(fold_scan_dense_kernel<D>, configured)) return rc;
-  fold_scan_dense_kernel<D><<<grid, kDenseThreads, LO::total(stages, p.R), st>>>(mk, mv, p);
+  if (launch_pdl(fold_scan_dense_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
+    return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
@@ -232,7 +247,8 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
   p.vr = vr;
   static int configured[64] = {0};
   if (int rc = opt_in_smem(fold_scan_gated_kernel<D>, configured)) return rc;
-  fold_scan_gated_kernel<D><<<grid, kGatedThreads, LO::total(stages, vr, p.R), st>>>(mk, mvs, p);
+  if (launch_pdl(fold_scan_gated_kernel<D>, grid, dim3(kGatedThreads), LO::total(stages, vr, p.R), st, mk, mvs, p) != cudaSuccess)
+    return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
@@ -240,7 +256,7 @@ int choose_splits(const fold_args *a, const Geometry &g) {
   const int max_chunks = num_chunks_of(a->kv.max_seqlen) > 0 ? num_chunks_of(a->kv.max_seqlen) : 1;
   if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
   const long long units = (long long)g.num_seqs * g.Hkv;
-  const long long target = 8LL * 296;
+  const long long target = 6LL * 296;
   long long per_cta = units * max_chunks / target;
   if (per_cta < 1) per_cta = 1;
   return (int)((max_chunks + per_cta - 1) / per_cta);
@@ -279,7 +295,6 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
   p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
 
-  if (cudaMemsetAsync(a->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
   const dim3 grid(p.num_splits, g.Hkv, g.num_seqs);
   p.box_min = 13;
   if (g.D == 128) return gated ? launch_gated<128>(mk, mv, p, grid, st) : launch_dense<128>(mk, mv, p, grid, st);
@@ -358,6 +373,8 @@ int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream str
   if (!args->workspace || !aligned(args->workspace, 256)) return FOLD_EINVAL;
   if (args->workspace_bytes < kHeaderBytes + g.slot_bytes) return FOLD_EWORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // header first, so that reference -> scan -> partial add are adjacent kernels in the stream
+  if (cudaMemsetAsync(args->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
   if (int rc = launch_reference(args, g, st)) return rc;
   if (int rc = launch_scan(args, g, st)) return rc;
   fill_partials(args, g, dst);
@@ -389,8 +406,13 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
   p.lse = lse; p.row_status = row_status;
   p.n_levels = n_levels; p.Hq = p0->num_q_heads; p.Hkv = p0->num_kv_heads;
   p.G = p0->num_q_heads / p0->num_kv_heads; p.D = p0->head_dim;
-  const dim3 grid(p.Hq, p0->batch), block(p.D, kMergeSlices);
-  fold_merge_kernel<<<grid, block, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  // slices per row: about 16 slots per thread, so short slot lists do not pay for idle threads
+  int total_slots = 0;
+  for (int l = 0; l < n_levels; ++l) total_slots += max_chunks_upto(levels[l]->max_seqlen);
+  int slices = (total_slots + 15) / 16;
+  slices = slices < 1 ? 1 : (slices > kMergeMaxSlices ? kMergeMaxSlices : slices);
+  const dim3 grid(p.Hq, p0->batch), block(p.D, slices);
+  if (launch_pdl(fold_merge_kernel, grid, block, 0, static_cast<cudaStream_t>(stream), p) != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 

@@ -72,11 +72,12 @@ constexpr int kEstSampleThreads = 4 * kEstSamples;       // 768
 template <int D>
 __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const EstParams p) {
   constexpr int QD = D / 4;                         // channels per thread
-  __shared__ float qs[kMaxRows][D + 4];             // quarter q padded by one float: no bank conflicts
-  __shared__ float sc[kMaxRows][kEstSamples];
+  __shared__ __align__(16) float qs[kMaxRows][D + 16];   // each quarter of q padded by 4 floats: aligned float4 reads, spread banks
+  __shared__ __align__(16) float sc[kMaxRows][kEstSamples];
   const int kvh = blockIdx.x, req = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G;
+  pdl_launch_dependents();                           // the scan may set up while the estimate runs
 
   int lens[kMaxLevels];
   int n = 0;
@@ -100,7 +101,7 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
   }
   for (int e = threadIdx.x; e < G * D; e += kEstSampleThreads) {
     const int g = e / D, d = e % D;
-    qs[g][(d / QD) * (QD + 1) + d % QD] =
+    qs[g][(d / QD) * (QD + 4) + d % QD] =
         __bfloat162float(p.q[(long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + d]);
   }
   __syncthreads();
@@ -117,43 +118,70 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
   }
   for (int g = 0; g < G; ++g) {
     float acc = 0.f;
+    const float4 *qv = reinterpret_cast<const float4 *>(&qs[g][part * (QD + 4)]);
 #pragma unroll
-    for (int e = 0; e < QD; ++e) acc = fmaf(kf[e], qs[g][part * (QD + 1) + e], acc);
+    for (int e = 0; e < QD / 4; ++e) {
+      const float4 t = qv[e];
+      acc = fmaf(kf[4 * e], t.x, acc);
+      acc = fmaf(kf[4 * e + 1], t.y, acc);
+      acc = fmaf(kf[4 * e + 2], t.z, acc);
+      acc = fmaf(kf[4 * e + 3], t.w, acc);
+    }
     acc += __shfl_xor_sync(0xffffffffu, acc, 1);
     acc += __shfl_xor_sync(0xffffffffu, acc, 2);
     if (part == 0 && i < n_samples) sc[g][i] = acc * p.scale_log2;
   }
   __syncthreads();
 
+  // row maxima (warp g), then every thread takes one (row, sample): its weight, and for a stratum
+  // centre its rank among the 128 centres (the 8 largest are dropped; ties broken by index)
+  __shared__ float rmax[kMaxRows];
+  __shared__ float wt[kMaxRows][kEstSamples];
+  for (int g = warp; g < G; g += kEstSampleThreads / 32) {
+    float m = -INFINITY;
+    for (int k = lane; k < n_samples; k += 32) m = fmaxf(m, sc[g][k]);
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+    if (lane == 0) rmax[g] = m;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < G * kEstSamples; e += kEstSampleThreads) {
+    const int g = e / kEstSamples, k = e % kEstSamples;
+    float wv = 0.f;
+    if (k < n_samples) {
+      const float sk = sc[g][k];
+      bool keep = true;
+      if (n > kEstSamples && k > kEstRecent) {
+        int rank = 0;
+        const float4 *cv = reinterpret_cast<const float4 *>(&sc[g][1 + kEstRecent]);
+#pragma unroll 8
+        for (int j4 = 0; j4 < kEstStrata / 4; ++j4) {
+          const float4 t = cv[j4];
+          const int j = 1 + kEstRecent + 4 * j4;
+          rank += (t.x > sk || (t.x == sk && j < k)) ? 1 : 0;
+          rank += (t.y > sk || (t.y == sk && j + 1 < k)) ? 1 : 0;
+          rank += (t.z > sk || (t.z == sk && j + 2 < k)) ? 1 : 0;
+          rank += (t.w > sk || (t.w == sk && j + 3 < k)) ? 1 : 0;
+        }
+        keep = rank >= kEstTrim;
+      }
+      if (keep) wv = exp2f(sk - rmax[g]);
+    }
+    wt[g][k] = wv;
+  }
+  __syncthreads();
   for (int g = warp; g < G; g += kEstSampleThreads / 32) {
     float zval = 0.f;
     if (n_samples > 0) {
-      float m = -INFINITY;
-      for (int k = lane; k < n_samples; k += 32) m = fmaxf(m, sc[g][k]);
-#pragma unroll
-      for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
-      float total = 0.f;
-      if (n <= kEstSamples) {
-        for (int k = lane; k < n_samples; k += 32) total += exp2f(sc[g][k] - m);
-      } else {
-        for (int k = lane; k <= kEstRecent; k += 32) total += exp2f(sc[g][k] - m);      // sink + 63 recent
-        // trimmed mean of the 128 centre weights: drop the 8 largest (ties broken by index)
-        float kept = 0.f;
-        for (int k = lane; k < kEstStrata; k += 32) {
-          const float wk = sc[g][1 + kEstRecent + k];
-          int rank = 0;
-#pragma unroll 8
-          for (int j = 0; j < kEstStrata; ++j) {
-            const float wj = sc[g][1 + kEstRecent + j];
-            rank += (wj > wk || (wj == wk && j < k)) ? 1 : 0;
-          }
-          if (rank >= kEstTrim) kept += exp2f(wk - m);
-        }
-        total += kept * ((float)(n - 1 - kEstRecent) / (float)(kEstStrata - kEstTrim));
-      }
+      float exact = 0.f, kept = 0.f;                 // fixed summation order: lane-strided, then a shuffle tree
+      const int n_exact = n <= kEstSamples ? n_samples : 1 + kEstRecent;
+      for (int k = lane; k < n_exact; k += 32) exact += wt[g][k];
+      if (n > kEstSamples)
+        for (int k = 1 + kEstRecent + lane; k < kEstSamples; k += 32) kept += wt[g][k];
+      float total = exact + kept * ((float)(n - 1 - kEstRecent) / (float)(kEstStrata - kEstTrim));
 #pragma unroll
       for (int k = 16; k > 0; k >>= 1) total += __shfl_xor_sync(0xffffffffu, total, k);
-      zval = m + log2f(total);
+      zval = rmax[g] + log2f(total);
     }
     if (lane == 0) p.z[(long long)req * p.Hq + kvh * G + g] = zval;
   }

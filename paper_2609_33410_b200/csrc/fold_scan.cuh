@@ -355,6 +355,8 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     mbar_fence_init();
   }
   __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();                                                // z (and the zeroed header) come from earlier work
 
   if (warp == kConsumerWarps) {
     if (lane == 0) produce_tiles<D, true, LO::kStage>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
@@ -452,6 +454,8 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     mbar_fence_init();
   }
   __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();                                                // z (and the zeroed header) come from earlier work
 
   if (warp == 2 * kConsumerWarps) {
     if (lane == 0) produce_tiles<D, false, LO::kKTile>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
@@ -482,9 +486,18 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     uint32_t phase = 0;
     unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
 
+#ifdef FOLD_PROFILE
+    long long pf[4] = {0, 0, 0, 0};
+#endif
     for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
       const int my_stage = stage;
+#ifdef FOLD_PROFILE
+      const long long c0 = clock64();
+#endif
       const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
+#ifdef FOLD_PROFILE
+      const long long c1 = clock64();
+#endif
       if (++stage == stages) { stage = 0; phase ^= 1u; }
       const int key0 = k.t * kTileKeys + sl * 16;
       uint32_t ah[4] = {0u, 0u, 0u, 0u}, al[4] = {0u, 0u, 0u, 0u};
@@ -504,7 +517,14 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         st_fetched += whole ? 16 : __popc(fetch16);
         st_skipped += (fetch16 == 0 && nvalid > 0) ? 1 : 0;
       }
+#ifdef FOLD_PROFILE
+      const long long c2 = clock64();
+      const bool vok = !vwrapped || mbar_wait(vempty + 8u * vs, vphase ^ 1u, dead);
+      const long long c3 = clock64();
+      if (vok) {
+#else
       if (!vwrapped || mbar_wait(vempty + 8u * vs, vphase ^ 1u, dead)) {
+#endif
         // publish the slice: weights as the value product's A-operand registers, and the verdict
         uint8_t *pe = pring + vs * pentry;
         if (rb.two_blocks) {
@@ -555,6 +575,10 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       }
       if (++vs == vr) { vs = 0; vwrapped = 1u; vphase ^= 1u; }
+#ifdef FOLD_PROFILE
+      const long long c4 = clock64();
+      pf[0] += c1 - c0; pf[1] += c2 - c1; pf[2] += c3 - c2; pf[3] += c4 - c3;
+#endif
       const int c_done = k.c;
       if (cursor_next(k, w, p.num_splits)) {
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
@@ -566,6 +590,10 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_fetched);
       atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
       if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
+#ifdef FOLD_PROFILE
+      if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && warp == 0)
+        for (int i = 0; i < 4; ++i) p.hdr->pad[i] = (unsigned long long)pf[i];
+#endif
     }
   } else {
     float o[D / 8][4];
