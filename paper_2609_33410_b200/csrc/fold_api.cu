@@ -17,6 +17,7 @@ constexpr size_t kHeaderBytes = 256;
 constexpr int kSmemPerSm = 233472;       // 228 KB per SM
 constexpr int kSmemPerCtaMax = 232448;   // 227 KB opt-in per CTA
 constexpr int kSmemCtaReserve = 1024;
+constexpr long long kMaxStackedRows = 4096;   // query rows stacked on one (sequence, kv head)
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
@@ -60,7 +61,7 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   if (need_out && (!a->out || !aligned(a->out, 2))) return FOLD_EINVAL;
   const int G = a->num_q_heads / a->num_kv_heads;
   const long long R = (long long)a->stack * G;
-  if (R > kMaxRows) return FOLD_EUNSUPPORTED;
+  if (G > kMaxRows || R > kMaxStackedRows) return FOLD_EUNSUPPORTED;
   g->B = a->batch; g->Hq = a->num_q_heads; g->Hkv = a->num_kv_heads; g->G = G; g->D = a->head_dim;
   g->stack = a->stack; g->R = (int)R; g->num_seqs = a->kv.num_seqs;
   g->max_slots = max_chunks_upto(a->kv.max_seqlen);
@@ -224,6 +225,30 @@ int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, di
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+// Stacked rows: the dense ring without reduction buffers; one CTA per (split, 64-row group).
+template <int D>
+int launch_stacked(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, bool gated, cudaStream_t st) {
+  using LO = DenseLayout<D>;
+  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  int stages = (per_cta2 - LO::total(0, 0)) / (LO::kStage + 16);
+  if (stages > 8) stages = 8;
+  if (stages < 2) return FOLD_EUNSUPPORTED;
+  p.stages = stages;
+  p.vr = 0;
+  grid.x *= (p.R + 63) / 64;
+  static int configured_g[64] = {0}, configured_d[64] = {0};
+  cudaError_t rc;
+  if (gated) {
+    if (int e = opt_in_smem(fold_scan_stacked_kernel<D, true>, configured_g)) return e;
+    rc = launch_pdl(fold_scan_stacked_kernel<D, true>, grid, dim3(kDenseThreads), LO::total(stages, 0), st, mk, mv, p);
+  } else {
+    if (int e = opt_in_smem(fold_scan_stacked_kernel<D, false>, configured_d)) return e;
+    rc = launch_pdl(fold_scan_stacked_kernel<D, false>, grid, dim3(kDenseThreads), LO::total(stages, 0), st, mk, mv, p);
+  }
+  if (rc != cudaSuccess) return FOLD_ECUDA;
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 // Gated scan: value slots hold rows whose requests can only be issued after scoring, so shared
 // memory is split between the key ring and the value slots of each slice.
 template <int D>
@@ -270,8 +295,9 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   CUtensorMap mk, mv;
   MapAxes axes;
   if (int rc = make_map(&mk, &axes, kv.k, kv, g.D, g.Hkv, box_tok)) return rc;
-  // dense: value tiles like key tiles; gated: a box of one 16-key slice
-  if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, gated ? 16 : box_tok)) return rc;
+  const bool stacked = g.R > kMaxRows;
+  // dense and stacked: value tiles like key tiles; gated: a box of one 16-key slice
+  if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, (gated && !stacked) ? 16 : box_tok)) return rc;
 
   ScanParams p;
   memset(&p, 0, sizeof(p));
@@ -297,6 +323,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
 
   const dim3 grid(p.num_splits, g.Hkv, g.num_seqs);
   p.box_min = 13;
+  if (stacked)
+    return g.D == 128 ? launch_stacked<128>(mk, mv, p, grid, gated, st) : launch_stacked<64>(mk, mv, p, grid, gated, st);
   if (g.D == 128) return gated ? launch_gated<128>(mk, mv, p, grid, st) : launch_dense<128>(mk, mv, p, grid, st);
   return gated ? launch_gated<64>(mk, mv, p, grid, st) : launch_dense<64>(mk, mv, p, grid, st);
 }
@@ -329,7 +357,7 @@ size_t fold_workspace_bytes(const fold_args *args) {
   if (tmp.num_q_heads % tmp.num_kv_heads || tmp.batch % tmp.stack) return 0;
   const int G = tmp.num_q_heads / tmp.num_kv_heads;
   const long long R = (long long)tmp.stack * G;
-  if (R > kMaxRows || tmp.kv.max_seqlen < 0) return 0;
+  if (G > kMaxRows || R > kMaxStackedRows || tmp.kv.max_seqlen < 0) return 0;
   g.max_slots = max_chunks_upto(tmp.kv.max_seqlen);
   if (g.max_slots < 1) g.max_slots = 1;
   g.slot_stride = R * tmp.head_dim + ((R + 3) / 4) * 4;

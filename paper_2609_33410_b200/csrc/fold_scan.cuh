@@ -28,13 +28,6 @@
 
 namespace fold {
 
-#ifndef FOLD_QK_CHAINS_DENSE
-#define FOLD_QK_CHAINS_DENSE 1
-#endif
-#ifndef FOLD_QK_CHAINS_GATED
-#define FOLD_QK_CHAINS_GATED 1
-#endif
-
 struct ScanParams {
   const __nv_bfloat16 *q;
   long long q_stride_b, q_stride_h;
@@ -179,11 +172,12 @@ struct RowBlock {
   bool rv_lo, rv_hi, two_blocks;
 };
 template <int D>
-__device__ __forceinline__ void load_rows(RowBlock<D> &rb, const ScanParams &p, int seq, int kvh, int lane) {
-  const int row_lo = lane >> 2, row_hi = row_lo + 8, qcol = (lane & 3) * 2;
+__device__ __forceinline__ void load_rows(RowBlock<D> &rb, const ScanParams &p, int seq, int kvh, int lane,
+                                          int row0 = 0) {
+  const int row_lo = row0 + (lane >> 2), row_hi = row_lo + 8, qcol = (lane & 3) * 2;
   rb.rv_lo = row_lo < p.R;
   rb.rv_hi = row_hi < p.R;
-  rb.two_blocks = p.R > 8;
+  rb.two_blocks = p.R > row0 + 8;
   const int req_lo = seq * p.stack + row_lo / p.G, head_lo = kvh * p.G + row_lo % p.G;
   const int req_hi = seq * p.stack + row_hi / p.G, head_hi = kvh * p.G + row_hi % p.G;
   const __nv_bfloat16 *ql = p.q + (long long)req_lo * p.q_stride_b + (long long)head_lo * p.q_stride_h;
@@ -387,7 +381,7 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       const uint32_t kt = base + my_stage * LO::kStage;
       const int key0 = t * kTileKeys + warp * 16;
       uint32_t ah[4], al[4];
-      const uint32_t fetch16 = score_slice<D, false, FOLD_QK_CHAINS_DENSE>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+      const uint32_t fetch16 = score_slice<D, false, 1>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
       st_total += min(16, max(0, n - key0));
       if (key0 + 16 > n) {                                   // ragged tail: value rows past n may hold anything
         for (int r = 0; r < 16; ++r)
@@ -410,6 +404,118 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     if (dead) atomicOr(&p.hdr->wait_timeouts, 2u);
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_total);
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Stacked rows (more than 16 query rows per (sequence, kv head): the shared-prefix level of a
+// cascade, Section 4 "Value product" / Appendix "Tile layouts").  K and V tiles arrive together by
+// TMA as in dense decode -- with this many rows every key is live for some row, so nothing can be
+// skipped -- and each of the four consumer warps owns a 16-row block and walks all four slices of
+// every tile.  A CTA covers 64 rows; CTAs of the same tile stream share it through L2.  The depth
+// gate still applies row by row.  Each warp writes its own rows of the chunk slot: no cross-warp add.
+template <int D, bool GATED>
+__global__ void __launch_bounds__(kDenseThreads, 2)
+fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                         const ScanParams p) {
+  using LO = DenseLayout<D>;
+  constexpr int C16 = D / 8;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row_groups = (p.R + 63) / 64;
+  const int rg = blockIdx.x % row_groups, split = blockIdx.x / row_groups;
+  const int kvh = blockIdx.y, seq = blockIdx.z;
+  const SeqWork w = seq_work(p, seq);
+  if (split >= w.n_chunks) return;
+  const int stages = p.stages, R = p.R, n = w.n;
+  const uint32_t full0 = base + LO::off_bar(stages, 0), empty0 = full0 + 8u * stages;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, kConsumerWarps);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();
+
+  if (warp == kConsumerWarps) {
+    if (lane == 0) produce_tiles<D, true, LO::kStage>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
+    return;
+  }
+
+  const int row0 = rg * 64 + warp * 16;
+  RowBlock<D> rb;
+  load_rows<D>(rb, p, seq, kvh, lane, row0);
+  float o[D / 8][4];
+#pragma unroll
+  for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float l_lo = 0.f, l_hi = 0.f;
+  bool dead = false;
+  int stage = 0;
+  uint32_t phase = 0;
+
+  for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
+    const int my_stage = stage;
+    const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
+    if (++stage == stages) { stage = 0; phase ^= 1u; }
+    if (ready) {
+      const uint32_t kt = base + my_stage * LO::kStage;
+      if (k.t * kTileKeys + kTileKeys > n) {                 // ragged tail: value rows past n may hold anything
+        // every warp reads every row: warp w clears the rows of slice w, then all four meet
+        for (int r = 0; r < 16; ++r)
+          if (k.t * kTileKeys + warp * 16 + r >= n && lane < C16)
+            *reinterpret_cast<uint4 *>(gen + my_stage * LO::kStage + LO::kKTile +
+                                       tile_off(warp * 16 + r, lane, kTileKeys)) = make_uint4(0, 0, 0, 0);
+        named_bar(1);
+      }
+#pragma unroll 1
+      for (int sl = 0; sl < 4; ++sl) {
+        const int key0 = k.t * kTileKeys + sl * 16;
+        if (key0 >= n) break;
+        uint32_t ah[4], al[4];
+        const uint32_t live16 = score_slice<D, GATED, 1>(rb, kt, sl, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        if (live16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, sl * 16, lane, ah, al);
+      }
+      if (k.t * kTileKeys + kTileKeys > n) fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);
+    }
+    const int c_done = k.c;
+    if (cursor_next(k, w, p.num_splits)) {
+      // this warp owns its rows of the slot outright
+      float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
+      const int r_lo = row0 + (lane >> 2), r_hi = r_lo + 8, qcol = (lane & 3) * 2;
+#pragma unroll
+      for (int nt = 0; nt < D / 8; ++nt) {
+        if (r_lo < R) *reinterpret_cast<float2 *>(slot + (long long)r_lo * D + nt * 8 + qcol) = make_float2(o[nt][0], o[nt][1]);
+        if (r_hi < R) *reinterpret_cast<float2 *>(slot + (long long)r_hi * D + nt * 8 + qcol) = make_float2(o[nt][2], o[nt][3]);
+        o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+      }
+      l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+      l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+      l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+      l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+      if ((lane & 3) == 0) {
+        if (r_lo < R) slot[(long long)R * D + r_lo] = l_lo;
+        if (r_hi < R) slot[(long long)R * D + r_hi] = l_hi;
+      }
+      l_lo = l_hi = 0.f;
+    }
+  }
+  if (lane == 0 && dead) atomicOr(&p.hdr->wait_timeouts, 2u);
+  if (threadIdx.x == 0 && rg == 0) {                          // every value row is read once per row group pass
+    unsigned long long keys = 0;
+    for (int c = split; c < w.n_chunks; c += p.num_splits)
+      keys += min((c + 1) * w.ctiles * kTileKeys, n) - c * w.ctiles * kTileKeys;
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), keys);
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), keys);
   }
 }
 
@@ -503,7 +609,7 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       uint32_t ah[4] = {0u, 0u, 0u, 0u}, al[4] = {0u, 0u, 0u, 0u};
       uint32_t fetch16 = 0;
       if (ready) {
-        fetch16 = score_slice<D, true, FOLD_QK_CHAINS_GATED>(rb, base + my_stage * LO::kKTile, sl, lane, key0, n,
+        fetch16 = score_slice<D, true, 1>(rb, base + my_stage * LO::kKTile, sl, lane, key0, n,
                                                             p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);   // the K tile is in registers: release it

@@ -42,6 +42,20 @@ def test_group_and_stack_shapes(Hq, Hkv, stack):
     compare(w, run_gpu(w, T=12.0), T=12.0)
 
 
+@pytest.mark.parametrize("Hq,Hkv,stack,D", [(8, 2, 5, 128), (8, 2, 16, 128), (8, 2, 20, 128), (4, 4, 33, 64),
+                                            (8, 2, 64, 128)])
+def test_stacked_rows_beyond_one_row_block(Hq, Hkv, stack, D):
+    # 20 .. 256 query rows per (sequence, kv head): the stacked-row kernel, with ragged 16- and 64-row groups
+    w = make_decode_workload(2 * stack, Hq, Hkv, D, [1500, 333], seed=9, device=DEV, stack=stack,
+                             poison_padding=True, capacity=1600)
+    rows = [(b, h) for b in (0, 1, stack - 1, stack, 2 * stack - 1) for h in (0, Hq - 1)]
+    compare(w, run_gpu(w), rows=rows, check_estimate=True)
+    compare(w, run_gpu(w, T=12.0), T=12.0, rows=rows)
+    p = make_decode_workload(stack, Hq, Hkv, D, [9000], seed=10, device=DEV, stack=stack, paged=True, page_size=32)
+    rows = [(b, h) for b in (0, stack // 2, stack - 1) for h in (1, Hq - 2)]
+    compare(p, run_gpu(p, T=16.0), T=16.0, rows=rows)
+
+
 @pytest.mark.parametrize("page_size", [16, 32, 64, 128])
 @pytest.mark.parametrize("D", [64, 128])
 def test_paged_layout_and_poisoned_tails(page_size, D):
@@ -163,7 +177,6 @@ def test_rejects_bad_arguments_with_status_codes():
     assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
     a = status(); a.q = a.q + 2
     assert F.lib().fold_decode(a, None) == F.FOLD_EINVAL
-    a = status(stack=1); a.stack = 16          # 16 * G = 32 rows: beyond one row block
-    a.batch = 16; a.kv.num_seqs = 1
+    a = status(); a.num_q_heads = 64; a.num_kv_heads = 2      # a group of 32 rows is wider than one row block
     assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
     torch.cuda.synchronize()
