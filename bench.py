@@ -33,6 +33,8 @@ WORKLOADS = {
                         page_size=64), T=16.0),
     "c1": dict(gen=dict(batch=1, num_q_heads=8, num_kv_heads=8, head_dim=128, seqlens=4096, seed=0, peak_frac=0.0),
                T=16.0),
+    "c4": dict(cascade=dict(batch=64, num_q_heads=32, num_kv_heads=8, head_dim=128, prefix_len=16384, suffix_lens=2048,
+                            seed=3), T=16.0),
     "c3_small": dict(gen=dict(batch=1, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=131072, seed=2, paged=True,
                               page_size=64), T=16.0),
     "c2_small": dict(gen=dict(batch=4, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=16384, seed=1), T=16.0),
@@ -125,11 +127,18 @@ def oracle_sample(w, T, units, z=None):
 
 
 def bounded_oracle(w, T, budget_s=12.0):
+    """Run the oracle unit by unit (cycling over the sample's units) until about budget_s seconds of
+    oracle time have been spent."""
     units_all = [(s, h) for s in range(w.num_seqs) for h in range(w.num_kv_heads)]
-    t1, b1, threads = oracle_sample(w, T, units_all[:1])
-    k = int(max(1, min(len(units_all) - 1, budget_s / max(t1, 1e-3))))
-    t, b, threads = oracle_sample(w, T, units_all[1:1 + k]) if k >= 1 and len(units_all) > 1 else (t1, b1, threads)
-    return dict(seconds=t, bytes=b, units=k, threads=threads)
+    oracle_sample(w, T, units_all[:1])                     # warm the BLAS threads, untimed
+    seconds = 0.0
+    nbytes = 0
+    done = 0
+    threads = 1
+    while seconds < budget_s and done < 4096:
+        t, b, threads = oracle_sample(w, T, [units_all[done % len(units_all)]])
+        seconds += t; nbytes += b; done += 1
+    return dict(seconds=seconds, bytes=nbytes, units=done, threads=threads)
 
 
 def run_reference(args, rank, world):
@@ -138,6 +147,9 @@ def run_reference(args, rank, world):
         return
     from paper_2609_33410_b200.workloads import make_decode_workload
     spec = WORKLOADS[args.workload]
+    if "gen" not in spec:
+        print(json.dumps({"impl": "reference", "unavailable": "the reference arm times flat decode workloads only"}))
+        return
     gen = dict(spec["gen"])
     gen["batch"] = min(gen["batch"], 2)                 # the sample never needs more than two requests
     w = make_decode_workload(device="cpu", **gen)
@@ -207,34 +219,54 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     spec = WORKLOADS[args.workload]
-    gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
-    w = make_decode_workload(device=dev, **gen)
     T = spec["T"]
-    cache = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table)
-    bufs = F.alloc_buffers(w.q, cache)
-    cache_bytes = w.cache_bytes()
     stream = torch.cuda.current_stream()
+    cascade = "cascade" in spec
+    if cascade:
+        from paper_2609_33410_b200.workloads import make_cascade_workload
+        gen = dict(spec["cascade"]); gen["seed"] = gen["seed"] + 1000 * rank
+        levels = list(make_cascade_workload(device=dev, **gen))           # prefix level (stacked), suffix level
+    else:
+        gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
+        levels = [make_decode_workload(device=dev, **gen)]
+    w = levels[-1]                                                        # the level that owns out / lse / z
+    caches = [F.KVCache(l.k, l.v, l.seqlens, l.max_seqlen, l.page_table) for l in levels]
+    lbufs = [F.alloc_buffers(l.q, c, l.stack) for l, c in zip(levels, caches)]
+    bufs = lbufs[-1]
+    cache_bytes = sum(l.cache_bytes() for l in levels)                    # unique bytes: a shared prefix counts once
+    flat_bytes = sum(l.cache_bytes() * l.stack for l in levels)           # what a flat decode of every request reads
 
     def make(depth, z_mode):
-        return F.make_args(w.q, cache, scale=w.scale, z_mode=z_mode, z=bufs.z, depth_T=depth,
-                           num_splits=args.num_splits, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse,
-                           row_status=bufs.row_status)
+        return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
+                            num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
+                            row_status=bufs.row_status) for l, c, b in zip(levels, caches, lbufs)]
+
+    def step_whole(a):
+        if cascade:
+            F.fold_decode_cascade(a, stream)
+        else:
+            F.fold_decode(a[0], stream)
 
     def step_split(a, evs):
-        # the three launches of fold_decode issued one by one, so each kernel can be timed on its own
+        # the same launches issued one by one, so each kernel can be timed on its own
         evs[0].record(stream)
-        F.fold_estimate_z([a], stream)
+        F.fold_estimate_z(a, stream)
         evs[1].record(stream)
-        part = F.fold_decode_split(a, stream)
+        parts = [F.fold_decode_split(x, stream) for x in a]
         evs[2].record(stream)
-        F.fold_cascade_merge([part], bufs.out, bufs.lse, bufs.row_status, stream)
+        F.fold_cascade_merge(parts, bufs.out, bufs.lse, bufs.row_status, stream)
         evs[3].record(stream)
 
+    def headers():
+        hs = [b.header() for b in lbufs]
+        return dict(fetched=[h.v_rows_fetched for h in hs], total=[h.v_rows_total for h in hs],
+                    timeouts=sum(h.wait_timeouts for h in hs))
+
     def timed(depth, steps, warmup, sample_clocks):
-        # (1) whole steps through fold_decode: estimate -> scan -> partial add, chained in the stream
+        # (1) whole steps: estimate -> scan(s) -> partial add, chained in the stream by one C-ABI call
         a = make(depth, F.Z_ESTIMATE)
         for _ in range(warmup):
-            F.fold_decode(a, stream)
+            step_whole(a)
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
@@ -244,14 +276,14 @@ def main():
         t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
         t0.record(stream)
         for i in range(steps):
-            F.fold_decode(a, stream)
+            step_whole(a)
         t1.record(stream)
         torch.cuda.synchronize()
         if ctx: ctx.__exit__()
         if world > 1:
             torch.distributed.barrier()
         total_ms = t0.elapsed_time(t1)
-        hdr = bufs.header()
+        hd = headers()
         # (2) the same launches with events between them, for the per-kernel durations
         g = make(depth, F.Z_GIVEN)
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
@@ -263,8 +295,7 @@ def main():
         mrg_ms = [e[2].elapsed_time(e[3]) for e in evs]
         return dict(ms_per_step=max_over_ranks(total_ms / steps, world, dev), scan_ms=statistics.mean(scan_ms),
                     scan_ms_min=min(scan_ms), est_ms=statistics.mean(est_ms), merge_ms=statistics.mean(mrg_ms),
-                    fetched=hdr.v_rows_fetched, total=hdr.v_rows_total, timeouts=hdr.wait_timeouts,
-                    clocks=sampler.summary() if sample_clocks else None)
+                    clocks=sampler.summary() if sample_clocks else None, **hd)
 
     warm = max(args.warmup, 3)
     r16 = timed(T, args.steps, warm, True)
@@ -273,40 +304,47 @@ def main():
         raise SystemExit("a bounded wait timed out inside the scan kernel: results invalid")
 
     D = w.head_dim
-    slot_bytes = F.fold_workspace_bytes(make(T, F.Z_GIVEN)) - 256
+    slot_bytes = sum(F.fold_workspace_bytes(x) - 256 for x in make(T, F.Z_GIVEN))
 
-    def actual_bytes(r):                                  # K in full + fetched V rows + slots written
-        return r["total"] * 2 * D + r["fetched"] * 2 * D + slot_bytes
+    def actual_bytes(r):                                  # K in full + fetched V rows + slots written, all levels
+        return sum(r["total"]) * 2 * D + sum(r["fetched"]) * 2 * D + slot_bytes
+
+    def fetched_frac(r):
+        return sum(r["fetched"]) / max(sum(r["total"]), 1)
 
     peak, peak_src = load_peaks()
     value = world * cache_bytes / (r16["ms_per_step"] * 1e-3) / 1e9
     ach16 = actual_bytes(r16) / (r16["scan_ms"] * 1e-3) / 1e9
     achinf = actual_bytes(rinf) / (rinf["scan_ms"] * 1e-3) / 1e9
+    scan_name = ("fold_scan_stacked_kernel + fold_scan_gated_kernel (prefix + suffix levels)" if cascade
+                 else "fold_scan_gated_kernel")
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
         "ms_per_step": r16["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 in, fp32 accumulate", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: " + json.dumps(spec["gen"], sort_keys=True), "depth_T": T,
+        "config": {"workload": f"{args.workload}: " + json.dumps(spec.get("gen", spec.get("cascade")), sort_keys=True),
+                   "depth_T": T,
                    "num_splits": args.num_splits or "auto", "l2": "inputs (cache) larger than L2, no flush needed"
                    if cache_bytes > 4 * 126e6 else "cache smaller than 4x L2: partly L2-resident",
-                   "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes},
+                   "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
+                   "flat_equivalent_bytes_per_gpu": flat_bytes},
         "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
         "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},
         "kernel_ms": {"estimate": r16["est_ms"], "scan_T16": r16["scan_ms"], "scan_Tinf": rinf["scan_ms"],
                       "merge": r16["merge_ms"]},
-        "v_rows_fetched_frac": {"T16": r16["fetched"] / max(r16["total"], 1), "Tinf": rinf["fetched"] / max(rinf["total"], 1)},
-        "roofline": {"bound": "hbm", "kernel": "fold_scan_kernel (T=16, gather path)", "achieved": ach16, "peak": peak,
+        "v_rows_fetched_frac": {"T16": fetched_frac(r16), "Tinf": fetched_frac(rinf)},
+        "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
                      "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src, "traffic": None,
                      "algorithmic_bytes_per_launch": actual_bytes(r16),
-                     "dense": {"kernel": "fold_scan_kernel (T=inf, TMA path)", "achieved": achinf, "frac": achinf / peak,
+                     "dense": {"kernel": "fold_scan_dense_kernel (T=inf)" if not cascade else "stacked + dense kernels (T=inf)", "achieved": achinf, "frac": achinf / peak,
                                "frac_of_nominal_8TBs": achinf / 8000.0,
                                "algorithmic_bytes_per_launch": actual_bytes(rinf)}},
         "gpu_launches": 3 * args.steps,   # estimate + scan + partial add per timed step (the extra per-kernel pass is not timed)
         "clocks": r16["clocks"],
     }
 
-    if rank == 0 and not args.no_e2e:
+    if rank == 0 and not args.no_e2e and not cascade:
         # end to end through the C ABI with HOST buffers: every step copies q and the whole cache
         # host -> device, decodes, and copies out / lse / status back
         hq, hk, hv = w.q.cpu().pin_memory(), w.k.cpu().pin_memory(), w.v.cpu().pin_memory()
@@ -335,7 +373,7 @@ def main():
                       "note": "fold_decode_host: whole cache copied from pinned host memory every step"}
         del staging, hk, hv
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not cascade:
         wc = make_decode_workload(device="cpu", **dict(spec["gen"], batch=min(spec["gen"]["batch"], 2)))
         ob = bounded_oracle(wc, T)
         out["cpu_baseline"] = {"value": ob["bytes"] / ob["seconds"] / 1e9, "unit": UNIT, "cores": ob["threads"],

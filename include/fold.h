@@ -174,6 +174,15 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
  * fold_decode_split followed by fold_cascade_merge over its one level. */
 int fold_decode(const fold_args *args, fold_stream stream);
 
+/* Shared-prefix cascade in one call (Section 4, "Value product"; Appendix "Cascades and drafts"):
+ * one reference estimate over each request's concatenated levels, one scan per level under
+ * that reference, one order-free add over all levels' partials.  levels[l] (HOST array of HOST
+ * pointers, n_levels in 1..4) describe the same requests: the same q, z, batch, head counts,
+ * head_dim, softmax_scale and depth_T; each level has its own kv, stack and workspace.
+ * levels[0]->z_mode is FOLD_Z_ESTIMATE (estimate over all levels, written to z) or FOLD_Z_GIVEN;
+ * out, lse and row_status are taken from levels[0]. */
+int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_stream stream);
+
 /* The same decode for callers whose tensors live in HOST memory (pinned for the copies to
  * be asynchronous): q, kv.k, kv.v, kv.page_table, kv.seqlens, z (if GIVEN), out, lse and
  * row_status of *host_args are HOST pointers laid out as described above (the cache is

@@ -56,7 +56,7 @@ class FoldWsHeader(C.Structure):
 
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
-           "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_host_staging_bytes",
+           "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
            "fold_decode_host", "fold_status_string", "fold_version"]
 
 _lib = None
@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
         L.fold_cascade_merge.argtypes = [C.POINTER(C.POINTER(FoldPartials)), C.c_int, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p]
         L.fold_decode.restype = C.c_int; L.fold_decode.argtypes = [C.POINTER(FoldArgs), C.c_void_p]
+        L.fold_decode_cascade.restype = C.c_int
+        L.fold_decode_cascade.argtypes = [C.POINTER(C.POINTER(FoldArgs)), C.c_int, C.c_void_p]
         L.fold_host_staging_bytes.restype = C.c_size_t; L.fold_host_staging_bytes.argtypes = [C.POINTER(FoldArgs)]
         L.fold_decode_host.restype = C.c_int
         L.fold_decode_host.argtypes = [C.POINTER(FoldArgs), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -203,6 +205,11 @@ def fold_cascade_merge(levels: Sequence[FoldPartials], out: torch.Tensor, lse: O
 
 def fold_decode(args: FoldArgs, stream=None) -> None:
     _check(lib().fold_decode(C.byref(args), _stream(stream)), "fold_decode")
+
+
+def fold_decode_cascade(levels: Sequence[FoldArgs], stream=None) -> None:
+    arr = (C.POINTER(FoldArgs) * len(levels))(*[C.pointer(a) for a in levels])
+    _check(lib().fold_decode_cascade(arr, len(levels), _stream(stream)), "fold_decode_cascade")
 
 
 def fold_host_staging_bytes(args: FoldArgs) -> int:

@@ -453,6 +453,33 @@ int fold_decode(const fold_args *args, fold_stream stream) {
   return fold_cascade_merge(lv, 1, args->out, args->lse, args->row_status, stream);
 }
 
+int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_stream stream) {
+  if (!levels || n_levels < 1 || n_levels > kMaxLevels || !levels[0]) return FOLD_EINVAL;
+  const fold_args *a0 = levels[0];
+  if (a0->z_mode != FOLD_Z_ESTIMATE && a0->z_mode != FOLD_Z_GIVEN) return FOLD_EINVAL;
+  fold_args lv[kMaxLevels];
+  for (int l = 0; l < n_levels; ++l) {
+    const fold_args *a = levels[l];
+    if (!a || a->q != a0->q || a->z != a0->z || a->batch != a0->batch || a->num_q_heads != a0->num_q_heads ||
+        a->num_kv_heads != a0->num_kv_heads || a->head_dim != a0->head_dim || a->depth_T != a0->depth_T ||
+        a->softmax_scale != a0->softmax_scale)
+      return FOLD_EINVAL;
+    Geometry g;
+    lv[l] = *a;
+    lv[l].z_mode = FOLD_Z_GIVEN;
+    if (int rc = check_args(&lv[l], &g, l == 0)) return rc;
+  }
+  if (a0->z_mode == FOLD_Z_ESTIMATE)
+    if (int rc = fold_estimate_z(levels, n_levels, stream)) return rc;
+  fold_partials parts[kMaxLevels];
+  const fold_partials *pp[kMaxLevels];
+  for (int l = 0; l < n_levels; ++l) {
+    if (int rc = fold_decode_split(&lv[l], &parts[l], stream)) return rc;
+    pp[l] = &parts[l];
+  }
+  return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
+}
+
 // ------------------------------------------------------------------ host-buffer variant
 namespace {
 struct HostPlan {

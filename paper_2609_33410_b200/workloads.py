@@ -153,6 +153,21 @@ def make_decode_workload(batch: int, num_q_heads: int, num_kv_heads: int, head_d
     return DecodeWorkload(q, kc, vc, seqlens_t, max_len, Hq, Hkv, D, stack, None, 0, 1.0 / D ** 0.5, meta)
 
 
+def make_cascade_workload(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, prefix_len: int,
+                          suffix_lens: Union[int, Sequence[int]], seed: int = 0, device="cpu", **kw):
+    """Requests that share one prefix and own private suffixes.  Returns (prefix level, suffix level):
+    two workloads over the same queries; the prefix level stacks all requests on one KV sequence."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(int(seed))
+    q = torch.randn(batch, num_q_heads, head_dim, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    pre = make_decode_workload(batch, num_q_heads, num_kv_heads, head_dim, prefix_len, seed=seed + 1, device=dev,
+                               stack=batch, q=q, **kw)
+    suf = make_decode_workload(batch, num_q_heads, num_kv_heads, head_dim, suffix_lens, seed=seed + 2, device=dev,
+                               q=q, sink_gain=1.0, **kw)
+    return pre, suf
+
+
 # The five benchmark configurations, by name.  `scale_down` shrinks context (and for the
 # sweep the batch) so the CPU oracle can check every row in seconds.
 def config_workload(name: str, device="cpu", small: bool = False, **over) -> DecodeWorkload:

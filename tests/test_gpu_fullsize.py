@@ -1,0 +1,83 @@
+"""The benchmark configurations at full size, in the launch configuration bench.py times
+(split hint 0 = the library's choice), checked against the oracle on sampled rows the
+oracle can compute one by one."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_33410_b200 as F
+from oracle import fold_oracle as O
+from paper_2609_33410_b200.workloads import make_decode_workload, make_cascade_workload, DecodeWorkload, bf16_bits
+from helpers import run_gpu, compare, cache_of, same_bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _free_gb():
+    free, _ = torch.cuda.mem_get_info()
+    return free / 2 ** 30
+
+
+def test_config2_gqa_batch16_32k_sampled_rows():
+    if _free_gb() < 12:
+        pytest.skip("not enough free device memory")
+    w = make_decode_workload(16, 32, 8, 128, 32768, seed=1, device=DEV)
+    rows = [(0, 0), (3, 13), (7, 31), (15, 18)]
+    b = run_gpu(w, T=16.0)
+    r = compare(w, b, T=16.0, rows=rows, check_estimate=True)
+    ref = b.out.clone()
+    assert same_bits(run_gpu(w, T=16.0, num_splits=8).out, ref)          # the configuration's 8-way split: same bits
+    compare(w, run_gpu(w), rows=rows)
+    del w
+    torch.cuda.empty_cache()
+
+
+def test_config3_paged_128k_sampled_rows():
+    if _free_gb() < 12:
+        pytest.skip("not enough free device memory")
+    w = make_decode_workload(4, 32, 8, 128, 131072, seed=2, device=DEV, paged=True, page_size=64)
+    rows = [(0, 5), (1, 30), (3, 0)]
+    b = run_gpu(w, T=16.0)
+    compare(w, b, T=16.0, rows=rows, check_estimate=True)
+    assert same_bits(run_gpu(w, T=16.0, num_splits=32).out, b.out.clone())
+    compare(w, run_gpu(w), rows=rows)
+    hdr = b.header()
+    del w
+    torch.cuda.empty_cache()
+
+
+def test_config4_shared_prefix_cascade_sampled_rows():
+    if _free_gb() < 8:
+        pytest.skip("not enough free device memory")
+    B, Hq, Hkv, D, P, S = 64, 32, 8, 128, 16384, 2048
+    pre, suf = make_cascade_workload(B, Hq, Hkv, D, P, S, seed=3, device=DEV)
+    cp, cs = cache_of(pre), cache_of(suf)
+    bp, bs = F.alloc_buffers(pre.q, cp, stack=B), F.alloc_buffers(pre.q, cs)
+    ap = F.make_args(pre.q, cp, z=bs.z, depth_T=16.0, stack=B, workspace=bp.workspace, out=bs.out, lse=bs.lse,
+                     row_status=bs.row_status)
+    as_ = F.make_args(pre.q, cs, z=bs.z, depth_T=16.0, workspace=bs.workspace, out=bs.out, lse=bs.lse,
+                      row_status=bs.row_status)
+    F.fold_decode_cascade([ap, as_])
+    torch.cuda.synchronize()
+    assert bp.header().wait_timeouts == 0 and bs.header().wait_timeouts == 0
+    out = bs.out.float().cpu().numpy().astype(np.float64)
+    z = bs.z.cpu().numpy().astype(np.float64)
+    num = den = ynum = 0.0
+    for (b, h) in [(0, 0), (17, 9), (63, 31)]:
+        kvh = h // 4
+        K = np.concatenate([O.widen_bf16(bf16_bits(pre.logical_rows("k", 0, kvh))),
+                            O.widen_bf16(bf16_bits(suf.logical_rows("k", b, kvh)))])
+        V = np.concatenate([O.widen_bf16(bf16_bits(pre.logical_rows("v", 0, kvh))),
+                            O.widen_bf16(bf16_bits(suf.logical_rows("v", b, kvh)))])
+        q = O.widen_bf16(bf16_bits(pre.q[b, h]))
+        s = O.scores(q, K)
+        assert abs(O.estimate_z(lambda i: s[i], len(s)) - z[b, h]) < 1e-3
+        ref, _, _, _ = O.fold_row(s, V, z[b, h], 16.0)
+        d = out[b, h] - ref
+        num += d @ d; den += ref @ ref
+        y = O.online_softmax_bf16(q, K, V) - O.dense_row(s, V)[0]
+        ynum += y @ y
+    assert math.sqrt(num / den) <= 1.5 * math.sqrt(ynum / den) + 1e-4
