@@ -41,6 +41,13 @@ WORKLOADS = {
 }
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one scan launch from the ncu captures
+# summarised in profiles/fold_scan_kernels_c2_small.md, per byte of cache the launch covers: the c2_small
+# capture (268.4 MB of K+V) moved 274.2 MB (gated, T=16) and 273.0 MB (dense).  Traffic grows in
+# proportion to the (sequence, kv head, key) units, so a launch is scaled by its cache bytes.
+NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 274.2 / 268.4, "dense": 273.0 / 268.4}
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -335,7 +342,9 @@ def main():
                       "merge": r16["merge_ms"]},
         "v_rows_fetched_frac": {"T16": fetched_frac(r16), "Tinf": fetched_frac(rinf)},
         "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
-                     "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src, "traffic": None,
+                     "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src,
+                     "traffic": None if cascade or args.workload != "c2" else NCU_TRAFFIC_PER_CACHE_BYTE["gated"] * cache_bytes,
+                     "traffic_source": "ncu capture on c2_small scaled by units (profiles/fold_scan_kernels_c2_small.md)",
                      "algorithmic_bytes_per_launch": actual_bytes(r16),
                      "dense": {"kernel": "fold_scan_dense_kernel (T=inf)" if not cascade else "stacked + dense kernels (T=inf)", "achieved": achinf, "frac": achinf / peak,
                                "frac_of_nominal_8TBs": achinf / 8000.0,
