@@ -40,7 +40,8 @@ typedef enum fold_status {
   FOLD_EINVAL = 1,        /* null / misaligned pointer, inconsistent sizes, T < 0 or NaN */
   FOLD_EUNSUPPORTED = 2,  /* head_dim not in {64,128}, page_size not a power of two >= 16, ... */
   FOLD_EWORKSPACE = 3,    /* workspace_bytes < fold_workspace_bytes(args) */
-  FOLD_ECUDA = 4          /* a CUDA runtime / driver call failed (launch error, no sm_100 device) */
+  FOLD_ECUDA = 4,         /* a CUDA runtime / driver call failed (launch error, no sm_100 device) */
+  FOLD_ETOOLARGE = 5      /* fold_decode_static only: the call needs more scratch than the built-in array holds */
 } fold_status;
 
 /* How the per-row reference Z_i (Section 3, "Choosing the reference") is obtained. */
@@ -192,6 +193,37 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
  * `stream`; the host buffers are valid after the caller synchronises the stream. */
 size_t fold_host_staging_bytes(const fold_args *host_args);
 int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_bytes, fold_stream stream);
+
+/* Decode without a caller workspace.  (The paper has no counterpart: this entry point exists for
+ * integration, not for the method.)
+ *
+ * Who needs it: callers that cannot hand the library device memory at call time because they are
+ * not allowed to allocate any -- a plugin inside a host program that owns the whole device heap and
+ * forbids cudaMalloc, a decode loop that must never reach the allocator because cudaMalloc /
+ * cudaFree synchronise the device and stall every stream, or code that is only given its input and
+ * output tensors and has nowhere to keep a buffer between calls.
+ *
+ * What it does: exactly fold_decode(args, stream), except that args->workspace and
+ * args->workspace_bytes are ignored and the scratch the scan and the partial add need (the
+ * fold_ws_header and the (A, L) slots) lives in an array built into the library:
+ * FOLD_STATIC_SCRATCH_BYTES bytes of device memory, 256-byte aligned, that every GPU which loads
+ * the library holds from load to exit.  The call allocates and frees nothing, on the host side of
+ * the CUDA API or through any other library.
+ *
+ * Limits and rules:
+ *  - A call whose fold_workspace_bytes(args) exceeds FOLD_STATIC_SCRATCH_BYTES is refused with
+ *    FOLD_ETOOLARGE before anything is enqueued (the default benchmark shape -- 16 requests x 8 kv
+ *    heads x 32768 keys, group 4, head_dim 128 -- needs 8.1 MiB).
+ *  - The first call on each device looks up the array's device address (with that device current);
+ *    make that first call outside any stream capture.  Later calls on the device reuse the address.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left.  The
+ *    library re-zeroes the part that must start at zero (the header) at the start of every call and
+ *    never reads a slot the same call has not written, so stale contents are harmless -- but two
+ *    calls that can overlap on the GPU (different streams, or a call racing a graph replay that
+ *    contains one) would write the same slots: order them yourself.
+ *  - The partials are not exposed: there is no split / cascade form of this entry point. */
+#define FOLD_STATIC_SCRATCH_BYTES (16u << 20)
+int fold_decode_static(const fold_args *args, fold_stream stream);
 
 const char *fold_status_string(int status);
 /* Library version as major*10000 + minor*100 + patch. */

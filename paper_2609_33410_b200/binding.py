@@ -17,7 +17,8 @@ import torch
 from . import build as _build
 
 # ------------------------------------------------------------------ C structs (mirror include/fold.h)
-FOLD_OK, FOLD_EINVAL, FOLD_EUNSUPPORTED, FOLD_EWORKSPACE, FOLD_ECUDA = range(5)
+FOLD_OK, FOLD_EINVAL, FOLD_EUNSUPPORTED, FOLD_EWORKSPACE, FOLD_ECUDA, FOLD_ETOOLARGE = range(6)
+STATIC_SCRATCH_BYTES = 16 << 20
 Z_ESTIMATE, Z_GIVEN, Z_EXACT_MAX, Z_ZERO = range(4)
 ROW_RANGE, ROW_NONFINITE, ROW_EMPTY = 1, 2, 4
 
@@ -57,7 +58,7 @@ class FoldWsHeader(C.Structure):
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
            "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
-           "fold_decode_host", "fold_status_string", "fold_version"]
+           "fold_decode_host", "fold_decode_static", "fold_status_string", "fold_version"]
 
 _lib = None
 
@@ -84,6 +85,7 @@ def lib() -> C.CDLL:
         L.fold_host_staging_bytes.restype = C.c_size_t; L.fold_host_staging_bytes.argtypes = [C.POINTER(FoldArgs)]
         L.fold_decode_host.restype = C.c_int
         L.fold_decode_host.argtypes = [C.POINTER(FoldArgs), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.fold_decode_static.restype = C.c_int; L.fold_decode_static.argtypes = [C.POINTER(FoldArgs), C.c_void_p]
         L.fold_status_string.restype = C.c_char_p; L.fold_status_string.argtypes = [C.c_int]
         L.fold_version.restype = C.c_int
         _lib = L
@@ -219,6 +221,14 @@ def fold_host_staging_bytes(args: FoldArgs) -> int:
 def fold_decode_host(host_args: FoldArgs, staging: torch.Tensor, stream=None) -> None:
     _check(lib().fold_decode_host(C.byref(host_args), staging.data_ptr(), staging.numel() * staging.element_size(),
                                   _stream(stream)), "fold_decode_host")
+
+
+def fold_decode_static(args: FoldArgs, stream=None) -> None:
+    """fold_decode for callers that may not allocate device memory: the workspace fields of `args` are
+    ignored and the library's built-in scratch array (STATIC_SCRATCH_BYTES per device) is used instead.
+    Raises FoldError(FOLD_ETOOLARGE) when the call would need more.  Calls on one device share that array:
+    do not let two of them overlap on the GPU; make the first call on a device outside stream capture."""
+    _check(lib().fold_decode_static(C.byref(args), _stream(stream)), "fold_decode_static")
 
 
 # ------------------------------------------------------------------ small conveniences for tests and the benchmark

@@ -563,6 +563,43 @@ int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, f
   return ok ? FOLD_OK : FOLD_ECUDA;
 }
 
+// ------------------------------------------------------------------ decode without a caller workspace
+// Scratch for callers that may not allocate: the header and (A, L) slots of one decode call live in
+// this array, which every device that loads the library holds until exit.  In host code the name
+// below is only a handle for cudaGetSymbolAddress, never a device address: kernels are given the
+// address that call returns (looked up once per device, with that device current).
+static __device__ __align__(256) unsigned char g_fold_static_scratch[FOLD_STATIC_SCRATCH_BYTES];
+
+namespace {
+void *g_static_scratch_addr[64] = {nullptr};   // device address of the array, per device ordinal
+
+int static_scratch_address(void **out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FOLD_ECUDA;
+  if (dev < 0 || dev >= 64) return FOLD_EUNSUPPORTED;
+  if (!g_static_scratch_addr[dev]) {           // first call on this device: resolve the symbol here, once
+    void *addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_fold_static_scratch) != cudaSuccess || !addr) return FOLD_ECUDA;
+    g_static_scratch_addr[dev] = addr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return FOLD_OK;
+}
+}  // namespace
+
+int fold_decode_static(const fold_args *args, fold_stream stream) {
+  if (!args) return FOLD_EINVAL;
+  const size_t need = fold_workspace_bytes(args);
+  if (need == 0) return FOLD_EINVAL;
+  if (need > (size_t)FOLD_STATIC_SCRATCH_BYTES) return FOLD_ETOOLARGE;
+  void *scratch = nullptr;
+  if (int rc = static_scratch_address(&scratch)) return rc;
+  fold_args a = *args;
+  a.workspace = scratch;                       // the header is re-zeroed by the scan's own memset; slots are
+  a.workspace_bytes = FOLD_STATIC_SCRATCH_BYTES;   // written before they are read, so nothing else needs clearing
+  return fold_decode(&a, stream);
+}
+
 const char *fold_status_string(int status) {
   switch (status) {
     case FOLD_OK: return "ok";
@@ -570,6 +607,7 @@ const char *fold_status_string(int status) {
     case FOLD_EUNSUPPORTED: return "unsupported shape or layout";
     case FOLD_EWORKSPACE: return "workspace too small";
     case FOLD_ECUDA: return "CUDA call failed";
+    case FOLD_ETOOLARGE: return "call needs more scratch than the library's built-in array holds";
     default: return "unknown status";
   }
 }
