@@ -434,13 +434,15 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
   p.lse = lse; p.row_status = row_status;
   p.n_levels = n_levels; p.Hq = p0->num_q_heads; p.Hkv = p0->num_kv_heads;
   p.G = p0->num_q_heads / p0->num_kv_heads; p.D = p0->head_dim;
-  // slices per row: about 16 slots per thread, so short slot lists do not pay for idle threads
+  // warps per row: about 8 slots per warp, so short slot lists do not pay for idle warps
   int total_slots = 0;
   for (int l = 0; l < n_levels; ++l) total_slots += max_chunks_upto(levels[l]->max_seqlen);
-  int slices = (total_slots + 15) / 16;
-  slices = slices < 1 ? 1 : (slices > kMergeMaxSlices ? kMergeMaxSlices : slices);
-  const dim3 grid(p.Hq, p0->batch), block(p.D, slices);
-  if (launch_pdl(fold_merge_kernel, grid, block, 0, static_cast<cudaStream_t>(stream), p) != cudaSuccess) return FOLD_ECUDA;
+  int warps = (total_slots + 7) / 8;
+  warps = warps < 1 ? 1 : (warps > kMergeMaxWarps ? kMergeMaxWarps : warps);
+  const dim3 grid(p.Hq, p0->batch), block(32, warps);
+  cudaError_t rc = p.D == 128 ? launch_pdl(fold_merge_kernel<4>, grid, block, 0, static_cast<cudaStream_t>(stream), p)
+                              : launch_pdl(fold_merge_kernel<2>, grid, block, 0, static_cast<cudaStream_t>(stream), p);
+  if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 

@@ -133,55 +133,47 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
   }
   __syncthreads();
 
-  // row maxima (warp g), then every thread takes one (row, sample): its weight, and for a stratum
-  // centre its rank among the 128 centres (the 8 largest are dropped; ties broken by index)
-  __shared__ float rmax[kMaxRows];
-  __shared__ float wt[kMaxRows][kEstSamples];
-  for (int g = warp; g < G; g += kEstSampleThreads / 32) {
-    float m = -INFINITY;
-    for (int k = lane; k < n_samples; k += 32) m = fmaxf(m, sc[g][k]);
-#pragma unroll
-    for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
-    if (lane == 0) rmax[g] = m;
-  }
-  __syncthreads();
-  for (int e = threadIdx.x; e < G * kEstSamples; e += kEstSampleThreads) {
-    const int g = e / kEstSamples, k = e % kEstSamples;
-    float wv = 0.f;
-    if (k < n_samples) {
-      const float sk = sc[g][k];
-      bool keep = true;
-      if (n > kEstSamples && k > kEstRecent) {
-        int rank = 0;
-        const float4 *cv = reinterpret_cast<const float4 *>(&sc[g][1 + kEstRecent]);
-#pragma unroll 8
-        for (int j4 = 0; j4 < kEstStrata / 4; ++j4) {
-          const float4 t = cv[j4];
-          const int j = 1 + kEstRecent + 4 * j4;
-          rank += (t.x > sk || (t.x == sk && j < k)) ? 1 : 0;
-          rank += (t.y > sk || (t.y == sk && j + 1 < k)) ? 1 : 0;
-          rank += (t.z > sk || (t.z == sk && j + 2 < k)) ? 1 : 0;
-          rank += (t.w > sk || (t.w == sk && j + 3 < k)) ? 1 : 0;
-        }
-        keep = rank >= kEstTrim;
-      }
-      if (keep) wv = exp2f(sk - rmax[g]);
-    }
-    wt[g][k] = wv;
-  }
-  __syncthreads();
+  // warp g finishes row g: maximum, exact part, trimmed stratified part
   for (int g = warp; g < G; g += kEstSampleThreads / 32) {
     float zval = 0.f;
     if (n_samples > 0) {
-      float exact = 0.f, kept = 0.f;                 // fixed summation order: lane-strided, then a shuffle tree
-      const int n_exact = n <= kEstSamples ? n_samples : 1 + kEstRecent;
-      for (int k = lane; k < n_exact; k += 32) exact += wt[g][k];
-      if (n > kEstSamples)
-        for (int k = 1 + kEstRecent + lane; k < kEstSamples; k += 32) kept += wt[g][k];
-      float total = exact + kept * ((float)(n - 1 - kEstRecent) / (float)(kEstStrata - kEstTrim));
+      float m = -INFINITY;
+      for (int k = lane; k < n_samples; k += 32) m = fmaxf(m, sc[g][k]);
+#pragma unroll
+      for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+      float total = 0.f;                             // fixed summation order: lane-strided, then a shuffle tree
+      if (n <= kEstSamples) {
+        for (int k = lane; k < n_samples; k += 32) total += exp2f(sc[g][k] - m);
+      } else {
+        for (int k = lane; k <= kEstRecent; k += 32) total += exp2f(sc[g][k] - m);      // sink + 63 recent
+        // the 128 centre scores, four per lane (centre lane + 32 i); drop the 8 largest, one per round:
+        // the warp-wide maximum, owned by the lowest index among equals
+        float c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c[i] = sc[g][1 + kEstRecent + lane + 32 * i];
+#pragma unroll 1
+        for (int r = 0; r < kEstTrim; ++r) {
+          float wm = fmaxf(fmaxf(c[0], c[1]), fmaxf(c[2], c[3]));
+#pragma unroll
+          for (int k = 16; k > 0; k >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, k));
+          bool found = false;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const unsigned owners = __ballot_sync(0xffffffffu, c[i] == wm);
+            if (!found && owners) {
+              if (lane == __ffs(owners) - 1) c[i] = -INFINITY;
+              found = true;
+            }
+          }
+        }
+        float kept = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kept += exp2f(c[i] - m);                              // dropped ones add 2^-inf = 0
+        total += kept * ((float)(n - 1 - kEstRecent) / (float)(kEstStrata - kEstTrim));
+      }
 #pragma unroll
       for (int k = 16; k > 0; k >>= 1) total += __shfl_xor_sync(0xffffffffu, total, k);
-      zval = rmax[g] + log2f(total);
+      zval = m + log2f(total);
     }
     if (lane == 0) p.z[(long long)req * p.Hq + kvh * G + g] = zval;
   }

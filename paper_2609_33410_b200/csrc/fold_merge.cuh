@@ -4,15 +4,15 @@
 // summed on an integer grid declared before the reduction (Eq. 3 / Prop. 2): the largest
 // magnitude among the C terms is found with an order-free integer maximum over their bit
 // patterns, the grid is alpha = 2^(61 - ceil(log2 C) - e_max - 1) (e_max >= -126: subnormal maxima
-// use their fixed scale), every term is rounded to nearest-even on it with integer shifts of its
-// mantissa and added as a 64-bit integer.
+// use their fixed scale), every term is rounded to nearest-even on it (exactly: a power-of-two
+// product in double, then a round-to-nearest-even conversion) and added as a 64-bit integer.
 #pragma once
 
 #include "fold_common.cuh"
 
 namespace fold {
 
-constexpr int kMergeMaxSlices = 8;
+constexpr int kMergeMaxWarps = 8;
 
 struct MergeLevel {
   const float *slots;
@@ -32,59 +32,43 @@ struct MergeParams {
 
 __device__ __forceinline__ int ceil_log2_u32(unsigned c) { return c <= 1 ? 0 : 32 - __clz(c - 1); }
 
-// Biased exponent of a bit pattern with subnormals counted as exponent 1 (their scale).
-__device__ __forceinline__ int norm_exp(unsigned bits) {
-  const int e = (int)((bits >> 23) & 0xffu);
-  return e == 0 ? 1 : e;
+// log2(alpha) for C terms whose largest magnitude has bit pattern maxbits (sign cleared); subnormal
+// maxima use their fixed scale (e_max = -126).
+__device__ __forceinline__ int grid_shift(unsigned maxbits, int clog2C) {
+  const int ef = (int)(maxbits >> 23);
+  const int e_max = ef == 0 ? -126 : ef - 127;
+  return 61 - (clog2C + e_max + 1);
 }
-// RNE(alpha * g) as an exact integer, alpha = 2^(61 - clog2C - (eb_max - 127) - 1): with g = m * 2^(e - 150),
-// alpha * g = m * 2^(e - eb_max + 37 - clog2C).  Integer shifts only; |result| < 2^61 / C.
-__device__ __forceinline__ long long to_grid(float g, int eb_max, int clog2C) {
-  const unsigned u = __float_as_uint(g);
-  const int e = (int)((u >> 23) & 0xffu);
-  unsigned m = u & 0x7fffffu;
-  if (e != 0) m |= 0x800000u;
-  const int s = (e == 0 ? 1 : e) - eb_max + 37 - clog2C;
-  long long v;
-  if (s >= 0) {
-    v = (long long)m << s;
-  } else if (s < -25) {
-    v = 0;
-  } else {
-    const int r = -s;
-    unsigned q = m >> r;
-    const unsigned rem = m & ((1u << r) - 1u), half = 1u << (r - 1);
-    if (rem > half || (rem == half && (q & 1u))) ++q;
-    v = q;
-  }
-  return (u >> 31) ? -v : v;
+__device__ __forceinline__ double pow2_double(int e) {       // 2^e, e in the normal range
+  return __longlong_as_double((long long)(e + 1023) << 52);
 }
-__device__ __forceinline__ float from_grid(long long sum, int eb_max, int clog2C) {
-  // alpha^-1 = 2^-(187 - clog2C - eb_max); exponent stays inside the double range
-  const int sh = 187 - clog2C - eb_max;
-  return (float)((double)sum * __longlong_as_double((long long)(1023 - sh) << 52));
-}
+// RNE(alpha * g) as an integer: the product with a power of two is exact in double, the conversion rounds to
+// nearest even; |result| < 2^61 / C.
+__device__ __forceinline__ long long to_grid(float g, double alpha) { return __double2ll_rn((double)g * alpha); }
 
-// grid (Hq, batch); block (D, S), S = blockDim.y <= kMergeMaxSlices chosen from the slot count.
-// Thread (x, y): element x of A over the slots y, y + S, ... of every level; the x == 0 threads
-// also carry L.  Two passes over the (cache-resident) slots: the maximum, then the integer sum.
-__global__ void __launch_bounds__(128 * kMergeMaxSlices) fold_merge_kernel(const MergeParams p) {
+// grid (Hq, batch); block (32, W), W = blockDim.y <= kMergeMaxWarps chosen from the slot count.  One CTA
+// per (request, q head).  Lane x of every warp owns EPT = D / 32 consecutive elements of A (one vector load
+// per slot); warp y takes the slots y, y + W, ... of every level; lane 0 also carries L.  Two passes over
+// the (cache-resident) slots: the order-free maximum, then the integer sum; warps combine through
+// shared-memory integer atomics, which are order-free by construction.
+template <int EPT>
+__global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const MergeParams p) {
   __shared__ unsigned s_max[129];
   __shared__ unsigned long long s_sum[129];
-  __shared__ float s_l;
   __shared__ int s_flags;
+  constexpr int D = 32 * EPT;
   const int h = blockIdx.x, b = blockIdx.y;
-  const int x = threadIdx.x, y = threadIdx.y, S = blockDim.y;
-  const int D = p.D, G = p.G, kvh = h / G;
-  const int tid = y * D + x;
+  const int x = threadIdx.x, y = threadIdx.y, W = blockDim.y;
+  const int G = p.G, kvh = h / G;
+  const int tid = y * 32 + x;
   const long long row = (long long)b * p.Hq + h;
   pdl_wait();                                        // slots and z come from the kernels before
   const float zrow = p.z[row];                       // requested early: only needed at the very end
 
-  for (int i = tid; i <= D; i += D * S) { s_max[i] = 0u; s_sum[i] = 0ull; }
+  for (int i = tid; i <= D; i += 32 * W) { s_max[i] = 0u; s_sum[i] = 0ull; }
   if (tid == 0) s_flags = 0;
 
-  // per level: this thread's first A element, the row's L element, the slot stride and count
+  // per level: this lane's first A vector, the row's L element, the slot stride and count
   const float *pa[kMaxLevels], *pl[kMaxLevels];
   long long step[kMaxLevels];
   int cnt[kMaxLevels];
@@ -101,69 +85,104 @@ __global__ void __launch_bounds__(128 * kMergeMaxSlices) fold_merge_kernel(const
       C += cnt[l];
       const int r = (b % L.stack) * G + (h % G);
       const float *s0 = L.slots + (((long long)seq * p.Hkv + kvh) * L.max_slots + y) * L.slot_stride;
-      pa[l] = s0 + r * D + x;
+      pa[l] = s0 + r * D + x * EPT;
       pl[l] = s0 + L.rows * D + r;
-      step[l] = L.slot_stride * S;
+      step[l] = L.slot_stride * W;
     }
   }
   const int clog2C = ceil_log2_u32(C);
 
+  auto load_vec = [](const float *a, float (&v)[EPT]) {
+    if (EPT == 4) {
+      const float4 t = *reinterpret_cast<const float4 *>(a);
+      v[0] = t.x; v[1] = t.y; v[EPT - 2] = t.z; v[EPT - 1] = t.w;
+    } else {
+      const float2 t = *reinterpret_cast<const float2 *>(a);
+      v[0] = t.x; v[1] = t.y;
+    }
+  };
+
   // pass 1: order-free maximum of |g| through the bit patterns
-  unsigned mx = 0u, mxl = 0u;
+  unsigned mx[EPT], mxl = 0u;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) mx[e] = 0u;
 #pragma unroll
   for (int l = 0; l < kMaxLevels; ++l) {
-    const float *a = pa[l];
+    const float *a = pa[l], *q = pl[l];
 #pragma unroll 4
-    for (int k = y; k < cnt[l]; k += S, a += step[l]) mx = max(mx, __float_as_uint(*a) & 0x7fffffffu);
-    if (x == 0) {
-      const float *q = pl[l];
-      for (int k = y; k < cnt[l]; k += S, q += step[l]) mxl = max(mxl, __float_as_uint(*q) & 0x7fffffffu);
+    for (int k = y; k < cnt[l]; k += W, a += step[l], q += step[l]) {
+      float v[EPT];
+      load_vec(a, v);
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) mx[e] = max(mx[e], __float_as_uint(v[e]) & 0x7fffffffu);
+      if (x == 0) mxl = max(mxl, __float_as_uint(*q) & 0x7fffffffu);
     }
   }
   __syncthreads();                                   // s_max / s_sum are zeroed
-  if (mx) atomicMax(&s_max[x], mx);
-  if (x == 0 && mxl) atomicMax(&s_max[D], mxl);
-  __syncthreads();
+  if (W > 1) {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) if (mx[e]) atomicMax(&s_max[x * EPT + e], mx[e]);
+    if (x == 0 && mxl) atomicMax(&s_max[D], mxl);
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) mx[e] = s_max[x * EPT + e];
+    mxl = s_max[D];
+  }
+  mxl = __shfl_sync(0xffffffffu, mxl, 0);
 
   // pass 2: integer sums on the declared grid
-  {
-    const unsigned ma = s_max[x], ml = s_max[D];
-    const int eb_a = norm_exp(ma), eb_l = norm_exp(ml);
-    const bool fin_a = (ma >> 23) != 255u, fin_l = (ml >> 23) != 255u;
-    long long acc = 0, accl = 0;
+  long long acc[EPT], accl = 0;
+  double alpha[EPT];
+  bool fin[EPT];
 #pragma unroll
-    for (int l = 0; l < kMaxLevels; ++l) {
-      const float *a = pa[l];
-      if (fin_a) {
+  for (int e = 0; e < EPT; ++e) {
+    acc[e] = 0;
+    alpha[e] = pow2_double(grid_shift(mx[e], clog2C));
+    fin[e] = (mx[e] >> 23) != 255u;
+  }
+  const double alpha_l = pow2_double(grid_shift(mxl, clog2C));
+  const bool fin_l = (mxl >> 23) != 255u;
+#pragma unroll
+  for (int l = 0; l < kMaxLevels; ++l) {
+    const float *a = pa[l], *q = pl[l];
 #pragma unroll 4
-        for (int k = y; k < cnt[l]; k += S, a += step[l]) acc += to_grid(*a, eb_a, clog2C);
-      }
-      if (x == 0 && fin_l) {
-        const float *q = pl[l];
-        for (int k = y; k < cnt[l]; k += S, q += step[l]) accl += to_grid(*q, eb_l, clog2C);
-      }
+    for (int k = y; k < cnt[l]; k += W, a += step[l], q += step[l]) {
+      float v[EPT];
+      load_vec(a, v);
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) if (fin[e]) acc[e] += to_grid(v[e], alpha[e]);
+      if (x == 0 && fin_l) accl += to_grid(*q, alpha_l);
     }
-    if (acc) atomicAdd(&s_sum[x], (unsigned long long)acc);
+  }
+  if (W > 1) {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) if (acc[e]) atomicAdd(&s_sum[x * EPT + e], (unsigned long long)acc[e]);
     if (x == 0 && accl) atomicAdd(&s_sum[D], (unsigned long long)accl);
+    __syncthreads();
+    if (y != 0) return;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) acc[e] = (long long)s_sum[x * EPT + e];
+    accl = (long long)s_sum[D];
   }
-  __syncthreads();
 
-  if (y != 0) return;
-  if (x == 0) {
-    const unsigned ml = s_max[D];
-    s_l = (ml >> 23) == 255u ? __int_as_float(0x7fc00000) : from_grid((long long)s_sum[D], norm_exp(ml), clog2C);
+  // warp 0 finishes the row
+  float Lf = fin_l ? (float)((double)accl * pow2_double(-grid_shift(mxl, clog2C))) : __int_as_float(0x7fc00000);
+  Lf = __shfl_sync(0xffffffffu, Lf, 0);
+  bool bad = false;
+  __nv_bfloat16 ob[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const float Af = fin[e] ? (float)((double)acc[e] * pow2_double(-grid_shift(mx[e], clog2C)))
+                            : __int_as_float(0x7fc00000);
+    const float ov = C == 0 ? 0.f : Af / Lf;
+    bad |= !(fabsf(ov) <= 3.4e38f);
+    ob[e] = __float2bfloat16_rn(ov);
   }
-  // only the y == 0 threads are left: a named barrier over those D threads
-  asm volatile("bar.sync 2, %0;" ::"r"(D) : "memory");
-  const float Lf = s_l;
-  const unsigned ma = s_max[x];
-  const float Af = (ma >> 23) == 255u ? __int_as_float(0x7fc00000) : from_grid((long long)s_sum[x], norm_exp(ma), clog2C);
-  float ov = C == 0 ? 0.f : Af / Lf;
-  p.out[row * D + x] = __float2bfloat16_rn(ov);
-  if (!(fabsf(ov) <= 3.4e38f)) atomicOr(&s_flags, FOLD_ROW_NONFINITE);
-  asm volatile("bar.sync 2, %0;" ::"r"(D) : "memory");
+  if (EPT == 4) *reinterpret_cast<uint2 *>(p.out + row * D + x * EPT) = *reinterpret_cast<uint2 *>(ob);
+  else *reinterpret_cast<uint32_t *>(p.out + row * D + x * EPT) = *reinterpret_cast<uint32_t *>(ob);
+  const unsigned any_bad = __ballot_sync(0xffffffffu, bad);
   if (x == 0) {
-    int flags = s_flags;
+    int flags = any_bad ? FOLD_ROW_NONFINITE : 0;
     float lse;
     if (C == 0) {
       flags = FOLD_ROW_EMPTY;
