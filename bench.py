@@ -194,6 +194,59 @@ def max_over_ranks(ms: float, world: int, device) -> float:
     return float(t.item())
 
 
+def run_sweep(args, dev):
+    """Configuration 5: MHA, 32 heads, D in {64,128}, batch {1,8,64}, context {1K,8K,32K,128K}, T in {8,16,inf}.
+    One JSON line with one record per cell; cells whose cache would not fit under the memory cap are
+    recorded as skipped (pages are never aliased to fake a large batch: L2 hits would inflate GB/s)."""
+    import paper_2609_33410_b200 as F
+    from paper_2609_33410_b200.workloads import make_decode_workload
+    stream = torch.cuda.current_stream()
+    peak, _ = load_peaks()
+    cells = []
+    for D in (64, 128):
+        for B in (1, 8, 64):
+            for n in (1024, 8192, 32768, 131072):
+                cache_bytes = B * n * 32 * 4 * D
+                base = dict(head_dim=D, batch=B, context=n, cache_mb=round(cache_bytes / 1e6, 1))
+                free, _tot = torch.cuda.mem_get_info()
+                if cache_bytes > args.sweep_cap_gb * 1e9 or cache_bytes * 1.3 > free:
+                    cells += [dict(base, T=t, skipped="memory cap") for t in ("8", "16", "inf")]
+                    continue
+                seed = 5000 + D * 7 + B * 131 + n
+                w = make_decode_workload(B, 32, 32, D, n, seed=seed, device=dev)
+                cache = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table)
+                bufs = F.alloc_buffers(w.q, cache)
+                # small caches are L2-resident unless evicted: stream a 512 MB buffer between samples
+                flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if cache_bytes < 4 * 126e6 else None
+                for t_name, T in (("8", 8.0), ("16", 16.0), ("inf", math.inf)):
+                    a = F.make_args(w.q, cache, scale=w.scale, z=bufs.z, depth_T=T, workspace=bufs.workspace,
+                                    out=bufs.out, lse=bufs.lse, row_status=bufs.row_status)
+                    for _ in range(3):
+                        F.fold_decode(a, stream)
+                    reps = 21 if cache_bytes < 2e9 else 7
+                    times = []
+                    for _ in range(reps):
+                        if flush is not None:
+                            flush.fill_(1)
+                        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                        e0.record(stream)
+                        F.fold_decode(a, stream)
+                        e1.record(stream)
+                        torch.cuda.synchronize()
+                        times.append(e0.elapsed_time(e1) * 1e3)
+                    times = sorted(times[1:])                 # drop the first sample, report the median
+                    us = times[len(times) // 2]
+                    h = bufs.header()
+                    lam = h.v_rows_fetched / max(h.v_rows_total, 1)
+                    cells.append(dict(base, T=t_name, us=round(us, 1), us_min=round(times[0], 1),
+                                      effective_gbs=round(cache_bytes / us / 1e3, 1),
+                                      actual_gbs=round(cache_bytes * (0.5 + 0.5 * lam) / us / 1e3, 1),
+                                      v_rows_fetched=round(lam, 4), l2_flush=flush is not None))
+                del w, cache, bufs, flush
+                torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "cells": cells}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -205,6 +258,8 @@ def main():
     ap.add_argument("--ref-units", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="run the MHA sweep (configuration 5) instead of one workload")
+    ap.add_argument("--sweep-cap-gb", type=float, default=40.0)
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -225,6 +280,9 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
+    if args.sweep:
+        run_sweep(args, dev)
+        return
     spec = WORKLOADS[args.workload]
     T = spec["T"]
     stream = torch.cuda.current_stream()
