@@ -258,6 +258,8 @@ def main():
     ap.add_argument("--ref-units", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cascade-streams", type=int, default=1, choices=[1, 2],
+                    help="cascade workloads: scan the levels on one stream (fold_decode_cascade) or on two")
     ap.add_argument("--sweep", action="store_true", help="run the MHA sweep (configuration 5) instead of one workload")
     ap.add_argument("--sweep-cap-gb", type=float, default=40.0)
     args = ap.parse_args()
@@ -306,11 +308,28 @@ def main():
                             num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
                             row_status=bufs.row_status) for l, c, b in zip(levels, caches, lbufs)]
 
+    # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
+    # is scanned on a side stream while the suffix level is scanned on the main one (fork / join with events).
+    side = torch.cuda.Stream(device=dev) if cascade and args.cascade_streams == 2 else None
+    ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
+
     def step_whole(a):
-        if cascade:
+        if not cascade:
+            F.fold_decode(a[0], stream)
+        elif side is None:
             F.fold_decode_cascade(a, stream)
         else:
-            F.fold_decode(a[0], stream)
+            F.fold_estimate_z(a, stream)
+            ev_fork.record(stream)
+            side.wait_event(ev_fork)
+            given = [F.FoldArgs.from_buffer_copy(bytes(x)) for x in a]
+            for x in given:
+                x.z_mode = F.Z_GIVEN
+            p0 = F.fold_decode_split(given[0], side)
+            ev_join.record(side)
+            p1 = F.fold_decode_split(given[1], stream)
+            stream.wait_event(ev_join)
+            F.fold_cascade_merge([p0, p1], bufs.out, bufs.lse, bufs.row_status, stream)
 
     def step_split(a, evs):
         # the same launches issued one by one, so each kernel can be timed on its own
@@ -393,6 +412,7 @@ def main():
                    "num_splits": args.num_splits or "auto", "l2": "inputs (cache) larger than L2, no flush needed"
                    if cache_bytes > 4 * 126e6 else "cache smaller than 4x L2: partly L2-resident",
                    "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
+                   "cascade_streams": args.cascade_streams if cascade else None,
                    "flat_equivalent_bytes_per_gpu": flat_bytes},
         "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
         "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},

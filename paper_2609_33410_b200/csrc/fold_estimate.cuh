@@ -64,16 +64,17 @@ __device__ __forceinline__ int est_sample_key(int i, int n) {
   return (e0 + e1) >> 1;
 }
 
-// One CTA per (kv head, request).  Four threads share a sampled key row (a quarter of its
-// channels each), so all 192 rows are requested at once and the kernel pays one memory
-// latency; warp g then reduces row g of the group.
-constexpr int kEstSampleThreads = 4 * kEstSamples;       // 768
+// One CTA per (kv head, request), 12 warps.  The 192 x G scores are one small matrix product: warp w
+// takes sampled keys 16w .. 16w+15 on M, the group's query rows on N (mma.sync m16n8k16, BF16 in,
+// FP32 accumulate).  Each lane loads its A fragments straight from the cache rows (all loads issued
+// before the first MMA, so the kernel pays one memory latency); warp g then reduces row g.
+constexpr int kEstWarps = kEstSamples / 16;              // 12
+constexpr int kEstSampleThreads = kEstWarps * 32;        // 384
 
 template <int D>
 __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const EstParams p) {
-  constexpr int QD = D / 4;                         // channels per thread
-  __shared__ __align__(16) float qs[kMaxRows][D + 16];   // each quarter of q padded by 4 floats: aligned float4 reads, spread banks
-  __shared__ __align__(16) float sc[kMaxRows][kEstSamples];
+  constexpr int KS = D / 16;
+  __shared__ float sc[kMaxRows][kEstSamples];
   const int kvh = blockIdx.x, req = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G;
@@ -86,50 +87,46 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
     n += lens[l];
   }
   const int n_samples = n < kEstSamples ? n : kEstSamples;
-  const int i = threadIdx.x >> 2, part = threadIdx.x & 3;
+  const int qcol = (lane & 3) * 2;
 
-  // request this thread's quarter row first, then stage q while it is in flight
-  uint4 raw[QD / 8];
+  if (warp * 16 < n_samples) {
+    // the two sampled key rows this lane reads fragments of
+    const __nv_bfloat16 *rowp[2];
 #pragma unroll
-  for (int c = 0; c < QD / 8; ++c) raw[c] = make_uint4(0, 0, 0, 0);
-  if (i < n_samples) {
-    int j = est_sample_key(i, n), l = 0;
-    while (l < p.n_levels - 1 && j >= lens[l]) { j -= lens[l]; ++l; }
-    const uint4 *row = reinterpret_cast<const uint4 *>(key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + part * QD);
-#pragma unroll
-    for (int c = 0; c < QD / 8; ++c) raw[c] = row[c];
-  }
-  for (int e = threadIdx.x; e < G * D; e += kEstSampleThreads) {
-    const int g = e / D, d = e % D;
-    qs[g][(d / QD) * (QD + 4) + d % QD] =
-        __bfloat162float(p.q[(long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + d]);
-  }
-  __syncthreads();
-
-  float kf[QD];
-#pragma unroll
-  for (int c = 0; c < QD / 8; ++c) {
-    const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      kf[c * 8 + 2 * e] = __uint_as_float(w[e] << 16);
-      kf[c * 8 + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+    for (int hlf = 0; hlf < 2; ++hlf) {
+      const int i = warp * 16 + (lane >> 2) + hlf * 8;
+      rowp[hlf] = nullptr;
+      if (i < n_samples) {
+        int j = est_sample_key(i, n), l = 0;
+        while (l < p.n_levels - 1 && j >= lens[l]) { j -= lens[l]; ++l; }
+        rowp[hlf] = key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + qcol;
+      }
     }
-  }
-  for (int g = 0; g < G; ++g) {
-    float acc = 0.f;
-    const float4 *qv = reinterpret_cast<const float4 *>(&qs[g][part * (QD + 4)]);
+    uint32_t a[KS][4];
 #pragma unroll
-    for (int e = 0; e < QD / 4; ++e) {
-      const float4 t = qv[e];
-      acc = fmaf(kf[4 * e], t.x, acc);
-      acc = fmaf(kf[4 * e + 1], t.y, acc);
-      acc = fmaf(kf[4 * e + 2], t.z, acc);
-      acc = fmaf(kf[4 * e + 3], t.w, acc);
+    for (int kk = 0; kk < KS; ++kk) {
+      a[kk][0] = rowp[0] ? *reinterpret_cast<const uint32_t *>(rowp[0] + kk * 16) : 0u;
+      a[kk][1] = rowp[1] ? *reinterpret_cast<const uint32_t *>(rowp[1] + kk * 16) : 0u;
+      a[kk][2] = rowp[0] ? *reinterpret_cast<const uint32_t *>(rowp[0] + kk * 16 + 8) : 0u;
+      a[kk][3] = rowp[1] ? *reinterpret_cast<const uint32_t *>(rowp[1] + kk * 16 + 8) : 0u;
     }
-    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-    if (part == 0 && i < n_samples) sc[g][i] = acc * p.scale_log2;
+    // query rows of the group as B fragments (n = lane / 4), eight rows per n-tile
+#pragma unroll 1
+    for (int nt = 0; nt * 8 < G; ++nt) {
+      const int g = nt * 8 + (lane >> 2);
+      const __nv_bfloat16 *qrow = p.q + (long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + qcol;
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int kk = 0; kk < KS; ++kk) {
+        const uint32_t b0 = g < G ? *reinterpret_cast<const uint32_t *>(qrow + kk * 16) : 0u;
+        const uint32_t b1 = g < G ? *reinterpret_cast<const uint32_t *>(qrow + kk * 16 + 8) : 0u;
+        mma_bf16(c, a[kk], b0, b1);
+      }
+      // c0, c1: key lane/4, rows 2*(lane%4) + {0,1};  c2, c3: key lane/4 + 8
+      const int i0 = warp * 16 + (lane >> 2), g0 = nt * 8 + qcol;
+      if (g0 < G) { sc[g0][i0] = c[0] * p.scale_log2; sc[g0][i0 + 8] = c[2] * p.scale_log2; }
+      if (g0 + 1 < G) { sc[g0 + 1][i0] = c[1] * p.scale_log2; sc[g0 + 1][i0 + 8] = c[3] * p.scale_log2; }
+    }
   }
   __syncthreads();
 
