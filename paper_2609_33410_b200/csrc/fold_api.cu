@@ -8,6 +8,7 @@
 #include "fold_estimate.cuh"
 #include "fold_merge.cuh"
 #include "fold_scan.cuh"
+#include "fold_scan_umma.cuh"
 
 using namespace fold;
 
@@ -249,6 +250,25 @@ int launch_stacked(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, 
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+// Stacked rows on tcgen05 (head_dim 128, at least 64 stacked rows): one CTA per (split, 128-row tile).
+int launch_stacked_umma(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, bool gated,
+                        cudaStream_t st) {
+  p.stages = kUmmaStages;
+  p.vr = 0;
+  grid.x *= (p.R + kUmmaRows - 1) / kUmmaRows;
+  static int configured_g[64] = {0}, configured_d[64] = {0};
+  cudaError_t rc;
+  if (gated) {
+    if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<true>, configured_g)) return e;
+    rc = launch_pdl(fold_scan_stacked_umma_kernel<true>, grid, dim3(kUmmaThreads), UmmaLayout::kTotal, st, mk, mv, p);
+  } else {
+    if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<false>, configured_d)) return e;
+    rc = launch_pdl(fold_scan_stacked_umma_kernel<false>, grid, dim3(kUmmaThreads), UmmaLayout::kTotal, st, mk, mv, p);
+  }
+  if (rc != cudaSuccess) return FOLD_ECUDA;
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 // Gated scan: value slots hold rows whose requests can only be issued after scoring, so shared
 // memory is split between the key ring and the value slots of each slice.
 template <int D>
@@ -323,8 +343,10 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
 
   const dim3 grid(p.num_splits, g.Hkv, g.num_seqs);
   p.box_min = 13;
-  if (stacked)
+  if (stacked) {
+    if (g.D == 128 && g.R >= 64) return launch_stacked_umma(mk, mv, p, grid, gated, st);
     return g.D == 128 ? launch_stacked<128>(mk, mv, p, grid, gated, st) : launch_stacked<64>(mk, mv, p, grid, gated, st);
+  }
   if (g.D == 128) return gated ? launch_gated<128>(mk, mv, p, grid, st) : launch_dense<128>(mk, mv, p, grid, st);
   return gated ? launch_gated<64>(mk, mv, p, grid, st) : launch_dense<64>(mk, mv, p, grid, st);
 }
