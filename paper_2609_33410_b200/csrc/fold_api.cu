@@ -297,14 +297,19 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+// CTAs per (sequence, kv head).  A CTA pays a few microseconds to start (barriers, first loads), so it should
+// walk at least ~32 tiles; below about one and a half waves of CTAs the machine is not filled, so short
+// batches are cut finer instead.  Only scheduling: the result does not depend on the choice.
 int choose_splits(const fold_args *a, const Geometry &g) {
-  const int max_chunks = num_chunks_of(a->kv.max_seqlen) > 0 ? num_chunks_of(a->kv.max_seqlen) : 1;
+  const int n = a->kv.max_seqlen;
+  const int max_chunks = num_chunks_of(n) > 0 ? num_chunks_of(n) : 1;
   if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
-  const long long units = (long long)g.num_seqs * g.Hkv;
-  const long long target = 6LL * 296;
-  long long per_cta = units * max_chunks / target;
-  if (per_cta < 1) per_cta = 1;
-  return (int)((max_chunks + per_cta - 1) / per_cta);
+  const long long units = (long long)g.num_seqs * g.Hkv * ((g.R + 127) / 128);
+  const int tiles_unit = max_chunks * (chunk_keys_of(n) / kTileKeys);
+  int s = tiles_unit / 32;
+  s = s < 1 ? 1 : (s > max_chunks ? max_chunks : s);
+  while (units * s < 444 && s < max_chunks) ++s;
+  return s;
 }
 
 int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
