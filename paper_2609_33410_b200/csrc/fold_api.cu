@@ -219,10 +219,17 @@ int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, di
   if (stages < 2) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = 0;
-  static int configured[64] = {0};
-  if (int rc = opt_in_smem(fold_scan_dense_kernel<D>, configured)) return rc;
-  if (launch_pdl(fold_scan_dense_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
-    return FOLD_ECUDA;
+  if (p.R <= 8) {                                            // rows on N: half the MMAs and accumulators
+    static int configured[64] = {0};
+    if (int rc = opt_in_smem(fold_scan_dense_kernel<D, true>, configured)) return rc;
+    if (launch_pdl(fold_scan_dense_kernel<D, true>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
+      return FOLD_ECUDA;
+  } else {
+    static int configured[64] = {0};
+    if (int rc = opt_in_smem(fold_scan_dense_kernel<D, false>, configured)) return rc;
+    if (launch_pdl(fold_scan_dense_kernel<D, false>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
+      return FOLD_ECUDA;
+  }
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
@@ -290,6 +297,24 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
   if (stages < 2 || vr < 1 || LO::total(stages, vr, p.R) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = vr;
+  if (p.R <= 8) {                                            // rows on N; unpadded value slices leave room for a deeper K ring
+    using LN = GatedNarrowLayout<D>;
+    int nvr = 2;
+    int nstages = (per_cta2 - LN::total(0, nvr)) / (LN::kKTile + 16);
+    if (nstages > 3) nstages = 3;                            // measured: a fourth stage buys nothing and costs L1
+#ifdef FOLD_TUNING
+    if (const char *e = getenv("FOLD_TUNE_STAGES")) nstages = atoi(e);
+    if (const char *e = getenv("FOLD_TUNE_VR")) nvr = atoi(e);
+#endif
+    if (nstages < 2 || nvr < 1 || LN::total(nstages, nvr) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
+    p.stages = nstages;
+    p.vr = nvr;
+    static int configured[64] = {0};
+    if (int rc = opt_in_smem(fold_scan_gated_narrow_kernel<D>, configured)) return rc;
+    if (launch_pdl(fold_scan_gated_narrow_kernel<D>, grid, dim3(kGatedThreads), LN::total(nstages, nvr), st, mk, mvs, p) != cudaSuccess)
+      return FOLD_ECUDA;
+    return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+  }
   static int configured[64] = {0};
   if (int rc = opt_in_smem(fold_scan_gated_kernel<D>, configured)) return rc;
   if (launch_pdl(fold_scan_gated_kernel<D>, grid, dim3(kGatedThreads), LO::total(stages, vr, p.R), st, mk, mvs, p) != cudaSuccess)

@@ -81,7 +81,27 @@ struct GatedLayout {
   }
 };
 
-__device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+// Narrow gated kernel: every value slice in the swizzled box layout (no row padding), and a two-warp
+// parking area for the chunk-end add.
+template <int D>
+struct GatedNarrowLayout {
+  static constexpr int kKTile = kTileKeys * D * 2;
+  static constexpr int kVSlice = 16 * D * 2;                 // [D/64 halves][16 rows][128 B], swizzled
+  static constexpr int kPEntry = 512 + 32;                   // 16 B of B-operand registers per lane + the verdict
+  static constexpr int kPark = D / 16 * 4 * 32 * 4;          // one warp's accumulators, fragment order
+  __host__ __device__ static int off_vring(int stages) { return stages * kKTile; }
+  __host__ __device__ static int off_pring(int stages, int vr) { return off_vring(stages) + kConsumerWarps * vr * kVSlice; }
+  __host__ __device__ static int off_red(int stages, int vr) { return off_pring(stages, vr) + kConsumerWarps * vr * kPEntry; }
+  __host__ __device__ static int off_redl(int stages, int vr) { return off_red(stages, vr) + 2 * kPark; }
+  __host__ __device__ static int off_bar(int stages, int vr) { return off_redl(stages, vr) + kConsumerWarps * kMaxRows * 4; }
+  __host__ __device__ static int total(int stages, int vr) {
+    return off_bar(stages, vr) + 2 * stages * 8 + 2 * kConsumerWarps * vr * 8 + 1024;
+  }
+};
+
+__device__ __forceinline__ void named_bar(int id, int threads = 128) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 
 // ------------------------------------------------------------------------------------------------
 // Geometry of the CTA's work: sequence length, tiles, chunks.
@@ -322,8 +342,204 @@ __device__ __forceinline__ void reduce_store_L(float &l_lo, float &l_hi, float *
 }
 
 // ------------------------------------------------------------------------------------------------
-// Dense decode (T = inf)
+// Narrow row blocks (at most 8 query rows per (sequence, kv head): every GQA group up to 8).
+// The products are turned round -- keys, then channels, on M and the query rows on N = 8 -- as
+// Algorithm 1 has them: half the MMAs and half the accumulator registers of the rows-on-M form.
+//   scores   S^T[16 keys, 8 rows] = K[16, D] Q^T            (A = K slice by ldmatrix, B = Q registers)
+//   values   A^T[D, 8 rows]      += V^T[D, 16 keys] P^T      (A = V slice by ldmatrix.trans, B = P^T)
+// P^T comes out of the score fragment by one movmatrix per 8x8 block.
 template <int D>
+struct RowBlockN {
+  uint32_t qb[D / 16][2];      // B fragments: row lane/4, channels kk*16 + (lane%4)*2 + {0,1} (+8)
+  float z0, z1;                // references of the two rows this thread's score fragment holds: (lane%4)*2 + {0,1}
+  bool v0, v1;
+};
+template <int D>
+__device__ __forceinline__ void load_rows_n(RowBlockN<D> &rb, const ScanParams &p, int seq, int kvh, int lane) {
+  {
+    const int r = lane >> 2;                                  // the row this lane feeds as B operand
+    const bool ok = r < p.R;
+    const int req = seq * p.stack + r / p.G, head = kvh * p.G + r % p.G;
+    const __nv_bfloat16 *q = p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + (lane & 3) * 2;
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+      rb.qb[kk][0] = ok ? *reinterpret_cast<const uint32_t *>(q + kk * 16) : 0u;
+      rb.qb[kk][1] = ok ? *reinterpret_cast<const uint32_t *>(q + kk * 16 + 8) : 0u;
+    }
+  }
+  const int r0 = (lane & 3) * 2;                              // the rows this lane holds scores of
+  rb.v0 = r0 < p.R;
+  rb.v1 = r0 + 1 < p.R;
+  const int req0 = seq * p.stack + r0 / p.G, head0 = kvh * p.G + r0 % p.G;
+  const int req1 = seq * p.stack + (r0 + 1) / p.G, head1 = kvh * p.G + (r0 + 1) % p.G;
+  rb.z0 = rb.v0 ? p.z[(long long)req0 * p.Hq + head0] : 0.f;
+  rb.z1 = rb.v1 ? p.z[(long long)req1 * p.Hq + head1] : 0.f;
+}
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
+// s[0], s[1]: key lane/4, rows (lane%4)*2 + {0,1};  s[2], s[3]: key lane/4 + 8.
+template <int D>
+__device__ __forceinline__ void qk_issue_n(const RowBlockN<D> &rb, uint32_t kt, int slice, int lane, float (&s)[4]) {
+  // ldmatrix matrix i = lane/8: keys (i&1)*8 + lane%8 of the slice, 16-byte chunk 2*kk + (i>>1)
+  const int k_key = slice * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
+  const uint32_t k_row = k_key * 128, k_x = (lane >> 4) ^ (k_key & 7);
+  s[0] = s[1] = s[2] = s[3] = 0.f;
+#pragma unroll
+  for (int kk = 0; kk < D / 16; ++kk) {
+    uint32_t a[4];
+    ldsm_x4(kt + (kk >> 2) * (kTileKeys * 128) + k_row + ((((2 * kk) & 7) ^ k_x) << 4), a[0], a[1], a[2], a[3]);
+    mma_bf16(s, a, rb.qb[kk][0], rb.qb[kk][1]);
+  }
+}
+
+// Final weights of a slice.  Returns the fetch mask; bh / bl receive P_hi^T / P_lo^T as B fragments of the
+// value product; l0 / l1 accumulate this thread's share of L for rows (lane%4)*2 + {0,1}.
+template <int D, bool GATED>
+__device__ __forceinline__ uint32_t weights_n(const RowBlockN<D> &rb, const float (&s)[4], int lane, int key0, int n,
+                                              float scale_log2, float neg_T, uint32_t (&bh)[2], uint32_t (&bl)[2],
+                                              float &l0, float &l1) {
+  const int klo = lane >> 2;
+  uint32_t livemask = 0;
+#pragma unroll
+  for (int kh = 0; kh < 2; ++kh) {                            // key lane/4, then key lane/4 + 8
+    const bool kvalid = (key0 + klo + 8 * kh) < n;
+    float pw[2], pm[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const bool ok = kvalid && (e ? rb.v1 : rb.v0);
+      const float x = ok ? fmaf(s[2 * kh + e], scale_log2, e ? -rb.z1 : -rb.z0) : -INFINITY;
+      const bool live = GATED ? (x >= neg_T) : ok;
+      pw[e] = ex2_approx(x);
+      pm[e] = live ? pw[e] : 0.f;
+      if (live) livemask |= 1u << (klo + 8 * kh);
+    }
+    const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
+    const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
+    const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
+    const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
+    l0 += (h0 + g0) + (pw[0] - pm[0]);
+    l1 += (h1 + g1) + (pw[1] - pm[1]);
+    bh[kh] = movmatrix_trans(hi2);                            // [key][row] block -> [row][key]: the B fragment
+    bl[kh] = movmatrix_trans(lo2);
+  }
+  return __reduce_or_sync(0xffffffffu, livemask);
+}
+
+// A^T += V^T (P_hi^T + P_lo^T) for one slice; o[mt]: channels 16*mt + lane/4 (+8), rows (lane%4)*2 + {0,1}.
+template <int D, bool SWIZZLED, int ROW_BYTES, int HALF_ROWS = kTileKeys>
+__device__ __forceinline__ void value_product_n(float (&o)[D / 16][4], uint32_t vbase, int row0, int lane,
+                                                const uint32_t (&bh)[2], const uint32_t (&bl)[2]) {
+  // ldmatrix.trans matrix i = lane/8: keys (i>>1)*8 + lane%8, 16-byte chunk 2*mt + (i&1)
+  const int v_key = ((lane >> 4) << 3) + (lane & 7);
+  const uint32_t sw_row = (row0 + v_key) * 128, sw_x = ((lane >> 3) & 1) ^ (v_key & 7);
+  const uint32_t pad_off = v_key * ROW_BYTES + ((lane >> 3) & 1) * 16;
+#pragma unroll
+  for (int mt = 0; mt < D / 16; ++mt) {
+    uint32_t a[4];
+    if (SWIZZLED) ldsm_x4_trans(vbase + (mt >> 2) * (HALF_ROWS * 128) + sw_row + ((((2 * mt) & 7) ^ sw_x) << 4), a[0], a[1], a[2], a[3]);
+    else ldsm_x4_trans(vbase + pad_off + mt * 32, a[0], a[1], a[2], a[3]);
+    mma_bf16(o[mt], a, bh[0], bh[1]);
+    mma_bf16(o[mt], a, bl[0], bl[1]);
+  }
+}
+
+// Chunk end for narrow blocks: park the warp's partial as [row][channel], add the warps in order, store.
+template <int D, int WARPS>
+__device__ __forceinline__ void reduce_store_A_n(float (&o)[D / 16][4], float *red, float *slot, int R, int warp,
+                                                 int lane, int tid, int bar_id) {
+  const int r0 = (lane & 3) * 2, c0 = lane >> 2;
+  float *mine = red + warp * R * D;
+#pragma unroll
+  for (int mt = 0; mt < D / 16; ++mt) {
+    if (r0 < R) { mine[r0 * D + mt * 16 + c0] = o[mt][0]; mine[r0 * D + mt * 16 + c0 + 8] = o[mt][2]; }
+    if (r0 + 1 < R) { mine[(r0 + 1) * D + mt * 16 + c0] = o[mt][1]; mine[(r0 + 1) * D + mt * 16 + c0 + 8] = o[mt][3]; }
+    o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+  }
+  named_bar(bar_id, WARPS * 32);
+  const int RD = R * D;
+  for (int i = tid; i < RD; i += WARPS * 32) {
+    float v = red[i];
+#pragma unroll
+    for (int wv = 1; wv < WARPS; ++wv) v += red[wv * RD + i];
+    slot[i] = v;
+  }
+  named_bar(bar_id, WARPS * 32);
+}
+// The same for four warps in a quarter of the room: warps 2, 3 park in fragment order, warps 0, 1 take them
+// in; warp 1 parks, warp 0 takes it in and stores:  (w0 + w2) + (w1 + w3), always in this order.
+template <int D>
+__device__ __forceinline__ void tree_store_A_n(float (&o)[D / 16][4], float *park, float *slot, int R, int warp,
+                                               int lane, int bar_id) {
+  constexpr int kPerWarp = D / 16 * 4 * 32;
+  if (warp >= 2) {
+#pragma unroll
+    for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) park[(warp - 2) * kPerWarp + (mt * 4 + j) * 32 + lane] = o[mt][j];
+  }
+  named_bar(bar_id, 128);
+  if (warp < 2) {
+#pragma unroll
+    for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) o[mt][j] += park[warp * kPerWarp + (mt * 4 + j) * 32 + lane];
+  }
+  named_bar(bar_id, 128);
+  if (warp == 1) {
+#pragma unroll
+    for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) park[(mt * 4 + j) * 32 + lane] = o[mt][j];
+  }
+  named_bar(bar_id, 128);
+  if (warp == 0) {
+    const int r0 = (lane & 3) * 2, c0 = lane >> 2;
+#pragma unroll
+    for (int mt = 0; mt < D / 16; ++mt) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int r = r0 + (j & 1);
+        const float v = o[mt][j] + park[(mt * 4 + j) * 32 + lane];
+        if (r < R) slot[r * D + mt * 16 + c0 + (j >> 1) * 8] = v;
+      }
+    }
+  }
+#pragma unroll
+  for (int mt = 0; mt < D / 16; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+  named_bar(bar_id, 128);
+}
+template <int WARPS>
+__device__ __forceinline__ void reduce_store_L_n(float &l0, float &l1, float *redl, float *slot_l, int R, int warp,
+                                                 int lane, int tid, int bar_id) {
+#pragma unroll
+  for (int m = 4; m <= 16; m <<= 1) {
+    l0 += __shfl_xor_sync(0xffffffffu, l0, m);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, m);
+  }
+  const int r0 = (lane & 3) * 2;
+  if (lane < 4) {
+    if (r0 < R) redl[warp * kMaxRows + r0] = l0;
+    if (r0 + 1 < R) redl[warp * kMaxRows + r0 + 1] = l1;
+  }
+  l0 = l1 = 0.f;
+  named_bar(bar_id, WARPS * 32);
+  if (tid < R) {
+    float v = redl[tid];
+#pragma unroll
+    for (int wv = 1; wv < WARPS; ++wv) v += redl[wv * kMaxRows + tid];
+    slot_l[tid] = v;
+  }
+  named_bar(bar_id, WARPS * 32);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Dense decode (T = inf)
+template <int D, bool NARROW>
 __global__ void __launch_bounds__(kDenseThreads, 2)
 fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const ScanParams p) {
@@ -357,11 +573,12 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     return;
   }
 
-  RowBlock<D> rb;
-  load_rows<D>(rb, p, seq, kvh, lane);
-  float o[D / 8][4];
+  // rows on M (up to 16 rows) or on N (up to 8 rows): see "Narrow row blocks"
+  typename std::conditional<NARROW, RowBlockN<D>, RowBlock<D>>::type rb;
+  if constexpr (NARROW) load_rows_n<D>(rb, p, seq, kvh, lane); else load_rows<D>(rb, p, seq, kvh, lane);
+  float o[NARROW ? D / 16 : D / 8][4];
 #pragma unroll
-  for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  for (int i = 0; i < (NARROW ? D / 16 : D / 8); ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
   float l_lo = 0.f, l_hi = 0.f;
   float *red = reinterpret_cast<float *>(gen + LO::off_red(stages));
   float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, R));
@@ -380,8 +597,6 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       if (!ready) continue;
       const uint32_t kt = base + my_stage * LO::kStage;
       const int key0 = t * kTileKeys + warp * 16;
-      uint32_t ah[4], al[4];
-      const uint32_t fetch16 = score_slice<D, false, 1>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
       st_total += min(16, max(0, n - key0));
       if (key0 + 16 > n) {                                   // ragged tail: value rows past n may hold anything
         for (int r = 0; r < 16; ++r)
@@ -390,14 +605,29 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
                                        tile_off(warp * 16 + r, lane, kTileKeys)) = make_uint4(0, 0, 0, 0);
         __syncwarp();
       }
-      if (fetch16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, ah, al);
+      if constexpr (NARROW) {
+        float s[4];
+        uint32_t bh[2], bl[2];
+        qk_issue_n<D>(rb, kt, warp, lane, s);
+        const uint32_t fetch16 = weights_n<D, false>(rb, s, lane, key0, n, p.scale_log2, p.neg_T, bh, bl, l_lo, l_hi);
+        if (fetch16 != 0) value_product_n<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, bh, bl);
+      } else {
+        uint32_t ah[4], al[4];
+        const uint32_t fetch16 = score_slice<D, false, 1>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        if (fetch16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, ah, al);
+      }
       if (key0 + 16 > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);
     }
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
-    reduce_store_L(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
-    reduce_store_A<D>(o, red, slot, R, warp, lane, threadIdx.x, 1);
+    if constexpr (NARROW) {
+      reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
+      reduce_store_A_n<D, kConsumerWarps>(o, red, slot, R, warp, lane, threadIdx.x, 1);
+    } else {
+      reduce_store_L(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
+      reduce_store_A<D>(o, red, slot, R, warp, lane, threadIdx.x, 1);
+    }
   }
 
   if (lane == 0) {
@@ -734,6 +964,185 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       if (cursor_next(k, w, p.num_splits)) {
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
         reduce_store_A<D>(o, red, slot, R, sl, lane, threadIdx.x - 128, 2);
+      }
+    }
+    if (lane == 0 && dead) atomicOr(&p.hdr->wait_timeouts, 4u);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Depth-gated decode for narrow row blocks (at most 8 rows): the same roles with the products turned
+// round (rows on N), which halves the MMAs and the accumulator registers.  Value slices always sit in
+// the swizzled box layout, whichever way they were fetched.
+template <int D>
+__global__ void __launch_bounds__(kGatedThreads, 2)
+fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
+                              const ScanParams p) {
+  using LO = GatedNarrowLayout<D>;
+  constexpr int C16 = D / 8;                                 // 16-byte chunks per value row
+  constexpr int RPI = 32 / C16;                              // rows one warp-wide async copy covers
+  constexpr int SW = kConsumerWarps;                         // scorer warps
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
+  const SeqWork w = seq_work(p, seq);
+  if (split >= w.n_chunks) return;
+  const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
+  const uint32_t full0 = base + LO::off_bar(stages, vr), empty0 = full0 + 8u * stages;
+  const uint32_t vfull0 = empty0 + 8u * stages, vempty0 = vfull0 + 8u * kConsumerWarps * vr;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, kConsumerWarps);
+    }
+    for (int s = 0; s < kConsumerWarps * vr; ++s) {
+      mbar_init(vfull0 + 8u * s, 1);
+      mbar_init(vempty0 + 8u * s, 1);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();                                                // z (and the zeroed header) come from earlier work
+
+  if (warp == SW + kConsumerWarps) {
+    if (lane == 0) produce_tiles<D, false, LO::kKTile>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
+    return;
+  }
+
+  const bool scorer = warp < SW;
+  const int sl = warp & 3;                                   // the slice of every tile this warp owns
+  constexpr int pentry = LO::kPEntry, pmask = 512;
+  uint8_t *pring = gen + LO::off_pring(stages, vr) + sl * vr * pentry;
+  const uint32_t vring = base + LO::off_vring(stages) + sl * vr * LO::kVSlice;
+  const uint32_t vfull = vfull0 + 8u * sl * vr, vempty = vempty0 + 8u * sl * vr;
+  bool dead = false;
+  int vs = 0;
+  uint32_t vphase = 0, vwrapped = 0;
+
+  if (scorer) {
+    RowBlockN<D> rb;
+    load_rows_n<D>(rb, p, seq, kvh, lane);
+    float l0 = 0.f, l1 = 0.f;
+    float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, vr));
+    const int page_mask = (1 << p.page_shift) - 1;
+    const uint64_t vpol = policy_evict_first();
+    // row-by-row fetch: lane covers 16-byte chunk (lane % C16) of rows (lane / C16) + RPI * i, swizzled as a box is
+    const uint32_t rdst0 = ((lane % C16) >> 3) * (16 * 128) + (lane / C16) * 128;
+    const long long rsrc0 = (long long)(lane / C16) * p.v_stride_tok + (lane % C16) * 8;
+    int stage = 0;
+    uint32_t phase = 0;
+    unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
+
+    for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
+      const int my_stage = stage, my_vs = vs;
+      const uint32_t my_phase = phase, my_vphase = vphase, my_wrapped = vwrapped;
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+      if (++vs == vr) { vs = 0; vwrapped = 1u; vphase ^= 1u; }
+      {
+        const bool ready = mbar_wait(full0 + 8u * my_stage, my_phase, dead);
+        const int key0 = k.t * kTileKeys + sl * 16;
+        uint32_t bh[2] = {0u, 0u}, bl[2] = {0u, 0u};
+        uint32_t fetch16 = 0;
+        if (ready) {
+          float s[4];
+          qk_issue_n<D>(rb, base + my_stage * LO::kKTile, sl, lane, s);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty0 + 8u * my_stage); // the K slice is consumed: release the tile
+          fetch16 = weights_n<D, true>(rb, s, lane, key0, n, p.scale_log2, p.neg_T, bh, bl, l0, l1);
+        }
+        const bool whole = (key0 + 16 <= n) && (__popc(fetch16) >= p.box_min);
+        {
+          const int nvalid = min(16, max(0, n - key0));
+          st_total += nvalid;
+          st_fetched += whole ? 16 : __popc(fetch16);
+          st_skipped += (fetch16 == 0 && nvalid > 0) ? 1 : 0;
+        }
+        if (!my_wrapped || mbar_wait(vempty + 8u * my_vs, my_vphase ^ 1u, dead)) {
+          uint8_t *pe = pring + my_vs * pentry;
+          *reinterpret_cast<uint4 *>(pe + lane * 16) = make_uint4(bh[0], bh[1], bl[0], bl[1]);
+          if (lane == 0) *reinterpret_cast<uint32_t *>(pe + pmask) = fetch16 | (whole ? 0x10000u : 0u);
+          const uint32_t bar = vfull + 8u * my_vs;
+          if (fetch16 != 0u) {
+            int c_seq = seq, c_tok = key0;
+            if (p.paged) {
+              const int pg = p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)];
+              c_seq = min(max(pg, 0), p.num_pages - 1);
+              c_tok = key0 & page_mask;
+            }
+            const uint32_t vdst = vring + my_vs * LO::kVSlice;
+            if (whole) {
+              fence_proxy_async_smem();                      // the slot's earlier generic-proxy traffic, then TMA writes
+              __syncwarp();
+              if (lane == 0) {
+                mbar_expect_tx(bar, 16 * D * 2);
+                const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
+                const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
+                const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
+#pragma unroll
+                for (int h = 0; h < D / 64; ++h) tma_load_4d(vdst + h * (16 * 128), &tmVs, bar, h * 64, c1, c2, c3, vpol);
+              }
+            } else {
+              const __nv_bfloat16 *src = p.v + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
+                                         (long long)kvh * p.v_stride_head + rsrc0;
+#pragma unroll
+              for (int i = 0; i < 16 / RPI; ++i) {
+                const int row = i * RPI + lane / C16;
+                const bool f = (fetch16 >> row) & 1u;
+                cp_async_16(vdst + rdst0 + i * (RPI * 128) + ((((lane % C16) ^ row) & 7) << 4), f ? src : p.v, f ? 16u : 0u);
+                src += (long long)RPI * p.v_stride_tok;
+              }
+              cp_async_mbar_arrive(bar);                     // this lane's copies hold the phase open
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar);
+            }
+          } else {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar);
+          }
+        }
+      }
+      const int c_done = k.c;
+      if (cursor_next(k, w, p.num_splits)) {
+        float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
+        reduce_store_L_n<SW>(l0, l1, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
+      }
+    }
+    if (lane == 0) {
+      if (dead) atomicOr(&p.hdr->wait_timeouts, 2u);
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_fetched);
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
+      if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
+    }
+  } else {
+    float o[D / 16][4];
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float *red = reinterpret_cast<float *>(gen + LO::off_red(stages, vr));
+    for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
+      const int my = vs;
+      const bool landed = mbar_wait(vfull + 8u * my, vphase, dead);
+      if (++vs == vr) { vs = 0; vphase ^= 1u; }
+      if (landed) {
+        const uint8_t *pe = pring + my * pentry;
+        const uint32_t verdict = *reinterpret_cast<const uint32_t *>(pe + pmask);
+        if (verdict != 0u) {
+          const uint4 a = *reinterpret_cast<const uint4 *>(pe + lane * 16);
+          const uint32_t bh[2] = {a.x, a.y}, bl[2] = {a.z, a.w};
+          value_product_n<D, true, 0, 16>(o, vring + my * LO::kVSlice, 0, lane, bh, bl);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(vempty + 8u * my);
+      }
+      const int c_done = k.c;
+      if (cursor_next(k, w, p.num_splits)) {
+        float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
+        tree_store_A_n<D>(o, red, slot, R, sl, lane, 2);
       }
     }
     if (lane == 0 && dead) atomicOr(&p.hdr->wait_timeouts, 4u);
