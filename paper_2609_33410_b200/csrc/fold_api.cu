@@ -206,9 +206,9 @@ int opt_in_smem(Kernel k, int *configured) {
 }
 
 // Ring depths: two CTAs per SM when a useful ring fits, else one CTA with a deeper ring.
-template <int D>
-int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
-  using LO = DenseLayout<D>;
+template <int D, bool NARROW>
+int launch_dense_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LO = DenseLayout<D, NARROW ? narrow_tile_keys<D>() : kTileKeys>;
   const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
   int stages = (per_cta2 - LO::total(0, p.R)) / (LO::kStage + 16);
   if (stages < 3) stages = (kSmemPerCtaMax - LO::total(0, p.R)) / (LO::kStage + 16);
@@ -219,18 +219,16 @@ int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, di
   if (stages < 2) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = 0;
-  if (p.R <= 8) {                                            // rows on N: half the MMAs and accumulators
-    static int configured[64] = {0};
-    if (int rc = opt_in_smem(fold_scan_dense_kernel<D, true>, configured)) return rc;
-    if (launch_pdl(fold_scan_dense_kernel<D, true>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
-      return FOLD_ECUDA;
-  } else {
-    static int configured[64] = {0};
-    if (int rc = opt_in_smem(fold_scan_dense_kernel<D, false>, configured)) return rc;
-    if (launch_pdl(fold_scan_dense_kernel<D, false>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
-      return FOLD_ECUDA;
-  }
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_dense_kernel<D, NARROW>, configured)) return rc;
+  if (launch_pdl(fold_scan_dense_kernel<D, NARROW>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
+    return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+template <int D>
+int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
+  // up to 8 rows: rows on N (half the MMAs and accumulators), 16 KB key tiles at either head dimension
+  return p.R <= kNarrowRows ? launch_dense_as<D, true>(mk, mv, p, grid, st) : launch_dense_as<D, false>(mk, mv, p, grid, st);
 }
 
 // Stacked rows: the dense ring without reduction buffers; one CTA per (split, 64-row group).
@@ -297,7 +295,7 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
   if (stages < 2 || vr < 1 || LO::total(stages, vr, p.R) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = vr;
-  if (p.R <= 8) {                                            // rows on N; unpadded value slices leave room for a deeper K ring
+  if (p.R <= kNarrowRows) {                                  // rows on N; unpadded value slices leave room for a deeper K ring
     using LN = GatedNarrowLayout<D>;
     int nvr = 2;
     int nstages = (per_cta2 - LN::total(0, nvr)) / (LN::kKTile + 16);
@@ -325,12 +323,12 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
 // CTAs per (sequence, kv head).  A CTA pays a few microseconds to start (barriers, first loads), so it should
 // walk at least ~32 tiles; below about one and a half waves of CTAs the machine is not filled, so short
 // batches are cut finer instead.  Only scheduling: the result does not depend on the choice.
-int choose_splits(const fold_args *a, const Geometry &g) {
+int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   const int n = a->kv.max_seqlen;
   const int max_chunks = num_chunks_of(n) > 0 ? num_chunks_of(n) : 1;
   if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
   const long long units = (long long)g.num_seqs * g.Hkv * ((g.R + 127) / 128);
-  const int tiles_unit = max_chunks * (chunk_keys_of(n) / kTileKeys);
+  const int tiles_unit = max_chunks * (chunk_keys_of(n) / tile_keys);
   int s = tiles_unit / 32;
   s = s < 1 ? 1 : (s > max_chunks ? max_chunks : s);
   while (units * s < 444 && s < max_chunks) ++s;
@@ -340,7 +338,9 @@ int choose_splits(const fold_args *a, const Geometry &g) {
 int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const fold_kv &kv = a->kv;
   const bool paged = kv.page_table != nullptr;
-  const int box_tok = paged ? (kv.page_size < kTileKeys ? kv.page_size : kTileKeys) : kTileKeys;
+  // narrow row blocks walk 16 KB key tiles: 128 keys at D = 64
+  const int tile_keys = (g.R <= kNarrowRows && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
+  const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   const bool gated = !isinf(a->depth_T);
   CUtensorMap mk, mv;
   MapAxes axes;
@@ -367,7 +367,7 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.max_pages = kv.max_pages_per_seq; p.num_pages = kv.num_pages > 0 ? kv.num_pages : 1;
   p.box_tok = box_tok;
   p.pos_tok = axes.pos_tok; p.pos_head = axes.pos_head; p.pos_seq = axes.pos_seq;
-  p.num_splits = choose_splits(a, g);
+  p.num_splits = choose_splits(a, g, tile_keys);
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
   p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
 

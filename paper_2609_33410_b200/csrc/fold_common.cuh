@@ -14,6 +14,11 @@
 namespace fold {
 
 constexpr int kTileKeys = 64;            // keys per tile (Algorithm 1 walks 64-key tiles)
+// Narrow row blocks walk 16 KB key tiles whatever the head dimension (64 keys at D = 128, 128 at D = 64), so a
+// warp's slice is always 4 KB of keys and the per-slice costs (waits, hand-offs) are paid per byte alike.
+constexpr int kNarrowRows = 8;           // row blocks up to this size put the rows on the MMA's N side
+template <int D>
+__host__ __device__ constexpr int narrow_tile_keys() { return 8192 / D; }
 constexpr int kConsumerWarps = 4;        // each owns 16 keys of every tile
 constexpr int kScanThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
 constexpr int kMaxRows = 16;             // query rows one row block holds (MMA M)
@@ -56,6 +61,9 @@ __device__ __forceinline__ void mbar_fence_init() {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {   // no arrival: bytes only
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");

@@ -51,9 +51,9 @@ constexpr int kDenseThreads = (kConsumerWarps + 1) * 32;        // 4 consumers +
 constexpr int kGatedThreads = (2 * kConsumerWarps + 1) * 32;    // 4 scorers + 4 multipliers + producer
 
 // Shared-memory carve-up.  All offsets are from a 1 KB-aligned base.
-template <int D>
+template <int D, int TK = kTileKeys>
 struct DenseLayout {
-  static constexpr int kKTile = kTileKeys * D * 2;
+  static constexpr int kKTile = TK * D * 2;
   static constexpr int kStage = 2 * kKTile;                                    // K tile then V tile
   __host__ __device__ static int off_red(int stages) { return stages * kStage; }
   __host__ __device__ static int off_redl(int stages, int R) { return off_red(stages) + kConsumerWarps * R * D * 4; }
@@ -85,9 +85,11 @@ struct GatedLayout {
 // parking area for the chunk-end add.
 template <int D>
 struct GatedNarrowLayout {
-  static constexpr int kKTile = kTileKeys * D * 2;
-  static constexpr int kVSlice = 16 * D * 2;                 // [D/64 halves][16 rows][128 B], swizzled
-  static constexpr int kPEntry = 512 + 32;                   // 16 B of B-operand registers per lane + the verdict
+  static constexpr int kTK = narrow_tile_keys<D>();          // keys per tile
+  static constexpr int kU = kTK / 64;                        // 16-key sub-slices per warp slice
+  static constexpr int kKTile = kTK * D * 2;
+  static constexpr int kVSlice = 16 * kU * D * 2;            // [D/64 halves][16 kU rows][128 B], swizzled
+  static constexpr int kPEntry = kU * 512 + 32;              // 16 B of B-operand registers per lane and sub-slice + the verdict
   static constexpr int kPark = D / 16 * 4 * 32 * 4;          // one warp's accumulators, fragment order
   __host__ __device__ static int off_vring(int stages) { return stages * kKTile; }
   __host__ __device__ static int off_pring(int stages, int vr) { return off_vring(stages) + kConsumerWarps * vr * kVSlice; }
@@ -108,12 +110,13 @@ __device__ __forceinline__ void named_bar(int id, int threads = 128) {
 struct SeqWork {
   int n, n_tiles, ctiles, n_chunks;
 };
+template <int TK = kTileKeys>
 __device__ __forceinline__ SeqWork seq_work(const ScanParams &p, int seq) {
   SeqWork w;
   int n = p.seqlens[seq];
   w.n = n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
-  w.n_tiles = (w.n + kTileKeys - 1) / kTileKeys;
-  w.ctiles = chunk_keys_of(w.n) / kTileKeys;
+  w.n_tiles = (w.n + TK - 1) / TK;
+  w.ctiles = chunk_keys_of(w.n) / TK;
   w.n_chunks = num_chunks_of(w.n);
   return w;
 }
@@ -139,23 +142,23 @@ __device__ __forceinline__ bool cursor_next(TileCursor &k, const SeqWork &w, int
 }
 
 // Producer thread: TMA-stage the tiles of chunks split, split + num_splits, ... in order.
-template <int D, bool WITH_V, int STAGE_BYTES>
+template <int D, bool WITH_V, int STAGE_BYTES, int TK = kTileKeys>
 __device__ __forceinline__ void produce_tiles(const CUtensorMap *tmK, const CUtensorMap *tmV, const ScanParams &p,
                                               const SeqWork &w, int split, int kvh, int seq, uint32_t ring,
                                               uint32_t full0, uint32_t empty0) {
   constexpr int HALVES = D / 64;
-  constexpr int KTILE = kTileKeys * D * 2;
+  constexpr int KTILE = TK * D * 2;
   tma_prefetch_desc(tmK);
   if (WITH_V) tma_prefetch_desc(tmV);
   const uint64_t pol = policy_evict_first();
   bool dead = false;
   int stage = 0;
   uint32_t wrapped = 0, phase = 0;                 // phase = parity of the ring round being refilled
-  const int boxes_per_tile = kTileKeys / p.box_tok;
+  const int boxes_per_tile = TK / p.box_tok;
   const int page_mask = (1 << p.page_shift) - 1;
   for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w); cursor_next(k, w, p.num_splits)) {
     if (wrapped && !mbar_wait(empty0 + 8u * stage, phase ^ 1u, dead)) break;
-    const int tok0 = k.t * kTileKeys;
+    const int tok0 = k.t * TK;
     const int nbox = min(boxes_per_tile, (w.n - tok0 + p.box_tok - 1) / p.box_tok);
     const uint32_t full = full0 + 8u * stage;
     mbar_expect_tx(full, nbox * p.box_tok * D * 2 * (WITH_V ? 2 : 1));
@@ -174,7 +177,7 @@ __device__ __forceinline__ void produce_tiles(const CUtensorMap *tmK, const CUte
       const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
 #pragma unroll
       for (int h = 0; h < HALVES; ++h) {
-        const uint32_t o = (h * kTileKeys + bx * p.box_tok) * 128;
+        const uint32_t o = (h * TK + bx * p.box_tok) * 128;
         tma_load_4d(kdst + o, tmK, full, h * 64, c1, c2, c3, pol);
         if (WITH_V) tma_load_4d(vdst + o, tmV, full, h * 64, c1, c2, c3, pol);
       }
@@ -383,7 +386,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 }
 
 // s[0], s[1]: key lane/4, rows (lane%4)*2 + {0,1};  s[2], s[3]: key lane/4 + 8.
-template <int D>
+template <int D, int TK = kTileKeys>
 __device__ __forceinline__ void qk_issue_n(const RowBlockN<D> &rb, uint32_t kt, int slice, int lane, float (&s)[4]) {
   // ldmatrix matrix i = lane/8: keys (i&1)*8 + lane%8 of the slice, 16-byte chunk 2*kk + (i>>1)
   const int k_key = slice * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
@@ -392,7 +395,7 @@ __device__ __forceinline__ void qk_issue_n(const RowBlockN<D> &rb, uint32_t kt, 
 #pragma unroll
   for (int kk = 0; kk < D / 16; ++kk) {
     uint32_t a[4];
-    ldsm_x4(kt + (kk >> 2) * (kTileKeys * 128) + k_row + ((((2 * kk) & 7) ^ k_x) << 4), a[0], a[1], a[2], a[3]);
+    ldsm_x4(kt + (kk >> 2) * (TK * 128) + k_row + ((((2 * kk) & 7) ^ k_x) << 4), a[0], a[1], a[2], a[3]);
     mma_bf16(s, a, rb.qb[kk][0], rb.qb[kk][1]);
   }
 }
@@ -543,7 +546,9 @@ template <int D, bool NARROW>
 __global__ void __launch_bounds__(kDenseThreads, 2)
 fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const ScanParams p) {
-  using LO = DenseLayout<D>;
+  constexpr int TK = NARROW ? narrow_tile_keys<D>() : kTileKeys;   // keys per tile
+  constexpr int U = TK / 64, KS = 16 * U;                          // 16-key sub-slices and keys per warp slice
+  using LO = DenseLayout<D, TK>;
   constexpr int C16 = D / 8;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -552,7 +557,7 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
-  const SeqWork w = seq_work(p, seq);
+  const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, R = p.R, n = w.n;
   const uint32_t full0 = base + LO::off_bar(stages, R), empty0 = full0 + 8u * stages;
@@ -569,7 +574,7 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   pdl_wait();                                                // z (and the zeroed header) come from earlier work
 
   if (warp == kConsumerWarps) {
-    if (lane == 0) produce_tiles<D, true, LO::kStage>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
+    if (lane == 0) produce_tiles<D, true, LO::kStage, TK>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
     return;
   }
 
@@ -596,27 +601,30 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       if (++stage == stages) { stage = 0; phase ^= 1u; }
       if (!ready) continue;
       const uint32_t kt = base + my_stage * LO::kStage;
-      const int key0 = t * kTileKeys + warp * 16;
-      st_total += min(16, max(0, n - key0));
-      if (key0 + 16 > n) {                                   // ragged tail: value rows past n may hold anything
-        for (int r = 0; r < 16; ++r)
+      const int key0 = t * TK + warp * KS;
+      st_total += min(KS, max(0, n - key0));
+      if (key0 + KS > n) {                                   // ragged tail: value rows past n may hold anything
+        for (int r = 0; r < KS; ++r)
           if (key0 + r >= n && lane < C16)
             *reinterpret_cast<uint4 *>(gen + my_stage * LO::kStage + LO::kKTile +
-                                       tile_off(warp * 16 + r, lane, kTileKeys)) = make_uint4(0, 0, 0, 0);
+                                       tile_off(warp * KS + r, lane, TK)) = make_uint4(0, 0, 0, 0);
         __syncwarp();
       }
       if constexpr (NARROW) {
-        float s[4];
-        uint32_t bh[2], bl[2];
-        qk_issue_n<D>(rb, kt, warp, lane, s);
-        const uint32_t fetch16 = weights_n<D, false>(rb, s, lane, key0, n, p.scale_log2, p.neg_T, bh, bl, l_lo, l_hi);
-        if (fetch16 != 0) value_product_n<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, bh, bl);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          float s[4];
+          uint32_t bh[2], bl[2];
+          qk_issue_n<D, TK>(rb, kt, warp * U + u, lane, s);
+          const uint32_t fetch16 = weights_n<D, false>(rb, s, lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh, bl, l_lo, l_hi);
+          if (fetch16 != 0) value_product_n<D, true, 0, TK>(o, kt + LO::kKTile, (warp * U + u) * 16, lane, bh, bl);
+        }
       } else {
         uint32_t ah[4], al[4];
         const uint32_t fetch16 = score_slice<D, false, 1>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
         if (fetch16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, ah, al);
       }
-      if (key0 + 16 > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
+      if (key0 + KS > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);
     }
@@ -979,6 +987,7 @@ __global__ void __launch_bounds__(kGatedThreads, 2)
 fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
                               const ScanParams p) {
   using LO = GatedNarrowLayout<D>;
+  constexpr int TK = LO::kTK, U = LO::kU, KS = 16 * U;       // keys per tile, sub-slices and keys per warp slice
   constexpr int C16 = D / 8;                                 // 16-byte chunks per value row
   constexpr int RPI = 32 / C16;                              // rows one warp-wide async copy covers
   constexpr int SW = kConsumerWarps;                         // scorer warps
@@ -989,7 +998,7 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
-  const SeqWork w = seq_work(p, seq);
+  const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
   const uint32_t full0 = base + LO::off_bar(stages, vr), empty0 = full0 + 8u * stages;
@@ -1011,13 +1020,13 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   pdl_wait();                                                // z (and the zeroed header) come from earlier work
 
   if (warp == SW + kConsumerWarps) {
-    if (lane == 0) produce_tiles<D, false, LO::kKTile>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
+    if (lane == 0) produce_tiles<D, false, LO::kKTile, TK>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
     return;
   }
 
   const bool scorer = warp < SW;
   const int sl = warp & 3;                                   // the slice of every tile this warp owns
-  constexpr int pentry = LO::kPEntry, pmask = 512;
+  constexpr int pentry = LO::kPEntry, pmask = U * 512;
   uint8_t *pring = gen + LO::off_pring(stages, vr) + sl * vr * pentry;
   const uint32_t vring = base + LO::off_vring(stages) + sl * vr * LO::kVSlice;
   const uint32_t vfull = vfull0 + 8u * sl * vr, vempty = vempty0 + 8u * sl * vr;
@@ -1033,7 +1042,7 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     const int page_mask = (1 << p.page_shift) - 1;
     const uint64_t vpol = policy_evict_first();
     // row-by-row fetch: lane covers 16-byte chunk (lane % C16) of rows (lane / C16) + RPI * i, swizzled as a box is
-    const uint32_t rdst0 = ((lane % C16) >> 3) * (16 * 128) + (lane / C16) * 128;
+    const uint32_t rdst0 = ((lane % C16) >> 3) * (KS * 128) + (lane / C16) * 128;
     const long long rsrc0 = (long long)(lane / C16) * p.v_stride_tok + (lane % C16) * 8;
     int stage = 0;
     uint32_t phase = 0;
@@ -1046,65 +1055,87 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       if (++vs == vr) { vs = 0; vwrapped = 1u; vphase ^= 1u; }
       {
         const bool ready = mbar_wait(full0 + 8u * my_stage, my_phase, dead);
-        const int key0 = k.t * kTileKeys + sl * 16;
-        uint32_t bh[2] = {0u, 0u}, bl[2] = {0u, 0u};
-        uint32_t fetch16 = 0;
+        const int key0 = k.t * TK + sl * KS;
+        uint32_t bh[U][2], bl[U][2];
+        uint32_t fetch = 0;                                  // bit 16 u + k: key k of sub-slice u is live for some row
+#pragma unroll
+        for (int u = 0; u < U; ++u) bh[u][0] = bh[u][1] = bl[u][0] = bl[u][1] = 0u;
         if (ready) {
-          float s[4];
-          qk_issue_n<D>(rb, base + my_stage * LO::kKTile, sl, lane, s);
+          float s[U][4];
+#pragma unroll
+          for (int u = 0; u < U; ++u) qk_issue_n<D, TK>(rb, base + my_stage * LO::kKTile, sl * U + u, lane, s[u]);
           __syncwarp();
           if (lane == 0) mbar_arrive(empty0 + 8u * my_stage); // the K slice is consumed: release the tile
-          fetch16 = weights_n<D, true>(rb, s, lane, key0, n, p.scale_log2, p.neg_T, bh, bl, l0, l1);
+#pragma unroll
+          for (int u = 0; u < U; ++u)
+            fetch |= weights_n<D, true>(rb, s[u], lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh[u], bl[u], l0, l1) << (16 * u);
         }
-        const bool whole = (key0 + 16 <= n) && (__popc(fetch16) >= p.box_min);
+        // a mostly-live sub-slice is cheaper to fetch whole (one TMA box per 64 channels) than row by row; rows nobody
+        // keeps then ride along under a zero weight.  Never past the sequence end: those rows may hold anything.
+        uint32_t whole = 0;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const uint32_t m = (fetch >> (16 * u)) & 0xffffu;
+          const bool wh = (key0 + 16 * u + 16 <= n) && (__popc(m) >= p.box_min);
+          whole |= wh ? (1u << u) : 0u;
+          st_fetched += wh ? 16 : __popc(m);
+        }
         {
-          const int nvalid = min(16, max(0, n - key0));
+          const int nvalid = min(KS, max(0, n - key0));
           st_total += nvalid;
-          st_fetched += whole ? 16 : __popc(fetch16);
-          st_skipped += (fetch16 == 0 && nvalid > 0) ? 1 : 0;
+          st_skipped += (fetch == 0 && nvalid > 0) ? 1 : 0;
         }
         if (!my_wrapped || mbar_wait(vempty + 8u * my_vs, my_vphase ^ 1u, dead)) {
+          // publish the slice: weights as the value product's B-operand registers, and the verdict
           uint8_t *pe = pring + my_vs * pentry;
-          *reinterpret_cast<uint4 *>(pe + lane * 16) = make_uint4(bh[0], bh[1], bl[0], bl[1]);
-          if (lane == 0) *reinterpret_cast<uint32_t *>(pe + pmask) = fetch16 | (whole ? 0x10000u : 0u);
+#pragma unroll
+          for (int u = 0; u < U; ++u)
+            *reinterpret_cast<uint4 *>(pe + u * 512 + lane * 16) = make_uint4(bh[u][0], bh[u][1], bl[u][0], bl[u][1]);
+          if (lane == 0) *reinterpret_cast<uint32_t *>(pe + pmask) = fetch;
           const uint32_t bar = vfull + 8u * my_vs;
-          if (fetch16 != 0u) {
-            int c_seq = seq, c_tok = key0;
+          const uint32_t vdst = vring + my_vs * LO::kVSlice;
+          if (whole) {
+            fence_proxy_async_smem();                        // the slot's earlier generic-proxy traffic, then TMA writes
+            __syncwarp();
+          }
+          bool rows = false;
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            const uint32_t m = (fetch >> (16 * u)) & 0xffffu;
+            if (m == 0u) continue;
+            int c_seq = seq, c_tok = key0 + 16 * u;
             if (p.paged) {
-              const int pg = p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)];
+              const int pg = p.page_table[(long long)seq * p.max_pages + (c_tok >> p.page_shift)];
               c_seq = min(max(pg, 0), p.num_pages - 1);
-              c_tok = key0 & page_mask;
+              c_tok &= page_mask;
             }
-            const uint32_t vdst = vring + my_vs * LO::kVSlice;
-            if (whole) {
-              fence_proxy_async_smem();                      // the slot's earlier generic-proxy traffic, then TMA writes
-              __syncwarp();
+            if ((whole >> u) & 1u) {
               if (lane == 0) {
-                mbar_expect_tx(bar, 16 * D * 2);
+                mbar_expect_tx_only(bar, 16 * D * 2);
                 const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
                 const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
                 const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
 #pragma unroll
-                for (int h = 0; h < D / 64; ++h) tma_load_4d(vdst + h * (16 * 128), &tmVs, bar, h * 64, c1, c2, c3, vpol);
+                for (int h = 0; h < D / 64; ++h)
+                  tma_load_4d(vdst + (h * KS + 16 * u) * 128, &tmVs, bar, h * 64, c1, c2, c3, vpol);
               }
             } else {
+              rows = true;
               const __nv_bfloat16 *src = p.v + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
                                          (long long)kvh * p.v_stride_head + rsrc0;
 #pragma unroll
               for (int i = 0; i < 16 / RPI; ++i) {
-                const int row = i * RPI + lane / C16;
-                const bool f = (fetch16 >> row) & 1u;
-                cp_async_16(vdst + rdst0 + i * (RPI * 128) + ((((lane % C16) ^ row) & 7) << 4), f ? src : p.v, f ? 16u : 0u);
+                const int row = i * RPI + lane / C16;        // row & 7 is the same within the sub-slice and the slice
+                const bool f = (m >> row) & 1u;
+                cp_async_16(vdst + rdst0 + (16 * u + i * RPI) * 128 + ((((lane % C16) ^ row) & 7) << 4), f ? src : p.v,
+                            f ? 16u : 0u);
                 src += (long long)RPI * p.v_stride_tok;
               }
-              cp_async_mbar_arrive(bar);                     // this lane's copies hold the phase open
-              __syncwarp();
-              if (lane == 0) mbar_arrive(bar);
             }
-          } else {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar);
           }
+          if (rows) cp_async_mbar_arrive(bar);               // this lane's copies hold the phase open
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar);
         }
       }
       const int c_done = k.c;
@@ -1131,10 +1162,12 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       if (landed) {
         const uint8_t *pe = pring + my * pentry;
         const uint32_t verdict = *reinterpret_cast<const uint32_t *>(pe + pmask);
-        if (verdict != 0u) {
-          const uint4 a = *reinterpret_cast<const uint4 *>(pe + lane * 16);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (((verdict >> (16 * u)) & 0xffffu) == 0u) continue;   // nobody keeps a key of this sub-slice
+          const uint4 a = *reinterpret_cast<const uint4 *>(pe + u * 512 + lane * 16);
           const uint32_t bh[2] = {a.x, a.y}, bl[2] = {a.z, a.w};
-          value_product_n<D, true, 0, 16>(o, vring + my * LO::kVSlice, 0, lane, bh, bl);
+          value_product_n<D, true, 0, KS>(o, vring + my * LO::kVSlice, 16 * u, lane, bh, bl);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(vempty + 8u * my);

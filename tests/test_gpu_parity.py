@@ -24,7 +24,7 @@ def test_config1_mha_dense_and_t16():
 
 
 @pytest.mark.parametrize("D", [64, 128])
-@pytest.mark.parametrize("n", [1, 63, 64, 65, 191, 192, 193, 255, 257, 1000])
+@pytest.mark.parametrize("n", [1, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 257, 1000])
 def test_edge_lengths(D, n):
     w = make_decode_workload(2, 4, 2, D, [n, max(1, n - 17)], seed=100 + n, device=DEV, poison_padding=True,
                              capacity=n + 70)
