@@ -371,7 +371,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
   p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
 
-  const dim3 grid(p.num_splits, g.Hkv, g.num_seqs);
+  // row-block kernels: kv heads on x (fastest), splits on y; stacked kernels: (row group, split) on x, heads on y
+  const dim3 grid = stacked ? dim3(p.num_splits, g.Hkv, g.num_seqs) : dim3(g.Hkv, p.num_splits, g.num_seqs);
   p.box_min = 13;
   if (stacked) {
     if (g.D == 128 && g.R >= 64) return launch_stacked_umma(mk, mv, p, grid, gated, st);

@@ -556,7 +556,8 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   uint8_t *gen = smem_raw + (base - raw);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
+  // kv heads fastest: CTAs that run together read the same tokens' rows, which sit side by side in memory
+  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
   const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, R = p.R, n = w.n;
@@ -778,7 +779,8 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   uint8_t *gen = smem_raw + (base - raw);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
+  // kv heads fastest: CTAs that run together read the same tokens' rows, which sit side by side in memory
+  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
   const SeqWork w = seq_work(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
@@ -997,7 +999,8 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   uint8_t *gen = smem_raw + (base - raw);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
+  // kv heads fastest: CTAs that run together read the same tokens' rows, which sit side by side in memory
+  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
   const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
