@@ -88,6 +88,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, bool &d
   dead = true;
   return false;
 }
+// The same with a non-suspending probe: a thread on a latency-critical hand-off polls instead of sleeping.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, bool &dead) {
+  if (dead) return false;
+  for (uint32_t i = 0; i < 16u * kWaitLimit; ++i)
+    if (mbar_test_wait(bar, parity)) return true;
+  dead = true;
+  return false;
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }

@@ -12,7 +12,7 @@
 
 namespace fold {
 
-constexpr int kMergeMaxWarps = 8;
+constexpr int kMergeMaxWarps = 16;
 
 struct MergeLevel {
   const float *slots;
@@ -46,51 +46,26 @@ __device__ __forceinline__ double pow2_double(int e) {       // 2^e, e in the no
 // nearest even; |result| < 2^61 / C.
 __device__ __forceinline__ long long to_grid(float g, double alpha) { return __double2ll_rn((double)g * alpha); }
 
-// grid (Hq, batch); block (32, W), W = blockDim.y <= kMergeMaxWarps chosen from the slot count.  One CTA
-// per (request, q head).  Lane x of every warp owns EPT = D / 32 consecutive elements of A (one vector load
-// per slot); warp y takes the slots y, y + W, ... of every level; lane 0 also carries L.  Two passes over
-// the (cache-resident) slots: the order-free maximum, then the integer sum; warps combine through
-// shared-memory integer atomics, which are order-free by construction.
+// One CTA of blockDim.x / 32 warps (at most kMergeMaxWarps) covers that many / W rows (a row = one (request, q head));
+// W in {1, 2, 4, 8, 16} warps share a row's slots (warp `sub` takes slots sub, sub + W, ... of every level).  Lane x owns EPT = D / 32
+// consecutive elements of A (one vector load per slot); lane 0 also carries L.  Two passes over the slots (the
+// second hits L1): the order-free maximum, then the integer sum.  The W warps of a row combine through staged
+// partials in shared memory: maxima by max, integer sums by integer addition, both exact, so neither the warp
+// count nor the slot order can change a bit.
 template <int EPT>
-__global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const MergeParams p) {
-  __shared__ unsigned s_max[129];
-  __shared__ unsigned long long s_sum[129];
-  __shared__ int s_flags;
+__global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const MergeParams p, const int W,
+                                                                         const long long n_rows) {
   constexpr int D = 32 * EPT;
-  const int h = blockIdx.x, b = blockIdx.y;
-  const int x = threadIdx.x, y = threadIdx.y, W = blockDim.y;
-  const int G = p.G, kvh = h / G;
-  const int tid = y * 32 + x;
-  const long long row = (long long)b * p.Hq + h;
+  __shared__ unsigned s_max[kMergeMaxWarps][D + 1];
+  __shared__ long long s_sum[kMergeMaxWarps][D + 1];
+  const int x = threadIdx.x & 31, wi = threadIdx.x >> 5;
+  const int sub = wi % W;
+  const long long row = (long long)blockIdx.x * ((blockDim.x >> 5) / W) + wi / W;
+  const bool active = row < n_rows;
+  const int b = active ? (int)(row / p.Hq) : 0, h = active ? (int)(row % p.Hq) : 0;
+  const int G = p.G, kvh = h / G, hg = h % G;
   pdl_wait();                                        // slots and z come from the kernels before
-  const float zrow = p.z[row];                       // requested early: only needed at the very end
-
-  for (int i = tid; i <= D; i += 32 * W) { s_max[i] = 0u; s_sum[i] = 0ull; }
-  if (tid == 0) s_flags = 0;
-
-  // per level: this lane's first A vector, the row's L element, the slot stride and count
-  const float *pa[kMaxLevels], *pl[kMaxLevels];
-  long long step[kMaxLevels];
-  int cnt[kMaxLevels];
-  unsigned C = 0;
-#pragma unroll
-  for (int l = 0; l < kMaxLevels; ++l) {
-    cnt[l] = 0; pa[l] = nullptr; pl[l] = nullptr; step[l] = 0;
-    if (l < p.n_levels) {
-      const MergeLevel &L = p.lv[l];
-      const int seq = b / L.stack;
-      int n = L.seqlens[seq];
-      n = n < 0 ? 0 : (n > L.max_seqlen ? L.max_seqlen : n);
-      cnt[l] = num_chunks_of(n);
-      C += cnt[l];
-      const int r = (b % L.stack) * G + (h % G);
-      const float *s0 = L.slots + (((long long)seq * p.Hkv + kvh) * L.max_slots + y) * L.slot_stride;
-      pa[l] = s0 + r * D + x * EPT;
-      pl[l] = s0 + L.rows * D + r;
-      step[l] = L.slot_stride * W;
-    }
-  }
-  const int clog2C = ceil_log2_u32(C);
+  const float zrow = active ? p.z[row] : 0.f;        // requested early: only needed at the very end
 
   auto load_vec = [](const float *a, float (&v)[EPT]) {
     if (EPT == 4) {
@@ -101,16 +76,31 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
       v[0] = t.x; v[1] = t.y;
     }
   };
+  // level l as this warp sees it: slot count, this lane's first A vector, the row's first L element, the step
+  auto level = [&](int l, int &cnt, const float *&a, const float *&q, long long &step) {
+    const MergeLevel &L = p.lv[l];
+    const int seq = b / L.stack;
+    int n = L.seqlens[seq];
+    n = n < 0 ? 0 : (n > L.max_seqlen ? L.max_seqlen : n);
+    cnt = active ? num_chunks_of(n) : 0;
+    const int r = (b % L.stack) * G + hg;
+    const float *s0 = L.slots + (((long long)seq * p.Hkv + kvh) * L.max_slots + sub) * L.slot_stride;
+    a = s0 + r * D + x * EPT;
+    q = s0 + L.rows * D + r;
+    step = L.slot_stride * W;
+  };
 
-  // pass 1: order-free maximum of |g| through the bit patterns
-  unsigned mx[EPT], mxl = 0u;
+  // pass 1: order-free maximum of |g| through the bit patterns; C = the number of terms
+  unsigned mx[EPT], mxl = 0u, C = 0;
 #pragma unroll
   for (int e = 0; e < EPT; ++e) mx[e] = 0u;
-#pragma unroll
-  for (int l = 0; l < kMaxLevels; ++l) {
-    const float *a = pa[l], *q = pl[l];
+#pragma unroll 1
+  for (int l = 0; l < p.n_levels; ++l) {
+    int cnt; const float *a, *q; long long step;
+    level(l, cnt, a, q, step);
+    C += cnt;
 #pragma unroll 4
-    for (int k = y; k < cnt[l]; k += W, a += step[l], q += step[l]) {
+    for (int k = sub; k < cnt; k += W, a += step, q += step) {
       float v[EPT];
       load_vec(a, v);
 #pragma unroll
@@ -118,17 +108,20 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
       if (x == 0) mxl = max(mxl, __float_as_uint(*q) & 0x7fffffffu);
     }
   }
-  __syncthreads();                                   // s_max / s_sum are zeroed
   if (W > 1) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) if (mx[e]) atomicMax(&s_max[x * EPT + e], mx[e]);
-    if (x == 0 && mxl) atomicMax(&s_max[D], mxl);
+    for (int e = 0; e < EPT; ++e) s_max[wi][e * 32 + x] = mx[e];
+    if (x == 0) s_max[wi][D] = mxl;
     __syncthreads();
+    const int w0 = wi - sub;
+    for (int o = 0; o < W; ++o) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) mx[e] = s_max[x * EPT + e];
-    mxl = s_max[D];
+      for (int e = 0; e < EPT; ++e) mx[e] = max(mx[e], s_max[w0 + o][e * 32 + x]);
+      mxl = max(mxl, s_max[w0 + o][D]);              // lanes other than 0 carry it along unused
+    }
   }
   mxl = __shfl_sync(0xffffffffu, mxl, 0);
+  const int clog2C = ceil_log2_u32(C);
 
   // pass 2: integer sums on the declared grid
   long long acc[EPT], accl = 0;
@@ -142,11 +135,12 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
   }
   const double alpha_l = pow2_double(grid_shift(mxl, clog2C));
   const bool fin_l = (mxl >> 23) != 255u;
-#pragma unroll
-  for (int l = 0; l < kMaxLevels; ++l) {
-    const float *a = pa[l], *q = pl[l];
+#pragma unroll 1
+  for (int l = 0; l < p.n_levels; ++l) {
+    int cnt; const float *a, *q; long long step;
+    level(l, cnt, a, q, step);
 #pragma unroll 4
-    for (int k = y; k < cnt[l]; k += W, a += step[l], q += step[l]) {
+    for (int k = sub; k < cnt; k += W, a += step, q += step) {
       float v[EPT];
       load_vec(a, v);
 #pragma unroll
@@ -156,16 +150,19 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
   }
   if (W > 1) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) if (acc[e]) atomicAdd(&s_sum[x * EPT + e], (unsigned long long)acc[e]);
-    if (x == 0 && accl) atomicAdd(&s_sum[D], (unsigned long long)accl);
+    for (int e = 0; e < EPT; ++e) s_sum[wi][e * 32 + x] = acc[e];
+    if (x == 0) s_sum[wi][D] = accl;
     __syncthreads();
-    if (y != 0) return;
+    if (sub != 0) return;
+    for (int o = 1; o < W; ++o) {
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) acc[e] = (long long)s_sum[x * EPT + e];
-    accl = (long long)s_sum[D];
+      for (int e = 0; e < EPT; ++e) acc[e] += s_sum[wi + o][e * 32 + x];
+      accl += s_sum[wi + o][D];
+    }
   }
+  if (!active) return;
 
-  // warp 0 finishes the row
+  // the row's first warp finishes it
   float Lf = fin_l ? (float)((double)accl * pow2_double(-grid_shift(mxl, clog2C))) : __int_as_float(0x7fc00000);
   Lf = __shfl_sync(0xffffffffu, Lf, 0);
   bool bad = false;

@@ -6,16 +6,20 @@
 // with the accumulators in tensor memory.  One CTA owns 128 query rows (M = 128) of one
 // (sequence, kv head) and walks the 64-key tiles of its canonical chunks:
 //
-//   producer warp   TMA: K and V tiles -> 3-stage shared-memory ring (same tiles as dense decode)
-//   MMA warp        S = Q K^T        (A = Q in smem, K-major;  B = K tile, K-major;  N = 64 keys)
-//                   O += P_hi V + P_lo V   (A = P in smem, K-major;  B = V tile, MN-major;  N = 128)
+//   producer warp   TMA: K and V tiles -> 6-stage shared-memory ring (same tiles as dense decode); the tiles come
+//                   from L2 (every row tile of a kv head reads them) and the ring has to cover that latency
+//   MMA warp        S = Q K^T        (A = Q in tensor memory;  B = K tile, K-major;  N = 64 keys)
+//                   O += P_hi V + P_lo V   (A = P in tensor memory;  B = V tile, MN-major;  N = 128)
 //   8 weight warps  two threads per query row (the row's TMEM lane; each takes 32 of the tile's 64 keys and
 //                   64 of the 128 channels): tcgen05.ld S, final weights 2^(s - Z) with the depth gate,
-//                   L in a register, two-term BF16 P -> smem
+//                   L in a register, two-term BF16 P -> tensor memory by tcgen05.st
 //
-// S is double-buffered in TMEM and P in shared memory, so the scores of tile t+1 are computed
-// while the weights of tile t are formed.  No maximum is tracked and nothing is rescaled: the
-// accumulator O is only ever added to.  At a chunk's end each thread reads its row of O from
+// Both A operands live in tensor memory (a row of A is a TMEM lane, two BF16 per 32-bit column), so the only
+// shared-memory traffic is the K and V tiles: with Q and P in shared memory the operand reads alone (112 KB per
+// tile) exceeded what the SM's shared memory delivers in the time the products take.  S is double-buffered, so
+// the scores of tile t+1 are computed while the weights of tile t are formed; P has one buffer (the value
+// product of tile t is over long before the weights of t+1 are ready).  No maximum is tracked and nothing is
+// rescaled: the accumulator O is only ever added to.  At a chunk's end each thread reads its row of O from
 // TMEM and writes it, with its L, to the chunk's slot.
 #pragma once
 
@@ -26,15 +30,14 @@ namespace fold {
 constexpr int kUmmaThreads = 10 * 32;                // producer, MMA, 8 weight warps
 constexpr int kUmmaWeightThreads = 8 * 32;
 constexpr int kUmmaRows = 128;                       // query rows per CTA (MMA M)
-constexpr int kUmmaStages = 3;
-constexpr int kUmmaTmemCols = 256;                   // S0 [0,64)  S1 [64,128)  O [128,256)
+constexpr int kUmmaStages = 6;
+constexpr int kUmmaTmemCols = 512;                   // S0 [0,64)  S1 [64,128)  O [128,256)  Q [256,320)  P_hi [320,352)  P_lo [352,384)
+constexpr int kUmmaColQ = 256, kUmmaColPhi = 320, kUmmaColPlo = 352;
 
 struct UmmaLayout {                                  // byte offsets from a 1 KB-aligned base
-  static constexpr int kQ = 0;                                   // [2 halves][128 rows][128 B], swizzled
-  static constexpr int kRing = 32768;                            // stages x (K tile 16 KB + V tile 16 KB)
+  static constexpr int kRing = 0;                                // stages x (K tile 16 KB + V tile 16 KB)
   static constexpr int kStage = 32768;
-  static constexpr int kP = kRing + kUmmaStages * kStage;        // 2 buffers x (hi 16 KB + lo 16 KB)
-  static constexpr int kBar = kP + 2 * 32768;
+  static constexpr int kBar = kRing + kUmmaStages * kStage;
   static constexpr int kLbuf = kBar + 256;                       // 128 floats: the second half-row's share of L
   static constexpr int kTotal = kLbuf + 512 + 1024;              // + alignment slack
 };
@@ -52,16 +55,41 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem], BF16 inputs, FP32 accumulate; issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// D[tmem] (+)= A * B, BF16 inputs, FP32 accumulate, issued by one thread, with the A operand in tensor memory (row r of A = TMEM lane r, K elements packed two per column).
+// The B descriptor comes as two 32-bit words: the issuing thread's instruction stream is the critical path of
+// the whole CTA, and stepping a descriptor is then one 32-bit add on the low word.
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 bd, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
       : "memory");
 }
+__device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                             bool accumulate) {
+  if (accumulate) umma_bf16_ta<true>(d_tmem, a_tmem, b_lo, b_hi, idesc);
+  else umma_bf16_ta<false>(d_tmem, a_tmem, b_lo, b_hi, idesc);
+}
+// Low and high words of a shared-memory matrix descriptor (128-byte swizzle, version 1); offsets in bytes.
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr, uint32_t lbo) {
+  return ((smem_addr >> 4) & 0x3fffu) | (((lbo >> 4) & 0x3fffu) << 16);
+}
+__host__ __device__ constexpr uint32_t umma_desc_hi(uint32_t sbo) {
+  return ((sbo >> 4) & 0x3fffu) | (1u << 14) | (2u << 29);
+}
+// 16 / 32 consecutive 32-bit columns of this thread's TMEM lane, written from registers.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // 32 consecutive FP32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
@@ -80,11 +108,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// Shared-memory matrix descriptor (128-byte swizzle, descriptor version 1).  Offsets in bytes.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
-  return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)((lbo >> 4) & 0x3fffu) << 16) |
-         ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46) | (2ull << 61);
-}
 // Instruction descriptor: FP32 accumulate, BF16 A and B, M = 128.
 __host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
@@ -110,47 +133,58 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   if (split >= w.n_chunks) return;
   const int R = p.R, n = w.n;
 
-  // barriers (8 bytes each): kv_full[3] kv_empty[3] s_full[2] s_empty[2] p_full[2] p_empty[2] o_full o_empty
+  // barriers (8 bytes each): kv_full[stages] pv_done[stages] s_full[2] s_empty[2] p_full o_empty.
+  // pv_done[stage] completes when the value product of the tile in `stage` has: it frees the stage for the producer,
+  // P for the weight warps, and at a chunk's end says that O is final -- one commit per tile serves all three (a
+  // commit holds the issuing thread for on the order of a hundred cycles).
   const uint32_t bar = base + LO::kBar;
-  const uint32_t kv_full = bar, kv_empty = bar + 24, s_full = bar + 48, s_empty = bar + 64, p_full = bar + 80,
-                 p_empty = bar + 96, o_full = bar + 112, o_empty = bar + 120, tmem_slot = bar + 128;
+  const uint32_t kv_full = bar, pv_done = bar + 8 * kUmmaStages, s_full = bar + 16 * kUmmaStages, s_empty = s_full + 16,
+                 p_full = s_full + 32, o_empty = s_full + 40, tmem_slot = bar + 192;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kUmmaStages; ++s) { mbar_init(kv_full + 8u * s, 1); mbar_init(kv_empty + 8u * s, 1); }
+    for (int s = 0; s < kUmmaStages; ++s) { mbar_init(kv_full + 8u * s, 1); mbar_init(pv_done + 8u * s, 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(s_full + 8u * b, 1);
-      mbar_init(s_empty + 8u * b, kUmmaWeightThreads);
-      mbar_init(p_full + 8u * b, kUmmaWeightThreads);
-      mbar_init(p_empty + 8u * b, 1);
+      mbar_init(s_empty + 8u * b, kUmmaWeightThreads / 32);      // one arrival per weight warp
     }
-    mbar_init(o_full, 1);
-    mbar_init(o_empty, kUmmaWeightThreads);
+    mbar_init(p_full, kUmmaWeightThreads / 32);
+    mbar_init(o_empty, kUmmaWeightThreads / 32);
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(tmem_slot, kUmmaTmemCols);
   pdl_launch_dependents();
   pdl_wait();                                                // q and z come from earlier work
 
-  // the weight warps stage their query rows: row r of the tile -> [half][r][128 B], 128-byte swizzle
+  tc_fence_before();
+  __syncthreads();                                           // barriers initialised, TMEM allocated
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(gen + LO::kBar + 192);
+
+  // the weight warps put their query rows into tensor memory: row r of the tile = lane r, channel pairs = columns
   const int row = (warp & 3) * 32 + lane;                    // TMEM lane == query row of the tile
   const int ch = warp >= 6 ? 1 : 0;                          // which half of the tile's keys / of the channels
   const int r_glob = rt * kUmmaRows + row;
+  const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
   float z_row = 0.f;
   if (warp >= 2) {
     const bool valid_row = r_glob < R;
     const int req = seq * p.stack + r_glob / p.G, head = kvh * p.G + r_glob % p.G;
     const uint4 *qrow = reinterpret_cast<const uint4 *>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h);
 #pragma unroll
-    for (int c = ch * 8; c < ch * 8 + 8; ++c) {
-      const uint4 v = valid_row ? qrow[c] : make_uint4(0, 0, 0, 0);
-      *reinterpret_cast<uint4 *>(gen + LO::kQ + tile_off(row, c, kUmmaRows)) = v;
+    for (int c = 0; c < 2; ++c) {                            // 16 columns = 32 channels at a time
+      uint32_t qw[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 v = valid_row ? qrow[ch * 8 + c * 4 + i] : make_uint4(0, 0, 0, 0);
+        qw[4 * i] = v.x; qw[4 * i + 1] = v.y; qw[4 * i + 2] = v.z; qw[4 * i + 3] = v.w;
+      }
+      tmem_st16(lane_addr + kUmmaColQ + ch * 32 + c * 16, qw);
     }
-    if (valid_row) z_row = p.z[(long long)req * p.Hq + head];
-    fence_proxy_async_smem();
+    tmem_st_wait();
+    z_row = valid_row ? p.z[(long long)req * p.Hq + head] : INFINITY;
   }
   tc_fence_before();
-  __syncthreads();
+  __syncthreads();                                           // Q is in tensor memory
   tc_fence_after();
-  const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(gen + LO::kBar + 128);
 
   bool dead = false;
   if (warp == 0) {
@@ -158,102 +192,120 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     if (lane == 0) {
       ScanParams pp = p;
       pp.stages = kUmmaStages;
-      produce_tiles<D, true, LO::kStage>(&tmK, &tmV, pp, w, split, kvh, seq, base + LO::kRing, kv_full, kv_empty);
+      produce_tiles<D, true, LO::kStage>(&tmK, &tmV, pp, w, split, kvh, seq, base + LO::kRing, kv_full, pv_done);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loop and its waits in step; one lane issues.  Everything an MMA takes as operand
+    // (tensor-memory addresses, descriptor words) is then the same in every lane, which lets it be kept in
+    // uniform registers instead of being moved there before every instruction.
+    {
+      const bool leader = lane == 0;
+      const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+      SeqWork wu;
+      wu.n = __shfl_sync(0xffffffffu, w.n, 0); wu.n_tiles = __shfl_sync(0xffffffffu, w.n_tiles, 0);
+      wu.ctiles = __shfl_sync(0xffffffffu, w.ctiles, 0); wu.n_chunks = __shfl_sync(0xffffffffu, w.n_chunks, 0);
       constexpr uint32_t idesc_qk = umma_idesc(64, 0), idesc_pv = umma_idesc(128, 1);
-      const uint32_t q_s = base + LO::kQ;
+      const uint32_t ring_lo = umma_desc_lo(base + LO::kRing, 0);
       auto issue_qk = [&](int it, int stage) {               // S[it & 1] = Q K^T for the tile in `stage`
         const int b = it & 1;
         if (!mbar_wait(kv_full + 8u * stage, (uint32_t)((it / kUmmaStages) & 1), dead)) return;
         if (it >= 2 && !mbar_wait(s_empty + 8u * b, (uint32_t)(((it >> 1) - 1) & 1), dead)) return;
         tc_fence_after();
-        const uint32_t k_s = base + LO::kRing + stage * LO::kStage;
+        // K tile [2 halves][64 keys][128 B]: K step kk = 32 bytes along the row, half kk / 4; LBO 16
+        const uint32_t k_lo = ring_lo + ((uint32_t)(stage * LO::kStage) >> 4) + (1u << 16);
+        const uint32_t s_t = tm + b * 64;
+        if (leader) {
+          umma_bf16_ta<false>(s_t, tm + kUmmaColQ, k_lo, umma_desc_hi(1024), idesc_qk);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2), sub = (kk & 3) * 32;
-          umma_bf16(tmem + b * 64, umma_desc(q_s + off * (kUmmaRows * 128) + sub, 16, 1024),
-                    umma_desc(k_s + off * (kTileKeys * 128) + sub, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+          for (int kk = 1; kk < D / 16; ++kk)
+            umma_bf16_ta<true>(s_t, tm + kUmmaColQ + kk * 8, k_lo + (((kk >> 2) * (kTileKeys * 128) + (kk & 3) * 32) >> 4),
+                               umma_desc_hi(1024), idesc_qk);
+          tc_commit(s_full + 8u * b);
         }
-        tc_commit(s_full + 8u * b);
+        __syncwarp();
       };
       int it = 0, chunk_i = 0;
-      TileCursor k = cursor_begin(w, split);
-      if (cursor_valid(k, w)) issue_qk(0, 0);
+      TileCursor k = cursor_begin(wu, split);
+      if (cursor_valid(k, wu)) issue_qk(0, 0);
       bool first_of_chunk = true;
-      while (cursor_valid(k, w) && !dead) {
-        const int stage = it % kUmmaStages, b = it & 1;
+      while (cursor_valid(k, wu) && !dead) {
+        const int stage = it % kUmmaStages;
         TileCursor kn = k;
-        const bool chunk_ends = cursor_next(kn, w, p.num_splits);
-        if (cursor_valid(kn, w)) issue_qk(it + 1, (it + 1) % kUmmaStages);
+        const bool chunk_ends = cursor_next(kn, wu, p.num_splits);
+        if (cursor_valid(kn, wu)) issue_qk(it + 1, (it + 1) % kUmmaStages);
         // O += P V for tile `it`
         if (first_of_chunk && chunk_i > 0 && !mbar_wait(o_empty, (uint32_t)((chunk_i - 1) & 1), dead)) break;
-        if (!mbar_wait(p_full + 8u * b, (uint32_t)((it >> 1) & 1), dead)) break;
+        if (!mbar_wait(p_full, (uint32_t)(it & 1), dead)) break;
         tc_fence_after();
-        const uint32_t v_s = base + LO::kRing + stage * LO::kStage + 16384;
-        const uint32_t p_s = base + LO::kP + b * 32768;
+        // V tile [2 halves][64 keys][128 B], MN-major: 16 keys = 2048 bytes per K step, halves 8192 bytes apart (LBO)
+        const uint32_t v_lo = ring_lo + ((uint32_t)(stage * LO::kStage + 16384) >> 4) + ((8192u >> 4) << 16);
+        if (leader) {
+          umma_bf16_ta(tm + 128, tm + kUmmaColPhi, v_lo, umma_desc_hi(1024), idesc_pv, !first_of_chunk);
 #pragma unroll
-        for (int term = 0; term < 2; ++term)
-#pragma unroll
-          for (int j = 0; j < kTileKeys / 16; ++j)
-            umma_bf16(tmem + 128, umma_desc(p_s + term * 16384 + j * 32, 16, 1024),
-                      umma_desc(v_s + j * 2048, 8192, 1024), idesc_pv, (first_of_chunk && term == 0 && j == 0) ? 0u : 1u);
-        tc_commit(p_empty + 8u * b);
-        tc_commit(kv_empty + 8u * stage);
-        if (chunk_ends) { tc_commit(o_full); ++chunk_i; }
+          for (int i = 1; i < 2 * (kTileKeys / 16); ++i) {
+            const int term = i / (kTileKeys / 16), j = i % (kTileKeys / 16);
+            umma_bf16_ta<true>(tm + 128, tm + (term ? kUmmaColPlo : kUmmaColPhi) + j * 8, v_lo + j * (2048 >> 4),
+                               umma_desc_hi(1024), idesc_pv);
+          }
+          tc_commit(pv_done + 8u * stage);
+        }
+        __syncwarp();
+        if (chunk_ends) ++chunk_i;
         first_of_chunk = chunk_ends;
         k = kn;
         ++it;
       }
-      if (dead) atomicOr(&p.hdr->wait_timeouts, 8u);
+      if (dead && leader) atomicOr(&p.hdr->wait_timeouts, 8u);
     }
   } else {
     // ------------------------------------------------------------ weight warps: one query row per thread
     const bool valid_row = r_glob < R;
-    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     float l_row = 0.f;
     int it = 0, chunk_i = 0;
     for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w); ++it) {
       const int b = it & 1, stage = it % kUmmaStages;
       const int key_base = k.t * kTileKeys;
       uint32_t ph[16], pl[16];                               // this thread's 32 weights, BF16 pairs: hi and lo terms
-      const bool have_s = mbar_wait(s_full + 8u * b, (uint32_t)((it >> 1) & 1), dead);
+      // the tcgen05 loads and stores below are warp-wide: the warp takes them together or not at all
+      const bool have_s = __all_sync(0xffffffffu, mbar_wait(s_full + 8u * b, (uint32_t)((it >> 1) & 1), dead));
       if (have_s) {
         tc_fence_after();
         float s[32];
         tmem_ld32(lane_addr + b * 64 + ch * 32, s);
+        // rows beyond R carry z = +inf, so their weights vanish by themselves; keys beyond n only occur in a tail tile
+        const int key_lim = n - (key_base + ch * 32);        // this thread's keys j < key_lim exist
+        auto weights = [&](auto tail) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          float pw[2], pm[2];
+          for (int j = 0; j < 32; j += 2) {
+            float pw[2], pm[2];
 #pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const bool ok = valid_row && (key_base + ch * 32 + j + e) < n;
-            const float x = ok ? fmaf(s[j + e], p.scale_log2, -z_row) : -INFINITY;
-            const bool live = GATED ? (x >= p.neg_T) : ok;
-            pw[e] = ex2_approx(x);
-            pm[e] = live ? pw[e] : 0.f;
+            for (int e = 0; e < 2; ++e) {
+              float x = fmaf(s[j + e], p.scale_log2, -z_row);
+              if (decltype(tail)::value) x = (j + e) < key_lim ? x : -INFINITY;
+              pw[e] = ex2_approx(x);
+              pm[e] = (!GATED || x >= p.neg_T) ? pw[e] : 0.f;
+            }
+            const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
+            const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
+            const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
+            const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
+            l_row += ((h0 + g0) + (pw[0] - pm[0])) + ((h1 + g1) + (pw[1] - pm[1]));
+            ph[j / 2] = hi2;
+            pl[j / 2] = lo2;
           }
-          const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
-          const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
-          const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
-          const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
-          l_row += ((h0 + g0) + (pw[0] - pm[0])) + ((h1 + g1) + (pw[1] - pm[1]));
-          ph[j / 2] = hi2;
-          pl[j / 2] = lo2;
-        }
+        };
+        if (key_lim >= 32) weights(std::false_type{}); else weights(std::true_type{});
         tc_fence_before();
       }
-      mbar_arrive(s_empty + 8u * b);                         // S[b] may be overwritten
-      if (it < 2 || mbar_wait(p_empty + 8u * b, (uint32_t)(((it >> 1) - 1) & 1), dead)) {
-        uint8_t *p_hi = gen + LO::kP + b * 32768, *p_lo = p_hi + 16384;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {                        // 8 keys = one 16-byte chunk, swizzled by the row
-          const uint32_t off = row * 128 + (((ch * 4 + c) ^ (row & 7)) << 4);
-          *reinterpret_cast<uint4 *>(p_hi + off) = make_uint4(ph[4 * c], ph[4 * c + 1], ph[4 * c + 2], ph[4 * c + 3]);
-          *reinterpret_cast<uint4 *>(p_lo + off) = make_uint4(pl[4 * c], pl[4 * c + 1], pl[4 * c + 2], pl[4 * c + 3]);
-        }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_empty + 8u * b);          // S[b] may be overwritten
+      // P is free once the value product of the tile before has completed
+      if (__all_sync(0xffffffffu, it < 1 || mbar_wait(pv_done + 8u * ((it - 1) % kUmmaStages),
+                                                        (uint32_t)(((it - 1) / kUmmaStages) & 1), dead))) {
+        tmem_st16(lane_addr + kUmmaColPhi + ch * 16, ph);    // this thread's 32 keys = 16 columns of its lane
+        tmem_st16(lane_addr + kUmmaColPlo + ch * 16, pl);
+        tmem_st_wait();
         if (key_base + kTileKeys > n) {                      // ragged tail: value rows past n may hold anything
           const int tw = threadIdx.x - 64;
           for (int i = tw; i < kTileKeys * 16; i += kUmmaWeightThreads) {
@@ -262,17 +314,19 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
               *reinterpret_cast<uint4 *>(gen + LO::kRing + stage * LO::kStage + 16384 + tile_off(vr_, c16, kTileKeys)) =
                   make_uint4(0, 0, 0, 0);
           }
+          fence_proxy_async_smem();                          // generic writes, then tensor-core (async proxy) reads
         }
-        fence_proxy_async_smem();                            // generic writes, then tensor-core (async proxy) reads
+        tc_fence_before();
       }
-      mbar_arrive(p_full + 8u * b);
+      __syncwarp();                                          // every lane's writes and proxy fence are done
+      if (lane == 0) mbar_arrive(p_full);
       const int c_done = k.c;
       if (cursor_next(k, w, p.num_splits)) {
         // chunk end: this thread's half of its row of O, and the row's L, go to the chunk's slot
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
         float *lbuf = reinterpret_cast<float *>(gen + LO::kLbuf);
         if (ch == 1) lbuf[row] = l_row;
-        if (mbar_wait(o_full, (uint32_t)(chunk_i & 1), dead)) {
+        if (__all_sync(0xffffffffu, mbar_wait(pv_done + 8u * stage, (uint32_t)((it / kUmmaStages) & 1), dead))) {
           tc_fence_after();
 #pragma unroll 1
           for (int q4 = ch * 2; q4 < ch * 2 + 2; ++q4) {
@@ -286,7 +340,8 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
           }
           tc_fence_before();
         }
-        mbar_arrive(o_empty);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(o_empty);
         asm volatile("bar.sync 1, %0;" ::"n"(kUmmaWeightThreads) : "memory");   // both halves of every row are in
         if (ch == 0 && valid_row) slot[(long long)R * D + r_glob] = l_row + lbuf[row];
         asm volatile("bar.sync 1, %0;" ::"n"(kUmmaWeightThreads) : "memory");   // lbuf may be rewritten
