@@ -274,6 +274,25 @@ int launch_stacked_umma(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+// More than 128 stacked rows: one CTA per (split, pair of 128-row tiles); the two tiles alternate on the tensor pipe.
+int launch_stacked_pair(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, bool gated,
+                        cudaStream_t st) {
+  p.stages = kPairStages;
+  p.vr = 0;
+  grid.x *= (p.R + kPairRows - 1) / kPairRows;
+  static int configured_g[64] = {0}, configured_d[64] = {0};
+  cudaError_t rc;
+  if (gated) {
+    if (int e = opt_in_smem(fold_scan_stacked_pair_kernel<true>, configured_g)) return e;
+    rc = launch_pdl(fold_scan_stacked_pair_kernel<true>, grid, dim3(kPairThreads), PairLayout::kTotal, st, mk, mv, p);
+  } else {
+    if (int e = opt_in_smem(fold_scan_stacked_pair_kernel<false>, configured_d)) return e;
+    rc = launch_pdl(fold_scan_stacked_pair_kernel<false>, grid, dim3(kPairThreads), PairLayout::kTotal, st, mk, mv, p);
+  }
+  if (rc != cudaSuccess) return FOLD_ECUDA;
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 // Gated scan: value slots hold rows whose requests can only be issued after scoring, so shared
 // memory is split between the key ring and the value slots of each slice.
 template <int D>
@@ -327,7 +346,7 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   const int n = a->kv.max_seqlen;
   const int max_chunks = num_chunks_of(n) > 0 ? num_chunks_of(n) : 1;
   if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
-  const long long units = (long long)g.num_seqs * g.Hkv * ((g.R + 127) / 128);
+  const long long units = (long long)g.num_seqs * g.Hkv * (g.R > 128 ? (g.R + 255) / 256 : 1);   // CTAs per split
   const int tiles_unit = max_chunks * (chunk_keys_of(n) / tile_keys);
   int s = tiles_unit / 32;
   s = s < 1 ? 1 : (s > max_chunks ? max_chunks : s);
@@ -375,6 +394,7 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const dim3 grid = stacked ? dim3(p.num_splits, g.Hkv, g.num_seqs) : dim3(g.Hkv, p.num_splits, g.num_seqs);
   p.box_min = 13;
   if (stacked) {
+    if (g.D == 128 && g.R > kUmmaRows) return launch_stacked_pair(mk, mv, p, grid, gated, st);
     if (g.D == 128 && g.R >= 64) return launch_stacked_umma(mk, mv, p, grid, gated, st);
     return g.D == 128 ? launch_stacked<128>(mk, mv, p, grid, gated, st) : launch_stacked<64>(mk, mv, p, grid, gated, st);
   }

@@ -368,4 +368,269 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Two row tiles per CTA (more than 128 stacked rows).  Both tiles (groups a and b, 128 rows each) share the CTA's
+// K and V tiles, and their products alternate on the tensor pipe: while the weight warps of one group turn S into P,
+// the pipe runs the other group's value product and next scores.  Per group S (64 columns) is overwritten in place
+// by P (each thread writes P_hi and P_lo over the 32 score columns it has just read), so no buffer is ever waited
+// for: the in-order pipe runs the scores of tile t+1 only after the value product of tile t has read P.
+//   tensor memory (512 columns): S/P_a [0,64)  S/P_b [64,128)  O_a [128,256)  O_b [256,384)  Q_a [384,448)  Q_b [448,512)
+constexpr int kPairThreads = (2 + 16) * 32;          // producer, MMA, 2 x 8 weight warps
+constexpr int kPairRows = 2 * kUmmaRows;
+constexpr int kPairStages = 6;
+
+struct PairLayout {                                  // byte offsets from a 1 KB-aligned base
+  static constexpr int kRing = 0;
+  static constexpr int kStage = 32768;
+  static constexpr int kBar = kRing + kPairStages * kStage;
+  static constexpr int kLbuf = kBar + 256;                       // 2 x 128 floats: the second half-row's share of L
+  static constexpr int kTotal = kLbuf + 1024 + 1024;
+};
+
+template <bool GATED>
+__global__ void __launch_bounds__(kPairThreads, 1)
+fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                              const ScanParams p) {
+  constexpr int D = 128;
+  using LO = PairLayout;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row_pairs = (p.R + kPairRows - 1) / kPairRows;
+  const int rp = blockIdx.x % row_pairs, split = blockIdx.x / row_pairs;
+  const int kvh = blockIdx.y, seq = blockIdx.z;
+  const SeqWork w = seq_work(p, seq);
+  if (split >= w.n_chunks) return;
+  const int R = p.R, n = w.n;
+
+  // barriers (8 bytes each): kv_full[stages]  pv_done[stages]  s_full[2]  p_full[2]  o_empty[2]
+  // pv_done[stage]: both groups' value products of the tile in `stage` have completed (frees the stage; at a
+  // chunk's end, O is final).
+  const uint32_t bar = base + LO::kBar;
+  const uint32_t kv_full = bar, pv_done = bar + 8 * kPairStages, s_full = bar + 16 * kPairStages, p_full = s_full + 16,
+                 o_empty = s_full + 32, tmem_slot = bar + 192;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(kv_full + 8u * s, 1); mbar_init(pv_done + 8u * s, 1); }
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(s_full + 8u * g, 1);
+      mbar_init(p_full + 8u * g, 8);                         // one arrival per weight warp of the group
+      mbar_init(o_empty + 8u * g, 8);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, 512);
+  pdl_launch_dependents();
+  pdl_wait();                                                // q and z come from earlier work
+  tc_fence_before();
+  __syncthreads();                                           // barriers initialised, TMEM allocated
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(gen + LO::kBar + 192);
+
+  // weight warps 2..17: group g, key/channel half ch, TMEM lane quarter warp % 4
+  const int wg = warp - 2;
+  const int g = wg >> 3, ch = (wg >> 2) & 1;
+  const int row = (warp & 3) * 32 + lane;                    // TMEM lane == query row of the group's tile
+  const int r_glob = rp * kPairRows + g * kUmmaRows + row;
+  const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+  const uint32_t col_s = g * 64, col_o = 128 + g * 128, col_q = 384 + g * 64;
+  float z_row = 0.f;
+  if (warp >= 2) {
+    const bool valid_row = r_glob < R;
+    const int req = seq * p.stack + r_glob / p.G, head = kvh * p.G + r_glob % p.G;
+    const uint4 *qrow = reinterpret_cast<const uint4 *>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h);
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {                            // 16 columns = 32 channels at a time
+      uint32_t qw[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 v = valid_row ? qrow[ch * 8 + c * 4 + i] : make_uint4(0, 0, 0, 0);
+        qw[4 * i] = v.x; qw[4 * i + 1] = v.y; qw[4 * i + 2] = v.z; qw[4 * i + 3] = v.w;
+      }
+      tmem_st16(lane_addr + col_q + ch * 32 + c * 16, qw);
+    }
+    tmem_st_wait();
+    z_row = valid_row ? p.z[(long long)req * p.Hq + head] : INFINITY;
+  }
+  tc_fence_before();
+  __syncthreads();                                           // Q is in tensor memory
+  tc_fence_after();
+
+  bool dead = false;
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0) {
+      ScanParams pp = p;
+      pp.stages = kPairStages;
+      produce_tiles<D, true, LO::kStage>(&tmK, &tmV, pp, w, split, kvh, seq, base + LO::kRing, kv_full, pv_done);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (the warp walks in step, one lane issues)
+    const bool leader = lane == 0;
+    const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+    constexpr uint32_t idesc_qk = umma_idesc(64, 0), idesc_pv = umma_idesc(128, 1);
+    const uint32_t ring_lo = umma_desc_lo(base + LO::kRing, 0);
+    // S_g = Q_g K^T for the tile in `stage` (K tile [2 halves][64 keys][128 B]: K step kk = 32 bytes along the row)
+    auto issue_qk = [&](int gg, int stage) {
+      const uint32_t k_lo = ring_lo + ((uint32_t)(stage * LO::kStage) >> 4) + (1u << 16);
+      if (leader) {
+        umma_bf16_ta<false>(tm + gg * 64, tm + 384 + gg * 64, k_lo, umma_desc_hi(1024), idesc_qk);
+#pragma unroll
+        for (int kk = 1; kk < D / 16; ++kk)
+          umma_bf16_ta<true>(tm + gg * 64, tm + 384 + gg * 64 + kk * 8,
+                             k_lo + (((kk >> 2) * (kTileKeys * 128) + (kk & 3) * 32) >> 4), umma_desc_hi(1024), idesc_qk);
+        tc_commit(s_full + 8u * gg);
+      }
+      __syncwarp();
+    };
+    // O_g += P_g V for the tile in `stage`; thread ch of a row holds keys ch*32.. : P_hi at its columns +0, P_lo at +16
+    auto issue_pv = [&](int gg, int stage, bool accumulate) {
+      const uint32_t v_lo = ring_lo + ((uint32_t)(stage * LO::kStage + 16384) >> 4) + ((8192u >> 4) << 16);
+      if (leader) {
+#pragma unroll
+        for (int i = 0; i < 2 * (kTileKeys / 16); ++i) {
+          const int term = i / (kTileKeys / 16), j = i % (kTileKeys / 16);       // keys 16 j ..: thread half j / 2
+          const uint32_t a = tm + gg * 64 + (j >> 1) * 32 + term * 16 + (j & 1) * 8;
+          if (i == 0) umma_bf16_ta(tm + 128 + gg * 128, a, v_lo, umma_desc_hi(1024), idesc_pv, accumulate);
+          else umma_bf16_ta<true>(tm + 128 + gg * 128, a, v_lo + j * (2048 >> 4), umma_desc_hi(1024), idesc_pv);
+        }
+      }
+      __syncwarp();
+    };
+    int it = 0, chunk_i = 0;
+    TileCursor k = cursor_begin(w, split);
+    if (cursor_valid(k, w) && mbar_wait(kv_full, 0u, dead)) {
+      tc_fence_after();
+      issue_qk(0, 0);
+      issue_qk(1, 0);
+    }
+    bool first_of_chunk = true;
+    while (cursor_valid(k, w) && !dead) {
+      const int stage = it % kPairStages, nstage = (it + 1) % kPairStages;
+      TileCursor kn = k;
+      const bool chunk_ends = cursor_next(kn, w, p.num_splits);
+      const bool more = cursor_valid(kn, w);
+      if (more && !mbar_wait(kv_full + 8u * nstage, (uint32_t)(((it + 1) / kPairStages) & 1), dead)) break;
+#pragma unroll
+      for (int gg = 0; gg < 2; ++gg) {
+        if (first_of_chunk && chunk_i > 0 && !mbar_wait(o_empty + 8u * gg, (uint32_t)((chunk_i - 1) & 1), dead)) break;
+        if (!mbar_wait(p_full + 8u * gg, (uint32_t)(it & 1), dead)) break;
+        tc_fence_after();
+        issue_pv(gg, stage, !first_of_chunk);
+        if (gg == 1) {
+          if (leader) tc_commit(pv_done + 8u * stage);
+          __syncwarp();
+        }
+        if (more) issue_qk(gg, nstage);
+      }
+      if (chunk_ends) ++chunk_i;
+      first_of_chunk = chunk_ends;
+      k = kn;
+      ++it;
+    }
+    if (dead && leader) atomicOr(&p.hdr->wait_timeouts, 8u);
+  } else {
+    // ------------------------------------------------------------ weight warps: two threads per query row
+    const bool valid_row = r_glob < R;
+    float l_row = 0.f;
+    int it = 0;
+    for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w); ++it) {
+      const int stage = it % kPairStages;
+      const int key_base = k.t * kTileKeys;
+      // the tcgen05 loads and stores below are warp-wide: the warp takes them together or not at all
+      if (__all_sync(0xffffffffu, mbar_wait(s_full + 8u * g, (uint32_t)(it & 1), dead))) {
+        tc_fence_after();
+        float s[32];
+        uint32_t ph[16], pl[16];                             // this thread's 32 weights, BF16 pairs: hi and lo terms
+        tmem_ld32(lane_addr + col_s + ch * 32, s);
+        // rows beyond R carry z = +inf, so their weights vanish by themselves; keys beyond n only occur in a tail tile
+        const int key_lim = n - (key_base + ch * 32);        // this thread's keys j < key_lim exist
+        auto weights = [&](auto tail) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float pw[2], pm[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              float x = fmaf(s[j + e], p.scale_log2, -z_row);
+              if (decltype(tail)::value) x = (j + e) < key_lim ? x : -INFINITY;
+              pw[e] = ex2_approx(x);
+              pm[e] = (!GATED || x >= p.neg_T) ? pw[e] : 0.f;
+            }
+            const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
+            const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
+            const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
+            const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
+            l_row += ((h0 + g0) + (pw[0] - pm[0])) + ((h1 + g1) + (pw[1] - pm[1]));
+            ph[j / 2] = hi2;
+            pl[j / 2] = lo2;
+          }
+        };
+        if (key_lim >= 32) weights(std::false_type{}); else weights(std::true_type{});
+        // P over the scores this thread has just read: P_hi in the first 16 of its 32 columns, P_lo in the rest
+        tmem_st16(lane_addr + col_s + ch * 32, ph);
+        tmem_st16(lane_addr + col_s + ch * 32 + 16, pl);
+        tmem_st_wait();
+        if (g == 0 && key_base + kTileKeys > n) {            // ragged tail: value rows past n may hold anything
+          const int tw = threadIdx.x - 64;                   // group a's 256 threads clear them for both groups
+          for (int i = tw; i < kTileKeys * 16; i += 256) {
+            const int vr_ = i >> 4, c16 = i & 15;
+            if (key_base + vr_ >= n)
+              *reinterpret_cast<uint4 *>(gen + LO::kRing + stage * LO::kStage + 16384 + tile_off(vr_, c16, kTileKeys)) =
+                  make_uint4(0, 0, 0, 0);
+          }
+          fence_proxy_async_smem();                          // generic writes, then tensor-core (async proxy) reads
+        }
+        tc_fence_before();
+      }
+      __syncwarp();                                          // every lane's stores and fences are done
+      if (lane == 0) mbar_arrive(p_full + 8u * g);
+      const int c_done = k.c;
+      if (cursor_next(k, w, p.num_splits)) {
+        // chunk end: this thread's half of its row of O, and the row's L, go to the chunk's slot
+        float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
+        float *lbuf = reinterpret_cast<float *>(gen + LO::kLbuf) + g * kUmmaRows;
+        if (ch == 1) lbuf[row] = l_row;
+        if (__all_sync(0xffffffffu, mbar_wait(pv_done + 8u * stage, (uint32_t)((it / kPairStages) & 1), dead))) {
+          tc_fence_after();
+#pragma unroll 1
+          for (int q4 = ch * 2; q4 < ch * 2 + 2; ++q4) {
+            float o[32];
+            tmem_ld32(lane_addr + col_o + q4 * 32, o);
+            if (valid_row) {
+              float4 *dst = reinterpret_cast<float4 *>(slot + (long long)r_glob * D + q4 * 32);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+            }
+          }
+          tc_fence_before();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(o_empty + 8u * g);
+        named_bar(1 + g, 256);                               // both halves of every row of the group are in
+        if (ch == 0 && valid_row) slot[(long long)R * D + r_glob] = l_row + lbuf[row];
+        named_bar(1 + g, 256);                               // lbuf may be rewritten
+        l_row = 0.f;
+      }
+    }
+    if (dead && lane == 0) atomicOr(&p.hdr->wait_timeouts, 16u);
+    if (threadIdx.x == 64 && rp == 0) {                      // every value row is read once per row-pair pass
+      unsigned long long keys = 0;
+      for (int c = split; c < w.n_chunks; c += p.num_splits)
+        keys += min((c + 1) * w.ctiles * kTileKeys, n) - c * w.ctiles * kTileKeys;
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), keys);
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), keys);
+    }
+  }
+
+  // every warp meets here; the allocating warp returns the tensor memory
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
 }  // namespace fold

@@ -43,9 +43,10 @@ def test_group_and_stack_shapes(Hq, Hkv, stack):
 
 
 @pytest.mark.parametrize("Hq,Hkv,stack,D", [(8, 2, 5, 128), (8, 2, 16, 128), (8, 2, 20, 128), (4, 4, 33, 64),
-                                            (8, 2, 64, 128)])
+                                            (8, 2, 64, 128), (8, 2, 40, 128), (4, 1, 75, 128)])
 def test_stacked_rows_beyond_one_row_block(Hq, Hkv, stack, D):
-    # 20 .. 256 query rows per (sequence, kv head): the stacked-row kernel, with ragged 16- and 64-row groups
+    # 20 .. 300 query rows per (sequence, kv head): the stacked-row kernels, with ragged 16-, 64- and 128-row groups
+    # (160 rows: a full and a partial 128-row tile in one pair; 300 rows: a second pair whose second tile is empty)
     w = make_decode_workload(2 * stack, Hq, Hkv, D, [1500, 333], seed=9, device=DEV, stack=stack,
                              poison_padding=True, capacity=1600)
     rows = [(b, h) for b in (0, 1, stack - 1, stack, 2 * stack - 1) for h in (0, Hq - 1)]
