@@ -351,7 +351,10 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   int s = tiles_unit / 32;
   s = s < 1 ? 1 : (s > max_chunks ? max_chunks : s);
   while (units * s < 444 && s < max_chunks) ++s;
-  return s;
+  // even shares: every CTA of the longest sequence gets the same whole number of chunks (14 splits of 16 chunks
+  // would finish no sooner than 8)
+  const int per = max_chunks / s > 1 ? max_chunks / s : 1;
+  return (max_chunks + per - 1) / per;
 }
 
 int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {

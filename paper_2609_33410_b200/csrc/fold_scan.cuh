@@ -1,27 +1,34 @@
 // Split-KV scan (Algorithm 1, rebuilt for a BF16 cache on sm_100a).
 //
-// A CTA walks the 64-key tiles of its canonical chunks for one (KV sequence, kv head).  A
-// producer thread stages tiles HBM -> shared memory with TMA through a ring of mbarriers.
-// Every tile is cut into four 16-key slices; slice w of every tile belongs to warp w of a
-// role, which keeps the instruction sequence that forms a chunk's (A, L) independent of the
-// grid, the batch and the split count.
+// A CTA walks the key tiles of its canonical chunks for one (KV sequence, kv head).  A producer thread
+// stages tiles HBM -> shared memory with TMA through a ring of mbarriers.  Every tile is cut into four
+// slices; slice w of every tile belongs to warp w of a role, which keeps the instruction sequence that
+// forms a chunk's (A, L) independent of the grid, the batch and the split count.
 //
-//   scores   BF16 mma.sync, query rows on M (padded to 16), the slice's 16 keys on N
-//   weights  p = 2^(s - Z) in FP32, final when computed; the depth gate s - Z >= -T decides
-//            per row whether a key's value is used; L sums every key's weight
-//   values   two-term BF16 weights (P_hi + P_lo) times V, rows on M, channels on N, the
-//            slice's 16 keys on K, FP32 accumulate
+//   scores   BF16 mma.sync over the slice's keys and the block's query rows
+//   weights  p = 2^(s - Z) in FP32, final when computed; the depth gate s - Z >= -T decides per row
+//            whether a key's value is used; L sums every key's weight
+//   values   two-term BF16 weights (P_hi + P_lo) times V, FP32 accumulate
 //
-// Two kernels share that arithmetic:
-//   fold_scan_dense_kernel (T = inf): K and V tiles arrive together by TMA; four consumer
+// Row blocks of up to 8 rows (every GQA group up to 8) put the rows on the MMA's N side (keys, then
+// channels, on M): half the MMAs and accumulators of the rows-on-M form, which blocks of 9..16 rows
+// use.  Narrow blocks walk 16 KB key tiles at either head dimension (a warp's slice is 4 KB of keys:
+// 16 keys at D = 128, 32 at D = 64); the rows-on-M kernels walk 64-key tiles with 16-key slices.
+//
+// Kernels:
+//   fold_scan_dense_kernel<D, NARROW> (T = inf): K and V tiles arrive together by TMA; four consumer
 //     warps score and multiply in place.
-//   fold_scan_gated_kernel (finite T): only K is prefetched.  Four scorer warps score a
-//     slice, publish its weights and request just the value rows some row of the group
-//     keeps (one bulk async copy per row); four multiplier warps wait for those rows and
-//     accumulate A.  Scoring never waits for values and values never wait for keys, so both
-//     memory latencies are covered by ring depth, and cut rows cost no traffic.
-// At the end of a chunk the four warps of a role add their partials in a fixed order and
-// write the chunk's slot.
+//   fold_scan_gated_narrow_kernel<D> / fold_scan_gated_kernel<D> (finite T): only K is prefetched.
+//     Four scorer warps score a slice, publish its weights and request just the value rows some row of
+//     the group keeps -- a whole 16-key sub-slice by one TMA box when most of it is live, else row by
+//     row with zero-filling 16-byte async copies; four multiplier warps wait for those rows and
+//     accumulate A.  Scoring never waits for values and values never wait for keys, so both memory
+//     latencies are covered by ring depth, and cut rows cost no traffic.
+//   fold_scan_stacked_kernel<D, GATED>: more than 16 rows per (sequence, kv head) on mma.sync (the
+//     tcgen05 kernels take head_dim 128 with 64 rows or more).
+// At the end of a chunk the four warps of a role add their partials in a fixed order and write the
+// chunk's slot.  Grid: kv heads on x, so CTAs that run together read neighbouring rows of the same
+// tokens; splits on y; KV sequences on z.
 #pragma once
 
 #include "fold_common.cuh"
@@ -221,7 +228,7 @@ __device__ __forceinline__ void load_rows(RowBlock<D> &rb, const ScanParams &p, 
 // Returns the slice's fetch mask (bit k: key k is live for some row); ah / al receive the
 // two-term BF16 weights as A-operand fragments of the value product; l_lo / l_hi accumulate
 // this thread's share of L.
-template <int D, bool GATED, int QK_CHAINS>
+template <int D, bool GATED>
 __device__ __forceinline__ uint32_t score_slice(const RowBlock<D> &rb, uint32_t kt, int warp, int lane, int key0,
                                                 int n, float scale_log2, float neg_T, uint32_t (&ah)[4],
                                                 uint32_t (&al)[4], float &l_lo, float &l_hi) {
@@ -229,30 +236,16 @@ __device__ __forceinline__ uint32_t score_slice(const RowBlock<D> &rb, uint32_t 
   // of the tile laid out [half][key][128 B] with the 128-byte swizzle.
   const int k_key = warp * 16 + ((lane >> 4) << 3) + (lane & 7);
   const uint32_t k_row = k_key * 128, k_x = ((lane >> 3) & 1) ^ (k_key & 7);
-  // QK_CHAINS independent accumulator chains keep the dependent-MMA depth short; they are added
-  // in a fixed order afterwards.
-  float acc[QK_CHAINS][2][4];
+  float s[2][4];
 #pragma unroll
-  for (int j = 0; j < QK_CHAINS; ++j)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[j][0][i] = acc[j][1][i] = 0.f;
+  for (int i = 0; i < 4; ++i) s[0][i] = s[1][i] = 0.f;
 #pragma unroll
   for (int kk = 0; kk < D / 16; ++kk) {
     uint32_t b0, b1, b2, b3;
     ldsm_x4(kt + (kk >> 2) * (kTileKeys * 128) + k_row + ((((2 * kk) & 7) ^ k_x) << 4), b0, b1, b2, b3);
-    mma_bf16(acc[kk % QK_CHAINS][0], rb.qf[kk], b0, b1);
-    mma_bf16(acc[kk % QK_CHAINS][1], rb.qf[kk], b2, b3);
+    mma_bf16(s[0], rb.qf[kk], b0, b1);
+    mma_bf16(s[1], rb.qf[kk], b2, b3);
   }
-  float s[2][4];
-#pragma unroll
-  for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float v = acc[0][nt][i];
-#pragma unroll
-      for (int j = 1; j < QK_CHAINS; ++j) v += acc[j][nt][i];
-      s[nt][i] = v;
-    }
   const int qcol = (lane & 3) * 2;
   uint32_t livemask = 0;
   ah[0] = ah[1] = ah[2] = ah[3] = 0u;
@@ -622,7 +615,7 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       } else {
         uint32_t ah[4], al[4];
-        const uint32_t fetch16 = score_slice<D, false, 1>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        const uint32_t fetch16 = score_slice<D, false>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
         if (fetch16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, ah, al);
       }
       if (key0 + KS > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
@@ -719,7 +712,7 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         const int key0 = k.t * kTileKeys + sl * 16;
         if (key0 >= n) break;
         uint32_t ah[4], al[4];
-        const uint32_t live16 = score_slice<D, GATED, 1>(rb, kt, sl, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        const uint32_t live16 = score_slice<D, GATED>(rb, kt, sl, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
         if (live16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, sl * 16, lane, ah, al);
       }
       if (k.t * kTileKeys + kTileKeys > n) fence_proxy_async_smem();
@@ -832,24 +825,15 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     uint32_t phase = 0;
     unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
 
-#ifdef FOLD_PROFILE
-    long long pf[4] = {0, 0, 0, 0};
-#endif
     for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
       const int my_stage = stage;
-#ifdef FOLD_PROFILE
-      const long long c0 = clock64();
-#endif
       const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
-#ifdef FOLD_PROFILE
-      const long long c1 = clock64();
-#endif
       if (++stage == stages) { stage = 0; phase ^= 1u; }
       const int key0 = k.t * kTileKeys + sl * 16;
       uint32_t ah[4] = {0u, 0u, 0u, 0u}, al[4] = {0u, 0u, 0u, 0u};
       uint32_t fetch16 = 0;
       if (ready) {
-        fetch16 = score_slice<D, true, 1>(rb, base + my_stage * LO::kKTile, sl, lane, key0, n,
+        fetch16 = score_slice<D, true>(rb, base + my_stage * LO::kKTile, sl, lane, key0, n,
                                                             p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);   // the K tile is in registers: release it
@@ -863,14 +847,7 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         st_fetched += whole ? 16 : __popc(fetch16);
         st_skipped += (fetch16 == 0 && nvalid > 0) ? 1 : 0;
       }
-#ifdef FOLD_PROFILE
-      const long long c2 = clock64();
-      const bool vok = !vwrapped || mbar_wait(vempty + 8u * vs, vphase ^ 1u, dead);
-      const long long c3 = clock64();
-      if (vok) {
-#else
       if (!vwrapped || mbar_wait(vempty + 8u * vs, vphase ^ 1u, dead)) {
-#endif
         // publish the slice: weights as the value product's A-operand registers, and the verdict
         uint8_t *pe = pring + vs * pentry;
         if (rb.two_blocks) {
@@ -921,10 +898,6 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         }
       }
       if (++vs == vr) { vs = 0; vwrapped = 1u; vphase ^= 1u; }
-#ifdef FOLD_PROFILE
-      const long long c4 = clock64();
-      pf[0] += c1 - c0; pf[1] += c2 - c1; pf[2] += c3 - c2; pf[3] += c4 - c3;
-#endif
       const int c_done = k.c;
       if (cursor_next(k, w, p.num_splits)) {
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
@@ -936,10 +909,6 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_fetched);
       atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
       if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
-#ifdef FOLD_PROFILE
-      if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && warp == 0)
-        for (int i = 0; i < 4; ++i) p.hdr->pad[i] = (unsigned long long)pf[i];
-#endif
     }
   } else {
     float o[D / 8][4];
