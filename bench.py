@@ -43,9 +43,9 @@ WORKLOADS = {
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one scan launch from the ncu captures
 # summarised in profiles/fold_scan_kernels_c2_small.md, per byte of cache the launch covers: the c2_small
-# capture (268.4 MB of K+V) moved 274.2 MB (gated, T=16) and 273.0 MB (dense).  Traffic grows in
+# capture (268.4 MB of K+V) moved 272.2 MB (gated, T=16) and 271.8 MB (dense).  Traffic grows in
 # proportion to the (sequence, kv head, key) units, so a launch is scaled by its cache bytes.
-NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 274.2 / 268.4, "dense": 273.0 / 268.4}
+NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 272.2 / 268.4, "dense": 271.8 / 268.4}
 
 
 def load_peaks():
@@ -400,8 +400,8 @@ def main():
     value = world * cache_bytes / (r16["ms_per_step"] * 1e-3) / 1e9
     ach16 = actual_bytes(r16) / (r16["scan_ms"] * 1e-3) / 1e9
     achinf = actual_bytes(rinf) / (rinf["scan_ms"] * 1e-3) / 1e9
-    scan_name = ("fold_scan_stacked_kernel + fold_scan_gated_kernel (prefix + suffix levels)" if cascade
-                 else "fold_scan_gated_kernel")
+    scan_name = ("fold_scan_stacked_pair_kernel + fold_scan_gated_narrow_kernel (prefix + suffix levels)" if cascade
+                 else "fold_scan_gated_narrow_kernel")
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
@@ -424,10 +424,11 @@ def main():
                      "traffic": None if cascade or args.workload != "c2" else NCU_TRAFFIC_PER_CACHE_BYTE["gated"] * cache_bytes,
                      "traffic_source": "ncu capture on c2_small scaled by units (profiles/fold_scan_kernels_c2_small.md)",
                      "algorithmic_bytes_per_launch": actual_bytes(r16),
-                     "dense": {"kernel": "fold_scan_dense_kernel (T=inf)" if not cascade else "stacked + dense kernels (T=inf)", "achieved": achinf, "frac": achinf / peak,
+                     "dense": {"kernel": "fold_scan_dense_kernel (T=inf)" if not cascade else "fold_scan_stacked_pair_kernel + fold_scan_dense_kernel (T=inf)", "achieved": achinf, "frac": achinf / peak,
                                "frac_of_nominal_8TBs": achinf / 8000.0,
                                "algorithmic_bytes_per_launch": actual_bytes(rinf)}},
-        "gpu_launches": 3 * args.steps,   # estimate + scan + partial add per timed step (the extra per-kernel pass is not timed)
+        # estimate + scan (one per level) + partial add per timed step (the extra per-kernel pass is not timed)
+        "gpu_launches": (2 + len(levels)) * args.steps,
         "clocks": r16["clocks"],
     }
 
