@@ -258,6 +258,8 @@ def main():
     ap.add_argument("--ref-units", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one whole decode call in a CUDA graph and time its replays (single stream only)")
     ap.add_argument("--cascade-streams", type=int, default=1, choices=[1, 2],
                     help="cascade workloads: scan the levels on one stream (fold_decode_cascade) or on two")
     ap.add_argument("--sweep", action="store_true", help="run the MHA sweep (configuration 5) instead of one workload")
@@ -313,7 +315,7 @@ def main():
     side = torch.cuda.Stream(device=dev) if cascade and args.cascade_streams == 2 else None
     ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
 
-    def step_whole(a):
+    def step_whole(a, stream=stream):
         if not cascade:
             F.fold_decode(a[0], stream)
         elif side is None:
@@ -351,6 +353,17 @@ def main():
         a = make(depth, F.Z_ESTIMATE)
         for _ in range(warmup):
             step_whole(a)
+        run_step = lambda: step_whole(a)
+        if args.graph:
+            # the whole call (memset + estimate + scan + partial add) captured once and replayed: takes the host's
+            # launch cost out of the step, which is what small workloads are bound by
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step_whole(a, torch.cuda.current_stream())
+            run_step = graph.replay
+            for _ in range(warmup):
+                run_step()
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
@@ -360,7 +373,7 @@ def main():
         t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
         t0.record(stream)
         for i in range(steps):
-            step_whole(a)
+            run_step()
         t1.record(stream)
         torch.cuda.synchronize()
         if ctx: ctx.__exit__()
@@ -413,6 +426,7 @@ def main():
                    if cache_bytes > 4 * 126e6 else "cache smaller than 4x L2: partly L2-resident",
                    "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
                    "cascade_streams": args.cascade_streams if cascade else None,
+                   "cuda_graph": bool(args.graph),
                    "flat_equivalent_bytes_per_gpu": flat_bytes},
         "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
         "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},

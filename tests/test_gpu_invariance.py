@@ -149,3 +149,26 @@ def test_shared_prefix_cascade_matches_oracle_and_flat_decode(T, B):
     # and the flat estimate equals the cascade's two-level estimate bit for bit
     fe = run_gpu(flat, T=T)
     assert same_bits(fe.z, bs.z)
+
+
+@pytest.mark.parametrize("T", [math.inf, 16.0])
+def test_graph_replay_equals_eager_call(T):
+    # the whole call (header memset, estimate, scan, partial add) is capturable: nothing allocates or synchronises
+    w = make_decode_workload(2, 8, 2, 128, [20000, 700], seed=71, device=DEV)
+    eager = run_gpu(w, T=T)
+    o, l, z = eager.out.clone(), eager.lse.clone(), eager.z.clone()
+    cache = cache_of(w)
+    bufs = F.alloc_buffers(w.q, cache, w.stack)
+    args = F.make_args(w.q, cache, scale=w.scale, z=bufs.z, depth_T=T, workspace=bufs.workspace, out=bufs.out,
+                       lse=bufs.lse, row_status=bufs.row_status)
+    F.fold_decode(args, torch.cuda.current_stream())          # first call outside capture: one-time set-up
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        F.fold_decode(args, torch.cuda.current_stream())
+    for _ in range(2):
+        bufs.out.zero_(); bufs.lse.zero_(); bufs.z.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert same_bits(bufs.out, o) and same_bits(bufs.lse, l) and same_bits(bufs.z, z)
+        assert bufs.header().wait_timeouts == 0
