@@ -16,6 +16,8 @@ What is here, with the passage each function restates:
   dense_row             Section 2: o = sum_j 2^s_j v_j / sum_j 2^s_j (max-subtracted)
   fold_partial          Eq. 2: F(I) = (A, L) for one key set, plus the depth-T cut
                         of Section 4 "Depth as a dial" (cut keys keep their mass)
+  block_means           Section 4 "Depth as a dial": the mean value of each 64-key block
+                        (the block model without its fitted rank-16 map), stored as BF16
   fold_row              Eq. 2 + Prop. 1(i): partials over key ranges, added
   merge_partials        Prop. 1(i): partials add; o = A/L, lse = Z + log2 L
   online_softmax_bf16   Section 2 online softmax with a running maximum; the
@@ -99,15 +101,44 @@ def live_mask(s: np.ndarray, Z: float, T: float) -> np.ndarray:
     return (s - Z) >= -T
 
 
-def fold_partial(s: np.ndarray, V: np.ndarray, Z: float, T: float = math.inf):
+BLOCK_KEYS = 64  # keys per block of the block model (Section 4, "Depth as a dial")
+
+
+def block_means(V: np.ndarray, block: int = BLOCK_KEYS) -> np.ndarray:
+    """Mean value row of each block of `block` consecutive keys (the last block may be
+    short: the mean is over the keys it has), rounded to BF16 as the cache stores it.
+    Section 4 "Depth as a dial": the block model's mean; its rank-16 key-to-deviation map
+    needs a fit on the prompt and is not part of this reading.  Returns [ceil(n/block), D]."""
+    V = np.asarray(V, dtype=np.float64)
+    n = V.shape[0]
+    nb = (n + block - 1) // block
+    out = np.zeros((nb, V.shape[1]))
+    for b in range(nb):
+        rows = V[b * block:min((b + 1) * block, n)]
+        out[b] = rows.sum(axis=0) / rows.shape[0]
+    return round_to_bf16(out)
+
+
+def fold_partial(s: np.ndarray, V: np.ndarray, Z: float, T: float = math.inf, tail=None):
     """F(I) of Eq. 2 over the keys given, with the depth-T cut: every key adds its
-    weight 2^(s-Z) to L; only live keys add weight*value to A.  Returns (A [D], L)."""
+    weight 2^(s-Z) to L; only live keys add weight*value to A.  Returns (A [D], L).
+
+    tail = (v_mean [num_blocks, D], block_of [len(s)]) switches the block tail on
+    (Section 4 "Depth as a dial"; Algorithm 1 "add the weights of cut keys to the tile's
+    virtual row"): a cut key j adds weight * v_mean[block_of[j]] to A instead of nothing."""
     s = np.asarray(s, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     p = np.exp2(s - Z)
     L = p.sum()
     live = live_mask(s, Z, T)
     A = (p[live, None] * V[live]).sum(axis=0)
+    if tail is not None:
+        v_mean, block_of = tail
+        v_mean = np.asarray(v_mean, dtype=np.float64)
+        block_of = np.asarray(block_of)
+        cut = ~live
+        for b in np.unique(block_of[cut]):
+            A = A + p[cut & (block_of == b)].sum() * v_mean[b]
     return A, L
 
 
@@ -126,17 +157,20 @@ def merge_partials(partials: Iterable, Z: float):
     return o, lse, A, L
 
 
-def fold_row(s, V, Z: float, T: float = math.inf, ranges: Optional[Sequence] = None):
+def fold_row(s, V, Z: float, T: float = math.inf, ranges: Optional[Sequence] = None, v_mean=None):
     """Declared-reference attention of one row.  `ranges` is a list of index arrays /
     slices that partition the keys (default: one range); each range's (A, L) is
-    formed on its own and the pairs are added.  Returns (o, lse2, A, L)."""
+    formed on its own and the pairs are added.  `v_mean` [ceil(n/64), D] switches the
+    block tail on (key j belongs to block j // 64).  Returns (o, lse2, A, L)."""
     s = np.asarray(s, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     if s.size == 0:
         return np.zeros(V.shape[-1]), -np.inf, np.zeros(V.shape[-1]), 0.0
     if ranges is None:
         ranges = [slice(None)]
-    return merge_partials((fold_partial(s[r], V[r], Z, T) for r in ranges), Z)
+    block_of = np.arange(s.size) // BLOCK_KEYS
+    return merge_partials((fold_partial(s[r], V[r], Z, T, None if v_mean is None else (v_mean, block_of[r]))
+                           for r in ranges), Z)
 
 
 def cut_report(s, V, Z: float, T: float, band: float = 2.0 ** -10):

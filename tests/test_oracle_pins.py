@@ -342,3 +342,85 @@ def test_grid_sum_order_free_and_within_prop2_bound():
     # FP32 partials that need no rounding on the grid add exactly
     g = [1.5, 2.0 ** -20, -0.75, 3.0]
     assert O.grid_sum(g)[0] == sum(g)
+
+
+# ------------------------------------------------------------------ block tail (Section 4, "Depth as a dial")
+def test_block_means_brute_force_and_short_last_block():
+    r = _rng(40)
+    V = _bf16ish(r.standard_normal((150, 8)))                 # blocks of 64, 64 and 22 keys
+    m = O.block_means(V)
+    assert m.shape == (3, 8)
+    for b, (lo, hi) in enumerate([(0, 64), (64, 128), (128, 150)]):
+        for d in range(8):
+            exact = Fraction(0)
+            for j in range(lo, hi):
+                exact += Fraction(float(V[j, d]))
+            exact /= (hi - lo)
+            # stored as BF16: within half a BF16 ulp of the exact rational mean
+            assert abs(Fraction(float(m[b, d])) - exact) <= abs(exact) * Fraction(1, 256) + Fraction(1, 2 ** 130)
+    # dyadic values with an exactly representable mean come back exactly
+    Vd = np.tile(np.array([[1.0, -2.0], [3.0, 6.0]]), (32, 1))           # 64 rows: mean (2, 2)
+    assert np.array_equal(O.block_means(Vd), np.array([[2.0, 2.0]]))
+
+
+def test_block_tail_is_exact_when_values_are_constant_within_blocks():
+    # if every key of a block holds the block's mean, replacing cut values by the mean changes nothing:
+    # the finite-depth result with the tail must equal dense attention, whatever T cuts
+    r = _rng(41)
+    n, D = 300, 16
+    q = _bf16ish(r.standard_normal(D)); K = _bf16ish(r.standard_normal((n, D)))
+    vb = _bf16ish(r.standard_normal(((n + 63) // 64, D)))
+    V = vb[np.arange(n) // 64]
+    s = O.scores(q, K)
+    o_dense, lse_dense = O.dense_row(s, V)
+    m = O.block_means(V)
+    assert np.array_equal(m, vb)
+    for Z in (lse_dense, lse_dense - 3.0):
+        for T in (0.5, 2.0, 6.0, 16.0):
+            assert (~O.live_mask(s, Z, T)).any() or T == 16.0
+            o, lse, _, _ = O.fold_row(s, V, Z, T, v_mean=m)
+            assert np.allclose(o, o_dense, rtol=1e-12, atol=1e-13) and abs(lse - lse_dense) < 1e-12
+            o_plain, _, _, _ = O.fold_row(s, V, Z, T)
+            if (~O.live_mask(s, Z, T)).any():
+                assert not np.allclose(o_plain, o_dense, rtol=1e-6)      # without the tail the cut shows
+
+
+def test_block_tail_identity_brute_force_and_partition_invariance():
+    q, K, V = _row(42, n=200, D=8)
+    s = O.scores(q, K)
+    _, lse = O.dense_row(s, V)
+    Z, T = lse - 1.0, 3.0
+    m = O.block_means(V)
+    o_tail, _, A_tail, L = O.fold_row(s, V, Z, T, v_mean=m)
+    o_plain, _, A_plain, L2 = O.fold_row(s, V, Z, T)
+    assert L == L2                                                       # the mass is the same either way
+    # brute force: A_tail - A_plain = sum over cut keys of p_j * mean of j's block
+    extra = np.zeros(8)
+    for j in range(200):
+        if s[j] - Z < -T:
+            extra += 2.0 ** (s[j] - Z) * m[j // 64]
+    assert np.allclose(A_tail - A_plain, extra, rtol=1e-12, atol=1e-15)
+    # T = inf: nothing is cut, the tail adds nothing
+    assert np.array_equal(O.fold_row(s, V, Z, math.inf, v_mean=m)[2], O.fold_row(s, V, Z, math.inf)[2])
+    # any partition of the keys, also one that splits blocks, adds up to the same pair
+    perm = _rng(43).permutation(200)
+    ranges = [perm[:37], perm[37:120], perm[120:]]
+    o_parts, _, A_parts, _ = O.fold_row(s, V, Z, T, ranges=ranges, v_mean=m)
+    assert np.allclose(A_parts, A_tail, rtol=1e-12, atol=1e-15)
+
+
+def test_block_tail_reduces_the_truncation_error_on_smooth_values():
+    # values that drift slowly along the sequence are well described by their block means
+    r = _rng(44)
+    n, D = 2000, 16
+    q = _bf16ish(r.standard_normal(D)); K = _bf16ish(r.standard_normal((n, D)))
+    t = np.arange(n)[:, None] / n
+    V = _bf16ish(np.sin(2 * np.pi * (t + np.arange(D)[None, :] / D)) + 0.01 * r.standard_normal((n, D)))
+    s = O.scores(q, K)
+    o_dense, lse = O.dense_row(s, V)
+    T = 11.0                                                             # weights sit near 2^-11: about half are cut
+    cut = ~O.live_mask(s, lse, T)
+    assert 0.2 < cut.mean() < 0.8
+    e_plain = np.linalg.norm(O.fold_row(s, V, lse, T)[0] - o_dense)
+    e_tail = np.linalg.norm(O.fold_row(s, V, lse, T, v_mean=O.block_means(V))[0] - o_dense)
+    assert e_tail < 0.3 * e_plain
