@@ -215,6 +215,8 @@ def run_sweep(args, dev):
                 seed = 5000 + D * 7 + B * 131 + n
                 w = make_decode_workload(B, 32, 32, D, n, seed=seed, device=dev)
                 cache = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table)
+                if args.tail:
+                    F.fold_block_means(cache, stream)
                 bufs = F.alloc_buffers(w.q, cache)
                 # small caches are L2-resident unless evicted: stream a 512 MB buffer between samples
                 flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if cache_bytes < 4 * 126e6 else None
@@ -244,7 +246,7 @@ def run_sweep(args, dev):
                                       v_rows_fetched=round(lam, 4), l2_flush=flush is not None))
                 del w, cache, bufs, flush
                 torch.cuda.empty_cache()
-    print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "cells": cells}))
+    print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "block_tail": bool(args.tail), "cells": cells}))
 
 
 def main():
@@ -258,6 +260,8 @@ def main():
     ap.add_argument("--ref-units", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--tail", action="store_true",
+                    help="finite-depth steps use the block tail (cut keys add weight x block-mean value)")
     ap.add_argument("--graph", action="store_true",
                     help="capture one whole decode call in a CUDA graph and time its replays (single stream only)")
     ap.add_argument("--cascade-streams", type=int, default=1, choices=[1, 2],
@@ -300,6 +304,13 @@ def main():
         levels = [make_decode_workload(device=dev, **gen)]
     w = levels[-1]                                                        # the level that owns out / lse / z
     caches = [F.KVCache(l.k, l.v, l.seqlens, l.max_seqlen, l.page_table) for l in levels]
+    if args.tail:
+        # block tail (the block model's mean): cut keys add weight x their 64-key block's mean value; the table is
+        # built once from the cache, outside the timed region (it belongs to cache write)
+        if cascade:
+            raise SystemExit("--tail: the block tail is built into the row-block scan only (no stacked prefix level)")
+        F.fold_block_means(caches[0], stream)
+        torch.cuda.synchronize()
     lbufs = [F.alloc_buffers(l.q, c, l.stack) for l, c in zip(levels, caches)]
     bufs = lbufs[-1]
     cache_bytes = sum(l.cache_bytes() for l in levels)                    # unique bytes: a shared prefix counts once
@@ -426,7 +437,7 @@ def main():
                    if cache_bytes > 4 * 126e6 else "cache smaller than 4x L2: partly L2-resident",
                    "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
                    "cascade_streams": args.cascade_streams if cascade else None,
-                   "cuda_graph": bool(args.graph),
+                   "cuda_graph": bool(args.graph), "block_tail": bool(args.tail),
                    "flat_equivalent_bytes_per_gpu": flat_bytes},
         "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
         "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},

@@ -71,7 +71,20 @@ enum {
  * Paged (page_table != NULL): logical token j of sequence `seq` is row
  *     (page = page_table[seq*max_pages_per_seq + j / page_size], j % page_size, head) at
  *     k + page*stride_seq + (j % page_size)*stride_tok + head*stride_head.
- * Rows at or beyond seqlens[seq] (and unused page tails) are never used, whatever they hold. */
+ * Rows at or beyond seqlens[seq] (and unused page tails) are never used, whatever they hold.
+ *
+ * Block tail (Section 4, "Depth as a dial": the block model, its mean only -- the fitted rank-16 map is
+ * not part of this library).  v_block_mean, when not NULL, holds for every LOGICAL block of 64
+ * consecutive keys [64 b, 64 b + 64) of every sequence the mean of that block's value rows as BF16
+ * (a short last block: the mean of the keys it has), row (seq, b, head) at
+ *     v_block_mean + seq*mean_stride_seq + b*mean_stride_block + head*mean_stride_head
+ * (elements; multiples of 8; rows 16-byte aligned; blocks are logical for paged caches too).  A decode
+ * at finite depth then adds, for every row, the summed weight of the keys that row cuts in a block
+ * times that block's mean to A, instead of nothing (Algorithm 1: "add the weights of cut keys to the
+ * tile's virtual row").  fold_block_means() fills the table from the cache; keeping it current when
+ * tokens are appended is the caller's business (only the last block changes).  Supported where up to
+ * 8 query rows share a (sequence, kv head); other shapes return FOLD_EUNSUPPORTED when it is set.
+ * Ignored at depth_T = INFINITY (nothing is cut). */
 typedef struct fold_kv {
   const void *k, *v;
   int64_t stride_seq, stride_tok, stride_head;   /* elements */
@@ -83,6 +96,8 @@ typedef struct fold_kv {
   int32_t num_seqs;                              /* KV sequences */
   const int32_t *seqlens;                        /* [num_seqs] keys per sequence */
   int32_t max_seqlen;                            /* HOST upper bound on seqlens[]; sizes grids and slots */
+  const void *v_block_mean;                      /* BF16 block means, or NULL: no block tail */
+  int64_t mean_stride_seq, mean_stride_block, mean_stride_head;   /* elements */
 } fold_kv;
 
 /* One decode call.  `batch` requests with one query token each; request b reads KV
@@ -184,13 +199,22 @@ int fold_decode(const fold_args *args, fold_stream stream);
  * out, lse and row_status are taken from levels[0]. */
 int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_stream stream);
 
+/* Fill kv->v_block_mean (DEVICE memory of the caller, laid out as the fold_kv comment says, at least
+ * ceil(kv->max_seqlen / 64) blocks per sequence) from kv->v: for every sequence, block b < ceil(n / 64)
+ * and kv head, the mean of the block's value rows, summed in float64 in key order, divided by the key
+ * count, rounded to FP32 and then to BF16 (both to nearest even) -- Section 4, "Depth as a dial".  Blocks
+ * at or beyond ceil(n / 64) are left untouched.  Asynchronous on `stream`; reads seqlens on the device.
+ * num_kv_heads / head_dim as in fold_args.  FOLD_EINVAL for a NULL or misaligned table. */
+int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, fold_stream stream);
+
 /* The same decode for callers whose tensors live in HOST memory (pinned for the copies to
  * be asynchronous): q, kv.k, kv.v, kv.page_table, kv.seqlens, z (if GIVEN), out, lse and
  * row_status of *host_args are HOST pointers laid out as described above (the cache is
  * copied as the single span its strides cover).  `staging` is DEVICE memory of at least
  * fold_host_staging_bytes(host_args) bytes, 256-byte aligned, which receives the copies,
  * the workspace and the results before they are copied back.  Everything is enqueued on
- * `stream`; the host buffers are valid after the caller synchronises the stream. */
+ * `stream`; the host buffers are valid after the caller synchronises the stream.  The block tail is
+ * not offered here: kv.v_block_mean must be NULL (FOLD_EUNSUPPORTED otherwise). */
 size_t fold_host_staging_bytes(const fold_args *host_args);
 int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_bytes, fold_stream stream);
 

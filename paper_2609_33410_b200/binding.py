@@ -28,7 +28,9 @@ class FoldKV(C.Structure):
                 ("stride_seq", C.c_int64), ("stride_tok", C.c_int64), ("stride_head", C.c_int64),
                 ("page_table", C.c_void_p), ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32),
                 ("num_pages", C.c_int32), ("capacity", C.c_int32), ("num_seqs", C.c_int32),
-                ("seqlens", C.c_void_p), ("max_seqlen", C.c_int32)]
+                ("seqlens", C.c_void_p), ("max_seqlen", C.c_int32),
+                ("v_block_mean", C.c_void_p), ("mean_stride_seq", C.c_int64), ("mean_stride_block", C.c_int64),
+                ("mean_stride_head", C.c_int64)]
 
 
 class FoldArgs(C.Structure):
@@ -58,7 +60,7 @@ class FoldWsHeader(C.Structure):
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
            "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
-           "fold_decode_host", "fold_decode_static", "fold_status_string", "fold_version"]
+           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_status_string", "fold_version"]
 
 _lib = None
 
@@ -86,6 +88,8 @@ def lib() -> C.CDLL:
         L.fold_decode_host.restype = C.c_int
         L.fold_decode_host.argtypes = [C.POINTER(FoldArgs), C.c_void_p, C.c_size_t, C.c_void_p]
         L.fold_decode_static.restype = C.c_int; L.fold_decode_static.argtypes = [C.POINTER(FoldArgs), C.c_void_p]
+        L.fold_block_means.restype = C.c_int
+        L.fold_block_means.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p]
         L.fold_status_string.restype = C.c_char_p; L.fold_status_string.argtypes = [C.c_int]
         L.fold_version.restype = C.c_int
         _lib = L
@@ -123,6 +127,7 @@ class KVCache:
     seqlens: torch.Tensor
     max_seqlen: int
     page_table: Optional[torch.Tensor] = None
+    v_block_mean: Optional[torch.Tensor] = None     # [num_seqs, ceil(max_seqlen / 64), Hkv, D] bf16: switches the block tail on
 
     def to_c(self) -> FoldKV:
         k, v = self.k, self.v
@@ -149,7 +154,21 @@ class KVCache:
             kv.max_pages_per_seq = 0
             kv.num_pages = 0
             kv.capacity = k.shape[1]
+        if self.v_block_mean is not None:
+            m = self.v_block_mean
+            assert m.dtype == torch.bfloat16 and m.dim() == 4 and m.stride(3) == 1 and m.shape[0] == kv.num_seqs
+            assert m.shape[1] * 64 >= kv.max_seqlen and m.shape[2:] == k.shape[2:]
+            kv.v_block_mean = m.data_ptr()
+            kv.mean_stride_seq, kv.mean_stride_block, kv.mean_stride_head = m.stride(0), m.stride(1), m.stride(2)
+        else:
+            kv.v_block_mean = None
         return kv
+
+    def alloc_block_means(self) -> torch.Tensor:
+        """An empty table of the shape fold_block_means fills (and the block tail reads)."""
+        nb = max((int(self.max_seqlen) + 63) // 64, 1)
+        return torch.zeros(self.seqlens.shape[0], nb, self.k.shape[2], self.k.shape[3], dtype=torch.bfloat16,
+                           device=self.k.device)
 
 
 def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None, z_mode: int = Z_ESTIMATE,
@@ -203,6 +222,16 @@ def fold_cascade_merge(levels: Sequence[FoldPartials], out: torch.Tensor, lse: O
     arr = (C.POINTER(FoldPartials) * len(levels))(*[C.pointer(p) for p in levels])
     _check(lib().fold_cascade_merge(arr, len(levels), out.data_ptr(), _ptr(lse), _ptr(row_status), _stream(stream)),
            "fold_cascade_merge")
+
+
+def fold_block_means(cache: KVCache, stream=None) -> torch.Tensor:
+    """Fill (allocating it if the cache has none) cache.v_block_mean from cache.v; returns the table."""
+    if cache.v_block_mean is None:
+        cache.v_block_mean = cache.alloc_block_means()
+    kv = cache.to_c()
+    _check(lib().fold_block_means(C.byref(kv), int(cache.k.shape[2]), int(cache.k.shape[3]), _stream(stream)),
+           "fold_block_means")
+    return cache.v_block_mean
 
 
 def fold_decode(args: FoldArgs, stream=None) -> None:

@@ -42,6 +42,11 @@ int check_kv(const fold_kv &kv, int D) {
   } else {
     if (kv.capacity < kv.max_seqlen || kv.capacity < 1) return FOLD_EINVAL;
   }
+  if (kv.v_block_mean) {
+    if (!aligned(kv.v_block_mean, 16)) return FOLD_EINVAL;
+    if (kv.mean_stride_seq < 0 || kv.mean_stride_block < D || kv.mean_stride_head < 0) return FOLD_EINVAL;
+    if (kv.mean_stride_seq % 8 || kv.mean_stride_block % 8 || kv.mean_stride_head % 8) return FOLD_EINVAL;
+  }
   return FOLD_OK;
 }
 
@@ -63,6 +68,8 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   const int G = a->num_q_heads / a->num_kv_heads;
   const long long R = (long long)a->stack * G;
   if (G > kMaxRows || R > kMaxStackedRows) return FOLD_EUNSUPPORTED;
+  // the block tail is built into the narrow row-block scan only
+  if (a->kv.v_block_mean && !isinf(a->depth_T) && R > kNarrowRows) return FOLD_EUNSUPPORTED;
   g->B = a->batch; g->Hq = a->num_q_heads; g->Hkv = a->num_kv_heads; g->G = G; g->D = a->head_dim;
   g->stack = a->stack; g->R = (int)R; g->num_seqs = a->kv.num_seqs;
   g->max_slots = max_chunks_upto(a->kv.max_seqlen);
@@ -293,10 +300,36 @@ int launch_stacked_pair(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+// Narrow row blocks (rows on N): unpadded value slices; three K stages (measured: a fourth buys nothing and costs L1).
+template <int D, bool TAIL>
+int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LN = GatedNarrowLayout<D, TAIL>;
+  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  int nvr = 2;
+  int nstages = (per_cta2 - LN::total(0, nvr)) / (LN::kKStage + 16);
+  if (nstages > 3) nstages = 3;
+#ifdef FOLD_TUNING
+  if (const char *e = getenv("FOLD_TUNE_STAGES")) nstages = atoi(e);
+  if (const char *e = getenv("FOLD_TUNE_VR")) nvr = atoi(e);
+  if (const char *e = getenv("FOLD_TUNE_BOXMIN")) p.box_min = atoi(e);
+#endif
+  if (nstages < 2 || nvr < 1 || LN::total(nstages, nvr) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
+  p.stages = nstages;
+  p.vr = nvr;
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_gated_narrow_kernel<D, TAIL>, configured)) return rc;
+  if (launch_pdl(fold_scan_gated_narrow_kernel<D, TAIL>, grid, dim3(kGatedThreads), LN::total(nstages, nvr), st, mk, mvs, p) !=
+      cudaSuccess)
+    return FOLD_ECUDA;
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 // Gated scan: value slots hold rows whose requests can only be issued after scoring, so shared
 // memory is split between the key ring and the value slots of each slice.
 template <int D>
 int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
+  if (p.R <= kNarrowRows)                                    // rows on N; with or without the block tail
+    return p.vmean ? launch_gated_narrow<D, true>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false>(mk, mvs, p, grid, st);
   using LO = GatedLayout<D>;
   const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
   int vr = 2;
@@ -314,24 +347,6 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
   if (stages < 2 || vr < 1 || LO::total(stages, vr, p.R) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = vr;
-  if (p.R <= kNarrowRows) {                                  // rows on N; unpadded value slices leave room for a deeper K ring
-    using LN = GatedNarrowLayout<D>;
-    int nvr = 2;
-    int nstages = (per_cta2 - LN::total(0, nvr)) / (LN::kKTile + 16);
-    if (nstages > 3) nstages = 3;                            // measured: a fourth stage buys nothing and costs L1
-#ifdef FOLD_TUNING
-    if (const char *e = getenv("FOLD_TUNE_STAGES")) nstages = atoi(e);
-    if (const char *e = getenv("FOLD_TUNE_VR")) nvr = atoi(e);
-#endif
-    if (nstages < 2 || nvr < 1 || LN::total(nstages, nvr) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
-    p.stages = nstages;
-    p.vr = nvr;
-    static int configured[64] = {0};
-    if (int rc = opt_in_smem(fold_scan_gated_narrow_kernel<D>, configured)) return rc;
-    if (launch_pdl(fold_scan_gated_narrow_kernel<D>, grid, dim3(kGatedThreads), LN::total(nstages, nvr), st, mk, mvs, p) != cudaSuccess)
-      return FOLD_ECUDA;
-    return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
-  }
   static int configured[64] = {0};
   if (int rc = opt_in_smem(fold_scan_gated_kernel<D>, configured)) return rc;
   if (launch_pdl(fold_scan_gated_kernel<D>, grid, dim3(kGatedThreads), LO::total(stages, vr, p.R), st, mk, mvs, p) != cudaSuccess)
@@ -380,6 +395,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.page_table = kv.page_table;
   p.v = static_cast<const __nv_bfloat16 *>(kv.v);
   p.v_stride_seq = kv.stride_seq; p.v_stride_tok = kv.stride_tok; p.v_stride_head = kv.stride_head;
+  p.vmean = static_cast<const __nv_bfloat16 *>(kv.v_block_mean);
+  p.vm_stride_seq = kv.mean_stride_seq; p.vm_stride_block = kv.mean_stride_block; p.vm_stride_head = kv.mean_stride_head;
   p.slots = reinterpret_cast<float *>(static_cast<uint8_t *>(a->workspace) + kHeaderBytes);
   p.slot_stride = g.slot_stride;
   p.hdr = static_cast<fold_ws_header *>(a->workspace);
@@ -530,6 +547,30 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, fold_stream stream) {
+  if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
+  if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
+  if (!kv->v_block_mean) return FOLD_EINVAL;
+  if (int rc = check_kv(*kv, head_dim)) return rc;
+  const int max_blocks = (kv->max_seqlen + 63) / 64;
+  if (max_blocks == 0) return FOLD_OK;
+  MeanParams p;
+  p.v = static_cast<const __nv_bfloat16 *>(kv->v);
+  p.v_stride_seq = kv->stride_seq; p.v_stride_tok = kv->stride_tok; p.v_stride_head = kv->stride_head;
+  p.mean = static_cast<__nv_bfloat16 *>(const_cast<void *>(kv->v_block_mean));
+  p.m_stride_seq = kv->mean_stride_seq; p.m_stride_block = kv->mean_stride_block; p.m_stride_head = kv->mean_stride_head;
+  p.seqlens = kv->seqlens; p.page_table = kv->page_table;
+  p.max_seqlen = kv->max_seqlen;
+  p.page_shift = kv->page_table ? ilog2(kv->page_size) : 0;
+  p.max_pages = kv->max_pages_per_seq; p.num_pages = kv->num_pages > 0 ? kv->num_pages : 1;
+  p.Hkv = num_kv_heads;
+  const dim3 grid((max_blocks + 3) / 4, num_kv_heads, kv->num_seqs), block(32, 4);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (head_dim == 128) fold_block_mean_kernel<128><<<grid, block, 0, st>>>(p);
+  else fold_block_mean_kernel<64><<<grid, block, 0, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 int fold_decode(const fold_args *args, fold_stream stream) {
   Geometry g;
   if (int rc = check_args(args, &g, true)) return rc;
@@ -612,6 +653,7 @@ int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, f
   if (!ha || !staging || !aligned(staging, 256)) return FOLD_EINVAL;
   if (!ha->q || !ha->kv.k || !ha->kv.v || !ha->kv.seqlens || !ha->out) return FOLD_EINVAL;
   if (ha->z_mode == FOLD_Z_GIVEN && !ha->z) return FOLD_EINVAL;
+  if (ha->kv.v_block_mean) return FOLD_EUNSUPPORTED;        // the block tail is not offered for host buffers
   HostPlan h;
   if (fold_workspace_bytes(ha) == 0 || !plan_host(ha, &h)) return FOLD_EINVAL;
   if (staging_bytes < h.total) return FOLD_EWORKSPACE;

@@ -222,4 +222,54 @@ __global__ void fold_fill_kernel(float *z, int count, float value) {
   if (i < count) z[i] = value;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Block means for the block tail (Section 4, "Depth as a dial"): one warp per (sequence, 64-key block, kv head),
+// each lane D / 32 channels; the block's value rows are summed in float64 in key order, divided by the key count
+// and rounded to FP32, then to BF16.
+struct MeanParams {
+  const __nv_bfloat16 *v;
+  long long v_stride_seq, v_stride_tok, v_stride_head;
+  __nv_bfloat16 *mean;
+  long long m_stride_seq, m_stride_block, m_stride_head;
+  const int *seqlens;
+  const int *page_table;
+  int max_seqlen, page_shift, max_pages, num_pages, Hkv;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128) fold_block_mean_kernel(const MeanParams p) {
+  constexpr int EPT = D / 32;
+  const int lane = threadIdx.x, blk = blockIdx.x * 4 + threadIdx.y, kvh = blockIdx.y, seq = blockIdx.z;
+  int n = p.seqlens[seq];
+  n = n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
+  const int j0 = blk * 64, j1 = min(j0 + 64, n);
+  if (j0 >= n) return;
+  double acc[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) acc[e] = 0.0;
+  const int page_mask = (1 << p.page_shift) - 1;
+  for (int j = j0; j < j1; ++j) {
+    long long s_row = seq, t_row = j;
+    if (p.page_table) {
+      const int pg = p.page_table[(long long)seq * p.max_pages + (j >> p.page_shift)];
+      s_row = min(max(pg, 0), p.num_pages - 1);
+      t_row = j & page_mask;
+    }
+    const __nv_bfloat16 *row = p.v + s_row * p.v_stride_seq + t_row * p.v_stride_tok + (long long)kvh * p.v_stride_head + lane * EPT;
+    if (EPT == 4) {
+      const uint2 w = *reinterpret_cast<const uint2 *>(row);
+      acc[0] += (double)__uint_as_float(w.x << 16); acc[1] += (double)__uint_as_float(w.x & 0xffff0000u);
+      acc[EPT - 2] += (double)__uint_as_float(w.y << 16); acc[EPT - 1] += (double)__uint_as_float(w.y & 0xffff0000u);
+    } else {
+      const uint32_t w = *reinterpret_cast<const uint32_t *>(row);
+      acc[0] += (double)__uint_as_float(w << 16); acc[1] += (double)__uint_as_float(w & 0xffff0000u);
+    }
+  }
+  const double cnt = (double)(j1 - j0);
+  __nv_bfloat16 *dst = p.mean + (long long)seq * p.m_stride_seq + (long long)blk * p.m_stride_block +
+                       (long long)kvh * p.m_stride_head + lane * EPT;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) dst[e] = __float2bfloat16_rn(__double2float_rn(acc[e] / cnt));
+}
+
 }  // namespace fold

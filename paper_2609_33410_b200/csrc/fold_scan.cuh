@@ -43,6 +43,8 @@ struct ScanParams {
   const int *page_table;
   const __nv_bfloat16 *v;                         // gated path reads value rows directly
   long long v_stride_seq, v_stride_tok, v_stride_head;
+  const __nv_bfloat16 *vmean;                     // block tail: mean value row of every 64-key block, or null
+  long long vm_stride_seq, vm_stride_block, vm_stride_head;
   float *slots;
   long long slot_stride;
   fold_ws_header *hdr;
@@ -90,15 +92,19 @@ struct GatedLayout {
 
 // Narrow gated kernel: every value slice in the swizzled box layout (no row padding), and a two-warp
 // parking area for the chunk-end add.
-template <int D>
+template <int D, bool TAIL = false>
 struct GatedNarrowLayout {
   static constexpr int kTK = narrow_tile_keys<D>();          // keys per tile
   static constexpr int kU = kTK / 64;                        // 16-key sub-slices per warp slice
   static constexpr int kKTile = kTK * D * 2;
   static constexpr int kVSlice = 16 * kU * D * 2;            // [D/64 halves][16 kU rows][128 B], swizzled
-  static constexpr int kPEntry = kU * 512 + 32;              // 16 B of B-operand registers per lane and sub-slice + the verdict
+  // per slice: 16 B of B-operand registers per lane and sub-slice; with the block tail each lane's cut mass of its
+  // two rows (8 B per lane) and the mean value row of the slice's block (D * 2 <= 256 B); the verdict words
+  static constexpr int kPEntry = kU * 512 + (TAIL ? 512 : 0) + 32;
+  static constexpr int kMeanBytes = (kTK / 64) * D * 2;      // mean rows that ride with a K tile: one per 64-key block
+  static constexpr int kKStage = kKTile + (TAIL ? 1024 : 0); // K tile (+ mean rows), 1 KB-aligned for the swizzle
   static constexpr int kPark = D / 16 * 4 * 32 * 4;          // one warp's accumulators, fragment order
-  __host__ __device__ static int off_vring(int stages) { return stages * kKTile; }
+  __host__ __device__ static int off_vring(int stages) { return stages * kKStage; }
   __host__ __device__ static int off_pring(int stages, int vr) { return off_vring(stages) + kConsumerWarps * vr * kVSlice; }
   __host__ __device__ static int off_red(int stages, int vr) { return off_pring(stages, vr) + kConsumerWarps * vr * kPEntry; }
   __host__ __device__ static int off_redl(int stages, int vr) { return off_red(stages, vr) + 2 * kPark; }
@@ -149,7 +155,8 @@ __device__ __forceinline__ bool cursor_next(TileCursor &k, const SeqWork &w, int
 }
 
 // Producer thread: TMA-stage the tiles of chunks split, split + num_splits, ... in order.
-template <int D, bool WITH_V, int STAGE_BYTES, int TK = kTileKeys>
+// WITH_MEAN: the mean value rows of the tile's 64-key blocks (block tail) follow the K tile in its stage.
+template <int D, bool WITH_V, int STAGE_BYTES, int TK = kTileKeys, bool WITH_MEAN = false>
 __device__ __forceinline__ void produce_tiles(const CUtensorMap *tmK, const CUtensorMap *tmV, const ScanParams &p,
                                               const SeqWork &w, int split, int kvh, int seq, uint32_t ring,
                                               uint32_t full0, uint32_t empty0) {
@@ -168,8 +175,14 @@ __device__ __forceinline__ void produce_tiles(const CUtensorMap *tmK, const CUte
     const int tok0 = k.t * TK;
     const int nbox = min(boxes_per_tile, (w.n - tok0 + p.box_tok - 1) / p.box_tok);
     const uint32_t full = full0 + 8u * stage;
-    mbar_expect_tx(full, nbox * p.box_tok * D * 2 * (WITH_V ? 2 : 1));
+    const int nmean = WITH_MEAN ? min(TK / 64, (w.n - tok0 + 63) / 64) : 0;
+    mbar_expect_tx(full, nbox * p.box_tok * D * 2 * (WITH_V ? 2 : 1) + nmean * D * 2);
     const uint32_t kdst = ring + stage * STAGE_BYTES;
+    if (WITH_MEAN) {
+      const __nv_bfloat16 *m = p.vmean + (long long)seq * p.vm_stride_seq + (long long)(tok0 / 64) * p.vm_stride_block +
+                               (long long)kvh * p.vm_stride_head;
+      for (int i = 0; i < nmean; ++i) bulk_load(kdst + KTILE + i * (D * 2), m + (long long)i * p.vm_stride_block, D * 2, full);
+    }
     const uint32_t vdst = kdst + KTILE;
     for (int bx = 0; bx < nbox; ++bx) {
       const int j0 = tok0 + bx * p.box_tok;
@@ -395,10 +408,11 @@ __device__ __forceinline__ void qk_issue_n(const RowBlockN<D> &rb, uint32_t kt, 
 
 // Final weights of a slice.  Returns the fetch mask; bh / bl receive P_hi^T / P_lo^T as B fragments of the
 // value product; l0 / l1 accumulate this thread's share of L for rows (lane%4)*2 + {0,1}.
-template <int D, bool GATED>
+// TAIL: c0 / c1 also accumulate the weight of this thread's cut keys (the block tail's virtual row, Algorithm 1).
+template <int D, bool GATED, bool TAIL = false>
 __device__ __forceinline__ uint32_t weights_n(const RowBlockN<D> &rb, const float (&s)[4], int lane, int key0, int n,
                                               float scale_log2, float neg_T, uint32_t (&bh)[2], uint32_t (&bl)[2],
-                                              float &l0, float &l1) {
+                                              float &l0, float &l1, float *c0 = nullptr, float *c1 = nullptr) {
   const int klo = lane >> 2;
   uint32_t livemask = 0;
 #pragma unroll
@@ -420,6 +434,7 @@ __device__ __forceinline__ uint32_t weights_n(const RowBlockN<D> &rb, const floa
     const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
     l0 += (h0 + g0) + (pw[0] - pm[0]);
     l1 += (h1 + g1) + (pw[1] - pm[1]);
+    if (TAIL) { *c0 += pw[0] - pm[0]; *c1 += pw[1] - pm[1]; }
     bh[kh] = movmatrix_trans(hi2);                            // [key][row] block -> [row][key]: the B fragment
     bl[kh] = movmatrix_trans(lo2);
   }
@@ -953,11 +968,16 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 // Depth-gated decode for narrow row blocks (at most 8 rows): the same roles with the products turned
 // round (rows on N), which halves the MMAs and the accumulator registers.  Value slices always sit in
 // the swizzled box layout, whichever way they were fetched.
-template <int D>
+// TAIL (block tail of Section 4 "Depth as a dial", mean only): a row's cut keys add their summed weight times
+// the mean value row of their 64-key block.  The mean rows ride with the K tiles (256 bytes per tile).  A slice lies
+// inside one block; its scorer publishes every lane's cut mass and a copy of the block's mean row with the slice;
+// the multiplier sums the cut mass per row and adds cut mass x mean after the slice's products.  A slice with no
+// live key still does that part.
+template <int D, bool TAIL>
 __global__ void __launch_bounds__(kGatedThreads, 2)
 fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
                               const ScanParams p) {
-  using LO = GatedNarrowLayout<D>;
+  using LO = GatedNarrowLayout<D, TAIL>;
   constexpr int TK = LO::kTK, U = LO::kU, KS = 16 * U;       // keys per tile, sub-slices and keys per warp slice
   constexpr int C16 = D / 8;                                 // 16-byte chunks per value row
   constexpr int RPI = 32 / C16;                              // rows one warp-wide async copy covers
@@ -992,13 +1012,13 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   pdl_wait();                                                // z (and the zeroed header) come from earlier work
 
   if (warp == SW + kConsumerWarps) {
-    if (lane == 0) produce_tiles<D, false, LO::kKTile, TK>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
+    if (lane == 0) produce_tiles<D, false, LO::kKStage, TK, TAIL>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
     return;
   }
 
   const bool scorer = warp < SW;
   const int sl = warp & 3;                                   // the slice of every tile this warp owns
-  constexpr int pentry = LO::kPEntry, pmask = U * 512;
+  constexpr int pentry = LO::kPEntry, pcut = U * 512, pmean = U * 512 + 256, pmask = pentry - 32;
   uint8_t *pring = gen + LO::off_pring(stages, vr) + sl * vr * pentry;
   const uint32_t vring = base + LO::off_vring(stages) + sl * vr * LO::kVSlice;
   const uint32_t vfull = vfull0 + 8u * sl * vr, vempty = vempty0 + 8u * sl * vr;
@@ -1029,19 +1049,26 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         const bool ready = mbar_wait(full0 + 8u * my_stage, my_phase, dead);
         const int key0 = k.t * TK + sl * KS;
         uint32_t bh[U][2], bl[U][2];
+        float cm0 = 0.f, cm1 = 0.f;                          // this lane's keys' cut mass for rows (lane%4)*2 + {0,1}
+        uint2 mean8 = make_uint2(0u, 0u);
         uint32_t fetch = 0;                                  // bit 16 u + k: key k of sub-slice u is live for some row
 #pragma unroll
         for (int u = 0; u < U; ++u) bh[u][0] = bh[u][1] = bl[u][0] = bl[u][1] = 0u;
         if (ready) {
           float s[U][4];
 #pragma unroll
-          for (int u = 0; u < U; ++u) qk_issue_n<D, TK>(rb, base + my_stage * LO::kKTile, sl * U + u, lane, s[u]);
+          for (int u = 0; u < U; ++u) qk_issue_n<D, TK>(rb, base + my_stage * LO::kKStage, sl * U + u, lane, s[u]);
+          if (TAIL && lane * 8 < D * 2)                      // this lane's 8 bytes of the slice's block mean row
+            mean8 = *reinterpret_cast<const uint2 *>(gen + my_stage * LO::kKStage + LO::kKTile +
+                                                     ((sl * KS) / 64) * (D * 2) + lane * 8);
           __syncwarp();
           if (lane == 0) mbar_arrive(empty0 + 8u * my_stage); // the K slice is consumed: release the tile
 #pragma unroll
           for (int u = 0; u < U; ++u)
-            fetch |= weights_n<D, true>(rb, s[u], lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh[u], bl[u], l0, l1) << (16 * u);
+            fetch |= weights_n<D, true, TAIL>(rb, s[u], lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh[u], bl[u], l0, l1,
+                                              &cm0, &cm1) << (16 * u);
         }
+        const bool tail = TAIL && __any_sync(0xffffffffu, cm0 > 0.f || cm1 > 0.f);
         // a mostly-live sub-slice is cheaper to fetch whole (one TMA box per 64 channels) than row by row; rows nobody
         // keeps then ride along under a zero weight.  Never past the sequence end: those rows may hold anything.
         uint32_t whole = 0;
@@ -1063,7 +1090,11 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
 #pragma unroll
           for (int u = 0; u < U; ++u)
             *reinterpret_cast<uint4 *>(pe + u * 512 + lane * 16) = make_uint4(bh[u][0], bh[u][1], bl[u][0], bl[u][1]);
-          if (lane == 0) *reinterpret_cast<uint32_t *>(pe + pmask) = fetch;
+          if (TAIL && tail) {
+            *reinterpret_cast<float2 *>(pe + pcut + lane * 8) = make_float2(cm0, cm1);
+            if (lane * 8 < D * 2) *reinterpret_cast<uint2 *>(pe + pmean + lane * 8) = mean8;
+          }
+          if (lane == 0) *reinterpret_cast<uint2 *>(pe + pmask) = make_uint2(fetch, tail ? 1u : 0u);
           const uint32_t bar = vfull + 8u * my_vs;
           const uint32_t vdst = vring + my_vs * LO::kVSlice;
           if (whole) {
@@ -1133,13 +1164,29 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       if (++vs == vr) { vs = 0; vphase ^= 1u; }
       if (landed) {
         const uint8_t *pe = pring + my * pentry;
-        const uint32_t verdict = *reinterpret_cast<const uint32_t *>(pe + pmask);
+        const uint2 vw = *reinterpret_cast<const uint2 *>(pe + pmask);
+        const uint32_t verdict = vw.x;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           if (((verdict >> (16 * u)) & 0xffffu) == 0u) continue;   // nobody keeps a key of this sub-slice
           const uint4 a = *reinterpret_cast<const uint4 *>(pe + u * 512 + lane * 16);
           const uint32_t bh[2] = {a.x, a.y}, bl[2] = {a.z, a.w};
           value_product_n<D, true, 0, KS>(o, vring + my * LO::kVSlice, 16 * u, lane, bh, bl);
+        }
+        if (TAIL && vw.y != 0u) {                            // o[mt]: channels 16 mt + lane/4 (+8), rows (lane%4)*2 + {0,1}
+          float2 c = make_float2(0.f, 0.f);                  // the rows' cut mass: over the 8 lanes that scored their keys
+#pragma unroll
+          for (int gsrc = 0; gsrc < 8; ++gsrc) {
+            const float2 t = *reinterpret_cast<const float2 *>(pe + pcut + (gsrc * 4 + (lane & 3)) * 8);
+            c.x += t.x; c.y += t.y;
+          }
+          const __nv_bfloat16 *mrow = reinterpret_cast<const __nv_bfloat16 *>(pe + pmean) + (lane >> 2);
+#pragma unroll
+          for (int mt = 0; mt < D / 16; ++mt) {
+            const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
+            o[mt][0] = fmaf(c.x, m0, o[mt][0]); o[mt][1] = fmaf(c.y, m0, o[mt][1]);
+            o[mt][2] = fmaf(c.x, m1, o[mt][2]); o[mt][3] = fmaf(c.y, m1, o[mt][3]);
+          }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(vempty + 8u * my);

@@ -25,12 +25,26 @@ Z_TOL = 1e-3
 LSE_TOL = 2e-3
 
 
-def cache_of(w: DecodeWorkload) -> F.KVCache:
-    return F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table)
+def cache_of(w: DecodeWorkload, v_block_mean=None) -> F.KVCache:
+    return F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table, v_block_mean)
 
 
-def run_gpu(w: DecodeWorkload, T=math.inf, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, bufs=None):
-    cache = cache_of(w)
+def oracle_block_means(w: DecodeWorkload) -> torch.Tensor:
+    """The block-mean table of a workload computed by the ORACLE (float64, rounded to BF16), as a device
+    tensor [num_seqs, blocks, Hkv, D]: the block tail's input in the parity tests."""
+    nb = max((w.max_seqlen + 63) // 64, 1)
+    t = torch.zeros(w.num_seqs, nb, w.num_kv_heads, w.head_dim, dtype=torch.float32)
+    for s in range(w.num_seqs):
+        for h in range(w.num_kv_heads):
+            V = O.widen_bf16(bf16_bits(w.logical_rows("v", s, h)))
+            if V.shape[0]:
+                m = O.block_means(V)
+                t[s, :m.shape[0], h] = torch.from_numpy(m).float()
+    return t.to(torch.bfloat16).to(w.k.device)                # exact: the oracle's means are BF16 values already
+
+
+def run_gpu(w: DecodeWorkload, T=math.inf, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, bufs=None, v_block_mean=None):
+    cache = cache_of(w, v_block_mean)
     if bufs is None:
         bufs = F.alloc_buffers(w.q, cache, w.stack)
     if z is not None:
@@ -54,9 +68,13 @@ def all_rows(w: DecodeWorkload):
     return [(b, h) for b in range(w.batch) for h in range(w.num_q_heads)]
 
 
-def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False, yardstick=True):
+def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False, yardstick=True, v_block_mean=None):
     """Element-by-element comparison of the CUDA outputs with the oracle run at the GPU's own
-    references.  Returns a dict of the measured errors; asserts the tolerances."""
+    references.  Returns a dict of the measured errors; asserts the tolerances.  `v_block_mean`
+    (the table the GPU was given) switches the oracle's block tail on; a key that flips at the threshold
+    then moves between its value and its block's mean, so the threshold slack counts twice."""
+    vm = None if v_block_mean is None else v_block_mean.float().cpu().numpy().astype(np.float64)
+    G = w.num_q_heads // w.num_kv_heads
     out = bufs.out.float().cpu().numpy().astype(np.float64)
     lse = bufs.lse.cpu().numpy().astype(np.float64)
     z = bufs.z.cpu().numpy().astype(np.float64)
@@ -73,7 +91,8 @@ def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False
             assert not out[b, h].any() and lse[b, h] == -np.inf and status[b, h] == F.ROW_EMPTY
             continue
         s = O.scores(q, K, w.scale)
-        o_ref, lse_ref, _, L = O.fold_row(s, V, z[b, h], T)
+        v_mean = None if vm is None else vm[b // w.stack, :(n + 63) // 64, h // G]
+        o_ref, lse_ref, _, L = O.fold_row(s, V, z[b, h], T, v_mean=v_mean)
         d = out[b, h] - o_ref
         num += float(d @ d); den += float(o_ref @ o_ref)
         max_abs = max(max_abs, float(np.abs(d).max())); vmax = max(vmax, float(np.abs(V).max()))
@@ -84,7 +103,7 @@ def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False
         if check_estimate:
             dz = max(dz, abs(O.estimate_z(lambda i: s[i], n) - z[b, h]))
         if not math.isinf(T):
-            slack_sum += O.cut_report(s, V, z[b, h], T)["slack"] ** 2 * V.shape[1]
+            slack_sum += ((2.0 if vm is not None else 1.0) * O.cut_report(s, V, z[b, h], T)["slack"]) ** 2 * V.shape[1]
             if yardstick:
                 o_dense, _ = O.dense_row(s, V)
                 y = O.online_softmax_bf16(q, K, V, w.scale) - o_dense
