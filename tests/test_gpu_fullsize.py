@@ -49,6 +49,25 @@ def test_config3_paged_128k_sampled_rows():
     torch.cuda.empty_cache()
 
 
+def test_config3_with_the_block_tail_sampled_rows():
+    if _free_gb() < 12:
+        pytest.skip("not enough free device memory")
+    w = make_decode_workload(4, 32, 8, 128, 131072, seed=2, device=DEV, paged=True, page_size=64)
+    cache = cache_of(w)
+    vm = F.fold_block_means(cache)                           # the library's table; sampled heads checked bit for bit
+    torch.cuda.synchronize()
+    for (s, kvh) in [(0, 1), (3, 7)]:
+        V = O.widen_bf16(bf16_bits(w.logical_rows("v", s, kvh)))
+        ref = torch.from_numpy(O.block_means(V)).float().to(torch.bfloat16).to(DEV)
+        assert same_bits(vm[s, :, kvh], ref)
+    rows = [(0, 5), (3, 28)]
+    b = run_gpu(w, T=16.0, v_block_mean=vm)
+    compare(w, b, T=16.0, rows=rows, v_block_mean=vm)
+    assert same_bits(run_gpu(w, T=16.0, num_splits=32, v_block_mean=vm).out, b.out.clone())
+    del w, vm, cache
+    torch.cuda.empty_cache()
+
+
 def test_config4_shared_prefix_cascade_sampled_rows():
     if _free_gb() < 8:
         pytest.skip("not enough free device memory")
