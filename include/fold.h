@@ -82,8 +82,8 @@ enum {
  * at finite depth then adds, for every row, the summed weight of the keys that row cuts in a block
  * times that block's mean to A, instead of nothing (Algorithm 1: "add the weights of cut keys to the
  * tile's virtual row").  fold_block_means() fills the table from the cache; keeping it current when
- * tokens are appended is the caller's business (only the last block changes).  Supported where up to
- * 8 query rows share a (sequence, kv head); other shapes return FOLD_EUNSUPPORTED when it is set.
+ * tokens are appended is the caller's business (only the last block changes).  Every row-block and
+ * stacked-row shape takes it (a stacked level with a table runs on the mma.sync kernel, not on tcgen05).
  * Ignored at depth_T = INFINITY (nothing is cut). */
 typedef struct fold_kv {
   const void *k, *v;

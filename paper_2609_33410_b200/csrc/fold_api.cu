@@ -68,8 +68,6 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   const int G = a->num_q_heads / a->num_kv_heads;
   const long long R = (long long)a->stack * G;
   if (G > kMaxRows || R > kMaxStackedRows) return FOLD_EUNSUPPORTED;
-  // the block tail is built into the narrow row-block scan only
-  if (a->kv.v_block_mean && !isinf(a->depth_T) && R > kNarrowRows) return FOLD_EUNSUPPORTED;
   g->B = a->batch; g->Hq = a->num_q_heads; g->Hkv = a->num_kv_heads; g->G = G; g->D = a->head_dim;
   g->stack = a->stack; g->R = (int)R; g->num_seqs = a->kv.num_seqs;
   g->max_slots = max_chunks_upto(a->kv.max_seqlen);
@@ -238,28 +236,30 @@ int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, di
   return p.R <= kNarrowRows ? launch_dense_as<D, true>(mk, mv, p, grid, st) : launch_dense_as<D, false>(mk, mv, p, grid, st);
 }
 
-// Stacked rows: the dense ring without reduction buffers; one CTA per (split, 64-row group).
-template <int D>
-int launch_stacked(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, bool gated, cudaStream_t st) {
+// Stacked rows: the dense ring without reduction buffers; one CTA per (split, 64-row group).  With the block tail
+// every stage also carries the tile's block-mean row (1 KB more per stage).
+template <int D, bool GATED, bool TAIL>
+int launch_stacked_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
   using LO = DenseLayout<D>;
+  constexpr int kStageBytes = LO::kStage + (TAIL ? 1024 : 0);
   const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
-  int stages = (per_cta2 - LO::total(0, 0)) / (LO::kStage + 16);
+  int stages = (per_cta2 - LO::total(0, 0)) / (kStageBytes + 16);
   if (stages > 8) stages = 8;
   if (stages < 2) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = 0;
   grid.x *= (p.R + 63) / 64;
-  static int configured_g[64] = {0}, configured_d[64] = {0};
-  cudaError_t rc;
-  if (gated) {
-    if (int e = opt_in_smem(fold_scan_stacked_kernel<D, true>, configured_g)) return e;
-    rc = launch_pdl(fold_scan_stacked_kernel<D, true>, grid, dim3(kDenseThreads), LO::total(stages, 0), st, mk, mv, p);
-  } else {
-    if (int e = opt_in_smem(fold_scan_stacked_kernel<D, false>, configured_d)) return e;
-    rc = launch_pdl(fold_scan_stacked_kernel<D, false>, grid, dim3(kDenseThreads), LO::total(stages, 0), st, mk, mv, p);
-  }
-  if (rc != cudaSuccess) return FOLD_ECUDA;
+  static int configured[64] = {0};
+  if (int e = opt_in_smem(fold_scan_stacked_kernel<D, GATED, TAIL>, configured)) return e;
+  if (launch_pdl(fold_scan_stacked_kernel<D, GATED, TAIL>, grid, dim3(kDenseThreads),
+                 LO::total(stages, 0) + stages * (kStageBytes - LO::kStage), st, mk, mv, p) != cudaSuccess)
+    return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+template <int D>
+int launch_stacked(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, bool gated, cudaStream_t st) {
+  if (!gated) return launch_stacked_as<D, false, false>(mk, mv, p, grid, st);
+  return p.vmean ? launch_stacked_as<D, true, true>(mk, mv, p, grid, st) : launch_stacked_as<D, true, false>(mk, mv, p, grid, st);
 }
 
 // Stacked rows on tcgen05 (head_dim 128, at least 64 stacked rows): one CTA per (split, 128-row tile).
@@ -326,17 +326,15 @@ int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParam
 
 // Gated scan: value slots hold rows whose requests can only be issued after scoring, so shared
 // memory is split between the key ring and the value slots of each slice.
-template <int D>
-int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
-  if (p.R <= kNarrowRows)                                    // rows on N; with or without the block tail
-    return p.vmean ? launch_gated_narrow<D, true>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false>(mk, mvs, p, grid, st);
-  using LO = GatedLayout<D>;
+template <int D, bool TAIL>
+int launch_gated_wide(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LO = GatedLayout<D, TAIL>;
   const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
   int vr = 2;
-  int stages = (per_cta2 - LO::total(0, vr, p.R)) / (LO::kKTile + 16);
+  int stages = (per_cta2 - LO::total(0, vr, p.R)) / (LO::kKStage + 16);
   if (stages < 2) {
     vr = 3;
-    stages = (kSmemPerCtaMax - LO::total(0, vr, p.R)) / (LO::kKTile + 16);
+    stages = (kSmemPerCtaMax - LO::total(0, vr, p.R)) / (LO::kKStage + 16);
   }
   if (stages > 8) stages = 8;
 #ifdef FOLD_TUNING
@@ -348,10 +346,17 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
   p.stages = stages;
   p.vr = vr;
   static int configured[64] = {0};
-  if (int rc = opt_in_smem(fold_scan_gated_kernel<D>, configured)) return rc;
-  if (launch_pdl(fold_scan_gated_kernel<D>, grid, dim3(kGatedThreads), LO::total(stages, vr, p.R), st, mk, mvs, p) != cudaSuccess)
+  if (int rc = opt_in_smem(fold_scan_gated_kernel<D, TAIL>, configured)) return rc;
+  if (launch_pdl(fold_scan_gated_kernel<D, TAIL>, grid, dim3(kGatedThreads), LO::total(stages, vr, p.R), st, mk, mvs, p) !=
+      cudaSuccess)
     return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+template <int D>
+int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
+  if (p.R <= kNarrowRows)                                    // rows on N; with or without the block tail
+    return p.vmean ? launch_gated_narrow<D, true>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false>(mk, mvs, p, grid, st);
+  return p.vmean ? launch_gated_wide<D, true>(mk, mvs, p, grid, st) : launch_gated_wide<D, false>(mk, mvs, p, grid, st);
 }
 
 // CTAs per (sequence, kv head).  A CTA pays a few microseconds to start (barriers, first loads), so it should
@@ -414,8 +419,10 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const dim3 grid = stacked ? dim3(p.num_splits, g.Hkv, g.num_seqs) : dim3(g.Hkv, p.num_splits, g.num_seqs);
   p.box_min = 13;
   if (stacked) {
-    if (g.D == 128 && g.R > kUmmaRows) return launch_stacked_pair(mk, mv, p, grid, gated, st);
-    if (g.D == 128 && g.R >= 64) return launch_stacked_umma(mk, mv, p, grid, gated, st);
+    // the tcgen05 kernels have no block tail yet: a gated stacked level with a mean table runs on mma.sync
+    const bool tail = gated && p.vmean != nullptr;
+    if (g.D == 128 && g.R > kUmmaRows && !tail) return launch_stacked_pair(mk, mv, p, grid, gated, st);
+    if (g.D == 128 && g.R >= 64 && !tail) return launch_stacked_umma(mk, mv, p, grid, gated, st);
     return g.D == 128 ? launch_stacked<128>(mk, mv, p, grid, gated, st) : launch_stacked<64>(mk, mv, p, grid, gated, st);
   }
   if (g.D == 128) return gated ? launch_gated<128>(mk, mv, p, grid, st) : launch_dense<128>(mk, mv, p, grid, st);

@@ -70,16 +70,18 @@ struct DenseLayout {
   __host__ __device__ static int total(int stages, int R) { return off_bar(stages, R) + 2 * stages * 8 + 1024; }
 };
 
-template <int D>
+template <int D, bool TAIL = false>
 struct GatedLayout {
   static constexpr int kKTile = kTileKeys * D * 2;
+  static constexpr int kKStage = kKTile + (TAIL ? 1024 : 0);   // K tile (+ the block's mean row)
   static constexpr int kVRow = D * 2 + 16;          // value row + 16 B pad: conflict-free ldmatrix
   // one slice's 16 value rows: padded rows (row-by-row fetch) or a swizzled TMA box (whole slice),
   // so the slot is 1 KB aligned
   static constexpr int kVSlice = ((16 * kVRow + 1023) / 1024) * 1024;
   // a slice's weights as A-operand registers (hi and lo terms; rows 8..15 only when present) + its fetch mask
-  __host__ __device__ static int pentry(int R) { return (R > 8 ? 1024 : 512) + 32; }
-  __host__ __device__ static int off_vring(int stages) { return stages * kKTile; }
+  // with the block tail: + every lane's cut mass of its two rows (256 B) + the block's mean row (256 B)
+  __host__ __device__ static int pentry(int R) { return (R > 8 ? 1024 : 512) + (TAIL ? 512 : 0) + 32; }
+  __host__ __device__ static int off_vring(int stages) { return stages * kKStage; }
   __host__ __device__ static int off_pring(int stages, int vr) { return off_vring(stages) + kConsumerWarps * vr * kVSlice; }
   __host__ __device__ static int off_red(int stages, int vr, int R) { return off_pring(stages, vr) + kConsumerWarps * vr * pentry(R); }
   __host__ __device__ static int off_redl(int stages, int vr, int R) { return off_red(stages, vr, R) + kConsumerWarps * R * D * 4; }
@@ -181,7 +183,8 @@ __device__ __forceinline__ void produce_tiles(const CUtensorMap *tmK, const CUte
     if (WITH_MEAN) {
       const __nv_bfloat16 *m = p.vmean + (long long)seq * p.vm_stride_seq + (long long)(tok0 / 64) * p.vm_stride_block +
                                (long long)kvh * p.vm_stride_head;
-      for (int i = 0; i < nmean; ++i) bulk_load(kdst + KTILE + i * (D * 2), m + (long long)i * p.vm_stride_block, D * 2, full);
+      for (int i = 0; i < nmean; ++i)
+        bulk_load(kdst + KTILE * (WITH_V ? 2 : 1) + i * (D * 2), m + (long long)i * p.vm_stride_block, D * 2, full);
     }
     const uint32_t vdst = kdst + KTILE;
     for (int bx = 0; bx < nbox; ++bx) {
@@ -241,10 +244,12 @@ __device__ __forceinline__ void load_rows(RowBlock<D> &rb, const ScanParams &p, 
 // Returns the slice's fetch mask (bit k: key k is live for some row); ah / al receive the
 // two-term BF16 weights as A-operand fragments of the value product; l_lo / l_hi accumulate
 // this thread's share of L.
-template <int D, bool GATED>
+// TAIL: c_lo / c_hi also accumulate the weight of this thread's cut keys for its two rows (block tail).
+template <int D, bool GATED, bool TAIL = false>
 __device__ __forceinline__ uint32_t score_slice(const RowBlock<D> &rb, uint32_t kt, int warp, int lane, int key0,
                                                 int n, float scale_log2, float neg_T, uint32_t (&ah)[4],
-                                                uint32_t (&al)[4], float &l_lo, float &l_hi) {
+                                                uint32_t (&al)[4], float &l_lo, float &l_hi, float *c_lo = nullptr,
+                                                float *c_hi = nullptr) {
   // S[rows, 16 keys] = Q K^T.  Lane l addresses key row (l>>4)*8 + (l&7), 16-byte chunk 2*kk + ((l>>3)&1)
   // of the tile laid out [half][key][128 B] with the 128-byte swizzle.
   const int k_key = warp * 16 + ((lane >> 4) << 3) + (lane & 7);
@@ -286,6 +291,10 @@ __device__ __forceinline__ uint32_t score_slice(const RowBlock<D> &rb, uint32_t 
       const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
       const float add = ((h0 + g0) + (pw[0] - pm[0])) + ((h1 + g1) + (pw[1] - pm[1]));
       if (blk) l_hi += add; else l_lo += add;
+      if (TAIL) {
+        const float cut = (pw[0] - pm[0]) + (pw[1] - pm[1]);
+        if (blk) *c_hi += cut; else *c_lo += cut;
+      }
       ah[nt * 2 + blk] = hi2;
       al[nt * 2 + blk] = lo2;
     }
@@ -310,6 +319,20 @@ __device__ __forceinline__ void value_product(float (&o)[D / 8][4], uint32_t vba
     mma_bf16(o[2 * pr], al, b0, b1);
     mma_bf16(o[2 * pr + 1], ah, b2, b3);
     mma_bf16(o[2 * pr + 1], al, b2, b3);
+  }
+}
+
+// Block tail for rows-on-M accumulators: o[nt] holds rows lane/4 (elements 0, 1) and lane/4 + 8 (elements 2, 3),
+// channels 8 nt + (lane%4)*2 + {0,1}.  c_lo / c_hi: the two rows' cut mass; mean: the block's mean value row.
+template <int D>
+__device__ __forceinline__ void tail_update(float (&o)[D / 8][4], float c_lo, float c_hi, const __nv_bfloat16 *mean, int lane) {
+  const uint32_t *m2 = reinterpret_cast<const uint32_t *>(mean) + (lane & 3);
+#pragma unroll
+  for (int nt = 0; nt < D / 8; ++nt) {
+    const uint32_t w = m2[nt * 4];
+    const float m0 = __uint_as_float(w << 16), m1 = __uint_as_float(w & 0xffff0000u);
+    o[nt][0] = fmaf(c_lo, m0, o[nt][0]); o[nt][1] = fmaf(c_lo, m1, o[nt][1]);
+    o[nt][2] = fmaf(c_hi, m0, o[nt][2]); o[nt][3] = fmaf(c_hi, m1, o[nt][3]);
   }
 }
 
@@ -661,12 +684,15 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 // skipped -- and each of the four consumer warps owns a 16-row block and walks all four slices of
 // every tile.  A CTA covers 64 rows; CTAs of the same tile stream share it through L2.  The depth
 // gate still applies row by row.  Each warp writes its own rows of the chunk slot: no cross-warp add.
-template <int D, bool GATED>
+// TAIL (with GATED): the tile's block-mean row rides behind the V tile; a warp sums its rows' cut mass over the tile
+// (= one 64-key block) and adds cut mass x mean once per tile.
+template <int D, bool GATED, bool TAIL = false>
 __global__ void __launch_bounds__(kDenseThreads, 2)
 fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                          const ScanParams p) {
   using LO = DenseLayout<D>;
   constexpr int C16 = D / 8;
+  constexpr int STAGE = LO::kStage + (TAIL ? 1024 : 0);      // K tile, V tile (, the block's mean row)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -679,7 +705,8 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   const SeqWork w = seq_work(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, R = p.R, n = w.n;
-  const uint32_t full0 = base + LO::off_bar(stages, 0), empty0 = full0 + 8u * stages;
+  // the ring's stages are STAGE bytes apart; what follows it keeps its place relative to the ring's end
+  const uint32_t full0 = base + stages * (STAGE - LO::kStage) + LO::off_bar(stages, 0), empty0 = full0 + 8u * stages;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -693,7 +720,7 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   pdl_wait();
 
   if (warp == kConsumerWarps) {
-    if (lane == 0) produce_tiles<D, true, LO::kStage>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
+    if (lane == 0) produce_tiles<D, true, STAGE, kTileKeys, TAIL>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
     return;
   }
 
@@ -713,22 +740,30 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
     const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
     if (++stage == stages) { stage = 0; phase ^= 1u; }
     if (ready) {
-      const uint32_t kt = base + my_stage * LO::kStage;
+      const uint32_t kt = base + my_stage * STAGE;
       if (k.t * kTileKeys + kTileKeys > n) {                 // ragged tail: value rows past n may hold anything
         // every warp reads every row: warp w clears the rows of slice w, then all four meet
         for (int r = 0; r < 16; ++r)
           if (k.t * kTileKeys + warp * 16 + r >= n && lane < C16)
-            *reinterpret_cast<uint4 *>(gen + my_stage * LO::kStage + LO::kKTile +
+            *reinterpret_cast<uint4 *>(gen + my_stage * STAGE + LO::kKTile +
                                        tile_off(warp * 16 + r, lane, kTileKeys)) = make_uint4(0, 0, 0, 0);
         named_bar(1);
       }
+      float c_lo = 0.f, c_hi = 0.f;                          // this tile's cut mass of the thread's two rows
 #pragma unroll 1
       for (int sl = 0; sl < 4; ++sl) {
         const int key0 = k.t * kTileKeys + sl * 16;
         if (key0 >= n) break;
         uint32_t ah[4], al[4];
-        const uint32_t live16 = score_slice<D, GATED>(rb, kt, sl, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        const uint32_t live16 = score_slice<D, GATED, TAIL>(rb, kt, sl, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo,
+                                                              l_hi, &c_lo, &c_hi);
         if (live16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, sl * 16, lane, ah, al);
+      }
+      if (TAIL) {
+        c_lo += __shfl_xor_sync(0xffffffffu, c_lo, 1); c_lo += __shfl_xor_sync(0xffffffffu, c_lo, 2);
+        c_hi += __shfl_xor_sync(0xffffffffu, c_hi, 1); c_hi += __shfl_xor_sync(0xffffffffu, c_hi, 2);
+        if (__any_sync(0xffffffffu, c_lo > 0.f || c_hi > 0.f))
+          tail_update<D>(o, c_lo, c_hi, reinterpret_cast<const __nv_bfloat16 *>(gen + my_stage * STAGE + LO::kStage), lane);
       }
       if (k.t * kTileKeys + kTileKeys > n) fence_proxy_async_smem();
       __syncwarp();
@@ -774,11 +809,13 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 // its slice's value ring -- the whole slice by TMA when most rows are live, else row by row
 // with zero-filling 16-byte async copies (cut rows are not read and become zero rows).
 // Multiplier warp w: waits for a slot to land, multiplies, hands the slot back.
-template <int D>
+// TAIL: the block tail, as in the narrow kernel below (mean rows ride with the K tiles; the scorer publishes every
+// lane's cut mass and the block's mean row with the slice; the multiplier adds cut mass x mean).
+template <int D, bool TAIL>
 __global__ void __launch_bounds__(kGatedThreads, 2)
 fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
                        const ScanParams p) {
-  using LO = GatedLayout<D>;
+  using LO = GatedLayout<D, TAIL>;
   constexpr int C16 = D / 8;                                 // 16-byte chunks per value row
   constexpr int RPI = 32 / C16;                              // rows one warp-wide async copy covers
   extern __shared__ uint8_t smem_raw[];
@@ -812,13 +849,13 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   pdl_wait();                                                // z (and the zeroed header) come from earlier work
 
   if (warp == 2 * kConsumerWarps) {
-    if (lane == 0) produce_tiles<D, false, LO::kKTile>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
+    if (lane == 0) produce_tiles<D, false, LO::kKStage, kTileKeys, TAIL>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
     return;
   }
 
   const bool scorer = warp < kConsumerWarps;
   const int sl = warp & 3;                                   // the slice of every tile this warp owns
-  const int pentry = LO::pentry(R), pmask = pentry - 32;
+  const int pentry = LO::pentry(R), pmask = pentry - 32, pcut = pmask - 512, pmean = pmask - 256;
   uint8_t *pring = gen + LO::off_pring(stages, vr) + sl * vr * pentry;
   const uint32_t vring = base + LO::off_vring(stages) + sl * vr * LO::kVSlice;
   const uint32_t vfull = vfull0 + 8u * sl * vr, vempty = vempty0 + 8u * sl * vr;
@@ -847,9 +884,13 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       const int key0 = k.t * kTileKeys + sl * 16;
       uint32_t ah[4] = {0u, 0u, 0u, 0u}, al[4] = {0u, 0u, 0u, 0u};
       uint32_t fetch16 = 0;
+      float c_lo = 0.f, c_hi = 0.f;                          // this lane's keys' cut mass for its two rows
+      uint2 mean8 = make_uint2(0u, 0u);
       if (ready) {
-        fetch16 = score_slice<D, true>(rb, base + my_stage * LO::kKTile, sl, lane, key0, n,
-                                                            p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        fetch16 = score_slice<D, true, TAIL>(rb, base + my_stage * LO::kKStage, sl, lane, key0, n, p.scale_log2, p.neg_T, ah,
+                                             al, l_lo, l_hi, &c_lo, &c_hi);
+        if (TAIL && lane * 8 < D * 2)                        // this lane's 8 bytes of the tile's block mean row
+          mean8 = *reinterpret_cast<const uint2 *>(gen + my_stage * LO::kKStage + LO::kKTile + lane * 8);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);   // the K tile is in registers: release it
       }
@@ -871,7 +912,12 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         } else {
           *reinterpret_cast<uint4 *>(pe + lane * 16) = make_uint4(ah[0], ah[2], al[0], al[2]);
         }
-        if (lane == 0) *reinterpret_cast<uint32_t *>(pe + pmask) = fetch16 | (whole ? 0x10000u : 0u);
+        const bool tail = TAIL && __any_sync(0xffffffffu, c_lo > 0.f || c_hi > 0.f);
+        if (TAIL && tail) {
+          *reinterpret_cast<float2 *>(pe + pcut + lane * 8) = make_float2(c_lo, c_hi);
+          if (lane * 8 < D * 2) *reinterpret_cast<uint2 *>(pe + pmean + lane * 8) = mean8;
+        }
+        if (lane == 0) *reinterpret_cast<uint2 *>(pe + pmask) = make_uint2(fetch16 | (whole ? 0x10000u : 0u), tail ? 1u : 0u);
         const uint32_t bar = vfull + 8u * vs;
         if (fetch16 != 0u) {
           int c_seq = seq, c_tok = key0;
@@ -936,7 +982,8 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       if (++vs == vr) { vs = 0; vphase ^= 1u; }
       if (landed) {
         const uint8_t *pe = pring + my * pentry;
-        const uint32_t verdict = *reinterpret_cast<const uint32_t *>(pe + pmask);
+        const uint2 vw = *reinterpret_cast<const uint2 *>(pe + pmask);
+        const uint32_t verdict = vw.x;
         if (verdict != 0u) {
           uint32_t ah[4], al[4];
           const uint4 a = *reinterpret_cast<const uint4 *>(pe + lane * 16);
@@ -950,6 +997,15 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           }
           if (verdict & 0x10000u) value_product<D, true, 0, 16>(o, vring + my * LO::kVSlice, 0, lane, ah, al);
           else value_product<D, false, LO::kVRow>(o, vring + my * LO::kVSlice, 0, lane, ah, al);
+        }
+        if (TAIL && vw.y != 0u) {                            // the rows' cut mass: over the four lanes that scored their keys
+          float c_lo = 0.f, c_hi = 0.f;
+#pragma unroll
+          for (int qsrc = 0; qsrc < 4; ++qsrc) {
+            const float2 t = *reinterpret_cast<const float2 *>(pe + pcut + ((lane & ~3) + qsrc) * 8);
+            c_lo += t.x; c_hi += t.y;
+          }
+          tail_update<D>(o, c_lo, c_hi, reinterpret_cast<const __nv_bfloat16 *>(pe + pmean), lane);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(vempty + 8u * my);

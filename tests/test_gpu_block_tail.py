@@ -78,13 +78,64 @@ def test_block_tail_is_exact_for_values_constant_within_blocks():
     assert bool(shallow.header().v_rows_fetched < 0.6 * shallow.header().v_rows_total)
 
 
-def test_block_tail_is_refused_where_it_is_not_built():
-    w = make_decode_workload(1, 16, 1, 128, [500], seed=89, device=DEV)        # 16 rows per kv head
+@pytest.mark.parametrize("Hq,Hkv,stack,D", [(16, 1, 1, 128), (12, 1, 1, 64), (8, 2, 4, 128), (8, 2, 5, 128), (4, 4, 33, 64),
+                                            (8, 2, 40, 128)])
+def test_block_tail_with_wider_row_blocks_and_stacked_rows(Hq, Hkv, stack, D):
+    # 9..16 rows per (sequence, kv head): the rows-on-M gated kernel; more: the stacked-row kernel
+    w = make_decode_workload(2 * stack, Hq, Hkv, D, [1500, 333], seed=91, device=DEV, stack=stack,
+                             poison_padding=True, capacity=1600)
     vm = oracle_block_means(w)
-    cache = cache_of(w, vm)
-    bufs = F.alloc_buffers(w.q, cache)
-    with pytest.raises(F.FoldError) as e:
-        F.decode(w.q, cache, bufs, depth_T=16.0)
-    assert e.value.status == F.FOLD_EUNSUPPORTED
-    F.decode(w.q, cache, bufs, depth_T=math.inf)               # dense decode ignores the table
+    rows = [(b, h) for b in (0, stack - 1, stack, 2 * stack - 1) for h in (0, Hq - 1)]
+    for T in (8.0, 14.0):
+        b = run_gpu(w, T=T, v_block_mean=vm)
+        compare(w, b, T=T, rows=rows, v_block_mean=vm)
+        plain = run_gpu(w, T=T, z_mode=F.Z_GIVEN, z=b.z.clone())
+        # the mass is the same either way (a stacked level without the table may run on another kernel: not the same bits)
+        assert torch.allclose(plain.lse, b.lse, atol=1e-4, rtol=0)
+        if T == 8.0:
+            assert not torch.equal(plain.out, b.out)
+    b1 = run_gpu(w, T=14.0, num_splits=1, v_block_mean=vm)
+    assert same_bits(b1.out, b.out)
+
+
+def test_block_tail_in_a_shared_prefix_cascade():
+    # each level has its own table (blocks are local to a level's sequence); the oracle walks prefix ++ suffix with
+    # the two tables one after the other
+    B, Hq, Hkv, D, P = 6, 8, 2, 128, 1000
+    suffixes = [300, 1, 0, 257, 64, 65]
+    g = torch.Generator(device=DEV); g.manual_seed(93)
+    q = torch.randn(B, Hq, D, generator=g, device=DEV).to(torch.bfloat16)
+    pre = make_decode_workload(B, Hq, Hkv, D, P, seed=94, device=DEV, stack=B, q=q)
+    suf = make_decode_workload(B, Hq, Hkv, D, suffixes, seed=95, device=DEV, q=q, sink_gain=1.0)
+    vmp, vms = oracle_block_means(pre), oracle_block_means(suf)
+    cp, cs = cache_of(pre, vmp), cache_of(suf, vms)
+    bp, bs = F.alloc_buffers(q, cp, stack=B), F.alloc_buffers(q, cs)
+    T = 10.0
+    ap = F.make_args(q, cp, z=bs.z, depth_T=T, stack=B, workspace=bp.workspace, out=bs.out, lse=bs.lse,
+                     row_status=bs.row_status)
+    as_ = F.make_args(q, cs, z=bs.z, depth_T=T, workspace=bs.workspace, out=bs.out, lse=bs.lse, row_status=bs.row_status)
+    F.fold_decode_cascade([ap, as_])
     torch.cuda.synchronize()
+    assert bp.header().wait_timeouts == 0 and bs.header().wait_timeouts == 0
+    out = bs.out.float().cpu().numpy().astype(np.float64)
+    z = bs.z.cpu().numpy().astype(np.float64)
+    mp, ms = vmp.float().cpu().numpy().astype(np.float64), vms.float().cpu().numpy().astype(np.float64)
+    nbp = (P + 63) // 64
+    num = den = 0.0
+    for b in range(B):
+        for h in (0, 3, 7):
+            kvh = h // (Hq // Hkv)
+            n_s = suffixes[b]
+            K = np.concatenate([O.widen_bf16(bf16_bits(pre.logical_rows("k", 0, kvh))),
+                                O.widen_bf16(bf16_bits(suf.logical_rows("k", b, kvh)))])
+            V = np.concatenate([O.widen_bf16(bf16_bits(pre.logical_rows("v", 0, kvh))),
+                                O.widen_bf16(bf16_bits(suf.logical_rows("v", b, kvh)))])
+            s = O.scores(O.widen_bf16(bf16_bits(q[b, h])), K)
+            table = np.concatenate([mp[0, :nbp, kvh], ms[b, :(n_s + 63) // 64, kvh]])
+            block_of = np.concatenate([np.arange(P) // 64, nbp + np.arange(n_s) // 64])
+            A, L = O.fold_partial(s, V, z[b, h], T, tail=(table, block_of))
+            d = out[b, h] - A / L
+            num += d @ d; den += (A / L) @ (A / L)
+    assert math.sqrt(num / den) < 4e-3
+
+
