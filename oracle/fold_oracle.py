@@ -16,6 +16,9 @@ What is here, with the passage each function restates:
   dense_row             Section 2: o = sum_j 2^s_j v_j / sum_j 2^s_j (max-subtracted)
   fold_partial          Eq. 2: F(I) = (A, L) for one key set, plus the depth-T cut
                         of Section 4 "Depth as a dial" (cut keys keep their mass)
+  draft_visible /
+  mask_draft_scores     Section 4 "Value product" (drafts and verification trees are extra query
+                        rows masked to their ancestors): which of the last m keys a row sees
   block_means           Section 4 "Depth as a dial": the mean value of each 64-key block
                         (the block model without its fitted rank-16 map), stored as BF16
   fold_row              Eq. 2 + Prop. 1(i): partials over key ranges, added
@@ -79,6 +82,27 @@ def scores(q: np.ndarray, K: np.ndarray, scale: Optional[float] = None) -> np.nd
 
 
 # --------------------------------------------------------------------------- dense
+def draft_visible(n: int, m: int, mask: int) -> np.ndarray:
+    """Keys a draft / tree-verification row sees (Section 4 "Value product"; Appendix "Cascades and
+    drafts").  The last m keys of the sequence are the draft tokens, already appended to the cache;
+    key n - m + t is visible iff bit t of `mask` is set (the row's ancestors and itself); every
+    earlier key is visible to every row.  If n < m only bits m - n .. m - 1 have a key.  Returns bool [n]."""
+    vis = np.ones(n, dtype=bool)
+    for t in range(m):
+        j = n - m + t
+        if j >= 0 and not (mask >> t) & 1:
+            vis[j] = False
+    return vis
+
+
+def mask_draft_scores(s: np.ndarray, m: int, mask: int) -> np.ndarray:
+    """Scores with the keys the row may not see set to -inf: their weight is exactly 0 in every
+    function of this module (dense, declared-reference, estimator)."""
+    s = np.array(s, dtype=np.float64)
+    s[~draft_visible(s.size, m, mask)] = -np.inf
+    return s
+
+
 def dense_row(s: np.ndarray, V: np.ndarray):
     """Textbook softmax attention of one row from base-2 scores: returns (o [D], lse2).
     The maximum is subtracted only to stay in range (Section 2)."""

@@ -424,3 +424,41 @@ def test_block_tail_reduces_the_truncation_error_on_smooth_values():
     e_plain = np.linalg.norm(O.fold_row(s, V, lse, T)[0] - o_dense)
     e_tail = np.linalg.norm(O.fold_row(s, V, lse, T, v_mean=O.block_means(V))[0] - o_dense)
     assert e_tail < 0.3 * e_plain
+
+
+# ------------------------------------------------------------------ drafts (Section 4 "Value product", Appendix "Cascades and drafts")
+def test_draft_chain_row_equals_attention_over_its_prefix():
+    # draft row r of a chain of m sees the committed keys and drafts 0..r: plain attention over a prefix of the keys
+    q, K, V = _row(50, n=300, D=16)
+    m = 5
+    s = O.scores(q, K)
+    for r in range(m):
+        sm = O.mask_draft_scores(s, m, (1 << (r + 1)) - 1)
+        o, lse = O.dense_row(sm, V)
+        keep = 300 - m + r + 1
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(q)[None, None, None, :], torch.from_numpy(K[:keep])[None, None], torch.from_numpy(V[:keep])[None, None])
+        assert np.allclose(o, ref[0, 0, 0].numpy(), rtol=1e-12, atol=1e-14)
+        o2, lse2 = O.dense_row(s[:keep], V[:keep])
+        assert np.allclose(o, o2, rtol=1e-13) and abs(lse - lse2) < 1e-12
+
+
+def test_draft_mask_conventions_and_tree_brute_force():
+    n, m = 40, 6
+    assert O.draft_visible(n, m, (1 << m) - 1).all()                     # every draft visible: no mask at all
+    assert O.draft_visible(n, 0, 0).all()
+    vis = O.draft_visible(n, m, 0b100101)                                # a tree row: drafts 0, 2 and 5 (itself)
+    assert vis[:n - m].all() and list(vis[n - m:]) == [True, False, True, False, False, True]
+    # fewer keys than drafts: only the bits that have a key count (key j = n - m + t >= 0)
+    assert list(O.draft_visible(2, 4, 0b0100)) == [True, False] and list(O.draft_visible(2, 4, 0b1000)) == [False, True]
+    # declared-reference attention over masked scores = the same over the visible keys alone, for every depth
+    q, K, V = _row(51, n=n, D=8)
+    s = O.scores(q, K)
+    sm = O.mask_draft_scores(s, m, 0b100101)
+    _, lse = O.dense_row(s[vis], V[vis])
+    for T in (math.inf, 6.0, 1.0):
+        a = O.fold_row(sm, V, lse - 0.5, T)
+        b = O.fold_row(s[vis], V[vis], lse - 0.5, T)
+        assert np.allclose(a[0], b[0], rtol=1e-13) and abs(a[1] - b[1]) < 1e-12 and abs(a[3] - b[3]) <= 1e-13 * b[3]
+    # the estimator sees the same mask (n <= 192: the exact log-sum-exp of the visible keys)
+    assert abs(O.estimate_z(lambda i: sm[i], n) - lse) < 1e-12
