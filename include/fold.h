@@ -104,7 +104,16 @@ typedef struct fold_kv {
  * sequence b / stack (stack consecutive requests share a sequence: stack = 1 for plain
  * decode; a cascade's shared-prefix level stacks the query rows of all requests that hold
  * the prefix, Section 4 "Value product" last sentence).  batch == kv.num_seqs * stack.
- * Query head h reads KV head h / (num_q_heads / num_kv_heads). */
+ * Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *
+ * Drafts and verification trees (Section 4 "Value product": extra query rows masked to their ancestors).
+ * With draft_len = m in 1..32 the last m keys of every sequence are draft tokens already appended to the
+ * cache: key n - m + t (n the sequence's length) is used by request b only if bit t of draft_mask[b] is
+ * set; earlier keys are used by every request; all heads of a request share its mask.  The requests that
+ * verify one sequence are the `stack` consecutive requests that read it (a chain of m drafts: stack = m,
+ * draft_mask[r] = 2^(r+1) - 1).  A key a row does not use has weight exactly 0 everywhere: in the
+ * reference estimate, in L and in A.  A row must use at least one key.  In a cascade only the level that
+ * holds the drafts (the last) carries them.  draft_len = 0: no masking. */
 typedef struct fold_args {
   int32_t batch, num_q_heads, num_kv_heads, head_dim;  /* head_dim in {64, 128} */
   int32_t stack;
@@ -122,6 +131,8 @@ typedef struct fold_args {
   void *out;                           /* BF16 [batch, num_q_heads, head_dim], contiguous */
   float *lse;                          /* [batch, num_q_heads] base-2 log-sum-exp, or NULL */
   int32_t *row_status;                 /* [batch, num_q_heads] bit flags, or NULL */
+  const uint32_t *draft_mask;          /* [batch] or NULL (draft_len = 0) */
+  int32_t draft_len;                   /* 0..32 */
 } fold_args;
 
 /* First 64 bytes of every workspace, zeroed at the start of each scan. */
@@ -214,7 +225,8 @@ int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, 
  * fold_host_staging_bytes(host_args) bytes, 256-byte aligned, which receives the copies,
  * the workspace and the results before they are copied back.  Everything is enqueued on
  * `stream`; the host buffers are valid after the caller synchronises the stream.  The block tail is
- * not offered here: kv.v_block_mean must be NULL (FOLD_EUNSUPPORTED otherwise). */
+ * not offered here: kv.v_block_mean must be NULL (FOLD_EUNSUPPORTED otherwise); nor are draft masks
+ * (draft_len must be 0). */
 size_t fold_host_staging_bytes(const fold_args *host_args);
 int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_bytes, fold_stream stream);
 

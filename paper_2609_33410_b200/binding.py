@@ -41,7 +41,8 @@ class FoldArgs(C.Structure):
                 ("softmax_scale", C.c_float), ("z_mode", C.c_int32), ("z", C.c_void_p),
                 ("depth_T", C.c_float), ("num_splits", C.c_int32),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("out", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p)]
+                ("out", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p),
+                ("draft_mask", C.c_void_p), ("draft_len", C.c_int32)]
 
 
 class FoldPartials(C.Structure):
@@ -174,7 +175,8 @@ class KVCache:
 def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None, z_mode: int = Z_ESTIMATE,
               z: Optional[torch.Tensor] = None, depth_T: float = math.inf, num_splits: int = 0, stack: int = 1,
               workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
-              lse: Optional[torch.Tensor] = None, row_status: Optional[torch.Tensor] = None) -> FoldArgs:
+              lse: Optional[torch.Tensor] = None, row_status: Optional[torch.Tensor] = None,
+              draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0) -> FoldArgs:
     assert q.dtype == torch.bfloat16 and q.dim() == 3 and q.stride(2) == 1
     B, Hq, D = q.shape
     a = FoldArgs()
@@ -190,6 +192,11 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
     a.workspace = _ptr(workspace)
     a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     a.out, a.lse, a.row_status = _ptr(out), _ptr(lse), _ptr(row_status)
+    if draft_len:
+        # int32 storage for the uint32 masks (torch has no uint32 arithmetic): the bit patterns are what is passed
+        assert draft_mask is not None and draft_mask.dtype == torch.int32 and draft_mask.numel() == B
+        assert draft_mask.is_contiguous()
+    a.draft_mask, a.draft_len = (_ptr(draft_mask), int(draft_len)) if draft_len else (None, 0)
     return a
 
 
@@ -291,9 +298,10 @@ def alloc_buffers(q: torch.Tensor, cache: KVCache, stack: int = 1) -> DecodeBuff
 
 def decode(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, depth_T: float = math.inf,
            z_mode: int = Z_ESTIMATE, num_splits: int = 0, scale: Optional[float] = None, stack: int = 1,
-           stream=None) -> FoldArgs:
+           draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, stream=None) -> FoldArgs:
     args = make_args(q, cache, scale=scale, z_mode=z_mode, z=bufs.z, depth_T=depth_T, num_splits=num_splits,
-                     stack=stack, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status)
+                     stack=stack, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status,
+                     draft_mask=draft_mask, draft_len=draft_len)
     fold_decode(args, stream)
     return args
 

@@ -65,6 +65,8 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   if (isnan(a->depth_T) || a->depth_T < 0.f) return FOLD_EINVAL;
   if (a->num_splits < 0) return FOLD_EINVAL;
   if (need_out && (!a->out || !aligned(a->out, 2))) return FOLD_EINVAL;
+  if (a->draft_len < 0 || a->draft_len > 32) return FOLD_EINVAL;
+  if (a->draft_len > 0 && (!a->draft_mask || !aligned(a->draft_mask, 4))) return FOLD_EINVAL;
   const int G = a->num_q_heads / a->num_kv_heads;
   const long long R = (long long)a->stack * G;
   if (G > kMaxRows || R > kMaxStackedRows) return FOLD_EUNSUPPORTED;
@@ -173,6 +175,8 @@ EstParams est_params(const fold_args *a, const Geometry &g) {
   p.z = a->z;
   p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
+  p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
+  p.draft_len = a->draft_len;
   return p;
 }
 
@@ -400,6 +404,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.page_table = kv.page_table;
   p.v = static_cast<const __nv_bfloat16 *>(kv.v);
   p.v_stride_seq = kv.stride_seq; p.v_stride_tok = kv.stride_tok; p.v_stride_head = kv.stride_head;
+  p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
+  p.draft_len = a->draft_len;
   p.vmean = static_cast<const __nv_bfloat16 *>(kv.v_block_mean);
   p.vm_stride_seq = kv.mean_stride_seq; p.vm_stride_block = kv.mean_stride_block; p.vm_stride_head = kv.mean_stride_head;
   p.slots = reinterpret_cast<float *>(static_cast<uint8_t *>(a->workspace) + kHeaderBytes);
@@ -479,6 +485,13 @@ int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream st
   g.B = a0->batch; g.Hq = a0->num_q_heads; g.Hkv = a0->num_kv_heads; g.G = G; g.D = a0->head_dim;
   EstParams p = est_params(a0, g);
   p.n_levels = n_levels;
+  {                                                          // drafts sit at the end of the last level
+    const fold_args *al = levels[n_levels - 1];
+    if (!al || al->draft_len < 0 || al->draft_len > 32) return FOLD_EINVAL;
+    if (al->draft_len > 0 && (!al->draft_mask || !aligned(al->draft_mask, 4))) return FOLD_EINVAL;
+    p.draft_mask = al->draft_len > 0 ? al->draft_mask : nullptr;
+    p.draft_len = al->draft_len;
+  }
   for (int l = 0; l < n_levels; ++l) {
     const fold_args *a = levels[l];
     if (!a || a->head_dim != a0->head_dim || a->num_kv_heads != a0->num_kv_heads || a->batch != a0->batch)
@@ -661,6 +674,7 @@ int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, f
   if (!ha->q || !ha->kv.k || !ha->kv.v || !ha->kv.seqlens || !ha->out) return FOLD_EINVAL;
   if (ha->z_mode == FOLD_Z_GIVEN && !ha->z) return FOLD_EINVAL;
   if (ha->kv.v_block_mean) return FOLD_EUNSUPPORTED;        // the block tail is not offered for host buffers
+  if (ha->draft_len != 0) return FOLD_EUNSUPPORTED;         // nor are draft masks
   HostPlan h;
   if (fold_workspace_bytes(ha) == 0 || !plan_host(ha, &h)) return FOLD_EINVAL;
   if (staging_bytes < h.total) return FOLD_EWORKSPACE;

@@ -33,6 +33,8 @@ struct EstParams {
   KvLevel lv[kMaxLevels];
   int n_levels, Hq, Hkv, G;
   float scale_log2;
+  const uint32_t *draft_mask;    // drafts: the last draft_len keys (of the concatenated levels) are used by request
+  int draft_len;                 // req only where its mask has the bit
 };
 
 __device__ __forceinline__ int level_len(const KvLevel &L, int req) {
@@ -124,6 +126,16 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
       }
       // c0, c1: key lane/4, rows 2*(lane%4) + {0,1};  c2, c3: key lane/4 + 8
       const int i0 = warp * 16 + (lane >> 2), g0 = nt * 8 + qcol;
+      if (p.draft_len) {                                     // a draft key the request does not use weighs nothing
+        const uint32_t dm = p.draft_mask[req];
+        const int dstart = n - p.draft_len;
+#pragma unroll
+        for (int hlf = 0; hlf < 2; ++hlf) {
+          const int i = i0 + 8 * hlf;
+          const int t = i < n_samples ? est_sample_key(i, n) - dstart : -1;
+          if (t >= 0 && t < 32 && !((dm >> t) & 1u)) c[2 * hlf] = c[2 * hlf + 1] = -INFINITY;
+        }
+      }
       if (g0 < G) { sc[g0][i0] = c[0] * p.scale_log2; sc[g0][i0 + 8] = c[2] * p.scale_log2; }
       if (g0 + 1 < G) { sc[g0 + 1][i0] = c[1] * p.scale_log2; sc[g0 + 1][i0 + 8] = c[3] * p.scale_log2; }
     }

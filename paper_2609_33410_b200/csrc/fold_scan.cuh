@@ -43,6 +43,8 @@ struct ScanParams {
   const int *page_table;
   const __nv_bfloat16 *v;                         // gated path reads value rows directly
   long long v_stride_seq, v_stride_tok, v_stride_head;
+  const uint32_t *draft_mask;                     // drafts: per request, which of the last draft_len keys it uses
+  int draft_len;
   const __nv_bfloat16 *vmean;                     // block tail: mean value row of every 64-key block, or null
   long long vm_stride_seq, vm_stride_block, vm_stride_head;
   float *slots;
@@ -215,6 +217,7 @@ template <int D>
 struct RowBlock {
   uint32_t qf[D / 16][4];
   float z_lo, z_hi;
+  uint32_t dm_lo, dm_hi;       // draft masks of the two rows' requests (all ones without drafts)
   bool rv_lo, rv_hi, two_blocks;
 };
 template <int D>
@@ -238,6 +241,16 @@ __device__ __forceinline__ void load_rows(RowBlock<D> &rb, const ScanParams &p, 
   }
   rb.z_lo = rb.rv_lo ? p.z[(long long)req_lo * p.Hq + head_lo] : 0.f;
   rb.z_hi = rb.rv_hi ? p.z[(long long)req_hi * p.Hq + head_hi] : 0.f;
+  rb.dm_lo = (p.draft_len && rb.rv_lo) ? p.draft_mask[req_lo] : 0xffffffffu;
+  rb.dm_hi = (p.draft_len && rb.rv_hi) ? p.draft_mask[req_hi] : 0xffffffffu;
+}
+
+// First draft key of a sequence of n keys (n itself without drafts): keys from here on are masked per request.
+__device__ __forceinline__ int draft_start(const ScanParams &p, int n) { return p.draft_len ? n - p.draft_len : n; }
+// Is key `key` (>= 0) usable under mask dm, the drafts starting at key dstart?
+__device__ __forceinline__ bool draft_ok(uint32_t dm, int key, int dstart) {
+  const int t = key - dstart;
+  return t < 0 || t > 31 || ((dm >> t) & 1u);
 }
 
 // Score one 16-key slice of the K tile at `kt` against the row block and form the weights.
@@ -249,7 +262,7 @@ template <int D, bool GATED, bool TAIL = false>
 __device__ __forceinline__ uint32_t score_slice(const RowBlock<D> &rb, uint32_t kt, int warp, int lane, int key0,
                                                 int n, float scale_log2, float neg_T, uint32_t (&ah)[4],
                                                 uint32_t (&al)[4], float &l_lo, float &l_hi, float *c_lo = nullptr,
-                                                float *c_hi = nullptr) {
+                                                float *c_hi = nullptr, int dstart = 0x7fffffff) {
   // S[rows, 16 keys] = Q K^T.  Lane l addresses key row (l>>4)*8 + (l&7), 16-byte chunk 2*kk + ((l>>3)&1)
   // of the tile laid out [half][key][128 B] with the 128-byte swizzle.
   const int k_key = warp * 16 + ((lane >> 4) << 3) + (lane & 7);
@@ -265,6 +278,16 @@ __device__ __forceinline__ uint32_t score_slice(const RowBlock<D> &rb, uint32_t 
     mma_bf16(s[1], rb.qf[kk], b2, b3);
   }
   const int qcol = (lane & 3) * 2;
+  if (key0 + 16 > dstart) {                                  // draft keys: a row only uses the ones its mask names
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int key = key0 + nt * 8 + qcol + e;
+        if (!draft_ok(rb.dm_lo, key, dstart)) s[nt][e] = -INFINITY;
+        if (!draft_ok(rb.dm_hi, key, dstart)) s[nt][2 + e] = -INFINITY;
+      }
+  }
   uint32_t livemask = 0;
   ah[0] = ah[1] = ah[2] = ah[3] = 0u;
   al[0] = al[1] = al[2] = al[3] = 0u;
@@ -384,6 +407,7 @@ template <int D>
 struct RowBlockN {
   uint32_t qb[D / 16][2];      // B fragments: row lane/4, channels kk*16 + (lane%4)*2 + {0,1} (+8)
   float z0, z1;                // references of the two rows this thread's score fragment holds: (lane%4)*2 + {0,1}
+  uint32_t dm0, dm1;           // their requests' draft masks (all ones without drafts)
   bool v0, v1;
 };
 template <int D>
@@ -406,6 +430,18 @@ __device__ __forceinline__ void load_rows_n(RowBlockN<D> &rb, const ScanParams &
   const int req1 = seq * p.stack + (r0 + 1) / p.G, head1 = kvh * p.G + (r0 + 1) % p.G;
   rb.z0 = rb.v0 ? p.z[(long long)req0 * p.Hq + head0] : 0.f;
   rb.z1 = rb.v1 ? p.z[(long long)req1 * p.Hq + head1] : 0.f;
+  rb.dm0 = (p.draft_len && rb.v0) ? p.draft_mask[req0] : 0xffffffffu;
+  rb.dm1 = (p.draft_len && rb.v1) ? p.draft_mask[req1] : 0xffffffffu;
+}
+// Draft keys of a 16-key sub-slice: scores of keys a row does not use become -inf (weight exactly 0).
+template <int D>
+__device__ __forceinline__ void mask_drafts_n(const RowBlockN<D> &rb, float (&s)[4], int lane, int key0, int dstart) {
+#pragma unroll
+  for (int kh = 0; kh < 2; ++kh) {
+    const int key = key0 + (lane >> 2) + 8 * kh;
+    if (!draft_ok(rb.dm0, key, dstart)) s[2 * kh] = -INFINITY;
+    if (!draft_ok(rb.dm1, key, dstart)) s[2 * kh + 1] = -INFINITY;
+  }
 }
 
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
@@ -592,6 +628,7 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, R = p.R, n = w.n;
+  const int dstart = draft_start(p, n);                     // keys from here on are per-request drafts
   const uint32_t full0 = base + LO::off_bar(stages, R), empty0 = full0 + 8u * stages;
 
   if (threadIdx.x == 0) {
@@ -648,12 +685,14 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           float s[4];
           uint32_t bh[2], bl[2];
           qk_issue_n<D, TK>(rb, kt, warp * U + u, lane, s);
+          if (key0 + 16 * u + 16 > dstart) mask_drafts_n<D>(rb, s, lane, key0 + 16 * u, dstart);
           const uint32_t fetch16 = weights_n<D, false>(rb, s, lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh, bl, l_lo, l_hi);
           if (fetch16 != 0) value_product_n<D, true, 0, TK>(o, kt + LO::kKTile, (warp * U + u) * 16, lane, bh, bl);
         }
       } else {
         uint32_t ah[4], al[4];
-        const uint32_t fetch16 = score_slice<D, false>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi);
+        const uint32_t fetch16 = score_slice<D, false>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi,
+                                                       nullptr, nullptr, dstart);
         if (fetch16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, ah, al);
       }
       if (key0 + KS > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
@@ -705,6 +744,7 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   const SeqWork w = seq_work(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, R = p.R, n = w.n;
+  const int dstart = draft_start(p, n);                     // keys from here on are per-request drafts
   // the ring's stages are STAGE bytes apart; what follows it keeps its place relative to the ring's end
   const uint32_t full0 = base + stages * (STAGE - LO::kStage) + LO::off_bar(stages, 0), empty0 = full0 + 8u * stages;
 
@@ -756,7 +796,7 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
         if (key0 >= n) break;
         uint32_t ah[4], al[4];
         const uint32_t live16 = score_slice<D, GATED, TAIL>(rb, kt, sl, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo,
-                                                              l_hi, &c_lo, &c_hi);
+                                                              l_hi, &c_lo, &c_hi, dstart);
         if (live16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, sl * 16, lane, ah, al);
       }
       if (TAIL) {
@@ -829,6 +869,7 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   const SeqWork w = seq_work(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
+  const int dstart = draft_start(p, n);                     // keys from here on are per-request drafts
   // barriers: K full / empty per stage; value full / empty per (slice, slot)
   const uint32_t full0 = base + LO::off_bar(stages, vr, R), empty0 = full0 + 8u * stages;
   const uint32_t vfull0 = empty0 + 8u * stages, vempty0 = vfull0 + 8u * kConsumerWarps * vr;
@@ -888,7 +929,7 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       uint2 mean8 = make_uint2(0u, 0u);
       if (ready) {
         fetch16 = score_slice<D, true, TAIL>(rb, base + my_stage * LO::kKStage, sl, lane, key0, n, p.scale_log2, p.neg_T, ah,
-                                             al, l_lo, l_hi, &c_lo, &c_hi);
+                                             al, l_lo, l_hi, &c_lo, &c_hi, dstart);
         if (TAIL && lane * 8 < D * 2)                        // this lane's 8 bytes of the tile's block mean row
           mean8 = *reinterpret_cast<const uint2 *>(gen + my_stage * LO::kKStage + LO::kKTile + lane * 8);
         __syncwarp();
@@ -1049,6 +1090,7 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
+  const int dstart = draft_start(p, n);                     // keys from here on are per-request drafts
   const uint32_t full0 = base + LO::off_bar(stages, vr), empty0 = full0 + 8u * stages;
   const uint32_t vfull0 = empty0 + 8u * stages, vempty0 = vfull0 + 8u * kConsumerWarps * vr;
 
@@ -1113,7 +1155,10 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         if (ready) {
           float s[U][4];
 #pragma unroll
-          for (int u = 0; u < U; ++u) qk_issue_n<D, TK>(rb, base + my_stage * LO::kKStage, sl * U + u, lane, s[u]);
+          for (int u = 0; u < U; ++u) {
+            qk_issue_n<D, TK>(rb, base + my_stage * LO::kKStage, sl * U + u, lane, s[u]);
+            if (key0 + 16 * u + 16 > dstart) mask_drafts_n<D>(rb, s[u], lane, key0 + 16 * u, dstart);
+          }
           if (TAIL && lane * 8 < D * 2)                      // this lane's 8 bytes of the slice's block mean row
             mean8 = *reinterpret_cast<const uint2 *>(gen + my_stage * LO::kKStage + LO::kKTile +
                                                      ((sl * KS) / 64) * (D * 2) + lane * 8);

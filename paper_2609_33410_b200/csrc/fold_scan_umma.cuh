@@ -132,6 +132,7 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   const SeqWork w = seq_work(p, seq);
   if (split >= w.n_chunks) return;
   const int R = p.R, n = w.n;
+  const int dstart = draft_start(p, n);
 
   // barriers (8 bytes each): kv_full[stages] pv_done[stages] s_full[2] s_empty[2] p_full o_empty.
   // pv_done[stage] completes when the value product of the tile in `stage` has: it frees the stage for the producer,
@@ -165,6 +166,7 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   const int r_glob = rt * kUmmaRows + row;
   const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
   float z_row = 0.f;
+  uint32_t dm_row = 0xffffffffu;                             // the row's request's draft mask
   if (warp >= 2) {
     const bool valid_row = r_glob < R;
     const int req = seq * p.stack + r_glob / p.G, head = kvh * p.G + r_glob % p.G;
@@ -181,6 +183,7 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     }
     tmem_st_wait();
     z_row = valid_row ? p.z[(long long)req * p.Hq + head] : INFINITY;
+    if (p.draft_len && valid_row) dm_row = p.draft_mask[req];
   }
   tc_fence_before();
   __syncthreads();                                           // Q is in tensor memory
@@ -275,6 +278,11 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         tmem_ld32(lane_addr + b * 64 + ch * 32, s);
         // rows beyond R carry z = +inf, so their weights vanish by themselves; keys beyond n only occur in a tail tile
         const int key_lim = n - (key_base + ch * 32);        // this thread's keys j < key_lim exist
+        if (key_base + kTileKeys > dstart) {                 // draft keys: the row only uses the ones its mask names
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (!draft_ok(dm_row, key_base + ch * 32 + j, dstart)) s[j] = -INFINITY;
+        }
         auto weights = [&](auto tail) {
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
@@ -405,6 +413,7 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   const SeqWork w = seq_work(p, seq);
   if (split >= w.n_chunks) return;
   const int R = p.R, n = w.n;
+  const int dstart = draft_start(p, n);
 
   // barriers (8 bytes each): kv_full[stages]  pv_done[stages]  s_full[2]  p_full[2]  o_empty[2]
   // pv_done[stage]: both groups' value products of the tile in `stage` have completed (frees the stage; at a
@@ -437,6 +446,7 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t col_s = g * 64, col_o = 128 + g * 128, col_q = 384 + g * 64;
   float z_row = 0.f;
+  uint32_t dm_row = 0xffffffffu;                             // the row's request's draft mask
   if (warp >= 2) {
     const bool valid_row = r_glob < R;
     const int req = seq * p.stack + r_glob / p.G, head = kvh * p.G + r_glob % p.G;
@@ -453,6 +463,7 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     }
     tmem_st_wait();
     z_row = valid_row ? p.z[(long long)req * p.Hq + head] : INFINITY;
+    if (p.draft_len && valid_row) dm_row = p.draft_mask[req];
   }
   tc_fence_before();
   __syncthreads();                                           // Q is in tensor memory
@@ -547,6 +558,11 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         tmem_ld32(lane_addr + col_s + ch * 32, s);
         // rows beyond R carry z = +inf, so their weights vanish by themselves; keys beyond n only occur in a tail tile
         const int key_lim = n - (key_base + ch * 32);        // this thread's keys j < key_lim exist
+        if (key_base + kTileKeys > dstart) {                 // draft keys: the row only uses the ones its mask names
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (!draft_ok(dm_row, key_base + ch * 32 + j, dstart)) s[j] = -INFINITY;
+        }
         auto weights = [&](auto tail) {
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {

@@ -168,6 +168,35 @@ def make_cascade_workload(batch: int, num_q_heads: int, num_kv_heads: int, head_
     return pre, suf
 
 
+def make_draft_workload(num_seqs: int, draft_len: int, num_q_heads: int, num_kv_heads: int, head_dim: int,
+                        context_lens: Union[int, Sequence[int]], seed: int = 0, device="cpu", tree: bool = False, **kw):
+    """Draft / tree verification: every sequence holds its committed context followed by `draft_len` draft tokens,
+    and `draft_len` requests (stacked on the sequence) verify them.  Returns (workload, masks, draft_len): request
+    seq * draft_len + r is draft row r; bit t of masks[request] says whether it uses draft key t.
+    Chain: row r uses drafts 0..r.  Tree: a random parent among the earlier drafts (or none) per draft; a row uses
+    its ancestors and itself.  Masks are int32 bit patterns."""
+    m = int(draft_len)
+    assert 1 <= m <= 32
+    ctx = [int(context_lens)] * num_seqs if isinstance(context_lens, int) else [int(x) for x in context_lens]
+    w = make_decode_workload(num_seqs * m, num_q_heads, num_kv_heads, head_dim, [c + m for c in ctx], seed=seed,
+                             device=device, stack=m, **kw)
+    g = torch.Generator(device="cpu")
+    g.manual_seed(int(seed) + 977)
+    masks = []
+    for _ in range(num_seqs):
+        row = []
+        for r in range(m):
+            if tree:
+                parent = int(torch.randint(-1, r, (1,), generator=g).item()) if r > 0 else -1
+                anc = row[parent] if parent >= 0 else 0
+            else:
+                anc = row[r - 1] if r > 0 else 0
+            row.append(anc | (1 << r))
+        masks += row
+    t = torch.tensor([x - (1 << 32) if x >= (1 << 31) else x for x in masks], dtype=torch.int32, device=device)
+    return w, t, m
+
+
 # The five benchmark configurations, by name.  `scale_down` shrinks context (and for the
 # sweep the batch) so the CPU oracle can check every row in seconds.
 def config_workload(name: str, device="cpu", small: bool = False, **over) -> DecodeWorkload:

@@ -43,13 +43,16 @@ def oracle_block_means(w: DecodeWorkload) -> torch.Tensor:
     return t.to(torch.bfloat16).to(w.k.device)                # exact: the oracle's means are BF16 values already
 
 
-def run_gpu(w: DecodeWorkload, T=math.inf, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, bufs=None, v_block_mean=None):
+def run_gpu(w: DecodeWorkload, T=math.inf, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, bufs=None, v_block_mean=None,
+            draft=None):
+    """`draft` = (masks int32 [batch], draft_len): draft / tree-verification rows."""
     cache = cache_of(w, v_block_mean)
     if bufs is None:
         bufs = F.alloc_buffers(w.q, cache, w.stack)
     if z is not None:
         bufs.z.copy_(z)
-    F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale)
+    F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale,
+             draft_mask=None if draft is None else draft[0], draft_len=0 if draft is None else draft[1])
     torch.cuda.synchronize()
     assert bufs.header().wait_timeouts == 0
     return bufs
@@ -68,12 +71,14 @@ def all_rows(w: DecodeWorkload):
     return [(b, h) for b in range(w.batch) for h in range(w.num_q_heads)]
 
 
-def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False, yardstick=True, v_block_mean=None):
+def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False, yardstick=True, v_block_mean=None,
+            draft=None):
     """Element-by-element comparison of the CUDA outputs with the oracle run at the GPU's own
     references.  Returns a dict of the measured errors; asserts the tolerances.  `v_block_mean`
     (the table the GPU was given) switches the oracle's block tail on; a key that flips at the threshold
     then moves between its value and its block's mean, so the threshold slack counts twice."""
     vm = None if v_block_mean is None else v_block_mean.float().cpu().numpy().astype(np.float64)
+    dmask = None if draft is None else [int(x) & 0xffffffff for x in draft[0].cpu().tolist()]
     G = w.num_q_heads // w.num_kv_heads
     out = bufs.out.float().cpu().numpy().astype(np.float64)
     lse = bufs.lse.cpu().numpy().astype(np.float64)
@@ -91,6 +96,8 @@ def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False
             assert not out[b, h].any() and lse[b, h] == -np.inf and status[b, h] == F.ROW_EMPTY
             continue
         s = O.scores(q, K, w.scale)
+        if draft is not None:                                 # keys the row does not use: weight exactly 0
+            s = O.mask_draft_scores(s, draft[1], dmask[b])
         v_mean = None if vm is None else vm[b // w.stack, :(n + 63) // 64, h // G]
         o_ref, lse_ref, _, L = O.fold_row(s, V, z[b, h], T, v_mean=v_mean)
         d = out[b, h] - o_ref
@@ -106,7 +113,8 @@ def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False
             slack_sum += ((2.0 if vm is not None else 1.0) * O.cut_report(s, V, z[b, h], T)["slack"]) ** 2 * V.shape[1]
             if yardstick:
                 o_dense, _ = O.dense_row(s, V)
-                y = O.online_softmax_bf16(q, K, V, w.scale) - o_dense
+                vis = np.isfinite(s)
+                y = O.online_softmax_bf16(q, K[vis], V[vis], w.scale) - o_dense
                 ynum += float(y @ y)
     res = dict(rel_l2=math.sqrt(num / max(den, 1e-300)), max_abs=max_abs, vmax=vmax,
                mean_rel=float(np.mean(rel_rows)) if rel_rows else 0.0, dz=dz)

@@ -55,3 +55,20 @@ def test_named_configs_small():
     assert (w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.max_seqlen) == (1, 8, 8, 128, 4096)
     w = config_workload("c3", small=True)
     assert w.paged and w.page_size == 64
+
+
+def test_draft_workload_masks_are_chains_or_ancestor_closed_trees():
+    from paper_2609_33410_b200.workloads import make_draft_workload
+    w, masks, m = make_draft_workload(3, 5, 4, 2, 64, [10, 20, 7], seed=5)
+    assert w.batch == 15 and w.stack == 5 and [int(x) for x in w.seqlens] == [15, 25, 12]
+    assert [int(x) for x in masks[:5]] == [1, 3, 7, 15, 31]
+    w, masks, m = make_draft_workload(4, 8, 4, 2, 64, 9, seed=6, tree=True)
+    for s in range(4):
+        row = [int(x) & 0xffffffff for x in masks[s * 8:(s + 1) * 8]]
+        for r, mk in enumerate(row):
+            assert (mk >> r) & 1 and mk < (1 << (r + 1))                  # itself, and nothing later
+            for t in range(r):
+                if (mk >> t) & 1:
+                    assert row[t] & mk == row[t]                          # an ancestor's ancestors are ancestors
+    w, masks, m = make_draft_workload(1, 32, 2, 2, 64, 3, seed=7)
+    assert int(masks[31]) == -1                                           # all 32 bits, stored as int32
