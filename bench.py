@@ -246,7 +246,7 @@ def run_sweep(args, dev):
                                       v_rows_fetched=round(lam, 4), l2_flush=flush is not None))
                 del w, cache, bufs, flush
                 torch.cuda.empty_cache()
-    print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "block_tail": bool(args.tail), "cells": cells}))
+    print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "block_tail": bool(args.tail), "drafts": args.drafts, "cells": cells}))
 
 
 def main():
@@ -260,6 +260,8 @@ def main():
     ap.add_argument("--ref-units", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--drafts", type=int, default=1,
+                    help="verify a chain of this many draft tokens per sequence (stacked rows with ancestor masks)")
     ap.add_argument("--tail", action="store_true",
                     help="finite-depth steps use the block tail (cut keys add weight x block-mean value)")
     ap.add_argument("--graph", action="store_true",
@@ -299,6 +301,15 @@ def main():
         from paper_2609_33410_b200.workloads import make_cascade_workload
         gen = dict(spec["cascade"]); gen["seed"] = gen["seed"] + 1000 * rank
         levels = list(make_cascade_workload(device=dev, **gen))           # prefix level (stacked), suffix level
+    elif args.drafts > 1:
+        # draft verification: every sequence keeps its length; its last `drafts` keys are draft tokens and `drafts`
+        # requests (a chain) verify them: the same bytes, `drafts` times the query rows
+        from paper_2609_33410_b200.workloads import make_draft_workload
+        gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
+        n_seqs, lens = gen.pop("batch"), gen.pop("seqlens")
+        lvl, draft_masks, _ = make_draft_workload(n_seqs, args.drafts, gen.pop("num_q_heads"), gen.pop("num_kv_heads"),
+                                                  gen.pop("head_dim"), lens - args.drafts, device=dev, **gen)
+        levels = [lvl]
     else:
         gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
         levels = [make_decode_workload(device=dev, **gen)]
@@ -319,7 +330,8 @@ def main():
     def make(depth, z_mode):
         return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
                             num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
-                            row_status=bufs.row_status) for l, c, b in zip(levels, caches, lbufs)]
+                            row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
+                            draft_len=args.drafts if args.drafts > 1 else 0) for l, c, b in zip(levels, caches, lbufs)]
 
     # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
     # is scanned on a side stream while the suffix level is scanned on the main one (fork / join with events).
