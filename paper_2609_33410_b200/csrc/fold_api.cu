@@ -547,22 +547,31 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
   p.lse = lse; p.row_status = row_status;
   p.n_levels = n_levels; p.Hq = p0->num_q_heads; p.Hkv = p0->num_kv_heads;
   p.G = p0->num_q_heads / p0->num_kv_heads; p.D = p0->head_dim;
-  // warps per row (a power of two up to 16): about 8 slots per warp, fewer warps when the rows alone fill the machine
+  // warps per row (a power of two up to 16): about 8 slots per warp.  One level whose slots then fit a warp's
+  // registers is merged in one load pass; otherwise two passes, and fewer warps when the rows alone fill the machine.
   int total_slots = 0;
   for (int l = 0; l < n_levels; ++l) total_slots += max_chunks_upto(levels[l]->max_seqlen);
   const long long n_rows = (long long)p0->batch * p.Hq;
   int warps = 1;
   while (warps < kMergeMaxWarps && warps * 8 < total_slots) warps <<= 1;
-  while (warps > 1 && n_rows * warps > 2048) warps >>= 1;
+  const bool resident = n_levels == 1 && (total_slots + warps - 1) / warps <= kMergeResident;
+  if (!resident)
+    while (warps > 1 && n_rows * warps > 2048) warps >>= 1;
 #ifdef FOLD_TUNING
   if (const char *e = getenv("FOLD_TUNE_MERGEW")) warps = atoi(e);
 #endif
   const int cta_warps = warps < 4 ? 4 : warps;
   const long long rows_per_cta = cta_warps / warps;
   const dim3 grid((unsigned)((n_rows + rows_per_cta - 1) / rows_per_cta)), block(32 * cta_warps);
-  cudaError_t rc = p.D == 128
-                       ? launch_pdl(fold_merge_kernel<4>, grid, block, 0, static_cast<cudaStream_t>(stream), p, warps, n_rows)
-                       : launch_pdl(fold_merge_kernel<2>, grid, block, 0, static_cast<cudaStream_t>(stream), p, warps, n_rows);
+  const cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool res = resident && (total_slots + warps - 1) / warps <= kMergeResident;
+  cudaError_t rc;
+  if (p.D == 128)
+    rc = res ? launch_pdl(fold_merge_kernel<4, true>, grid, block, 0, st, p, warps, n_rows)
+             : launch_pdl(fold_merge_kernel<4, false>, grid, block, 0, st, p, warps, n_rows);
+  else
+    rc = res ? launch_pdl(fold_merge_kernel<2, true>, grid, block, 0, st, p, warps, n_rows)
+             : launch_pdl(fold_merge_kernel<2, false>, grid, block, 0, st, p, warps, n_rows);
   if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }

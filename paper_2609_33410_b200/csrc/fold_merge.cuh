@@ -52,7 +52,10 @@ __device__ __forceinline__ long long to_grid(float g, double alpha) { return __d
 // second hits L1): the order-free maximum, then the integer sum.  The W warps of a row combine through staged
 // partials in shared memory: maxima by max, integer sums by integer addition, both exact, so neither the warp
 // count nor the slot order can change a bit.
-template <int EPT>
+// RESIDENT (one level, at most kMergeResident slots per warp): the slots are loaded once and stay in registers for
+// the second pass.
+constexpr int kMergeResident = 8;
+template <int EPT, bool RESIDENT>
 __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const MergeParams p, const int W,
                                                                          const long long n_rows) {
   constexpr int D = 32 * EPT;
@@ -94,8 +97,28 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
   unsigned mx[EPT], mxl = 0u, C = 0;
 #pragma unroll
   for (int e = 0; e < EPT; ++e) mx[e] = 0u;
+  float rv[RESIDENT ? kMergeResident : 1][EPT], rl[RESIDENT ? kMergeResident : 1];
+  if (RESIDENT) {
+    int cnt; const float *a, *q; long long step;
+    level(0, cnt, a, q, step);
+    C = cnt;
+#pragma unroll
+    for (int i = 0; i < kMergeResident; ++i) {
+      const bool on = sub + i * W < cnt;
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) rv[i][e] = 0.f;
+      rl[i] = 0.f;
+      if (on) {
+        load_vec(a + i * step, rv[i]);
+        if (x == 0) rl[i] = q[i * step];
+      }
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) mx[e] = max(mx[e], __float_as_uint(rv[i][e]) & 0x7fffffffu);
+      mxl = max(mxl, __float_as_uint(rl[i]) & 0x7fffffffu);
+    }
+  }
 #pragma unroll 1
-  for (int l = 0; l < p.n_levels; ++l) {
+  for (int l = 0; l < (RESIDENT ? 0 : p.n_levels); ++l) {
     int cnt; const float *a, *q; long long step;
     level(l, cnt, a, q, step);
     C += cnt;
@@ -135,8 +158,16 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
   }
   const double alpha_l = pow2_double(grid_shift(mxl, clog2C));
   const bool fin_l = (mxl >> 23) != 255u;
+  if (RESIDENT) {                                    // absent slots hold zeros, which add nothing
+#pragma unroll
+    for (int i = 0; i < kMergeResident; ++i) {
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) if (fin[e]) acc[e] += to_grid(rv[i][e], alpha[e]);
+      if (x == 0 && fin_l) accl += to_grid(rl[i], alpha_l);
+    }
+  }
 #pragma unroll 1
-  for (int l = 0; l < p.n_levels; ++l) {
+  for (int l = 0; l < (RESIDENT ? 0 : p.n_levels); ++l) {
     int cnt; const float *a, *q; long long step;
     level(l, cnt, a, q, step);
 #pragma unroll 4
