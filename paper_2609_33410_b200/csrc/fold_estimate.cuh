@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
   }
   const int n_samples = n < kEstSamples ? n : kEstSamples;
   const int qcol = (lane & 3) * 2;
+  const int qcol4 = (lane & 3) * 8;                          // this lane's 8 consecutive channels of every 32
 
   if (warp * 16 < n_samples) {
     // the two sampled key rows this lane reads fragments of
@@ -101,28 +102,32 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
       if (i < n_samples) {
         int j = est_sample_key(i, n), l = 0;
         while (l < p.n_levels - 1 && j >= lens[l]) { j -= lens[l]; ++l; }
-        rowp[hlf] = key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + qcol;
+        rowp[hlf] = key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + qcol4;
       }
     }
+    // A dot product does not care in which order its terms meet: the k slots of each pair of MMAs are assigned so
+    // that a lane's fragments of 32 channels are 8 CONSECUTIVE channels of its row (one 16-byte load) -- MMA 2j takes
+    // channels 32j + 8t + {0,1 | 2,3} in its slots {2t,2t+1 | 2t+8,2t+9}, MMA 2j+1 takes 32j + 8t + {4,5 | 6,7} -- and
+    // the query fragments below follow the same assignment.
     uint32_t a[KS][4];
 #pragma unroll
-    for (int kk = 0; kk < KS; ++kk) {
-      a[kk][0] = rowp[0] ? *reinterpret_cast<const uint32_t *>(rowp[0] + kk * 16) : 0u;
-      a[kk][1] = rowp[1] ? *reinterpret_cast<const uint32_t *>(rowp[1] + kk * 16) : 0u;
-      a[kk][2] = rowp[0] ? *reinterpret_cast<const uint32_t *>(rowp[0] + kk * 16 + 8) : 0u;
-      a[kk][3] = rowp[1] ? *reinterpret_cast<const uint32_t *>(rowp[1] + kk * 16 + 8) : 0u;
+    for (int j = 0; j < KS / 2; ++j) {
+      const uint4 r0 = rowp[0] ? *reinterpret_cast<const uint4 *>(rowp[0] + j * 32) : make_uint4(0, 0, 0, 0);
+      const uint4 r1 = rowp[1] ? *reinterpret_cast<const uint4 *>(rowp[1] + j * 32) : make_uint4(0, 0, 0, 0);
+      a[2 * j][0] = r0.x; a[2 * j][1] = r1.x; a[2 * j][2] = r0.y; a[2 * j][3] = r1.y;
+      a[2 * j + 1][0] = r0.z; a[2 * j + 1][1] = r1.z; a[2 * j + 1][2] = r0.w; a[2 * j + 1][3] = r1.w;
     }
     // query rows of the group as B fragments (n = lane / 4), eight rows per n-tile
 #pragma unroll 1
     for (int nt = 0; nt * 8 < G; ++nt) {
       const int g = nt * 8 + (lane >> 2);
-      const __nv_bfloat16 *qrow = p.q + (long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + qcol;
+      const __nv_bfloat16 *qrow = p.q + (long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + qcol4;
       float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int kk = 0; kk < KS; ++kk) {
-        const uint32_t b0 = g < G ? *reinterpret_cast<const uint32_t *>(qrow + kk * 16) : 0u;
-        const uint32_t b1 = g < G ? *reinterpret_cast<const uint32_t *>(qrow + kk * 16 + 8) : 0u;
-        mma_bf16(c, a[kk], b0, b1);
+      for (int j = 0; j < KS / 2; ++j) {
+        const uint4 b = g < G ? *reinterpret_cast<const uint4 *>(qrow + j * 32) : make_uint4(0, 0, 0, 0);
+        mma_bf16(c, a[2 * j], b.x, b.y);
+        mma_bf16(c, a[2 * j + 1], b.z, b.w);
       }
       // c0, c1: key lane/4, rows 2*(lane%4) + {0,1};  c2, c3: key lane/4 + 8
       const int i0 = warp * 16 + (lane >> 2), g0 = nt * 8 + qcol;
