@@ -42,7 +42,7 @@ WORKLOADS = {
 
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one scan launch from the ncu captures
-# summarised in profiles/fold_scan_kernels_c2_small.md, per byte of cache the launch covers: the c2_small
+# of the c2_small workload (`--workload c2_small`), per byte of cache the launch covers: the c2_small
 # capture (268.4 MB of K+V) moved 272.2 MB (gated, T=16) and 271.8 MB (dense).  Traffic grows in
 # proportion to the (sequence, kv head, key) units, so a launch is scaled by its cache bytes.
 NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 272.2 / 268.4, "dense": 271.8 / 268.4}
@@ -459,7 +459,7 @@ def main():
         "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
                      "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src,
                      "traffic": None if cascade or args.workload != "c2" else NCU_TRAFFIC_PER_CACHE_BYTE["gated"] * cache_bytes,
-                     "traffic_source": "ncu capture on c2_small scaled by units (profiles/fold_scan_kernels_c2_small.md)",
+                     "traffic_source": "ncu dram__bytes_read+write of the same kernel captured on workload c2_small, scaled by units",
                      "algorithmic_bytes_per_launch": actual_bytes(r16),
                      "dense": {"kernel": "fold_scan_dense_kernel (T=inf)" if not cascade else "fold_scan_stacked_pair_kernel + fold_scan_dense_kernel (T=inf)", "achieved": achinf, "frac": achinf / peak,
                                "frac_of_nominal_8TBs": achinf / 8000.0,
