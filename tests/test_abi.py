@@ -115,6 +115,31 @@ def test_host_checks_answer_before_any_cuda_call():
     assert L.fold_estimate_z(None, 0, None) == F.FOLD_EINVAL
 
 
+def test_host_checks_of_draft_masks_and_block_means():
+    L = F.lib()
+    a, keep = _cpu_args()
+    ws = torch.zeros(F.fold_workspace_bytes(a) + 256, dtype=torch.uint8)
+    a.workspace = ws.data_ptr() + ((-ws.data_ptr()) % 256)
+    a.workspace_bytes = ws.numel() - 256
+    masks = torch.ones(64, dtype=torch.int32)
+    for length, ptr, want in [(33, masks.data_ptr(), F.FOLD_EINVAL), (-1, masks.data_ptr(), F.FOLD_EINVAL),
+                              (4, None, F.FOLD_EINVAL), (4, masks.data_ptr() + 2, F.FOLD_EINVAL)]:
+        a.draft_len, a.draft_mask = length, ptr
+        assert L.fold_decode(a, None) == want, (length, ptr)
+    a.draft_len, a.draft_mask = 0, None
+    means = torch.zeros(4096, dtype=torch.bfloat16)
+    a.kv.v_block_mean = means.data_ptr() + 2                        # rows must start on 16 bytes
+    a.kv.mean_stride_seq, a.kv.mean_stride_block, a.kv.mean_stride_head = 1024, 256, 128
+    assert L.fold_decode(a, None) == F.FOLD_EINVAL
+    a.kv.v_block_mean = means.data_ptr() + ((-means.data_ptr()) % 16)
+    a.kv.mean_stride_block = 100                                    # not a multiple of 8, shorter than a row
+    assert L.fold_decode(a, None) == F.FOLD_EINVAL
+    kv = F.FoldKV()
+    assert L.fold_block_means(None, 2, 128, None) == F.FOLD_EINVAL
+    assert L.fold_block_means(kv, 2, 96, None) == F.FOLD_EUNSUPPORTED
+    assert L.fold_block_means(kv, 2, 128, None) == F.FOLD_EINVAL    # no table to fill
+
+
 @pytest.mark.skipif(torch.cuda.is_available(), reason="only meaningful without a device")
 def test_no_device_means_a_loud_error_not_a_fallback():
     a, keep = _cpu_args()
