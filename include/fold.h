@@ -207,7 +207,10 @@ int fold_decode(const fold_args *args, fold_stream stream);
  * pointers, n_levels in 1..4) describe the same requests: the same q, z, batch, head counts,
  * head_dim, softmax_scale and depth_T; each level has its own kv, stack and workspace.
  * levels[0]->z_mode is FOLD_Z_ESTIMATE (estimate over all levels, written to z) or FOLD_Z_GIVEN;
- * out, lse and row_status are taken from levels[0]. */
+ * out, lse and row_status are taken from levels[0].
+ * With two or more levels the first level is scanned on a stream the library keeps per device (created, with two
+ * events, at the first such call on the device: make that call outside stream capture), forked from and joined
+ * back into `stream` with events, so to the caller the call is still one ordered piece of work on `stream`. */
 int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_stream stream);
 
 /* Fill kv->v_block_mean (DEVICE memory of the caller, laid out as the fold_kv comment says, at least

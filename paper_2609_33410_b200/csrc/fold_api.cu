@@ -4,6 +4,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "fold_common.cuh"
 #include "fold_estimate.cuh"
 #include "fold_merge.cuh"
@@ -445,6 +447,30 @@ void fill_partials(const fold_args *a, const Geometry &g, fold_partials *dst) {
   dst->max_seqlen = a->kv.max_seqlen;
 }
 
+// One non-blocking stream and two events per device for fold_decode_cascade's fork / join, created at the first
+// cascade call on the device.  Null if they cannot be created: the cascade then runs on the caller's stream alone.
+struct CascadeSide {
+  std::mutex mu;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  int state = 0;                                             // 0 untried, 1 ready, -1 unavailable
+};
+CascadeSide *cascade_side() {
+  static CascadeSide sides[64];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  CascadeSide *s = &sides[dev];
+  std::lock_guard<std::mutex> lock(s->mu);
+  if (s->state == 0) {
+    const bool ok = cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&s->join, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) (void)cudaGetLastError();
+    s->state = ok ? 1 : -1;
+  }
+  return s->state == 1 ? s : nullptr;
+}
+
 }  // namespace
 
 extern "C" {
@@ -629,10 +655,26 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
     if (int rc = fold_estimate_z(levels, n_levels, stream)) return rc;
   fold_partials parts[kMaxLevels];
   const fold_partials *pp[kMaxLevels];
-  for (int l = 0; l < n_levels; ++l) {
-    if (int rc = fold_decode_split(&lv[l], &parts[l], stream)) return rc;
-    pp[l] = &parts[l];
+  for (int l = 0; l < n_levels; ++l) pp[l] = &parts[l];
+  // Once the reference is fixed the levels are independent: the first level (the shared prefix: a tensor-bound
+  // kernel on fewer CTAs than SMs) is scanned on a side stream of the library's while the others are scanned on the
+  // caller's stream, forked and joined with events, so the caller still sees one ordered call on `stream`.
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CascadeSide *side = n_levels >= 2 ? cascade_side() : nullptr;
+  if (side) {
+    std::lock_guard<std::mutex> lock(side->mu);               // the events are shared by every call on the device
+    if (cudaEventRecord(side->fork, st) != cudaSuccess || cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess)
+      return FOLD_ECUDA;
+    int rc = fold_decode_split(&lv[0], &parts[0], side->stream);
+    const bool recorded = cudaEventRecord(side->join, side->stream) == cudaSuccess;
+    for (int l = 1; l < n_levels && rc == FOLD_OK; ++l) rc = fold_decode_split(&lv[l], &parts[l], stream);
+    // join in every case, so that the side stream never holds work the caller's stream does not wait for
+    if (!recorded || cudaStreamWaitEvent(st, side->join, 0) != cudaSuccess) return FOLD_ECUDA;
+    if (rc) return rc;
+    return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
   }
+  for (int l = 0; l < n_levels; ++l)
+    if (int rc = fold_decode_split(&lv[l], &parts[l], stream)) return rc;
   return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
 }
 

@@ -172,3 +172,29 @@ def test_graph_replay_equals_eager_call(T):
         torch.cuda.synchronize()
         assert same_bits(bufs.out, o) and same_bits(bufs.lse, l) and same_bits(bufs.z, z)
         assert bufs.header().wait_timeouts == 0
+
+
+def test_cascade_call_is_graph_capturable_with_its_side_stream():
+    # the cascade forks its first level onto a stream of the library's and joins it back: still one capturable call
+    B, Hq, Hkv, D = 6, 8, 2, 128
+    suffixes = [300, 1, 0, 257, 64, 65]
+    g = torch.Generator(device=DEV); g.manual_seed(97)
+    q = torch.randn(B, Hq, D, generator=g, device=DEV).to(torch.bfloat16)
+    pre = make_decode_workload(B, Hq, Hkv, D, 2000, seed=98, device=DEV, stack=B, q=q)
+    suf = make_decode_workload(B, Hq, Hkv, D, suffixes, seed=99, device=DEV, q=q, sink_gain=1.0)
+    cp, cs = cache_of(pre), cache_of(suf)
+    bp, bs = F.alloc_buffers(q, cp, stack=B), F.alloc_buffers(q, cs)
+    common = dict(z=bs.z, depth_T=16.0, out=bs.out, lse=bs.lse, row_status=bs.row_status)
+    levels = [F.make_args(q, cp, stack=B, workspace=bp.workspace, **common), F.make_args(q, cs, workspace=bs.workspace, **common)]
+    F.fold_decode_cascade(levels, torch.cuda.current_stream())           # first call outside capture
+    torch.cuda.synchronize()
+    o, l = bs.out.clone(), bs.lse.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        F.fold_decode_cascade(levels, torch.cuda.current_stream())
+    for _ in range(2):
+        bs.out.zero_(); bs.lse.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert same_bits(bs.out, o) and same_bits(bs.lse, l)
+        assert bp.header().wait_timeouts == 0 and bs.header().wait_timeouts == 0
