@@ -236,10 +236,30 @@ int launch_dense_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p,
     return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
+// 9..16 rows: rows on N in two 8-row tiles per warp.
+template <int D>
+int launch_dense_nt2(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LO = DenseWideLayout<D>;
+  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  int stages = (per_cta2 - LO::total(0)) / (LO::kStage + 16);
+  if (stages > 8) stages = 8;
+  if (stages < 2) return FOLD_EUNSUPPORTED;
+  p.stages = stages;
+  p.vr = 0;
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_dense_nt2_kernel<D>, configured)) return rc;
+  if (launch_pdl(fold_scan_dense_nt2_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages), st, mk, mv, p) != cudaSuccess)
+    return FOLD_ECUDA;
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
 template <int D>
 int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
   // up to 8 rows: rows on N (half the MMAs and accumulators), 16 KB key tiles at either head dimension
-  return p.R <= kNarrowRows ? launch_dense_as<D, true>(mk, mv, p, grid, st) : launch_dense_as<D, false>(mk, mv, p, grid, st);
+  if (p.R <= kNarrowRows) return launch_dense_as<D, true>(mk, mv, p, grid, st);
+#ifdef FOLD_TUNING
+  if (getenv("FOLD_TUNE_WIDE")) return launch_dense_as<D, false>(mk, mv, p, grid, st);
+#endif
+  return launch_dense_nt2<D>(mk, mv, p, grid, st);
 }
 
 // Stacked rows: the dense ring without reduction buffers; one CTA per (split, 64-row group).  With the block tail
@@ -387,7 +407,12 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const fold_kv &kv = a->kv;
   const bool paged = kv.page_table != nullptr;
   // narrow row blocks walk 16 KB key tiles: 128 keys at D = 64
-  const int tile_keys = (g.R <= kNarrowRows && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
+  // (so do 9..16-row blocks at T = inf, which run the two-tile rows-on-N kernel)
+  bool narrow_tiles = g.R <= kNarrowRows || (g.R <= kMaxRows && isinf(a->depth_T));
+#ifdef FOLD_TUNING
+  if (getenv("FOLD_TUNE_WIDE") && g.R > kNarrowRows) narrow_tiles = false;
+#endif
+  const int tile_keys = (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
   const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   const bool gated = !isinf(a->depth_T);
   CUtensorMap mk, mv;

@@ -410,10 +410,11 @@ struct RowBlockN {
   uint32_t dm0, dm1;           // their requests' draft masks (all ones without drafts)
   bool v0, v1;
 };
+// `row0`: first row of this 8-row N tile within the (sequence, kv head)'s row block (0, or 8 for the second tile).
 template <int D>
-__device__ __forceinline__ void load_rows_n(RowBlockN<D> &rb, const ScanParams &p, int seq, int kvh, int lane) {
+__device__ __forceinline__ void load_rows_n(RowBlockN<D> &rb, const ScanParams &p, int seq, int kvh, int lane, int row0 = 0) {
   {
-    const int r = lane >> 2;                                  // the row this lane feeds as B operand
+    const int r = row0 + (lane >> 2);                         // the row this lane feeds as B operand
     const bool ok = r < p.R;
     const int req = seq * p.stack + r / p.G, head = kvh * p.G + r % p.G;
     const __nv_bfloat16 *q = p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + (lane & 3) * 2;
@@ -423,7 +424,7 @@ __device__ __forceinline__ void load_rows_n(RowBlockN<D> &rb, const ScanParams &
       rb.qb[kk][1] = ok ? *reinterpret_cast<const uint32_t *>(q + kk * 16 + 8) : 0u;
     }
   }
-  const int r0 = (lane & 3) * 2;                              // the rows this lane holds scores of
+  const int r0 = row0 + (lane & 3) * 2;                       // the rows this lane holds scores of
   rb.v0 = r0 < p.R;
   rb.v1 = r0 + 1 < p.R;
   const int req0 = seq * p.stack + r0 / p.G, head0 = kvh * p.G + r0 % p.G;
@@ -462,6 +463,22 @@ __device__ __forceinline__ void qk_issue_n(const RowBlockN<D> &rb, uint32_t kt, 
     uint32_t a[4];
     ldsm_x4(kt + (kk >> 2) * (TK * 128) + k_row + ((((2 * kk) & 7) ^ k_x) << 4), a[0], a[1], a[2], a[3]);
     mma_bf16(s, a, rb.qb[kk][0], rb.qb[kk][1]);
+  }
+}
+
+// The same for NT 8-row N tiles at once: one ldmatrix of the K slice feeds every tile's MMA.
+template <int D, int TK, int NT>
+__device__ __forceinline__ void qk_issue_nt(const RowBlockN<D> (&rb)[NT], uint32_t kt, int slice, int lane, float (&s)[NT][4]) {
+  const int k_key = slice * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
+  const uint32_t k_row = k_key * 128, k_x = (lane >> 4) ^ (k_key & 7);
+#pragma unroll
+  for (int t = 0; t < NT; ++t) s[t][0] = s[t][1] = s[t][2] = s[t][3] = 0.f;
+#pragma unroll
+  for (int kk = 0; kk < D / 16; ++kk) {
+    uint32_t a[4];
+    ldsm_x4(kt + (kk >> 2) * (TK * 128) + k_row + ((((2 * kk) & 7) ^ k_x) << 4), a[0], a[1], a[2], a[3]);
+#pragma unroll
+    for (int t = 0; t < NT; ++t) mma_bf16(s[t], a, rb[t].qb[kk][0], rb[t].qb[kk][1]);
   }
 }
 
@@ -515,6 +532,25 @@ __device__ __forceinline__ void value_product_n(float (&o)[D / 16][4], uint32_t 
     else ldsm_x4_trans(vbase + pad_off + mt * 32, a[0], a[1], a[2], a[3]);
     mma_bf16(o[mt], a, bh[0], bh[1]);
     mma_bf16(o[mt], a, bl[0], bl[1]);
+  }
+}
+
+// The same for NT N tiles: one ldmatrix.trans of the V slice feeds every tile's MMAs.
+template <int D, int HALF_ROWS, int NT>
+__device__ __forceinline__ void value_product_nt(float (&o)[NT][D / 16][4], uint32_t vbase, int row0, int lane,
+                                                 const uint32_t (&bh)[NT][2], const uint32_t (&bl)[NT][2], uint32_t skip) {
+  const int v_key = ((lane >> 4) << 3) + (lane & 7);
+  const uint32_t sw_row = (row0 + v_key) * 128, sw_x = ((lane >> 3) & 1) ^ (v_key & 7);
+#pragma unroll
+  for (int mt = 0; mt < D / 16; ++mt) {
+    uint32_t a[4];
+    ldsm_x4_trans(vbase + (mt >> 2) * (HALF_ROWS * 128) + sw_row + ((((2 * mt) & 7) ^ sw_x) << 4), a[0], a[1], a[2], a[3]);
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      if ((skip >> t) & 1u) continue;                        // no key of the slice is live for this tile's rows
+      mma_bf16(o[t][mt], a, bh[t][0], bh[t][1]);
+      mma_bf16(o[t][mt], a, bl[t][0], bl[t][1]);
+    }
   }
 }
 
@@ -706,6 +742,125 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     } else {
       reduce_store_L(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
       reduce_store_A<D>(o, red, slot, R, warp, lane, threadIdx.x, 1);
+    }
+  }
+
+  if (lane == 0) {
+    if (dead) atomicOr(&p.hdr->wait_timeouts, 2u);
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_total);
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Dense decode for row blocks of 9..16 rows: the rows-on-N form with two 8-row N tiles per warp.  A warp still
+// owns slice w of every tile; each ldmatrix of keys or values feeds both tiles' MMAs.
+template <int D>
+struct DenseWideLayout {
+  static constexpr int kTK = narrow_tile_keys<D>();
+  static constexpr int kKTile = kTK * D * 2;
+  static constexpr int kStage = 2 * kKTile;                    // K tile then V tile
+  static constexpr int kPark = D / 16 * 4 * 32 * 4;            // one warp's accumulators of one N tile, fragment order
+  __host__ __device__ static int off_park(int stages) { return stages * kStage; }
+  __host__ __device__ static int off_redl(int stages) { return off_park(stages) + 2 * kPark; }
+  __host__ __device__ static int off_bar(int stages) { return off_redl(stages) + kConsumerWarps * kMaxRows * 4; }
+  __host__ __device__ static int total(int stages) { return off_bar(stages) + 2 * stages * 8 + 1024; }
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDenseThreads, 2)
+fold_scan_dense_nt2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                           const ScanParams p) {
+  using LO = DenseWideLayout<D>;
+  constexpr int TK = LO::kTK, U = TK / 64, KS = 16 * U, NT = 2, C16 = D / 8;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
+  const SeqWork w = seq_work<TK>(p, seq);
+  if (split >= w.n_chunks) return;
+  const int stages = p.stages, R = p.R, n = w.n;
+  const int dstart = draft_start(p, n);
+  const uint32_t full0 = base + LO::off_bar(stages), empty0 = full0 + 8u * stages;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, kConsumerWarps);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();                                                // z (and the zeroed header) come from earlier work
+
+  if (warp == kConsumerWarps) {
+    if (lane == 0) produce_tiles<D, true, LO::kStage, TK>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
+    return;
+  }
+
+  RowBlockN<D> rb[NT];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) load_rows_n<D>(rb[t], p, seq, kvh, lane, 8 * t);
+  float o[NT][D / 16][4];
+#pragma unroll
+  for (int t = 0; t < NT; ++t)
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) o[t][i][0] = o[t][i][1] = o[t][i][2] = o[t][i][3] = 0.f;
+  float l0[NT] = {0.f, 0.f}, l1[NT] = {0.f, 0.f};
+  float *park = reinterpret_cast<float *>(gen + LO::off_park(stages));
+  float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages));
+
+  bool dead = false;
+  int stage = 0;
+  uint32_t phase = 0;
+  unsigned long long st_total = 0;
+
+  for (int c = split; c < w.n_chunks; c += p.num_splits) {
+    const int t_end = min((c + 1) * w.ctiles, w.n_tiles);
+    for (int t = c * w.ctiles; t < t_end; ++t) {
+      const int my_stage = stage;
+      const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+      if (!ready) continue;
+      const uint32_t kt = base + my_stage * LO::kStage;
+      const int key0 = t * TK + warp * KS;
+      st_total += min(KS, max(0, n - key0));
+      if (key0 + KS > n) {                                   // ragged tail: value rows past n may hold anything
+        for (int r = 0; r < KS; ++r)
+          if (key0 + r >= n && lane < C16)
+            *reinterpret_cast<uint4 *>(gen + my_stage * LO::kStage + LO::kKTile +
+                                       tile_off(warp * KS + r, lane, TK)) = make_uint4(0, 0, 0, 0);
+        __syncwarp();
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float s[NT][4];
+        uint32_t bh[NT][2], bl[NT][2];
+        qk_issue_nt<D, TK, NT>(rb, kt, warp * U + u, lane, s);
+        uint32_t skip = 0;
+#pragma unroll
+        for (int q = 0; q < NT; ++q) {
+          if (key0 + 16 * u + 16 > dstart) mask_drafts_n<D>(rb[q], s[q], lane, key0 + 16 * u, dstart);
+          const uint32_t live = weights_n<D, false>(rb[q], s[q], lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh[q], bl[q],
+                                                    l0[q], l1[q]);
+          skip |= live ? 0u : (1u << q);
+        }
+        if (skip != (1u << NT) - 1u) value_product_nt<D, TK, NT>(o, kt + LO::kKTile, (warp * U + u) * 16, lane, bh, bl, skip);
+      }
+      if (key0 + KS > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);
+    }
+    float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
+#pragma unroll
+    for (int q = 0; q < NT; ++q) {
+      const int rows = min(8, R - 8 * q);                    // 8, then what is left (1..8)
+      reduce_store_L_n<kConsumerWarps>(l0[q], l1[q], redl, slot + R * D + 8 * q, rows, warp, lane, threadIdx.x, 1);
+      tree_store_A_n<D>(o[q], park, slot + 8 * q * D, rows, warp, lane, 1);
     }
   }
 
