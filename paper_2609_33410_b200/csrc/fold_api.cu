@@ -327,9 +327,9 @@ int launch_stacked_pair(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams
 }
 
 // Narrow row blocks (rows on N): unpadded value slices; three K stages (measured: a fourth buys nothing and costs L1).
-template <int D, bool TAIL>
+template <int D, bool TAIL, int NT>
 int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
-  using LN = GatedNarrowLayout<D, TAIL>;
+  using LN = GatedNarrowLayout<D, TAIL, NT>;
   const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
   int nvr = 2;
   int nstages = (per_cta2 - LN::total(0, nvr)) / (LN::kKStage + 16);
@@ -343,8 +343,8 @@ int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParam
   p.stages = nstages;
   p.vr = nvr;
   static int configured[64] = {0};
-  if (int rc = opt_in_smem(fold_scan_gated_narrow_kernel<D, TAIL>, configured)) return rc;
-  if (launch_pdl(fold_scan_gated_narrow_kernel<D, TAIL>, grid, dim3(kGatedThreads), LN::total(nstages, nvr), st, mk, mvs, p) !=
+  if (int rc = opt_in_smem(fold_scan_gated_narrow_kernel<D, TAIL, NT>, configured)) return rc;
+  if (launch_pdl(fold_scan_gated_narrow_kernel<D, TAIL, NT>, grid, dim3(kGatedThreads), LN::total(nstages, nvr), st, mk, mvs, p) !=
       cudaSuccess)
     return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
@@ -381,8 +381,13 @@ int launch_gated_wide(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams 
 template <int D>
 int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
   if (p.R <= kNarrowRows)                                    // rows on N; with or without the block tail
-    return p.vmean ? launch_gated_narrow<D, true>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false>(mk, mvs, p, grid, st);
-  return p.vmean ? launch_gated_wide<D, true>(mk, mvs, p, grid, st) : launch_gated_wide<D, false>(mk, mvs, p, grid, st);
+    return p.vmean ? launch_gated_narrow<D, true, 1>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false, 1>(mk, mvs, p, grid, st);
+#ifdef FOLD_TUNING
+  if (getenv("FOLD_TUNE_WIDE"))
+    return p.vmean ? launch_gated_wide<D, true>(mk, mvs, p, grid, st) : launch_gated_wide<D, false>(mk, mvs, p, grid, st);
+#endif
+  // 9..16 rows: two 8-row N tiles per warp
+  return p.vmean ? launch_gated_narrow<D, true, 2>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false, 2>(mk, mvs, p, grid, st);
 }
 
 // CTAs per (sequence, kv head).  A CTA pays a few microseconds to start (barriers, first loads), so it should
@@ -407,8 +412,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const fold_kv &kv = a->kv;
   const bool paged = kv.page_table != nullptr;
   // narrow row blocks walk 16 KB key tiles: 128 keys at D = 64
-  // (so do 9..16-row blocks at T = inf, which run the two-tile rows-on-N kernel)
-  bool narrow_tiles = g.R <= kNarrowRows || (g.R <= kMaxRows && isinf(a->depth_T));
+  // (row blocks of 9..16 rows run the same kernels with two N tiles per warp)
+  bool narrow_tiles = g.R <= kMaxRows;
 #ifdef FOLD_TUNING
   if (getenv("FOLD_TUNE_WIDE") && g.R > kNarrowRows) narrow_tiles = false;
 #endif

@@ -96,7 +96,7 @@ struct GatedLayout {
 
 // Narrow gated kernel: every value slice in the swizzled box layout (no row padding), and a two-warp
 // parking area for the chunk-end add.
-template <int D, bool TAIL = false>
+template <int D, bool TAIL = false, int NT = 1>
 struct GatedNarrowLayout {
   static constexpr int kTK = narrow_tile_keys<D>();          // keys per tile
   static constexpr int kU = kTK / 64;                        // 16-key sub-slices per warp slice
@@ -104,7 +104,7 @@ struct GatedNarrowLayout {
   static constexpr int kVSlice = 16 * kU * D * 2;            // [D/64 halves][16 kU rows][128 B], swizzled
   // per slice: 16 B of B-operand registers per lane and sub-slice; with the block tail each lane's cut mass of its
   // two rows (8 B per lane) and the mean value row of the slice's block (D * 2 <= 256 B); the verdict words
-  static constexpr int kPEntry = kU * 512 + (TAIL ? 512 : 0) + 32;
+  static constexpr int kPEntry = kU * NT * 512 + (TAIL ? NT * 256 + 256 : 0) + 32;   // NT: 8-row N tiles per warp
   static constexpr int kMeanBytes = (kTK / 64) * D * 2;      // mean rows that ride with a K tile: one per 64-key block
   static constexpr int kKStage = kKTile + (TAIL ? 1024 : 0); // K tile (+ mean rows), 1 KB-aligned for the swizzle
   static constexpr int kPark = D / 16 * 4 * 32 * 4;          // one warp's accumulators, fragment order
@@ -1225,11 +1225,13 @@ fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 // inside one block; its scorer publishes every lane's cut mass and a copy of the block's mean row with the slice;
 // the multiplier sums the cut mass per row and adds cut mass x mean after the slice's products.  A slice with no
 // live key still does that part.
-template <int D, bool TAIL>
+// NT = 2: row blocks of 9..16 rows as two 8-row N tiles per warp (one ldmatrix feeds both tiles' MMAs; the verdict is
+// ORed over all 16 rows).
+template <int D, bool TAIL, int NT>
 __global__ void __launch_bounds__(kGatedThreads, 2)
 fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
                               const ScanParams p) {
-  using LO = GatedNarrowLayout<D, TAIL>;
+  using LO = GatedNarrowLayout<D, TAIL, NT>;
   constexpr int TK = LO::kTK, U = LO::kU, KS = 16 * U;       // keys per tile, sub-slices and keys per warp slice
   constexpr int C16 = D / 8;                                 // 16-byte chunks per value row
   constexpr int RPI = 32 / C16;                              // rows one warp-wide async copy covers
@@ -1271,7 +1273,7 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
 
   const bool scorer = warp < SW;
   const int sl = warp & 3;                                   // the slice of every tile this warp owns
-  constexpr int pentry = LO::kPEntry, pcut = U * 512, pmean = U * 512 + 256, pmask = pentry - 32;
+  constexpr int pentry = LO::kPEntry, pcut = U * NT * 512, pmean = pcut + NT * 256, pmask = pentry - 32;
   uint8_t *pring = gen + LO::off_pring(stages, vr) + sl * vr * pentry;
   const uint32_t vring = base + LO::off_vring(stages) + sl * vr * LO::kVSlice;
   const uint32_t vfull = vfull0 + 8u * sl * vr, vempty = vempty0 + 8u * sl * vr;
@@ -1280,9 +1282,13 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   uint32_t vphase = 0, vwrapped = 0;
 
   if (scorer) {
-    RowBlockN<D> rb;
-    load_rows_n<D>(rb, p, seq, kvh, lane);
-    float l0 = 0.f, l1 = 0.f;
+    RowBlockN<D> rb[NT];
+    float l0[NT], l1[NT];
+#pragma unroll
+    for (int q = 0; q < NT; ++q) {
+      load_rows_n<D>(rb[q], p, seq, kvh, lane, 8 * q);
+      l0[q] = l1[q] = 0.f;
+    }
     float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, vr));
     const int page_mask = (1 << p.page_shift) - 1;
     const uint64_t vpol = policy_evict_first();
@@ -1301,18 +1307,26 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       {
         const bool ready = mbar_wait(full0 + 8u * my_stage, my_phase, dead);
         const int key0 = k.t * TK + sl * KS;
-        uint32_t bh[U][2], bl[U][2];
-        float cm0 = 0.f, cm1 = 0.f;                          // this lane's keys' cut mass for rows (lane%4)*2 + {0,1}
+        uint32_t bh[U][NT][2], bl[U][NT][2];
+        float cm0[NT], cm1[NT];                              // this lane's keys' cut mass for rows 8 q + (lane%4)*2 + {0,1}
         uint2 mean8 = make_uint2(0u, 0u);
         uint32_t fetch = 0;                                  // bit 16 u + k: key k of sub-slice u is live for some row
+        uint32_t tile_live = 0;                              // bit NT u + q: some key of sub-slice u is live for N tile q
 #pragma unroll
-        for (int u = 0; u < U; ++u) bh[u][0] = bh[u][1] = bl[u][0] = bl[u][1] = 0u;
+        for (int q = 0; q < NT; ++q) {
+          cm0[q] = cm1[q] = 0.f;
+#pragma unroll
+          for (int u = 0; u < U; ++u) bh[u][q][0] = bh[u][q][1] = bl[u][q][0] = bl[u][q][1] = 0u;
+        }
         if (ready) {
-          float s[U][4];
+          float s[U][NT][4];
 #pragma unroll
           for (int u = 0; u < U; ++u) {
-            qk_issue_n<D, TK>(rb, base + my_stage * LO::kKStage, sl * U + u, lane, s[u]);
-            if (key0 + 16 * u + 16 > dstart) mask_drafts_n<D>(rb, s[u], lane, key0 + 16 * u, dstart);
+            qk_issue_nt<D, TK, NT>(rb, base + my_stage * LO::kKStage, sl * U + u, lane, s[u]);
+            if (key0 + 16 * u + 16 > dstart) {
+#pragma unroll
+              for (int q = 0; q < NT; ++q) mask_drafts_n<D>(rb[q], s[u][q], lane, key0 + 16 * u, dstart);
+            }
           }
           if (TAIL && lane * 8 < D * 2)                      // this lane's 8 bytes of the slice's block mean row
             mean8 = *reinterpret_cast<const uint2 *>(gen + my_stage * LO::kKStage + LO::kKTile +
@@ -1321,10 +1335,18 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
           if (lane == 0) mbar_arrive(empty0 + 8u * my_stage); // the K slice is consumed: release the tile
 #pragma unroll
           for (int u = 0; u < U; ++u)
-            fetch |= weights_n<D, true, TAIL>(rb, s[u], lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh[u], bl[u], l0, l1,
-                                              &cm0, &cm1) << (16 * u);
+#pragma unroll
+            for (int q = 0; q < NT; ++q) {
+              const uint32_t live = weights_n<D, true, TAIL>(rb[q], s[u][q], lane, key0 + 16 * u, n, p.scale_log2, p.neg_T,
+                                                             bh[u][q], bl[u][q], l0[q], l1[q], &cm0[q], &cm1[q]);
+              fetch |= live << (16 * u);
+              tile_live |= live ? (1u << (NT * u + q)) : 0u;
+            }
         }
-        const bool tail = TAIL && __any_sync(0xffffffffu, cm0 > 0.f || cm1 > 0.f);
+        bool any_cut = false;
+#pragma unroll
+        for (int q = 0; q < NT; ++q) any_cut |= cm0[q] > 0.f || cm1[q] > 0.f;
+        const bool tail = TAIL && __any_sync(0xffffffffu, any_cut);
         // a mostly-live sub-slice is cheaper to fetch whole (one TMA box per 64 channels) than row by row; rows nobody
         // keeps then ride along under a zero weight.  Never past the sequence end: those rows may hold anything.
         uint32_t whole = 0;
@@ -1345,12 +1367,17 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
           uint8_t *pe = pring + my_vs * pentry;
 #pragma unroll
           for (int u = 0; u < U; ++u)
-            *reinterpret_cast<uint4 *>(pe + u * 512 + lane * 16) = make_uint4(bh[u][0], bh[u][1], bl[u][0], bl[u][1]);
+#pragma unroll
+            for (int q = 0; q < NT; ++q)
+              *reinterpret_cast<uint4 *>(pe + (u * NT + q) * 512 + lane * 16) =
+                  make_uint4(bh[u][q][0], bh[u][q][1], bl[u][q][0], bl[u][q][1]);
           if (TAIL && tail) {
-            *reinterpret_cast<float2 *>(pe + pcut + lane * 8) = make_float2(cm0, cm1);
+#pragma unroll
+            for (int q = 0; q < NT; ++q) *reinterpret_cast<float2 *>(pe + pcut + q * 256 + lane * 8) = make_float2(cm0[q], cm1[q]);
             if (lane * 8 < D * 2) *reinterpret_cast<uint2 *>(pe + pmean + lane * 8) = mean8;
           }
-          if (lane == 0) *reinterpret_cast<uint2 *>(pe + pmask) = make_uint2(fetch, tail ? 1u : 0u);
+          // verdict words: the fetch mask; bit 0 = block tail present, bits 8.. = which N tiles have a live key per sub-slice
+          if (lane == 0) *reinterpret_cast<uint2 *>(pe + pmask) = make_uint2(fetch, (tail ? 1u : 0u) | (tile_live << 8));
           const uint32_t bar = vfull + 8u * my_vs;
           const uint32_t vdst = vring + my_vs * LO::kVSlice;
           if (whole) {
@@ -1400,7 +1427,9 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       const int c_done = k.c;
       if (cursor_next(k, w, p.num_splits)) {
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
-        reduce_store_L_n<SW>(l0, l1, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
+#pragma unroll
+        for (int q = 0; q < NT; ++q)
+          reduce_store_L_n<SW>(l0[q], l1[q], redl, slot + R * D + 8 * q, min(8, R - 8 * q), warp, lane, threadIdx.x, 1);
       }
     }
     if (lane == 0) {
@@ -1410,9 +1439,11 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
     }
   } else {
-    float o[D / 16][4];
+    float o[NT][D / 16][4];
 #pragma unroll
-    for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    for (int q = 0; q < NT; ++q)
+#pragma unroll
+      for (int i = 0; i < D / 16; ++i) o[q][i][0] = o[q][i][1] = o[q][i][2] = o[q][i][3] = 0.f;
     float *red = reinterpret_cast<float *>(gen + LO::off_red(stages, vr));
     for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
       const int my = vs;
@@ -1425,23 +1456,31 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           if (((verdict >> (16 * u)) & 0xffffu) == 0u) continue;   // nobody keeps a key of this sub-slice
-          const uint4 a = *reinterpret_cast<const uint4 *>(pe + u * 512 + lane * 16);
-          const uint32_t bh[2] = {a.x, a.y}, bl[2] = {a.z, a.w};
-          value_product_n<D, true, 0, KS>(o, vring + my * LO::kVSlice, 16 * u, lane, bh, bl);
-        }
-        if (TAIL && vw.y != 0u) {                            // o[mt]: channels 16 mt + lane/4 (+8), rows (lane%4)*2 + {0,1}
-          float2 c = make_float2(0.f, 0.f);                  // the rows' cut mass: over the 8 lanes that scored their keys
+          uint32_t bh[NT][2], bl[NT][2];
 #pragma unroll
-          for (int gsrc = 0; gsrc < 8; ++gsrc) {
-            const float2 t = *reinterpret_cast<const float2 *>(pe + pcut + (gsrc * 4 + (lane & 3)) * 8);
-            c.x += t.x; c.y += t.y;
+          for (int q = 0; q < NT; ++q) {
+            const uint4 a = *reinterpret_cast<const uint4 *>(pe + (u * NT + q) * 512 + lane * 16);
+            bh[q][0] = a.x; bh[q][1] = a.y; bl[q][0] = a.z; bl[q][1] = a.w;
           }
+          const uint32_t skip = ~(vw.y >> (8 + NT * u)) & ((1u << NT) - 1u);
+          value_product_nt<D, KS, NT>(o, vring + my * LO::kVSlice, 16 * u, lane, bh, bl, skip);
+        }
+        if (TAIL && (vw.y & 1u)) {                           // o[q][mt]: channels 16 mt + lane/4 (+8), rows 8 q + (lane%4)*2 + {0,1}
           const __nv_bfloat16 *mrow = reinterpret_cast<const __nv_bfloat16 *>(pe + pmean) + (lane >> 2);
 #pragma unroll
-          for (int mt = 0; mt < D / 16; ++mt) {
-            const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
-            o[mt][0] = fmaf(c.x, m0, o[mt][0]); o[mt][1] = fmaf(c.y, m0, o[mt][1]);
-            o[mt][2] = fmaf(c.x, m1, o[mt][2]); o[mt][3] = fmaf(c.y, m1, o[mt][3]);
+          for (int q = 0; q < NT; ++q) {
+            float2 c = make_float2(0.f, 0.f);                // the rows' cut mass: over the 8 lanes that scored their keys
+#pragma unroll
+            for (int gsrc = 0; gsrc < 8; ++gsrc) {
+              const float2 t = *reinterpret_cast<const float2 *>(pe + pcut + q * 256 + (gsrc * 4 + (lane & 3)) * 8);
+              c.x += t.x; c.y += t.y;
+            }
+#pragma unroll
+            for (int mt = 0; mt < D / 16; ++mt) {
+              const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
+              o[q][mt][0] = fmaf(c.x, m0, o[q][mt][0]); o[q][mt][1] = fmaf(c.y, m0, o[q][mt][1]);
+              o[q][mt][2] = fmaf(c.x, m1, o[q][mt][2]); o[q][mt][3] = fmaf(c.y, m1, o[q][mt][3]);
+            }
           }
         }
         __syncwarp();
@@ -1450,7 +1489,8 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       const int c_done = k.c;
       if (cursor_next(k, w, p.num_splits)) {
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
-        tree_store_A_n<D>(o, red, slot, R, sl, lane, 2);
+#pragma unroll
+        for (int q = 0; q < NT; ++q) tree_store_A_n<D>(o[q], red, slot + 8 * q * D, min(8, R - 8 * q), sl, lane, 2);
       }
     }
     if (lane == 0 && dead) atomicOr(&p.hdr->wait_timeouts, 4u);
