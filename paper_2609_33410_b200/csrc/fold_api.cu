@@ -217,9 +217,9 @@ int opt_in_smem(Kernel k, int *configured) {
 }
 
 // Ring depths: two CTAs per SM when a useful ring fits, else one CTA with a deeper ring.
-template <int D, bool NARROW>
-int launch_dense_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
-  using LO = DenseLayout<D, NARROW ? narrow_tile_keys<D>() : kTileKeys>;
+template <int D>
+int launch_dense_n(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
+  using LO = DenseLayout<D, narrow_tile_keys<D>()>;
   const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
   int stages = (per_cta2 - LO::total(0, p.R)) / (LO::kStage + 16);
   if (stages < 3) stages = (kSmemPerCtaMax - LO::total(0, p.R)) / (LO::kStage + 16);
@@ -231,11 +231,12 @@ int launch_dense_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p,
   p.stages = stages;
   p.vr = 0;
   static int configured[64] = {0};
-  if (int rc = opt_in_smem(fold_scan_dense_kernel<D, NARROW>, configured)) return rc;
-  if (launch_pdl(fold_scan_dense_kernel<D, NARROW>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
+  if (int rc = opt_in_smem(fold_scan_dense_kernel<D>, configured)) return rc;
+  if (launch_pdl(fold_scan_dense_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
     return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
+
 // 9..16 rows: rows on N in two 8-row tiles per warp.
 template <int D>
 int launch_dense_nt2(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
@@ -254,12 +255,8 @@ int launch_dense_nt2(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p
 }
 template <int D>
 int launch_dense(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, cudaStream_t st) {
-  // up to 8 rows: rows on N (half the MMAs and accumulators), 16 KB key tiles at either head dimension
-  if (p.R <= kNarrowRows) return launch_dense_as<D, true>(mk, mv, p, grid, st);
-#ifdef FOLD_TUNING
-  if (getenv("FOLD_TUNE_WIDE")) return launch_dense_as<D, false>(mk, mv, p, grid, st);
-#endif
-  return launch_dense_nt2<D>(mk, mv, p, grid, st);
+  // rows on N (half the MMAs and accumulators of rows on M), 16 KB key tiles at either head dimension
+  return p.R <= kNarrowRows ? launch_dense_n<D>(mk, mv, p, grid, st) : launch_dense_nt2<D>(mk, mv, p, grid, st);
 }
 
 // Stacked rows: the dense ring without reduction buffers; one CTA per (split, 64-row group).  With the block tail
@@ -352,40 +349,10 @@ int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParam
 
 // Gated scan: value slots hold rows whose requests can only be issued after scoring, so shared
 // memory is split between the key ring and the value slots of each slice.
-template <int D, bool TAIL>
-int launch_gated_wide(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
-  using LO = GatedLayout<D, TAIL>;
-  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
-  int vr = 2;
-  int stages = (per_cta2 - LO::total(0, vr, p.R)) / (LO::kKStage + 16);
-  if (stages < 2) {
-    vr = 3;
-    stages = (kSmemPerCtaMax - LO::total(0, vr, p.R)) / (LO::kKStage + 16);
-  }
-  if (stages > 8) stages = 8;
-#ifdef FOLD_TUNING
-  if (const char *e = getenv("FOLD_TUNE_STAGES")) stages = atoi(e);
-  if (const char *e = getenv("FOLD_TUNE_VR")) vr = atoi(e);
-  if (const char *e = getenv("FOLD_TUNE_BOXMIN")) p.box_min = atoi(e);
-#endif
-  if (stages < 2 || vr < 1 || LO::total(stages, vr, p.R) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
-  p.stages = stages;
-  p.vr = vr;
-  static int configured[64] = {0};
-  if (int rc = opt_in_smem(fold_scan_gated_kernel<D, TAIL>, configured)) return rc;
-  if (launch_pdl(fold_scan_gated_kernel<D, TAIL>, grid, dim3(kGatedThreads), LO::total(stages, vr, p.R), st, mk, mvs, p) !=
-      cudaSuccess)
-    return FOLD_ECUDA;
-  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
-}
 template <int D>
 int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
   if (p.R <= kNarrowRows)                                    // rows on N; with or without the block tail
     return p.vmean ? launch_gated_narrow<D, true, 1>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false, 1>(mk, mvs, p, grid, st);
-#ifdef FOLD_TUNING
-  if (getenv("FOLD_TUNE_WIDE"))
-    return p.vmean ? launch_gated_wide<D, true>(mk, mvs, p, grid, st) : launch_gated_wide<D, false>(mk, mvs, p, grid, st);
-#endif
   // 9..16 rows: two 8-row N tiles per warp
   return p.vmean ? launch_gated_narrow<D, true, 2>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false, 2>(mk, mvs, p, grid, st);
 }
@@ -413,10 +380,7 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const bool paged = kv.page_table != nullptr;
   // narrow row blocks walk 16 KB key tiles: 128 keys at D = 64
   // (row blocks of 9..16 rows run the same kernels with two N tiles per warp)
-  bool narrow_tiles = g.R <= kMaxRows;
-#ifdef FOLD_TUNING
-  if (getenv("FOLD_TUNE_WIDE") && g.R > kNarrowRows) narrow_tiles = false;
-#endif
+  const bool narrow_tiles = g.R <= kMaxRows;
   const int tile_keys = (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
   const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   const bool gated = !isinf(a->depth_T);

@@ -10,15 +10,16 @@
 //            whether a key's value is used; L sums every key's weight
 //   values   two-term BF16 weights (P_hi + P_lo) times V, FP32 accumulate
 //
-// Row blocks of up to 8 rows (every GQA group up to 8) put the rows on the MMA's N side (keys, then
-// channels, on M): half the MMAs and accumulators of the rows-on-M form, which blocks of 9..16 rows
-// use.  Narrow blocks walk 16 KB key tiles at either head dimension (a warp's slice is 4 KB of keys:
-// 16 keys at D = 128, 32 at D = 64); the rows-on-M kernels walk 64-key tiles with 16-key slices.
+// Row blocks (up to 16 rows per (sequence, kv head)) put the rows on the MMA's N side (keys, then
+// channels, on M) in one or two 8-row N tiles: half the MMAs and accumulators of a rows-on-M form,
+// which only the mma.sync stacked-row kernel still uses.  Row-block kernels walk 16 KB key tiles at
+// either head dimension (a warp's slice is 4 KB of keys: 16 keys at D = 128, 32 at D = 64); the
+// stacked-row kernel walks 64-key tiles with 16-key slices.
 //
 // Kernels:
-//   fold_scan_dense_kernel<D, NARROW> (T = inf): K and V tiles arrive together by TMA; four consumer
-//     warps score and multiply in place.
-//   fold_scan_gated_narrow_kernel<D> / fold_scan_gated_kernel<D> (finite T): only K is prefetched.
+//   fold_scan_dense_kernel<D> / fold_scan_dense_nt2_kernel<D> (T = inf; up to 8 / 9..16 rows): K and V
+//     tiles arrive together by TMA; four consumer warps score and multiply in place.
+//   fold_scan_gated_narrow_kernel<D, TAIL, NT> (finite T): only K is prefetched.
 //     Four scorer warps score a slice, publish its weights and request just the value rows some row of
 //     the group keeps -- a whole 16-key sub-slice by one TMA box when most of it is live, else row by
 //     row with zero-filling 16-byte async copies; four multiplier warps wait for those rows and
@@ -70,28 +71,6 @@ struct DenseLayout {
   __host__ __device__ static int off_redl(int stages, int R) { return off_red(stages) + kConsumerWarps * R * D * 4; }
   __host__ __device__ static int off_bar(int stages, int R) { return off_redl(stages, R) + kConsumerWarps * kMaxRows * 4; }
   __host__ __device__ static int total(int stages, int R) { return off_bar(stages, R) + 2 * stages * 8 + 1024; }
-};
-
-template <int D, bool TAIL = false>
-struct GatedLayout {
-  static constexpr int kKTile = kTileKeys * D * 2;
-  static constexpr int kKStage = kKTile + (TAIL ? 1024 : 0);   // K tile (+ the block's mean row)
-  static constexpr int kVRow = D * 2 + 16;          // value row + 16 B pad: conflict-free ldmatrix
-  // one slice's 16 value rows: padded rows (row-by-row fetch) or a swizzled TMA box (whole slice),
-  // so the slot is 1 KB aligned
-  static constexpr int kVSlice = ((16 * kVRow + 1023) / 1024) * 1024;
-  // a slice's weights as A-operand registers (hi and lo terms; rows 8..15 only when present) + its fetch mask
-  // with the block tail: + every lane's cut mass of its two rows (256 B) + the block's mean row (256 B)
-  __host__ __device__ static int pentry(int R) { return (R > 8 ? 1024 : 512) + (TAIL ? 512 : 0) + 32; }
-  __host__ __device__ static int off_vring(int stages) { return stages * kKStage; }
-  __host__ __device__ static int off_pring(int stages, int vr) { return off_vring(stages) + kConsumerWarps * vr * kVSlice; }
-  __host__ __device__ static int off_red(int stages, int vr, int R) { return off_pring(stages, vr) + kConsumerWarps * vr * pentry(R); }
-  __host__ __device__ static int off_redl(int stages, int vr, int R) { return off_red(stages, vr, R) + kConsumerWarps * R * D * 4; }
-  __host__ __device__ static int off_bar(int stages, int vr, int R) { return off_redl(stages, vr, R) + kConsumerWarps * kMaxRows * 4; }
-  // barriers: K full / empty per stage, then value full / empty per (slice, slot)
-  __host__ __device__ static int total(int stages, int vr, int R) {
-    return off_bar(stages, vr, R) + 2 * stages * 8 + 2 * kConsumerWarps * vr * 8 + 1024;
-  }
 };
 
 // Narrow gated kernel: every value slice in the swizzled box layout (no row padding), and a two-warp
@@ -359,43 +338,6 @@ __device__ __forceinline__ void tail_update(float (&o)[D / 8][4], float c_lo, fl
   }
 }
 
-// Chunk end, A part: the four warps of a role park their partials, then 128 threads add them in
-// warp order and store the chunk slot's A.  `bar_id` is the role's named barrier.
-template <int D>
-__device__ __forceinline__ void reduce_store_A(float (&o)[D / 8][4], float *red, float *slot, int R, int warp,
-                                               int lane, int tid128, int bar_id) {
-  const int row_lo = lane >> 2, row_hi = row_lo + 8, qcol = (lane & 3) * 2;
-  float *mine = red + warp * R * D;
-#pragma unroll
-  for (int nt = 0; nt < D / 8; ++nt) {
-    if (row_lo < R) *reinterpret_cast<float2 *>(mine + row_lo * D + nt * 8 + qcol) = make_float2(o[nt][0], o[nt][1]);
-    if (row_hi < R) *reinterpret_cast<float2 *>(mine + row_hi * D + nt * 8 + qcol) = make_float2(o[nt][2], o[nt][3]);
-    o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-  }
-  named_bar(bar_id);
-  const int RD = R * D;
-  for (int i = tid128; i < RD; i += 128) slot[i] = ((red[i] + red[RD + i]) + red[2 * RD + i]) + red[3 * RD + i];
-  named_bar(bar_id);
-}
-// Chunk end, L part.
-__device__ __forceinline__ void reduce_store_L(float &l_lo, float &l_hi, float *redl, float *slot_l, int R, int warp,
-                                               int lane, int tid128, int bar_id) {
-  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
-  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
-  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-  const int row_lo = lane >> 2, row_hi = row_lo + 8;
-  if ((lane & 3) == 0) {
-    if (row_lo < R) redl[warp * kMaxRows + row_lo] = l_lo;
-    if (row_hi < R) redl[warp * kMaxRows + row_hi] = l_hi;
-  }
-  l_lo = l_hi = 0.f;
-  named_bar(bar_id);
-  if (tid128 < R)
-    slot_l[tid128] = ((redl[tid128] + redl[kMaxRows + tid128]) + redl[2 * kMaxRows + tid128]) + redl[3 * kMaxRows + tid128];
-  named_bar(bar_id);
-}
-
 // ------------------------------------------------------------------------------------------------
 // Narrow row blocks (at most 8 query rows per (sequence, kv head): every GQA group up to 8).
 // The products are turned round -- keys, then channels, on M and the query rows on N = 8 -- as
@@ -645,11 +587,11 @@ __device__ __forceinline__ void reduce_store_L_n(float &l0, float &l1, float *re
 
 // ------------------------------------------------------------------------------------------------
 // Dense decode (T = inf)
-template <int D, bool NARROW>
+template <int D>
 __global__ void __launch_bounds__(kDenseThreads, 2)
 fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                        const ScanParams p) {
-  constexpr int TK = NARROW ? narrow_tile_keys<D>() : kTileKeys;   // keys per tile
+  constexpr int TK = narrow_tile_keys<D>();                        // keys per tile
   constexpr int U = TK / 64, KS = 16 * U;                          // 16-key sub-slices and keys per warp slice
   using LO = DenseLayout<D, TK>;
   constexpr int C16 = D / 8;
@@ -683,12 +625,11 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     return;
   }
 
-  // rows on M (up to 16 rows) or on N (up to 8 rows): see "Narrow row blocks"
-  typename std::conditional<NARROW, RowBlockN<D>, RowBlock<D>>::type rb;
-  if constexpr (NARROW) load_rows_n<D>(rb, p, seq, kvh, lane); else load_rows<D>(rb, p, seq, kvh, lane);
-  float o[NARROW ? D / 16 : D / 8][4];
+  RowBlockN<D> rb;                                           // rows on N: see "Narrow row blocks"
+  load_rows_n<D>(rb, p, seq, kvh, lane);
+  float o[D / 16][4];
 #pragma unroll
-  for (int i = 0; i < (NARROW ? D / 16 : D / 8); ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
   float l_lo = 0.f, l_hi = 0.f;
   float *red = reinterpret_cast<float *>(gen + LO::off_red(stages));
   float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, R));
@@ -715,34 +656,22 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
                                        tile_off(warp * KS + r, lane, TK)) = make_uint4(0, 0, 0, 0);
         __syncwarp();
       }
-      if constexpr (NARROW) {
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          float s[4];
-          uint32_t bh[2], bl[2];
-          qk_issue_n<D, TK>(rb, kt, warp * U + u, lane, s);
-          if (key0 + 16 * u + 16 > dstart) mask_drafts_n<D>(rb, s, lane, key0 + 16 * u, dstart);
-          const uint32_t fetch16 = weights_n<D, false>(rb, s, lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh, bl, l_lo, l_hi);
-          if (fetch16 != 0) value_product_n<D, true, 0, TK>(o, kt + LO::kKTile, (warp * U + u) * 16, lane, bh, bl);
-        }
-      } else {
-        uint32_t ah[4], al[4];
-        const uint32_t fetch16 = score_slice<D, false>(rb, kt, warp, lane, key0, n, p.scale_log2, p.neg_T, ah, al, l_lo, l_hi,
-                                                       nullptr, nullptr, dstart);
-        if (fetch16 != 0) value_product<D, true, 0>(o, kt + LO::kKTile, warp * 16, lane, ah, al);
+      for (int u = 0; u < U; ++u) {
+        float s[4];
+        uint32_t bh[2], bl[2];
+        qk_issue_n<D, TK>(rb, kt, warp * U + u, lane, s);
+        if (key0 + 16 * u + 16 > dstart) mask_drafts_n<D>(rb, s, lane, key0 + 16 * u, dstart);
+        const uint32_t fetch16 = weights_n<D, false>(rb, s, lane, key0 + 16 * u, n, p.scale_log2, p.neg_T, bh, bl, l_lo, l_hi);
+        if (fetch16 != 0) value_product_n<D, true, 0, TK>(o, kt + LO::kKTile, (warp * U + u) * 16, lane, bh, bl);
       }
       if (key0 + KS > n) fence_proxy_async_smem();           // generic writes before the next TMA fill
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);
     }
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
-    if constexpr (NARROW) {
-      reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
-      reduce_store_A_n<D, kConsumerWarps>(o, red, slot, R, warp, lane, threadIdx.x, 1);
-    } else {
-      reduce_store_L(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
-      reduce_store_A<D>(o, red, slot, R, warp, lane, threadIdx.x, 1);
-    }
+    reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
+    reduce_store_A_n<D, kConsumerWarps>(o, red, slot, R, warp, lane, threadIdx.x, 1);
   }
 
   if (lane == 0) {
@@ -993,226 +922,6 @@ fold_scan_stacked_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       keys += min((c + 1) * w.ctiles * kTileKeys, n) - c * w.ctiles * kTileKeys;
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), keys);
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), keys);
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Depth-gated decode (finite T)
-//
-// Roles.  Scorer warp w: waits for a K tile, scores slice w, releases the tile, publishes the
-// slice's weights and verdict and requests the value rows the verdict asks for into a slot of
-// its slice's value ring -- the whole slice by TMA when most rows are live, else row by row
-// with zero-filling 16-byte async copies (cut rows are not read and become zero rows).
-// Multiplier warp w: waits for a slot to land, multiplies, hands the slot back.
-// TAIL: the block tail, as in the narrow kernel below (mean rows ride with the K tiles; the scorer publishes every
-// lane's cut mass and the block's mean row with the slice; the multiplier adds cut mass x mean).
-template <int D, bool TAIL>
-__global__ void __launch_bounds__(kGatedThreads, 2)
-fold_scan_gated_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVs,
-                       const ScanParams p) {
-  using LO = GatedLayout<D, TAIL>;
-  constexpr int C16 = D / 8;                                 // 16-byte chunks per value row
-  constexpr int RPI = 32 / C16;                              // rows one warp-wide async copy covers
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;
-  uint8_t *gen = smem_raw + (base - raw);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // kv heads fastest: CTAs that run together read the same tokens' rows, which sit side by side in memory
-  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
-  const SeqWork w = seq_work(p, seq);
-  if (split >= w.n_chunks) return;
-  const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
-  const int dstart = draft_start(p, n);                     // keys from here on are per-request drafts
-  // barriers: K full / empty per stage; value full / empty per (slice, slot)
-  const uint32_t full0 = base + LO::off_bar(stages, vr, R), empty0 = full0 + 8u * stages;
-  const uint32_t vfull0 = empty0 + 8u * stages, vempty0 = vfull0 + 8u * kConsumerWarps * vr;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(full0 + 8u * s, 1);
-      mbar_init(empty0 + 8u * s, kConsumerWarps);
-    }
-    for (int s = 0; s < kConsumerWarps * vr; ++s) {
-      mbar_init(vfull0 + 8u * s, 1);
-      mbar_init(vempty0 + 8u * s, 1);
-    }
-    mbar_fence_init();
-  }
-  __syncthreads();
-  pdl_launch_dependents();
-  pdl_wait();                                                // z (and the zeroed header) come from earlier work
-
-  if (warp == 2 * kConsumerWarps) {
-    if (lane == 0) produce_tiles<D, false, LO::kKStage, kTileKeys, TAIL>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
-    return;
-  }
-
-  const bool scorer = warp < kConsumerWarps;
-  const int sl = warp & 3;                                   // the slice of every tile this warp owns
-  const int pentry = LO::pentry(R), pmask = pentry - 32, pcut = pmask - 512, pmean = pmask - 256;
-  uint8_t *pring = gen + LO::off_pring(stages, vr) + sl * vr * pentry;
-  const uint32_t vring = base + LO::off_vring(stages) + sl * vr * LO::kVSlice;
-  const uint32_t vfull = vfull0 + 8u * sl * vr, vempty = vempty0 + 8u * sl * vr;
-  bool dead = false;
-  int vs = 0;
-  uint32_t vphase = 0, vwrapped = 0;
-
-  if (scorer) {
-    RowBlock<D> rb;
-    load_rows<D>(rb, p, seq, kvh, lane);
-    float l_lo = 0.f, l_hi = 0.f;
-    float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, vr, R));
-    const int page_mask = (1 << p.page_shift) - 1;
-    const uint64_t vpol = policy_evict_first();
-    // row-by-row fetch: lane covers 16-byte chunk (lane % C16) of rows (lane / C16) + RPI * i
-    const uint32_t rdst0 = (lane / C16) * LO::kVRow + (lane % C16) * 16;
-    const long long rsrc0 = (long long)(lane / C16) * p.v_stride_tok + (lane % C16) * 8;
-    int stage = 0;
-    uint32_t phase = 0;
-    unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
-
-    for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
-      const int my_stage = stage;
-      const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
-      if (++stage == stages) { stage = 0; phase ^= 1u; }
-      const int key0 = k.t * kTileKeys + sl * 16;
-      uint32_t ah[4] = {0u, 0u, 0u, 0u}, al[4] = {0u, 0u, 0u, 0u};
-      uint32_t fetch16 = 0;
-      float c_lo = 0.f, c_hi = 0.f;                          // this lane's keys' cut mass for its two rows
-      uint2 mean8 = make_uint2(0u, 0u);
-      if (ready) {
-        fetch16 = score_slice<D, true, TAIL>(rb, base + my_stage * LO::kKStage, sl, lane, key0, n, p.scale_log2, p.neg_T, ah,
-                                             al, l_lo, l_hi, &c_lo, &c_hi, dstart);
-        if (TAIL && lane * 8 < D * 2)                        // this lane's 8 bytes of the tile's block mean row
-          mean8 = *reinterpret_cast<const uint2 *>(gen + my_stage * LO::kKStage + LO::kKTile + lane * 8);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);   // the K tile is in registers: release it
-      }
-      // a mostly-live slice is cheaper to fetch whole (two TMA boxes) than row by row; rows nobody keeps
-      // then ride along under a zero weight.  Never past the sequence end: those rows may hold anything.
-      const bool whole = (key0 + 16 <= n) && (__popc(fetch16) >= p.box_min);
-      {
-        const int nvalid = min(16, max(0, n - key0));
-        st_total += nvalid;
-        st_fetched += whole ? 16 : __popc(fetch16);
-        st_skipped += (fetch16 == 0 && nvalid > 0) ? 1 : 0;
-      }
-      if (!vwrapped || mbar_wait(vempty + 8u * vs, vphase ^ 1u, dead)) {
-        // publish the slice: weights as the value product's A-operand registers, and the verdict
-        uint8_t *pe = pring + vs * pentry;
-        if (rb.two_blocks) {
-          *reinterpret_cast<uint4 *>(pe + lane * 16) = make_uint4(ah[0], ah[1], ah[2], ah[3]);
-          *reinterpret_cast<uint4 *>(pe + 512 + lane * 16) = make_uint4(al[0], al[1], al[2], al[3]);
-        } else {
-          *reinterpret_cast<uint4 *>(pe + lane * 16) = make_uint4(ah[0], ah[2], al[0], al[2]);
-        }
-        const bool tail = TAIL && __any_sync(0xffffffffu, c_lo > 0.f || c_hi > 0.f);
-        if (TAIL && tail) {
-          *reinterpret_cast<float2 *>(pe + pcut + lane * 8) = make_float2(c_lo, c_hi);
-          if (lane * 8 < D * 2) *reinterpret_cast<uint2 *>(pe + pmean + lane * 8) = mean8;
-        }
-        if (lane == 0) *reinterpret_cast<uint2 *>(pe + pmask) = make_uint2(fetch16 | (whole ? 0x10000u : 0u), tail ? 1u : 0u);
-        const uint32_t bar = vfull + 8u * vs;
-        if (fetch16 != 0u) {
-          int c_seq = seq, c_tok = key0;
-          if (p.paged) {
-            const int pg = p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)];
-            c_seq = min(max(pg, 0), p.num_pages - 1);
-            c_tok = key0 & page_mask;
-          }
-          const uint32_t vdst = vring + vs * LO::kVSlice;
-          if (whole) {
-            fence_proxy_async_smem();                        // the slot's earlier generic-proxy traffic, then TMA writes
-            __syncwarp();
-            if (lane == 0) {
-              mbar_expect_tx(bar, 16 * D * 2);
-              const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
-              const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
-              const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
-#pragma unroll
-              for (int h = 0; h < D / 64; ++h) tma_load_4d(vdst + h * (16 * 128), &tmVs, bar, h * 64, c1, c2, c3, vpol);
-            }
-          } else {
-            const __nv_bfloat16 *src = p.v + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
-                                       (long long)kvh * p.v_stride_head + rsrc0;
-            uint32_t dst = vdst + rdst0;
-#pragma unroll
-            for (int i = 0; i < 16 / RPI; ++i) {
-              const bool f = (fetch16 >> (i * RPI + lane / C16)) & 1u;
-              cp_async_16(dst, f ? src : p.v, f ? 16u : 0u);
-              dst += RPI * LO::kVRow;
-              src += (long long)RPI * p.v_stride_tok;
-            }
-            cp_async_mbar_arrive(bar);                       // this lane's copies hold the phase open
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar);
-          }
-        } else {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar);
-        }
-      }
-      if (++vs == vr) { vs = 0; vwrapped = 1u; vphase ^= 1u; }
-      const int c_done = k.c;
-      if (cursor_next(k, w, p.num_splits)) {
-        float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
-        reduce_store_L(l_lo, l_hi, redl, slot + R * D, R, sl, lane, threadIdx.x, 1);
-      }
-    }
-    if (lane == 0) {
-      if (dead) atomicOr(&p.hdr->wait_timeouts, 2u);
-      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_fetched);
-      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
-      if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
-    }
-  } else {
-    float o[D / 8][4];
-#pragma unroll
-    for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-    float *red = reinterpret_cast<float *>(gen + LO::off_red(stages, vr, R));
-    for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w);) {
-      const int my = vs;
-      const bool landed = mbar_wait(vfull + 8u * my, vphase, dead);
-      if (++vs == vr) { vs = 0; vphase ^= 1u; }
-      if (landed) {
-        const uint8_t *pe = pring + my * pentry;
-        const uint2 vw = *reinterpret_cast<const uint2 *>(pe + pmask);
-        const uint32_t verdict = vw.x;
-        if (verdict != 0u) {
-          uint32_t ah[4], al[4];
-          const uint4 a = *reinterpret_cast<const uint4 *>(pe + lane * 16);
-          if (R > 8) {
-            const uint4 b = *reinterpret_cast<const uint4 *>(pe + 512 + lane * 16);
-            ah[0] = a.x; ah[1] = a.y; ah[2] = a.z; ah[3] = a.w;
-            al[0] = b.x; al[1] = b.y; al[2] = b.z; al[3] = b.w;
-          } else {
-            ah[0] = a.x; ah[1] = 0u; ah[2] = a.y; ah[3] = 0u;
-            al[0] = a.z; al[1] = 0u; al[2] = a.w; al[3] = 0u;
-          }
-          if (verdict & 0x10000u) value_product<D, true, 0, 16>(o, vring + my * LO::kVSlice, 0, lane, ah, al);
-          else value_product<D, false, LO::kVRow>(o, vring + my * LO::kVSlice, 0, lane, ah, al);
-        }
-        if (TAIL && vw.y != 0u) {                            // the rows' cut mass: over the four lanes that scored their keys
-          float c_lo = 0.f, c_hi = 0.f;
-#pragma unroll
-          for (int qsrc = 0; qsrc < 4; ++qsrc) {
-            const float2 t = *reinterpret_cast<const float2 *>(pe + pcut + ((lane & ~3) + qsrc) * 8);
-            c_lo += t.x; c_hi += t.y;
-          }
-          tail_update<D>(o, c_lo, c_hi, reinterpret_cast<const __nv_bfloat16 *>(pe + pmean), lane);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(vempty + 8u * my);
-      }
-      const int c_done = k.c;
-      if (cursor_next(k, w, p.num_splits)) {
-        float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
-        reduce_store_A<D>(o, red, slot, R, sl, lane, threadIdx.x - 128, 2);
-      }
-    }
-    if (lane == 0 && dead) atomicOr(&p.hdr->wait_timeouts, 4u);
   }
 }
 
