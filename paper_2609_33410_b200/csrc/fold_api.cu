@@ -357,6 +357,15 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
   return p.vmean ? launch_gated_narrow<D, true, 2>(mk, mvs, p, grid, st) : launch_gated_narrow<D, false, 2>(mk, mvs, p, grid, st);
 }
 
+// Rows per (sequence, kv head) up to which the row-block kernels run (in 16-row groups, each its own CTA sharing the
+// kv head's tiles through L2); beyond, the stacked-row kernels.
+int row_block_rows() {
+#ifdef FOLD_TUNING
+  if (const char *e = getenv("FOLD_TUNE_RGMAX")) return atoi(e);
+#endif
+  return 2 * kMaxRows;
+}
+
 // CTAs per (sequence, kv head).  A CTA pays a few microseconds to start (barriers, first loads), so it should
 // walk at least ~32 tiles; below about one and a half waves of CTAs the machine is not filled, so short
 // batches are cut finer instead.  Only scheduling: the result does not depend on the choice.
@@ -364,7 +373,8 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   const int n = a->kv.max_seqlen;
   const int max_chunks = num_chunks_of(n) > 0 ? num_chunks_of(n) : 1;
   if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
-  const long long units = (long long)g.num_seqs * g.Hkv * (g.R > 128 ? (g.R + 255) / 256 : 1);   // CTAs per split
+  const long long units = (long long)g.num_seqs * g.Hkv *
+                          (g.R > 128 ? (g.R + 255) / 256 : (g.R <= row_block_rows() ? (g.R + kMaxRows - 1) / kMaxRows : 1));   // CTAs per split
   const int tiles_unit = max_chunks * (chunk_keys_of(n) / tile_keys);
   int s = tiles_unit / 32;
   s = s < 1 ? 1 : (s > max_chunks ? max_chunks : s);
@@ -380,14 +390,14 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const bool paged = kv.page_table != nullptr;
   // narrow row blocks walk 16 KB key tiles: 128 keys at D = 64
   // (row blocks of 9..16 rows run the same kernels with two N tiles per warp)
-  const bool narrow_tiles = g.R <= kMaxRows;
+  const bool narrow_tiles = g.R <= row_block_rows();
   const int tile_keys = (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
   const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   const bool gated = !isinf(a->depth_T);
   CUtensorMap mk, mv;
   MapAxes axes;
   if (int rc = make_map(&mk, &axes, kv.k, kv, g.D, g.Hkv, box_tok)) return rc;
-  const bool stacked = g.R > kMaxRows;
+  const bool stacked = g.R > row_block_rows();
   // dense and stacked: value tiles like key tiles; gated: a box of one 16-key slice
   if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, (gated && !stacked) ? 16 : box_tok)) return rc;
 
@@ -418,7 +428,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
 
   // row-block kernels: kv heads on x (fastest), splits on y; stacked kernels: (row group, split) on x, heads on y
-  const dim3 grid = stacked ? dim3(p.num_splits, g.Hkv, g.num_seqs) : dim3(g.Hkv, p.num_splits, g.num_seqs);
+  p.row_groups = stacked || g.R <= kMaxRows ? 1 : (g.R + kMaxRows - 1) / kMaxRows;
+  const dim3 grid = stacked ? dim3(p.num_splits, g.Hkv, g.num_seqs) : dim3(g.Hkv * p.row_groups, p.num_splits, g.num_seqs);
   p.box_min = 13;
   if (stacked) {
     // the tcgen05 kernels have no block tail yet: a gated stacked level with a mean table runs on mma.sync

@@ -55,6 +55,7 @@ struct ScanParams {
   int paged, page_shift, max_pages, num_pages, box_tok;
   int num_splits, stages, vr;
   int pos_tok, pos_head, pos_seq;                 // which tensor-map coordinate (1..3) each axis is
+  int row_groups;                                 // row-block kernels: 16-row groups per (sequence, kv head), each its own CTA
   int box_min;                                    // gated: fetch a whole slice by one TMA box from this many live rows on
   float scale_log2, neg_T;
 };
@@ -708,7 +709,9 @@ fold_scan_dense_nt2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
   uint8_t *gen = smem_raw + (base - raw);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
+  // x = row group + row_groups * kv head: the 16-row groups of a kv head sit side by side and share its tiles in L2
+  const int rg = blockIdx.x % p.row_groups, kvh = blockIdx.x / p.row_groups, split = blockIdx.y, seq = blockIdx.z;
+  const int rbase = rg * 16;                                 // first row of this CTA's group
   const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, R = p.R, n = w.n;
@@ -733,7 +736,7 @@ fold_scan_dense_nt2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
 
   RowBlockN<D> rb[NT];
 #pragma unroll
-  for (int t = 0; t < NT; ++t) load_rows_n<D>(rb[t], p, seq, kvh, lane, 8 * t);
+  for (int t = 0; t < NT; ++t) load_rows_n<D>(rb[t], p, seq, kvh, lane, rbase + 8 * t);
   float o[NT][D / 16][4];
 #pragma unroll
   for (int t = 0; t < NT; ++t)
@@ -787,9 +790,9 @@ fold_scan_dense_nt2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
 #pragma unroll
     for (int q = 0; q < NT; ++q) {
-      const int rows = min(8, R - 8 * q);                    // 8, then what is left (1..8)
-      reduce_store_L_n<kConsumerWarps>(l0[q], l1[q], redl, slot + R * D + 8 * q, rows, warp, lane, threadIdx.x, 1);
-      tree_store_A_n<D>(o[q], park, slot + 8 * q * D, rows, warp, lane, 1);
+      const int rows = min(8, R - rbase - 8 * q);            // 8, then what is left (possibly none)
+      reduce_store_L_n<kConsumerWarps>(l0[q], l1[q], redl, slot + R * D + rbase + 8 * q, rows, warp, lane, threadIdx.x, 1);
+      tree_store_A_n<D>(o[q], park, slot + (rbase + 8 * q) * D, rows, warp, lane, 1);
     }
   }
 
@@ -952,7 +955,9 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // kv heads fastest: CTAs that run together read the same tokens' rows, which sit side by side in memory
-  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
+  // x = row group + row_groups * kv head (row groups only with NT = 2: more than 16 rows)
+  const int rg = blockIdx.x % p.row_groups, kvh = blockIdx.x / p.row_groups, split = blockIdx.y, seq = blockIdx.z;
+  const int rbase = rg * 16;                                 // first row of this CTA's group
   const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
   const int stages = p.stages, vr = p.vr, R = p.R, n = w.n;
@@ -995,7 +1000,7 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     float l0[NT], l1[NT];
 #pragma unroll
     for (int q = 0; q < NT; ++q) {
-      load_rows_n<D>(rb[q], p, seq, kvh, lane, 8 * q);
+      load_rows_n<D>(rb[q], p, seq, kvh, lane, rbase + 8 * q);
       l0[q] = l1[q] = 0.f;
     }
     float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages, vr));
@@ -1138,7 +1143,8 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
 #pragma unroll
         for (int q = 0; q < NT; ++q)
-          reduce_store_L_n<SW>(l0[q], l1[q], redl, slot + R * D + 8 * q, min(8, R - 8 * q), warp, lane, threadIdx.x, 1);
+          reduce_store_L_n<SW>(l0[q], l1[q], redl, slot + R * D + rbase + 8 * q, min(8, R - rbase - 8 * q), warp, lane,
+                               threadIdx.x, 1);
       }
     }
     if (lane == 0) {
@@ -1199,7 +1205,7 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       if (cursor_next(k, w, p.num_splits)) {
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
 #pragma unroll
-        for (int q = 0; q < NT; ++q) tree_store_A_n<D>(o[q], red, slot + 8 * q * D, min(8, R - 8 * q), sl, lane, 2);
+        for (int q = 0; q < NT; ++q) tree_store_A_n<D>(o[q], red, slot + (rbase + 8 * q) * D, min(8, R - rbase - 8 * q), sl, lane, 2);
       }
     }
     if (lane == 0 && dead) atomicOr(&p.hdr->wait_timeouts, 4u);
