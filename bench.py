@@ -426,11 +426,12 @@ def main():
     D = w.head_dim
     slot_bytes = sum(F.fold_workspace_bytes(x) - 256 for x in make(T, F.Z_GIVEN))
 
-    def actual_bytes(r):                                  # K in full + fetched V rows + slots written, all levels
-        return sum(r["total"]) * 2 * D + sum(r["fetched"]) * 2 * D + slot_bytes
-
     def fetched_frac(r):
         return sum(r["fetched"]) / max(sum(r["total"]), 1)
+
+    def actual_bytes(r):                                  # K in full + the fetched share of V + slots written, all levels
+        # (from the fetched FRACTION: row groups of one kv head count their keys once each, but share the tiles in L2)
+        return cache_bytes // 2 + int(cache_bytes // 2 * fetched_frac(r)) + slot_bytes
 
     peak, peak_src = load_peaks()
     value = world * cache_bytes / (r16["ms_per_step"] * 1e-3) / 1e9
