@@ -68,6 +68,23 @@ def test_config3_with_the_block_tail_sampled_rows():
     torch.cuda.empty_cache()
 
 
+def test_config5_cell_mha_head_dim_64_sampled_rows():
+    # one cell of the sweep at full size: MHA, 32 heads, D = 64 (128-key tiles), batch 8, 32768 keys, T in {8, 16, inf}
+    if _free_gb() < 12:
+        pytest.skip("not enough free device memory")
+    w = make_decode_workload(8, 32, 32, 64, 32768, seed=5000 + 64 * 7 + 8 * 131 + 32768, device=DEV)
+    rows = [(0, 0), (3, 17), (7, 31)]
+    for T in (8.0, 16.0, math.inf):
+        b = run_gpu(w, T=T)
+        compare(w, b, T=T, rows=rows, check_estimate=True)
+        if T == 8.0:
+            h = b.header()
+            assert h.v_rows_fetched < 0.05 * h.v_rows_total          # nearly every value row is cut and not read
+            assert same_bits(run_gpu(w, T=T, num_splits=4).out, b.out.clone())
+    del w
+    torch.cuda.empty_cache()
+
+
 def test_config4_shared_prefix_cascade_sampled_rows():
     if _free_gb() < 8:
         pytest.skip("not enough free device memory")
