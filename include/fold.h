@@ -141,7 +141,7 @@ typedef struct fold_ws_header {
   uint32_t reserved;
   uint64_t v_rows_fetched;     /* value rows actually requested from memory, all (seq, kv head) */
   uint64_t v_rows_total;       /* value rows a dense decode would read (= keys scanned) */
-  uint64_t v_slices_skipped;   /* 16-key slices of a tile whose value work was skipped entirely */
+  uint64_t v_slices_skipped;   /* warp slices (16 keys at head_dim 128, 32 at 64) whose value work was skipped entirely */
   uint64_t pad[4];
 } fold_ws_header;
 
