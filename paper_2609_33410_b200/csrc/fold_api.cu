@@ -587,7 +587,7 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
   while (warps < kMergeMaxWarps && warps * 8 < total_slots) warps <<= 1;
   const bool resident = n_levels == 1 && (total_slots + warps - 1) / warps <= kMergeResident;
   if (!resident)
-    while (warps > 1 && n_rows * warps > 2048) warps >>= 1;
+    while (warps > 1 && n_rows * warps > 4096) warps >>= 1;
 #ifdef FOLD_TUNING
   if (const char *e = getenv("FOLD_TUNE_MERGEW")) warps = atoi(e);
 #endif
