@@ -415,14 +415,16 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   const int R = p.R, n = w.n;
   const int dstart = draft_start(p, n);
 
-  // barriers (8 bytes each): kv_full[stages]  pv_done[stages]  s_full[2]  p_full[2]  o_empty[2]
-  // pv_done[stage]: both groups' value products of the tile in `stage` have completed (frees the stage; at a
-  // chunk's end, O is final).
+  // barriers (8 bytes each): kv_full[stages]  xa[stages]  xb[stages]  s0[2]  p_full[2]  o_empty[2]
+  // One commit per group and tile: x{a,b}[stage] completes when that group's value product of the tile in `stage` AND
+  // its scores of the next tile have (the pipe runs in order), so it tells the group's weight warps both that S of the
+  // next tile is ready and, at a chunk's end, that O is final.  xb (`pv_done` below) is committed after everything
+  // issued for the tile and also frees the stage for the producer.  s0[g] (`s_full`): the very first scores.
   const uint32_t bar = base + LO::kBar;
-  const uint32_t kv_full = bar, pv_done = bar + 8 * kPairStages, s_full = bar + 16 * kPairStages, p_full = s_full + 16,
-                 o_empty = s_full + 32, tmem_slot = bar + 192;
+  const uint32_t kv_full = bar, xa = bar + 8 * kPairStages, pv_done = bar + 16 * kPairStages, s_full = bar + 24 * kPairStages,
+                 p_full = s_full + 16, o_empty = s_full + 32, tmem_slot = bar + 224;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kPairStages; ++s) { mbar_init(kv_full + 8u * s, 1); mbar_init(pv_done + 8u * s, 1); }
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(kv_full + 8u * s, 1); mbar_init(xa + 8u * s, 1); mbar_init(pv_done + 8u * s, 1); }
     for (int g = 0; g < 2; ++g) {
       mbar_init(s_full + 8u * g, 1);
       mbar_init(p_full + 8u * g, 8);                         // one arrival per weight warp of the group
@@ -436,7 +438,7 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   tc_fence_before();
   __syncthreads();                                           // barriers initialised, TMEM allocated
   tc_fence_after();
-  const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(gen + LO::kBar + 192);
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(gen + LO::kBar + 224);
 
   // weight warps 2..17: group g, key/channel half ch, TMEM lane quarter warp % 4
   const int wg = warp - 2;
@@ -484,7 +486,7 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     constexpr uint32_t idesc_qk = umma_idesc(64, 0), idesc_pv = umma_idesc(128, 1);
     const uint32_t ring_lo = umma_desc_lo(base + LO::kRing, 0);
     // S_g = Q_g K^T for the tile in `stage` (K tile [2 halves][64 keys][128 B]: K step kk = 32 bytes along the row)
-    auto issue_qk = [&](int gg, int stage) {
+    auto issue_qk = [&](int gg, int stage, bool first) {
       const uint32_t k_lo = ring_lo + ((uint32_t)(stage * LO::kStage) >> 4) + (1u << 16);
       if (leader) {
         umma_bf16_ta<false>(tm + gg * 64, tm + 384 + gg * 64, k_lo, umma_desc_hi(1024), idesc_qk);
@@ -492,7 +494,7 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         for (int kk = 1; kk < D / 16; ++kk)
           umma_bf16_ta<true>(tm + gg * 64, tm + 384 + gg * 64 + kk * 8,
                              k_lo + (((kk >> 2) * (kTileKeys * 128) + (kk & 3) * 32) >> 4), umma_desc_hi(1024), idesc_qk);
-        tc_commit(s_full + 8u * gg);
+        if (first) tc_commit(s_full + 8u * gg);               // later scores are announced by the group's x barrier
       }
       __syncwarp();
     };
@@ -514,8 +516,8 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     TileCursor k = cursor_begin(w, split);
     if (cursor_valid(k, w) && mbar_wait(kv_full, 0u, dead)) {
       tc_fence_after();
-      issue_qk(0, 0);
-      issue_qk(1, 0);
+      issue_qk(0, 0, true);
+      issue_qk(1, 0, true);
     }
     bool first_of_chunk = true;
     while (cursor_valid(k, w) && !dead) {
@@ -530,11 +532,9 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         if (!mbar_wait(p_full + 8u * gg, (uint32_t)(it & 1), dead)) break;
         tc_fence_after();
         issue_pv(gg, stage, !first_of_chunk);
-        if (gg == 1) {
-          if (leader) tc_commit(pv_done + 8u * stage);
-          __syncwarp();
-        }
-        if (more) issue_qk(gg, nstage);
+        if (more) issue_qk(gg, nstage, false);
+        if (leader) tc_commit((gg == 0 ? xa : pv_done) + 8u * stage);
+        __syncwarp();
       }
       if (chunk_ends) ++chunk_i;
       first_of_chunk = chunk_ends;
@@ -551,7 +551,10 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
       const int stage = it % kPairStages;
       const int key_base = k.t * kTileKeys;
       // the tcgen05 loads and stores below are warp-wide: the warp takes them together or not at all
-      if (__all_sync(0xffffffffu, mbar_wait(s_full + 8u * g, (uint32_t)(it & 1), dead))) {
+      const uint32_t xg = g == 0 ? xa : pv_done;             // this group's per-stage barrier
+      const bool have_s = it == 0 ? mbar_wait(s_full + 8u * g, 0u, dead)
+                                  : mbar_wait(xg + 8u * ((it - 1) % kPairStages), (uint32_t)(((it - 1) / kPairStages) & 1), dead);
+      if (__all_sync(0xffffffffu, have_s)) {
         tc_fence_after();
         float s[32];
         uint32_t ph[16], pl[16];                             // this thread's 32 weights, BF16 pairs: hi and lo terms
@@ -608,7 +611,7 @@ fold_scan_stacked_pair_kernel(const __grid_constant__ CUtensorMap tmK, const __g
         float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c_done) * p.slot_stride;
         float *lbuf = reinterpret_cast<float *>(gen + LO::kLbuf) + g * kUmmaRows;
         if (ch == 1) lbuf[row] = l_row;
-        if (__all_sync(0xffffffffu, mbar_wait(pv_done + 8u * stage, (uint32_t)((it / kPairStages) & 1), dead))) {
+        if (__all_sync(0xffffffffu, mbar_wait(xg + 8u * stage, (uint32_t)((it / kPairStages) & 1), dead))) {
           tc_fence_after();
 #pragma unroll 1
           for (int q4 = ch * 2; q4 < ch * 2 + 2; ++q4) {
