@@ -133,6 +133,49 @@ def oracle_sample(w, T, units, z=None):
     return time.perf_counter() - t0, nbytes, threads
 
 
+def accuracy_sample(w, run, T, n_units=16, seed=4242):
+    """Errors of the CUDA path on a seeded sample of (sequence, kv head) units (every query row of each), against
+    the float64 oracle: the declared-reference result at the GPU's own Z and T, float64 softmax attention, and the
+    emulated BF16 online-softmax yardstick beside them.  `run(depth)` runs one decode step and returns
+    (out, z) as float64 numpy arrays.  Part of the CPU-baseline leg: the only place the bench touches the oracle."""
+    import numpy as np
+    from oracle import fold_oracle as O
+    from paper_2609_33410_b200.workloads import bf16_bits
+    rng = np.random.default_rng(seed)
+    G = w.num_q_heads // w.num_kv_heads
+    units = [(s, h) for s in range(w.num_seqs) for h in range(w.num_kv_heads)]
+    pick = [units[i] for i in rng.choice(len(units), size=min(n_units, len(units)), replace=False)]
+    out_t, z_t = run(T)
+    out_d, _ = run(math.inf)
+    acc = dict(t_ref=0.0, t_dense=0.0, d_dense=0.0, yard=0.0, ref=0.0, dense=0.0)
+    cut_mass, live, rows = [], [], 0
+    for (seq, kvh) in pick:
+        K = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh)))
+        V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
+        if K.shape[0] == 0:
+            continue
+        for r in range(w.stack * G):
+            b, h = seq * w.stack + r // G, kvh * G + r % G
+            q = O.widen_bf16(bf16_bits(w.q[b, h]))
+            s = O.scores(q, K, w.scale)
+            o_ref = O.fold_row(s, V, z_t[b, h], T)[0]
+            o_dense = O.dense_row(s, V)[0]
+            y = O.online_softmax_bf16(q, K, V, w.scale)
+            rep = O.cut_report(s, V, z_t[b, h], T)
+            for key, d in (("t_ref", out_t[b, h] - o_ref), ("t_dense", out_t[b, h] - o_dense),
+                           ("d_dense", out_d[b, h] - o_dense), ("yard", y - o_dense)):
+                acc[key] += float(d @ d)
+            acc["ref"] += float(o_ref @ o_ref); acc["dense"] += float(o_dense @ o_dense)
+            cut_mass.append(rep["cut_mass"]); live.append(rep["live_frac"]); rows += 1
+    rel = lambda num, den: math.sqrt(acc[num] / max(acc[den], 1e-300))
+    return {"rows": rows, "sample": f"{len(pick)} seeded (sequence, kv head) units, all their query rows",
+            "rel_l2_T_vs_oracle_same_Z_T": rel("t_ref", "ref"), "rel_l2_T_vs_float64_softmax": rel("t_dense", "dense"),
+            "rel_l2_Tinf_vs_float64_softmax": rel("d_dense", "dense"),
+            "rel_l2_bf16_online_softmax_vs_float64_softmax": rel("yard", "dense"),
+            "cut_mass_mean": float(np.mean(cut_mass)) if rows else 0.0,
+            "live_key_frac_mean": float(np.mean(live)) if rows else 0.0, "depth_T": T}
+
+
 def bounded_oracle(w, T, budget_s=12.0):
     """Run the oracle unit by unit (cycling over the sample's units) until about budget_s seconds of
     oracle time have been spent."""
@@ -506,6 +549,12 @@ def main():
                                "kind": "oracle",
                                "sample": f"{ob['units']} (sequence, kv head) units of {args.workload} "
                                          f"({ob['seconds']:.1f} s of float64 numpy; estimate + declared-Z row per q head)"}
+        if args.drafts <= 1 and not args.tail:
+            def run_once(depth):
+                step_whole(make(depth, F.Z_ESTIMATE))
+                torch.cuda.synchronize()
+                return bufs.out.float().cpu().numpy().astype("float64"), bufs.z.cpu().numpy().astype("float64")
+            out["accuracy"] = accuracy_sample(w, run_once, T)
 
     if rank == 0:
         print(json.dumps(out))
