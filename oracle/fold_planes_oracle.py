@@ -1,0 +1,170 @@
+"""CPU oracle for the two-plane INT8 key cache of fold decode.
+
+TEST INFRASTRUCTURE ONLY, like ``fold_oracle``: the slow, plain statement of what the
+two-plane path computes.  It shares no code with the CUDA library; only the tests, the smoke
+check and the benchmark's CPU-baseline leg call it.
+
+What is here, with the passage each function restates (Section 4, "Cache format" and
+"Weight-gated reads"; Algorithm 1):
+  hadamard            the orthonormal (Sylvester) Hadamard matrix, float64: the definition the
+                      fast transform below is pinned against
+  rotate_f32          the same rotation as the cache writer performs it: FP32 butterflies in a
+                      fixed order, then one multiply by fp32(1/sqrt(D))
+  split_planes        k = e (a + b/256): BF16 scale rounded up so plane A never saturates, two
+                      INT8 planes.  The codes are integers decided by FP32 arithmetic, so this
+                      function works in FP32, operation by operation, as the writer does
+  quantize_rows       rotate_f32 + split_planes for an array of rows (keys at cache write, the
+                      query rows at every step: "the query is split the same way")
+  dequantize          e (a + b/256) in float64
+  plane_products      the four integer products c^aa, c^ab, c^ba, c^bb (exact)
+  coarse_scores /
+  refined_scores      Algorithm 1: eta e (c^aa + c^ab/256) and the plane-B correction, float64
+  auto_refine_tau     the refine gate when the caller gives none (a reading; see its docstring)
+  fold_group_planes   Algorithm 1 for one (sequence, kv head): verdict bits ORed over the
+                      group's rows, final weights, (A, L) per row; also counts the bytes the
+                      gates ask for (130 + 128 r_K + 256 lambda per key at D = 128)
+"""
+from __future__ import annotations
+
+import math
+from typing import Optional
+
+import numpy as np
+
+from . import fold_oracle as O
+
+F32 = np.float32
+
+
+# --------------------------------------------------------------------------- rotation
+def hadamard(D: int) -> np.ndarray:
+    """Orthonormal Sylvester-Hadamard matrix H_D (D a power of two), float64: H H^T = I."""
+    assert D >= 1 and D & (D - 1) == 0
+    H = np.ones((1, 1))
+    while H.shape[0] < D:
+        H = np.block([[H, H], [H, -H]])
+    return H / math.sqrt(D)
+
+
+def rotate_f32(x: np.ndarray) -> np.ndarray:
+    """Rows of x [.., D] (values exactly representable in FP32) times H_D, computed as the cache
+    writer computes it: log2(D) butterfly stages with strides 1, 2, 4, ..., each an FP32 add and
+    an FP32 subtract ((lo, hi) -> (lo + hi, lo - hi)), then one FP32 multiply by fp32(1/sqrt(D))."""
+    y = np.array(x, dtype=F32)
+    D = y.shape[-1]
+    assert D & (D - 1) == 0
+    h = 1
+    while h < D:
+        y = y.reshape(y.shape[:-1] + (D // (2 * h), 2, h))
+        lo, hi = y[..., 0, :], y[..., 1, :]
+        y = np.stack([(lo + hi).astype(F32), (lo - hi).astype(F32)], axis=-2).reshape(y.shape[:-3] + (D,))
+        h *= 2
+    return (y * F32(1.0 / math.sqrt(D))).astype(F32)
+
+
+# --------------------------------------------------------------------------- planes
+def bf16_round_up(x: np.ndarray) -> np.ndarray:
+    """Smallest BF16 value >= x, for x >= 0 finite FP32; returned as FP32."""
+    u = np.asarray(x, dtype=F32).view(np.uint32)
+    up = np.where((u & np.uint32(0xFFFF)) != 0, (u >> np.uint32(16)) + np.uint32(1), u >> np.uint32(16))
+    return (up.astype(np.uint32) << np.uint32(16)).view(F32)
+
+
+def split_planes(y: np.ndarray):
+    """y [.., D] FP32 -> (a int8, b int8, e FP32 holding a BF16 value) with y ~ e (a + b/256).
+    Section 4 "Cache format": a scale per row, rounded UP so plane A never saturates; a row's code
+    depends on that row alone.  Every step is one FP32 operation (the reading of how the codes are
+    decided):  e = bf16_up(max|y| / 127)  (1 when the row is all zero);  t = y / e;
+    a = rint(t) kept within +-127;  b = rint((t - a) * 256) kept within [-128, 127]."""
+    y = np.asarray(y, dtype=F32)
+    m = np.abs(y).max(axis=-1)
+    e = np.where(m > 0, bf16_round_up((m / F32(127.0)).astype(F32)), F32(1.0)).astype(F32)
+    t = (y / e[..., None]).astype(F32)
+    a = np.clip(np.rint(t), -127, 127).astype(F32)
+    r = (t - a).astype(F32)                                   # exact: t minus its nearest integer
+    b = np.clip(np.rint((r * F32(256.0)).astype(F32)), -128, 127)
+    return a.astype(np.int8), b.astype(np.int8), e
+
+
+def quantize_rows(x: np.ndarray):
+    """Rotate and split rows x [.., D] (FP32-representable values): returns (a, b, e)."""
+    return split_planes(rotate_f32(x))
+
+
+def dequantize(a, b, e) -> np.ndarray:
+    return np.asarray(e, dtype=np.float64)[..., None] * (np.asarray(a, dtype=np.float64) + np.asarray(b, dtype=np.float64) / 256.0)
+
+
+# --------------------------------------------------------------------------- scores
+def plane_products(ka, kb, qa, qb):
+    """The four integer products of Algorithm 1 for one query row: keys [n, D] int8, query [D] int8.
+    Returns (c_aa, c_ab, c_ba, c_bb), int64 [n] each, exact."""
+    ka = np.asarray(ka, dtype=np.int64); kb = np.asarray(kb, dtype=np.int64)
+    qa = np.asarray(qa, dtype=np.int64); qb = np.asarray(qb, dtype=np.int64)
+    return ka @ qa, ka @ qb, kb @ qa, kb @ qb
+
+
+def coarse_scores(ka, ke, qa, qb, eta: float) -> np.ndarray:
+    """Algorithm 1, coarse score (before the reference is subtracted): eta e_j (c^aa_j + c^ab_j / 256).
+    `eta` is the query row's scale times log2(e) times the softmax scale, so the result is in binades."""
+    ka = np.asarray(ka, dtype=np.int64)
+    c_aa = ka @ np.asarray(qa, dtype=np.int64)
+    c_ab = ka @ np.asarray(qb, dtype=np.int64)
+    return float(eta) * np.asarray(ke, dtype=np.float64) * (c_aa + c_ab / 256.0)
+
+
+def refine_terms(kb, ke, qa, qb, eta: float) -> np.ndarray:
+    """Algorithm 1, the plane-B correction: eta e_j (c^ba_j + c^bb_j / 256) / 256."""
+    kb = np.asarray(kb, dtype=np.int64)
+    c_ba = kb @ np.asarray(qa, dtype=np.int64)
+    c_bb = kb @ np.asarray(qb, dtype=np.int64)
+    return float(eta) * np.asarray(ke, dtype=np.float64) * (c_ba + c_bb / 256.0) / 256.0
+
+
+def refined_scores(ka, kb, ke, qa, qb, eta: float) -> np.ndarray:
+    return coarse_scores(ka, ke, qa, qb, eta) + refine_terms(kb, ke, qa, qb, eta)
+
+
+def auto_refine_tau(n: int) -> float:
+    """The refine gate tau_K used when the caller gives none.  The paper says only that the refine
+    thresholds follow each request's own length and are set where the second plane starts to matter at
+    the error target.  Reading: a key whose coarse weight is below 2^-tau moves the output by at most
+    its weight times the coarse score error (a fraction of a binade), and n such keys by n times that,
+    so  tau_K = log2(n) + 7  holds the unrefined keys' total to about 2^-8 of the row's mass."""
+    return math.log2(max(n, 1)) + 7.0
+
+
+def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None):
+    """Algorithm 1 for the rows of one (sequence, kv head) group over all its keys.
+    ka, kb [n, D] int8; ke [n]; V [n, D]; qa, qb [R, D] int8; eta [R]; Z [R] (binades).
+    tau: refine gate in binades (None: auto_refine_tau(n); inf: refine every live key; negative:
+    never).  Per key j:  live_j = OR_i [coarse_ij - Z_i >= -T];  refine_j = live_j AND
+    OR_i [coarse_ij - Z_i >= -tau];  s_ij = coarse_ij (+ correction_ij if refine_j);  the weight
+    2^(s_ij - Z_i) always adds to L_i and adds weight x value to A_i iff live_j and s_ij - Z_i >= -T.
+    Returns (A [R, D], L [R], info) with info = live / refine masks and the bytes-per-key count."""
+    ka = np.asarray(ka); kb = np.asarray(kb)
+    V = np.asarray(V, dtype=np.float64)
+    n, D = ka.shape
+    R = len(eta)
+    if tau is None:
+        tau = auto_refine_tau(n)
+    coarse = np.stack([coarse_scores(ka, ke, qa[i], qb[i], eta[i]) - Z[i] for i in range(R)])      # [R, n]
+    live = np.ones(n, dtype=bool) if math.isinf(T) else (coarse >= -T).any(axis=0)
+    refine = live & ((coarse >= -tau).any(axis=0) if tau >= 0 else np.zeros(n, dtype=bool))
+    A = np.zeros((R, D)); L = np.zeros(R)
+    for i in range(R):
+        s = coarse[i] + np.where(refine, refine_terms(kb, ke, qa[i], qb[i], eta[i]), 0.0)
+        p = np.exp2(s)
+        keep = live if math.isinf(T) else (live & (s >= -T))
+        L[i] = p.sum()
+        A[i] = (p[keep, None] * V[keep]).sum(axis=0)
+    info = dict(live=live, refine=refine, coarse=coarse,
+                bytes_per_key=(D + 2) + D * float(refine.mean() if n else 0.0) + 2 * D * float(live.mean() if n else 0.0))
+    return A, L, info
+
+
+def estimate_z_planes(ka, kb, ke, qa, qb, eta: float) -> float:
+    """The 192-key reference estimate (``fold_oracle.estimate_z``) on two-plane scores: the sampled keys
+    are scored with both planes."""
+    n = ka.shape[0]
+    return O.estimate_z(lambda idx: refined_scores(ka[idx], kb[idx], np.asarray(ke)[idx], qa, qb, eta), n)

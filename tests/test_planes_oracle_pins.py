@@ -1,0 +1,224 @@
+"""Pins of the two-plane INT8 key oracle (Section 4 "Cache format", "Weight-gated reads"; Algorithm 1)
+to things other than itself: the matrix definition of the rotation, hand-worked codes, closed-form
+bounds, special cases that reduce to the plain declared-reference functions, and a per-key
+brute-force restatement of Algorithm 1."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import fold_oracle as O
+from oracle import fold_planes_oracle as P
+
+
+def rng_rows(seed, n, D, spread=1.0):
+    r = np.random.default_rng(seed)
+    x = r.standard_normal((n, D)) * spread
+    x[:, 3] *= 9.0                                          # an outlier channel, as real keys have
+    return O.round_to_bf16(x)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_rotation_is_the_orthonormal_hadamard_matrix(D):
+    H = P.hadamard(D)
+    assert np.allclose(H @ H.T, np.eye(D), atol=1e-14)
+    assert np.allclose(np.abs(H), 1 / math.sqrt(D))
+    x = rng_rows(1, 17, D)
+    y = P.rotate_f32(x).astype(np.float64)
+    assert np.abs(y - x @ H).max() <= 2e-6 * np.abs(x).max() * math.sqrt(D)      # fp32 butterflies vs the definition
+    # a unit vector picks out one row of H: pins the butterfly indexing element by element
+    for j in (0, 1, 5, D - 1):
+        e = np.zeros((1, D)); e[0, j] = 1.0
+        assert np.array_equal(P.rotate_f32(e)[0].astype(np.float64), np.float32(1 / math.sqrt(D)).astype(np.float64) * np.sign(H[j]))
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_rotation_keeps_every_inner_product(D):
+    k = rng_rows(2, 50, D); q = rng_rows(3, 4, D)
+    exact = q @ k.T
+    rot = P.rotate_f32(q).astype(np.float64) @ P.rotate_f32(k).astype(np.float64).T
+    assert np.abs(rot - exact).max() <= 1e-5 * np.abs(exact).max()
+
+
+def test_bf16_round_up_values():
+    x = np.array([1.0, 1.0 + 2.0 ** -10, 0.3, 3.0e-5, 127.0], dtype=np.float32)
+    up = P.bf16_round_up(x)
+    assert up[0] == 1.0 and up[1] == 1.0078125 and up[4] == 127.0
+    assert np.all(up >= x)
+    assert np.all((up.view(np.uint32) & 0xFFFF) == 0)                            # BF16 values
+    below = ((up.view(np.uint32) >> 16) - 1).astype(np.uint32) << 16             # the BF16 just below
+    assert np.all((below.view(np.float32) < x) | (up == x))
+
+
+def test_split_planes_hand_worked_row():
+    # max = 127 -> e = 1; t = y.  rint(-63.5) = -64 (ties to even), remainder +0.5 -> 128 -> kept at 127;
+    # 0.25 -> a = 0, b = 64;  100.75 -> a = 101, b = -64
+    y = np.array([[127.0, -63.5, 0.25, 0.0, 100.75, -0.001953125]], dtype=np.float32)
+    a, b, e = P.split_planes(y)
+    assert e[0] == 1.0
+    assert a[0].tolist() == [127, -64, 0, 0, 101, 0]
+    assert b[0].tolist() == [0, 127, 64, 0, -64, 0]            # -0.001953125 * 256 = -0.5 -> rint -> -0 (ties to even)
+    # a scale that is not a power of two: max = 100 -> 100/127 = 0.78740156 -> BF16 up = 0.7890625
+    a, b, e = P.split_planes(np.array([[100.0, 50.0]], dtype=np.float32))
+    assert e[0] == 0.7890625
+    assert a[0].tolist() == [127, 63] and b[0].tolist() == [-68, 94]   # 100/e = 126.7327 (-0.2673 * 256 = -68.4), 50/e = 63.3663 (0.3663 * 256 = 93.8)
+    # an all-zero row
+    a, b, e = P.split_planes(np.zeros((1, 8), dtype=np.float32))
+    assert e[0] == 1.0 and not a.any() and not b.any()
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_codes_never_saturate_and_reconstruct_within_half_a_step(D):
+    x = rng_rows(4, 400, D, spread=3.0)
+    y = P.rotate_f32(x)
+    a, b, e = P.split_planes(y)
+    t = y.astype(np.float64) / e[:, None].astype(np.float64)
+    assert np.abs(np.rint(t)).max() <= 127                                      # the clip on plane A never acts
+    assert np.abs(a.astype(int)).max() <= 127 and b.min() >= -128 and b.max() <= 127
+    assert np.all(e.astype(np.float64) >= np.abs(y).max(axis=1) / 127.0 * (1 - 2.0 ** -23))   # scale rounded up
+    assert np.all(e.astype(np.float64) <= np.abs(y).max(axis=1) / 127.0 * (1 + 2.0 ** -7))    # by less than a BF16 step
+    err = np.abs(P.dequantize(a, b, e) - y.astype(np.float64))
+    # half a plane-B step (e/512), one whole step where +128 was kept at 127, plus the fp32 division's rounding
+    assert np.all(err <= e[:, None].astype(np.float64) * (1.0 / 256 + 1e-5))
+    assert np.mean(err <= e[:, None].astype(np.float64) * (1.0 / 512 + 1e-5)) > 0.99
+    # plane A alone is within half a coarse step
+    assert np.all(np.abs(P.dequantize(a, 0 * b, e) - y.astype(np.float64)) <= e[:, None] * (0.5 + 1e-5))
+
+
+def test_scores_are_the_product_of_the_dequantized_codes():
+    D = 128
+    ka, kb, ke = P.quantize_rows(rng_rows(5, 60, D))
+    qa, qb, qe = P.quantize_rows(rng_rows(6, 1, D))
+    eta = float(qe[0]) * 0.1275
+    kd = P.dequantize(ka, kb, ke); qd = P.dequantize(qa, qb, qe)[0]
+    assert np.allclose(P.refined_scores(ka, kb, ke, qa[0], qb[0], eta), 0.1275 * kd @ qd, rtol=1e-12, atol=1e-12)
+    # coarse = plane A of the key against BOTH planes of the query
+    ka_only = P.dequantize(ka, 0 * kb, ke)
+    assert np.allclose(P.coarse_scores(ka, ke, qa[0], qb[0], eta), 0.1275 * ka_only @ qd, rtol=1e-12, atol=1e-12)
+    c = P.plane_products(ka, kb, qa[0], qb[0])
+    assert all(v.dtype == np.int64 for v in c)
+    j = 7
+    assert c[1][j] == sum(int(ka[j, d]) * int(qb[0, d]) for d in range(D))      # c^ab: key plane A, query plane B
+    assert c[2][j] == sum(int(kb[j, d]) * int(qa[0, d]) for d in range(D))      # c^ba: key plane B, query plane A
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_two_plane_scores_sit_within_the_quantisation_bound_of_the_exact_scores(D):
+    k = rng_rows(7, 300, D); q = rng_rows(8, 3, D)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    c = O.LOG2E / math.sqrt(D)
+    for i in range(3):
+        exact = O.scores(q[i], k)
+        two = P.refined_scores(ka, kb, ke, qa[i], qb[i], float(qe[i]) * c)
+        one = P.coarse_scores(ka, ke, qa[i], qb[i], float(qe[i]) * c)
+        kn = np.linalg.norm(k, axis=1); qn = np.linalg.norm(q[i])
+        # Cauchy-Schwarz with per-channel code errors e/256 (both planes) and e/2 (plane A only)
+        b2 = c * (ke * math.sqrt(D) / 256 * qn + float(qe[i]) * math.sqrt(D) / 256 * kn) * 1.01 + 1e-4
+        b1 = c * (ke * math.sqrt(D) / 2 * qn) * 1.01 + b2
+        assert np.all(np.abs(two - exact) <= b2)
+        assert np.all(np.abs(one - exact) <= b1)
+        assert np.abs(two - exact).max() < 0.02 and np.abs(one - exact).max() > np.abs(two - exact).max()
+
+
+def brute_force_algorithm_1(ka, kb, ke, V, qa, qb, eta, Z, T, tau):
+    """Algorithm 1, key by key, in plain Python."""
+    n, D = ka.shape
+    R = len(eta)
+    A = [[0.0] * D for _ in range(R)]; L = [0.0] * R
+    n_live = n_ref = 0
+    for j in range(n):
+        co = []
+        for i in range(R):
+            caa = sum(int(ka[j, d]) * int(qa[i][d]) for d in range(D))
+            cab = sum(int(ka[j, d]) * int(qb[i][d]) for d in range(D))
+            co.append(float(eta[i]) * float(ke[j]) * (caa + cab / 256.0) - Z[i])
+        live = any(x >= -T for x in co)
+        refine = live and tau >= 0 and any(x >= -tau for x in co)
+        n_live += live; n_ref += refine
+        for i in range(R):
+            s = co[i]
+            if refine:
+                cba = sum(int(kb[j, d]) * int(qa[i][d]) for d in range(D))
+                cbb = sum(int(kb[j, d]) * int(qb[i][d]) for d in range(D))
+                s += float(eta[i]) * float(ke[j]) * (cba + cbb / 256.0) / 256.0
+            p = 2.0 ** s
+            L[i] += p
+            if live and s >= -T:
+                for d in range(D):
+                    A[i][d] += p * V[j, d]
+    return np.array(A), np.array(L), n_live, n_ref
+
+
+@pytest.mark.parametrize("T,tau", [(math.inf, math.inf), (math.inf, 3.0), (6.0, 2.0), (4.0, -1.0), (5.0, math.inf)])
+def test_group_fold_matches_a_key_by_key_restatement_of_algorithm_1(T, tau):
+    D, n, R = 64, 90, 3
+    k = rng_rows(9, n, D); q = rng_rows(10, R, D); V = rng_rows(11, n, D)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    Z = np.array([P.coarse_scores(ka, ke, qa[i], qb[i], eta[i]).max() for i in range(R)]) + np.array([0.0, -0.5, 0.25])
+    A, L, info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T, tau)
+    A2, L2, n_live, n_ref = brute_force_algorithm_1(ka, kb, ke, V, qa, qb, eta, Z, T, tau)
+    assert np.allclose(A, A2, rtol=1e-12, atol=1e-300) and np.allclose(L, L2, rtol=1e-12)
+    assert info["live"].sum() == n_live and info["refine"].sum() == n_ref
+    if not math.isinf(T):
+        assert 0 < n_live < n                                 # the case exercises the gate
+    if 0 <= tau < 10:
+        assert 0 < n_ref < n_live
+
+
+def test_special_cases_reduce_to_the_plain_declared_reference_functions():
+    D, n, R = 128, 500, 4
+    k = rng_rows(12, n, D); q = rng_rows(13, R, D); V = rng_rows(14, n, D)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    Z = np.zeros(R)
+    # dense, every key refined: plain softmax attention on the two-plane scores
+    A, L, info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, math.inf, math.inf)
+    for i in range(R):
+        s = P.refined_scores(ka, kb, ke, qa[i], qb[i], eta[i])
+        o, lse = O.dense_row(s, V)
+        assert np.allclose(A[i] / L[i], o, rtol=1e-12) and abs(math.log2(L[i]) - lse) < 1e-12
+    assert info["bytes_per_key"] == 514.0                      # 130 + 128 + 256: both planes, the scale, a BF16 value row
+    # never refined, finite depth, ONE row: the plain depth-T fold on the coarse scores
+    for i in range(R):
+        s = P.coarse_scores(ka, ke, qa[i], qb[i], eta[i])
+        Zi = O.dense_row(s, V)[1]
+        A1, L1, info1 = P.fold_group_planes(ka, kb, ke, V, qa[i:i + 1], qb[i:i + 1], eta[i:i + 1], [Zi], 8.0, -1.0)
+        o, lse, A0, L0 = O.fold_row(s, V, Zi, 8.0)
+        assert np.allclose(A1[0], A0, rtol=1e-12) and np.isclose(L1[0], L0, rtol=1e-12)
+        assert info1["bytes_per_key"] == 130.0 + 256.0 * info1["live"].mean()
+    # without refinement L does not depend on the depth
+    La = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, 3.0, -1.0)[1]
+    Lb = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, math.inf, -1.0)[1]
+    assert np.array_equal(La, Lb)
+
+
+def test_verdicts_are_ored_over_the_group_but_weights_are_cut_per_row():
+    D = 64
+    k = rng_rows(15, 200, D); V = np.ones((200, D)); q = rng_rows(16, 2, D)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    Z = np.array([P.coarse_scores(ka, ke, qa[i], qb[i], eta[i]).max() for i in range(2)])
+    T = 3.0
+    A, L, info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T, -1.0)
+    own = [(info["coarse"][i] >= -T) for i in range(2)]
+    assert np.array_equal(info["live"], own[0] | own[1])
+    assert (own[0] & ~own[1]).any()                            # keys fetched for row 0 alone ...
+    for i in range(2):                                         # ... add nothing to row 1's A (V = 1: A counts kept mass)
+        assert np.isclose(A[i][0], np.exp2(info["coarse"][i][own[i]]).sum(), rtol=1e-12)
+
+
+def test_auto_refine_gate_follows_the_request_length_only():
+    assert P.auto_refine_tau(1024) == 17.0 and P.auto_refine_tau(32768) == 22.0
+    assert P.auto_refine_tau(2048) - P.auto_refine_tau(1024) == 1.0
+
+
+def test_estimate_on_planes_is_the_plain_estimate_of_the_two_plane_scores():
+    D, n = 128, 1000
+    k = rng_rows(17, n, D); q = rng_rows(18, 1, D)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = float(qe[0]) * O.LOG2E / math.sqrt(D)
+    s = P.refined_scores(ka, kb, ke, qa[0], qb[0], eta)
+    assert P.estimate_z_planes(ka, kb, ke, qa[0], qb[0], eta) == O.estimate_z(lambda i: s[i], n)
+    short = P.estimate_z_planes(ka[:100], kb[:100], ke[:100], qa[0], qb[0], eta)
+    assert abs(short - O.dense_row(s[:100], np.zeros((100, 1)))[1]) < 1e-12
