@@ -84,7 +84,22 @@ enum {
  * tile's virtual row").  fold_block_means() fills the table from the cache; keeping it current when
  * tokens are appended is the caller's business (only the last block changes).  Every row-block and
  * stacked-row shape takes it (a stacked level with a table runs on the mma.sync kernel, not on tcgen05).
- * Ignored at depth_T = INFINITY (nothing is cut). */
+ * Ignored at depth_T = INFINITY (nothing is cut).
+ *
+ * Two-plane INT8 keys (Section 4, "Cache format"; Algorithm 1).  When k_plane_a is not NULL the decode
+ * reads keys from two INT8 planes and a BF16 scale per (token, kv head) instead of from k:
+ *     H k_j ~ e_j (a_j + b_j / 256),   H the orthonormal Hadamard matrix of order head_dim,
+ * written by fold_quantize_keys() (below, which states the arithmetic).  Plane rows are head_dim bytes,
+ * contiguous, 16-byte aligned: row (seq-or-page, tok, head) of plane X at
+ *     k_plane_X + seq*plane_stride_seq + tok*plane_stride_tok + head*plane_stride_head   (bytes; multiples of 16),
+ * both planes with the same strides, paged exactly as k is (same page_table).  The scales lie token-fastest,
+ *     k_scale + seq*scale_stride_seq + head*scale_stride_head + tok                       (BF16 elements; multiples of 8),
+ * and every (sequence-or-page, head) scale row must be readable up to the next multiple of 8 tokens past
+ * capacity (page_size).  With planes, k may be NULL for the decode calls; v stays BF16.  Each scan scores every
+ * key against plane A alone (head_dim + 2 bytes per key), ORs the verdicts over the rows that share the kv head,
+ * and only then requests plane B rows (refined keys) and value rows (live keys).  This path takes row blocks of
+ * at most 8 rows (stack * group <= 8), no draft masks, no block tail, one level (no cascade), and no
+ * FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED. */
 typedef struct fold_kv {
   const void *k, *v;
   int64_t stride_seq, stride_tok, stride_head;   /* elements */
@@ -98,6 +113,10 @@ typedef struct fold_kv {
   int32_t max_seqlen;                            /* HOST upper bound on seqlens[]; sizes grids and slots */
   const void *v_block_mean;                      /* BF16 block means, or NULL: no block tail */
   int64_t mean_stride_seq, mean_stride_block, mean_stride_head;   /* elements */
+  const int8_t *k_plane_a, *k_plane_b;           /* INT8 key planes, or NULL: BF16 keys from k */
+  int64_t plane_stride_seq, plane_stride_tok, plane_stride_head;  /* bytes */
+  const void *k_scale;                           /* BF16 scale per (token, kv head), token-fastest */
+  int64_t scale_stride_seq, scale_stride_head;   /* elements */
 } fold_kv;
 
 /* One decode call.  `batch` requests with one query token each; request b reads KV
@@ -133,6 +152,10 @@ typedef struct fold_args {
   int32_t *row_status;                 /* [batch, num_q_heads] bit flags, or NULL */
   const uint32_t *draft_mask;          /* [batch] or NULL (draft_len = 0) */
   int32_t draft_len;                   /* 0..32 */
+  float refine_tau;                    /* two-plane keys only: the refine gate tau_K of Algorithm 1, binades.  A live key
+                                          reads plane B iff some row of its group has coarse weight >= 2^-refine_tau.
+                                          0 = choose: log2(n) + 7 for a sequence of n keys (its own length only);
+                                          INFINITY = every live key; negative = none (plane A scores only) */
 } fold_args;
 
 /* First 64 bytes of every workspace, zeroed at the start of each scan. */
@@ -142,7 +165,8 @@ typedef struct fold_ws_header {
   uint64_t v_rows_fetched;     /* value rows actually requested from memory, all (seq, kv head) */
   uint64_t v_rows_total;       /* value rows a dense decode would read (= keys scanned) */
   uint64_t v_slices_skipped;   /* warp slices (16 keys at head_dim 128, 32 at 64) whose value work was skipped entirely */
-  uint64_t pad[4];
+  uint64_t k_rows_refined;     /* two-plane keys: plane B rows requested from memory */
+  uint64_t pad[3];
 } fold_ws_header;
 
 /* The (A, L) partial pairs one scan leaves in its workspace (Algorithm 1, last line).
@@ -170,8 +194,9 @@ typedef struct fold_partials {
 int32_t fold_chunk_keys(int32_t n);
 int32_t fold_num_chunks(int32_t n);
 
-/* Bytes of workspace fold_decode / fold_decode_split need for `args` (header + slots).
- * Depends only on shapes and kv.max_seqlen.  Returns 0 if args is invalid. */
+/* Bytes of workspace fold_decode / fold_decode_split need for `args` (header + slots; with two-plane keys
+ * also the split query rows).  Depends only on shapes, kv.max_seqlen and whether kv.k_plane_a is set.
+ * Returns 0 if args is invalid. */
 size_t fold_workspace_bytes(const fold_args *args);
 
 /* Reference estimate (Section 3): writes levels[0]->z for every (request, q head).
@@ -221,6 +246,21 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
  * num_kv_heads / head_dim as in fold_args.  FOLD_EINVAL for a NULL or misaligned table. */
 int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, fold_stream stream);
 
+/* Cache write for two-plane INT8 keys (Section 4, "Cache format"): for every sequence s, kv head and token
+ * first_token[s] <= j < seqlens[s] (first_token == NULL: from 0; a DEVICE array otherwise -- pass the old lengths
+ * to quantize only appended tokens) read the BF16 key row from kv->k, rotate it and write its two planes and
+ * scale into kv->k_plane_a / k_plane_b / k_scale (DEVICE memory of the caller; written although the struct
+ * says const).  A row's code depends on that row alone.  The arithmetic is FP32, one rounding per step, so the
+ * codes are reproducible bit for bit:
+ *   y = H x:   log2(head_dim) butterfly stages with strides 1, 2, 4, ..., each (lo, hi) -> (lo + hi, lo - hi),
+ *              then one multiply by fp32(1 / sqrt(head_dim));
+ *   e = the smallest BF16 value >= max|y| / 127 (1 if the row is all zero), so plane A never saturates;
+ *   t = y / e;   a = rint(t) within +-127;   b = rint((t - a) * 256) within [-128, 127]   (ties to even).
+ * The decode splits each query row the same way at every step (into its workspace) and carries
+ * eta = e_q * fp32(log2(e) * softmax_scale).  Asynchronous on `stream`. */
+int fold_quantize_keys(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, const int32_t *first_token,
+                       fold_stream stream);
+
 /* The same decode for callers whose tensors live in HOST memory (pinned for the copies to
  * be asynchronous): q, kv.k, kv.v, kv.page_table, kv.seqlens, z (if GIVEN), out, lse and
  * row_status of *host_args are HOST pointers laid out as described above (the cache is
@@ -229,7 +269,7 @@ int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, 
  * the workspace and the results before they are copied back.  Everything is enqueued on
  * `stream`; the host buffers are valid after the caller synchronises the stream.  The block tail is
  * not offered here: kv.v_block_mean must be NULL (FOLD_EUNSUPPORTED otherwise); nor are draft masks
- * (draft_len must be 0). */
+ * (draft_len must be 0) or two-plane keys (kv.k_plane_a must be NULL). */
 size_t fold_host_staging_bytes(const fold_args *host_args);
 int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_bytes, fold_stream stream);
 

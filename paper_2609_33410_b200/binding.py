@@ -30,7 +30,10 @@ class FoldKV(C.Structure):
                 ("num_pages", C.c_int32), ("capacity", C.c_int32), ("num_seqs", C.c_int32),
                 ("seqlens", C.c_void_p), ("max_seqlen", C.c_int32),
                 ("v_block_mean", C.c_void_p), ("mean_stride_seq", C.c_int64), ("mean_stride_block", C.c_int64),
-                ("mean_stride_head", C.c_int64)]
+                ("mean_stride_head", C.c_int64),
+                ("k_plane_a", C.c_void_p), ("k_plane_b", C.c_void_p),
+                ("plane_stride_seq", C.c_int64), ("plane_stride_tok", C.c_int64), ("plane_stride_head", C.c_int64),
+                ("k_scale", C.c_void_p), ("scale_stride_seq", C.c_int64), ("scale_stride_head", C.c_int64)]
 
 
 class FoldArgs(C.Structure):
@@ -42,7 +45,7 @@ class FoldArgs(C.Structure):
                 ("depth_T", C.c_float), ("num_splits", C.c_int32),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("out", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p),
-                ("draft_mask", C.c_void_p), ("draft_len", C.c_int32)]
+                ("draft_mask", C.c_void_p), ("draft_len", C.c_int32), ("refine_tau", C.c_float)]
 
 
 class FoldPartials(C.Structure):
@@ -56,12 +59,13 @@ class FoldPartials(C.Structure):
 class FoldWsHeader(C.Structure):
     _fields_ = [("wait_timeouts", C.c_uint32), ("reserved", C.c_uint32),
                 ("v_rows_fetched", C.c_uint64), ("v_rows_total", C.c_uint64),
-                ("v_slices_skipped", C.c_uint64), ("pad", C.c_uint64 * 4)]
+                ("v_slices_skipped", C.c_uint64), ("k_rows_refined", C.c_uint64), ("pad", C.c_uint64 * 3)]
 
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
            "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
-           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_status_string", "fold_version"]
+           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_quantize_keys", "fold_status_string",
+           "fold_version"]
 
 _lib = None
 
@@ -91,6 +95,8 @@ def lib() -> C.CDLL:
         L.fold_decode_static.restype = C.c_int; L.fold_decode_static.argtypes = [C.POINTER(FoldArgs), C.c_void_p]
         L.fold_block_means.restype = C.c_int
         L.fold_block_means.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p]
+        L.fold_quantize_keys.restype = C.c_int
+        L.fold_quantize_keys.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.fold_status_string.restype = C.c_char_p; L.fold_status_string.argtypes = [C.c_int]
         L.fold_version.restype = C.c_int
         _lib = L
@@ -129,6 +135,10 @@ class KVCache:
     max_seqlen: int
     page_table: Optional[torch.Tensor] = None
     v_block_mean: Optional[torch.Tensor] = None     # [num_seqs, ceil(max_seqlen / 64), Hkv, D] bf16: switches the block tail on
+    # two-plane INT8 keys (alloc_key_planes + fold_quantize_keys): planes shaped like k, scales [seqs-or-pages, Hkv, tokens]
+    k_plane_a: Optional[torch.Tensor] = None
+    k_plane_b: Optional[torch.Tensor] = None
+    k_scale: Optional[torch.Tensor] = None
 
     def to_c(self) -> FoldKV:
         k, v = self.k, self.v
@@ -163,7 +173,26 @@ class KVCache:
             kv.mean_stride_seq, kv.mean_stride_block, kv.mean_stride_head = m.stride(0), m.stride(1), m.stride(2)
         else:
             kv.v_block_mean = None
+        if self.k_plane_a is not None:
+            pa, pb, sc = self.k_plane_a, self.k_plane_b, self.k_scale
+            assert pa.dtype == torch.int8 and pb.dtype == torch.int8 and pa.shape == k.shape and pb.shape == k.shape
+            assert pa.stride() == pb.stride() and pa.stride(3) == 1
+            assert sc.dtype == torch.bfloat16 and sc.dim() == 3 and sc.stride(2) == 1 and sc.shape[:2] == (k.shape[0], k.shape[2])
+            assert sc.shape[2] >= (k.shape[1] + 7) // 8 * 8
+            kv.k_plane_a, kv.k_plane_b, kv.k_scale = pa.data_ptr(), pb.data_ptr(), sc.data_ptr()
+            kv.plane_stride_seq, kv.plane_stride_tok, kv.plane_stride_head = pa.stride(0), pa.stride(1), pa.stride(2)
+            kv.scale_stride_seq, kv.scale_stride_head = sc.stride(0), sc.stride(1)
+        else:
+            kv.k_plane_a = kv.k_plane_b = kv.k_scale = None
         return kv
+
+    def alloc_key_planes(self) -> None:
+        """Allocate the two INT8 key planes and the scales (fold_quantize_keys fills them)."""
+        k = self.k
+        self.k_plane_a = torch.zeros(k.shape, dtype=torch.int8, device=k.device)
+        self.k_plane_b = torch.zeros(k.shape, dtype=torch.int8, device=k.device)
+        toks = (k.shape[1] + 127) // 128 * 128
+        self.k_scale = torch.zeros(k.shape[0], k.shape[2], toks, dtype=torch.bfloat16, device=k.device)
 
     def alloc_block_means(self) -> torch.Tensor:
         """An empty table of the shape fold_block_means fills (and the block tail reads)."""
@@ -176,7 +205,7 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
               z: Optional[torch.Tensor] = None, depth_T: float = math.inf, num_splits: int = 0, stack: int = 1,
               workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
               lse: Optional[torch.Tensor] = None, row_status: Optional[torch.Tensor] = None,
-              draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0) -> FoldArgs:
+              draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0) -> FoldArgs:
     assert q.dtype == torch.bfloat16 and q.dim() == 3 and q.stride(2) == 1
     B, Hq, D = q.shape
     a = FoldArgs()
@@ -197,6 +226,7 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
         assert draft_mask is not None and draft_mask.dtype == torch.int32 and draft_mask.numel() == B
         assert draft_mask.is_contiguous()
     a.draft_mask, a.draft_len = (_ptr(draft_mask), int(draft_len)) if draft_len else (None, 0)
+    a.refine_tau = float(refine_tau)
     return a
 
 
@@ -239,6 +269,18 @@ def fold_block_means(cache: KVCache, stream=None) -> torch.Tensor:
     _check(lib().fold_block_means(C.byref(kv), int(cache.k.shape[2]), int(cache.k.shape[3]), _stream(stream)),
            "fold_block_means")
     return cache.v_block_mean
+
+
+def fold_quantize_keys(cache: KVCache, first_token: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Cache write for two-plane INT8 keys: rotate and split the BF16 key rows of tokens first_token[s] .. seqlens[s]-1
+    (all tokens when first_token is None) into cache.k_plane_a / k_plane_b / k_scale (allocated here if absent)."""
+    if cache.k_plane_a is None:
+        cache.alloc_key_planes()
+    if first_token is not None:
+        assert first_token.dtype == torch.int32 and first_token.is_contiguous() and first_token.numel() == cache.seqlens.numel()
+    kv = cache.to_c()
+    _check(lib().fold_quantize_keys(C.byref(kv), int(cache.k.shape[2]), int(cache.k.shape[3]), _ptr(first_token),
+                                    _stream(stream)), "fold_quantize_keys")
 
 
 def fold_decode(args: FoldArgs, stream=None) -> None:
@@ -298,10 +340,11 @@ def alloc_buffers(q: torch.Tensor, cache: KVCache, stack: int = 1) -> DecodeBuff
 
 def decode(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, depth_T: float = math.inf,
            z_mode: int = Z_ESTIMATE, num_splits: int = 0, scale: Optional[float] = None, stack: int = 1,
-           draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, stream=None) -> FoldArgs:
+           draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0,
+           stream=None) -> FoldArgs:
     args = make_args(q, cache, scale=scale, z_mode=z_mode, z=bufs.z, depth_T=depth_T, num_splits=num_splits,
                      stack=stack, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status,
-                     draft_mask=draft_mask, draft_len=draft_len)
+                     draft_mask=draft_mask, draft_len=draft_len, refine_tau=refine_tau)
     fold_decode(args, stream)
     return args
 

@@ -9,6 +9,7 @@
 #include "fold_common.cuh"
 #include "fold_estimate.cuh"
 #include "fold_merge.cuh"
+#include "fold_planes.cuh"
 #include "fold_scan.cuh"
 #include "fold_scan_umma.cuh"
 
@@ -29,11 +30,26 @@ struct Geometry {
   int B, Hq, Hkv, G, D, stack, R, num_seqs, max_slots;
   long long slot_stride;
   size_t slot_bytes;
+  bool planes;            // two-plane INT8 keys
+  size_t q_off, ws_bytes; // workspace: where the split query rows start (planes), and the total
 };
 
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+// bytes after the slots for the split query rows: codes [rows][2][D], then one eta per row
+inline size_t qplane_bytes(long long rows, int D) { return round_up((size_t)rows * 2 * D, 256) + round_up((size_t)rows * 4, 256); }
+
 int check_kv(const fold_kv &kv, int D) {
-  if (!kv.k || !kv.v || !kv.seqlens) return FOLD_EINVAL;
+  const bool planes = kv.k_plane_a != nullptr;
+  if ((!kv.k && !planes) || !kv.v || !kv.seqlens) return FOLD_EINVAL;
   if (!aligned(kv.k, 16) || !aligned(kv.v, 16)) return FOLD_EINVAL;
+  if (planes) {
+    if (!kv.k_plane_b || !kv.k_scale) return FOLD_EINVAL;
+    if (!aligned(kv.k_plane_a, 16) || !aligned(kv.k_plane_b, 16) || !aligned(kv.k_scale, 16)) return FOLD_EINVAL;
+    if (kv.plane_stride_tok < D || kv.plane_stride_head < 0 || kv.plane_stride_seq < 0) return FOLD_EINVAL;
+    if (kv.plane_stride_tok % 16 || kv.plane_stride_head % 16 || kv.plane_stride_seq % 16) return FOLD_EINVAL;
+    if (kv.scale_stride_seq < 0 || kv.scale_stride_head < 0 || kv.scale_stride_seq % 8 || kv.scale_stride_head % 8)
+      return FOLD_EINVAL;
+  }
   if (kv.num_seqs < 1 || kv.max_seqlen < 0) return FOLD_EINVAL;
   if (kv.stride_tok < D || kv.stride_head < 0 || kv.stride_seq < 0) return FOLD_EINVAL;
   if (kv.stride_tok % 8 || kv.stride_head % 8 || kv.stride_seq % 8) return FOLD_EINVAL;
@@ -78,6 +94,15 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   if (g->max_slots < 1) g->max_slots = 1;
   g->slot_stride = (long long)g->R * g->D + ((g->R + 3) / 4) * 4;
   g->slot_bytes = (size_t)g->num_seqs * g->Hkv * g->max_slots * g->slot_stride * sizeof(float);
+  g->planes = a->kv.k_plane_a != nullptr;
+  g->q_off = round_up(kHeaderBytes + g->slot_bytes, 256);
+  g->ws_bytes = g->planes ? g->q_off + qplane_bytes((long long)g->B * g->Hq, g->D) : kHeaderBytes + g->slot_bytes;
+  if (g->planes) {
+    if (isnan(a->refine_tau)) return FOLD_EINVAL;
+    // the two-plane scan: one 8-row block, no drafts, no block tail, no exact-maximum pass
+    if (R > kNarrowRows || a->draft_len > 0 || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
+    if (a->kv.v_block_mean && !isinf(a->depth_T)) return FOLD_EUNSUPPORTED;
+  }
   return FOLD_OK;
 }
 
@@ -182,7 +207,48 @@ EstParams est_params(const fold_args *a, const Geometry &g) {
   return p;
 }
 
+PlaneView plane_view(const fold_kv &kv) {
+  PlaneView v;
+  v.a = kv.k_plane_a; v.b = kv.k_plane_b;
+  v.stride_seq = kv.plane_stride_seq; v.stride_tok = kv.plane_stride_tok; v.stride_head = kv.plane_stride_head;
+  v.scale = static_cast<const __nv_bfloat16 *>(kv.k_scale);
+  v.sc_stride_seq = kv.scale_stride_seq; v.sc_stride_head = kv.scale_stride_head;
+  v.page_table = kv.page_table; v.seqlens = kv.seqlens;
+  v.paged = kv.page_table != nullptr;
+  v.page_shift = v.paged ? ilog2(kv.page_size) : 0;
+  v.max_pages = kv.max_pages_per_seq;
+  v.num_pages = kv.num_pages > 0 ? kv.num_pages : 1;
+  v.max_seqlen = kv.max_seqlen;
+  return v;
+}
+
+// Two-plane keys: the front kernel splits the query rows into the workspace whatever the reference mode, and
+// forms the estimate when asked to.
+int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st) {
+  FrontParams p;
+  memset(&p, 0, sizeof(p));
+  p.q = static_cast<const __nv_bfloat16 *>(a->q);
+  p.q_stride_b = a->q_stride_b; p.q_stride_h = a->q_stride_h;
+  uint8_t *ws = static_cast<uint8_t *>(a->workspace);
+  p.qplanes = reinterpret_cast<int8_t *>(ws + g.q_off);
+  p.qeta = reinterpret_cast<float *>(ws + g.q_off + round_up((size_t)g.B * g.Hq * 2 * g.D, 256));
+  p.z = a->z;
+  p.kv = plane_view(a->kv);
+  p.write_z = a->z_mode == FOLD_Z_ESTIMATE;
+  p.stack = g.stack; p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
+  p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
+  if (a->z_mode == FOLD_Z_ZERO) {
+    const int rows = g.B * g.Hq;
+    fold_fill_kernel<<<(rows + 255) / 256, 256, 0, st>>>(a->z, rows, 0.f);
+  }
+  const dim3 grid(g.Hkv, g.B);
+  if (g.D == 128) fold_planes_front_kernel<128><<<grid, kFrontThreads, 0, st>>>(p);
+  else fold_planes_front_kernel<64><<<grid, kFrontThreads, 0, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st) {
+  if (g.planes) return launch_planes_front(a, g, st);
   if (a->z_mode == FOLD_Z_GIVEN) return FOLD_OK;
   const int rows = g.B * g.Hq;
   if (a->z_mode == FOLD_Z_ZERO) {
@@ -385,7 +451,105 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   return (max_chunks + per - 1) / per;
 }
 
+// 4-D view of key plane A (INT8): axis 0 is the channel (one box spans the whole D-byte row), then token / head /
+// sequence-or-page by stride as in make_map.  128-byte swizzle for 128-byte rows, 64-byte swizzle for 64-byte rows.
+int make_plane_map(CUtensorMap *map, MapAxes *axes, const fold_kv &kv, int D, int Hkv, int box_tok) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return FOLD_ECUDA;
+  const bool paged = kv.page_table != nullptr;
+  struct Axis { cuuint64_t extent, stride; cuuint32_t box; int id; };
+  Axis ax[3] = {{(cuuint64_t)(paged ? kv.page_size : kv.capacity), (cuuint64_t)kv.plane_stride_tok, (cuuint32_t)box_tok, 0},
+                {(cuuint64_t)Hkv, (cuuint64_t)kv.plane_stride_head, 1u, 1},
+                {(cuuint64_t)(paged ? kv.num_pages : kv.num_seqs), (cuuint64_t)kv.plane_stride_seq, 1u, 2}};
+  for (int i = 0; i < 3; ++i)
+    for (int j = i + 1; j < 3; ++j) {
+      const bool i_one = ax[i].extent == 1, j_one = ax[j].extent == 1;
+      if ((i_one && !j_one) || (i_one == j_one && ax[j].stride < ax[i].stride)) { Axis t = ax[i]; ax[i] = ax[j]; ax[j] = t; }
+    }
+  cuuint64_t prev_stride = (cuuint64_t)D, prev_extent = 1;
+  for (int i = 0; i < 3; ++i) {
+    if (ax[i].extent == 1 || ax[i].stride == 0) ax[i].stride = prev_stride * prev_extent;
+    prev_stride = ax[i].stride; prev_extent = ax[i].extent;
+  }
+  cuuint64_t dims[4] = {(cuuint64_t)D, ax[0].extent, ax[1].extent, ax[2].extent};
+  cuuint64_t strides[3] = {ax[0].stride, ax[1].stride, ax[2].stride};
+  cuuint32_t box[4] = {(cuuint32_t)D, ax[0].box, ax[1].box, ax[2].box};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  for (int i = 0; i < 3; ++i) {
+    if (ax[i].id == 0) axes->pos_tok = i + 1;
+    if (ax[i].id == 1) axes->pos_head = i + 1;
+    if (ax[i].id == 2) axes->pos_seq = i + 1;
+  }
+  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t *>(kv.k_plane_a), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, D == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? FOLD_OK : FOLD_ECUDA;
+}
+
+// Two-plane keys: one kernel for dense and finite depth (the depth gate is a comparison against -T = -inf).
+int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
+  const fold_kv &kv = a->kv;
+  const bool paged = kv.page_table != nullptr;
+  const int tile_keys = kPlaneTileKeys;
+  const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
+  CUtensorMap ma;
+  MapAxes axes;
+  if (int rc = make_plane_map(&ma, &axes, kv, g.D, g.Hkv, box_tok)) return rc;
+  PlaneScanParams pp;
+  memset(&pp, 0, sizeof(pp));
+  ScanParams &p = pp.s;
+  p.z = a->z;
+  p.seqlens = kv.seqlens;
+  p.page_table = kv.page_table;
+  p.v = static_cast<const __nv_bfloat16 *>(kv.v);
+  p.v_stride_seq = kv.stride_seq; p.v_stride_tok = kv.stride_tok; p.v_stride_head = kv.stride_head;
+  p.slots = reinterpret_cast<float *>(static_cast<uint8_t *>(a->workspace) + kHeaderBytes);
+  p.slot_stride = g.slot_stride;
+  p.hdr = static_cast<fold_ws_header *>(a->workspace);
+  p.max_slots = g.max_slots; p.max_seqlen = kv.max_seqlen;
+  p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.stack = g.stack; p.R = g.R;
+  p.paged = paged; p.page_shift = paged ? ilog2(kv.page_size) : 0;
+  p.max_pages = kv.max_pages_per_seq; p.num_pages = kv.num_pages > 0 ? kv.num_pages : 1;
+  p.box_tok = box_tok;
+  p.pos_tok = axes.pos_tok; p.pos_head = axes.pos_head; p.pos_seq = axes.pos_seq;
+  p.num_splits = choose_splits(a, g, tile_keys);
+  p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
+  p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
+  p.row_groups = 1;
+  pp.kv = plane_view(kv);
+  uint8_t *ws = static_cast<uint8_t *>(a->workspace);
+  pp.qplanes = reinterpret_cast<const int8_t *>(ws + g.q_off);
+  pp.qeta = reinterpret_cast<const float *>(ws + g.q_off + round_up((size_t)g.B * g.Hq * 2 * g.D, 256));
+  pp.auto_tau = a->refine_tau == 0.f;
+  pp.neg_tau = a->refine_tau < 0.f ? INFINITY : -a->refine_tau;      // tau = inf -> -inf: every live key
+  const dim3 grid(g.Hkv, p.num_splits, g.num_seqs);
+  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  int stages;
+  static int cfg128[64] = {0}, cfg64[64] = {0};
+  if (g.D == 128) {
+    using LO = PlaneLayout<128>;
+    stages = (per_cta2 - LO::total(0)) / (LO::kStage + 16);
+    if (stages > 4) stages = 4;
+    if (stages < 2) return FOLD_EUNSUPPORTED;
+    p.stages = stages;
+    if (int rc = opt_in_smem(fold_scan_planes_kernel<128>, cfg128)) return rc;
+    if (launch_pdl(fold_scan_planes_kernel<128>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, pp) != cudaSuccess)
+      return FOLD_ECUDA;
+  } else {
+    using LO = PlaneLayout<64>;
+    stages = (per_cta2 - LO::total(0)) / (LO::kStage + 16);
+    if (stages > 4) stages = 4;
+    if (stages < 2) return FOLD_EUNSUPPORTED;
+    p.stages = stages;
+    if (int rc = opt_in_smem(fold_scan_planes_kernel<64>, cfg64)) return rc;
+    if (launch_pdl(fold_scan_planes_kernel<64>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, pp) != cudaSuccess)
+      return FOLD_ECUDA;
+  }
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
+  if (g.planes) return launch_scan_planes(a, g, st);
   const fold_kv &kv = a->kv;
   const bool paged = kv.page_table != nullptr;
   // narrow row blocks walk 16 KB key tiles: 128 keys at D = 64
@@ -498,13 +662,27 @@ size_t fold_workspace_bytes(const fold_args *args) {
   g.max_slots = max_chunks_upto(tmp.kv.max_seqlen);
   if (g.max_slots < 1) g.max_slots = 1;
   g.slot_stride = R * tmp.head_dim + ((R + 3) / 4) * 4;
-  return kHeaderBytes + (size_t)(tmp.batch / tmp.stack) * tmp.num_kv_heads * g.max_slots * g.slot_stride * sizeof(float);
+  const size_t base = kHeaderBytes + (size_t)(tmp.batch / tmp.stack) * tmp.num_kv_heads * g.max_slots * g.slot_stride * sizeof(float);
+  if (!tmp.kv.k_plane_a) return base;
+  return round_up(base, 256) + qplane_bytes((long long)tmp.batch * tmp.num_q_heads, tmp.head_dim);
 }
 
 int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream stream) {
   if (!levels || n_levels < 1 || n_levels > kMaxLevels) return FOLD_EINVAL;
   const fold_args *a0 = levels[0];
   if (!a0) return FOLD_EINVAL;
+  for (int l = 1; l < n_levels; ++l)
+    if (levels[l] && levels[l]->kv.k_plane_a) return FOLD_EUNSUPPORTED;
+  if (a0->kv.k_plane_a) {                                    // two-plane keys: one level; the split rows go to its workspace
+    if (n_levels != 1) return FOLD_EUNSUPPORTED;
+    Geometry g;
+    fold_args tmp = *a0;
+    tmp.z_mode = FOLD_Z_ESTIMATE;
+    if (int rc = check_args(&tmp, &g, false)) return rc;
+    if (!tmp.workspace || !aligned(tmp.workspace, 256)) return FOLD_EINVAL;
+    if (tmp.workspace_bytes < g.ws_bytes) return FOLD_EWORKSPACE;
+    return launch_planes_front(&tmp, g, static_cast<cudaStream_t>(stream));
+  }
   if (a0->head_dim != 64 && a0->head_dim != 128) return FOLD_EUNSUPPORTED;
   if (a0->batch < 1 || a0->num_q_heads < 1 || a0->num_kv_heads < 1 || a0->num_q_heads % a0->num_kv_heads)
     return FOLD_EINVAL;
@@ -543,7 +721,7 @@ int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream str
   if (int rc = check_args(args, &g, false)) return rc;
   if (!dst) return FOLD_EINVAL;
   if (!args->workspace || !aligned(args->workspace, 256)) return FOLD_EINVAL;
-  if (args->workspace_bytes < kHeaderBytes + g.slot_bytes) return FOLD_EWORKSPACE;
+  if (args->workspace_bytes < g.ws_bytes) return FOLD_EWORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // header first, so that reference -> scan -> partial add are adjacent kernels in the stream
   if (cudaMemsetAsync(args->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
@@ -631,6 +809,27 @@ int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, 
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+int fold_quantize_keys(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, const int32_t *first_token,
+                       fold_stream stream) {
+  if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
+  if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
+  if (!kv->k || !kv->k_plane_a) return FOLD_EINVAL;
+  if (int rc = check_kv(*kv, head_dim)) return rc;
+  if (kv->max_seqlen == 0) return FOLD_OK;
+  QuantParams p;
+  memset(&p, 0, sizeof(p));
+  p.k = static_cast<const __nv_bfloat16 *>(kv->k);
+  p.k_stride_seq = kv->stride_seq; p.k_stride_tok = kv->stride_tok; p.k_stride_head = kv->stride_head;
+  p.kv = plane_view(*kv);
+  p.first_token = first_token;
+  const dim3 grid((kv->max_seqlen + kQuantRowsPerCta - 1) / kQuantRowsPerCta, num_kv_heads, kv->num_seqs);
+  const dim3 block(32, kQuantRowsPerCta);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (head_dim == 128) fold_quantize_keys_kernel<128><<<grid, block, 0, st>>>(p);
+  else fold_quantize_keys_kernel<64><<<grid, block, 0, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
 int fold_decode(const fold_args *args, fold_stream stream) {
   Geometry g;
   if (int rc = check_args(args, &g, true)) return rc;
@@ -644,6 +843,8 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
   if (!levels || n_levels < 1 || n_levels > kMaxLevels || !levels[0]) return FOLD_EINVAL;
   const fold_args *a0 = levels[0];
   if (a0->z_mode != FOLD_Z_ESTIMATE && a0->z_mode != FOLD_Z_GIVEN) return FOLD_EINVAL;
+  for (int l = 0; l < n_levels; ++l)
+    if (levels[l] && levels[l]->kv.k_plane_a) return FOLD_EUNSUPPORTED;   // two-plane keys: fold_decode only
   fold_args lv[kMaxLevels];
   for (int l = 0; l < n_levels; ++l) {
     const fold_args *a = levels[l];
@@ -731,6 +932,7 @@ int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, f
   if (ha->z_mode == FOLD_Z_GIVEN && !ha->z) return FOLD_EINVAL;
   if (ha->kv.v_block_mean) return FOLD_EUNSUPPORTED;        // the block tail is not offered for host buffers
   if (ha->draft_len != 0) return FOLD_EUNSUPPORTED;         // nor are draft masks
+  if (ha->kv.k_plane_a) return FOLD_EUNSUPPORTED;           // nor two-plane keys
   HostPlan h;
   if (fold_workspace_bytes(ha) == 0 || !plan_host(ha, &h)) return FOLD_EINVAL;
   if (staging_bytes < h.total) return FOLD_EWORKSPACE;

@@ -66,6 +66,52 @@ __device__ __forceinline__ int est_sample_key(int i, int n) {
   return (e0 + e1) >> 1;
 }
 
+// One warp finishes one row from its sampled scores row[0 .. n_samples): maximum, exact part, trimmed
+// stratified part.  n = the row's key count.  Every lane returns the row's reference.
+__device__ __forceinline__ float est_reduce_row(const float *row, int n, int n_samples, int lane) {
+  float zval = 0.f;
+  if (n_samples > 0) {
+    float m = -INFINITY;
+    for (int k = lane; k < n_samples; k += 32) m = fmaxf(m, row[k]);
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+    float total = 0.f;                             // fixed summation order: lane-strided, then a shuffle tree
+    if (n <= kEstSamples) {
+      for (int k = lane; k < n_samples; k += 32) total += exp2f(row[k] - m);
+    } else {
+      for (int k = lane; k <= kEstRecent; k += 32) total += exp2f(row[k] - m);      // sink + 63 recent
+      // the 128 centre scores, four per lane (centre lane + 32 i); drop the 8 largest, one per round:
+      // the warp-wide maximum, owned by the lowest index among equals
+      float c[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) c[i] = row[1 + kEstRecent + lane + 32 * i];
+#pragma unroll 1
+      for (int r = 0; r < kEstTrim; ++r) {
+        float wm = fmaxf(fmaxf(c[0], c[1]), fmaxf(c[2], c[3]));
+#pragma unroll
+        for (int k = 16; k > 0; k >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, k));
+        bool found = false;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const unsigned owners = __ballot_sync(0xffffffffu, c[i] == wm);
+          if (!found && owners) {
+            if (lane == __ffs(owners) - 1) c[i] = -INFINITY;
+            found = true;
+          }
+        }
+      }
+      float kept = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) kept += exp2f(c[i] - m);                              // dropped ones add 2^-inf = 0
+      total += kept * ((float)(n - 1 - kEstRecent) / (float)(kEstStrata - kEstTrim));
+    }
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) total += __shfl_xor_sync(0xffffffffu, total, k);
+    zval = m + log2f(total);
+  }
+  return zval;
+}
+
 // One CTA per (kv head, request), 12 warps.  The 192 x G scores are one small matrix product: warp w
 // takes sampled keys 16w .. 16w+15 on M, the group's query rows on N (mma.sync m16n8k16, BF16 in,
 // FP32 accumulate).  Each lane loads its A fragments straight from the cache rows (all loads issued
@@ -147,48 +193,9 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
   }
   __syncthreads();
 
-  // warp g finishes row g: maximum, exact part, trimmed stratified part
+  // warp g finishes row g
   for (int g = warp; g < G; g += kEstSampleThreads / 32) {
-    float zval = 0.f;
-    if (n_samples > 0) {
-      float m = -INFINITY;
-      for (int k = lane; k < n_samples; k += 32) m = fmaxf(m, sc[g][k]);
-#pragma unroll
-      for (int k = 16; k > 0; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
-      float total = 0.f;                             // fixed summation order: lane-strided, then a shuffle tree
-      if (n <= kEstSamples) {
-        for (int k = lane; k < n_samples; k += 32) total += exp2f(sc[g][k] - m);
-      } else {
-        for (int k = lane; k <= kEstRecent; k += 32) total += exp2f(sc[g][k] - m);      // sink + 63 recent
-        // the 128 centre scores, four per lane (centre lane + 32 i); drop the 8 largest, one per round:
-        // the warp-wide maximum, owned by the lowest index among equals
-        float c[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) c[i] = sc[g][1 + kEstRecent + lane + 32 * i];
-#pragma unroll 1
-        for (int r = 0; r < kEstTrim; ++r) {
-          float wm = fmaxf(fmaxf(c[0], c[1]), fmaxf(c[2], c[3]));
-#pragma unroll
-          for (int k = 16; k > 0; k >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, k));
-          bool found = false;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const unsigned owners = __ballot_sync(0xffffffffu, c[i] == wm);
-            if (!found && owners) {
-              if (lane == __ffs(owners) - 1) c[i] = -INFINITY;
-              found = true;
-            }
-          }
-        }
-        float kept = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) kept += exp2f(c[i] - m);                              // dropped ones add 2^-inf = 0
-        total += kept * ((float)(n - 1 - kEstRecent) / (float)(kEstStrata - kEstTrim));
-      }
-#pragma unroll
-      for (int k = 16; k > 0; k >>= 1) total += __shfl_xor_sync(0xffffffffu, total, k);
-      zval = m + log2f(total);
-    }
+    const float zval = est_reduce_row(sc[g], n, n_samples, lane);
     if (lane == 0) p.z[(long long)req * p.Hq + kvh * G + g] = zval;
   }
 }

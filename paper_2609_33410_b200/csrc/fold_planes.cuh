@@ -1,0 +1,550 @@
+// Two-plane INT8 keys (Section 4, "Cache format" and "Weight-gated reads"; Algorithm 1).
+//
+//   cache write   fold_quantize_keys_kernel: rotate a BF16 key row by the orthonormal Hadamard matrix, split
+//                 it into two INT8 planes and a BF16 scale rounded up:  H k = e (a + b / 256)
+//   front         fold_planes_front_kernel: split every query row the same way (into the workspace) and
+//                 form the 192-key reference estimate on two-plane scores
+//   scan          fold_scan_planes_kernel: every key is scored against plane A alone (INT8 products, keys
+//                 on M, the group's rows on N); the verdict bits live / refine are ORed over the group, and
+//                 only then are plane B rows (refined keys) and value rows (live keys) requested; a second
+//                 INT8 product adds plane B; final FP32 weights feed the BF16 value product.
+#pragma once
+
+#include "fold_common.cuh"
+#include "fold_estimate.cuh"
+#include "fold_scan.cuh"
+
+namespace fold {
+
+// The key planes as the kernels see them.
+struct PlaneView {
+  const int8_t *a, *b;
+  long long stride_seq, stride_tok, stride_head;              // bytes
+  const __nv_bfloat16 *scale;
+  long long sc_stride_seq, sc_stride_head;                    // elements; tokens are contiguous
+  const int *page_table;
+  const int *seqlens;
+  int paged, page_shift, max_pages, num_pages, max_seqlen;
+};
+
+// (sequence-or-page, token-in-it) of logical token j
+__device__ __forceinline__ void plane_locate(const PlaneView &kv, int seq, int j, long long &s, long long &t) {
+  s = seq; t = j;
+  if (kv.paged) {
+    int pg = kv.page_table[(long long)seq * kv.max_pages + (j >> kv.page_shift)];
+    s = min(max(pg, 0), kv.num_pages - 1);
+    t = j & ((1 << kv.page_shift) - 1);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rotation and split of one row held by a warp: lane l has channels l * D/32 .. + D/32 - 1 in x[].
+// FP32, one rounding per step, in this order (the codes are integers decided by this arithmetic, so the order
+// is part of the format): butterfly stages with strides 1, 2, 4, ..., D/2, each (lo, hi) -> (lo + hi, lo - hi);
+// one multiply by fp32(1 / sqrt(D)); e = the smallest BF16 >= max|y| / 127 (1 for an all-zero row);
+// t = y / e; a = rint(t) within +-127; b = rint((t - a) * 256) within [-128, 127].  Returns e.
+template <int D>
+__device__ __forceinline__ float rotate_split(float (&x)[D / 32], int lane, int (&a)[D / 32], int (&b)[D / 32]) {
+  constexpr int EPL = D / 32;
+#pragma unroll
+  for (int h = 1; h < EPL; h <<= 1)
+#pragma unroll
+    for (int i = 0; i < EPL; ++i)
+      if (!(i & h)) {
+        const float lo = x[i], hi = x[i + h];
+        x[i] = __fadd_rn(lo, hi);
+        x[i + h] = __fsub_rn(lo, hi);
+      }
+#pragma unroll
+  for (int m = 1; m < 32; m <<= 1)
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+      const float other = __shfl_xor_sync(0xffffffffu, x[i], m);
+      x[i] = (lane & m) ? __fsub_rn(other, x[i]) : __fadd_rn(x[i], other);
+    }
+  const float r_sqrt_d = D == 64 ? 0.125f : __uint_as_float(0x3db504f3u);      // fp32(1 / sqrt(D))
+  float mx = 0.f;
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    x[i] = __fmul_rn(x[i], r_sqrt_d);
+    mx = fmaxf(mx, fabsf(x[i]));
+  }
+#pragma unroll
+  for (int m = 16; m > 0; m >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, m));
+  float e = 1.f;
+  if (mx > 0.f) {
+    const uint32_t u = __float_as_uint(__fdiv_rn(mx, 127.f));
+    e = __uint_as_float((u & 0xffffu) ? ((u >> 16) + 1u) << 16 : u);
+    if (!(e > 0.f)) e = 1.f;
+  }
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const float t = __fdiv_rn(x[i], e);
+    const float af = fminf(fmaxf(rintf(t), -127.f), 127.f);
+    const float bf = fminf(fmaxf(rintf(__fmul_rn(__fsub_rn(t, af), 256.f)), -128.f), 127.f);
+    a[i] = (int)af;
+    b[i] = (int)bf;
+  }
+  return e;
+}
+
+template <int EPL>
+__device__ __forceinline__ void load_bf16_row(const __nv_bfloat16 *row, float (&x)[EPL]) {
+  if (EPL == 4) {
+    const uint2 w = *reinterpret_cast<const uint2 *>(row);
+    x[0] = __uint_as_float(w.x << 16); x[1] = __uint_as_float(w.x & 0xffff0000u);
+    x[EPL - 2] = __uint_as_float(w.y << 16); x[EPL - 1] = __uint_as_float(w.y & 0xffff0000u);
+  } else {
+    const uint32_t w = *reinterpret_cast<const uint32_t *>(row);
+    x[0] = __uint_as_float(w << 16); x[1] = __uint_as_float(w & 0xffff0000u);
+  }
+}
+template <int EPL>
+__device__ __forceinline__ void store_codes(int8_t *dst, const int (&c)[EPL]) {       // EPL consecutive bytes
+  if (EPL == 4) {
+    *reinterpret_cast<uint32_t *>(dst) = (uint32_t)(c[0] & 0xff) | ((uint32_t)(c[1] & 0xff) << 8) |
+                                         ((uint32_t)(c[EPL - 2] & 0xff) << 16) | ((uint32_t)(c[EPL - 1] & 0xff) << 24);
+  } else {
+    *reinterpret_cast<uint16_t *>(dst) = (uint16_t)((c[0] & 0xff) | ((c[1] & 0xff) << 8));
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Cache write: one warp per (sequence, token, kv head) row.
+struct QuantParams {
+  const __nv_bfloat16 *k;
+  long long k_stride_seq, k_stride_tok, k_stride_head;
+  PlaneView kv;                                               // destinations (written)
+  const int *first_token;                                     // per sequence, or null: from token 0
+};
+constexpr int kQuantRowsPerCta = 8;
+
+template <int D>
+__global__ void __launch_bounds__(32 * kQuantRowsPerCta) fold_quantize_keys_kernel(const QuantParams p) {
+  constexpr int EPL = D / 32;
+  const int lane = threadIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
+  int n = p.kv.seqlens[seq];
+  n = n < 0 ? 0 : (n > p.kv.max_seqlen ? p.kv.max_seqlen : n);
+  const int first = p.first_token ? max(p.first_token[seq], 0) : 0;
+  const int j = first + blockIdx.x * kQuantRowsPerCta + threadIdx.y;
+  if (j >= n) return;
+  long long s, t;
+  plane_locate(p.kv, seq, j, s, t);
+  float x[EPL];
+  load_bf16_row<EPL>(p.k + s * p.k_stride_seq + t * p.k_stride_tok + (long long)kvh * p.k_stride_head + lane * EPL, x);
+  int a[EPL], b[EPL];
+  const float e = rotate_split<D>(x, lane, a, b);
+  const long long off = s * p.kv.stride_seq + t * p.kv.stride_tok + (long long)kvh * p.kv.stride_head + lane * EPL;
+  store_codes<EPL>(const_cast<int8_t *>(p.kv.a) + off, a);
+  store_codes<EPL>(const_cast<int8_t *>(p.kv.b) + off, b);
+  if (lane == 0)
+    const_cast<__nv_bfloat16 *>(p.kv.scale)[s * p.kv.sc_stride_seq + (long long)kvh * p.kv.sc_stride_head + t] =
+        __float2bfloat16_rn(e);                              // exact: e is a BF16 value
+}
+
+// ------------------------------------------------------------------------------------------------
+// Front kernel: one CTA per (kv head, request).  Splits the group's query rows (rows of the workspace:
+// [request * Hq + head][2][D] codes and one eta = e_q * scale_log2 per row), then, if the reference is to be
+// estimated, thread i scores sampled key i with both planes (exact integer dot products) and warp g
+// reduces row g.
+struct FrontParams {
+  const __nv_bfloat16 *q;
+  long long q_stride_b, q_stride_h;
+  int8_t *qplanes;
+  float *qeta;
+  float *z;
+  PlaneView kv;
+  int write_z, stack, Hq, Hkv, G;
+  float scale_log2;
+};
+constexpr int kFrontThreads = kEstSamples;                    // 192
+
+template <int D>
+__global__ void __launch_bounds__(kFrontThreads) fold_planes_front_kernel(const FrontParams p) {
+  constexpr int EPL = D / 32, W = D / 4;                      // W: 32-bit words per plane row
+  __shared__ uint32_t sq[kMaxRows][2][W];
+  __shared__ float seta[kMaxRows];
+  __shared__ float sc[kMaxRows][kEstSamples];
+  const int kvh = blockIdx.x, req = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = p.G;
+  pdl_launch_dependents();
+
+  for (int g = warp; g < G; g += kFrontThreads / 32) {
+    const int head = kvh * G + g;
+    float x[EPL];
+    load_bf16_row<EPL>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + lane * EPL, x);
+    int a[EPL], b[EPL];
+    const float e = rotate_split<D>(x, lane, a, b);
+    const float eta = __fmul_rn(e, p.scale_log2);
+    int8_t *dst = p.qplanes + ((long long)req * p.Hq + head) * (2 * D);
+    store_codes<EPL>(dst + lane * EPL, a);
+    store_codes<EPL>(dst + D + lane * EPL, b);
+    store_codes<EPL>(reinterpret_cast<int8_t *>(&sq[g][0][0]) + lane * EPL, a);
+    store_codes<EPL>(reinterpret_cast<int8_t *>(&sq[g][1][0]) + lane * EPL, b);
+    if (lane == 0) { p.qeta[(long long)req * p.Hq + head] = eta; seta[g] = eta; }
+  }
+  if (!p.write_z) return;
+  __syncthreads();
+
+  const int seq = req / p.stack;
+  int n = p.kv.seqlens[seq];
+  n = n < 0 ? 0 : (n > p.kv.max_seqlen ? p.kv.max_seqlen : n);
+  const int n_samples = n < kEstSamples ? n : kEstSamples;
+  const int i = threadIdx.x;
+  if (i < n_samples) {
+    long long s, t;
+    plane_locate(p.kv, seq, est_sample_key(i, n), s, t);
+    const long long off = s * p.kv.stride_seq + t * p.kv.stride_tok + (long long)kvh * p.kv.stride_head;
+    const float e = __bfloat162float(p.kv.scale[s * p.kv.sc_stride_seq + (long long)kvh * p.kv.sc_stride_head + t]);
+    uint32_t ka[W], kb[W];
+#pragma unroll
+    for (int w4 = 0; w4 < W / 4; ++w4) {
+      const uint4 va = *reinterpret_cast<const uint4 *>(p.kv.a + off + w4 * 16);
+      const uint4 vb = *reinterpret_cast<const uint4 *>(p.kv.b + off + w4 * 16);
+      ka[4 * w4] = va.x; ka[4 * w4 + 1] = va.y; ka[4 * w4 + 2] = va.z; ka[4 * w4 + 3] = va.w;
+      kb[4 * w4] = vb.x; kb[4 * w4 + 1] = vb.y; kb[4 * w4 + 2] = vb.z; kb[4 * w4 + 3] = vb.w;
+    }
+    for (int g = 0; g < G; ++g) {
+      int caa = 0, cab = 0, cba = 0, cbb = 0;
+#pragma unroll
+      for (int w = 0; w < W; ++w) {
+        const int qa = (int)sq[g][0][w], qb = (int)sq[g][1][w];
+        caa = __dp4a((int)ka[w], qa, caa); cab = __dp4a((int)ka[w], qb, cab);
+        cba = __dp4a((int)kb[w], qa, cba); cbb = __dp4a((int)kb[w], qb, cbb);
+      }
+      const float f = ((float)caa + (float)cab * 0.00390625f) + ((float)cba + (float)cbb * 0.00390625f) * 0.00390625f;
+      sc[g][i] = f * (seta[g] * e);
+    }
+  }
+  __syncthreads();
+  for (int g = warp; g < G; g += kFrontThreads / 32) {
+    const float zval = est_reduce_row(sc[g], n, n_samples, lane);
+    if (lane == 0) p.z[(long long)req * p.Hq + kvh * G + g] = zval;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Scan.
+struct PlaneScanParams {
+  ScanParams s;                                               // rows, references, value cache, slots, geometry
+  PlaneView kv;
+  const int8_t *qplanes;
+  const float *qeta;
+  float neg_tau;                                              // -tau_K; -inf: refine every live key; +inf: none
+  int auto_tau;                                               // tau_K = log2(n) + 7 from the sequence's own length
+};
+
+constexpr int kPlaneTileKeys = 128;                           // keys per plane-A tile
+constexpr int kPlaneBufs = 2;                                 // gather buffers per warp (one in flight, one in use)
+
+template <int D>
+struct PlaneLayout {
+  static constexpr int kTK = kPlaneTileKeys;
+  static constexpr int kATile = kTK * D;                      // plane A codes, swizzled as the tensor map writes them
+  static constexpr int kStage = kATile + 1024;                // + the tile's scales (kTK * 2 bytes), 1 KB-aligned
+  static constexpr int kBBuf = 16 * D;                        // plane B rows of one 16-key sub-slice
+  static constexpr int kVBuf = 16 * D * 2;                    // value rows of one sub-slice, [D/64][16][128 B] swizzled
+  static constexpr int kWarpBufs = kPlaneBufs * (kBBuf + kVBuf);
+  __host__ __device__ static int off_bufs(int stages) { return stages * kStage; }
+  // the chunk-end reduction parks in the gather buffers (drained by then): 4 warps x R x D floats <= 4 x kWarpBufs
+  __host__ __device__ static int off_redl(int stages) { return off_bufs(stages) + kConsumerWarps * kWarpBufs; }
+  __host__ __device__ static int off_bar(int stages) { return off_redl(stages) + kConsumerWarps * kMaxRows * 4; }
+  __host__ __device__ static int total(int stages) { return off_bar(stages) + 2 * stages * 8 + 1024; }
+};
+
+// Byte offset of 16-byte chunk `ch` of key row `key` in a tile of D-byte rows: the 128-byte swizzle for 128-byte
+// rows, the 64-byte swizzle for 64-byte rows (what the tensor map writes; the gather buffers use the same).
+template <int D>
+__device__ __forceinline__ uint32_t plane_off(int key, int ch) {
+  return D == 128 ? (uint32_t)(key * 128 + ((ch ^ (key & 7)) << 4)) : (uint32_t)(key * 64 + ((ch ^ ((key >> 1) & 3)) << 4));
+}
+
+__device__ __forceinline__ void mma_s8(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// c^xa, c^xb [16 keys, 8 rows] = plane X of 16 keys (rows key0.. of the tile at `tile`) times [Q^a; Q^b]^T.
+// c[0], c[1]: key lane/4, rows (lane%4)*2 + {0,1};  c[2], c[3]: key lane/4 + 8.
+template <int D>
+__device__ __forceinline__ void plane_products(uint32_t tile, int key0, int lane, const uint32_t (&qa)[D / 32][2],
+                                               const uint32_t (&qb)[D / 32][2], int (&ca)[4], int (&cb)[4]) {
+  // ldmatrix matrix i = lane/8: keys (i&1)*8 + lane%8, 16-byte chunk 2*kk + (i>>1)
+  const int key = key0 + (((lane >> 3) & 1) << 3) + (lane & 7);
+  ca[0] = ca[1] = ca[2] = ca[3] = 0;
+  cb[0] = cb[1] = cb[2] = cb[3] = 0;
+#pragma unroll
+  for (int kk = 0; kk < D / 32; ++kk) {
+    uint32_t a[4];
+    ldsm_x4(tile + plane_off<D>(key, 2 * kk + (lane >> 4)), a[0], a[1], a[2], a[3]);
+    mma_s8(ca, a, qa[kk][0], qa[kk][1]);
+    mma_s8(cb, a, qb[kk][0], qb[kk][1]);
+  }
+}
+
+// Producer thread: plane A tiles by TMA, their scales by bulk copies, one stage per 128-key tile.
+template <int D>
+__device__ __forceinline__ void produce_plane_tiles(const CUtensorMap *tmA, const PlaneScanParams &pp, const SeqWork &w,
+                                                    int split, int kvh, int seq, uint32_t ring, uint32_t full0,
+                                                    uint32_t empty0) {
+  using LO = PlaneLayout<D>;
+  const ScanParams &p = pp.s;
+  tma_prefetch_desc(tmA);
+  const uint64_t pol = policy_evict_first();
+  bool dead = false;
+  int stage = 0;
+  uint32_t wrapped = 0, phase = 0;
+  const int boxes_per_tile = LO::kTK / p.box_tok;
+  const int page_mask = (1 << p.page_shift) - 1;
+  for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w); cursor_next(k, w, p.num_splits)) {
+    if (wrapped && !mbar_wait(empty0 + 8u * stage, phase ^ 1u, dead)) break;
+    const int tok0 = k.t * LO::kTK;
+    const int nbox = min(boxes_per_tile, (w.n - tok0 + p.box_tok - 1) / p.box_tok);
+    const uint32_t full = full0 + 8u * stage;
+    int sc_tokens = 0;                                       // scale tokens copied: whole groups of 8 (16 bytes)
+    for (int bx = 0; bx < nbox; ++bx) sc_tokens += min(p.box_tok, (w.n - (tok0 + bx * p.box_tok) + 7) & ~7);
+    mbar_expect_tx(full, nbox * p.box_tok * D + sc_tokens * 2);
+    const uint32_t dst = ring + stage * LO::kStage;
+    for (int bx = 0; bx < nbox; ++bx) {
+      const int j0 = tok0 + bx * p.box_tok;
+      int c_seq = seq, c_tok = j0;
+      if (p.paged) {
+        c_seq = min(max(p.page_table[(long long)seq * p.max_pages + (j0 >> p.page_shift)], 0), p.num_pages - 1);
+        c_tok = j0 & page_mask;
+      }
+      const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
+      const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
+      const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
+      tma_load_4d(dst + bx * p.box_tok * D, tmA, full, 0, c1, c2, c3, pol);
+      const int cnt = min(p.box_tok, (w.n - j0 + 7) & ~7);
+      bulk_load(dst + LO::kATile + bx * p.box_tok * 2,
+                pp.kv.scale + (long long)c_seq * pp.kv.sc_stride_seq + (long long)kvh * pp.kv.sc_stride_head + c_tok,
+                cnt * 2, full);
+    }
+    if (++stage == p.stages) { stage = 0; wrapped = 1u; phase ^= 1u; }
+  }
+  if (dead) atomicOr(&p.hdr->wait_timeouts, 1u);
+}
+
+// One sub-slice (16 keys) between its coarse pass and its second pass.
+struct PlanePending {
+  float x[4];            // coarse score minus reference: key lane/4 (+8), rows (lane%4)*2 + {0,1}; -inf if unused
+  float e[2];            // the two keys' scales
+  uint32_t live, refine; // verdict bits of the 16 keys, ORed over the rows
+  int buf;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDenseThreads, 2)
+fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const PlaneScanParams pp) {
+  using LO = PlaneLayout<D>;
+  constexpr int TK = LO::kTK, U = TK / (16 * kConsumerWarps);          // sub-slices per warp and tile
+  constexpr int CV = D / 8, CB = D / 16;                               // 16-byte chunks per value row / plane row
+  const ScanParams &p = pp.s;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
+  const SeqWork w = seq_work<TK>(p, seq);
+  if (split >= w.n_chunks) return;
+  const int stages = p.stages, R = p.R, n = w.n;
+  const uint32_t full0 = base + LO::off_bar(stages), empty0 = full0 + 8u * stages;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, kConsumerWarps);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();                                                // z, the split query rows and the zeroed header
+
+  if (warp == kConsumerWarps) {
+    if (lane == 0) produce_plane_tiles<D>(&tmA, pp, w, split, kvh, seq, base, full0, empty0);
+    return;
+  }
+
+  // query rows: B fragments of the INT8 products (row lane/4), scales and references of the score rows
+  uint32_t qa[D / 32][2], qb[D / 32][2];
+  {
+    const int r = lane >> 2;
+    const bool ok = r < R;
+    const int req = seq * p.stack + r / p.G, head = kvh * p.G + r % p.G;
+    const int8_t *qp = pp.qplanes + ((long long)req * p.Hq + head) * (2 * D) + (lane & 3) * 4;
+#pragma unroll
+    for (int kk = 0; kk < D / 32; ++kk) {
+      qa[kk][0] = ok ? *reinterpret_cast<const uint32_t *>(qp + kk * 32) : 0u;
+      qa[kk][1] = ok ? *reinterpret_cast<const uint32_t *>(qp + kk * 32 + 16) : 0u;
+      qb[kk][0] = ok ? *reinterpret_cast<const uint32_t *>(qp + D + kk * 32) : 0u;
+      qb[kk][1] = ok ? *reinterpret_cast<const uint32_t *>(qp + D + kk * 32 + 16) : 0u;
+    }
+  }
+  float eta[2], zr[2];
+  bool rv[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int r = (lane & 3) * 2 + e;
+    rv[e] = r < R;
+    const long long row = (long long)(seq * p.stack + r / p.G) * p.Hq + kvh * p.G + r % p.G;
+    eta[e] = rv[e] ? pp.qeta[row] : 0.f;
+    zr[e] = rv[e] ? p.z[row] : 0.f;
+  }
+  const float neg_T = p.neg_T;
+  const float neg_tau = pp.auto_tau ? -(log2f((float)max(n, 1)) + 7.f) : pp.neg_tau;
+
+  float o[D / 16][4];
+#pragma unroll
+  for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float l_lo = 0.f, l_hi = 0.f;
+  const uint32_t bufs = base + LO::off_bufs(stages) + warp * LO::kWarpBufs;
+  float *red = reinterpret_cast<float *>(gen + LO::off_bufs(stages));
+  float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages));
+  const int klo = lane >> 2;
+
+  // second pass of a sub-slice: plane B product, final weights, value product
+  auto finish = [&](const PlanePending &pd) {
+    const uint32_t bbuf = bufs + pd.buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
+    int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
+    if (pd.refine) plane_products<D>(bbuf, 0, lane, qa, qb, ca, cb);      // unrefined keys' rows were zero-filled
+    uint32_t bh[2], bl[2];
+#pragma unroll
+    for (int kh = 0; kh < 2; ++kh) {
+      const bool klive = (pd.live >> (klo + 8 * kh)) & 1u;
+      float pw[2], pm[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int i = 2 * kh + e;
+        const float corr = ((float)ca[i] + (float)cb[i] * 0.00390625f) * 0.00390625f;
+        const float x = fmaf(corr, eta[e] * pd.e[kh], pd.x[i]);
+        const bool live = klive && (x >= neg_T);
+        pw[e] = ex2_approx(x);
+        pm[e] = live ? pw[e] : 0.f;
+      }
+      const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
+      const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
+      const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
+      const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
+      l_lo += (h0 + g0) + (pw[0] - pm[0]);
+      l_hi += (h1 + g1) + (pw[1] - pm[1]);
+      bh[kh] = movmatrix_trans(hi2);
+      bl[kh] = movmatrix_trans(lo2);
+    }
+    if (pd.live) value_product_n<D, true, 0, 16>(o, vbuf, 0, lane, bh, bl);
+  };
+
+  bool dead = false, have = false;
+  int stage = 0, buf = 0;
+  uint32_t phase = 0;
+  unsigned long long st_total = 0, st_live = 0, st_ref = 0;
+  PlanePending pend;
+  const int page_mask = (1 << p.page_shift) - 1;
+
+  for (int c = split; c < w.n_chunks; c += p.num_splits) {
+    const int t_end = min((c + 1) * w.ctiles, w.n_tiles);
+    for (int t = c * w.ctiles; t < t_end; ++t) {
+      const int my_stage = stage;
+      const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
+      if (++stage == stages) { stage = 0; phase ^= 1u; }
+      if (!ready) continue;
+      const uint32_t at = base + my_stage * LO::kStage;
+      const __nv_bfloat16 *scales = reinterpret_cast<const __nv_bfloat16 *>(gen + my_stage * LO::kStage + LO::kATile);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int sub = warp * U + u;                         // 16-key sub-slice of the tile
+        const int key0 = t * TK + sub * 16;
+        if (key0 >= n) continue;                              // warp-uniform
+        st_total += min(16, n - key0);
+        // coarse pass: plane A against both query planes
+        PlanePending cur;
+        int ca[4], cb[4];
+        plane_products<D>(at, sub * 16, lane, qa, qb, ca, cb);
+        uint32_t lm = 0, rm = 0;
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh) {
+          const int key = key0 + klo + 8 * kh;
+          cur.e[kh] = key < n ? __bfloat162float(scales[sub * 16 + klo + 8 * kh]) : 0.f;
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int i = 2 * kh + e;
+            const bool ok = key < n && rv[e];
+            const float f = (float)ca[i] + (float)cb[i] * 0.00390625f;
+            const float x = ok ? fmaf(f, eta[e] * cur.e[kh], -zr[e]) : -INFINITY;
+            cur.x[i] = x;
+            if (ok && x >= neg_T) lm |= 1u << (klo + 8 * kh);
+            if (ok && x >= neg_tau) rm |= 1u << (klo + 8 * kh);
+          }
+        }
+        cur.live = __reduce_or_sync(0xffffffffu, lm);
+        cur.refine = __reduce_or_sync(0xffffffffu, rm) & cur.live;
+        cur.buf = buf;
+        st_live += __popc(cur.live);
+        st_ref += __popc(cur.refine);
+        // only now are bytes requested: plane B rows of refined keys, value rows of live keys (others zero-filled)
+        __syncwarp();                                         // the buffer's last readers are done
+        const uint32_t bbuf = bufs + buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
+        if (cur.live) {
+          long long s_row = seq, t_row = key0;
+          if (p.paged) {
+            s_row = min(max(p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)], 0), p.num_pages - 1);
+            t_row = key0 & page_mask;
+          }
+          if (cur.refine) {
+            const int8_t *src0 = pp.kv.b + s_row * pp.kv.stride_seq + t_row * pp.kv.stride_tok + (long long)kvh * pp.kv.stride_head;
+#pragma unroll
+            for (int i = 0; i < CB / 2; ++i) {
+              const int cidx = lane + 32 * i, key = cidx / CB, ch = cidx % CB;
+              const bool f = (cur.refine >> key) & 1u;
+              cp_async_16(bbuf + plane_off<D>(key, ch), f ? src0 + (long long)key * pp.kv.stride_tok + ch * 16 : pp.kv.b, f ? 16u : 0u);
+            }
+          }
+          const __nv_bfloat16 *v0 = p.v + s_row * p.v_stride_seq + t_row * p.v_stride_tok + (long long)kvh * p.v_stride_head;
+#pragma unroll
+          for (int i = 0; i < CV / 2; ++i) {
+            const int cidx = lane + 32 * i, key = cidx / CV, ch = cidx % CV;
+            const bool f = (cur.live >> key) & 1u;
+            cp_async_16(vbuf + (ch >> 3) * (16 * 128) + key * 128 + (((ch & 7) ^ (key & 7)) << 4),
+                        f ? v0 + (long long)key * p.v_stride_tok + ch * 8 : p.v, f ? 16u : 0u);
+          }
+        }
+        cp_async_commit();
+        if (have) {                                           // the sub-slice before this one: its rows have landed
+          cp_async_wait<1>();
+          __syncwarp();
+          finish(pend);
+        }
+        pend = cur;
+        have = true;
+        buf ^= 1;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);     // plane A and the scales are no longer needed
+    }
+    if (have) {
+      cp_async_wait<0>();
+      __syncwarp();
+      finish(pend);
+      have = false;
+    }
+    named_bar(1, kConsumerWarps * 32);                        // every warp's buffers are drained: park there
+    float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
+    reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
+    reduce_store_A_n<D, kConsumerWarps>(o, red, slot, R, warp, lane, threadIdx.x, 1);
+  }
+
+  if (lane == 0) {
+    if (dead) atomicOr(&p.hdr->wait_timeouts, 2u);
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_live);
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
+    atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->k_rows_refined), st_ref);
+  }
+}
+
+}  // namespace fold

@@ -1,0 +1,290 @@
+"""Two-plane INT8 keys on the GPU against the oracle: the cache writer and the query split bit for bit
+(integer codes decided by FP32 arithmetic both sides perform identically), the decode within the build's
+tolerances of Algorithm 1 evaluated in float64 at the GPU's own references."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_33410_b200 as F
+from oracle import fold_oracle as O
+from oracle import fold_planes_oracle as P
+from paper_2609_33410_b200.workloads import make_decode_workload, bf16_bits
+from helpers import cache_of, same_bits, DENSE_MAX_ABS, DENSE_MEAN_REL, FINITE_T_FACTOR, LSE_TOL, Z_TOL
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+BAND = 2.0 ** -10          # binades around a gate within which fp32 and fp64 scores may decide differently
+
+
+def scale_log2_f32(w):
+    return np.float32(np.float64(np.float32(w.scale)) * 1.4426950408889634)
+
+
+def plane_cache(w):
+    cache = cache_of(w)
+    F.fold_quantize_keys(cache)
+    torch.cuda.synchronize()
+    return cache
+
+
+def logical_planes(w, cache, seq, kvh):
+    """(a, b, e) of the logical keys of one (sequence, kv head), read back from the device planes."""
+    n = int(w.seqlens[seq])
+    j = torch.arange(n, device=cache.k.device)
+    if w.paged:
+        ps = cache.k.shape[1]
+        pg = w.page_table[seq].long()[j // ps]
+        a = cache.k_plane_a[pg, j % ps, kvh]; b = cache.k_plane_b[pg, j % ps, kvh]; e = cache.k_scale[pg, kvh, j % ps]
+    else:
+        a = cache.k_plane_a[seq, :n, kvh]; b = cache.k_plane_b[seq, :n, kvh]; e = cache.k_scale[seq, kvh, :n]
+    return a.cpu().numpy(), b.cpu().numpy(), e.float().cpu().numpy()
+
+
+def split_queries(w, bufs):
+    """The split query rows the front kernel left in the workspace: (qa, qb [B, Hq, D] int8, eta [B, Hq] fp32)."""
+    B, Hq, D = w.q.shape
+    probe = F.make_args(w.q, cache_of(w), stack=w.stack)
+    q_off = (F.fold_workspace_bytes(probe) + 255) // 256 * 256
+    codes = bufs.workspace[q_off: q_off + B * Hq * 2 * D].view(torch.int8).view(B, Hq, 2, D).cpu().numpy()
+    e_off = q_off + (B * Hq * 2 * D + 255) // 256 * 256
+    eta = bufs.workspace[e_off: e_off + B * Hq * 4].view(torch.float32).view(B, Hq).cpu().numpy()
+    return codes[:, :, 0], codes[:, :, 1], eta
+
+
+def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0, z=None):
+    bufs = F.alloc_buffers(w.q, cache, w.stack)
+    if z is not None:
+        bufs.z.copy_(z)
+    F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale, refine_tau=tau)
+    torch.cuda.synchronize()
+    assert bufs.header().wait_timeouts == 0
+    return bufs
+
+
+def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estimate=False, check_counts=True):
+    G = w.num_q_heads // w.num_kv_heads
+    R = w.stack * G
+    out = bufs.out.float().cpu().numpy().astype(np.float64)
+    lse = bufs.lse.cpu().numpy().astype(np.float64)
+    z = bufs.z.cpu().numpy().astype(np.float64)
+    status = bufs.row_status.cpu().numpy()
+    qa, qb, eta = split_queries(w, bufs)
+    units = units if units is not None else [(s, h) for s in range(w.num_seqs) for h in range(w.num_kv_heads)]
+    num = den = ynum = slack2 = 0.0
+    max_abs = vmax = dz = 0.0
+    rel_rows = []
+    n_live = n_ref = n_keys = 0
+    for (seq, kvh) in units:
+        n = int(w.seqlens[seq])
+        rows = [(seq * w.stack + r // G, kvh * G + r % G) for r in range(R)]
+        if n == 0:
+            for (b, h) in rows:
+                assert not out[b, h].any() and lse[b, h] == -np.inf and status[b, h] == F.ROW_EMPTY
+            continue
+        ka, kb, ke = logical_planes(w, cache, seq, kvh)
+        V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
+        Kx = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh)))
+        rqa = np.stack([qa[b, h] for (b, h) in rows]); rqb = np.stack([qb[b, h] for (b, h) in rows])
+        reta = np.array([eta[b, h] for (b, h) in rows], dtype=np.float64)
+        rz = np.array([z[b, h] for (b, h) in rows])
+        tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
+        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff)
+        n_live += int(info["live"].sum()); n_ref += int(info["refine"].sum()); n_keys += n
+        vinf = np.abs(V).max(axis=1)
+        near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
+        near_tau = (np.abs(info["coarse"] + tau_eff) <= BAND).any(axis=0) if 0 <= tau_eff < math.inf else np.zeros(n, bool)
+        for i, (b, h) in enumerate(rows):
+            o_ref = A[i] / L[i]
+            d = out[b, h] - o_ref
+            num += float(d @ d); den += float(o_ref @ o_ref)
+            max_abs = max(max_abs, float(np.abs(d).max())); vmax = max(vmax, float(vinf.max()))
+            rel_rows.append(np.linalg.norm(d) / max(np.linalg.norm(o_ref), 1e-300))
+            assert abs(lse[b, h] - (rz[i] + math.log2(L[i]))) <= LSE_TOL, (b, h)
+            if 0.5 <= L[i] <= 2.0 ** 100:
+                assert status[b, h] == 0, (b, h, status[b, h], L[i])
+            corr = P.refine_terms(kb, ke, rqa[i], rqb[i], reta[i])
+            s_fin = info["coarse"][i] + np.where(info["refine"], corr, 0.0)
+            p = np.exp2(s_fin)
+            if check_estimate:
+                dz = max(dz, abs(P.estimate_z_planes(ka, kb, ke, rqa[i], rqb[i], reta[i]) - z[b, h]))
+            if not math.isinf(T):
+                near = near_T | (np.abs(s_fin + T) <= BAND)
+                sl = float((p[near] * vinf[near]).sum() / L[i])
+                sl += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum() / L[i])
+                slack2 += sl ** 2 * V.shape[1]
+                o_dense = O.dense_row(O.scores(O.widen_bf16(bf16_bits(w.q[b, h])), Kx, w.scale), V)[0]
+                y = O.online_softmax_bf16(O.widen_bf16(bf16_bits(w.q[b, h])), Kx, V, w.scale) - o_dense
+                ynum += float(y @ y)
+    res = dict(rel_l2=math.sqrt(num / max(den, 1e-300)), max_abs=max_abs, vmax=vmax,
+               mean_rel=float(np.mean(rel_rows)) if rel_rows else 0.0, dz=dz,
+               live_frac=n_live / max(n_keys, 1), refine_frac=n_ref / max(n_keys, 1))
+    if math.isinf(T):
+        assert max_abs <= DENSE_MAX_ABS * vmax, res
+        assert res["mean_rel"] <= DENSE_MEAN_REL, res
+    else:
+        res["yard"] = math.sqrt(ynum / max(den, 1e-300)); res["slack"] = math.sqrt(slack2 / max(den, 1e-300))
+        assert res["rel_l2"] <= FINITE_T_FACTOR * res["yard"] + res["slack"] + 1e-12, res
+    if check_estimate:
+        assert dz <= Z_TOL, res
+    if check_counts and len(units) == w.num_seqs * w.num_kv_heads:
+        h = bufs.header()
+        assert h.v_rows_total == n_keys
+        assert abs(h.v_rows_fetched - n_live) <= max(2, 2e-3 * n_keys), (h.v_rows_fetched, n_live)
+        assert abs(h.k_rows_refined - n_ref) <= max(2, 2e-3 * n_keys), (h.k_rows_refined, n_ref)
+    return res
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("paged", [False, True])
+def test_cache_writer_and_query_split_match_the_oracle_bit_for_bit(D, paged):
+    w = make_decode_workload(3, 8, 2, D, [700, 64, 333], seed=41, device=DEV, paged=paged, page_size=32,
+                             poison_padding=True)
+    cache = plane_cache(w)
+    for seq in range(3):
+        for kvh in range(2):
+            a, b, e = logical_planes(w, cache, seq, kvh)
+            K = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh)))
+            ra, rb, re = P.quantize_rows(K)
+            assert np.array_equal(a, ra) and np.array_equal(b, rb) and np.array_equal(e, re)
+    bufs = run_planes(w, cache)
+    qa, qb, eta = split_queries(w, bufs)
+    q = O.widen_bf16(bf16_bits(w.q.reshape(-1, D))).reshape(3, 8, D)
+    ra, rb, re = P.quantize_rows(q)
+    assert np.array_equal(qa, ra) and np.array_equal(qb, rb)
+    assert np.array_equal(eta, (re * scale_log2_f32(w)).astype(np.float32))
+
+
+def test_appending_tokens_quantizes_only_the_new_rows():
+    w = make_decode_workload(2, 4, 2, 128, [500, 200], seed=43, device=DEV, capacity=640)
+    cache = plane_cache(w)
+    a0, b0, s0 = cache.k_plane_a.clone(), cache.k_plane_b.clone(), cache.k_scale.clone()
+    old = w.seqlens.clone()
+    w.seqlens += torch.tensor([3, 40], dtype=torch.int32, device=DEV)
+    w.max_seqlen = int(w.seqlens.max())
+    cache2 = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, None, None, cache.k_plane_a, cache.k_plane_b, cache.k_scale)
+    cache.k_plane_a[0, :500].fill_(77)                         # rows below first_token must not be rewritten
+    F.fold_quantize_keys(cache2, first_token=old)
+    torch.cuda.synchronize()
+    assert bool((cache.k_plane_a[0, :500] == 77).all())
+    cache.k_plane_a[0, :500] = a0[0, :500]
+    full = cache_of(w); F.fold_quantize_keys(full); torch.cuda.synchronize()
+    for seq, n in enumerate(w.seqlens.tolist()):
+        assert torch.equal(cache.k_plane_a[seq, :n], full.k_plane_a[seq, :n])
+        assert torch.equal(cache.k_plane_b[seq, :n], full.k_plane_b[seq, :n])
+        assert torch.equal(cache.k_scale[seq, :, :n], full.k_scale[seq, :, :n])
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 127, 128, 129, 255, 257, 1000])
+def test_edge_lengths(D, n):
+    w = make_decode_workload(2, 4, 2, D, [n, max(1, n - 17)], seed=200 + n, device=DEV, poison_padding=True,
+                             capacity=n + 70)
+    cache = plane_cache(w)
+    compare_planes(w, cache, run_planes(w, cache), check_estimate=True)
+    compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0)
+    compare_planes(w, cache, run_planes(w, cache, T=4.0, tau=2.0), T=4.0, tau=2.0)
+
+
+@pytest.mark.parametrize("Hq,Hkv,stack", [(1, 1, 1), (8, 8, 1), (4, 2, 1), (8, 1, 1), (8, 2, 2), (2, 2, 4), (3, 1, 2)])
+def test_group_and_stack_shapes(Hq, Hkv, stack):
+    w = make_decode_workload(2 * stack, Hq, Hkv, 128, [700, 300], seed=47, device=DEV, stack=stack)
+    cache = plane_cache(w)
+    compare_planes(w, cache, run_planes(w, cache))
+    compare_planes(w, cache, run_planes(w, cache, T=12.0), T=12.0)
+
+
+@pytest.mark.parametrize("page_size", [16, 32, 64, 128, 256])
+@pytest.mark.parametrize("D", [64, 128])
+def test_paged_layout_and_poisoned_tails(page_size, D):
+    w = make_decode_workload(3, 8, 2, D, [1500, 64, 333], seed=53, device=DEV, paged=True, page_size=page_size,
+                             poison_padding=True)
+    cache = plane_cache(w)
+    compare_planes(w, cache, run_planes(w, cache), check_estimate=True)
+    compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0)
+
+
+@pytest.mark.parametrize("tau", [-1.0, 3.0, 12.0, math.inf])
+def test_refine_gate_settings(tau):
+    w = make_decode_workload(2, 8, 2, 128, [3000, 1111], seed=59, device=DEV)
+    cache = plane_cache(w)
+    r = compare_planes(w, cache, run_planes(w, cache, tau=tau), tau=tau)
+    if tau < 0:
+        assert r["refine_frac"] == 0.0
+    if math.isinf(tau):
+        assert r["refine_frac"] == 1.0
+    if tau == 3.0:
+        assert 0.0 < r["refine_frac"] < 0.5
+    r = compare_planes(w, cache, run_planes(w, cache, T=10.0, tau=tau), T=10.0, tau=tau)
+    assert r["refine_frac"] <= r["live_frac"] < 1.0
+
+
+def test_long_context_several_chunks_and_two_plane_accuracy():
+    # > 8192 keys: 1024-key chunks; the two-plane dense result is also within the BF16 tolerances of EXACT attention
+    w = make_decode_workload(2, 8, 2, 128, [20000, 9001], seed=61, device=DEV)
+    cache = plane_cache(w)
+    units = [(0, 0), (1, 1)]
+    b = run_planes(w, cache, tau=math.inf)
+    compare_planes(w, cache, b, tau=math.inf, units=units, check_estimate=True)
+    out = b.out.float().cpu().numpy().astype(np.float64)
+    for (seq, kvh) in units:
+        K = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh))); V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
+        for g in range(4):
+            h = kvh * 4 + g
+            o = O.dense_row(O.scores(O.widen_bf16(bf16_bits(w.q[seq, h])), K, w.scale), V)[0]
+            assert np.linalg.norm(out[seq, h] - o) <= 1e-2 * np.linalg.norm(o)
+    compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0, units=units)
+
+
+def test_split_count_and_reference_modes():
+    w = make_decode_workload(2, 8, 2, 128, [9000, 2500], seed=67, device=DEV)
+    cache = plane_cache(w)
+    base = run_planes(w, cache, T=14.0)
+    for s in (1, 3, 9):
+        other = run_planes(w, cache, T=14.0, num_splits=s)
+        assert same_bits(base.out, other.out) and same_bits(base.lse, other.lse) and same_bits(base.z, other.z)
+    given = run_planes(w, cache, T=14.0, z_mode=F.Z_GIVEN, z=base.z)
+    assert same_bits(base.out, given.out) and same_bits(base.lse, given.lse)
+    compare_planes(w, cache, run_planes(w, cache, z_mode=F.Z_ZERO))
+    compare_planes(w, cache, run_planes(w, cache, z_mode=F.Z_GIVEN, z=base.lse + 30.0), check_counts=False)
+
+
+def test_empty_sequences_and_unsupported_shapes():
+    w = make_decode_workload(3, 4, 2, 128, [0, 500, 0], seed=71, device=DEV, capacity=512)
+    cache = plane_cache(w)
+    compare_planes(w, cache, run_planes(w, cache))
+    compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0)
+    wide = make_decode_workload(1, 16, 1, 128, [300], seed=73, device=DEV)              # 16 rows: beyond the two-plane scan
+    c2 = plane_cache(wide)
+    bufs = F.alloc_buffers(wide.q, cache_of(wide))
+    a = F.make_args(wide.q, c2, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse)
+    assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
+    a = F.make_args(w.q, cache, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, z_mode=F.Z_EXACT_MAX)
+    assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
+    torch.cuda.synchronize()
+
+
+def test_decode_without_the_bf16_keys_and_graph_replay():
+    w = make_decode_workload(2, 8, 2, 128, [4000, 1000], seed=79, device=DEV)
+    cache = plane_cache(w)
+    ref = run_planes(w, cache, T=16.0)
+    nok = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, None, None, cache.k_plane_a, cache.k_plane_b, cache.k_scale)
+    bufs = F.alloc_buffers(w.q, nok)
+    args = F.make_args(w.q, nok, depth_T=16.0, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse,
+                       row_status=bufs.row_status)
+    args.kv.k = None                                            # the planes are all the decode reads of the keys
+    F.fold_decode(args)
+    torch.cuda.synchronize()
+    assert same_bits(bufs.out, ref.out) and same_bits(bufs.lse, ref.lse)
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        F.fold_decode(args, s)
+        s.synchronize()
+        bufs.out.zero_()
+        with torch.cuda.graph(g, stream=s):
+            F.fold_decode(args, s)
+    g.replay()
+    torch.cuda.synchronize()
+    assert same_bits(bufs.out, ref.out) and same_bits(bufs.lse, ref.lse)
