@@ -307,6 +307,10 @@ def main():
                     help="verify a chain of this many draft tokens per sequence (stacked rows with ancestor masks)")
     ap.add_argument("--tail", action="store_true",
                     help="finite-depth steps use the block tail (cut keys add weight x block-mean value)")
+    ap.add_argument("--planes", action="store_true",
+                    help="keys as two INT8 planes + a BF16 scale per key (quantized once, outside the timed region)")
+    ap.add_argument("--refine-tau", type=float, default=0.0,
+                    help="--planes: the refine gate in binades (0 = max(log2(n) - 2, 4); inf = every live key; negative = none)")
     ap.add_argument("--graph", action="store_true",
                     help="capture one whole decode call in a CUDA graph and time its replays (single stream only)")
     ap.add_argument("--cascade-streams", type=int, default=1, choices=[1, 2],
@@ -365,6 +369,17 @@ def main():
             raise SystemExit("--tail: the block tail is built into the row-block scan only (no stacked prefix level)")
         F.fold_block_means(caches[0], stream)
         torch.cuda.synchronize()
+    quant_ms = None
+    if args.planes:
+        if cascade or args.drafts > 1 or args.tail:
+            raise SystemExit("--planes: flat decode only (no cascade, drafts or block tail)")
+        F.fold_quantize_keys(caches[0], None, stream)                   # allocates the planes, warms the kernel
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        F.fold_quantize_keys(caches[0], None, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        quant_ms = e0.elapsed_time(e1)
     lbufs = [F.alloc_buffers(l.q, c, l.stack) for l, c in zip(levels, caches)]
     bufs = lbufs[-1]
     cache_bytes = sum(l.cache_bytes() for l in levels)                    # unique bytes: a shared prefix counts once
@@ -374,7 +389,8 @@ def main():
         return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
                             num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
                             row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
-                            draft_len=args.drafts if args.drafts > 1 else 0) for l, c, b in zip(levels, caches, lbufs)]
+                            draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau)
+                for l, c, b in zip(levels, caches, lbufs)]
 
     # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
     # is scanned on a side stream while the suffix level is scanned on the main one (fork / join with events).
@@ -412,7 +428,7 @@ def main():
     def headers():
         hs = [b.header() for b in lbufs]
         return dict(fetched=[h.v_rows_fetched for h in hs], total=[h.v_rows_total for h in hs],
-                    timeouts=sum(h.wait_timeouts for h in hs))
+                    refined=[h.k_rows_refined for h in hs], timeouts=sum(h.wait_timeouts for h in hs))
 
     def timed(depth, steps, warmup, sample_clocks):
         # (1) whole steps: estimate -> scan(s) -> partial add, chained in the stream by one C-ABI call
@@ -472,8 +488,14 @@ def main():
     def fetched_frac(r):
         return sum(r["fetched"]) / max(sum(r["total"]), 1)
 
+    def refined_frac(r):
+        return sum(r["refined"]) / max(sum(r["total"]), 1)
+
     def actual_bytes(r):                                  # K in full + the fetched share of V + slots written, all levels
         # (from the fetched FRACTION: row groups of one kv head count their keys once each, but share the tiles in L2)
+        if args.planes:                                   # per key: plane A + scale, the refined share of plane B, the live share of V
+            keys = cache_bytes // (4 * D)
+            return int(keys * ((D + 2) + D * refined_frac(r) + 2 * D * fetched_frac(r))) + slot_bytes
         return cache_bytes // 2 + int(cache_bytes // 2 * fetched_frac(r)) + slot_bytes
 
     peak, peak_src = load_peaks()
@@ -481,7 +503,7 @@ def main():
     ach16 = actual_bytes(r16) / (r16["scan_ms"] * 1e-3) / 1e9
     achinf = actual_bytes(rinf) / (rinf["scan_ms"] * 1e-3) / 1e9
     scan_name = ("fold_scan_stacked_pair_kernel + fold_scan_gated_narrow_kernel (prefix + suffix levels)" if cascade
-                 else "fold_scan_gated_narrow_kernel")
+                 else "fold_scan_planes_kernel" if args.planes else "fold_scan_gated_narrow_kernel")
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
@@ -494,18 +516,25 @@ def main():
                    "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
                    "cascade_streams": args.cascade_streams if cascade else None,
                    "cuda_graph": bool(args.graph), "block_tail": bool(args.tail),
+                   "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16",
+                   "refine_tau": (args.refine_tau or "auto: max(log2(n) - 2, 4)") if args.planes else None,
                    "flat_equivalent_bytes_per_gpu": flat_bytes},
         "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
         "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},
         "kernel_ms": {"estimate": r16["est_ms"], "scan_T16": r16["scan_ms"], "scan_Tinf": rinf["scan_ms"],
                       "merge": r16["merge_ms"]},
         "v_rows_fetched_frac": {"T16": fetched_frac(r16), "Tinf": fetched_frac(rinf)},
+        "planes": None if not args.planes else {
+            "k_rows_refined_frac": {"T16": refined_frac(r16), "Tinf": refined_frac(rinf)},
+            "bytes_per_key": {"T16": (D + 2) + D * refined_frac(r16) + 2 * D * fetched_frac(r16),
+                              "Tinf": (D + 2) + D * refined_frac(rinf) + 2 * D * fetched_frac(rinf), "bf16_cache": 4 * D},
+            "cache_write_ms": quant_ms},
         "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
                      "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src,
-                     "traffic": None if cascade or args.workload != "c2" else NCU_TRAFFIC_PER_CACHE_BYTE["gated"] * cache_bytes,
+                     "traffic": None if cascade or args.planes or args.workload != "c2" else NCU_TRAFFIC_PER_CACHE_BYTE["gated"] * cache_bytes,
                      "traffic_source": "ncu dram__bytes_read+write of the same kernel captured on workload c2_small, scaled by units",
                      "algorithmic_bytes_per_launch": actual_bytes(r16),
-                     "dense": {"kernel": "fold_scan_dense_kernel (T=inf)" if not cascade else "fold_scan_stacked_pair_kernel + fold_scan_dense_kernel (T=inf)", "achieved": achinf, "frac": achinf / peak,
+                     "dense": {"kernel": "fold_scan_planes_kernel (T=inf)" if args.planes else "fold_scan_dense_kernel (T=inf)" if not cascade else "fold_scan_stacked_pair_kernel + fold_scan_dense_kernel (T=inf)", "achieved": achinf, "frac": achinf / peak,
                                "frac_of_nominal_8TBs": achinf / 8000.0,
                                "algorithmic_bytes_per_launch": actual_bytes(rinf)}},
         # estimate + scan (one per level) + partial add per timed step (the extra per-kernel pass is not timed)
@@ -513,7 +542,7 @@ def main():
         "clocks": r16["clocks"],
     }
 
-    if rank == 0 and not args.no_e2e and not cascade:
+    if rank == 0 and not args.no_e2e and not cascade and not args.planes:
         # end to end through the C ABI with HOST buffers: every step copies q and the whole cache
         # host -> device, decodes, and copies out / lse / status back
         hq, hk, hv = w.q.cpu().pin_memory(), w.k.cpu().pin_memory(), w.v.cpu().pin_memory()
@@ -549,7 +578,7 @@ def main():
                                "kind": "oracle",
                                "sample": f"{ob['units']} (sequence, kv head) units of {args.workload} "
                                          f"({ob['seconds']:.1f} s of float64 numpy; estimate + declared-Z row per q head)"}
-        if args.drafts <= 1 and not args.tail:
+        if args.drafts <= 1 and not args.tail and not args.planes:
             def run_once(depth):
                 step_whole(make(depth, F.Z_ESTIMATE))
                 torch.cuda.synchronize()

@@ -154,7 +154,8 @@ typedef struct fold_args {
   int32_t draft_len;                   /* 0..32 */
   float refine_tau;                    /* two-plane keys only: the refine gate tau_K of Algorithm 1, binades.  A live key
                                           reads plane B iff some row of its group has coarse weight >= 2^-refine_tau.
-                                          0 = choose: log2(n) + 7 for a sequence of n keys (its own length only);
+                                          0 = choose: max(log2(n) - 2, 4) for a sequence of n keys (its own length only:
+                                          a key is refined when some row gives it >= 4/n of the row's mass);
                                           INFINITY = every live key; negative = none (plane A scores only) */
 } fold_args;
 

@@ -495,8 +495,16 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   CUtensorMap ma;
   MapAxes axes;
   if (int rc = make_plane_map(&ma, &axes, kv, g.D, g.Hkv, box_tok)) return rc;
+  CUtensorMap mv;                                            // value rows of one 16-key sub-slice as a box
+  MapAxes vaxes;
+  if (int rc = make_map(&mv, &vaxes, kv.v, kv, g.D, g.Hkv, 16)) return rc;
   PlaneScanParams pp;
   memset(&pp, 0, sizeof(pp));
+  pp.vpos_tok = vaxes.pos_tok; pp.vpos_head = vaxes.pos_head; pp.vpos_seq = vaxes.pos_seq;
+  pp.box_min = 13;
+#ifdef FOLD_TUNING
+  if (const char *e = getenv("FOLD_TUNE_BOXMIN")) pp.box_min = atoi(e);
+#endif
   ScanParams &p = pp.s;
   p.z = a->z;
   p.seqlens = kv.seqlens;
@@ -523,7 +531,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   pp.auto_tau = a->refine_tau == 0.f;
   pp.neg_tau = a->refine_tau < 0.f ? INFINITY : -a->refine_tau;      // tau = inf -> -inf: every live key
   const dim3 grid(g.Hkv, p.num_splits, g.num_seqs);
-  const int per_cta2 = kSmemPerSm / 2 - kSmemCtaReserve;
+  const int per_cta2 = kSmemPerSm / kPlaneCtasPerSm - kSmemCtaReserve;
   int stages;
   static int cfg128[64] = {0}, cfg64[64] = {0};
   if (g.D == 128) {
@@ -533,7 +541,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
     if (stages < 2) return FOLD_EUNSUPPORTED;
     p.stages = stages;
     if (int rc = opt_in_smem(fold_scan_planes_kernel<128>, cfg128)) return rc;
-    if (launch_pdl(fold_scan_planes_kernel<128>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, pp) != cudaSuccess)
+    if (launch_pdl(fold_scan_planes_kernel<128>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) != cudaSuccess)
       return FOLD_ECUDA;
   } else {
     using LO = PlaneLayout<64>;
@@ -542,7 +550,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
     if (stages < 2) return FOLD_EUNSUPPORTED;
     p.stages = stages;
     if (int rc = opt_in_smem(fold_scan_planes_kernel<64>, cfg64)) return rc;
-    if (launch_pdl(fold_scan_planes_kernel<64>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, pp) != cudaSuccess)
+    if (launch_pdl(fold_scan_planes_kernel<64>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) != cudaSuccess)
       return FOLD_ECUDA;
   }
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;

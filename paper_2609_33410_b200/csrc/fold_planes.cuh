@@ -231,26 +231,34 @@ struct PlaneScanParams {
   PlaneView kv;
   const int8_t *qplanes;
   const float *qeta;
+  int vpos_tok, vpos_head, vpos_seq;                          // coordinate order of the value tensor map
+  int box_min;                                                // value rows of a sub-slice come as one box from this many live keys on
   float neg_tau;                                              // -tau_K; -inf: refine every live key; +inf: none
-  int auto_tau;                                               // tau_K = log2(n) + 7 from the sequence's own length
+  int auto_tau;                                               // tau_K = max(log2(n) - 2, 4) from the sequence's own length
 };
 
-constexpr int kPlaneTileKeys = 128;                           // keys per plane-A tile
-constexpr int kPlaneBufs = 2;                                 // gather buffers per warp (one in flight, one in use)
+// 64-key plane-A tiles (Algorithm 1's tile), two gather buffers per warp, three CTAs per SM: the kernel is bound by
+// its warps' instruction latencies, so more resident warps beat deeper rings (measured: 2 CTAs/SM 321 us, 3 CTAs/SM
+// 285 us on 16 x 8 x 32768 keys; a third gather buffer or 128-key tiles gain nothing).
+constexpr int kPlaneTileKeys = 64;                            // keys per plane-A tile
+constexpr int kPlaneBufs = 2;                                 // gather buffers per warp: kPlaneBufs - 1 sub-slices in flight
+constexpr int kPlaneCtasPerSm = 3;
 
 template <int D>
 struct PlaneLayout {
   static constexpr int kTK = kPlaneTileKeys;
   static constexpr int kATile = kTK * D;                      // plane A codes, swizzled as the tensor map writes them
   static constexpr int kStage = kATile + 1024;                // + the tile's scales (kTK * 2 bytes), 1 KB-aligned
-  static constexpr int kBBuf = 16 * D;                        // plane B rows of one 16-key sub-slice
+  static constexpr int kBBuf = 16 * D;                        // plane B rows of one 16-key sub-slice, swizzled like a tile
   static constexpr int kVBuf = 16 * D * 2;                    // value rows of one sub-slice, [D/64][16][128 B] swizzled
   static constexpr int kWarpBufs = kPlaneBufs * (kBBuf + kVBuf);
   __host__ __device__ static int off_bufs(int stages) { return stages * kStage; }
   // the chunk-end reduction parks in the gather buffers (drained by then): 4 warps x R x D floats <= 4 x kWarpBufs
   __host__ __device__ static int off_redl(int stages) { return off_bufs(stages) + kConsumerWarps * kWarpBufs; }
   __host__ __device__ static int off_bar(int stages) { return off_redl(stages) + kConsumerWarps * kMaxRows * 4; }
-  __host__ __device__ static int total(int stages) { return off_bar(stages) + 2 * stages * 8 + 1024; }
+  __host__ __device__ static int total(int stages) {
+    return off_bar(stages) + 2 * stages * 8 + kConsumerWarps * kPlaneBufs * 8 + 1024;
+  }
 };
 
 // Byte offset of 16-byte chunk `ch` of key row `key` in a tile of D-byte rows: the 128-byte swizzle for 128-byte
@@ -279,7 +287,8 @@ __device__ __forceinline__ void plane_products(uint32_t tile, int key0, int lane
 #pragma unroll
   for (int kk = 0; kk < D / 32; ++kk) {
     uint32_t a[4];
-    ldsm_x4(tile + plane_off<D>(key, 2 * kk + (lane >> 4)), a[0], a[1], a[2], a[3]);
+    const int ch = 2 * kk + (lane >> 4);
+    ldsm_x4(tile + plane_off<D>(key, ch), a[0], a[1], a[2], a[3]);
     mma_s8(ca, a, qa[kk][0], qa[kk][1]);
     mma_s8(cb, a, qb[kk][0], qb[kk][1]);
   }
@@ -334,12 +343,13 @@ struct PlanePending {
   float x[4];            // coarse score minus reference: key lane/4 (+8), rows (lane%4)*2 + {0,1}; -inf if unused
   float e[2];            // the two keys' scales
   uint32_t live, refine; // verdict bits of the 16 keys, ORed over the rows
-  int buf;
+  int buf;               // the gather buffer its rows land in
 };
 
 template <int D>
-__global__ void __launch_bounds__(kDenseThreads, 2)
-fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const PlaneScanParams pp) {
+__global__ void __launch_bounds__(kDenseThreads, kPlaneCtasPerSm)
+fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmV,
+                        const PlaneScanParams pp) {
   using LO = PlaneLayout<D>;
   constexpr int TK = LO::kTK, U = TK / (16 * kConsumerWarps);          // sub-slices per warp and tile
   constexpr int CV = D / 8, CB = D / 16;                               // 16-byte chunks per value row / plane row
@@ -355,12 +365,14 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const PlaneScan
   if (split >= w.n_chunks) return;
   const int stages = p.stages, R = p.R, n = w.n;
   const uint32_t full0 = base + LO::off_bar(stages), empty0 = full0 + 8u * stages;
+  const uint32_t gbar0 = empty0 + 8u * stages;               // one barrier per (warp, gather buffer)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(full0 + 8u * s, 1);
       mbar_init(empty0 + 8u * s, kConsumerWarps);
     }
+    for (int i = 0; i < kConsumerWarps * kPlaneBufs; ++i) mbar_init(gbar0 + 8u * i, 1);
     mbar_fence_init();
   }
   __syncthreads();
@@ -398,7 +410,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const PlaneScan
     zr[e] = rv[e] ? p.z[row] : 0.f;
   }
   const float neg_T = p.neg_T;
-  const float neg_tau = pp.auto_tau ? -(log2f((float)max(n, 1)) + 7.f) : pp.neg_tau;
+  const float neg_tau = pp.auto_tau ? -fmaxf(log2f((float)max(n, 1)) - 2.f, 4.f) : pp.neg_tau;
 
   float o[D / 16][4];
 #pragma unroll
@@ -408,21 +420,28 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const PlaneScan
   float *red = reinterpret_cast<float *>(gen + LO::off_bufs(stages));
   float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages));
   const int klo = lane >> 2;
+  const uint32_t gbar_w = gbar0 + 8u * (warp * kPlaneBufs);
+  bool dead = false;
 
+  uint32_t gphase = 0;                                       // bit b: parity of buffer b's next completed phase
   // second pass of a sub-slice: plane B product, final weights, value product
   auto finish = [&](const PlanePending &pd) {
     const uint32_t bbuf = bufs + pd.buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
+    const bool landed = mbar_wait(gbar_w + 8u * pd.buf, (gphase >> pd.buf) & 1u, dead);
+    gphase ^= 1u << pd.buf;
+    if (!landed) return;
     int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
-    if (pd.refine) plane_products<D>(bbuf, 0, lane, qa, qb, ca, cb);      // unrefined keys' rows were zero-filled
+    if (pd.refine) plane_products<D>(bbuf, 0, lane, qa, qb, ca, cb);
     uint32_t bh[2], bl[2];
 #pragma unroll
     for (int kh = 0; kh < 2; ++kh) {
       const bool klive = (pd.live >> (klo + 8 * kh)) & 1u;
+      const bool kref = (pd.refine >> (klo + 8 * kh)) & 1u;   // an unrefined key's buffer row is stale: no correction
       float pw[2], pm[2];
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const int i = 2 * kh + e;
-        const float corr = ((float)ca[i] + (float)cb[i] * 0.00390625f) * 0.00390625f;
+        const float corr = kref ? ((float)ca[i] + (float)cb[i] * 0.00390625f) * 0.00390625f : 0.f;
         const float x = fmaf(corr, eta[e] * pd.e[kh], pd.x[i]);
         const bool live = klive && (x >= neg_T);
         pw[e] = ex2_approx(x);
@@ -440,12 +459,12 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const PlaneScan
     if (pd.live) value_product_n<D, true, 0, 16>(o, vbuf, 0, lane, bh, bl);
   };
 
-  bool dead = false, have = false;
-  int stage = 0, buf = 0;
+  int stage = 0, buf = 0, n_pend = 0;
   uint32_t phase = 0;
   unsigned long long st_total = 0, st_live = 0, st_ref = 0;
-  PlanePending pend;
+  PlanePending pend[kPlaneBufs - 1];
   const int page_mask = (1 << p.page_shift) - 1;
+  const uint64_t vpol = policy_evict_first();
 
   for (int c = split; c < w.n_chunks; c += p.num_splits) {
     const int t_end = min((c + 1) * w.ctiles, w.n_tiles);
@@ -487,52 +506,73 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const PlaneScan
         cur.buf = buf;
         st_live += __popc(cur.live);
         st_ref += __popc(cur.refine);
-        // only now are bytes requested: plane B rows of refined keys, value rows of live keys (others zero-filled)
+        // only now are bytes requested: plane B rows of refined keys, value rows of live keys.  A sub-slice with (nearly)
+        // every key live takes its value rows as one tensor-map box; otherwise rows are copied one by one, the
+        // others zero-filled (their weight is 0, and the buffer may hold anything).  Plane B rows of unrefined keys are
+        // not touched: their correction is masked in registers.
         __syncwarp();                                         // the buffer's last readers are done
-        const uint32_t bbuf = bufs + buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
-        if (cur.live) {
-          long long s_row = seq, t_row = key0;
-          if (p.paged) {
-            s_row = min(max(p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)], 0), p.num_pages - 1);
-            t_row = key0 & page_mask;
-          }
-          if (cur.refine) {
-            const int8_t *src0 = pp.kv.b + s_row * pp.kv.stride_seq + t_row * pp.kv.stride_tok + (long long)kvh * pp.kv.stride_head;
-#pragma unroll
-            for (int i = 0; i < CB / 2; ++i) {
-              const int cidx = lane + 32 * i, key = cidx / CB, ch = cidx % CB;
-              const bool f = (cur.refine >> key) & 1u;
-              cp_async_16(bbuf + plane_off<D>(key, ch), f ? src0 + (long long)key * pp.kv.stride_tok + ch * 16 : pp.kv.b, f ? 16u : 0u);
+        {
+          const uint32_t bbuf = bufs + buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
+          const uint32_t gbar = gbar_w + 8u * buf;
+          if (cur.live) {
+            long long s_row = seq, t_row = key0;
+            if (p.paged) {
+              s_row = min(max(p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)], 0), p.num_pages - 1);
+              t_row = key0 & page_mask;
             }
-          }
-          const __nv_bfloat16 *v0 = p.v + s_row * p.v_stride_seq + t_row * p.v_stride_tok + (long long)kvh * p.v_stride_head;
+            const bool box = __popc(cur.live) >= pp.box_min && key0 + 16 <= n;
+            if (box) {
+              fence_proxy_async_smem();                       // the buffer's earlier generic-proxy traffic, then TMA writes
+              __syncwarp();
+              if (lane == 0) {
+                mbar_expect_tx_only(gbar, 16 * D * 2);
+                const int c_seq = (int)s_row, c_tok = (int)t_row;
+                const int c1 = pp.vpos_tok == 1 ? c_tok : (pp.vpos_head == 1 ? kvh : c_seq);
+                const int c2 = pp.vpos_tok == 2 ? c_tok : (pp.vpos_head == 2 ? kvh : c_seq);
+                const int c3 = pp.vpos_tok == 3 ? c_tok : (pp.vpos_head == 3 ? kvh : c_seq);
 #pragma unroll
-          for (int i = 0; i < CV / 2; ++i) {
-            const int cidx = lane + 32 * i, key = cidx / CV, ch = cidx % CV;
-            const bool f = (cur.live >> key) & 1u;
-            cp_async_16(vbuf + (ch >> 3) * (16 * 128) + key * 128 + (((ch & 7) ^ (key & 7)) << 4),
-                        f ? v0 + (long long)key * p.v_stride_tok + ch * 8 : p.v, f ? 16u : 0u);
+                for (int h = 0; h < D / 64; ++h) tma_load_4d(vbuf + h * (16 * 128), &tmV, gbar, h * 64, c1, c2, c3, vpol);
+              }
+            } else {
+              const __nv_bfloat16 *v0 = p.v + s_row * p.v_stride_seq + t_row * p.v_stride_tok + (long long)kvh * p.v_stride_head;
+#pragma unroll
+              for (int i = 0; i < CV / 2; ++i) {
+                const int cidx = lane + 32 * i, key = cidx / CV, ch = cidx % CV;
+                const bool f = (cur.live >> key) & 1u;
+                cp_async_16(vbuf + (ch >> 3) * (16 * 128) + key * 128 + (((ch & 7) ^ (key & 7)) << 4),
+                            f ? v0 + (long long)key * p.v_stride_tok + ch * 8 : p.v, f ? 16u : 0u);
+              }
+            }
+            if (cur.refine) {
+              const int8_t *src0 = pp.kv.b + s_row * pp.kv.stride_seq + t_row * pp.kv.stride_tok + (long long)kvh * pp.kv.stride_head;
+#pragma unroll
+              for (int i = 0; i < CB / 2; ++i) {
+                const int cidx = lane + 32 * i, key = cidx / CB, ch = cidx % CB;
+                if ((cur.refine >> key) & 1u)
+                  cp_async_16(bbuf + plane_off<D>(key, ch), src0 + (long long)key * pp.kv.stride_tok + ch * 16, 16u);
+              }
+            }
+            if (!box || cur.refine) cp_async_mbar_arrive(gbar);   // this lane's copies hold the phase open
+            __syncwarp();
           }
+          if (lane == 0) mbar_arrive(gbar);
         }
-        cp_async_commit();
-        if (have) {                                           // the sub-slice before this one: its rows have landed
-          cp_async_wait<1>();
-          __syncwarp();
-          finish(pend);
-        }
-        pend = cur;
-        have = true;
-        buf ^= 1;
+        // with every buffer now taken, the oldest sub-slice in flight is finished while the newest one's rows travel
+        // (the queue is kept at the tail of pend[], so every index is a constant and the entries stay in registers)
+        if (n_pend == kPlaneBufs - 1) finish(pend[0]);
+        else ++n_pend;
+#pragma unroll
+        for (int i = 0; i + 1 < kPlaneBufs - 1; ++i) pend[i] = pend[i + 1];
+        pend[kPlaneBufs - 2] = cur;
+        buf = buf + 1 == kPlaneBufs ? 0 : buf + 1;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);     // plane A and the scales are no longer needed
     }
-    if (have) {
-      cp_async_wait<0>();
-      __syncwarp();
-      finish(pend);
-      have = false;
-    }
+#pragma unroll
+    for (int i = 0; i < kPlaneBufs - 1; ++i)
+      if (i >= kPlaneBufs - 1 - n_pend) finish(pend[i]);
+    n_pend = 0;
     named_bar(1, kConsumerWarps * 32);                        // every warp's buffers are drained: park there
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
     reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);

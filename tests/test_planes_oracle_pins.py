@@ -209,7 +209,7 @@ def test_verdicts_are_ored_over_the_group_but_weights_are_cut_per_row():
 
 
 def test_auto_refine_gate_follows_the_request_length_only():
-    assert P.auto_refine_tau(1024) == 17.0 and P.auto_refine_tau(32768) == 22.0
+    assert P.auto_refine_tau(1024) == 8.0 and P.auto_refine_tau(32768) == 13.0 and P.auto_refine_tau(16) == 4.0
     assert P.auto_refine_tau(2048) - P.auto_refine_tau(1024) == 1.0
 
 
