@@ -423,6 +423,14 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   const uint32_t gbar_w = gbar0 + 8u * (warp * kPlaneBufs);
   bool dead = false;
 
+  // The buffers must never hold bit patterns that read as non-finite BF16: zero them before the first rows land and
+  // after the chunk-end reduction has parked FP32 partials in them.
+  auto clear_bufs = [&]() {
+    for (int i = lane; i < LO::kWarpBufs / 16; i += 32)
+      *reinterpret_cast<uint4 *>(gen + LO::off_bufs(stages) + warp * LO::kWarpBufs + i * 16) = make_uint4(0, 0, 0, 0);
+    __syncwarp();
+  };
+  clear_bufs();
   uint32_t gphase = 0;                                       // bit b: parity of buffer b's next completed phase
   // second pass of a sub-slice: plane B product, final weights, value product
   auto finish = [&](const PlanePending &pd) {
@@ -507,9 +515,9 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         st_live += __popc(cur.live);
         st_ref += __popc(cur.refine);
         // only now are bytes requested: plane B rows of refined keys, value rows of live keys.  A sub-slice with (nearly)
-        // every key live takes its value rows as one tensor-map box; otherwise rows are copied one by one, the
-        // others zero-filled (their weight is 0, and the buffer may hold anything).  Plane B rows of unrefined keys are
-        // not touched: their correction is masked in registers.
+        // every key live takes its value rows as one tensor-map box; otherwise the live rows are copied one by one.
+        // A row that is not fetched keeps what the buffer held -- zeros or an earlier value row, finite either way,
+        // times a weight of exactly 0; an unrefined key's plane B row likewise, its correction masked in registers.
         __syncwarp();                                         // the buffer's last readers are done
         {
           const uint32_t bbuf = bufs + buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
@@ -534,22 +542,29 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 for (int h = 0; h < D / 64; ++h) tma_load_4d(vbuf + h * (16 * 128), &tmV, gbar, h * 64, c1, c2, c3, vpol);
               }
             } else {
-              const __nv_bfloat16 *v0 = p.v + s_row * p.v_stride_seq + t_row * p.v_stride_tok + (long long)kvh * p.v_stride_head;
+              // lane -> chunk lane % CV of keys lane / CV, + 32 / CV, ...: one pointer step per copy
+              constexpr int VK = 32 / CV;
+              const int ch = lane % CV, k0 = lane / CV;
+              const __nv_bfloat16 *src = p.v + s_row * p.v_stride_seq + (t_row + k0) * p.v_stride_tok +
+                                         (long long)kvh * p.v_stride_head + ch * 8;
+              const uint32_t dst = vbuf + (ch >> 3) * (16 * 128) + k0 * 128;
 #pragma unroll
-              for (int i = 0; i < CV / 2; ++i) {
-                const int cidx = lane + 32 * i, key = cidx / CV, ch = cidx % CV;
-                const bool f = (cur.live >> key) & 1u;
-                cp_async_16(vbuf + (ch >> 3) * (16 * 128) + key * 128 + (((ch & 7) ^ (key & 7)) << 4),
-                            f ? v0 + (long long)key * p.v_stride_tok + ch * 8 : p.v, f ? 16u : 0u);
+              for (int i = 0; i < 16 / VK; ++i) {
+                const int key = k0 + i * VK;
+                if ((cur.live >> key) & 1u) cp_async_16(dst + i * VK * 128 + (((ch & 7) ^ (key & 7)) << 4), src, 16u);
+                src += VK * p.v_stride_tok;
               }
             }
             if (cur.refine) {
-              const int8_t *src0 = pp.kv.b + s_row * pp.kv.stride_seq + t_row * pp.kv.stride_tok + (long long)kvh * pp.kv.stride_head;
+              constexpr int BK = 32 / CB;
+              const int ch = lane % CB, k0 = lane / CB;
+              const int8_t *src = pp.kv.b + s_row * pp.kv.stride_seq + (t_row + k0) * pp.kv.stride_tok +
+                                  (long long)kvh * pp.kv.stride_head + ch * 16;
 #pragma unroll
-              for (int i = 0; i < CB / 2; ++i) {
-                const int cidx = lane + 32 * i, key = cidx / CB, ch = cidx % CB;
-                if ((cur.refine >> key) & 1u)
-                  cp_async_16(bbuf + plane_off<D>(key, ch), src0 + (long long)key * pp.kv.stride_tok + ch * 16, 16u);
+              for (int i = 0; i < 16 / BK; ++i) {
+                const int key = k0 + i * BK;
+                if ((cur.refine >> key) & 1u) cp_async_16(bbuf + plane_off<D>(key, ch), src, 16u);
+                src += BK * pp.kv.stride_tok;
               }
             }
             if (!box || cur.refine) cp_async_mbar_arrive(gbar);   // this lane's copies hold the phase open
@@ -577,6 +592,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
     reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
     reduce_store_A_n<D, kConsumerWarps>(o, red, slot, R, warp, lane, threadIdx.x, 1);
+    if (c + p.num_splits < w.n_chunks) clear_bufs();
   }
 
   if (lane == 0) {

@@ -288,3 +288,33 @@ def test_decode_without_the_bf16_keys_and_graph_replay():
     g.replay()
     torch.cuda.synchronize()
     assert same_bits(bufs.out, ref.out) and same_bits(bufs.lse, ref.lse)
+
+
+def test_config2_full_size_two_plane_keys_sampled_units():
+    # the benchmark's workload (16 x 8 kv heads x 32768 keys, group 4) in the launch configuration bench.py --planes times
+    free, _ = torch.cuda.mem_get_info()
+    if free / 2 ** 30 < 14:
+        pytest.skip("not enough free device memory")
+    w = make_decode_workload(16, 32, 8, 128, 32768, seed=1, device=DEV)
+    cache = plane_cache(w)
+    units = [(0, 0), (7, 5), (15, 7)]
+    for seq, kvh in units[:2]:                                  # the writer at full size, bit for bit
+        a, b, e = logical_planes(w, cache, seq, kvh)
+        ra, rb, re = P.quantize_rows(O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh))))
+        assert np.array_equal(a, ra) and np.array_equal(b, rb) and np.array_equal(e, re)
+    b16 = run_planes(w, cache, T=16.0)
+    r = compare_planes(w, cache, b16, T=16.0, units=units, check_estimate=True)
+    assert 0.1 < r["refine_frac"] < 0.3 and r["live_frac"] > 0.9
+    assert same_bits(run_planes(w, cache, T=16.0, num_splits=8).out, b16.out)
+    compare_planes(w, cache, run_planes(w, cache), units=units)
+    del w, cache
+    torch.cuda.empty_cache()
+
+
+def test_head_dim_64_mha_long_rows_sampled_units():
+    w = make_decode_workload(4, 16, 16, 64, 32768, seed=83, device=DEV, paged=True, page_size=64)
+    cache = plane_cache(w)
+    units = [(0, 0), (3, 15)]
+    compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0, units=units, check_estimate=True)
+    compare_planes(w, cache, run_planes(w, cache, T=8.0), T=8.0, units=units)
+    compare_planes(w, cache, run_planes(w, cache), units=units)
