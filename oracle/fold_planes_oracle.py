@@ -19,7 +19,8 @@ What is here, with the passage each function restates (Section 4, "Cache format"
   plane_products      the four integer products c^aa, c^ab, c^ba, c^bb (exact)
   coarse_scores /
   refined_scores      Algorithm 1: eta e (c^aa + c^ab/256) and the plane-B correction, float64
-  auto_refine_tau     the refine gate when the caller gives none (a reading; see its docstring)
+  auto_refine_tau     the refine gate when the caller gives none.  PARITY UNPINNED by the paper (it
+                      gives no formula); the reading taken is in the docstring
   fold_group_planes   Algorithm 1 for one (sequence, kv head): verdict bits ORed over the
                       group's rows, final weights, (A, L) per row; also counts the bytes the
                       gates ask for (130 + 128 r_K + 256 lambda per key at D = 128)
