@@ -318,3 +318,39 @@ def test_head_dim_64_mha_long_rows_sampled_units():
     compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0, units=units, check_estimate=True)
     compare_planes(w, cache, run_planes(w, cache, T=8.0), T=8.0, units=units)
     compare_planes(w, cache, run_planes(w, cache), units=units)
+
+
+PLANE_LENGTHS = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 1000, 2047, 5000, 9000]
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_random_shapes_match_the_oracle(seed):
+    """Seeded random shapes of the two-plane path: head dimension, rows per kv head (1..8), lengths around every tile /
+    chunk / estimator boundary, paged or contiguous, depth and refine gate drawn together."""
+    import random
+    rnd = random.Random(7300 + seed)
+    for i in range(8):
+        D = rnd.choice([64, 128])
+        G, stack = rnd.choice([(1, 1), (2, 1), (3, 1), (4, 1), (8, 1), (5, 1), (1, 3), (2, 4), (4, 2), (1, 8), (2, 2)])
+        Hkv = rnd.choice([1, 2, 3])
+        nseq = rnd.choice([1, 2, 3])
+        lens = [rnd.choice(PLANE_LENGTHS) for _ in range(nseq)]
+        if max(lens) == 0:
+            lens[0] = 33
+        T = rnd.choice([math.inf, 16.0, 12.0, 8.0])
+        tau = rnd.choice([0.0, 0.0, -1.0, 3.0, 9.0, math.inf])
+        kw = dict(device=DEV, poison_padding=True)
+        if rnd.random() < 0.4:
+            kw.update(paged=True, page_size=rnd.choice([16, 32, 64, 128]))
+        else:
+            kw.update(capacity=max(lens) + rnd.choice([0, 5, 100]))
+        case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw)
+        w = make_decode_workload(nseq * stack, G * Hkv, Hkv, D, lens, seed=seed * 100 + i, stack=stack, **kw)
+        cache = plane_cache(w)
+        try:
+            b = run_planes(w, cache, T=T, tau=tau)
+            compare_planes(w, cache, b, T=T, tau=tau, check_estimate=True)
+            s = run_planes(w, cache, T=T, tau=tau, num_splits=rnd.choice([1, 2, 5]))
+            assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse), "split count changed a bit"
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: {e}") from e
