@@ -260,12 +260,14 @@ def run_sweep(args, dev):
                 cache = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table)
                 if args.tail:
                     F.fold_block_means(cache, stream)
+                if args.planes:                               # two INT8 key planes (+33 % device memory for the cell)
+                    F.fold_quantize_keys(cache, None, stream)
                 bufs = F.alloc_buffers(w.q, cache)
                 # small caches are L2-resident unless evicted: stream a 512 MB buffer between samples
                 flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if cache_bytes < 4 * 126e6 else None
                 for t_name, T in (("8", 8.0), ("16", 16.0), ("inf", math.inf)):
                     a = F.make_args(w.q, cache, scale=w.scale, z=bufs.z, depth_T=T, workspace=bufs.workspace,
-                                    out=bufs.out, lse=bufs.lse, row_status=bufs.row_status)
+                                    out=bufs.out, lse=bufs.lse, row_status=bufs.row_status, refine_tau=args.refine_tau)
                     for _ in range(3):
                         F.fold_decode(a, stream)
                     reps = 21 if cache_bytes < 2e9 else 7
@@ -283,13 +285,19 @@ def run_sweep(args, dev):
                     us = times[len(times) // 2]
                     h = bufs.header()
                     lam = h.v_rows_fetched / max(h.v_rows_total, 1)
+                    rk = h.k_rows_refined / max(h.v_rows_total, 1)
+                    # bytes read per key as a share of the BF16 cache's 4 D: K in full + the live share of V, or
+                    # plane A + scale + the refined share of plane B + the live share of V
+                    share = ((D + 2) + D * rk + 2 * D * lam) / (4 * D) if args.planes else 0.5 + 0.5 * lam
                     cells.append(dict(base, T=t_name, us=round(us, 1), us_min=round(times[0], 1),
                                       effective_gbs=round(cache_bytes / us / 1e3, 1),
-                                      actual_gbs=round(cache_bytes * (0.5 + 0.5 * lam) / us / 1e3, 1),
-                                      v_rows_fetched=round(lam, 4), l2_flush=flush is not None))
+                                      actual_gbs=round(cache_bytes * share / us / 1e3, 1),
+                                      v_rows_fetched=round(lam, 4), l2_flush=flush is not None,
+                                      **({"k_rows_refined": round(rk, 4)} if args.planes else {})))
                 del w, cache, bufs, flush
                 torch.cuda.empty_cache()
-    print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "block_tail": bool(args.tail), "drafts": args.drafts, "cells": cells}))
+    print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "block_tail": bool(args.tail), "drafts": args.drafts,
+                      "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16", "cells": cells}))
 
 
 def main():
