@@ -149,3 +149,50 @@ def test_no_device_means_a_loud_error_not_a_fallback():
     with pytest.raises(F.FoldError) as e:
         F.fold_decode(a, stream=0)
     assert e.value.status == F.FOLD_ECUDA
+
+
+def test_host_checks_of_two_plane_keys():
+    L = F.lib()
+    a, keep = _cpu_args()
+    plain = F.fold_workspace_bytes(a)
+    k = keep[1]
+    pa, pb = torch.zeros(k.shape, dtype=torch.int8), torch.zeros(k.shape, dtype=torch.int8)
+    sc = torch.zeros(k.shape[0], k.shape[2], 1024, dtype=torch.bfloat16)
+    a.kv.k_plane_a, a.kv.k_plane_b, a.kv.k_scale = pa.data_ptr(), pb.data_ptr(), sc.data_ptr()
+    a.kv.plane_stride_seq, a.kv.plane_stride_tok, a.kv.plane_stride_head = pa.stride(0), pa.stride(1), pa.stride(2)
+    a.kv.scale_stride_seq, a.kv.scale_stride_head = sc.stride(0), sc.stride(1)
+    # the workspace also holds the split query rows: [row][2][D] codes and one scale per row, each part 256-aligned
+    assert F.fold_workspace_bytes(a) == (plain + 255) // 256 * 256 + 2 * 8 * 2 * 128 + 256
+    ws = torch.zeros(F.fold_workspace_bytes(a) + 256, dtype=torch.uint8)
+    a.workspace = ws.data_ptr() + ((-ws.data_ptr()) % 256)
+    a.workspace_bytes = plain                                      # enough for BF16 keys, not for the planes
+    assert L.fold_decode(a, None) == F.FOLD_EWORKSPACE
+    a.workspace_bytes = ws.numel() - 256
+    for field, value, want in [("k_plane_b", None, F.FOLD_EINVAL), ("k_scale", None, F.FOLD_EINVAL),
+                               ("k_plane_a", pa.data_ptr() + 4, F.FOLD_EINVAL), ("plane_stride_tok", 100, F.FOLD_EINVAL),
+                               ("plane_stride_head", 72, F.FOLD_EINVAL), ("scale_stride_head", 1001, F.FOLD_EINVAL)]:
+        old = getattr(a.kv, field)
+        setattr(a.kv, field, value)
+        assert L.fold_decode(a, None) == want, field
+        setattr(a.kv, field, old)
+    a.refine_tau = float("nan")
+    assert L.fold_decode(a, None) == F.FOLD_EINVAL
+    a.refine_tau = 0.0
+    for field, value in [("z_mode", F.Z_EXACT_MAX), ("draft_len", 2), ("stack", 2)]:
+        old = getattr(a, field)
+        setattr(a, field, value)
+        if field == "draft_len":
+            masks = torch.ones(2, dtype=torch.int32); a.draft_mask = masks.data_ptr()
+        if field == "stack":                                        # 2 requests x group 4 on one sequence: 8 rows is the limit,
+            a.num_q_heads, a.num_kv_heads = 8, 1                    # 16 is beyond it
+            a.kv.num_seqs = 1
+        assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED, field
+        setattr(a, field, old)
+        a.draft_mask = None; a.num_q_heads, a.num_kv_heads = 8, 2; a.kv.num_seqs = 2
+    args2 = (F.FoldArgs * 2)(a, a)
+    ptrs = (C.POINTER(F.FoldArgs) * 2)(C.pointer(args2[0]), C.pointer(args2[1]))
+    assert L.fold_decode_cascade(ptrs, 2, None) == F.FOLD_EUNSUPPORTED     # two-plane keys: one level only
+    assert L.fold_quantize_keys(None, 2, 128, None, None) == F.FOLD_EINVAL
+    kv = F.FoldKV()
+    assert L.fold_quantize_keys(kv, 2, 96, None, None) == F.FOLD_EUNSUPPORTED
+    assert L.fold_quantize_keys(kv, 2, 128, None, None) == F.FOLD_EINVAL  # nothing to read or write
