@@ -377,12 +377,11 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   }
   __syncthreads();
   pdl_launch_dependents();
-  pdl_wait();                                                // z, the split query rows and the zeroed header
-
-  if (warp == kConsumerWarps) {
+  if (warp == kConsumerWarps) {                              // plane A and the scales depend on nothing the front kernel writes
     if (lane == 0) produce_plane_tiles<D>(&tmA, pp, w, split, kvh, seq, base, full0, empty0);
     return;
   }
+  pdl_wait();                                                // z and the split query rows come from the kernel before
 
   // query rows: B fragments of the INT8 products (row lane/4), scales and references of the score rows
   uint32_t qa[D / 32][2], qb[D / 32][2];

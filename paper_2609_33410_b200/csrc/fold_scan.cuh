@@ -619,12 +619,11 @@ fold_scan_dense_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
   }
   __syncthreads();
   pdl_launch_dependents();
-  pdl_wait();                                                // z (and the zeroed header) come from earlier work
-
-  if (warp == kConsumerWarps) {
+  if (warp == kConsumerWarps) {                              // the tiles depend on nothing the reference kernel writes:
     if (lane == 0) produce_tiles<D, true, LO::kStage, TK>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
-    return;
+    return;                                                  // the ring fills while that kernel drains
   }
+  pdl_wait();                                                // z comes from the kernel before
 
   RowBlockN<D> rb;                                           // rows on N: see "Narrow row blocks"
   load_rows_n<D>(rb, p, seq, kvh, lane);
@@ -727,12 +726,11 @@ fold_scan_dense_nt2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
   }
   __syncthreads();
   pdl_launch_dependents();
-  pdl_wait();                                                // z (and the zeroed header) come from earlier work
-
-  if (warp == kConsumerWarps) {
+  if (warp == kConsumerWarps) {                              // the tiles depend on nothing the reference kernel writes:
     if (lane == 0) produce_tiles<D, true, LO::kStage, TK>(&tmK, &tmV, p, w, split, kvh, seq, base, full0, empty0);
-    return;
+    return;                                                  // the ring fills while that kernel drains
   }
+  pdl_wait();                                                // z comes from the kernel before
 
   RowBlockN<D> rb[NT];
 #pragma unroll
@@ -978,12 +976,11 @@ fold_scan_gated_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __g
   }
   __syncthreads();
   pdl_launch_dependents();
-  pdl_wait();                                                // z (and the zeroed header) come from earlier work
-
-  if (warp == SW + kConsumerWarps) {
+  if (warp == SW + kConsumerWarps) {                         // the key tiles depend on nothing the reference kernel writes
     if (lane == 0) produce_tiles<D, false, LO::kKStage, TK, TAIL>(&tmK, &tmK, p, w, split, kvh, seq, base, full0, empty0);
     return;
   }
+  pdl_wait();                                                // z comes from the kernel before
 
   const bool scorer = warp < SW;
   const int sl = warp & 3;                                   // the slice of every tile this warp owns
