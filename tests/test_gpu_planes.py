@@ -354,3 +354,15 @@ def test_random_shapes_match_the_oracle(seed):
             assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse), "split count changed a bit"
         except AssertionError as e:
             raise AssertionError(f"case {case}: {e}") from e
+
+
+def test_static_scratch_entry_point_takes_two_plane_keys():
+    w = make_decode_workload(2, 8, 2, 128, [3000, 900], seed=89, device=DEV, paged=True, page_size=64)
+    cache = plane_cache(w)
+    ref = run_planes(w, cache, T=16.0)
+    out = torch.zeros_like(ref.out); lse = torch.zeros_like(ref.lse); z = torch.zeros_like(ref.z)
+    st = torch.zeros_like(ref.row_status)
+    args = F.make_args(w.q, cache, depth_T=16.0, z=z, out=out, lse=lse, row_status=st)       # no workspace
+    F.fold_decode_static(args)
+    torch.cuda.synchronize()
+    assert same_bits(out, ref.out) and same_bits(lse, ref.lse) and same_bits(z, ref.z) and not st.any()
