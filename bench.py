@@ -38,6 +38,8 @@ WORKLOADS = {
     "c3_small": dict(gen=dict(batch=1, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=131072, seed=2, paged=True,
                               page_size=64), T=16.0),
     "c2_small": dict(gen=dict(batch=4, num_q_heads=32, num_kv_heads=8, head_dim=128, seqlens=16384, seed=1), T=16.0),
+    # one small cell of the MHA sweep (configuration 5) at depth 8, for profiler captures
+    "c5_small": dict(gen=dict(batch=4, num_q_heads=32, num_kv_heads=32, head_dim=128, seqlens=32768, seed=5), T=8.0),
 }
 
 

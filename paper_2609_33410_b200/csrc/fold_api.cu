@@ -537,7 +537,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   if (g.D == 128) {
     using LO = PlaneLayout<128>;
     stages = (per_cta2 - LO::total(0)) / (LO::kStage + 16);
-    if (stages > 4) stages = 4;
+    if (stages > LO::kMaxStages) stages = LO::kMaxStages;
     if (stages < 2) return FOLD_EUNSUPPORTED;
     p.stages = stages;
     if (int rc = opt_in_smem(fold_scan_planes_kernel<128>, cfg128)) return rc;
@@ -546,7 +546,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   } else {
     using LO = PlaneLayout<64>;
     stages = (per_cta2 - LO::total(0)) / (LO::kStage + 16);
-    if (stages > 4) stages = 4;
+    if (stages > LO::kMaxStages) stages = LO::kMaxStages;
     if (stages < 2) return FOLD_EUNSUPPORTED;
     p.stages = stages;
     if (int rc = opt_in_smem(fold_scan_planes_kernel<64>, cfg64)) return rc;

@@ -248,11 +248,14 @@ template <int D>
 struct PlaneLayout {
   static constexpr int kTK = kPlaneTileKeys;
   static constexpr int kATile = kTK * D;                      // plane A codes, swizzled as the tensor map writes them
-  static constexpr int kStage = kATile + 1024;                // + the tile's scales (kTK * 2 bytes), 1 KB-aligned
+  static constexpr int kStage = kATile;                       // a ring stage (1 KB-aligned); the tiles' scales have a ring of their own
+  static constexpr int kScales = kTK * 2;                     // one tile's scales
+  static constexpr int kMaxStages = 8;
   static constexpr int kBBuf = 16 * D;                        // plane B rows of one 16-key sub-slice, swizzled like a tile
   static constexpr int kVBuf = 16 * D * 2;                    // value rows of one sub-slice, [D/64][16][128 B] swizzled
   static constexpr int kWarpBufs = kPlaneBufs * (kBBuf + kVBuf);
-  __host__ __device__ static int off_bufs(int stages) { return stages * kStage; }
+  __host__ __device__ static int off_scales(int stages) { return stages * kStage; }
+  __host__ __device__ static int off_bufs(int stages) { return off_scales(stages) + kMaxStages * kScales; }   // 1 KB-aligned
   // the chunk-end reduction parks in the gather buffers (drained by then): 4 warps x R x D floats <= 4 x kWarpBufs
   __host__ __device__ static int off_redl(int stages) { return off_bufs(stages) + kConsumerWarps * kWarpBufs; }
   __host__ __device__ static int off_bar(int stages) { return off_redl(stages) + kConsumerWarps * kMaxRows * 4; }
@@ -329,7 +332,7 @@ __device__ __forceinline__ void produce_plane_tiles(const CUtensorMap *tmA, cons
       const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
       tma_load_4d(dst + bx * p.box_tok * D, tmA, full, 0, c1, c2, c3, pol);
       const int cnt = min(p.box_tok, (w.n - j0 + 7) & ~7);
-      bulk_load(dst + LO::kATile + bx * p.box_tok * 2,
+      bulk_load(ring + LO::off_scales(p.stages) + stage * LO::kScales + bx * p.box_tok * 2,
                 pp.kv.scale + (long long)c_seq * pp.kv.sc_stride_seq + (long long)kvh * pp.kv.sc_stride_head + c_tok,
                 cnt * 2, full);
     }
@@ -481,7 +484,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       if (++stage == stages) { stage = 0; phase ^= 1u; }
       if (!ready) continue;
       const uint32_t at = base + my_stage * LO::kStage;
-      const __nv_bfloat16 *scales = reinterpret_cast<const __nv_bfloat16 *>(gen + my_stage * LO::kStage + LO::kATile);
+      const __nv_bfloat16 *scales = reinterpret_cast<const __nv_bfloat16 *>(gen + LO::off_scales(stages) + my_stage * LO::kScales);
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int sub = warp * U + u;                         // 16-key sub-slice of the tile
@@ -513,6 +516,16 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         cur.buf = buf;
         st_live += __popc(cur.live);
         st_ref += __popc(cur.refine);
+        if (cur.live == 0u) {
+          // every key of the sub-slice is cut for every row: no bytes are asked for, nothing is queued, and the weights
+          // (the coarse scores are all this scan will ever have for these keys) only add to L
+#pragma unroll
+          for (int kh = 0; kh < 2; ++kh) {
+            l_lo += ex2_approx(cur.x[2 * kh]);
+            l_hi += ex2_approx(cur.x[2 * kh + 1]);
+          }
+          continue;
+        }
         // only now are bytes requested: plane B rows of refined keys, value rows of live keys.  A sub-slice with (nearly)
         // every key live takes its value rows as one tensor-map box; otherwise the live rows are copied one by one.
         // A row that is not fetched keeps what the buffer held -- zeros or an earlier value row, finite either way,
