@@ -241,7 +241,6 @@ struct PlaneScanParams {
 // its warps' instruction latencies, so more resident warps beat deeper rings (measured: 2 CTAs/SM 321 us, 3 CTAs/SM
 // 285 us on 16 x 8 x 32768 keys; a third gather buffer or 128-key tiles gain nothing).
 constexpr int kPlaneTileKeys = 64;                            // keys per plane-A tile
-constexpr int kPlaneBufs = 2;                                 // gather buffers per warp: kPlaneBufs - 1 sub-slices in flight
 constexpr int kPlaneCtasPerSm = 3;
 
 template <int D>
@@ -253,14 +252,17 @@ struct PlaneLayout {
   static constexpr int kMaxStages = 8;
   static constexpr int kBBuf = 16 * D;                        // plane B rows of one 16-key sub-slice, swizzled like a tile
   static constexpr int kVBuf = 16 * D * 2;                    // value rows of one sub-slice, [D/64][16][128 B] swizzled
-  static constexpr int kWarpBufs = kPlaneBufs * (kBBuf + kVBuf);
+  // gather buffers per warp: kBufs - 1 sub-slices' rows in flight while one is multiplied (measured: three at D = 128
+  // cost a CTA per SM and lose; four at D = 64 fit and still lose -- there the instruction streams bind, not the rows in flight)
+  static constexpr int kBufs = 2;
+  static constexpr int kWarpBufs = kBufs * (kBBuf + kVBuf);
   __host__ __device__ static int off_scales(int stages) { return stages * kStage; }
   __host__ __device__ static int off_bufs(int stages) { return off_scales(stages) + kMaxStages * kScales; }   // 1 KB-aligned
   // the chunk-end reduction parks in the gather buffers (drained by then): 4 warps x R x D floats <= 4 x kWarpBufs
   __host__ __device__ static int off_redl(int stages) { return off_bufs(stages) + kConsumerWarps * kWarpBufs; }
   __host__ __device__ static int off_bar(int stages) { return off_redl(stages) + kConsumerWarps * kMaxRows * 4; }
   __host__ __device__ static int total(int stages) {
-    return off_bar(stages) + 2 * stages * 8 + kConsumerWarps * kPlaneBufs * 8 + 1024;
+    return off_bar(stages) + 2 * stages * 8 + kConsumerWarps * kBufs * 8 + 1024;
   }
 };
 
@@ -375,7 +377,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       mbar_init(full0 + 8u * s, 1);
       mbar_init(empty0 + 8u * s, kConsumerWarps);
     }
-    for (int i = 0; i < kConsumerWarps * kPlaneBufs; ++i) mbar_init(gbar0 + 8u * i, 1);
+    for (int i = 0; i < kConsumerWarps * LO::kBufs; ++i) mbar_init(gbar0 + 8u * i, 1);
     mbar_fence_init();
   }
   __syncthreads();
@@ -422,7 +424,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   float *red = reinterpret_cast<float *>(gen + LO::off_bufs(stages));
   float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages));
   const int klo = lane >> 2;
-  const uint32_t gbar_w = gbar0 + 8u * (warp * kPlaneBufs);
+  const uint32_t gbar_w = gbar0 + 8u * (warp * LO::kBufs);
   bool dead = false;
 
   // The buffers must never hold bit patterns that read as non-finite BF16: zero them before the first rows land and
@@ -472,7 +474,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   int stage = 0, buf = 0, n_pend = 0;
   uint32_t phase = 0;
   unsigned long long st_total = 0, st_live = 0, st_ref = 0;
-  PlanePending pend[kPlaneBufs - 1];
+  PlanePending pend[LO::kBufs - 1];
   const int page_mask = (1 << p.page_shift) - 1;
   const uint64_t vpol = policy_evict_first();
 
@@ -586,19 +588,19 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
         // with every buffer now taken, the oldest sub-slice in flight is finished while the newest one's rows travel
         // (the queue is kept at the tail of pend[], so every index is a constant and the entries stay in registers)
-        if (n_pend == kPlaneBufs - 1) finish(pend[0]);
+        if (n_pend == LO::kBufs - 1) finish(pend[0]);
         else ++n_pend;
 #pragma unroll
-        for (int i = 0; i + 1 < kPlaneBufs - 1; ++i) pend[i] = pend[i + 1];
-        pend[kPlaneBufs - 2] = cur;
-        buf = buf + 1 == kPlaneBufs ? 0 : buf + 1;
+        for (int i = 0; i + 1 < LO::kBufs - 1; ++i) pend[i] = pend[i + 1];
+        pend[LO::kBufs - 2] = cur;
+        buf = buf + 1 == LO::kBufs ? 0 : buf + 1;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8u * my_stage);     // plane A and the scales are no longer needed
     }
 #pragma unroll
-    for (int i = 0; i < kPlaneBufs - 1; ++i)
-      if (i >= kPlaneBufs - 1 - n_pend) finish(pend[i]);
+    for (int i = 0; i < LO::kBufs - 1; ++i)
+      if (i >= LO::kBufs - 1 - n_pend) finish(pend[i]);
     n_pend = 0;
     named_bar(1, kConsumerWarps * 32);                        // every warp's buffers are drained: park there
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
