@@ -125,43 +125,59 @@ EncodeTiledFn encode_fn() {
 }
 
 // 4-D view of a cache tensor: axis 0 is the channel, the token / head / sequence-or-page axes
-// follow in order of increasing stride (pos[] returns where each landed).  Box = 64 channels
-// x box_tok tokens, 128-byte swizzle, out-of-range elements read as zero.
+// follow in order of increasing stride (MapAxes returns where each landed).  Box = box_ch channels
+// x box_tok tokens, swizzled, out-of-range elements read as zero.
 struct MapAxes { int pos_tok, pos_head, pos_seq; };
 
-int make_map(CUtensorMap *map, MapAxes *axes, const void *ptr, const fold_kv &kv, int D, int Hkv, int box_tok) {
+// `elem` bytes per element (2: BF16 rows, 1: INT8 plane rows), strides in elements; the box spans `box_ch` channels.
+int make_map_of(CUtensorMap *map, MapAxes *axes, const void *ptr, const fold_kv &kv, int D, int Hkv, int box_tok, int elem,
+                long long stride_tok, long long stride_head, long long stride_seq, int box_ch, CUtensorMapSwizzle swizzle,
+                CUtensorMapL2promotion promo) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return FOLD_ECUDA;
   const bool paged = kv.page_table != nullptr;
   struct Axis { cuuint64_t extent, stride; cuuint32_t box; int id; };
-  Axis ax[3] = {{(cuuint64_t)(paged ? kv.page_size : kv.capacity), (cuuint64_t)kv.stride_tok * 2, (cuuint32_t)box_tok, 0},
-                {(cuuint64_t)Hkv, (cuuint64_t)kv.stride_head * 2, 1u, 1},
-                {(cuuint64_t)(paged ? kv.num_pages : kv.num_seqs), (cuuint64_t)kv.stride_seq * 2, 1u, 2}};
+  Axis ax[3] = {{(cuuint64_t)(paged ? kv.page_size : kv.capacity), (cuuint64_t)stride_tok * elem, (cuuint32_t)box_tok, 0},
+                {(cuuint64_t)Hkv, (cuuint64_t)stride_head * elem, 1u, 1},
+                {(cuuint64_t)(paged ? kv.num_pages : kv.num_seqs), (cuuint64_t)stride_seq * elem, 1u, 2}};
   // extent-1 axes carry no information: sort them last, the rest by stride
   for (int i = 0; i < 3; ++i)
     for (int j = i + 1; j < 3; ++j) {
       const bool i_one = ax[i].extent == 1, j_one = ax[j].extent == 1;
       if ((i_one && !j_one) || (i_one == j_one && ax[j].stride < ax[i].stride)) { Axis t = ax[i]; ax[i] = ax[j]; ax[j] = t; }
     }
-  cuuint64_t prev_stride = (cuuint64_t)D * 2, prev_extent = 1;
+  cuuint64_t prev_stride = (cuuint64_t)D * elem, prev_extent = 1;
   for (int i = 0; i < 3; ++i) {
     if (ax[i].extent == 1 || ax[i].stride == 0) ax[i].stride = prev_stride * prev_extent;
     prev_stride = ax[i].stride; prev_extent = ax[i].extent;
   }
   cuuint64_t dims[4] = {(cuuint64_t)D, ax[0].extent, ax[1].extent, ax[2].extent};
   cuuint64_t strides[3] = {ax[0].stride, ax[1].stride, ax[2].stride};
-  cuuint32_t box[4] = {64u, ax[0].box, ax[1].box, ax[2].box};
+  cuuint32_t box[4] = {(cuuint32_t)box_ch, ax[0].box, ax[1].box, ax[2].box};
   cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
   for (int i = 0; i < 3; ++i) {
     if (ax[i].id == 0) axes->pos_tok = i + 1;
     if (ax[i].id == 1) axes->pos_head = i + 1;
     if (ax[i].id == 2) axes->pos_seq = i + 1;
   }
-  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                   D == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+  CUresult rc = fn(map, elem == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
+                   const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promo,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? FOLD_OK : FOLD_ECUDA;
+}
+
+// BF16 key / value rows: a box of 64 channels x box_tok tokens, 128-byte swizzle.
+int make_map(CUtensorMap *map, MapAxes *axes, const void *ptr, const fold_kv &kv, int D, int Hkv, int box_tok) {
+  return make_map_of(map, axes, ptr, kv, D, Hkv, box_tok, 2, kv.stride_tok, kv.stride_head, kv.stride_seq, 64,
+                     CU_TENSOR_MAP_SWIZZLE_128B,
+                     D == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+}
+
+// Key plane A (INT8): one box spans the whole D-byte row; 128-byte swizzle for 128-byte rows, 64-byte for 64-byte rows.
+int make_plane_map(CUtensorMap *map, MapAxes *axes, const fold_kv &kv, int D, int Hkv, int box_tok) {
+  return make_map_of(map, axes, kv.k_plane_a, kv, D, Hkv, box_tok, 1, kv.plane_stride_tok, kv.plane_stride_head,
+                     kv.plane_stride_seq, D, D == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
 // ------------------------------------------------------------------ launches
@@ -451,39 +467,20 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   return (max_chunks + per - 1) / per;
 }
 
-// 4-D view of key plane A (INT8): axis 0 is the channel (one box spans the whole D-byte row), then token / head /
-// sequence-or-page by stride as in make_map.  128-byte swizzle for 128-byte rows, 64-byte swizzle for 64-byte rows.
-int make_plane_map(CUtensorMap *map, MapAxes *axes, const fold_kv &kv, int D, int Hkv, int box_tok) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return FOLD_ECUDA;
-  const bool paged = kv.page_table != nullptr;
-  struct Axis { cuuint64_t extent, stride; cuuint32_t box; int id; };
-  Axis ax[3] = {{(cuuint64_t)(paged ? kv.page_size : kv.capacity), (cuuint64_t)kv.plane_stride_tok, (cuuint32_t)box_tok, 0},
-                {(cuuint64_t)Hkv, (cuuint64_t)kv.plane_stride_head, 1u, 1},
-                {(cuuint64_t)(paged ? kv.num_pages : kv.num_seqs), (cuuint64_t)kv.plane_stride_seq, 1u, 2}};
-  for (int i = 0; i < 3; ++i)
-    for (int j = i + 1; j < 3; ++j) {
-      const bool i_one = ax[i].extent == 1, j_one = ax[j].extent == 1;
-      if ((i_one && !j_one) || (i_one == j_one && ax[j].stride < ax[i].stride)) { Axis t = ax[i]; ax[i] = ax[j]; ax[j] = t; }
-    }
-  cuuint64_t prev_stride = (cuuint64_t)D, prev_extent = 1;
-  for (int i = 0; i < 3; ++i) {
-    if (ax[i].extent == 1 || ax[i].stride == 0) ax[i].stride = prev_stride * prev_extent;
-    prev_stride = ax[i].stride; prev_extent = ax[i].extent;
-  }
-  cuuint64_t dims[4] = {(cuuint64_t)D, ax[0].extent, ax[1].extent, ax[2].extent};
-  cuuint64_t strides[3] = {ax[0].stride, ax[1].stride, ax[2].stride};
-  cuuint32_t box[4] = {(cuuint32_t)D, ax[0].box, ax[1].box, ax[2].box};
-  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  for (int i = 0; i < 3; ++i) {
-    if (ax[i].id == 0) axes->pos_tok = i + 1;
-    if (ax[i].id == 1) axes->pos_head = i + 1;
-    if (ax[i].id == 2) axes->pos_seq = i + 1;
-  }
-  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t *>(kv.k_plane_a), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, D == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return rc == CUDA_SUCCESS ? FOLD_OK : FOLD_ECUDA;
+// As many plane-A stages as fit beside the gather buffers with kPlaneCtasPerSm CTAs on an SM.
+template <int D>
+int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
+  using LO = PlaneLayout<D>;
+  const int per_cta = kSmemPerSm / kPlaneCtasPerSm - kSmemCtaReserve;
+  int stages = (per_cta - LO::total(0)) / (LO::kStage + 16);
+  if (stages > LO::kMaxStages) stages = LO::kMaxStages;
+  if (stages < 2) return FOLD_EUNSUPPORTED;
+  pp.s.stages = stages;
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_planes_kernel<D>, configured)) return rc;
+  if (launch_pdl(fold_scan_planes_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) != cudaSuccess)
+    return FOLD_ECUDA;
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
 // Two-plane keys: one kernel for dense and finite depth (the depth gate is a comparison against -T = -inf).
@@ -531,29 +528,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   pp.auto_tau = a->refine_tau == 0.f;
   pp.neg_tau = a->refine_tau < 0.f ? INFINITY : -a->refine_tau;      // tau = inf -> -inf: every live key
   const dim3 grid(g.Hkv, p.num_splits, g.num_seqs);
-  const int per_cta2 = kSmemPerSm / kPlaneCtasPerSm - kSmemCtaReserve;
-  int stages;
-  static int cfg128[64] = {0}, cfg64[64] = {0};
-  if (g.D == 128) {
-    using LO = PlaneLayout<128>;
-    stages = (per_cta2 - LO::total(0)) / (LO::kStage + 16);
-    if (stages > LO::kMaxStages) stages = LO::kMaxStages;
-    if (stages < 2) return FOLD_EUNSUPPORTED;
-    p.stages = stages;
-    if (int rc = opt_in_smem(fold_scan_planes_kernel<128>, cfg128)) return rc;
-    if (launch_pdl(fold_scan_planes_kernel<128>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) != cudaSuccess)
-      return FOLD_ECUDA;
-  } else {
-    using LO = PlaneLayout<64>;
-    stages = (per_cta2 - LO::total(0)) / (LO::kStage + 16);
-    if (stages > LO::kMaxStages) stages = LO::kMaxStages;
-    if (stages < 2) return FOLD_EUNSUPPORTED;
-    p.stages = stages;
-    if (int rc = opt_in_smem(fold_scan_planes_kernel<64>, cfg64)) return rc;
-    if (launch_pdl(fold_scan_planes_kernel<64>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) != cudaSuccess)
-      return FOLD_ECUDA;
-  }
-  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+  return g.D == 128 ? launch_planes_kernel<128>(ma, mv, pp, grid, st) : launch_planes_kernel<64>(ma, mv, pp, grid, st);
 }
 
 int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
