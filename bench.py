@@ -584,8 +584,16 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not cascade:
         wc = make_decode_workload(device="cpu", **dict(spec["gen"], batch=min(spec["gen"]["batch"], 2)))
         ob = bounded_oracle(wc, T)
+        one = None
+        try:                                              # the same oracle held to one thread, a shorter sample
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                o1 = bounded_oracle(wc, T, budget_s=5.0)
+            one = o1["bytes"] / o1["seconds"] / 1e9
+        except Exception:
+            pass
         out["cpu_baseline"] = {"value": ob["bytes"] / ob["seconds"] / 1e9, "unit": UNIT, "cores": ob["threads"],
-                               "kind": "oracle",
+                               "value_1_thread": one, "kind": "oracle",
                                "sample": f"{ob['units']} (sequence, kv head) units of {args.workload} "
                                          f"({ob['seconds']:.1f} s of float64 numpy; estimate + declared-Z row per q head)"}
         if args.drafts <= 1 and not args.tail and not args.planes:
