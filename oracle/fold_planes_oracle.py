@@ -137,13 +137,16 @@ def auto_refine_tau(n: int) -> float:
     return max(math.log2(max(n, 1)) - 2.0, 4.0)
 
 
-def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None):
+def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None, visible=None):
     """Algorithm 1 for the rows of one (sequence, kv head) group over all its keys.
     ka, kb [n, D] int8; ke [n]; V [n, D]; qa, qb [R, D] int8; eta [R]; Z [R] (binades).
     tau: refine gate in binades (None: auto_refine_tau(n); inf: refine every live key; negative:
     never).  Per key j:  live_j = OR_i [coarse_ij - Z_i >= -T];  refine_j = live_j AND
     OR_i [coarse_ij - Z_i >= -tau];  s_ij = coarse_ij (+ correction_ij if refine_j);  the weight
     2^(s_ij - Z_i) always adds to L_i and adds weight x value to A_i iff live_j and s_ij - Z_i >= -T.
+    visible [R, n] bool (drafts and verification trees, Section 4 "Value product": extra query rows masked to
+    their ancestors): a key a row does not see has coarse score -inf for that row -- weight exactly 0, and no
+    say in the verdicts.
     Returns (A [R, D], L [R], info) with info = live / refine masks and the bytes-per-key count."""
     ka = np.asarray(ka); kb = np.asarray(kb)
     V = np.asarray(V, dtype=np.float64)
@@ -152,7 +155,9 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
     if tau is None:
         tau = auto_refine_tau(n)
     coarse = np.stack([coarse_scores(ka, ke, qa[i], qb[i], eta[i]) - Z[i] for i in range(R)])      # [R, n]
-    live = np.ones(n, dtype=bool) if math.isinf(T) else (coarse >= -T).any(axis=0)
+    if visible is not None:
+        coarse = np.where(np.asarray(visible, dtype=bool), coarse, -np.inf)
+    live = np.isfinite(coarse).any(axis=0) if math.isinf(T) else (coarse >= -T).any(axis=0)
     refine = live & ((coarse >= -tau).any(axis=0) if tau >= 0 else np.zeros(n, dtype=bool))
     A = np.zeros((R, D)); L = np.zeros(R)
     for i in range(R):

@@ -99,8 +99,8 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   g->ws_bytes = g->planes ? g->q_off + qplane_bytes((long long)g->B * g->Hq, g->D) : kHeaderBytes + g->slot_bytes;
   if (g->planes) {
     if (isnan(a->refine_tau)) return FOLD_EINVAL;
-    // the two-plane scan: one 8-row block, no drafts, no block tail, no exact-maximum pass
-    if (R > kNarrowRows || a->draft_len > 0 || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
+    // the two-plane scan: one 8-row block, no block tail, no exact-maximum pass
+    if (R > kNarrowRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
     if (a->kv.v_block_mean && !isinf(a->depth_T)) return FOLD_EUNSUPPORTED;
   }
   return FOLD_OK;
@@ -253,6 +253,8 @@ int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st) 
   p.write_z = a->z_mode == FOLD_Z_ESTIMATE;
   p.stack = g.stack; p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
+  p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
+  p.draft_len = a->draft_len;
   if (a->z_mode == FOLD_Z_ZERO) {
     const int rows = g.B * g.Hq;
     fold_fill_kernel<<<(rows + 255) / 256, 256, 0, st>>>(a->z, rows, 0.f);
@@ -476,10 +478,16 @@ int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScan
   if (stages > LO::kMaxStages) stages = LO::kMaxStages;
   if (stages < 2) return FOLD_EUNSUPPORTED;
   pp.s.stages = stages;
-  static int configured[64] = {0};
-  if (int rc = opt_in_smem(fold_scan_planes_kernel<D>, configured)) return rc;
-  if (launch_pdl(fold_scan_planes_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) != cudaSuccess)
-    return FOLD_ECUDA;
+  static int configured[2][64] = {{0}, {0}};
+  cudaError_t rc;
+  if (pp.s.draft_len > 0) {
+    if (int e = opt_in_smem(fold_scan_planes_kernel<D, true>, configured[1])) return e;
+    rc = launch_pdl(fold_scan_planes_kernel<D, true>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp);
+  } else {
+    if (int e = opt_in_smem(fold_scan_planes_kernel<D, false>, configured[0])) return e;
+    rc = launch_pdl(fold_scan_planes_kernel<D, false>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp);
+  }
+  if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
@@ -521,6 +529,8 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
   p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
   p.row_groups = 1;
+  p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
+  p.draft_len = a->draft_len;
   pp.kv = plane_view(kv);
   uint8_t *ws = static_cast<uint8_t *>(a->workspace);
   pp.qplanes = reinterpret_cast<const int8_t *>(ws + g.q_off);

@@ -156,6 +156,8 @@ struct FrontParams {
   PlaneView kv;
   int write_z, stack, Hq, Hkv, G;
   float scale_log2;
+  const uint32_t *draft_mask;                                  // drafts: the last draft_len keys are used by request req only
+  int draft_len;                                               // where its mask has the bit
 };
 constexpr int kFrontThreads = kEstSamples;                    // 192
 
@@ -215,6 +217,11 @@ __global__ void __launch_bounds__(kFrontThreads) fold_planes_front_kernel(const 
       }
       const float f = ((float)caa + (float)cab * 0.00390625f) + ((float)cba + (float)cbb * 0.00390625f) * 0.00390625f;
       sc[g][i] = f * (seta[g] * e);
+    }
+    if (p.draft_len) {                                         // a draft key the request does not use weighs nothing
+      const int t = est_sample_key(i, n) - (n - p.draft_len);
+      if (t >= 0 && t < 32 && !((p.draft_mask[req] >> t) & 1u))
+        for (int g = 0; g < G; ++g) sc[g][i] = -INFINITY;
     }
   }
   __syncthreads();
@@ -351,7 +358,8 @@ struct PlanePending {
   int buf;               // the gather buffer its rows land in
 };
 
-template <int D>
+// DRAFTS: the rows carry draft masks (a separate instantiation: the plain one is at its register limit).
+template <int D, bool DRAFTS>
 __global__ void __launch_bounds__(kDenseThreads, kPlaneCtasPerSm)
 fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmV,
                         const PlaneScanParams pp) {
@@ -404,15 +412,19 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     }
   }
   float eta[2], zr[2];
+  uint32_t dm[2];                                            // the rows' requests' draft masks (all ones without drafts)
   bool rv[2];
 #pragma unroll
   for (int e = 0; e < 2; ++e) {
     const int r = (lane & 3) * 2 + e;
     rv[e] = r < R;
-    const long long row = (long long)(seq * p.stack + r / p.G) * p.Hq + kvh * p.G + r % p.G;
+    const int req = seq * p.stack + r / p.G;
+    const long long row = (long long)req * p.Hq + kvh * p.G + r % p.G;
     eta[e] = rv[e] ? pp.qeta[row] : 0.f;
     zr[e] = rv[e] ? p.z[row] : 0.f;
+    dm[e] = (DRAFTS && rv[e]) ? p.draft_mask[req] : 0xffffffffu;
   }
+  const int dstart = DRAFTS ? draft_start(p, n) : n;         // keys from here on are per-request drafts
   const float neg_T = p.neg_T;
   const float neg_tau = pp.auto_tau ? -fmaxf(log2f((float)max(n, 1)) - 2.f, 4.f) : pp.neg_tau;
 
@@ -505,7 +517,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             const int i = 2 * kh + e;
-            const bool ok = key < n && rv[e];
+            const bool ok = key < n && rv[e] && (!DRAFTS || draft_ok(dm[e], key, dstart));   // an unused draft key: -inf
             const float f = (float)ca[i] + (float)cb[i] * 0.00390625f;
             const float x = ok ? fmaf(f, eta[e] * cur.e[kh], -zr[e]) : -INFINITY;
             cur.x[i] = x;

@@ -178,17 +178,15 @@ def test_host_checks_of_two_plane_keys():
     a.refine_tau = float("nan")
     assert L.fold_decode(a, None) == F.FOLD_EINVAL
     a.refine_tau = 0.0
-    for field, value in [("z_mode", F.Z_EXACT_MAX), ("draft_len", 2), ("stack", 2)]:
+    for field, value in [("z_mode", F.Z_EXACT_MAX), ("stack", 2)]:
         old = getattr(a, field)
         setattr(a, field, value)
-        if field == "draft_len":
-            masks = torch.ones(2, dtype=torch.int32); a.draft_mask = masks.data_ptr()
         if field == "stack":                                        # 2 requests x group 4 on one sequence: 8 rows is the limit,
             a.num_q_heads, a.num_kv_heads = 8, 1                    # 16 is beyond it
             a.kv.num_seqs = 1
         assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED, field
         setattr(a, field, old)
-        a.draft_mask = None; a.num_q_heads, a.num_kv_heads = 8, 2; a.kv.num_seqs = 2
+        a.num_q_heads, a.num_kv_heads = 8, 2; a.kv.num_seqs = 2
     args2 = (F.FoldArgs * 2)(a, a)
     ptrs = (C.POINTER(F.FoldArgs) * 2)(C.pointer(args2[0]), C.pointer(args2[1]))
     assert L.fold_decode_cascade(ptrs, 2, None) == F.FOLD_EUNSUPPORTED     # two-plane keys: one level only

@@ -29,6 +29,11 @@ def plane_cache(w):
     return cache
 
 
+def cache_after(w, cache):
+    """The same planes over the workload's (modified) BF16 tensors."""
+    return F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table, None, cache.k_plane_a, cache.k_plane_b, cache.k_scale)
+
+
 def logical_planes(w, cache, seq, kvh):
     """(a, b, e) of the logical keys of one (sequence, kv head), read back from the device planes."""
     n = int(w.seqlens[seq])
@@ -53,17 +58,20 @@ def split_queries(w, bufs):
     return codes[:, :, 0], codes[:, :, 1], eta
 
 
-def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0, z=None):
+def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, draft=None):
+    """`draft` = (masks int32 [batch], draft_len): draft / tree-verification rows."""
     bufs = F.alloc_buffers(w.q, cache, w.stack)
     if z is not None:
         bufs.z.copy_(z)
-    F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale, refine_tau=tau)
+    F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale, refine_tau=tau,
+             draft_mask=None if draft is None else draft[0], draft_len=0 if draft is None else draft[1])
     torch.cuda.synchronize()
     assert bufs.header().wait_timeouts == 0
     return bufs
 
 
-def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estimate=False, check_counts=True):
+def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estimate=False, check_counts=True, draft=None):
+    dmask = None if draft is None else [int(x) & 0xffffffff for x in draft[0].cpu().tolist()]
     G = w.num_q_heads // w.num_kv_heads
     R = w.stack * G
     out = bufs.out.float().cpu().numpy().astype(np.float64)
@@ -90,7 +98,8 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
         reta = np.array([eta[b, h] for (b, h) in rows], dtype=np.float64)
         rz = np.array([z[b, h] for (b, h) in rows])
         tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
-        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff)
+        vis = None if draft is None else np.stack([O.draft_visible(n, draft[1], dmask[b]) for (b, h) in rows])
+        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis)
         n_live += int(info["live"].sum()); n_ref += int(info["refine"].sum()); n_keys += n
         vinf = np.abs(V).max(axis=1)
         near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
@@ -108,14 +117,18 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
             s_fin = info["coarse"][i] + np.where(info["refine"], corr, 0.0)
             p = np.exp2(s_fin)
             if check_estimate:
-                dz = max(dz, abs(P.estimate_z_planes(ka, kb, ke, rqa[i], rqb[i], reta[i]) - z[b, h]))
+                s_all = P.refined_scores(ka, kb, ke, rqa[i], rqb[i], reta[i])
+                if vis is not None:
+                    s_all = np.where(vis[i], s_all, -np.inf)
+                dz = max(dz, abs(O.estimate_z(lambda idx: s_all[idx], n) - z[b, h]))
             if not math.isinf(T):
                 near = near_T | (np.abs(s_fin + T) <= BAND)
                 sl = float((p[near] * vinf[near]).sum() / L[i])
                 sl += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum() / L[i])
                 slack2 += sl ** 2 * V.shape[1]
-                o_dense = O.dense_row(O.scores(O.widen_bf16(bf16_bits(w.q[b, h])), Kx, w.scale), V)[0]
-                y = O.online_softmax_bf16(O.widen_bf16(bf16_bits(w.q[b, h])), Kx, V, w.scale) - o_dense
+                keep = slice(None) if vis is None else vis[i]
+                o_dense = O.dense_row(O.scores(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], w.scale), V[keep])[0]
+                y = O.online_softmax_bf16(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], V[keep], w.scale) - o_dense
                 ynum += float(y @ y)
     res = dict(rel_l2=math.sqrt(num / max(den, 1e-300)), max_abs=max_abs, vmax=vmax,
                mean_rel=float(np.mean(rel_rows)) if rel_rows else 0.0, dz=dz,
@@ -366,3 +379,22 @@ def test_static_scratch_entry_point_takes_two_plane_keys():
     F.fold_decode_static(args)
     torch.cuda.synchronize()
     assert same_bits(out, ref.out) and same_bits(lse, ref.lse) and same_bits(z, ref.z) and not st.any()
+
+
+@pytest.mark.parametrize("Hq,Hkv,m,tree", [(8, 2, 2, False), (4, 2, 4, True), (2, 2, 8, False), (3, 1, 2, True)])
+def test_draft_rows_on_two_plane_keys(Hq, Hkv, m, tree):
+    from paper_2609_33410_b200.workloads import make_draft_workload
+    w, masks, m = make_draft_workload(2, m, Hq, Hkv, 128, [700, 190], seed=97, device=DEV, tree=tree, poison_padding=True)
+    cache = plane_cache(w)
+    d = (masks, m)
+    b = run_planes(w, cache, draft=d)
+    compare_planes(w, cache, b, check_estimate=True, draft=d)
+    compare_planes(w, cache, run_planes(w, cache, T=12.0, draft=d), T=12.0, draft=d)
+    s = run_planes(w, cache, num_splits=1, draft=d)
+    assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse)
+    # a row's masked-out draft keys change nothing: flipping their value rows leaves that row's output bit-identical
+    keep = b.out.clone()
+    n0 = int(w.seqlens[0])
+    w.v[0, n0 - 1] = -w.v[0, n0 - 1]                            # the LAST draft key: row 0 of a chain / tree never uses it
+    again = run_planes(w, cache_after(w, cache), draft=d)
+    assert same_bits(again.out[0], keep[0])

@@ -222,3 +222,28 @@ def test_estimate_on_planes_is_the_plain_estimate_of_the_two_plane_scores():
     assert P.estimate_z_planes(ka, kb, ke, qa[0], qb[0], eta) == O.estimate_z(lambda i: s[i], n)
     short = P.estimate_z_planes(ka[:100], kb[:100], ke[:100], qa[0], qb[0], eta)
     assert abs(short - O.dense_row(s[:100], np.zeros((100, 1)))[1]) < 1e-12
+
+
+def test_rows_that_do_not_see_a_key_give_it_no_weight_and_no_vote():
+    # drafts / verification trees: a masked key is as good as absent for that row, and cannot make the key live
+    D, n = 64, 120
+    k = rng_rows(19, n, D); V = rng_rows(20, n, D); q = rng_rows(21, 2, D)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    Z = np.array([P.coarse_scores(ka, ke, qa[i], qb[i], eta[i]).max() for i in range(2)])
+    vis = np.ones((2, n), dtype=bool); vis[1, -7:] = False; vis[1, 3] = False
+    A, L, info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, math.inf, -1.0, visible=vis)
+    sub = vis[1]
+    A1, L1, _ = P.fold_group_planes(ka[sub], kb[sub], ke[sub], V[sub], qa[1:], qb[1:], eta[1:], Z[1:], math.inf, -1.0)
+    assert np.allclose(A[1], A1[0], rtol=1e-12) and np.isclose(L[1], L1[0], rtol=1e-12)
+    A0, L0, _ = P.fold_group_planes(ka, kb, ke, V, qa[:1], qb[:1], eta[:1], Z[:1], math.inf, -1.0)
+    assert np.allclose(A[0], A0[0], rtol=1e-12) and np.isclose(L[0], L0[0], rtol=1e-12)
+    # a key nobody sees is not live even in dense decode (its value row is never asked for)
+    vis[0, 5] = vis[1, 5] = False
+    info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, math.inf, -1.0, visible=vis)[2]
+    assert not info["live"][5] and info["live"].sum() == n - 1
+    # at finite depth a masked row has no vote: the key is live only through the rows that see it
+    T = 3.0
+    info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T, -1.0, visible=vis)[2]
+    own0 = np.where(vis[0], info["coarse"][0] >= -T, False); own1 = np.where(vis[1], info["coarse"][1] >= -T, False)
+    assert np.array_equal(info["live"], own0 | own1)
