@@ -98,8 +98,8 @@ enum {
  * capacity (page_size).  With planes, k may be NULL for the decode calls; v stays BF16.  Each scan scores every
  * key against plane A alone (head_dim + 2 bytes per key), ORs the verdicts over the rows that share the kv head,
  * and only then requests plane B rows (refined keys) and value rows (live keys).  This path takes row blocks of
- * at most 8 rows (stack * group <= 8, draft rows included), no block tail, one level (no cascade), and no
- * FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED. */
+ * at most 8 rows (stack * group <= 8, draft rows included) and one level (no cascade), with or without the block
+ * tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED. */
 typedef struct fold_kv {
   const void *k, *v;
   int64_t stride_seq, stride_tok, stride_head;   /* elements */

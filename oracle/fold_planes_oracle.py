@@ -137,7 +137,8 @@ def auto_refine_tau(n: int) -> float:
     return max(math.log2(max(n, 1)) - 2.0, 4.0)
 
 
-def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None, visible=None):
+def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None, visible=None,
+                      v_mean=None):
     """Algorithm 1 for the rows of one (sequence, kv head) group over all its keys.
     ka, kb [n, D] int8; ke [n]; V [n, D]; qa, qb [R, D] int8; eta [R]; Z [R] (binades).
     tau: refine gate in binades (None: auto_refine_tau(n); inf: refine every live key; negative:
@@ -147,6 +148,9 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
     visible [R, n] bool (drafts and verification trees, Section 4 "Value product": extra query rows masked to
     their ancestors): a key a row does not see has coarse score -inf for that row -- weight exactly 0, and no
     say in the verdicts.
+    v_mean [ceil(n/64), D] switches the block tail on (``fold_oracle.block_means``; Algorithm 1 "add the weights of
+    cut keys to the tile's virtual row"): a key whose weight row i does not keep in A adds weight x the mean value row
+    of its 64-key block to A_i instead of nothing.
     Returns (A [R, D], L [R], info) with info = live / refine masks and the bytes-per-key count."""
     ka = np.asarray(ka); kb = np.asarray(kb)
     V = np.asarray(V, dtype=np.float64)
@@ -166,6 +170,11 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
         keep = live if math.isinf(T) else (live & (s >= -T))
         L[i] = p.sum()
         A[i] = (p[keep, None] * V[keep]).sum(axis=0)
+        if v_mean is not None:
+            vm = np.asarray(v_mean, dtype=np.float64)
+            block_of = np.arange(n) // O.BLOCK_KEYS
+            for b in np.unique(block_of[~keep]):
+                A[i] = A[i] + p[~keep & (block_of == b)].sum() * vm[b]
     info = dict(live=live, refine=refine, coarse=coarse,
                 bytes_per_key=(D + 2) + D * float(refine.mean() if n else 0.0) + 2 * D * float(live.mean() if n else 0.0))
     return A, L, info

@@ -99,9 +99,8 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   g->ws_bytes = g->planes ? g->q_off + qplane_bytes((long long)g->B * g->Hq, g->D) : kHeaderBytes + g->slot_bytes;
   if (g->planes) {
     if (isnan(a->refine_tau)) return FOLD_EINVAL;
-    // the two-plane scan: one 8-row block, no block tail, no exact-maximum pass
+    // the two-plane scan: one 8-row block, no exact-maximum pass
     if (R > kNarrowRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
-    if (a->kv.v_block_mean && !isinf(a->depth_T)) return FOLD_EUNSUPPORTED;
   }
   return FOLD_OK;
 }
@@ -470,25 +469,26 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
 }
 
 // As many plane-A stages as fit beside the gather buffers with kPlaneCtasPerSm CTAs on an SM.
-template <int D>
-int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
-  using LO = PlaneLayout<D>;
+template <int D, bool DRAFTS, bool TAIL>
+int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
+  using LO = PlaneLayout<D, TAIL>;
   const int per_cta = kSmemPerSm / kPlaneCtasPerSm - kSmemCtaReserve;
   int stages = (per_cta - LO::total(0)) / (LO::kStage + 16);
   if (stages > LO::kMaxStages) stages = LO::kMaxStages;
   if (stages < 2) return FOLD_EUNSUPPORTED;
   pp.s.stages = stages;
-  static int configured[2][64] = {{0}, {0}};
-  cudaError_t rc;
-  if (pp.s.draft_len > 0) {
-    if (int e = opt_in_smem(fold_scan_planes_kernel<D, true>, configured[1])) return e;
-    rc = launch_pdl(fold_scan_planes_kernel<D, true>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp);
-  } else {
-    if (int e = opt_in_smem(fold_scan_planes_kernel<D, false>, configured[0])) return e;
-    rc = launch_pdl(fold_scan_planes_kernel<D, false>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp);
-  }
-  if (rc != cudaSuccess) return FOLD_ECUDA;
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_planes_kernel<D, DRAFTS, TAIL>, configured)) return rc;
+  if (launch_pdl(fold_scan_planes_kernel<D, DRAFTS, TAIL>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) !=
+      cudaSuccess)
+    return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+template <int D>
+int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
+  const bool drafts = pp.s.draft_len > 0, tail = pp.s.vmean != nullptr;      // (separate instantiations: registers)
+  if (drafts) return tail ? launch_planes_as<D, true, true>(ma, mv, pp, grid, st) : launch_planes_as<D, true, false>(ma, mv, pp, grid, st);
+  return tail ? launch_planes_as<D, false, true>(ma, mv, pp, grid, st) : launch_planes_as<D, false, false>(ma, mv, pp, grid, st);
 }
 
 // Two-plane keys: one kernel for dense and finite depth (the depth gate is a comparison against -T = -inf).
@@ -531,6 +531,10 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.row_groups = 1;
   p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
   p.draft_len = a->draft_len;
+  if (!isinf(a->depth_T)) {                                  // block tail: nothing is cut in dense decode
+    p.vmean = static_cast<const __nv_bfloat16 *>(kv.v_block_mean);
+    p.vm_stride_seq = kv.mean_stride_seq; p.vm_stride_block = kv.mean_stride_block; p.vm_stride_head = kv.mean_stride_head;
+  }
   pp.kv = plane_view(kv);
   uint8_t *ws = static_cast<uint8_t *>(a->workspace);
   pp.qplanes = reinterpret_cast<const int8_t *>(ws + g.q_off);

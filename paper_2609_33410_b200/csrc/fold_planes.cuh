@@ -250,13 +250,15 @@ struct PlaneScanParams {
 constexpr int kPlaneTileKeys = 64;                            // keys per plane-A tile
 constexpr int kPlaneCtasPerSm = 3;
 
-template <int D>
+// TAIL: the block tail's mean value rows (one per 64-key tile = block) ride along in a ring of stages + 1 slots.
+template <int D, bool TAIL = false>
 struct PlaneLayout {
   static constexpr int kTK = kPlaneTileKeys;
   static constexpr int kATile = kTK * D;                      // plane A codes, swizzled as the tensor map writes them
   static constexpr int kStage = kATile;                       // a ring stage (1 KB-aligned); the tiles' scales have a ring of their own
   static constexpr int kScales = kTK * 2;                     // one tile's scales
-  static constexpr int kMaxStages = 8;
+  static constexpr int kMeans = TAIL ? 1024 : 0;              // the mean ring: at most 1024 / (2 D) slots
+  static constexpr int kMaxStages = TAIL ? 1024 / (2 * D) - 1 : 8;
   static constexpr int kBBuf = 16 * D;                        // plane B rows of one 16-key sub-slice, swizzled like a tile
   static constexpr int kVBuf = 16 * D * 2;                    // value rows of one sub-slice, [D/64][16][128 B] swizzled
   // gather buffers per warp: kBufs - 1 sub-slices' rows in flight while one is multiplied (measured: three at D = 128
@@ -264,7 +266,8 @@ struct PlaneLayout {
   static constexpr int kBufs = 2;
   static constexpr int kWarpBufs = kBufs * (kBBuf + kVBuf);
   __host__ __device__ static int off_scales(int stages) { return stages * kStage; }
-  __host__ __device__ static int off_bufs(int stages) { return off_scales(stages) + kMaxStages * kScales; }   // 1 KB-aligned
+  __host__ __device__ static int off_means(int stages) { return off_scales(stages) + 1024; }                  // scales: <= 8 x 128 B
+  __host__ __device__ static int off_bufs(int stages) { return off_means(stages) + kMeans; }                 // 1 KB-aligned
   // the chunk-end reduction parks in the gather buffers (drained by then): 4 warps x R x D floats <= 4 x kWarpBufs
   __host__ __device__ static int off_redl(int stages) { return off_bufs(stages) + kConsumerWarps * kWarpBufs; }
   __host__ __device__ static int off_bar(int stages) { return off_redl(stages) + kConsumerWarps * kMaxRows * 4; }
@@ -307,16 +310,16 @@ __device__ __forceinline__ void plane_products(uint32_t tile, int key0, int lane
 }
 
 // Producer thread: plane A tiles by TMA, their scales by bulk copies, one stage per 128-key tile.
-template <int D>
+template <int D, bool TAIL>
 __device__ __forceinline__ void produce_plane_tiles(const CUtensorMap *tmA, const PlaneScanParams &pp, const SeqWork &w,
                                                     int split, int kvh, int seq, uint32_t ring, uint32_t full0,
                                                     uint32_t empty0) {
-  using LO = PlaneLayout<D>;
+  using LO = PlaneLayout<D, TAIL>;
   const ScanParams &p = pp.s;
   tma_prefetch_desc(tmA);
   const uint64_t pol = policy_evict_first();
   bool dead = false;
-  int stage = 0;
+  int stage = 0, mslot = 0;
   uint32_t wrapped = 0, phase = 0;
   const int boxes_per_tile = LO::kTK / p.box_tok;
   const int page_mask = (1 << p.page_shift) - 1;
@@ -327,8 +330,14 @@ __device__ __forceinline__ void produce_plane_tiles(const CUtensorMap *tmA, cons
     const uint32_t full = full0 + 8u * stage;
     int sc_tokens = 0;                                       // scale tokens copied: whole groups of 8 (16 bytes)
     for (int bx = 0; bx < nbox; ++bx) sc_tokens += min(p.box_tok, (w.n - (tok0 + bx * p.box_tok) + 7) & ~7);
-    mbar_expect_tx(full, nbox * p.box_tok * D + sc_tokens * 2);
+    mbar_expect_tx(full, nbox * p.box_tok * D + sc_tokens * 2 + (TAIL ? D * 2 : 0));
     const uint32_t dst = ring + stage * LO::kStage;
+    if (TAIL) {                                               // the tile is one 64-key block: its mean value row
+      bulk_load(ring + LO::off_means(p.stages) + mslot * (D * 2),
+                p.vmean + (long long)seq * p.vm_stride_seq + (long long)k.t * p.vm_stride_block + (long long)kvh * p.vm_stride_head,
+                D * 2, full);
+      if (++mslot == p.stages + 1) mslot = 0;
+    }
     for (int bx = 0; bx < nbox; ++bx) {
       const int j0 = tok0 + bx * p.box_tok;
       int c_seq = seq, c_tok = j0;
@@ -356,14 +365,17 @@ struct PlanePending {
   float e[2];            // the two keys' scales
   uint32_t live, refine; // verdict bits of the 16 keys, ORed over the rows
   int buf;               // the gather buffer its rows land in
+  int ms;                // block tail: the ring slot of its tile's mean value row
 };
 
 // DRAFTS: the rows carry draft masks (a separate instantiation: the plain one is at its register limit).
-template <int D, bool DRAFTS>
+// TAIL: cut keys add weight x the mean value row of their 64-key block (Section 4, "Depth as a dial").
+template <int D, bool DRAFTS, bool TAIL>
 __global__ void __launch_bounds__(kDenseThreads, kPlaneCtasPerSm)
 fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmV,
                         const PlaneScanParams pp) {
-  using LO = PlaneLayout<D>;
+  using LO = PlaneLayout<D, TAIL>;
+  static_assert(!TAIL || LO::kTK == 64, "a tile is one block of the block model");
   constexpr int TK = LO::kTK, U = TK / (16 * kConsumerWarps);          // sub-slices per warp and tile
   constexpr int CV = D / 8, CB = D / 16;                               // 16-byte chunks per value row / plane row
   const ScanParams &p = pp.s;
@@ -391,7 +403,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   __syncthreads();
   pdl_launch_dependents();
   if (warp == kConsumerWarps) {                              // plane A and the scales depend on nothing the front kernel writes
-    if (lane == 0) produce_plane_tiles<D>(&tmA, pp, w, split, kvh, seq, base, full0, empty0);
+    if (lane == 0) produce_plane_tiles<D, TAIL>(&tmA, pp, w, split, kvh, seq, base, full0, empty0);
     return;
   }
   pdl_wait();                                                // z and the split query rows come from the kernel before
@@ -449,6 +461,23 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   clear_bufs();
   uint32_t gphase = 0;                                       // bit b: parity of buffer b's next completed phase
   // second pass of a sub-slice: plane B product, final weights, value product
+  // Block tail: c0 / c1 = this thread's share of the mass rows (lane%4)*2 + {0,1} cut in the sub-slice; the eight lanes that
+  // scored the rows' keys are summed, then every channel this thread accumulates takes cut mass x the block's mean value.
+  const __nv_bfloat16 *means = reinterpret_cast<const __nv_bfloat16 *>(gen + LO::off_means(stages));
+  auto add_tail = [&](float c0, float c1, int ms) {
+#pragma unroll
+    for (int m = 4; m <= 16; m <<= 1) {
+      c0 += __shfl_xor_sync(0xffffffffu, c0, m);
+      c1 += __shfl_xor_sync(0xffffffffu, c1, m);
+    }
+    const __nv_bfloat16 *mrow = means + ms * D + klo;
+#pragma unroll
+    for (int mt = 0; mt < D / 16; ++mt) {
+      const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
+      o[mt][0] = fmaf(c0, m0, o[mt][0]); o[mt][1] = fmaf(c1, m0, o[mt][1]);
+      o[mt][2] = fmaf(c0, m1, o[mt][2]); o[mt][3] = fmaf(c1, m1, o[mt][3]);
+    }
+  };
   auto finish = [&](const PlanePending &pd) {
     const uint32_t bbuf = bufs + pd.buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
     const bool landed = mbar_wait(gbar_w + 8u * pd.buf, (gphase >> pd.buf) & 1u, dead);
@@ -457,6 +486,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
     if (pd.refine) plane_products<D>(bbuf, 0, lane, qa, qb, ca, cb);
     uint32_t bh[2], bl[2];
+    float cut0 = 0.f, cut1 = 0.f;
 #pragma unroll
     for (int kh = 0; kh < 2; ++kh) {
       const bool klive = (pd.live >> (klo + 8 * kh)) & 1u;
@@ -477,13 +507,15 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
       l_lo += (h0 + g0) + (pw[0] - pm[0]);
       l_hi += (h1 + g1) + (pw[1] - pm[1]);
+      if (TAIL) { cut0 += pw[0] - pm[0]; cut1 += pw[1] - pm[1]; }
       bh[kh] = movmatrix_trans(hi2);
       bl[kh] = movmatrix_trans(lo2);
     }
     if (pd.live) value_product_n<D, true, 0, 16>(o, vbuf, 0, lane, bh, bl);
+    if (TAIL) add_tail(cut0, cut1, pd.ms);
   };
 
-  int stage = 0, buf = 0, n_pend = 0;
+  int stage = 0, buf = 0, n_pend = 0, mslot = 0;
   uint32_t phase = 0;
   unsigned long long st_total = 0, st_live = 0, st_ref = 0;
   PlanePending pend[LO::kBufs - 1];
@@ -493,9 +525,10 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   for (int c = split; c < w.n_chunks; c += p.num_splits) {
     const int t_end = min((c + 1) * w.ctiles, w.n_tiles);
     for (int t = c * w.ctiles; t < t_end; ++t) {
-      const int my_stage = stage;
+      const int my_stage = stage, my_ms = mslot;
       const bool ready = mbar_wait(full0 + 8u * my_stage, phase, dead);
       if (++stage == stages) { stage = 0; phase ^= 1u; }
+      if (TAIL && ++mslot == stages + 1) mslot = 0;
       if (!ready) continue;
       const uint32_t at = base + my_stage * LO::kStage;
       const __nv_bfloat16 *scales = reinterpret_cast<const __nv_bfloat16 *>(gen + LO::off_scales(stages) + my_stage * LO::kScales);
@@ -528,15 +561,28 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         cur.live = __reduce_or_sync(0xffffffffu, lm);
         cur.refine = __reduce_or_sync(0xffffffffu, rm) & cur.live;
         cur.buf = buf;
+        cur.ms = my_ms;
         st_live += __popc(cur.live);
         st_ref += __popc(cur.refine);
         if (cur.live == 0u) {
           // every key of the sub-slice is cut for every row: no bytes are asked for, nothing is queued, and the weights
           // (the coarse scores are all this scan will ever have for these keys) only add to L
+          float cut0 = 0.f, cut1 = 0.f;
 #pragma unroll
           for (int kh = 0; kh < 2; ++kh) {
-            l_lo += ex2_approx(cur.x[2 * kh]);
-            l_hi += ex2_approx(cur.x[2 * kh + 1]);
+            cut0 += ex2_approx(cur.x[2 * kh]);
+            cut1 += ex2_approx(cur.x[2 * kh + 1]);
+          }
+          l_lo += cut0;
+          l_hi += cut1;
+          if (TAIL) {
+            add_tail(cut0, cut1, my_ms);
+            // a queued sub-slice must be finished while its tile's mean row is still in the ring (stages + 1 slots):
+            // with the tail on, a dead sub-slice does not let it wait any longer than a live one would
+#pragma unroll
+            for (int i = 0; i < LO::kBufs - 1; ++i)
+              if (i >= LO::kBufs - 1 - n_pend) finish(pend[i]);
+            n_pend = 0;
           }
           continue;
         }

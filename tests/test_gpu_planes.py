@@ -11,7 +11,7 @@ import paper_2609_33410_b200 as F
 from oracle import fold_oracle as O
 from oracle import fold_planes_oracle as P
 from paper_2609_33410_b200.workloads import make_decode_workload, bf16_bits
-from helpers import cache_of, same_bits, DENSE_MAX_ABS, DENSE_MEAN_REL, FINITE_T_FACTOR, LSE_TOL, Z_TOL
+from helpers import cache_of, oracle_block_means, same_bits, DENSE_MAX_ABS, DENSE_MEAN_REL, FINITE_T_FACTOR, LSE_TOL, Z_TOL
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -58,6 +58,11 @@ def split_queries(w, bufs):
     return codes[:, :, 0], codes[:, :, 1], eta
 
 
+def with_means(cache, vm):
+    return F.KVCache(cache.k, cache.v, cache.seqlens, cache.max_seqlen, cache.page_table, vm, cache.k_plane_a,
+                     cache.k_plane_b, cache.k_scale)
+
+
 def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, draft=None):
     """`draft` = (masks int32 [batch], draft_len): draft / tree-verification rows."""
     bufs = F.alloc_buffers(w.q, cache, w.stack)
@@ -70,7 +75,11 @@ def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0,
     return bufs
 
 
-def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estimate=False, check_counts=True, draft=None):
+def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estimate=False, check_counts=True, draft=None,
+                   v_block_mean=None):
+    """`v_block_mean`: the table the GPU was given (block tail); a key that flips at a gate then moves between its value
+    and its block's mean, so the threshold slack counts twice."""
+    vmt = None if v_block_mean is None else v_block_mean.float().cpu().numpy().astype(np.float64)
     dmask = None if draft is None else [int(x) & 0xffffffff for x in draft[0].cpu().tolist()]
     G = w.num_q_heads // w.num_kv_heads
     R = w.stack * G
@@ -99,7 +108,8 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
         rz = np.array([z[b, h] for (b, h) in rows])
         tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
         vis = None if draft is None else np.stack([O.draft_visible(n, draft[1], dmask[b]) for (b, h) in rows])
-        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis)
+        vm = None if vmt is None else vmt[seq, :(n + 63) // 64, kvh]
+        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis, v_mean=vm)
         n_live += int(info["live"].sum()); n_ref += int(info["refine"].sum()); n_keys += n
         vinf = np.abs(V).max(axis=1)
         near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
@@ -123,7 +133,7 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
                 dz = max(dz, abs(O.estimate_z(lambda idx: s_all[idx], n) - z[b, h]))
             if not math.isinf(T):
                 near = near_T | (np.abs(s_fin + T) <= BAND)
-                sl = float((p[near] * vinf[near]).sum() / L[i])
+                sl = (2.0 if vmt is not None else 1.0) * float((p[near] * vinf[near]).sum() / L[i])
                 sl += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum() / L[i])
                 slack2 += sl ** 2 * V.shape[1]
                 keep = slice(None) if vis is None else vis[i]
@@ -339,7 +349,7 @@ PLANE_LENGTHS = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255
 @pytest.mark.parametrize("seed", range(5))
 def test_random_shapes_match_the_oracle(seed):
     """Seeded random shapes of the two-plane path: head dimension, rows per kv head (1..8), lengths around every tile /
-    chunk / estimator boundary, paged or contiguous, depth and refine gate drawn together."""
+    chunk / estimator boundary, paged or contiguous, depth, refine gate, block tail and draft masks drawn together."""
     import random
     rnd = random.Random(7300 + seed)
     for i in range(8):
@@ -357,13 +367,26 @@ def test_random_shapes_match_the_oracle(seed):
             kw.update(paged=True, page_size=rnd.choice([16, 32, 64, 128]))
         else:
             kw.update(capacity=max(lens) + rnd.choice([0, 5, 100]))
-        case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw)
-        w = make_decode_workload(nseq * stack, G * Hkv, Hkv, D, lens, seed=seed * 100 + i, stack=stack, **kw)
+        tail = (not math.isinf(T)) and rnd.random() < 0.4
+        drafts = stack > 1 and rnd.random() < 0.5
+        case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw, tail=tail, drafts=drafts)
+        draft = None
+        if drafts:
+            from paper_2609_33410_b200.workloads import make_draft_workload
+            kw.pop("capacity", None)
+            w, masks, m = make_draft_workload(nseq, stack, G * Hkv, Hkv, D, [max(n, 1) for n in lens], seed=seed * 100 + i,
+                                              tree=rnd.random() < 0.5, **kw)
+            draft = (masks, m)
+        else:
+            w = make_decode_workload(nseq * stack, G * Hkv, Hkv, D, lens, seed=seed * 100 + i, stack=stack, **kw)
         cache = plane_cache(w)
+        vm = oracle_block_means(w) if tail else None
+        if tail:
+            cache = with_means(cache, vm)
         try:
-            b = run_planes(w, cache, T=T, tau=tau)
-            compare_planes(w, cache, b, T=T, tau=tau, check_estimate=True)
-            s = run_planes(w, cache, T=T, tau=tau, num_splits=rnd.choice([1, 2, 5]))
+            b = run_planes(w, cache, T=T, tau=tau, draft=draft)
+            compare_planes(w, cache, b, T=T, tau=tau, check_estimate=True, draft=draft, v_block_mean=vm)
+            s = run_planes(w, cache, T=T, tau=tau, num_splits=rnd.choice([1, 2, 5]), draft=draft)
             assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse), "split count changed a bit"
         except AssertionError as e:
             raise AssertionError(f"case {case}: {e}") from e
@@ -398,3 +421,25 @@ def test_draft_rows_on_two_plane_keys(Hq, Hkv, m, tree):
     w.v[0, n0 - 1] = -w.v[0, n0 - 1]                            # the LAST draft key: row 0 of a chain / tree never uses it
     again = run_planes(w, cache_after(w, cache), draft=d)
     assert same_bits(again.out[0], keep[0])
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,paged", [(8, 2, 128, False), (8, 8, 64, True), (4, 1, 128, True), (2, 2, 64, False)])
+def test_block_tail_on_two_plane_keys(Hq, Hkv, D, paged):
+    kw = dict(paged=True, page_size=32) if paged else dict(capacity=3100)
+    w = make_decode_workload(2, Hq, Hkv, D, [3000, 733], seed=101, device=DEV, poison_padding=True, **kw)
+    vm = oracle_block_means(w)
+    cache = with_means(plane_cache(w), vm)
+    plain = plane_cache(w)
+    for T in (6.0, 12.0, 16.0):
+        b = run_planes(w, cache, T=T)
+        r = compare_planes(w, cache, b, T=T, v_block_mean=vm)
+        s = run_planes(w, cache, T=T, num_splits=1)
+        assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse)
+        assert same_bits(b.lse, run_planes(w, plain, T=T).lse)          # the tail moves A only: L and lse are untouched
+    assert same_bits(run_planes(w, cache).out, run_planes(w, plain).out)  # nothing is cut in dense decode
+    # constant values: the tail gives back what the cut took away
+    w.v.fill_(1.5)
+    vm2 = oracle_block_means(w)
+    t = run_planes(w, with_means(plain, vm2), T=6.0)
+    ok = t.row_status.cpu().numpy() == 0
+    assert np.allclose(t.out.float().cpu().numpy()[ok], 1.5, rtol=1e-2)

@@ -247,3 +247,22 @@ def test_rows_that_do_not_see_a_key_give_it_no_weight_and_no_vote():
     info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T, -1.0, visible=vis)[2]
     own0 = np.where(vis[0], info["coarse"][0] >= -T, False); own1 = np.where(vis[1], info["coarse"][1] >= -T, False)
     assert np.array_equal(info["live"], own0 | own1)
+
+
+def test_block_tail_on_planes_reduces_to_the_plain_block_tail():
+    # one row, no refinement: the two-plane fold with a mean table is the plain depth-T fold with that table on the
+    # coarse scores; with constant values the tail restores exactly what the cut took away
+    D, n = 64, 300
+    k = rng_rows(22, n, D); V = rng_rows(23, n, D); q = rng_rows(24, 1, D)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    s = P.coarse_scores(ka, ke, qa[0], qb[0], eta[0])
+    Z = float(s.max()) - 1.0
+    vm = O.block_means(V)
+    A, L, info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, [Z], 4.0, -1.0, v_mean=vm)
+    o, lse, A0, L0 = O.fold_row(s, V, Z, 4.0, v_mean=vm)
+    assert 0 < info["live"].sum() < n
+    assert np.allclose(A[0], A0, rtol=1e-12) and np.isclose(L[0], L0, rtol=1e-12)
+    Vc = np.full((n, D), 1.5)
+    A, L, _ = P.fold_group_planes(ka, kb, ke, Vc, qa, qb, eta, [Z], 4.0, -1.0, v_mean=O.block_means(Vc))
+    assert np.allclose(A[0] / L[0], 1.5, rtol=1e-12)
