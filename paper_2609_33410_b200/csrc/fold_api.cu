@@ -239,7 +239,7 @@ PlaneView plane_view(const fold_kv &kv) {
 
 // Two-plane keys: the front kernel splits the query rows into the workspace whatever the reference mode, and
 // forms the estimate when asked to.
-int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st) {
+int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st, bool zero_header = false) {
   FrontParams p;
   memset(&p, 0, sizeof(p));
   p.q = static_cast<const __nv_bfloat16 *>(a->q);
@@ -254,6 +254,7 @@ int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st) 
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
   p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
   p.draft_len = a->draft_len;
+  p.hdr = zero_header ? static_cast<fold_ws_header *>(a->workspace) : nullptr;
   if (a->z_mode == FOLD_Z_ZERO) {
     const int rows = g.B * g.Hq;
     fold_fill_kernel<<<(rows + 255) / 256, 256, 0, st>>>(a->z, rows, 0.f);
@@ -264,8 +265,11 @@ int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st) 
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
-int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st) {
-  if (g.planes) return launch_planes_front(a, g, st);
+// zero_header: the kernel launched here also zeroes the first 64 bytes of a->workspace; header_zeroed_by_reference()
+// says whether this call's mode launches such a kernel
+bool header_zeroed_by_reference(const fold_args *a, const Geometry &g) { return g.planes || a->z_mode == FOLD_Z_ESTIMATE; }
+int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st, bool zero_header = false) {
+  if (g.planes) return launch_planes_front(a, g, st, zero_header);
   if (a->z_mode == FOLD_Z_GIVEN) return FOLD_OK;
   const int rows = g.B * g.Hq;
   if (a->z_mode == FOLD_Z_ZERO) {
@@ -275,6 +279,7 @@ int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st) {
     EstParams p = est_params(a, g);
     p.n_levels = 1;
     p.lv[0] = kv_level(a->kv, a->stack);
+    p.hdr = (zero_header && a->z_mode == FOLD_Z_ESTIMATE) ? static_cast<fold_ws_header *>(a->workspace) : nullptr;
     const dim3 grid(g.Hkv, g.B);
     if (a->z_mode == FOLD_Z_ESTIMATE) {
       if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstSampleThreads, 0, st>>>(p);
@@ -720,9 +725,11 @@ int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream str
   if (!args->workspace || !aligned(args->workspace, 256)) return FOLD_EINVAL;
   if (args->workspace_bytes < g.ws_bytes) return FOLD_EWORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // header first, so that reference -> scan -> partial add are adjacent kernels in the stream
-  if (cudaMemsetAsync(args->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
-  if (int rc = launch_reference(args, g, st)) return rc;
+  // the header is zeroed by the reference kernel where one runs (estimate, or the two-plane front kernel), else by a
+  // memset issued first, so that reference -> scan -> partial add stay adjacent kernels in the stream
+  const bool by_kernel = header_zeroed_by_reference(args, g);
+  if (!by_kernel && cudaMemsetAsync(args->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
+  if (int rc = launch_reference(args, g, st, by_kernel)) return rc;
   if (int rc = launch_scan(args, g, st)) return rc;
   fill_partials(args, g, dst);
   return FOLD_OK;

@@ -158,6 +158,7 @@ struct FrontParams {
   float scale_log2;
   const uint32_t *draft_mask;                                  // drafts: the last draft_len keys are used by request req only
   int draft_len;                                               // where its mask has the bit
+  fold_ws_header *hdr;                                         // not null: also zero the scan's workspace header
 };
 constexpr int kFrontThreads = kEstSamples;                    // 192
 
@@ -171,6 +172,7 @@ __global__ void __launch_bounds__(kFrontThreads) fold_planes_front_kernel(const 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G;
   pdl_launch_dependents();
+  if (p.hdr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16) reinterpret_cast<uint32_t *>(p.hdr)[threadIdx.x] = 0u;
 
   for (int g = warp; g < G; g += kFrontThreads / 32) {
     const int head = kvh * G + g;
