@@ -279,7 +279,7 @@ int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st, boo
     EstParams p = est_params(a, g);
     p.n_levels = 1;
     p.lv[0] = kv_level(a->kv, a->stack);
-    p.hdr = (zero_header && a->z_mode == FOLD_Z_ESTIMATE) ? static_cast<fold_ws_header *>(a->workspace) : nullptr;
+    p.hdr[0] = (zero_header && a->z_mode == FOLD_Z_ESTIMATE) ? static_cast<fold_ws_header *>(a->workspace) : nullptr;
     const dim3 grid(g.Hkv, g.B);
     if (a->z_mode == FOLD_Z_ESTIMATE) {
       if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstSampleThreads, 0, st>>>(p);
@@ -669,7 +669,11 @@ size_t fold_workspace_bytes(const fold_args *args) {
   return round_up(base, 256) + qplane_bytes((long long)tmp.batch * tmp.num_q_heads, tmp.head_dim);
 }
 
-int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream stream) {
+}  // extern "C"
+
+namespace {
+// zero_headers: the estimate kernel also zeroes every level's workspace header (the cascade's scans then need no memset)
+int estimate_levels(const fold_args *const *levels, int n_levels, fold_stream stream, bool zero_headers) {
   if (!levels || n_levels < 1 || n_levels > kMaxLevels) return FOLD_EINVAL;
   const fold_args *a0 = levels[0];
   if (!a0) return FOLD_EINVAL;
@@ -710,6 +714,11 @@ int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream st
     if (a->stack < 1 || a->batch % a->stack || a->batch / a->stack != a->kv.num_seqs) return FOLD_EINVAL;
     if (int rc = check_kv(a->kv, a->head_dim)) return rc;
     p.lv[l] = kv_level(a->kv, a->stack);
+    if (zero_headers) {
+      if (!a->workspace || !aligned(a->workspace, 256)) return FOLD_EINVAL;
+      if (a->workspace_bytes < kHeaderBytes) return FOLD_EWORKSPACE;
+      p.hdr[l] = static_cast<fold_ws_header *>(a->workspace);
+    }
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(g.Hkv, g.B);
@@ -718,7 +727,8 @@ int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream st
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
-int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream stream) {
+// header_done: the workspace header has been zeroed by a kernel already in the stream
+int decode_split_impl(const fold_args *args, fold_partials *dst, fold_stream stream, bool header_done) {
   Geometry g;
   if (int rc = check_args(args, &g, false)) return rc;
   if (!dst) return FOLD_EINVAL;
@@ -728,11 +738,22 @@ int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream str
   // the header is zeroed by the reference kernel where one runs (estimate, or the two-plane front kernel), else by a
   // memset issued first, so that reference -> scan -> partial add stay adjacent kernels in the stream
   const bool by_kernel = header_zeroed_by_reference(args, g);
-  if (!by_kernel && cudaMemsetAsync(args->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
+  if (!by_kernel && !header_done && cudaMemsetAsync(args->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
   if (int rc = launch_reference(args, g, st, by_kernel)) return rc;
   if (int rc = launch_scan(args, g, st)) return rc;
   fill_partials(args, g, dst);
   return FOLD_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream stream) {
+  return estimate_levels(levels, n_levels, stream, false);
+}
+
+int fold_decode_split(const fold_args *args, fold_partials *dst, fold_stream stream) {
+  return decode_split_impl(args, dst, stream, false);
 }
 
 int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *out, float *lse, int32_t *row_status,
@@ -861,8 +882,9 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
     lv[l].z_mode = FOLD_Z_GIVEN;
     if (int rc = check_args(&lv[l], &g, l == 0)) return rc;
   }
-  if (a0->z_mode == FOLD_Z_ESTIMATE)
-    if (int rc = fold_estimate_z(levels, n_levels, stream)) return rc;
+  const bool est = a0->z_mode == FOLD_Z_ESTIMATE;            // the estimate kernel then zeroes every level's header too
+  if (est)
+    if (int rc = estimate_levels(levels, n_levels, stream, true)) return rc;
   fold_partials parts[kMaxLevels];
   const fold_partials *pp[kMaxLevels];
   for (int l = 0; l < n_levels; ++l) pp[l] = &parts[l];
@@ -875,16 +897,16 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
     std::lock_guard<std::mutex> lock(side->mu);               // the events are shared by every call on the device
     if (cudaEventRecord(side->fork, st) != cudaSuccess || cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess)
       return FOLD_ECUDA;
-    int rc = fold_decode_split(&lv[0], &parts[0], side->stream);
+    int rc = decode_split_impl(&lv[0], &parts[0], side->stream, est);
     const bool recorded = cudaEventRecord(side->join, side->stream) == cudaSuccess;
-    for (int l = 1; l < n_levels && rc == FOLD_OK; ++l) rc = fold_decode_split(&lv[l], &parts[l], stream);
+    for (int l = 1; l < n_levels && rc == FOLD_OK; ++l) rc = decode_split_impl(&lv[l], &parts[l], stream, est);
     // join in every case, so that the side stream never holds work the caller's stream does not wait for
     if (!recorded || cudaStreamWaitEvent(st, side->join, 0) != cudaSuccess) return FOLD_ECUDA;
     if (rc) return rc;
     return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
   }
   for (int l = 0; l < n_levels; ++l)
-    if (int rc = fold_decode_split(&lv[l], &parts[l], stream)) return rc;
+    if (int rc = decode_split_impl(&lv[l], &parts[l], stream, est)) return rc;
   return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
 }
 

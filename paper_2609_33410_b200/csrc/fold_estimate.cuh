@@ -35,7 +35,7 @@ struct EstParams {
   float scale_log2;
   const uint32_t *draft_mask;    // drafts: the last draft_len keys (of the concatenated levels) are used by request
   int draft_len;                 // req only where its mask has the bit
-  fold_ws_header *hdr;           // not null: this launch also zeroes the scan's workspace header (one memset less)
+  fold_ws_header *hdr[kMaxLevels];   // not null: this launch also zeroes that level's workspace header (a memset less)
 };
 
 __device__ __forceinline__ int level_len(const KvLevel &L, int req) {
@@ -128,8 +128,9 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G;
   pdl_launch_dependents();                           // the scan may set up while the estimate runs
-  if (p.hdr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16)
-    reinterpret_cast<uint32_t *>(p.hdr)[threadIdx.x] = 0u;   // the scan touches the header only after its dependency wait
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16)
+    for (int l = 0; l < p.n_levels; ++l)                  // the scans touch their headers only after their dependency wait
+      if (p.hdr[l]) reinterpret_cast<uint32_t *>(p.hdr[l])[threadIdx.x] = 0u;
 
   int lens[kMaxLevels];
   int n = 0;
