@@ -86,19 +86,19 @@ __device__ __forceinline__ float est_reduce_row(const float *row, int n, int n_s
       float c[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) c[i] = row[1 + kEstRecent + lane + 32 * i];
+      // (floats compared as order-preserving unsigned keys, so that the warp-wide maximum is one redux instruction)
+      auto key_of = [](float f) { const uint32_t b = __float_as_uint(f); return (b & 0x80000000u) ? ~b : (b | 0x80000000u); };
 #pragma unroll 1
       for (int r = 0; r < kEstTrim; ++r) {
-        float wm = fmaxf(fmaxf(c[0], c[1]), fmaxf(c[2], c[3]));
-#pragma unroll
-        for (int k = 16; k > 0; k >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, k));
-        bool found = false;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const unsigned owners = __ballot_sync(0xffffffffu, c[i] == wm);
-          if (!found && owners) {
-            if (lane == __ffs(owners) - 1) c[i] = -INFINITY;
-            found = true;
-          }
+        const uint32_t k0 = key_of(c[0]), k1 = key_of(c[1]), k2 = key_of(c[2]), k3 = key_of(c[3]);
+        const uint32_t mine = max(max(k0, k1), max(k2, k3));
+        const uint32_t wm = __reduce_max_sync(0xffffffffu, mine);
+        const unsigned owners = __ballot_sync(0xffffffffu, mine == wm);
+        if (lane == __ffs(owners) - 1) {                     // the lowest lane among equals drops one of its own
+          if (k0 == wm) c[0] = -INFINITY;
+          else if (k1 == wm) c[1] = -INFINITY;
+          else if (k2 == wm) c[2] = -INFINITY;
+          else c[3] = -INFINITY;
         }
       }
       float kept = 0.f;
