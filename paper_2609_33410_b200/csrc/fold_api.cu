@@ -260,8 +260,9 @@ int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st, 
     fold_fill_kernel<<<(rows + 255) / 256, 256, 0, st>>>(a->z, rows, 0.f);
   }
   const dim3 grid(g.Hkv, g.B);
-  if (g.D == 128) fold_planes_front_kernel<128><<<grid, kFrontThreads, 0, st>>>(p);
-  else fold_planes_front_kernel<64><<<grid, kFrontThreads, 0, st>>>(p);
+  const cudaError_t rc = g.D == 128 ? launch_pdl(fold_planes_front_kernel<128>, grid, dim3(kFrontThreads), 0, st, p)
+                                    : launch_pdl(fold_planes_front_kernel<64>, grid, dim3(kFrontThreads), 0, st, p);
+  if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
@@ -282,8 +283,9 @@ int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st, boo
     p.hdr[0] = (zero_header && a->z_mode == FOLD_Z_ESTIMATE) ? static_cast<fold_ws_header *>(a->workspace) : nullptr;
     const dim3 grid(g.Hkv, g.B);
     if (a->z_mode == FOLD_Z_ESTIMATE) {
-      if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstSampleThreads, 0, st>>>(p);
-      else fold_estimate_kernel<64><<<grid, kEstSampleThreads, 0, st>>>(p);
+      const cudaError_t rc = g.D == 128 ? launch_pdl(fold_estimate_kernel<128>, grid, dim3(kEstSampleThreads), 0, st, p)
+                                        : launch_pdl(fold_estimate_kernel<64>, grid, dim3(kEstSampleThreads), 0, st, p);
+      if (rc != cudaSuccess) return FOLD_ECUDA;
     } else {
       if (g.D == 128) fold_exact_max_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
       else fold_exact_max_kernel<64><<<grid, kEstThreads, 0, st>>>(p);
@@ -722,8 +724,9 @@ int estimate_levels(const fold_args *const *levels, int n_levels, fold_stream st
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(g.Hkv, g.B);
-  if (g.D == 128) fold_estimate_kernel<128><<<grid, kEstSampleThreads, 0, st>>>(p);
-  else fold_estimate_kernel<64><<<grid, kEstSampleThreads, 0, st>>>(p);
+  const cudaError_t rc = g.D == 128 ? launch_pdl(fold_estimate_kernel<128>, grid, dim3(kEstSampleThreads), 0, st, p)
+                                    : launch_pdl(fold_estimate_kernel<64>, grid, dim3(kEstSampleThreads), 0, st, p);
+  if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 

@@ -128,9 +128,6 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G;
   pdl_launch_dependents();                           // the scan may set up while the estimate runs
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16)
-    for (int l = 0; l < p.n_levels; ++l)                  // the scans touch their headers only after their dependency wait
-      if (p.hdr[l]) reinterpret_cast<uint32_t *>(p.hdr[l])[threadIdx.x] = 0u;
 
   int lens[kMaxLevels];
   int n = 0;
@@ -196,6 +193,13 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
     }
   }
   __syncthreads();
+  // Everything above reads only the caller's inputs.  What follows writes: z, which the partial add of a call before
+  // this one may still be reading, and the workspace headers -- so it waits for the kernels before (a no-op unless this
+  // kernel was launched early behind one that allows it).
+  pdl_wait();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16)
+    for (int l = 0; l < p.n_levels; ++l)                  // the scans touch their headers only after their dependency wait
+      if (p.hdr[l]) reinterpret_cast<uint32_t *>(p.hdr[l])[threadIdx.x] = 0u;
 
   // warp g finishes row g
   for (int g = warp; g < G; g += kEstSampleThreads / 32) {

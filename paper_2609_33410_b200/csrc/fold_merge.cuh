@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
   const bool active = row < n_rows;
   const int b = active ? (int)(row / p.Hq) : 0, h = active ? (int)(row % p.Hq) : 0;
   const int G = p.G, kvh = h / G, hg = h % G;
+  pdl_launch_dependents();                           // the next call's reference kernel may set up and load meanwhile
   pdl_wait();                                        // slots and z come from the kernels before
   const float zrow = active ? p.z[row] : 0.f;        // requested early: only needed at the very end
 

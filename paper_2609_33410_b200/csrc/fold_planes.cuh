@@ -172,24 +172,31 @@ __global__ void __launch_bounds__(kFrontThreads) fold_planes_front_kernel(const 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G;
   pdl_launch_dependents();
-  if (p.hdr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16) reinterpret_cast<uint32_t *>(p.hdr)[threadIdx.x] = 0u;
 
+  // Everything up to the dependency wait below reads only the caller's inputs and writes shared memory: launched
+  // early behind the partial add of a call before this one, it overlaps it.
   for (int g = warp; g < G; g += kFrontThreads / 32) {
     const int head = kvh * G + g;
     float x[EPL];
     load_bf16_row<EPL>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + lane * EPL, x);
     int a[EPL], b[EPL];
     const float e = rotate_split<D>(x, lane, a, b);
-    const float eta = __fmul_rn(e, p.scale_log2);
-    int8_t *dst = p.qplanes + ((long long)req * p.Hq + head) * (2 * D);
-    store_codes<EPL>(dst + lane * EPL, a);
-    store_codes<EPL>(dst + D + lane * EPL, b);
     store_codes<EPL>(reinterpret_cast<int8_t *>(&sq[g][0][0]) + lane * EPL, a);
     store_codes<EPL>(reinterpret_cast<int8_t *>(&sq[g][1][0]) + lane * EPL, b);
-    if (lane == 0) { p.qeta[(long long)req * p.Hq + head] = eta; seta[g] = eta; }
+    if (lane == 0) seta[g] = __fmul_rn(e, p.scale_log2);
   }
-  if (!p.write_z) return;
   __syncthreads();
+  // the workspace (split rows, header) may still be read by the scan of a call before this one, z by its partial add
+  auto publish = [&]() {
+    pdl_wait();
+    if (p.hdr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16) reinterpret_cast<uint32_t *>(p.hdr)[threadIdx.x] = 0u;
+    for (int i = threadIdx.x; i < G * 2 * W; i += kFrontThreads) {          // rows kvh * G .. + G - 1 are contiguous
+      const int g = i / (2 * W), w = i % (2 * W);
+      reinterpret_cast<uint32_t *>(p.qplanes + ((long long)req * p.Hq + kvh * G + g) * (2 * D))[w] = sq[g][w / W][w % W];
+    }
+    if (threadIdx.x < G) p.qeta[(long long)req * p.Hq + kvh * G + threadIdx.x] = seta[threadIdx.x];
+  };
+  if (!p.write_z) { publish(); return; }
 
   const int seq = req / p.stack;
   int n = p.kv.seqlens[seq];
@@ -227,6 +234,7 @@ __global__ void __launch_bounds__(kFrontThreads) fold_planes_front_kernel(const 
     }
   }
   __syncthreads();
+  publish();
   for (int g = warp; g < G; g += kFrontThreads / 32) {
     const float zval = est_reduce_row(sc[g], n, n_samples, lane);
     if (lane == 0) p.z[(long long)req * p.Hq + kvh * G + g] = zval;
