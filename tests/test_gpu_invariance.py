@@ -198,3 +198,32 @@ def test_cascade_call_is_graph_capturable_with_its_side_stream():
         torch.cuda.synchronize()
         assert same_bits(bs.out, o) and same_bits(bs.lse, l)
         assert bp.header().wait_timeouts == 0 and bs.header().wait_timeouts == 0
+
+
+@pytest.mark.parametrize("planes", [False, True])
+def test_back_to_back_calls_that_share_z_and_workspace_do_not_disturb_each_other(planes):
+    # The reference kernel of a call may start while the partial add of the call before it is still running (programmatic
+    # dependent launch); it must not write z, the header or the workspace before that add is done.  Two different
+    # workloads of one shape alternate on ONE z buffer and ONE workspace, without a host synchronisation between calls.
+    wa = make_decode_workload(4, 8, 2, 128, [9000, 700, 4000, 33], seed=71, device=DEV)
+    wb = make_decode_workload(4, 8, 2, 128, [8000, 9000, 100, 5000], seed=72, device=DEV, capacity=wa.k.shape[1])
+    ca, cb = cache_of(wa), cache_of(wb)
+    if planes:
+        F.fold_quantize_keys(ca); F.fold_quantize_keys(cb)
+    ref = []
+    for w, c in ((wa, ca), (wb, cb)):
+        b = F.alloc_buffers(w.q, c)
+        F.decode(w.q, c, b, depth_T=16.0)
+        torch.cuda.synchronize()
+        ref.append((b.out.clone(), b.lse.clone()))
+    shared = F.alloc_buffers(wa.q, ca)
+    outs = [torch.empty_like(ref[0][0]) for _ in range(2)]
+    lses = [torch.empty_like(ref[0][1]) for _ in range(2)]
+    args = [F.make_args(w.q, c, depth_T=16.0, z=shared.z, workspace=shared.workspace, out=outs[i], lse=lses[i],
+                        row_status=shared.row_status) for i, (w, c) in enumerate(((wa, ca), (wb, cb)))]
+    for _ in range(25):
+        F.fold_decode(args[0])
+        F.fold_decode(args[1])
+    torch.cuda.synchronize()
+    for i in range(2):
+        assert same_bits(outs[i], ref[i][0]) and same_bits(lses[i], ref[i][1]), i
