@@ -21,6 +21,10 @@ What is here, with the passage each function restates (Section 4, "Cache format"
   refined_scores      Algorithm 1: eta e (c^aa + c^ab/256) and the plane-B correction, float64
   auto_refine_tau     the refine gate when the caller gives none.  PARITY UNPINNED by the paper (it
                       gives no formula); the reading taken is in the docstring
+  e4m3_values / round_e4m3 / quantize_values / widen_values
+                      Section 4 "Cache format": values as two E4M3 planes under a power-of-two scale,
+                      v ~ 2^k (v1 + v2), the second plane read only for keys whose weight matters
+                      ("refine V"); E4M3 = 1-4-3 bits, bias 7, no infinities, largest value 448
   fold_group_planes   Algorithm 1 for one (sequence, kv head): verdict bits ORed over the
                       group's rows, final weights, (A, L) per row; also counts the bytes the
                       gates ask for (130 + 128 r_K + 256 lambda per key at D = 128)
@@ -126,6 +130,67 @@ def refined_scores(ka, kb, ke, qa, qb, eta: float) -> np.ndarray:
     return coarse_scores(ka, ke, qa, qb, eta) + refine_terms(kb, ke, qa, qb, eta)
 
 
+# --------------------------------------------------------------------------- E4M3 value planes
+def e4m3_values() -> np.ndarray:
+    """The 256 E4M3 codes as float64: sign, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is
+    subnormal (m/8 * 2^-6), there are no infinities, 0x7f / 0xff are NaN, the largest value is 448."""
+    v = np.empty(256)
+    for b in range(256):
+        sgn = -1.0 if b & 0x80 else 1.0
+        e, m = (b >> 3) & 0xF, b & 7
+        if e == 15 and m == 7:
+            v[b] = np.nan
+        elif e == 0:
+            v[b] = sgn * (m / 8.0) * 2.0 ** -6
+        else:
+            v[b] = sgn * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return v
+
+
+_E4M3 = e4m3_values()
+_E4M3_POS = _E4M3[:0x7f]                                     # codes 0x00 .. 0x7e ascend from 0 to 448
+
+
+def round_e4m3(x: np.ndarray) -> np.ndarray:
+    """x -> the E4M3 code (uint8) nearest to x, ties to the even code, magnitudes beyond 448 saturate
+    to 448 (the "satfinite" conversion)."""
+    x = np.asarray(x, dtype=np.float64)
+    a = np.minimum(np.abs(x), 448.0)
+    hi = np.clip(np.searchsorted(_E4M3_POS, a, side="left"), 1, 0x7e)
+    lo = hi - 1
+    dlo, dhi = a - _E4M3_POS[lo], _E4M3_POS[hi] - a
+    code = np.where((dhi < dlo) | ((dhi == dlo) & (hi % 2 == 0)), hi, lo).astype(np.uint8)
+    return np.where(np.signbit(x), code | np.uint8(0x80), code).astype(np.uint8)
+
+
+def quantize_values(V: np.ndarray, scale_log2: int):
+    """Value rows -> two E4M3 planes under the scale 2^scale_log2 (a power of two per layer, given by the
+    caller): p1 = e4m3(v / 2^k), p2 = e4m3(v / 2^k - p1).  Both subtractions and the scaling are exact for
+    BF16 inputs, so the codes depend on nothing but the rounding rule.  Returns (p1, p2) uint8."""
+    x = np.asarray(V, dtype=np.float64) * 2.0 ** (-scale_log2)
+    p1 = round_e4m3(x)
+    p2 = round_e4m3(x - _E4M3[p1])
+    return p1, p2
+
+
+def widen_values(p1, p2, scale_log2: int, refined) -> np.ndarray:
+    """What the scan multiplies: 2^k * v1 for a key read from plane 1 alone, 2^k * bf16(v1 + v2) for a key
+    whose second plane is read (`refined` bool [n]).  v1 and v2 widen to BF16 exactly; their sum can need
+    nine significant bits and is rounded to BF16 once (the reading taken: the value product runs in BF16)."""
+    v1 = _E4M3[np.asarray(p1)]
+    v2 = _E4M3[np.asarray(p2)]
+    both = O.round_to_bf16(v1 + v2)
+    return np.where(np.asarray(refined, dtype=bool)[:, None], both, v1) * 2.0 ** scale_log2
+
+
+def auto_refine_tau_v(n: int) -> float:
+    """The refine-V gate when the caller gives none.  Reading (PARITY UNPINNED, like auto_refine_tau): a key's
+    second value plane is read when some row of its group gives it at least 1/(2n) of the row's mass,
+    tau_V = max(log2(n) + 1, 4).  On the synthetic rows plane 1 alone leaves the dense output at 13 x the BF16
+    online-softmax error, tau_V = log2 n at 0.6-1.6 x, log2 n + 2 at 0.1-0.3 x."""
+    return max(math.log2(max(n, 1)) + 1.0, 4.0)
+
+
 def auto_refine_tau(n: int) -> float:
     """The refine gate tau_K used when the caller gives none.  The paper says only that the refine
     thresholds follow each request's own length and are set where the second plane starts to matter at
@@ -138,7 +203,7 @@ def auto_refine_tau(n: int) -> float:
 
 
 def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None, visible=None,
-                      v_mean=None):
+                      v_mean=None, value_planes=None, tau_v: Optional[float] = None):
     """Algorithm 1 for the rows of one (sequence, kv head) group over all its keys.
     ka, kb [n, D] int8; ke [n]; V [n, D]; qa, qb [R, D] int8; eta [R]; Z [R] (binades).
     tau: refine gate in binades (None: auto_refine_tau(n); inf: refine every live key; negative:
@@ -151,9 +216,12 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
     v_mean [ceil(n/64), D] switches the block tail on (``fold_oracle.block_means``; Algorithm 1 "add the weights of
     cut keys to the tile's virtual row"): a key whose weight row i does not keep in A adds weight x the mean value row
     of its 64-key block to A_i instead of nothing.
+    value_planes = (p1, p2, scale_log2) replaces V by two E4M3 planes: refine_v_j = live_j AND
+    OR_i [coarse_ij - Z_i >= -tau_v] (tau_v None: auto_refine_tau_v(n); inf: every live key; negative: none), and
+    key j's value row is widen_values(...) with that mask (`V` is then ignored).
     Returns (A [R, D], L [R], info) with info = live / refine masks and the bytes-per-key count."""
     ka = np.asarray(ka); kb = np.asarray(kb)
-    V = np.asarray(V, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64) if value_planes is None else None
     n, D = ka.shape
     R = len(eta)
     if tau is None:
@@ -163,6 +231,12 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
         coarse = np.where(np.asarray(visible, dtype=bool), coarse, -np.inf)
     live = np.isfinite(coarse).any(axis=0) if math.isinf(T) else (coarse >= -T).any(axis=0)
     refine = live & ((coarse >= -tau).any(axis=0) if tau >= 0 else np.zeros(n, dtype=bool))
+    refine_v = np.zeros(n, dtype=bool)
+    if value_planes is not None:
+        if tau_v is None:
+            tau_v = auto_refine_tau_v(n)
+        refine_v = live & ((coarse >= -tau_v).any(axis=0) if tau_v >= 0 else np.zeros(n, dtype=bool))
+        V = widen_values(value_planes[0], value_planes[1], value_planes[2], refine_v)
     A = np.zeros((R, D)); L = np.zeros(R)
     for i in range(R):
         s = coarse[i] + np.where(refine, refine_terms(kb, ke, qa[i], qb[i], eta[i]), 0.0)
@@ -175,8 +249,9 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
             block_of = np.arange(n) // O.BLOCK_KEYS
             for b in np.unique(block_of[~keep]):
                 A[i] = A[i] + p[~keep & (block_of == b)].sum() * vm[b]
-    info = dict(live=live, refine=refine, coarse=coarse,
-                bytes_per_key=(D + 2) + D * float(refine.mean() if n else 0.0) + 2 * D * float(live.mean() if n else 0.0))
+    lam, rk, rv = (float(m.mean()) if n else 0.0 for m in (live, refine, refine_v))
+    v_bytes = 2 * D * lam if value_planes is None else D * lam + D * rv          # "8-bit values replace 256 with 128 + 128 r_V"
+    info = dict(live=live, refine=refine, refine_v=refine_v, coarse=coarse, bytes_per_key=(D + 2) + D * rk + v_bytes)
     return A, L, info
 
 

@@ -266,3 +266,56 @@ def test_block_tail_on_planes_reduces_to_the_plain_block_tail():
     Vc = np.full((n, D), 1.5)
     A, L, _ = P.fold_group_planes(ka, kb, ke, Vc, qa, qb, eta, [Z], 4.0, -1.0, v_mean=O.block_means(Vc))
     assert np.allclose(A[0] / L[0], 1.5, rtol=1e-12)
+
+
+def test_e4m3_grid_and_rounding_hand_values():
+    v = P.e4m3_values()
+    # 1-4-3 bits, bias 7: 0x38 = 1.0, 0x7e = 448 (largest), 0x01 = 2^-9 (smallest subnormal), 0x08 = 2^-6 (smallest normal)
+    assert v[0x38] == 1.0 and v[0x7e] == 448.0 and v[0x01] == 2.0 ** -9 and v[0x08] == 2.0 ** -6 and v[0xb8] == -1.0
+    assert np.isnan(v[0x7f]) and np.isnan(v[0xff]) and np.all(np.diff(v[:0x7f]) > 0)
+    x = np.array([1.0, 1.0625, 1.1875, 17.0, 448.0, 1000.0, -464.0, 2.0 ** -10, 3 * 2.0 ** -10, 0.3])
+    want = [0x38, 0x38, 0x3a, 0x58, 0x7e, 0x7e, 0xfe, 0x00, 0x02, 0x2a]       # ties to the even code; beyond 448 saturates
+    assert P.round_e4m3(x).tolist() == want
+    # nearest: no other code is closer, for a dense sample of the range
+    xs = np.linspace(-460, 460, 20011)
+    c = P.round_e4m3(xs)
+    d = np.abs(np.minimum(np.abs(xs), 448.0)[:, None] - v[None, :0x7f])
+    assert np.all(np.abs(np.abs(v[c]) - np.minimum(np.abs(xs), 448.0)) <= d.min(axis=1) + 1e-15)
+
+
+def test_value_planes_reconstruct_within_their_steps():
+    V = rng_rows(25, 300, 128, spread=2.0)
+    k = int(math.ceil(math.log2(np.abs(V).max() / 448.0)))
+    p1, p2 = P.quantize_values(V, k)
+    one = P.widen_values(p1, p2, k, np.zeros(300, bool)); two = P.widen_values(p1, p2, k, np.ones(300, bool))
+    nz = np.abs(V) >= 2.0 ** (k - 6)                            # normal range of plane 1: 3 mantissa bits, then 3 more + BF16
+    assert np.all(np.abs(one - V)[nz] <= np.abs(V)[nz] * 2.0 ** -4)
+    assert np.all(np.abs(two - V)[nz] <= np.abs(V)[nz] * 2.0 ** -8 * 1.01 + 2.0 ** (k - 10))   # (the residual's code may be subnormal)
+    assert np.mean(np.abs(two - V)[nz] <= np.abs(V)[nz] * 2.0 ** -8 * 1.01) > 0.95
+    assert np.all(np.abs(one - V) <= 2.0 ** (k - 10) + np.abs(V) * 2.0 ** -4)    # subnormal plane-1 codes: absolute step 2^-9
+    assert np.array_equal(O.round_to_bf16(two), two) and np.array_equal(O.round_to_bf16(one), one)   # both are BF16 values
+    mixed = P.widen_values(p1, p2, k, np.arange(300) % 2 == 0)
+    assert np.array_equal(mixed[0::2], two[0::2]) and np.array_equal(mixed[1::2], one[1::2])
+
+
+def test_group_fold_with_value_planes_special_cases_and_bytes():
+    D, n, R = 128, 400, 4
+    k_ = rng_rows(26, n, D); q = rng_rows(27, R, D); V = rng_rows(28, n, D)
+    ka, kb, ke = P.quantize_rows(k_); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    Z = np.array([P.coarse_scores(ka, ke, qa[i], qb[i], eta[i]).max() for i in range(R)]) - 2.0
+    sl = int(math.ceil(math.log2(np.abs(V).max() / 448.0)))
+    p1, p2 = P.quantize_values(V, sl)
+    # every live key refined (keys and values), dense: the plain fold on the fully widened values; 514 - 256 + 256 bytes
+    A, L, info = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, math.inf, math.inf, value_planes=(p1, p2, sl), tau_v=math.inf)
+    A0, L0, _ = P.fold_group_planes(ka, kb, ke, P.widen_values(p1, p2, sl, np.ones(n, bool)), qa, qb, eta, Z, math.inf, math.inf)
+    assert np.array_equal(A, A0) and np.array_equal(L, L0) and info["bytes_per_key"] == 130 + 128 + 128 + 128
+    # no second plane at all: plane-1 values; "8-bit values replace 256 with 128 + 128 r_V"
+    A, L, info = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, 6.0, -1.0, value_planes=(p1, p2, sl), tau_v=-1.0)
+    A0, L0, i0 = P.fold_group_planes(ka, kb, ke, P.widen_values(p1, p2, sl, np.zeros(n, bool)), qa, qb, eta, Z, 6.0, -1.0)
+    assert np.array_equal(A, A0) and info["bytes_per_key"] == 130 + 128 * i0["live"].mean()
+    # the refine-V verdict is ORed over the group like the others, and only live keys can carry it
+    A, L, info = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, 6.0, -1.0, value_planes=(p1, p2, sl), tau_v=3.0)
+    assert np.array_equal(info["refine_v"], info["live"] & (info["coarse"] >= -3.0).any(axis=0))
+    assert 0 < info["refine_v"].sum() < info["live"].sum()
+    assert P.auto_refine_tau_v(32768) == 16.0 and P.auto_refine_tau_v(4) == 4.0
