@@ -99,7 +99,16 @@ enum {
  * key against plane A alone (head_dim + 2 bytes per key), ORs the verdicts over the rows that share the kv head,
  * and only then requests plane B rows (refined keys) and value rows (live keys).  This path takes row blocks of
  * at most 8 rows (stack * group <= 8, draft rows included) and one level (no cascade), with or without the block
- * tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED. */
+ * tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED.
+ *
+ * Two E4M3 value planes (Section 4, "Cache format": "two E4M3 planes under a power-of-two scale per layer"; only
+ * together with the two-plane keys).  When v_plane_1 is not NULL the scan reads values from
+ *     v_j ~ 2^v_scale_log2 * (v1_j + v2_j),   v1, v2 E4M3 codes (1-4-3 bits, bias 7, largest value 448),
+ * written by fold_quantize_values(): rows of head_dim bytes laid out exactly like the key planes (the same
+ * plane_stride_* and paging).  A live key's plane-1 row is always read; its plane-2 row only when some row of
+ * the group gives the key a coarse weight >= 2^-refine_tau_v ("refine V"): head_dim + head_dim * r_V bytes per live
+ * key instead of 2 * head_dim.  The codes widen to BF16 exactly; v1 + v2 is rounded to BF16 once.  v may then be
+ * NULL for the decode calls.  Not offered with draft masks or the block tail (FOLD_EUNSUPPORTED). */
 typedef struct fold_kv {
   const void *k, *v;
   int64_t stride_seq, stride_tok, stride_head;   /* elements */
@@ -117,6 +126,8 @@ typedef struct fold_kv {
   int64_t plane_stride_seq, plane_stride_tok, plane_stride_head;  /* bytes */
   const void *k_scale;                           /* BF16 scale per (token, kv head), token-fastest */
   int64_t scale_stride_seq, scale_stride_head;   /* elements */
+  const uint8_t *v_plane_1, *v_plane_2;          /* E4M3 value planes (strides: plane_stride_*), or NULL: BF16 values from v */
+  int32_t v_scale_log2;                          /* the value planes' power-of-two scale */
 } fold_kv;
 
 /* One decode call.  `batch` requests with one query token each; request b reads KV
@@ -157,6 +168,8 @@ typedef struct fold_args {
                                           0 = choose: max(log2(n) - 2, 4) for a sequence of n keys (its own length only:
                                           a key is refined when some row gives it >= 4/n of the row's mass);
                                           INFINITY = every live key; negative = none (plane A scores only) */
+  float refine_tau_v;                  /* E4M3 value planes only: the refine-V gate, binades, like refine_tau.
+                                          0 = choose: max(log2(n) + 1, 4); INFINITY = every live key; negative = none */
 } fold_args;
 
 /* First 64 bytes of every workspace, zeroed at the start of each scan. */
@@ -167,7 +180,8 @@ typedef struct fold_ws_header {
   uint64_t v_rows_total;       /* value rows a dense decode would read (= keys scanned) */
   uint64_t v_slices_skipped;   /* warp slices (16 keys at head_dim 128, 32 at 64) whose value work was skipped entirely */
   uint64_t k_rows_refined;     /* two-plane keys: plane B rows requested from memory */
-  uint64_t pad[3];
+  uint64_t v2_rows_refined;    /* E4M3 value planes: plane-2 rows requested from memory */
+  uint64_t pad[2];
 } fold_ws_header;
 
 /* The (A, L) partial pairs one scan leaves in its workspace (Algorithm 1, last line).
@@ -261,6 +275,15 @@ int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, 
  * eta = e_q * fp32(log2(e) * softmax_scale).  Asynchronous on `stream`. */
 int fold_quantize_keys(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, const int32_t *first_token,
                        fold_stream stream);
+
+/* Cache write for the E4M3 value planes: for every sequence, kv head and token first_token[s] <= j < seqlens[s]
+ * (first_token as in fold_quantize_keys) read the BF16 value row from kv->v and write
+ *     p1 = e4m3(v / 2^v_scale_log2),   p2 = e4m3(v / 2^v_scale_log2 - p1)
+ * (round to nearest, ties to even, magnitudes beyond 448 saturate; both subtractions and the scaling are exact)
+ * into kv->v_plane_1 / v_plane_2 (DEVICE memory of the caller, written although the struct says const).  The scale
+ * is the caller's: 2^v_scale_log2 >= max|v| / 448 keeps plane 1 from saturating.  Asynchronous on `stream`. */
+int fold_quantize_values(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, const int32_t *first_token,
+                         fold_stream stream);
 
 /* The same decode for callers whose tensors live in HOST memory (pinned for the copies to
  * be asynchronous): q, kv.k, kv.v, kv.page_table, kv.seqlens, z (if GIVEN), out, lse and

@@ -33,7 +33,8 @@ class FoldKV(C.Structure):
                 ("mean_stride_head", C.c_int64),
                 ("k_plane_a", C.c_void_p), ("k_plane_b", C.c_void_p),
                 ("plane_stride_seq", C.c_int64), ("plane_stride_tok", C.c_int64), ("plane_stride_head", C.c_int64),
-                ("k_scale", C.c_void_p), ("scale_stride_seq", C.c_int64), ("scale_stride_head", C.c_int64)]
+                ("k_scale", C.c_void_p), ("scale_stride_seq", C.c_int64), ("scale_stride_head", C.c_int64),
+                ("v_plane_1", C.c_void_p), ("v_plane_2", C.c_void_p), ("v_scale_log2", C.c_int32)]
 
 
 class FoldArgs(C.Structure):
@@ -45,7 +46,8 @@ class FoldArgs(C.Structure):
                 ("depth_T", C.c_float), ("num_splits", C.c_int32),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("out", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p),
-                ("draft_mask", C.c_void_p), ("draft_len", C.c_int32), ("refine_tau", C.c_float)]
+                ("draft_mask", C.c_void_p), ("draft_len", C.c_int32), ("refine_tau", C.c_float),
+                ("refine_tau_v", C.c_float)]
 
 
 class FoldPartials(C.Structure):
@@ -59,12 +61,13 @@ class FoldPartials(C.Structure):
 class FoldWsHeader(C.Structure):
     _fields_ = [("wait_timeouts", C.c_uint32), ("reserved", C.c_uint32),
                 ("v_rows_fetched", C.c_uint64), ("v_rows_total", C.c_uint64),
-                ("v_slices_skipped", C.c_uint64), ("k_rows_refined", C.c_uint64), ("pad", C.c_uint64 * 3)]
+                ("v_slices_skipped", C.c_uint64), ("k_rows_refined", C.c_uint64), ("v2_rows_refined", C.c_uint64),
+                ("pad", C.c_uint64 * 2)]
 
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
            "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
-           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_quantize_keys", "fold_status_string",
+           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_quantize_keys", "fold_quantize_values", "fold_status_string",
            "fold_version"]
 
 _lib = None
@@ -97,6 +100,8 @@ def lib() -> C.CDLL:
         L.fold_block_means.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p]
         L.fold_quantize_keys.restype = C.c_int
         L.fold_quantize_keys.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.fold_quantize_values.restype = C.c_int
+        L.fold_quantize_values.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.fold_status_string.restype = C.c_char_p; L.fold_status_string.argtypes = [C.c_int]
         L.fold_version.restype = C.c_int
         _lib = L
@@ -139,6 +144,10 @@ class KVCache:
     k_plane_a: Optional[torch.Tensor] = None
     k_plane_b: Optional[torch.Tensor] = None
     k_scale: Optional[torch.Tensor] = None
+    # two E4M3 value planes (uint8, shaped and strided like the key planes) under the scale 2^v_scale_log2
+    v_plane_1: Optional[torch.Tensor] = None
+    v_plane_2: Optional[torch.Tensor] = None
+    v_scale_log2: int = 0
 
     def to_c(self) -> FoldKV:
         k, v = self.k, self.v
@@ -184,6 +193,13 @@ class KVCache:
             kv.scale_stride_seq, kv.scale_stride_head = sc.stride(0), sc.stride(1)
         else:
             kv.k_plane_a = kv.k_plane_b = kv.k_scale = None
+        if self.v_plane_1 is not None:
+            p1, p2 = self.v_plane_1, self.v_plane_2
+            assert self.k_plane_a is not None and p1.dtype == torch.uint8 and p2.dtype == torch.uint8
+            assert p1.shape == k.shape and p2.shape == k.shape and p1.stride() == self.k_plane_a.stride() == p2.stride()
+            kv.v_plane_1, kv.v_plane_2, kv.v_scale_log2 = p1.data_ptr(), p2.data_ptr(), int(self.v_scale_log2)
+        else:
+            kv.v_plane_1 = kv.v_plane_2 = None
         return kv
 
     def alloc_key_planes(self) -> None:
@@ -205,7 +221,8 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
               z: Optional[torch.Tensor] = None, depth_T: float = math.inf, num_splits: int = 0, stack: int = 1,
               workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
               lse: Optional[torch.Tensor] = None, row_status: Optional[torch.Tensor] = None,
-              draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0) -> FoldArgs:
+              draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0,
+              refine_tau_v: float = 0.0) -> FoldArgs:
     assert q.dtype == torch.bfloat16 and q.dim() == 3 and q.stride(2) == 1
     B, Hq, D = q.shape
     a = FoldArgs()
@@ -227,6 +244,7 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
         assert draft_mask.is_contiguous()
     a.draft_mask, a.draft_len = (_ptr(draft_mask), int(draft_len)) if draft_len else (None, 0)
     a.refine_tau = float(refine_tau)
+    a.refine_tau_v = float(refine_tau_v)
     return a
 
 
@@ -281,6 +299,19 @@ def fold_quantize_keys(cache: KVCache, first_token: Optional[torch.Tensor] = Non
     kv = cache.to_c()
     _check(lib().fold_quantize_keys(C.byref(kv), int(cache.k.shape[2]), int(cache.k.shape[3]), _ptr(first_token),
                                     _stream(stream)), "fold_quantize_keys")
+
+
+def fold_quantize_values(cache: KVCache, scale_log2: int, first_token: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Cache write for the E4M3 value planes (allocated here if absent; the key planes must exist): p1, p2 of every
+    value row of tokens first_token[s] .. seqlens[s]-1 under the scale 2^scale_log2."""
+    assert cache.k_plane_a is not None, "E4M3 value planes go with two-plane keys"
+    if cache.v_plane_1 is None:
+        cache.v_plane_1 = torch.zeros(cache.k.shape, dtype=torch.uint8, device=cache.k.device)
+        cache.v_plane_2 = torch.zeros(cache.k.shape, dtype=torch.uint8, device=cache.k.device)
+    cache.v_scale_log2 = int(scale_log2)
+    kv = cache.to_c()
+    _check(lib().fold_quantize_values(C.byref(kv), int(cache.k.shape[2]), int(cache.k.shape[3]), _ptr(first_token),
+                                      _stream(stream)), "fold_quantize_values")
 
 
 def fold_decode(args: FoldArgs, stream=None) -> None:
@@ -341,10 +372,10 @@ def alloc_buffers(q: torch.Tensor, cache: KVCache, stack: int = 1) -> DecodeBuff
 def decode(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, depth_T: float = math.inf,
            z_mode: int = Z_ESTIMATE, num_splits: int = 0, scale: Optional[float] = None, stack: int = 1,
            draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0,
-           stream=None) -> FoldArgs:
+           refine_tau_v: float = 0.0, stream=None) -> FoldArgs:
     args = make_args(q, cache, scale=scale, z_mode=z_mode, z=bufs.z, depth_T=depth_T, num_splits=num_splits,
                      stack=stack, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status,
-                     draft_mask=draft_mask, draft_len=draft_len, refine_tau=refine_tau)
+                     draft_mask=draft_mask, draft_len=draft_len, refine_tau=refine_tau, refine_tau_v=refine_tau_v)
     fold_decode(args, stream)
     return args
 

@@ -39,8 +39,13 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline size_t qplane_bytes(long long rows, int D) { return round_up((size_t)rows * 2 * D, 256) + round_up((size_t)rows * 4, 256); }
 
 int check_kv(const fold_kv &kv, int D) {
-  const bool planes = kv.k_plane_a != nullptr;
-  if ((!kv.k && !planes) || !kv.v || !kv.seqlens) return FOLD_EINVAL;
+  const bool planes = kv.k_plane_a != nullptr, vplanes = kv.v_plane_1 != nullptr;
+  if ((!kv.k && !planes) || (!kv.v && !vplanes) || !kv.seqlens) return FOLD_EINVAL;
+  if (vplanes) {
+    if (!planes) return FOLD_EUNSUPPORTED;                   // the E4M3 value planes go with the two-plane keys
+    if (!kv.v_plane_2 || !aligned(kv.v_plane_1, 16) || !aligned(kv.v_plane_2, 16)) return FOLD_EINVAL;
+    if (kv.v_scale_log2 < -100 || kv.v_scale_log2 > 100) return FOLD_EINVAL;
+  }
   if (!aligned(kv.k, 16) || !aligned(kv.v, 16)) return FOLD_EINVAL;
   if (planes) {
     if (!kv.k_plane_b || !kv.k_scale) return FOLD_EINVAL;
@@ -101,6 +106,10 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
     if (isnan(a->refine_tau)) return FOLD_EINVAL;
     // the two-plane scan: one 8-row block, no exact-maximum pass
     if (R > kNarrowRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
+    if (a->kv.v_plane_1) {
+      if (isnan(a->refine_tau_v)) return FOLD_EINVAL;
+      if (a->draft_len > 0 || (a->kv.v_block_mean && !isinf(a->depth_T))) return FOLD_EUNSUPPORTED;
+    }
   }
   return FOLD_OK;
 }
@@ -234,6 +243,8 @@ PlaneView plane_view(const fold_kv &kv) {
   v.max_pages = kv.max_pages_per_seq;
   v.num_pages = kv.num_pages > 0 ? kv.num_pages : 1;
   v.max_seqlen = kv.max_seqlen;
+  v.v1 = kv.v_plane_1; v.v2 = kv.v_plane_2;
+  v.v_scale = ldexpf(1.f, kv.v_scale_log2);
   return v;
 }
 
@@ -476,7 +487,7 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
 }
 
 // As many plane-A stages as fit beside the gather buffers with kPlaneCtasPerSm CTAs on an SM.
-template <int D, bool DRAFTS, bool TAIL>
+template <int D, bool DRAFTS, bool TAIL, bool VFP8 = false>
 int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
   using LO = PlaneLayout<D, TAIL>;
   const int per_cta = kSmemPerSm / kPlaneCtasPerSm - kSmemCtaReserve;
@@ -485,14 +496,15 @@ int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanPara
   if (stages < 2) return FOLD_EUNSUPPORTED;
   pp.s.stages = stages;
   static int configured[64] = {0};
-  if (int rc = opt_in_smem(fold_scan_planes_kernel<D, DRAFTS, TAIL>, configured)) return rc;
-  if (launch_pdl(fold_scan_planes_kernel<D, DRAFTS, TAIL>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) !=
+  if (int rc = opt_in_smem(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8>, configured)) return rc;
+  if (launch_pdl(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) !=
       cudaSuccess)
     return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 template <int D>
 int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
+  if (pp.kv.v1) return launch_planes_as<D, false, false, true>(ma, mv, pp, grid, st);    // E4M3 values: no drafts, no tail
   const bool drafts = pp.s.draft_len > 0, tail = pp.s.vmean != nullptr;      // (separate instantiations: registers)
   if (drafts) return tail ? launch_planes_as<D, true, true>(ma, mv, pp, grid, st) : launch_planes_as<D, true, false>(ma, mv, pp, grid, st);
   return tail ? launch_planes_as<D, false, true>(ma, mv, pp, grid, st) : launch_planes_as<D, false, false>(ma, mv, pp, grid, st);
@@ -507,9 +519,10 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   CUtensorMap ma;
   MapAxes axes;
   if (int rc = make_plane_map(&ma, &axes, kv, g.D, g.Hkv, box_tok)) return rc;
-  CUtensorMap mv;                                            // value rows of one 16-key sub-slice as a box
-  MapAxes vaxes;
-  if (int rc = make_map(&mv, &vaxes, kv.v, kv, g.D, g.Hkv, 16)) return rc;
+  CUtensorMap mv = ma;                                       // value rows of one 16-key sub-slice as a box (BF16 values)
+  MapAxes vaxes = axes;
+  if (!kv.v_plane_1)
+    if (int rc = make_map(&mv, &vaxes, kv.v, kv, g.D, g.Hkv, 16)) return rc;
   PlaneScanParams pp;
   memset(&pp, 0, sizeof(pp));
   pp.vpos_tok = vaxes.pos_tok; pp.vpos_head = vaxes.pos_head; pp.vpos_seq = vaxes.pos_seq;
@@ -546,6 +559,8 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   uint8_t *ws = static_cast<uint8_t *>(a->workspace);
   pp.qplanes = reinterpret_cast<const int8_t *>(ws + g.q_off);
   pp.qeta = reinterpret_cast<const float *>(ws + g.q_off + round_up((size_t)g.B * g.Hq * 2 * g.D, 256));
+  pp.auto_tau_v = a->refine_tau_v == 0.f;
+  pp.neg_tau_v = a->refine_tau_v < 0.f ? INFINITY : -a->refine_tau_v;
   pp.auto_tau = a->refine_tau == 0.f;
   pp.neg_tau = a->refine_tau < 0.f ? INFINITY : -a->refine_tau;      // tau = inf -> -inf: every live key
   const dim3 grid(g.Hkv, p.num_splits, g.num_seqs);
@@ -855,6 +870,28 @@ int fold_quantize_keys(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (head_dim == 128) fold_quantize_keys_kernel<128><<<grid, block, 0, st>>>(p);
   else fold_quantize_keys_kernel<64><<<grid, block, 0, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+int fold_quantize_values(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, const int32_t *first_token,
+                         fold_stream stream) {
+  if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
+  if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
+  if (!kv->v || !kv->v_plane_1) return FOLD_EINVAL;
+  if (int rc = check_kv(*kv, head_dim)) return rc;
+  if (kv->max_seqlen == 0) return FOLD_OK;
+  QuantValueParams p;
+  memset(&p, 0, sizeof(p));
+  p.v = static_cast<const __nv_bfloat16 *>(kv->v);
+  p.v_stride_seq = kv->stride_seq; p.v_stride_tok = kv->stride_tok; p.v_stride_head = kv->stride_head;
+  p.kv = plane_view(*kv);
+  p.first_token = first_token;
+  p.inv_scale = ldexpf(1.f, -kv->v_scale_log2);
+  const dim3 grid((kv->max_seqlen + kQuantRowsPerCta - 1) / kQuantRowsPerCta, num_kv_heads, kv->num_seqs);
+  const dim3 block(32, kQuantRowsPerCta);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (head_dim == 128) fold_quantize_values_kernel<128><<<grid, block, 0, st>>>(p);
+  else fold_quantize_values_kernel<64><<<grid, block, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 

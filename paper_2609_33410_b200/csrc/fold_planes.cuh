@@ -10,6 +10,9 @@
 //                 INT8 product adds plane B; final FP32 weights feed the BF16 value product.
 #pragma once
 
+#include <cuda_fp8.h>
+#include <cuda_fp16.h>
+
 #include "fold_common.cuh"
 #include "fold_estimate.cuh"
 #include "fold_scan.cuh"
@@ -25,6 +28,8 @@ struct PlaneView {
   const int *page_table;
   const int *seqlens;
   int paged, page_shift, max_pages, num_pages, max_seqlen;
+  const uint8_t *v1, *v2;                                     // E4M3 value planes (strides as a / b), or null
+  float v_scale;                                              // 2^v_scale_log2
 };
 
 // (sequence-or-page, token-in-it) of logical token j
@@ -142,6 +147,42 @@ __global__ void __launch_bounds__(32 * kQuantRowsPerCta) fold_quantize_keys_kern
         __float2bfloat16_rn(e);                              // exact: e is a BF16 value
 }
 
+// Cache write of the E4M3 value planes: p1 = e4m3(v / scale), p2 = e4m3(v / scale - p1), one warp per row.
+struct QuantValueParams {
+  const __nv_bfloat16 *v;
+  long long v_stride_seq, v_stride_tok, v_stride_head;
+  PlaneView kv;                                               // destinations v1 / v2 (written)
+  const int *first_token;
+  float inv_scale;                                            // 2^-v_scale_log2
+};
+template <int D>
+__global__ void __launch_bounds__(32 * kQuantRowsPerCta) fold_quantize_values_kernel(const QuantValueParams p) {
+  constexpr int EPL = D / 32;
+  const int lane = threadIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
+  int n = p.kv.seqlens[seq];
+  n = n < 0 ? 0 : (n > p.kv.max_seqlen ? p.kv.max_seqlen : n);
+  const int first = p.first_token ? max(p.first_token[seq], 0) : 0;
+  const int j = first + blockIdx.x * kQuantRowsPerCta + threadIdx.y;
+  if (j >= n) return;
+  long long s, t;
+  plane_locate(p.kv, seq, j, s, t);
+  float x[EPL];
+  load_bf16_row<EPL>(p.v + s * p.v_stride_seq + t * p.v_stride_tok + (long long)kvh * p.v_stride_head + lane * EPL, x);
+  int c1[EPL], c2[EPL];
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const float y = __fmul_rn(x[i], p.inv_scale);             // exact: a power of two
+    const __nv_fp8_storage_t a = __nv_cvt_float_to_fp8(y, __NV_SATFINITE, __NV_E4M3);
+    const float ya = __half2float(__half(__nv_cvt_fp8_to_halfraw(a, __NV_E4M3)));
+    const __nv_fp8_storage_t b = __nv_cvt_float_to_fp8(__fsub_rn(y, ya), __NV_SATFINITE, __NV_E4M3);   // exact difference
+    c1[i] = (int)a;
+    c2[i] = (int)b;
+  }
+  const long long off = s * p.kv.stride_seq + t * p.kv.stride_tok + (long long)kvh * p.kv.stride_head + lane * EPL;
+  store_codes<EPL>(reinterpret_cast<int8_t *>(const_cast<uint8_t *>(p.kv.v1)) + off, c1);
+  store_codes<EPL>(reinterpret_cast<int8_t *>(const_cast<uint8_t *>(p.kv.v2)) + off, c2);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Front kernel: one CTA per (kv head, request).  Splits the group's query rows (rows of the workspace:
 // [request * Hq + head][2][D] codes and one eta = e_q * scale_log2 per row), then, if the reference is to be
@@ -251,6 +292,8 @@ struct PlaneScanParams {
   int vpos_tok, vpos_head, vpos_seq;                          // coordinate order of the value tensor map
   int box_min;                                                // value rows of a sub-slice come as one box from this many live keys on
   float neg_tau;                                              // -tau_K; -inf: refine every live key; +inf: none
+  float neg_tau_v;                                            // the same for the refine-V gate (E4M3 value planes)
+  int auto_tau_v;                                             // tau_V = max(log2(n) + 1, 4)
   int auto_tau;                                               // tau_K = max(log2(n) - 2, 4) from the sequence's own length
 };
 
@@ -374,13 +417,15 @@ struct PlanePending {
   float x[4];            // coarse score minus reference: key lane/4 (+8), rows (lane%4)*2 + {0,1}; -inf if unused
   float e[2];            // the two keys' scales
   uint32_t live, refine; // verdict bits of the 16 keys, ORed over the rows
+  uint32_t refv;         // E4M3 value planes: keys whose second value plane is read
   int buf;               // the gather buffer its rows land in
   int ms;                // block tail: the ring slot of its tile's mean value row
 };
 
 // DRAFTS: the rows carry draft masks (a separate instantiation: the plain one is at its register limit).
 // TAIL: cut keys add weight x the mean value row of their 64-key block (Section 4, "Depth as a dial").
-template <int D, bool DRAFTS, bool TAIL>
+// VFP8: values come from two E4M3 planes (plane 1 for live keys, plane 2 for refine-V keys), widened to BF16 in place.
+template <int D, bool DRAFTS, bool TAIL, bool VFP8 = false>
 __global__ void __launch_bounds__(kDenseThreads, kPlaneCtasPerSm)
 fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmV,
                         const PlaneScanParams pp) {
@@ -449,6 +494,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   const int dstart = DRAFTS ? draft_start(p, n) : n;         // keys from here on are per-request drafts
   const float neg_T = p.neg_T;
   const float neg_tau = pp.auto_tau ? -fmaxf(log2f((float)max(n, 1)) - 2.f, 4.f) : pp.neg_tau;
+  const float neg_tau_v = pp.auto_tau_v ? -fmaxf(log2f((float)max(n, 1)) + 1.f, 4.f) : pp.neg_tau_v;
 
   float o[D / 16][4];
 #pragma unroll
@@ -521,13 +567,51 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       bh[kh] = movmatrix_trans(hi2);
       bl[kh] = movmatrix_trans(lo2);
     }
+    if (VFP8 && pd.live) {
+      // widen the landed E4M3 rows to BF16 in place: all reads (two planes, D / 32 units of 16 codes per lane), then
+      // all writes into the [D/64][16][128 B] swizzled layout the value product reads.  v1 and v2 widen exactly (to
+      // FP16 here), their sum is exact in FP16 and is rounded to BF16 once; rows of keys that are not live become zeros.
+      constexpr int UPL = CB / 2;                            // units per lane and plane
+      uint4 w1[UPL], w2[UPL];
+      uint8_t *vb = gen + (vbuf - base);
+#pragma unroll
+      for (int i = 0; i < UPL; ++i) {
+        const int idx = lane + 32 * i, key = idx / CB, u = idx % CB;
+        const bool lv = (pd.live >> key) & 1u, r2 = (pd.refv >> key) & 1u;
+        w1[i] = lv ? *reinterpret_cast<const uint4 *>(vb + key * D + u * 16) : make_uint4(0, 0, 0, 0);
+        w2[i] = r2 ? *reinterpret_cast<const uint4 *>(vb + 16 * D + key * D + u * 16) : make_uint4(0, 0, 0, 0);
+      }
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < UPL; ++i) {
+        const int idx = lane + 32 * i, key = idx / CB, u = idx % CB;
+        const uint32_t a[4] = {w1[i].x, w1[i].y, w1[i].z, w1[i].w}, b[4] = {w2[i].x, w2[i].y, w2[i].z, w2[i].w};
+        uint32_t outw[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+          for (int hl = 0; hl < 2; ++hl) {
+            const __half2 h1 = __half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(a[j] >> (16 * hl)), __NV_E4M3));
+            const __half2 h2 = __half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(b[j] >> (16 * hl)), __NV_E4M3));
+            const float2 f = __half22float2(__hadd2(h1, h2));
+            outw[2 * j + hl] = pack_bf16(f.x * pp.kv.v_scale, f.y * pp.kv.v_scale);
+          }
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+          const int oc = 2 * u + c2;                          // 16-byte chunk of the BF16 row: channels 8 oc .. 8 oc + 7
+          *reinterpret_cast<uint4 *>(vb + (oc >> 3) * (16 * 128) + key * 128 + (((oc & 7) ^ (key & 7)) << 4)) =
+              make_uint4(outw[4 * c2], outw[4 * c2 + 1], outw[4 * c2 + 2], outw[4 * c2 + 3]);
+        }
+      }
+      __syncwarp();
+    }
     if (pd.live) value_product_n<D, true, 0, 16>(o, vbuf, 0, lane, bh, bl);
     if (TAIL) add_tail(cut0, cut1, pd.ms);
   };
 
   int stage = 0, buf = 0, n_pend = 0, mslot = 0;
   uint32_t phase = 0;
-  unsigned long long st_total = 0, st_live = 0, st_ref = 0;
+  unsigned long long st_total = 0, st_live = 0, st_ref = 0, st_refv = 0;
   PlanePending pend[LO::kBufs - 1];
   const int page_mask = (1 << p.page_shift) - 1;
   const uint64_t vpol = policy_evict_first();
@@ -552,7 +636,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         PlanePending cur;
         int ca[4], cb[4];
         plane_products<D>(at, sub * 16, lane, qa, qb, ca, cb);
-        uint32_t lm = 0, rm = 0;
+        uint32_t lm = 0, rm = 0, vm = 0;
 #pragma unroll
         for (int kh = 0; kh < 2; ++kh) {
           const int key = key0 + klo + 8 * kh;
@@ -566,10 +650,13 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             cur.x[i] = x;
             if (ok && x >= neg_T) lm |= 1u << (klo + 8 * kh);
             if (ok && x >= neg_tau) rm |= 1u << (klo + 8 * kh);
+            if (VFP8 && ok && x >= neg_tau_v) vm |= 1u << (klo + 8 * kh);
           }
         }
         cur.live = __reduce_or_sync(0xffffffffu, lm);
         cur.refine = __reduce_or_sync(0xffffffffu, rm) & cur.live;
+        cur.refv = VFP8 ? __reduce_or_sync(0xffffffffu, vm) & cur.live : 0u;
+        if (VFP8) st_refv += __popc(cur.refv);
         cur.buf = buf;
         cur.ms = my_ms;
         st_live += __popc(cur.live);
@@ -610,8 +697,23 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
               s_row = min(max(p.page_table[(long long)seq * p.max_pages + (key0 >> p.page_shift)], 0), p.num_pages - 1);
               t_row = key0 & page_mask;
             }
-            const bool box = __popc(cur.live) >= pp.box_min && key0 + 16 <= n;
-            if (box) {
+            const bool box = !VFP8 && __popc(cur.live) >= pp.box_min && key0 + 16 <= n;
+            if (VFP8) {
+              // E4M3 planes: plane-1 rows of live keys into the first half of the value buffer (16 rows of D bytes),
+              // plane-2 rows of refine-V keys into the second half; the second pass widens them in place
+              constexpr int BK = 32 / CB;
+              const int ch = lane % CB, k0 = lane / CB;
+              const long long off = s_row * pp.kv.stride_seq + (t_row + k0) * pp.kv.stride_tok + (long long)kvh * pp.kv.stride_head + ch * 16;
+              const uint8_t *s1 = pp.kv.v1 + off, *s2 = pp.kv.v2 + off;
+#pragma unroll
+              for (int i = 0; i < 16 / BK; ++i) {
+                const int key = k0 + i * BK;
+                if ((cur.live >> key) & 1u) cp_async_16(vbuf + key * D + ch * 16, s1, 16u);
+                if ((cur.refv >> key) & 1u) cp_async_16(vbuf + 16 * D + key * D + ch * 16, s2, 16u);
+                s1 += BK * pp.kv.stride_tok;
+                s2 += BK * pp.kv.stride_tok;
+              }
+            } else if (box) {
               fence_proxy_async_smem();                       // the buffer's earlier generic-proxy traffic, then TMA writes
               __syncwarp();
               if (lane == 0) {
@@ -682,6 +784,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), st_live);
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
     atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->k_rows_refined), st_ref);
+    if (VFP8) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v2_rows_refined), st_refv);
   }
 }
 

@@ -63,20 +63,39 @@ def with_means(cache, vm):
                      cache.k_plane_b, cache.k_scale)
 
 
-def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, draft=None):
+def value_planes_of(w, cache):
+    """Quantize the values into two E4M3 planes under the smallest power-of-two scale that keeps plane 1 unsaturated."""
+    vmax = float(torch.nan_to_num(w.v.float(), nan=0.0).abs().max())          # (padding rows may be poisoned with NaN)
+    k = int(math.ceil(math.log2(max(vmax, 1e-30) / 448.0)))
+    F.fold_quantize_values(cache, k)
+    torch.cuda.synchronize()
+    return cache
+
+
+def logical_value_planes(w, cache, seq, kvh):
+    n = int(w.seqlens[seq])
+    j = torch.arange(n, device=cache.k.device)
+    if w.paged:
+        ps = cache.k.shape[1]
+        pg = w.page_table[seq].long()[j // ps]
+        return cache.v_plane_1[pg, j % ps, kvh].cpu().numpy(), cache.v_plane_2[pg, j % ps, kvh].cpu().numpy()
+    return cache.v_plane_1[seq, :n, kvh].cpu().numpy(), cache.v_plane_2[seq, :n, kvh].cpu().numpy()
+
+
+def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, draft=None, tau_v=0.0):
     """`draft` = (masks int32 [batch], draft_len): draft / tree-verification rows."""
     bufs = F.alloc_buffers(w.q, cache, w.stack)
     if z is not None:
         bufs.z.copy_(z)
     F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale, refine_tau=tau,
-             draft_mask=None if draft is None else draft[0], draft_len=0 if draft is None else draft[1])
+             refine_tau_v=tau_v, draft_mask=None if draft is None else draft[0], draft_len=0 if draft is None else draft[1])
     torch.cuda.synchronize()
     assert bufs.header().wait_timeouts == 0
     return bufs
 
 
 def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estimate=False, check_counts=True, draft=None,
-                   v_block_mean=None):
+                   v_block_mean=None, tau_v=0.0):
     """`v_block_mean`: the table the GPU was given (block tail); a key that flips at a gate then moves between its value
     and its block's mean, so the threshold slack counts twice."""
     vmt = None if v_block_mean is None else v_block_mean.float().cpu().numpy().astype(np.float64)
@@ -92,7 +111,8 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
     num = den = ynum = slack2 = 0.0
     max_abs = vmax = dz = 0.0
     rel_rows = []
-    n_live = n_ref = n_keys = 0
+    n_live = n_ref = n_keys = n_refv = 0
+    vfp8 = cache.v_plane_1 is not None
     for (seq, kvh) in units:
         n = int(w.seqlens[seq])
         rows = [(seq * w.stack + r // G, kvh * G + r % G) for r in range(R)]
@@ -109,7 +129,14 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
         tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
         vis = None if draft is None else np.stack([O.draft_visible(n, draft[1], dmask[b]) for (b, h) in rows])
         vm = None if vmt is None else vmt[seq, :(n + 63) // 64, kvh]
-        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis, v_mean=vm)
+        vpl, tau_v_eff = None, None
+        if vfp8:
+            p1, p2 = logical_value_planes(w, cache, seq, kvh)
+            vpl = (p1, p2, cache.v_scale_log2)
+            tau_v_eff = P.auto_refine_tau_v(n) if tau_v == 0.0 else tau_v
+        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis, v_mean=vm,
+                                         value_planes=vpl, tau_v=tau_v_eff)
+        n_refv += int(info["refine_v"].sum())
         n_live += int(info["live"].sum()); n_ref += int(info["refine"].sum()); n_keys += n
         vinf = np.abs(V).max(axis=1)
         near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
@@ -156,6 +183,8 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
         assert h.v_rows_total == n_keys
         assert abs(h.v_rows_fetched - n_live) <= max(2, 2e-3 * n_keys), (h.v_rows_fetched, n_live)
         assert abs(h.k_rows_refined - n_ref) <= max(2, 2e-3 * n_keys), (h.k_rows_refined, n_ref)
+        if vfp8:
+            assert abs(h.v2_rows_refined - n_refv) <= max(2, 2e-3 * n_keys), (h.v2_rows_refined, n_refv)
     return res
 
 
@@ -443,3 +472,47 @@ def test_block_tail_on_two_plane_keys(Hq, Hkv, D, paged):
     t = run_planes(w, with_means(plain, vm2), T=6.0)
     ok = t.row_status.cpu().numpy() == 0
     assert np.allclose(t.out.float().cpu().numpy()[ok], 1.5, rtol=1e-2)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("paged", [False, True])
+def test_value_plane_writer_matches_the_oracle_bit_for_bit(D, paged):
+    w = make_decode_workload(3, 8, 2, D, [700, 64, 333], seed=103, device=DEV, paged=paged, page_size=32, poison_padding=True)
+    w.v[..., 5] *= 300.0                                         # a wide range: saturating and subnormal codes both occur
+    cache = plane_cache(w)
+    for k in (0, -3):
+        F.fold_quantize_values(cache, k)
+        torch.cuda.synchronize()
+        for seq in range(3):
+            for kvh in range(2):
+                p1, p2 = logical_value_planes(w, cache, seq, kvh)
+                r1, r2 = P.quantize_values(O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh))), k)
+                assert np.array_equal(p1, r1) and np.array_equal(p2, r2), (k, seq, kvh)
+    assert (p1 & 0x7f).max() == 0x7e and ((p1 & 0x78) == 0).any()
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,paged", [(8, 2, 128, False), (8, 8, 64, True), (4, 1, 128, True), (1, 1, 64, False)])
+def test_decode_on_e4m3_value_planes(Hq, Hkv, D, paged):
+    kw = dict(paged=True, page_size=32) if paged else dict(capacity=3100)
+    w = make_decode_workload(2, Hq, Hkv, D, [3000, 733], seed=107, device=DEV, poison_padding=True, **kw)
+    cache = value_planes_of(w, plane_cache(w))
+    for T, tau_v in ((math.inf, 0.0), (math.inf, math.inf), (16.0, 0.0), (12.0, -1.0), (6.0, 3.0)):
+        b = run_planes(w, cache, T=T, tau_v=tau_v)
+        r = compare_planes(w, cache, b, T=T, tau_v=tau_v, check_estimate=True)
+        s = run_planes(w, cache, T=T, tau_v=tau_v, num_splits=1)
+        assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse)
+    # the decode reads no BF16 value: the same bits with v taken away
+    nov = F.KVCache(w.k, w.v, w.seqlens, w.max_seqlen, w.page_table, None, cache.k_plane_a, cache.k_plane_b, cache.k_scale,
+                    cache.v_plane_1, cache.v_plane_2, cache.v_scale_log2)
+    bufs = F.alloc_buffers(w.q, nov)
+    args = F.make_args(w.q, nov, depth_T=16.0, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status)
+    args.kv.v = None; args.kv.k = None
+    F.fold_decode(args)
+    torch.cuda.synchronize()
+    ref = run_planes(w, cache, T=16.0)
+    assert same_bits(bufs.out, ref.out) and same_bits(bufs.lse, ref.lse)
+    # with every second plane read, the dense result is the BF16 result up to the planes' own step (2^-8 per value)
+    full = run_planes(w, cache, tau_v=math.inf)
+    plain = run_planes(w, plane_cache(w))
+    d = (full.out.float() - plain.out.float()).norm() / plain.out.float().norm()
+    assert float(d) < 5e-3
