@@ -301,7 +301,8 @@ def run_sweep(args, dev):
                 del w, cache, bufs, flush
                 torch.cuda.empty_cache()
     print(json.dumps({"sweep": "config5", "heads": 32, "peak_gbs": peak, "block_tail": bool(args.tail), "drafts": args.drafts,
-                      "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16", "cells": cells}))
+                      "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16",
+                   "value_format": "two E4M3 planes, power-of-two scale" if args.fp8v else "bf16", "cells": cells}))
 
 
 def main():
@@ -321,6 +322,10 @@ def main():
                     help="finite-depth steps use the block tail (cut keys add weight x block-mean value)")
     ap.add_argument("--planes", action="store_true",
                     help="keys as two INT8 planes + a BF16 scale per key (quantized once, outside the timed region)")
+    ap.add_argument("--fp8v", action="store_true",
+                    help="--planes: values as two E4M3 planes under a power-of-two scale (quantized outside the timed region)")
+    ap.add_argument("--refine-tau-v", type=float, default=0.0,
+                    help="--fp8v: the refine-V gate in binades (0 = max(log2(n) + 1, 4); inf = every live key; negative = none)")
     ap.add_argument("--refine-tau", type=float, default=0.0,
                     help="--planes: the refine gate in binades (0 = max(log2(n) - 2, 4); inf = every live key; negative = none)")
     ap.add_argument("--graph", action="store_true",
@@ -392,6 +397,17 @@ def main():
         e1.record(stream)
         torch.cuda.synchronize()
         quant_ms = e0.elapsed_time(e1)
+        if args.fp8v:
+            vmax = float(levels[0].v.float().abs().max())
+            vk = int(math.ceil(math.log2(max(vmax, 1e-30) / 448.0)))
+            F.fold_quantize_values(caches[0], vk, None, stream)
+            e0.record(stream)
+            F.fold_quantize_values(caches[0], vk, None, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            quant_ms += e0.elapsed_time(e1)
+    elif args.fp8v:
+        raise SystemExit("--fp8v goes with --planes")
     lbufs = [F.alloc_buffers(l.q, c, l.stack) for l, c in zip(levels, caches)]
     bufs = lbufs[-1]
     cache_bytes = sum(l.cache_bytes() for l in levels)                    # unique bytes: a shared prefix counts once
@@ -401,7 +417,8 @@ def main():
         return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
                             num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
                             row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
-                            draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau)
+                            draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau,
+                            refine_tau_v=args.refine_tau_v)
                 for l, c, b in zip(levels, caches, lbufs)]
 
     # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
@@ -440,7 +457,8 @@ def main():
     def headers():
         hs = [b.header() for b in lbufs]
         return dict(fetched=[h.v_rows_fetched for h in hs], total=[h.v_rows_total for h in hs],
-                    refined=[h.k_rows_refined for h in hs], timeouts=sum(h.wait_timeouts for h in hs))
+                    refined=[h.k_rows_refined for h in hs], refined_v=[h.v2_rows_refined for h in hs],
+                    timeouts=sum(h.wait_timeouts for h in hs))
 
     def timed(depth, steps, warmup, sample_clocks):
         # (1) whole steps: estimate -> scan(s) -> partial add, chained in the stream by one C-ABI call
@@ -520,11 +538,17 @@ def main():
     def refined_frac(r):
         return sum(r["refined"]) / max(sum(r["total"]), 1)
 
+    def refined_v_frac(r):
+        return sum(r["refined_v"]) / max(sum(r["total"]), 1)
+
+    def value_bytes(r):                                   # per key: BF16 rows of live keys, or plane 1 + the refined share of plane 2
+        return D * fetched_frac(r) + D * refined_v_frac(r) if args.fp8v else 2 * D * fetched_frac(r)
+
     def actual_bytes(r):                                  # K in full + the fetched share of V + slots written, all levels
         # (from the fetched FRACTION: row groups of one kv head count their keys once each, but share the tiles in L2)
         if args.planes:                                   # per key: plane A + scale, the refined share of plane B, the live share of V
             keys = cache_bytes // (4 * D)
-            return int(keys * ((D + 2) + D * refined_frac(r) + 2 * D * fetched_frac(r))) + slot_bytes
+            return int(keys * ((D + 2) + D * refined_frac(r) + value_bytes(r))) + slot_bytes
         return cache_bytes // 2 + int(cache_bytes // 2 * fetched_frac(r)) + slot_bytes
 
     peak, peak_src = load_peaks()
@@ -546,6 +570,7 @@ def main():
                    "cascade_streams": args.cascade_streams if cascade else None,
                    "cuda_graph": bool(args.graph), "block_tail": bool(args.tail),
                    "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16",
+                   "value_format": "two E4M3 planes, power-of-two scale" if args.fp8v else "bf16",
                    "refine_tau": (args.refine_tau or "auto: max(log2(n) - 2, 4)") if args.planes else None,
                    "flat_equivalent_bytes_per_gpu": flat_bytes},
         "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
@@ -555,8 +580,9 @@ def main():
         "v_rows_fetched_frac": {"T16": fetched_frac(r16), "Tinf": fetched_frac(rinf)},
         "planes": None if not args.planes else {
             "k_rows_refined_frac": {"T16": refined_frac(r16), "Tinf": refined_frac(rinf)},
-            "bytes_per_key": {"T16": (D + 2) + D * refined_frac(r16) + 2 * D * fetched_frac(r16),
-                              "Tinf": (D + 2) + D * refined_frac(rinf) + 2 * D * fetched_frac(rinf), "bf16_cache": 4 * D},
+            "v2_rows_refined_frac": {"T16": refined_v_frac(r16), "Tinf": refined_v_frac(rinf)} if args.fp8v else None,
+            "bytes_per_key": {"T16": (D + 2) + D * refined_frac(r16) + value_bytes(r16),
+                              "Tinf": (D + 2) + D * refined_frac(rinf) + value_bytes(rinf), "bf16_cache": 4 * D},
             "cache_write_ms": quant_ms},
         "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
                      "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src,

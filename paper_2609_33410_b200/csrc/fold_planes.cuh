@@ -564,16 +564,26 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       l_lo += (h0 + g0) + (pw[0] - pm[0]);
       l_hi += (h1 + g1) + (pw[1] - pm[1]);
       if (TAIL) { cut0 += pw[0] - pm[0]; cut1 += pw[1] - pm[1]; }
-      bh[kh] = movmatrix_trans(hi2);
-      bl[kh] = movmatrix_trans(lo2);
+      if (VFP8) {
+        // E4M3 values enter the product without their power-of-two scale: it multiplies the weights' BF16 terms instead
+        // (exactly: a power of two), while L keeps the weights themselves
+        const float vs = pp.kv.v_scale;
+        bh[kh] = movmatrix_trans(pack_bf16(h0 * vs, h1 * vs));
+        bl[kh] = movmatrix_trans(pack_bf16(g0 * vs, g1 * vs));
+      } else {
+        bh[kh] = movmatrix_trans(hi2);
+        bl[kh] = movmatrix_trans(lo2);
+      }
     }
     if (VFP8 && pd.live) {
       // widen the landed E4M3 rows to BF16 in place: all reads (two planes, D / 32 units of 16 codes per lane), then
       // all writes into the [D/64][16][128 B] swizzled layout the value product reads.  v1 and v2 widen exactly (to
       // FP16 here), their sum is exact in FP16 and is rounded to BF16 once; rows of keys that are not live become zeros.
       constexpr int UPL = CB / 2;                            // units per lane and plane
+      // (the planes' power-of-two scale rides on the weights instead: see the weights above)
       uint4 w1[UPL], w2[UPL];
       uint8_t *vb = gen + (vbuf - base);
+      const bool any2 = pd.refv != 0u;                       // warp-uniform: is any second plane there at all?
 #pragma unroll
       for (int i = 0; i < UPL; ++i) {
         const int idx = lane + 32 * i, key = idx / CB, u = idx % CB;
@@ -591,10 +601,10 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         for (int j = 0; j < 4; ++j)
 #pragma unroll
           for (int hl = 0; hl < 2; ++hl) {
-            const __half2 h1 = __half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(a[j] >> (16 * hl)), __NV_E4M3));
-            const __half2 h2 = __half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(b[j] >> (16 * hl)), __NV_E4M3));
-            const float2 f = __half22float2(__hadd2(h1, h2));
-            outw[2 * j + hl] = pack_bf16(f.x * pp.kv.v_scale, f.y * pp.kv.v_scale);
+            __half2 h = __half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(a[j] >> (16 * hl)), __NV_E4M3));
+            if (any2) h = __hadd2(h, __half2(__nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(b[j] >> (16 * hl)), __NV_E4M3)));
+            const float2 f = __half22float2(h);
+            outw[2 * j + hl] = pack_bf16(f.x, f.y);
           }
 #pragma unroll
         for (int c2 = 0; c2 < 2; ++c2) {
