@@ -194,3 +194,37 @@ def test_host_checks_of_two_plane_keys():
     kv = F.FoldKV()
     assert L.fold_quantize_keys(kv, 2, 96, None, None) == F.FOLD_EUNSUPPORTED
     assert L.fold_quantize_keys(kv, 2, 128, None, None) == F.FOLD_EINVAL  # nothing to read or write
+
+
+def test_host_checks_of_e4m3_value_planes():
+    L = F.lib()
+    a, keep = _cpu_args()
+    k = keep[1]
+    pa, pb = torch.zeros(k.shape, dtype=torch.int8), torch.zeros(k.shape, dtype=torch.int8)
+    sc = torch.zeros(k.shape[0], k.shape[2], 1024, dtype=torch.bfloat16)
+    v1, v2 = torch.zeros(k.shape, dtype=torch.uint8), torch.zeros(k.shape, dtype=torch.uint8)
+    a.kv.v_plane_1, a.kv.v_plane_2 = v1.data_ptr(), v2.data_ptr()
+    ws = torch.zeros(1 << 20, dtype=torch.uint8)
+    a.workspace = ws.data_ptr() + ((-ws.data_ptr()) % 256)
+    a.workspace_bytes = ws.numel() - 256
+    assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED             # value planes without the two-plane keys
+    a.kv.k_plane_a, a.kv.k_plane_b, a.kv.k_scale = pa.data_ptr(), pb.data_ptr(), sc.data_ptr()
+    a.kv.plane_stride_seq, a.kv.plane_stride_tok, a.kv.plane_stride_head = pa.stride(0), pa.stride(1), pa.stride(2)
+    a.kv.scale_stride_seq, a.kv.scale_stride_head = sc.stride(0), sc.stride(1)
+    for field, value, want in [("v_plane_2", None, F.FOLD_EINVAL), ("v_plane_1", v1.data_ptr() + 8, F.FOLD_EINVAL),
+                               ("v_scale_log2", 500, F.FOLD_EINVAL)]:
+        old = getattr(a.kv, field)
+        setattr(a.kv, field, value)
+        assert L.fold_decode(a, None) == want, field
+        setattr(a.kv, field, old)
+    a.refine_tau_v = float("nan")
+    assert L.fold_decode(a, None) == F.FOLD_EINVAL
+    a.refine_tau_v = 0.0
+    masks = torch.ones(2, dtype=torch.int32)
+    a.draft_len, a.draft_mask = 1, masks.data_ptr()
+    assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED             # no draft rows on the value planes
+    a.draft_len, a.draft_mask = 0, None
+    kv = F.FoldKV()
+    assert L.fold_quantize_values(None, 2, 128, None, None) == F.FOLD_EINVAL
+    assert L.fold_quantize_values(kv, 2, 96, None, None) == F.FOLD_EUNSUPPORTED
+    assert L.fold_quantize_values(kv, 2, 128, None, None) == F.FOLD_EINVAL

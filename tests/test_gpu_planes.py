@@ -378,7 +378,7 @@ PLANE_LENGTHS = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255
 @pytest.mark.parametrize("seed", range(5))
 def test_random_shapes_match_the_oracle(seed):
     """Seeded random shapes of the two-plane path: head dimension, rows per kv head (1..8), lengths around every tile /
-    chunk / estimator boundary, paged or contiguous, depth, refine gate, block tail and draft masks drawn together."""
+    chunk / estimator boundary, paged or contiguous, depth, refine gates, block tail, draft masks and E4M3 value planes drawn together."""
     import random
     rnd = random.Random(7300 + seed)
     for i in range(8):
@@ -398,7 +398,9 @@ def test_random_shapes_match_the_oracle(seed):
             kw.update(capacity=max(lens) + rnd.choice([0, 5, 100]))
         tail = (not math.isinf(T)) and rnd.random() < 0.4
         drafts = stack > 1 and rnd.random() < 0.5
-        case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw, tail=tail, drafts=drafts)
+        vfp8 = (not tail) and (not drafts) and rnd.random() < 0.4
+        tau_v = rnd.choice([0.0, 0.0, -1.0, 5.0, math.inf])
+        case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw, tail=tail, drafts=drafts, vfp8=vfp8, tau_v=tau_v)
         draft = None
         if drafts:
             from paper_2609_33410_b200.workloads import make_draft_workload
@@ -412,10 +414,12 @@ def test_random_shapes_match_the_oracle(seed):
         vm = oracle_block_means(w) if tail else None
         if tail:
             cache = with_means(cache, vm)
+        if vfp8:
+            value_planes_of(w, cache)
         try:
-            b = run_planes(w, cache, T=T, tau=tau, draft=draft)
-            compare_planes(w, cache, b, T=T, tau=tau, check_estimate=True, draft=draft, v_block_mean=vm)
-            s = run_planes(w, cache, T=T, tau=tau, num_splits=rnd.choice([1, 2, 5]), draft=draft)
+            b = run_planes(w, cache, T=T, tau=tau, draft=draft, tau_v=tau_v)
+            compare_planes(w, cache, b, T=T, tau=tau, check_estimate=True, draft=draft, v_block_mean=vm, tau_v=tau_v)
+            s = run_planes(w, cache, T=T, tau=tau, num_splits=rnd.choice([1, 2, 5]), draft=draft, tau_v=tau_v)
             assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse), "split count changed a bit"
         except AssertionError as e:
             raise AssertionError(f"case {case}: {e}") from e
