@@ -108,7 +108,7 @@ enum {
  * plane_stride_* and paging).  A live key's plane-1 row is always read; its plane-2 row only when some row of
  * the group gives the key a coarse weight >= 2^-refine_tau_v ("refine V"): head_dim + head_dim * r_V bytes per live
  * key instead of 2 * head_dim.  The codes widen to BF16 exactly; v1 + v2 is rounded to BF16 once.  v may then be
- * NULL for the decode calls.  Not offered with draft masks or the block tail (FOLD_EUNSUPPORTED). */
+ * NULL for the decode calls.  Draft masks apply as on BF16 values; the block tail is not offered (FOLD_EUNSUPPORTED). */
 typedef struct fold_kv {
   const void *k, *v;
   int64_t stride_seq, stride_tok, stride_head;   /* elements */

@@ -108,7 +108,7 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
     if (R > kNarrowRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
     if (a->kv.v_plane_1) {
       if (isnan(a->refine_tau_v)) return FOLD_EINVAL;
-      if (a->draft_len > 0 || (a->kv.v_block_mean && !isinf(a->depth_T))) return FOLD_EUNSUPPORTED;
+      if (a->kv.v_block_mean && !isinf(a->depth_T)) return FOLD_EUNSUPPORTED;
     }
   }
   return FOLD_OK;
@@ -504,8 +504,9 @@ int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanPara
 }
 template <int D>
 int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
-  if (pp.kv.v1) return launch_planes_as<D, false, false, true>(ma, mv, pp, grid, st);    // E4M3 values: no drafts, no tail
   const bool drafts = pp.s.draft_len > 0, tail = pp.s.vmean != nullptr;      // (separate instantiations: registers)
+  if (pp.kv.v1)                                              // E4M3 values: no block tail
+    return drafts ? launch_planes_as<D, true, false, true>(ma, mv, pp, grid, st) : launch_planes_as<D, false, false, true>(ma, mv, pp, grid, st);
   if (drafts) return tail ? launch_planes_as<D, true, true>(ma, mv, pp, grid, st) : launch_planes_as<D, true, false>(ma, mv, pp, grid, st);
   return tail ? launch_planes_as<D, false, true>(ma, mv, pp, grid, st) : launch_planes_as<D, false, false>(ma, mv, pp, grid, st);
 }

@@ -220,10 +220,11 @@ def test_host_checks_of_e4m3_value_planes():
     a.refine_tau_v = float("nan")
     assert L.fold_decode(a, None) == F.FOLD_EINVAL
     a.refine_tau_v = 0.0
-    masks = torch.ones(2, dtype=torch.int32)
-    a.draft_len, a.draft_mask = 1, masks.data_ptr()
-    assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED             # no draft rows on the value planes
-    a.draft_len, a.draft_mask = 0, None
+    vm = torch.zeros(k.shape[0], 16, k.shape[2], k.shape[3], dtype=torch.bfloat16)
+    a.kv.v_block_mean, a.depth_T = vm.data_ptr(), 12.0
+    a.kv.mean_stride_seq, a.kv.mean_stride_block, a.kv.mean_stride_head = vm.stride(0), vm.stride(1), vm.stride(2)
+    assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED             # no block tail on the value planes
+    a.kv.v_block_mean, a.depth_T = None, float("inf")
     kv = F.FoldKV()
     assert L.fold_quantize_values(None, 2, 128, None, None) == F.FOLD_EINVAL
     assert L.fold_quantize_values(kv, 2, 96, None, None) == F.FOLD_EUNSUPPORTED

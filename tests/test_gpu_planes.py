@@ -398,7 +398,7 @@ def test_random_shapes_match_the_oracle(seed):
             kw.update(capacity=max(lens) + rnd.choice([0, 5, 100]))
         tail = (not math.isinf(T)) and rnd.random() < 0.4
         drafts = stack > 1 and rnd.random() < 0.5
-        vfp8 = (not tail) and (not drafts) and rnd.random() < 0.4
+        vfp8 = (not tail) and rnd.random() < 0.4
         tau_v = rnd.choice([0.0, 0.0, -1.0, 5.0, math.inf])
         case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw, tail=tail, drafts=drafts, vfp8=vfp8, tau_v=tau_v)
         draft = None
@@ -520,3 +520,16 @@ def test_decode_on_e4m3_value_planes(Hq, Hkv, D, paged):
     plain = run_planes(w, plane_cache(w))
     d = (full.out.float() - plain.out.float()).norm() / plain.out.float().norm()
     assert float(d) < 5e-3
+
+
+@pytest.mark.parametrize("Hq,Hkv,m,tree", [(4, 1, 2, False), (2, 2, 4, True), (1, 1, 8, False)])
+def test_draft_rows_on_e4m3_value_planes(Hq, Hkv, m, tree):
+    from paper_2609_33410_b200.workloads import make_draft_workload
+    w, masks, m = make_draft_workload(2, m, Hq, Hkv, 128, [700, 190], seed=109, device=DEV, tree=tree, poison_padding=True)
+    cache = value_planes_of(w, plane_cache(w))
+    d = (masks, m)
+    for T, tau_v in ((math.inf, 0.0), (12.0, 0.0), (12.0, 4.0)):
+        b = run_planes(w, cache, T=T, draft=d, tau_v=tau_v)
+        compare_planes(w, cache, b, T=T, check_estimate=True, draft=d, tau_v=tau_v)
+        s = run_planes(w, cache, T=T, num_splits=1, draft=d, tau_v=tau_v)
+        assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse)
