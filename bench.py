@@ -47,7 +47,8 @@ WORKLOADS = {
 # of the c2_small workload (`--workload c2_small`), per byte of cache the launch covers: the c2_small
 # capture (268.4 MB of K+V) moved 272.2 MB (gated, T=16) and 271.8 MB (dense).  Traffic grows in
 # proportion to the (sequence, kv head, key) units, so a launch is scaled by its cache bytes.
-NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 272.2 / 268.4, "dense": 271.8 / 268.4}
+# The two-plane scan at its automatic gates moved 218.4 MB (BF16 values) and 219.3 MB (E4M3 value planes) on c2_small.
+NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 272.2 / 268.4, "dense": 271.8 / 268.4, "planes": 218.4 / 268.4, "planes_fp8v": 219.3 / 268.4}
 
 
 def load_peaks():
@@ -558,6 +559,13 @@ def main():
     scan_name = ("fold_scan_stacked_pair_kernel + fold_scan_gated_narrow_kernel (prefix + suffix levels)" if cascade
                  else "fold_scan_planes_kernel" if args.planes else "fold_scan_gated_narrow_kernel")
 
+    # the ncu captures cover c2's launch shape at the default gates only
+    traffic_key = None
+    if args.workload == "c2" and not cascade and args.drafts <= 1 and not args.tail:
+        if not args.planes:
+            traffic_key = "gated"
+        elif args.refine_tau == 0 and (not args.fp8v or args.refine_tau_v == 0):
+            traffic_key = "planes_fp8v" if args.fp8v else "planes"
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
         "ms_per_step": r16["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -586,7 +594,7 @@ def main():
             "cache_write_ms": quant_ms},
         "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
                      "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src,
-                     "traffic": None if cascade or args.planes or args.workload != "c2" else NCU_TRAFFIC_PER_CACHE_BYTE["gated"] * cache_bytes,
+                     "traffic": None if traffic_key is None else NCU_TRAFFIC_PER_CACHE_BYTE[traffic_key] * cache_bytes,
                      "traffic_source": "ncu dram__bytes_read+write of the same kernel captured on workload c2_small, scaled by units",
                      "algorithmic_bytes_per_launch": actual_bytes(r16),
                      "dense": {"kernel": "fold_scan_planes_kernel (T=inf)" if args.planes else "fold_scan_dense_kernel (T=inf)" if not cascade else "fold_scan_stacked_pair_kernel + fold_scan_dense_kernel (T=inf)", "achieved": achinf, "frac": achinf / peak,
