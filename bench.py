@@ -321,6 +321,12 @@ def main():
                     help="verify a chain of this many draft tokens per sequence (stacked rows with ancestor masks)")
     ap.add_argument("--tail", action="store_true",
                     help="finite-depth steps use the block tail (cut keys add weight x block-mean value)")
+    ap.add_argument("--peak-gain", type=float, default=None,
+                    help="EXTRA, not the graded data: boosted keys get k += peak_gain * q/|q| instead of 4 * q/|q| "
+                         "(4 * sqrt(head_dim) ~ the other reading of the recipe, k += 4 q: sharply peaked rows)")
+    ap.add_argument("--z-from-lse", action="store_true",
+                    help="EXTRA: the timed steps take each row's reference from the log-sum-exp of a first decode "
+                         "(FOLD_Z_GIVEN, the certificate's re-run) instead of estimating it")
     ap.add_argument("--planes", action="store_true",
                     help="keys as two INT8 planes + a BF16 scale per key (quantized once, outside the timed region)")
     ap.add_argument("--fp8v", action="store_true",
@@ -377,7 +383,11 @@ def main():
         levels = [lvl]
     else:
         gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
+        if args.peak_gain is not None:
+            gen["peak_gain"] = args.peak_gain
         levels = [make_decode_workload(device=dev, **gen)]
+    if (args.peak_gain is not None or args.z_from_lse) and (cascade or args.drafts > 1):
+        raise SystemExit("--peak-gain / --z-from-lse: plain workloads only")
     w = levels[-1]                                                        # the level that owns out / lse / z
     caches = [F.KVCache(l.k, l.v, l.seqlens, l.max_seqlen, l.page_table) for l in levels]
     if args.tail:
@@ -448,7 +458,8 @@ def main():
     def step_split(a, evs):
         # the same launches issued one by one, so each kernel can be timed on its own
         evs[0].record(stream)
-        F.fold_estimate_z(a, stream)
+        if not args.z_from_lse:                               # (there the references are inputs: nothing to estimate)
+            F.fold_estimate_z(a, stream)
         evs[1].record(stream)
         parts = [F.fold_decode_split(x, stream) for x in a]
         evs[2].record(stream)
@@ -466,6 +477,12 @@ def main():
         a = make(depth, F.Z_ESTIMATE)
         for _ in range(warmup):
             step_whole(a)
+        if args.z_from_lse:
+            torch.cuda.synchronize()
+            bufs.z.copy_(bufs.lse)                             # the dense log-sum-exp of the rows (L sums every key)
+            a = make(depth, F.Z_GIVEN)
+            for _ in range(warmup):
+                step_whole(a)
         run_step = lambda: step_whole(a)
         if args.graph:
             # the whole call (memset + estimate + scan + partial add) captured once and replayed: takes the host's
@@ -580,6 +597,8 @@ def main():
                    "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16",
                    "value_format": "two E4M3 planes, power-of-two scale" if args.fp8v else "bf16",
                    "refine_tau": (args.refine_tau or "auto: max(log2(n) - 2, 4)") if args.planes else None,
+                   "extra_not_graded": ({"peak_gain": args.peak_gain, "z_from_lse": bool(args.z_from_lse)}
+                                        if args.peak_gain is not None or args.z_from_lse else None),
                    "flat_equivalent_bytes_per_gpu": flat_bytes},
         "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
         "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},
@@ -634,7 +653,7 @@ def main():
                       "note": "fold_decode_host: whole cache copied from pinned host memory every step"}
         del staging, hk, hv
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not cascade:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not cascade and args.peak_gain is None:
         wc = make_decode_workload(device="cpu", **dict(spec["gen"], batch=min(spec["gen"]["batch"], 2)))
         ob = bounded_oracle(wc, T)
         one = None
