@@ -359,6 +359,15 @@ def test_config2_full_size_two_plane_keys_sampled_units():
     assert 0.1 < r["refine_frac"] < 0.3 and r["live_frac"] > 0.9
     assert same_bits(run_planes(w, cache, T=16.0, num_splits=8).out, b16.out)
     compare_planes(w, cache, run_planes(w, cache), units=units)
+    # the same cache with its values in two E4M3 planes (bench.py --planes --fp8v): writer bit for bit on one unit,
+    # gated decode at the automatic gates on the sampled units
+    cache = value_planes_of(w, cache)
+    p1, p2 = logical_value_planes(w, cache, 7, 5)
+    r1, r2 = P.quantize_values(O.widen_bf16(bf16_bits(w.logical_rows("v", 7, 5))), cache.v_scale_log2)
+    assert np.array_equal(p1, r1) and np.array_equal(p2, r2)
+    v16 = run_planes(w, cache, T=16.0)
+    compare_planes(w, cache, v16, T=16.0, units=units[1:], check_estimate=True)
+    assert same_bits(run_planes(w, cache, T=16.0, num_splits=8).out, v16.out)
     del w, cache
     torch.cuda.empty_cache()
 
