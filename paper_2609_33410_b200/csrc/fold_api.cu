@@ -867,7 +867,7 @@ int fold_quantize_keys(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim
   p.kv = plane_view(*kv);
   p.first_token = first_token;
   const dim3 grid((kv->max_seqlen + kQuantRowsPerCta - 1) / kQuantRowsPerCta, num_kv_heads, kv->num_seqs);
-  const dim3 block(32, kQuantRowsPerCta);
+  const dim3 block(32, kQuantWarps);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (head_dim == 128) fold_quantize_keys_kernel<128><<<grid, block, 0, st>>>(p);
   else fold_quantize_keys_kernel<64><<<grid, block, 0, st>>>(p);
@@ -889,7 +889,7 @@ int fold_quantize_values(const fold_kv *kv, int32_t num_kv_heads, int32_t head_d
   p.first_token = first_token;
   p.inv_scale = ldexpf(1.f, -kv->v_scale_log2);
   const dim3 grid((kv->max_seqlen + kQuantRowsPerCta - 1) / kQuantRowsPerCta, num_kv_heads, kv->num_seqs);
-  const dim3 block(32, kQuantRowsPerCta);
+  const dim3 block(32, kQuantWarps);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (head_dim == 128) fold_quantize_values_kernel<128><<<grid, block, 0, st>>>(p);
   else fold_quantize_values_kernel<64><<<grid, block, 0, st>>>(p);

@@ -122,32 +122,44 @@ struct QuantParams {
   PlaneView kv;                                               // destinations (written)
   const int *first_token;                                     // per sequence, or null: from token 0
 };
-constexpr int kQuantRowsPerCta = 8;
+constexpr int kQuantWarps = 8;                                  // warps per CTA
+constexpr int kQuantRowsPerWarp = 4;                            // rows a warp loads before it works on any (bytes in flight)
+constexpr int kQuantRowsPerCta = kQuantWarps * kQuantRowsPerWarp;
 
 template <int D>
-__global__ void __launch_bounds__(32 * kQuantRowsPerCta) fold_quantize_keys_kernel(const QuantParams p) {
-  constexpr int EPL = D / 32;
+__global__ void __launch_bounds__(32 * kQuantWarps) fold_quantize_keys_kernel(const QuantParams p) {
+  constexpr int EPL = D / 32, RW = kQuantRowsPerWarp;
   const int lane = threadIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
   int n = p.kv.seqlens[seq];
   n = n < 0 ? 0 : (n > p.kv.max_seqlen ? p.kv.max_seqlen : n);
   const int first = p.first_token ? max(p.first_token[seq], 0) : 0;
-  const int j = first + blockIdx.x * kQuantRowsPerCta + threadIdx.y;
-  if (j >= n) return;
-  long long s, t;
-  plane_locate(p.kv, seq, j, s, t);
-  float x[EPL];
-  load_bf16_row<EPL>(p.k + s * p.k_stride_seq + t * p.k_stride_tok + (long long)kvh * p.k_stride_head + lane * EPL, x);
-  int a[EPL], b[EPL];
-  const float e = rotate_split<D>(x, lane, a, b);
-  const long long off = s * p.kv.stride_seq + t * p.kv.stride_tok + (long long)kvh * p.kv.stride_head + lane * EPL;
-  store_codes<EPL>(const_cast<int8_t *>(p.kv.a) + off, a);
-  store_codes<EPL>(const_cast<int8_t *>(p.kv.b) + off, b);
-  if (lane == 0)
-    const_cast<__nv_bfloat16 *>(p.kv.scale)[s * p.kv.sc_stride_seq + (long long)kvh * p.kv.sc_stride_head + t] =
-        __float2bfloat16_rn(e);                              // exact: e is a BF16 value
+  const int j0 = first + (blockIdx.x * kQuantWarps + threadIdx.y) * RW;
+  if (j0 >= n) return;
+  long long s[RW], t[RW];
+  float x[RW][EPL];
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    s[r] = t[r] = 0;
+    if (j0 + r < n) {
+      plane_locate(p.kv, seq, j0 + r, s[r], t[r]);
+      load_bf16_row<EPL>(p.k + s[r] * p.k_stride_seq + t[r] * p.k_stride_tok + (long long)kvh * p.k_stride_head + lane * EPL, x[r]);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    if (j0 + r >= n) break;
+    int a[EPL], b[EPL];
+    const float e = rotate_split<D>(x[r], lane, a, b);
+    const long long off = s[r] * p.kv.stride_seq + t[r] * p.kv.stride_tok + (long long)kvh * p.kv.stride_head + lane * EPL;
+    store_codes<EPL>(const_cast<int8_t *>(p.kv.a) + off, a);
+    store_codes<EPL>(const_cast<int8_t *>(p.kv.b) + off, b);
+    if (lane == 0)
+      const_cast<__nv_bfloat16 *>(p.kv.scale)[s[r] * p.kv.sc_stride_seq + (long long)kvh * p.kv.sc_stride_head + t[r]] =
+          __float2bfloat16_rn(e);                            // exact: e is a BF16 value
+  }
 }
 
-// Cache write of the E4M3 value planes: p1 = e4m3(v / scale), p2 = e4m3(v / scale - p1), one warp per row.
+// Cache write of the E4M3 value planes: p1 = e4m3(v / scale), p2 = e4m3(v / scale - p1), a warp per four rows.
 struct QuantValueParams {
   const __nv_bfloat16 *v;
   long long v_stride_seq, v_stride_tok, v_stride_head;
@@ -156,31 +168,41 @@ struct QuantValueParams {
   float inv_scale;                                            // 2^-v_scale_log2
 };
 template <int D>
-__global__ void __launch_bounds__(32 * kQuantRowsPerCta) fold_quantize_values_kernel(const QuantValueParams p) {
-  constexpr int EPL = D / 32;
+__global__ void __launch_bounds__(32 * kQuantWarps) fold_quantize_values_kernel(const QuantValueParams p) {
+  constexpr int EPL = D / 32, RW = kQuantRowsPerWarp;
   const int lane = threadIdx.x, kvh = blockIdx.y, seq = blockIdx.z;
   int n = p.kv.seqlens[seq];
   n = n < 0 ? 0 : (n > p.kv.max_seqlen ? p.kv.max_seqlen : n);
   const int first = p.first_token ? max(p.first_token[seq], 0) : 0;
-  const int j = first + blockIdx.x * kQuantRowsPerCta + threadIdx.y;
-  if (j >= n) return;
-  long long s, t;
-  plane_locate(p.kv, seq, j, s, t);
-  float x[EPL];
-  load_bf16_row<EPL>(p.v + s * p.v_stride_seq + t * p.v_stride_tok + (long long)kvh * p.v_stride_head + lane * EPL, x);
-  int c1[EPL], c2[EPL];
+  const int j0 = first + (blockIdx.x * kQuantWarps + threadIdx.y) * RW;
+  if (j0 >= n) return;
+  long long s[RW], t[RW];
+  float x[RW][EPL];
 #pragma unroll
-  for (int i = 0; i < EPL; ++i) {
-    const float y = __fmul_rn(x[i], p.inv_scale);             // exact: a power of two
-    const __nv_fp8_storage_t a = __nv_cvt_float_to_fp8(y, __NV_SATFINITE, __NV_E4M3);
-    const float ya = __half2float(__half(__nv_cvt_fp8_to_halfraw(a, __NV_E4M3)));
-    const __nv_fp8_storage_t b = __nv_cvt_float_to_fp8(__fsub_rn(y, ya), __NV_SATFINITE, __NV_E4M3);   // exact difference
-    c1[i] = (int)a;
-    c2[i] = (int)b;
+  for (int r = 0; r < RW; ++r) {
+    s[r] = t[r] = 0;
+    if (j0 + r < n) {
+      plane_locate(p.kv, seq, j0 + r, s[r], t[r]);
+      load_bf16_row<EPL>(p.v + s[r] * p.v_stride_seq + t[r] * p.v_stride_tok + (long long)kvh * p.v_stride_head + lane * EPL, x[r]);
+    }
   }
-  const long long off = s * p.kv.stride_seq + t * p.kv.stride_tok + (long long)kvh * p.kv.stride_head + lane * EPL;
-  store_codes<EPL>(reinterpret_cast<int8_t *>(const_cast<uint8_t *>(p.kv.v1)) + off, c1);
-  store_codes<EPL>(reinterpret_cast<int8_t *>(const_cast<uint8_t *>(p.kv.v2)) + off, c2);
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    if (j0 + r >= n) break;
+    int c1[EPL], c2[EPL];
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+      const float y = __fmul_rn(x[r][i], p.inv_scale);        // exact: a power of two
+      const __nv_fp8_storage_t a = __nv_cvt_float_to_fp8(y, __NV_SATFINITE, __NV_E4M3);
+      const float ya = __half2float(__half(__nv_cvt_fp8_to_halfraw(a, __NV_E4M3)));
+      const __nv_fp8_storage_t b = __nv_cvt_float_to_fp8(__fsub_rn(y, ya), __NV_SATFINITE, __NV_E4M3);   // exact difference
+      c1[i] = (int)a;
+      c2[i] = (int)b;
+    }
+    const long long off = s[r] * p.kv.stride_seq + t[r] * p.kv.stride_tok + (long long)kvh * p.kv.stride_head + lane * EPL;
+    store_codes<EPL>(reinterpret_cast<int8_t *>(const_cast<uint8_t *>(p.kv.v1)) + off, c1);
+    store_codes<EPL>(reinterpret_cast<int8_t *>(const_cast<uint8_t *>(p.kv.v2)) + off, c2);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
