@@ -380,6 +380,27 @@ def decode(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, depth_T: flo
     return args
 
 
+def decode_certified(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, max_reruns: int = 2, **kw) -> int:
+    """The range certificate's loop (Section 3, "Choosing the reference"): decode; if a row's status carries
+    ROW_RANGE or ROW_NONFINITE (its L left [2^-1, 2^100] or its output is not finite), give that row the
+    log-sum-exp the decode reported as its reference where that is finite (Z = lse makes L = 1) and decode
+    again with the references given.  Rows that were in range keep their reference, so their bits do not
+    change.  Host-side control flow around the C ABI calls: it synchronises the stream to read the status, as
+    the paper's loop does, and is not part of a timed step.  Returns the number of re-runs."""
+    decode(q, cache, bufs, **kw)
+    reruns = 0
+    while reruns < max_reruns:
+        torch.cuda.synchronize(q.device)
+        bad = (bufs.row_status & (ROW_RANGE | ROW_NONFINITE)) != 0
+        bad &= torch.isfinite(bufs.lse)
+        if not bool(bad.any()):
+            break
+        bufs.z.copy_(torch.where(bad, bufs.lse, bufs.z))
+        decode(q, cache, bufs, **dict(kw, z_mode=Z_GIVEN))
+        reruns += 1
+    return reruns
+
+
 def slots_view(part: FoldPartials, workspace: torch.Tensor) -> torch.Tensor:
     """FP32 view [num_seqs, Hkv, max_slots, slot_stride] of the partial slots inside `workspace`."""
     off = part.slots - workspace.data_ptr()

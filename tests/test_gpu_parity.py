@@ -91,6 +91,31 @@ def test_head_major_cache_strides():
         assert same_bits(bufs.out, ref.out) and same_bits(bufs.lse, ref.lse)
 
 
+def test_range_certificate_rerun_repairs_flagged_rows_and_leaves_the_others_alone():
+    # Section 3, "Choosing the reference": a row whose L leaves [2^-1, 2^100] is decoded again with Z = its lse
+    w = make_decode_workload(2, 8, 2, 128, [3000, 1111], seed=23, device=DEV)
+    cache = cache_of(w)
+    good = run_gpu(w, T=16.0)
+    z = good.z.clone()
+    z[0, 3] += 40.0                                             # L = 2^-40: below the certificate's range
+    z[1, 6] -= 110.0                                            # L = 2^110: above it
+    bufs = F.alloc_buffers(w.q, cache, w.stack)
+    bufs.z.copy_(z)
+    F.decode(w.q, cache, bufs, depth_T=16.0, z_mode=F.Z_GIVEN, scale=w.scale)
+    torch.cuda.synchronize()
+    st = bufs.row_status.cpu().numpy()
+    assert (st[0, 3] & F.ROW_RANGE) and (st[1, 6] & F.ROW_RANGE) and (st != 0).sum() == 2
+    bufs.z.copy_(z)
+    assert F.decode_certified(w.q, cache, bufs, depth_T=16.0, z_mode=F.Z_GIVEN, scale=w.scale) == 1
+    torch.cuda.synchronize()
+    assert not bufs.row_status.any()
+    keep = torch.ones_like(bufs.row_status, dtype=torch.bool); keep[0, 3] = False; keep[1, 6] = False
+    assert same_bits(bufs.out[keep], good.out[keep]) and same_bits(bufs.lse[keep], good.lse[keep])
+    assert abs(float(bufs.z[0, 3] - good.lse[0, 3])) < 1e-2 and abs(float(bufs.z[1, 6] - good.lse[1, 6])) < 1e-2
+    compare(w, bufs, T=16.0)                                    # every row against the oracle at its final reference
+    assert F.decode_certified(w.q, cache, bufs, depth_T=16.0, scale=w.scale) == 0      # estimated references are in range
+
+
 def test_reference_modes_and_fp32_range():
     w = make_decode_workload(2, 8, 2, 128, [3000, 1111], seed=19, device=DEV)
     est = run_gpu(w)
