@@ -117,3 +117,18 @@ def test_config4_shared_prefix_cascade_sampled_rows():
         y = O.online_softmax_bf16(q, K, V) - O.dense_row(s, V)[0]
         ynum += y @ y
     assert math.sqrt(num / den) <= 1.5 * math.sqrt(ynum / den) + 1e-4
+
+
+@pytest.mark.parametrize("n,Hq,Hkv,D,paged", [(2_000_003, 2, 1, 128, False), (4_194_304 + 17, 1, 1, 64, True)])
+def test_multi_million_key_sequences(n, Hq, Hkv, D, paged):
+    # far beyond the paper's 128K contexts: thousands of canonical chunks per row, token offsets past 2^31 bytes
+    if _free_gb() < 6:
+        pytest.skip("not enough free device memory")
+    kw = dict(paged=True, page_size=64) if paged else {}
+    w = make_decode_workload(1, Hq, Hkv, D, n, seed=5, device=DEV, **kw)
+    for T in (math.inf, 16.0):
+        b = run_gpu(w, T=T)
+        compare(w, b, T=T, rows=[(0, Hq - 1)], check_estimate=True)
+        assert same_bits(run_gpu(w, T=T, num_splits=3).out, b.out)
+    del w
+    torch.cuda.empty_cache()
