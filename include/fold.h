@@ -38,7 +38,7 @@ typedef void *fold_stream;            /* a cudaStream_t; NULL is the legacy defa
 typedef enum fold_status {
   FOLD_OK = 0,
   FOLD_EINVAL = 1,        /* null / misaligned pointer, inconsistent sizes, T < 0 or NaN */
-  FOLD_EUNSUPPORTED = 2,  /* head_dim not in {64,128}, page_size not a power of two >= 16, ... */
+  FOLD_EUNSUPPORTED = 2,  /* head_dim not in {64,128}, page_size not a power of two >= 16, batch > 65535, ... */
   FOLD_EWORKSPACE = 3,    /* workspace_bytes < fold_workspace_bytes(args) */
   FOLD_ECUDA = 4,         /* a CUDA runtime / driver call failed (launch error, no sm_100 device) */
   FOLD_ETOOLARGE = 5      /* fold_decode_static only: the call needs more scratch than the built-in array holds */

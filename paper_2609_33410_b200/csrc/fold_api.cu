@@ -79,6 +79,7 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   if (a->batch < 1 || a->num_q_heads < 1 || a->num_kv_heads < 1 || a->stack < 1) return FOLD_EINVAL;
   if (a->num_q_heads % a->num_kv_heads) return FOLD_EINVAL;
   if (a->batch % a->stack || a->batch / a->stack != a->kv.num_seqs) return FOLD_EINVAL;
+  if (a->batch > 65535) return FOLD_EUNSUPPORTED;           // requests and sequences index a grid's y / z dimension
   if (!a->q || !aligned(a->q, 16) || a->q_stride_b % 8 || a->q_stride_h % 8) return FOLD_EINVAL;
   if (a->q_stride_h < a->head_dim && a->num_q_heads > 1) return FOLD_EINVAL;
   if (int rc = check_kv(a->kv, a->head_dim)) return rc;

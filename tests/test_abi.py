@@ -113,6 +113,9 @@ def test_host_checks_answer_before_any_cuda_call():
     assert L.fold_decode(a, None) == F.FOLD_EINVAL                # table cannot hold max_seqlen
     assert L.fold_cascade_merge(None, 1, None, None, None, None) == F.FOLD_EINVAL
     assert L.fold_estimate_z(None, 0, None) == F.FOLD_EINVAL
+    a.kv.page_table = None
+    a.batch, a.kv.num_seqs = 70000, 70000                         # requests index a grid dimension: at most 65535
+    assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED
 
 
 def test_host_checks_of_draft_masks_and_block_means():
