@@ -473,7 +473,8 @@ int row_block_rows() {
 // batches are cut finer instead.  Only scheduling: the result does not depend on the choice.
 int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   const int n = a->kv.max_seqlen;
-  const int max_chunks = num_chunks_of(n) > 0 ? num_chunks_of(n) : 1;
+  int max_chunks = num_chunks_of(n) > 0 ? num_chunks_of(n) : 1;
+  if (max_chunks > 65535) max_chunks = 65535;               // splits index a grid dimension (a split walks several chunks)
   if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
   const long long units = (long long)g.num_seqs * g.Hkv *
                           (g.R > 128 ? (g.R + 255) / 256 : (g.R <= row_block_rows() ? (g.R + kMaxRows - 1) / kMaxRows : 1));   // CTAs per split
