@@ -286,6 +286,10 @@ def test_estimator_index_structure():
         edges = [1 + (k * n_mid) // 128 for k in range(129)]
         assert all(edges[k] <= centres[k] < edges[k + 1] for k in range(128))
         assert edges[0] == 1 and edges[-1] == n - 63
+        # the key in the MIDDLE of each stratum stands for it (not its first key)
+        assert all(centres[k] - edges[k] == (edges[k + 1] - edges[k]) // 2 for k in range(128))
+    # strata of exactly 10 keys: 1..10, 11..20, ...: centres 6, 16, 26, ...
+    assert np.array_equal(O.estimator_indices(64 + 1280)[2], 6 + 10 * np.arange(128))
     assert O.estimator_indices(192) is None and O.estimator_indices(1) is None
 
 

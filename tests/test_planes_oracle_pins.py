@@ -62,6 +62,9 @@ def test_split_planes_hand_worked_row():
     a, b, e = P.split_planes(np.array([[100.0, 50.0]], dtype=np.float32))
     assert e[0] == 0.7890625
     assert a[0].tolist() == [127, 63] and b[0].tolist() == [-68, 94]   # 100/e = 126.7327 (-0.2673 * 256 = -68.4), 50/e = 63.3663 (0.3663 * 256 = 93.8)
+    # the other end of plane B: t = 3.5 -> a = 4 (ties to even), remainder -0.5 -> -128, which an int8 holds
+    a, b, e = P.split_planes(np.array([[127.0, 3.5, -2.5]], dtype=np.float32))
+    assert e[0] == 1.0 and a[0].tolist() == [127, 4, -2] and b[0].tolist() == [0, -128, -128]
     # an all-zero row
     a, b, e = P.split_planes(np.zeros((1, 8), dtype=np.float32))
     assert e[0] == 1.0 and not a.any() and not b.any()
@@ -294,6 +297,18 @@ def test_value_planes_reconstruct_within_their_steps():
     assert np.mean(np.abs(two - V)[nz] <= np.abs(V)[nz] * 2.0 ** -8 * 1.01) > 0.95
     assert np.all(np.abs(one - V) <= 2.0 ** (k - 10) + np.abs(V) * 2.0 ** -4)    # subnormal plane-1 codes: absolute step 2^-9
     assert np.array_equal(O.round_to_bf16(two), two) and np.array_equal(O.round_to_bf16(one), one)   # both are BF16 values
+    # v1 + v2 can need nine significant bits; it is rounded to BF16 once, ties to even: 1 + 2^-5 + 2^-8 -> 1 + 2^-5
+    # (codes 0x38 = 1, 0x11 = 1.125 * 2^-5) and 1 + 2^-5 + 2^-7 + 2^-8 -> 1 + 2^-5 + 2^-6 (0x13 = 1.375 * 2^-5)
+    w = P.widen_values(np.array([[0x38, 0x38]], dtype=np.uint8), np.array([[0x11, 0x13]], dtype=np.uint8), 3, np.ones(1, bool))
+    assert w[0].tolist() == [8.0 * (1 + 2.0 ** -5), 8.0 * (1 + 2.0 ** -5 + 2.0 ** -6)]
+    # values that are not BF16 themselves (the writer takes any float): the widened rows still are, and for BF16
+    # inputs the sum of the planes never needs the rounding at all
+    Vf = np.random.default_rng(31).standard_normal((200, 64)) * 2.0
+    f1, f2 = P.quantize_values(Vf, k)
+    twof = P.widen_values(f1, f2, k, np.ones(200, bool))
+    assert np.array_equal(O.round_to_bf16(twof), twof)
+    assert not np.array_equal(P.e4m3_values()[f1] + P.e4m3_values()[f2], twof * 2.0 ** -k)
+    assert np.array_equal((P.e4m3_values()[p1] + P.e4m3_values()[p2]) * 2.0 ** k, two)
     mixed = P.widen_values(p1, p2, k, np.arange(300) % 2 == 0)
     assert np.array_equal(mixed[0::2], two[0::2]) and np.array_equal(mixed[1::2], one[1::2])
 
