@@ -153,6 +153,29 @@ def test_worked_example_z4_golden():
     oa, la = O.dense_row(s[:2], v[:2]); ob, lb = O.dense_row(s[2:], v[2:])
     om, lm = O.lse_merge(oa, la, ob, lb)
     assert abs(om[0] - o[0]) < 1e-15 and abs(lm - lse) < 1e-15
+    # ... in either order and for an uneven cut (the two log-sum-exps differ, whichever is larger)
+    for cut in (1, 4):
+        oa, la = O.dense_row(s[:cut], v[:cut]); ob, lb = O.dense_row(s[cut:], v[cut:])
+        assert la != lb
+        for (x, lx, y, ly) in ((oa, la, ob, lb), (ob, lb, oa, la)):
+            om, lm = O.lse_merge(x, lx, y, ly)
+            assert abs(om[0] - o[0]) < 1e-15 and abs(lm - lse) < 1e-15
+
+
+def test_bf16_online_softmax_two_key_example():
+    # the yardstick's defining choices on two keys, by hand: P is rounded to BF16 for the value product, L sums the
+    # unrounded FP32 weights, the output is rounded to BF16.  Scores 0 and -0.5 binades: p = (1, 2^-0.5 = 0.70710677),
+    # bf16(p_2) = 0.70703125; values (0, 12.5625): A = 0.70703125 * 12.5625 = 8.88208, L = 1.70710677 -> 5.203002,
+    # just below the BF16 tie 5.203125 -> 5.1875.  With P left unrounded it would be 5.203558 -> 5.21875.
+    D = 4
+    q = np.zeros(D); q[0] = 1.0
+    K = np.zeros((2, D)); K[1, 0] = -0.5 / (O.LOG2E / math.sqrt(D))
+    V = np.zeros((2, D)); V[1, 0] = 12.5625
+    got = O.online_softmax_bf16(q, K, V)
+    assert got[0] == 5.1875 and not got[1:].any()
+    # the other way round, one key per tile: the first key's weight is 1 when it is multiplied, and the maximum found
+    # afterwards rescales A and L by the FP32 factor 2^-0.5, which is never rounded to BF16: the other side of the tie
+    assert O.online_softmax_bf16(q, K[::-1], V[::-1], tile=1)[0] == 5.21875
 
 
 def test_mass_is_kept_for_every_depth():
@@ -262,6 +285,7 @@ def test_bf16_online_softmax_error_band():
         V = _bf16ish(r.standard_normal((n, D))); K[0] = _bf16ish(K[0] * 8)
         ref, _ = O.dense_row(O.scores(q, K), V)
         got = O.online_softmax_bf16(q, K, V)
+        assert np.array_equal(O.round_to_bf16(got), got)          # a BF16 kernel writes BF16
         errs.append(np.linalg.norm(got - ref) / np.linalg.norm(ref))
     assert 5e-4 < np.mean(errs) < 6e-3, errs
 
@@ -343,6 +367,14 @@ def test_grid_sum_order_free_and_within_prop2_bound():
         assert abs(Fraction(val) - exact) <= Fraction(C * B) * Fraction(2) ** -61 + Fraction(abs(val)) * Fraction(2) ** -52
         assert abs(total) < 2 ** 62                 # fits the (b+2)-bit accumulator
     assert O.grid_sum([]) == (0.0, 0, 0) and O.grid_sum([0.0, 0.0])[0] == 0.0
+    # Eq. 3 by hand on a coarse grid (b = 4): C = 2 terms, largest 1.0 -> B = 2 * 2^1, alpha = 2^(4 - 2) = 4;
+    # 4 * 0.625 = 2.5 -> 2 and 4 * 0.375 = 1.5 -> 2 (ties to even), 4 * 0.875 = 3.5 -> 4, 4 * 0.3 = 1.2 -> 1
+    assert O.grid_sum([1.0, 0.625], b=4) == (1.5, 6, 2)
+    assert O.grid_sum([1.0, 0.375], b=4) == (1.5, 6, 2)
+    assert O.grid_sum([1.0, 0.875], b=4) == (2.0, 8, 2)
+    assert O.grid_sum([1.0, -0.3], b=4) == (0.75, 3, 2)
+    # C = 5 terms: ceil(log2 5) = 3 -> alpha = 2^(6 - 3 - 1) = 4 for a largest term in [1, 2)
+    assert O.grid_sum([1.5, 0.25, 0.25, 0.25, 0.25], b=6) == (2.5, 10, 2)
     # FP32 partials that need no rounding on the grid add exactly
     g = [1.5, 2.0 ** -20, -0.75, 3.0]
     assert O.grid_sum(g)[0] == sum(g)

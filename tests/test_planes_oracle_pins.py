@@ -271,6 +271,31 @@ def test_block_tail_on_planes_reduces_to_the_plain_block_tail():
     assert np.allclose(A[0] / L[0], 1.5, rtol=1e-12)
 
 
+def test_block_tail_on_planes_counts_what_each_row_cuts():
+    # several rows: a key another row keeps live (so it is fetched) is still cut for a row whose own final score is
+    # below the depth, and that row's weight goes to the block's mean.  Brute force, key by key.
+    D, n, R, T = 64, 200, 3, 5.0
+    k = rng_rows(32, n, D); V = rng_rows(33, n, D); q = rng_rows(34, R, D, spread=2.0)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    Z = np.array([P.coarse_scores(ka, ke, qa[i], qb[i], eta[i]).max() for i in range(R)]) - 1.0
+    vm = O.block_means(V)
+    A, L, info = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T, 2.0, v_mean=vm)
+    A0, L0, _ = P.fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T, 2.0)
+    assert np.array_equal(L, L0)
+    shared = 0
+    for i in range(R):
+        extra = np.zeros(D)
+        for j in range(n):
+            s = info["coarse"][i, j] + (P.refine_terms(kb[j:j + 1], ke[j:j + 1], qa[i], qb[i], eta[i])[0] if info["refine"][j] else 0.0)
+            kept = info["live"][j] and s >= -T
+            if not kept:
+                extra += 2.0 ** s * vm[j // 64]
+            shared += int(info["live"][j] and not kept)
+        assert np.allclose(A[i] - A0[i], extra, rtol=1e-9, atol=1e-12)
+    assert shared > 0                                             # the case the test is about does occur
+
+
 def test_e4m3_grid_and_rounding_hand_values():
     v = P.e4m3_values()
     # 1-4-3 bits, bias 7: 0x38 = 1.0, 0x7e = 448 (largest), 0x01 = 2^-9 (smallest subnormal), 0x08 = 2^-6 (smallest normal)
