@@ -178,6 +178,18 @@ def test_bf16_online_softmax_two_key_example():
     assert O.online_softmax_bf16(q, K[::-1], V[::-1], tile=1)[0] == 5.21875
 
 
+def test_cut_report_by_hand():
+    # Z = 0, T = 4: keys at 0, -3, -4 (on the threshold: live), -4.0005 (just cut), -9 binades; band 2^-10 holds keys 2, 3
+    s = np.array([0.0, -3.0, -4.0, -4.0005, -9.0])
+    V = np.array([[1.0, -2.0], [0.5, 0.25], [3.0, -7.0], [-5.0, 4.0], [100.0, 100.0]])
+    p = 2.0 ** s
+    rep = O.cut_report(s, V, 0.0, 4.0)
+    assert rep["live_frac"] == 3 / 5
+    assert abs(rep["cut_mass"] - (p[3] + p[4]) / p.sum()) < 1e-15
+    assert abs(rep["slack"] - (p[2] * 7.0 + p[3] * 5.0) / p.sum()) < 1e-15      # weight x the row's largest |value|
+    assert O.cut_report(s, V, 0.0, math.inf) == {"live_frac": 1.0, "cut_mass": 0.0, "slack": 0.0}
+
+
 def test_mass_is_kept_for_every_depth():
     # cut keys add weight to L and nothing to A ("Depth as a dial")
     q, K, V = _row(30, 2000, 64)
