@@ -542,3 +542,34 @@ def test_draft_rows_on_e4m3_value_planes(Hq, Hkv, m, tree):
         compare_planes(w, cache, b, T=T, check_estimate=True, draft=d, tau_v=tau_v)
         s = run_planes(w, cache, T=T, num_splits=1, draft=d, tau_v=tau_v)
         assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse)
+
+
+@pytest.mark.parametrize("vfp8", [False, True])
+def test_head_major_plane_strides(vfp8):
+    # planes stored [seq, head, token, D] and viewed as [seq, token, head, D]: only the strides differ, not a bit of the result
+    w = make_decode_workload(2, 8, 4, 128, [900, 400], seed=113, device=DEV)
+    cache = plane_cache(w)
+    if vfp8:
+        cache = value_planes_of(w, cache)
+    hm = lambda t: None if t is None else t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    other = F.KVCache(hm(w.k), hm(w.v), w.seqlens, w.max_seqlen, None, None, hm(cache.k_plane_a), hm(cache.k_plane_b),
+                      cache.k_scale, hm(cache.v_plane_1), hm(cache.v_plane_2), cache.v_scale_log2)
+    assert other.k_plane_a.stride() != cache.k_plane_a.stride()
+    for T in (math.inf, 16.0, 8.0):
+        a = run_planes(w, cache, T=T)
+        b = run_planes(w, other, T=T)
+        assert same_bits(a.out, b.out) and same_bits(a.lse, b.lse)
+    # the writers into head-major planes: the same codes
+    fresh = F.KVCache(hm(w.k), hm(w.v), w.seqlens, w.max_seqlen, None, None, torch.zeros_like(other.k_plane_a),
+                      torch.zeros_like(other.k_plane_b), torch.zeros_like(cache.k_scale),
+                      torch.zeros_like(other.k_plane_a).view(torch.uint8) if vfp8 else None,
+                      torch.zeros_like(other.k_plane_a).view(torch.uint8) if vfp8 else None, cache.v_scale_log2)
+    F.fold_quantize_keys(fresh)
+    if vfp8:
+        F.fold_quantize_values(fresh, cache.v_scale_log2)
+    torch.cuda.synchronize()
+    for s, n in enumerate([900, 400]):
+        assert torch.equal(fresh.k_plane_a[s, :n], cache.k_plane_a[s, :n]) and torch.equal(fresh.k_plane_b[s, :n], cache.k_plane_b[s, :n])
+        assert torch.equal(fresh.k_scale[s, :, :n], cache.k_scale[s, :, :n])
+        if vfp8:
+            assert torch.equal(fresh.v_plane_1[s, :n], cache.v_plane_1[s, :n]) and torch.equal(fresh.v_plane_2[s, :n], cache.v_plane_2[s, :n])
