@@ -25,6 +25,8 @@ What is here, with the passage each function restates (Section 4, "Cache format"
                       Section 4 "Cache format": values as two E4M3 planes under a power-of-two scale,
                       v ~ 2^k (v1 + v2), the second plane read only for keys whose weight matters
                       ("refine V"); E4M3 = 1-4-3 bits, bias 7, no infinities, largest value 448
+  running_mean        Section 4 "Depth as a dial": the cut model of the 8-bit value format, the mean value row of
+                      the sequence (BF16)
   fold_group_planes   Algorithm 1 for one (sequence, kv head): verdict bits ORed over the
                       group's rows, final weights, (A, L) per row; also counts the bytes the
                       gates ask for (130 + 128 r_K + 256 lambda per key at D = 128)
@@ -183,6 +185,14 @@ def widen_values(p1, p2, scale_log2: int, refined) -> np.ndarray:
     return np.where(np.asarray(refined, dtype=bool)[:, None], both, v1) * 2.0 ** scale_log2
 
 
+def running_mean(V: np.ndarray) -> np.ndarray:
+    """The cut model of the 8-bit value format (Section 4, "Depth as a dial": "for 8-bit values the model is the
+    request's running mean, which needs no fit"): the mean of all the value rows the sequence holds so far (for one
+    kv head), rounded to BF16 as the cache stores it.  V [n, D] -> [D]."""
+    V = np.asarray(V, dtype=np.float64)
+    return O.round_to_bf16(V.sum(axis=0) / V.shape[0])
+
+
 def auto_refine_tau_v(n: int) -> float:
     """The refine-V gate when the caller gives none.  Reading (PARITY UNPINNED, like auto_refine_tau): a key's
     second value plane is read when some row of its group gives it at least 1/(2n) of the row's mass,
@@ -203,7 +213,7 @@ def auto_refine_tau(n: int) -> float:
 
 
 def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None, visible=None,
-                      v_mean=None, value_planes=None, tau_v: Optional[float] = None):
+                      v_mean=None, value_planes=None, tau_v: Optional[float] = None, v_run_mean=None):
     """Algorithm 1 for the rows of one (sequence, kv head) group over all its keys.
     ka, kb [n, D] int8; ke [n]; V [n, D]; qa, qb [R, D] int8; eta [R]; Z [R] (binades).
     tau: refine gate in binades (None: auto_refine_tau(n); inf: refine every live key; negative:
@@ -219,6 +229,8 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
     value_planes = (p1, p2, scale_log2) replaces V by two E4M3 planes: refine_v_j = live_j AND
     OR_i [coarse_ij - Z_i >= -tau_v] (tau_v None: auto_refine_tau_v(n); inf: every live key; negative: none), and
     key j's value row is widen_values(...) with that mask (`V` is then ignored).
+    v_run_mean [D] (with value_planes; `running_mean`): the 8-bit format's cut model -- a key whose weight row i does
+    not keep in A adds weight x the sequence's mean value row to A_i.
     Returns (A [R, D], L [R], info) with info = live / refine masks and the bytes-per-key count."""
     ka = np.asarray(ka); kb = np.asarray(kb)
     V = np.asarray(V, dtype=np.float64) if value_planes is None else None
@@ -249,6 +261,8 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
             block_of = np.arange(n) // O.BLOCK_KEYS
             for b in np.unique(block_of[~keep]):
                 A[i] = A[i] + p[~keep & (block_of == b)].sum() * vm[b]
+        if v_run_mean is not None:
+            A[i] = A[i] + p[~keep].sum() * np.asarray(v_run_mean, dtype=np.float64)
     lam, rk, rv = (float(m.mean()) if n else 0.0 for m in (live, refine, refine_v))
     v_bytes = 2 * D * lam if value_planes is None else D * lam + D * rv          # "8-bit values replace 256 with 128 + 128 r_V"
     info = dict(live=live, refine=refine, refine_v=refine_v, coarse=coarse, bytes_per_key=(D + 2) + D * rk + v_bytes)

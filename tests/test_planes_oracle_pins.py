@@ -359,3 +359,47 @@ def test_group_fold_with_value_planes_special_cases_and_bytes():
     assert np.array_equal(info["refine_v"], info["live"] & (info["coarse"] >= -3.0).any(axis=0))
     assert 0 < info["refine_v"].sum() < info["live"].sum()
     assert P.auto_refine_tau_v(32768) == 16.0 and P.auto_refine_tau_v(4) == 4.0
+
+
+def test_running_mean_cut_model_of_the_value_planes():
+    # Section 4, "Depth as a dial": with 8-bit values a cut key's weight goes to the sequence's mean value row
+    D, n, R, T = 64, 300, 3, 5.0
+    k = rng_rows(40, n, D); V = rng_rows(41, n, D); q = rng_rows(42, R, D, spread=2.0)
+    ka, kb, ke = P.quantize_rows(k); qa, qb, qe = P.quantize_rows(q)
+    eta = qe.astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    Z = np.array([P.coarse_scores(ka, ke, qa[i], qb[i], eta[i]).max() for i in range(R)]) - 1.0
+    sl = int(math.ceil(math.log2(np.abs(V).max() / 448.0)))
+    vp = P.quantize_values(V, sl) + (sl,)
+    # the mean by hand: exact rationals on small integers, then the BF16 rounding (257 / 3 = 85.67 -> 85.5)
+    assert P.running_mean(np.array([[1.0, 2.0], [2.0, 255.0], [6.0, 0.0]])).tolist() == [3.0, 85.5]
+    m = P.running_mean(V)
+    assert np.array_equal(O.round_to_bf16(m), m) and np.allclose(m, V.mean(axis=0), rtol=2.0 ** -8, atol=1e-12)
+    A, L, info = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, T, 2.0, value_planes=vp, tau_v=3.0, v_run_mean=m)
+    A0, L0, i0 = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, T, 2.0, value_planes=vp, tau_v=3.0)
+    assert np.array_equal(L, L0) and np.array_equal(info["refine_v"], i0["refine_v"])
+    # brute force, key by key: what a row does not keep adds weight x mean
+    for i in range(R):
+        cut = 0.0
+        for j in range(n):
+            s = info["coarse"][i, j] + (P.refine_terms(kb[j:j + 1], ke[j:j + 1], qa[i], qb[i], eta[i])[0] if info["refine"][j] else 0.0)
+            if not (info["live"][j] and s >= -T):
+                cut += 2.0 ** s
+        assert cut > 0 and np.allclose(A[i] - A0[i], cut * m, rtol=1e-9, atol=1e-12)
+    # dense decode cuts nothing: no effect
+    Ai, Li, _ = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, math.inf, 2.0, value_planes=vp, tau_v=3.0, v_run_mean=m)
+    Aj, Lj, _ = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, math.inf, 2.0, value_planes=vp, tau_v=3.0)
+    assert np.array_equal(Ai, Aj)
+    # constant values that the planes hold exactly: the model restores exactly what the cut took, at any depth
+    Vc = np.full((n, D), 1.5)
+    vc = P.quantize_values(Vc, 0) + (0,)
+    A, L, _ = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, 3.0, -1.0, value_planes=vc, tau_v=-1.0, v_run_mean=P.running_mean(Vc))
+    assert np.allclose(A / L[:, None], 1.5, rtol=1e-12)
+    # a sequence of at most 64 keys is one block: the running mean is the block model's mean, and the two tails agree
+    ks, Vs = k[:50], V[:50]
+    a2, b2, e2 = P.quantize_rows(ks)
+    vs = P.quantize_values(Vs, sl) + (sl,)
+    Z2 = np.array([P.coarse_scores(a2, e2, qa[i], qb[i], eta[i]).max() for i in range(R)]) - 1.0
+    assert np.array_equal(P.running_mean(Vs), O.block_means(Vs)[0])
+    Ar, Lr, _ = P.fold_group_planes(a2, b2, e2, None, qa, qb, eta, Z2, 3.0, 1.0, value_planes=vs, tau_v=2.0, v_run_mean=P.running_mean(Vs))
+    Ab, Lb, _ = P.fold_group_planes(a2, b2, e2, None, qa, qb, eta, Z2, 3.0, 1.0, value_planes=vs, tau_v=2.0, v_mean=O.block_means(Vs))
+    assert np.allclose(Ar, Ab, rtol=1e-12) and np.array_equal(Lr, Lb)
