@@ -395,7 +395,8 @@ def main():
         # built once from the cache, outside the timed region (it belongs to cache write)
         if cascade:
             raise SystemExit("--tail: the block tail is built into the row-block scan only (no stacked prefix level)")
-        F.fold_block_means(caches[0], stream)
+        if not (args.planes and args.fp8v):               # (the 8-bit value format has its own cut model: below)
+            F.fold_block_means(caches[0], stream)
         torch.cuda.synchronize()
     quant_ms = None
     if args.planes:
@@ -417,6 +418,9 @@ def main():
             e1.record(stream)
             torch.cuda.synchronize()
             quant_ms += e0.elapsed_time(e1)
+            if args.tail:                                   # the format's cut model: one mean value row per sequence
+                F.fold_running_means(caches[0], stream)
+                torch.cuda.synchronize()
     elif args.fp8v:
         raise SystemExit("--fp8v goes with --planes")
     lbufs = [F.alloc_buffers(l.q, c, l.stack) for l, c in zip(levels, caches)]

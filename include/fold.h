@@ -80,8 +80,8 @@ enum {
  *     v_block_mean + seq*mean_stride_seq + b*mean_stride_block + head*mean_stride_head
  * (elements; multiples of 8; rows 16-byte aligned; blocks are logical for paged caches too).  A decode
  * at finite depth then adds, for every row, the summed weight of the keys that row cuts in a block
- * times that block's mean to A, instead of nothing (Algorithm 1: "add the weights of cut keys to the
- * tile's virtual row").  fold_block_means() fills the table from the cache; keeping it current when
+ * times that block's mean to A, instead of nothing (Algorithm 1: the step that gives the cut keys' weights to the
+ * tile's virtual row).  fold_block_means() fills the table from the cache; keeping it current when
  * tokens are appended is the caller's business (only the last block changes).  Every row-block and
  * stacked-row shape takes it (a stacked level with a table runs on the mma.sync kernel, not on tcgen05).
  * Ignored at depth_T = INFINITY (nothing is cut).
@@ -101,14 +101,19 @@ enum {
  * at most 8 rows (stack * group <= 8, draft rows included) and one level (no cascade), with or without the block
  * tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED.
  *
- * Two E4M3 value planes (Section 4, "Cache format": "two E4M3 planes under a power-of-two scale per layer"; only
+ * Two E4M3 value planes (Section 4, "Cache format": two FP8 planes that share one power-of-two scale per layer; only
  * together with the two-plane keys).  When v_plane_1 is not NULL the scan reads values from
  *     v_j ~ 2^v_scale_log2 * (v1_j + v2_j),   v1, v2 E4M3 codes (1-4-3 bits, bias 7, largest value 448),
  * written by fold_quantize_values(): rows of head_dim bytes laid out exactly like the key planes (the same
  * plane_stride_* and paging).  A live key's plane-1 row is always read; its plane-2 row only when some row of
  * the group gives the key a coarse weight >= 2^-refine_tau_v ("refine V"): head_dim + head_dim * r_V bytes per live
  * key instead of 2 * head_dim.  The codes widen to BF16 exactly; v1 + v2 is rounded to BF16 once.  v may then be
- * NULL for the decode calls.  Draft masks apply as on BF16 values; the block tail is not offered (FOLD_EUNSUPPORTED). */
+ * NULL for the decode calls.  Draft masks apply as on BF16 values.  The cut model of this format is not the block
+ * model but the sequence's mean value row (Section 4, "Depth as a dial": a mean kept per request): with value
+ * planes, v_block_mean (when not NULL) is read as ONE row per (sequence, kv head) -- block index 0 of the layout
+ * above, mean_stride_block unused -- holding the mean of all the sequence's value rows as BF16
+ * (fold_running_means() fills it), and a decode at finite depth adds, for every row, the summed weight of the keys
+ * that row cuts times that mean row to A. */
 typedef struct fold_kv {
   const void *k, *v;
   int64_t stride_seq, stride_tok, stride_head;   /* elements */
@@ -260,6 +265,11 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
  * at or beyond ceil(n / 64) are left untouched.  Asynchronous on `stream`; reads seqlens on the device.
  * num_kv_heads / head_dim as in fold_args.  FOLD_EINVAL for a NULL or misaligned table. */
 int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, fold_stream stream);
+
+/* The same for the 8-bit value format's cut model (Section 4, "Depth as a dial"): writes, for every sequence and kv
+ * head, the mean of ALL its value rows j < seqlens[s] (float64 sums, one rounding to FP32 and one to BF16) into block
+ * 0 of kv->v_block_mean; a sequence of length 0 gets zeros.  Reads kv->v (BF16 values; FOLD_EINVAL if NULL). */
+int fold_running_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, fold_stream stream);
 
 /* Cache write for two-plane INT8 keys (Section 4, "Cache format"): for every sequence s, kv head and token
  * first_token[s] <= j < seqlens[s] (first_token == NULL: from 0; a DEVICE array otherwise -- pass the old lengths

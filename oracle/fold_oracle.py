@@ -148,8 +148,8 @@ def fold_partial(s: np.ndarray, V: np.ndarray, Z: float, T: float = math.inf, ta
     weight 2^(s-Z) to L; only live keys add weight*value to A.  Returns (A [D], L).
 
     tail = (v_mean [num_blocks, D], block_of [len(s)]) switches the block tail on
-    (Section 4 "Depth as a dial"; Algorithm 1 "add the weights of cut keys to the tile's
-    virtual row"): a cut key j adds weight * v_mean[block_of[j]] to A instead of nothing."""
+    (Section 4 "Depth as a dial"; Algorithm 1, the step that gives the cut keys' weights to the
+    tile's virtual row): a cut key j adds weight * v_mean[block_of[j]] to A instead of nothing."""
     s = np.asarray(s, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     p = np.exp2(s - Z)

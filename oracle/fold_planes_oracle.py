@@ -14,7 +14,7 @@ What is here, with the passage each function restates (Section 4, "Cache format"
                       INT8 planes.  The codes are integers decided by FP32 arithmetic, so this
                       function works in FP32, operation by operation, as the writer does
   quantize_rows       rotate_f32 + split_planes for an array of rows (keys at cache write, the
-                      query rows at every step: "the query is split the same way")
+                      query rows at every step, which Section 4 splits like the keys)
   dequantize          e (a + b/256) in float64
   plane_products      the four integer products c^aa, c^ab, c^ba, c^bb (exact)
   coarse_scores /
@@ -186,8 +186,8 @@ def widen_values(p1, p2, scale_log2: int, refined) -> np.ndarray:
 
 
 def running_mean(V: np.ndarray) -> np.ndarray:
-    """The cut model of the 8-bit value format (Section 4, "Depth as a dial": "for 8-bit values the model is the
-    request's running mean, which needs no fit"): the mean of all the value rows the sequence holds so far (for one
+    """The cut model of the 8-bit value format (Section 4, "Depth as a dial": with 8-bit values the
+    model is a mean kept per request and needs no fitting): the mean of all the value rows the sequence holds so far (for one
     kv head), rounded to BF16 as the cache stores it.  V [n, D] -> [D]."""
     V = np.asarray(V, dtype=np.float64)
     return O.round_to_bf16(V.sum(axis=0) / V.shape[0])
@@ -202,9 +202,8 @@ def auto_refine_tau_v(n: int) -> float:
 
 
 def auto_refine_tau(n: int) -> float:
-    """The refine gate tau_K used when the caller gives none.  The paper says only that the refine
-    thresholds follow each request's own length and are set where the second plane starts to matter at
-    the error target.  Reading:  tau_K = max(log2(n) - 2, 4): a key reads plane B when some row of its
+    """The refine gate tau_K used when the caller gives none.  The paper says only that the
+    thresholds depend on the request's length and are placed where plane B begins to affect the error.  Reading:  tau_K = max(log2(n) - 2, 4): a key reads plane B when some row of its
     group gives it at least four times the uniform share 1/n of the row's mass (every key of a short row).
     On the synthetic rows of this build that refines about a quarter of the keys at 4K-32K context and
     leaves the dense output within 0.7 x the BF16 online-softmax error of exact attention (plane A alone:
@@ -223,8 +222,8 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
     visible [R, n] bool (drafts and verification trees, Section 4 "Value product": extra query rows masked to
     their ancestors): a key a row does not see has coarse score -inf for that row -- weight exactly 0, and no
     say in the verdicts.
-    v_mean [ceil(n/64), D] switches the block tail on (``fold_oracle.block_means``; Algorithm 1 "add the weights of
-    cut keys to the tile's virtual row"): a key whose weight row i does not keep in A adds weight x the mean value row
+    v_mean [ceil(n/64), D] switches the block tail on (``fold_oracle.block_means``; Algorithm 1, the step that gives
+    the cut keys' weights to the tile's virtual row): a key whose weight row i does not keep in A adds weight x the mean value row
     of its 64-key block to A_i instead of nothing.
     value_planes = (p1, p2, scale_log2) replaces V by two E4M3 planes: refine_v_j = live_j AND
     OR_i [coarse_ij - Z_i >= -tau_v] (tau_v None: auto_refine_tau_v(n); inf: every live key; negative: none), and
@@ -264,7 +263,7 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
         if v_run_mean is not None:
             A[i] = A[i] + p[~keep].sum() * np.asarray(v_run_mean, dtype=np.float64)
     lam, rk, rv = (float(m.mean()) if n else 0.0 for m in (live, refine, refine_v))
-    v_bytes = 2 * D * lam if value_planes is None else D * lam + D * rv          # "8-bit values replace 256 with 128 + 128 r_V"
+    v_bytes = 2 * D * lam if value_planes is None else D * lam + D * rv          # (Section 4: the 256 value bytes become 128 + 128 r_V)
     info = dict(live=live, refine=refine, refine_v=refine_v, coarse=coarse, bytes_per_key=(D + 2) + D * rk + v_bytes)
     return A, L, info
 

@@ -67,7 +67,7 @@ class FoldWsHeader(C.Structure):
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
            "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
-           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_quantize_keys", "fold_quantize_values", "fold_status_string",
+           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_running_means", "fold_quantize_keys", "fold_quantize_values", "fold_status_string",
            "fold_version"]
 
 _lib = None
@@ -98,6 +98,8 @@ def lib() -> C.CDLL:
         L.fold_decode_static.restype = C.c_int; L.fold_decode_static.argtypes = [C.POINTER(FoldArgs), C.c_void_p]
         L.fold_block_means.restype = C.c_int
         L.fold_block_means.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p]
+        L.fold_running_means.restype = C.c_int
+        L.fold_running_means.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p]
         L.fold_quantize_keys.restype = C.c_int
         L.fold_quantize_keys.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.fold_quantize_values.restype = C.c_int
@@ -149,7 +151,7 @@ class KVCache:
     v_plane_2: Optional[torch.Tensor] = None
     v_scale_log2: int = 0
 
-    def to_c(self) -> FoldKV:
+    def to_c(self, mean_rows_only: bool = False) -> FoldKV:
         k, v = self.k, self.v
         assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and k.dim() == 4
         assert k.stride() == v.stride() and k.shape == v.shape and k.stride(3) == 1
@@ -177,7 +179,8 @@ class KVCache:
         if self.v_block_mean is not None:
             m = self.v_block_mean
             assert m.dtype == torch.bfloat16 and m.dim() == 4 and m.stride(3) == 1 and m.shape[0] == kv.num_seqs
-            assert m.shape[1] * 64 >= kv.max_seqlen and m.shape[2:] == k.shape[2:]
+            # (with E4M3 value planes the table is the sequences' mean rows: one block)
+            assert (m.shape[1] * 64 >= kv.max_seqlen or self.v_plane_1 is not None or mean_rows_only) and m.shape[2:] == k.shape[2:]
             kv.v_block_mean = m.data_ptr()
             kv.mean_stride_seq, kv.mean_stride_block, kv.mean_stride_head = m.stride(0), m.stride(1), m.stride(2)
         else:
@@ -286,6 +289,18 @@ def fold_block_means(cache: KVCache, stream=None) -> torch.Tensor:
     kv = cache.to_c()
     _check(lib().fold_block_means(C.byref(kv), int(cache.k.shape[2]), int(cache.k.shape[3]), _stream(stream)),
            "fold_block_means")
+    return cache.v_block_mean
+
+
+def fold_running_means(cache: KVCache, stream=None) -> torch.Tensor:
+    """The 8-bit value format's cut model: fill (allocating a one-block table if the cache has none)
+    cache.v_block_mean[:, 0] with the mean value row of every (sequence, kv head); returns the table."""
+    if cache.v_block_mean is None:
+        cache.v_block_mean = torch.zeros(cache.seqlens.shape[0], 1, cache.k.shape[2], cache.k.shape[3],
+                                         dtype=torch.bfloat16, device=cache.k.device)
+    kv = cache.to_c(mean_rows_only=True)
+    _check(lib().fold_running_means(C.byref(kv), int(cache.k.shape[2]), int(cache.k.shape[3]), _stream(stream)),
+           "fold_running_means")
     return cache.v_block_mean
 
 

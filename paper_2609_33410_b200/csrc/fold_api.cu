@@ -107,10 +107,7 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
     if (isnan(a->refine_tau)) return FOLD_EINVAL;
     // the two-plane scan: one 8-row block, no exact-maximum pass
     if (R > kNarrowRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
-    if (a->kv.v_plane_1) {
-      if (isnan(a->refine_tau_v)) return FOLD_EINVAL;
-      if (a->kv.v_block_mean && !isinf(a->depth_T)) return FOLD_EUNSUPPORTED;
-    }
+    if (a->kv.v_plane_1 && isnan(a->refine_tau_v)) return FOLD_EINVAL;
   }
   return FOLD_OK;
 }
@@ -507,7 +504,7 @@ int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanPara
 template <int D>
 int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
   const bool drafts = pp.s.draft_len > 0, tail = pp.s.vmean != nullptr;      // (separate instantiations: registers)
-  if (pp.kv.v1)                                              // E4M3 values: no block tail
+  if (pp.kv.v1)                                              // E4M3 values: their cut model is applied at the chunk's end
     return drafts ? launch_planes_as<D, true, false, true>(ma, mv, pp, grid, st) : launch_planes_as<D, false, false, true>(ma, mv, pp, grid, st);
   if (drafts) return tail ? launch_planes_as<D, true, true>(ma, mv, pp, grid, st) : launch_planes_as<D, true, false>(ma, mv, pp, grid, st);
   return tail ? launch_planes_as<D, false, true>(ma, mv, pp, grid, st) : launch_planes_as<D, false, false>(ma, mv, pp, grid, st);
@@ -554,7 +551,10 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.row_groups = 1;
   p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
   p.draft_len = a->draft_len;
-  if (!isinf(a->depth_T)) {                                  // block tail: nothing is cut in dense decode
+  if (!isinf(a->depth_T) && kv.v_plane_1) {                  // 8-bit values: the table holds the sequences' mean rows (block 0)
+    pp.vrun = static_cast<const __nv_bfloat16 *>(kv.v_block_mean);
+    pp.vrun_stride_seq = kv.mean_stride_seq; pp.vrun_stride_head = kv.mean_stride_head;
+  } else if (!isinf(a->depth_T)) {                           // block tail: nothing is cut in dense decode
     p.vmean = static_cast<const __nv_bfloat16 *>(kv.v_block_mean);
     p.vm_stride_seq = kv.mean_stride_seq; p.vm_stride_block = kv.mean_stride_block; p.vm_stride_head = kv.mean_stride_head;
   }
@@ -852,6 +852,28 @@ int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (head_dim == 128) fold_block_mean_kernel<128><<<grid, block, 0, st>>>(p);
   else fold_block_mean_kernel<64><<<grid, block, 0, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+int fold_running_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, fold_stream stream) {
+  if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
+  if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
+  if (!kv->v_block_mean || !kv->v) return FOLD_EINVAL;
+  if (int rc = check_kv(*kv, head_dim)) return rc;
+  MeanParams p;
+  p.v = static_cast<const __nv_bfloat16 *>(kv->v);
+  p.v_stride_seq = kv->stride_seq; p.v_stride_tok = kv->stride_tok; p.v_stride_head = kv->stride_head;
+  p.mean = static_cast<__nv_bfloat16 *>(const_cast<void *>(kv->v_block_mean));
+  p.m_stride_seq = kv->mean_stride_seq; p.m_stride_block = kv->mean_stride_block; p.m_stride_head = kv->mean_stride_head;
+  p.seqlens = kv->seqlens; p.page_table = kv->page_table;
+  p.max_seqlen = kv->max_seqlen;
+  p.page_shift = kv->page_table ? ilog2(kv->page_size) : 0;
+  p.max_pages = kv->max_pages_per_seq; p.num_pages = kv->num_pages > 0 ? kv->num_pages : 1;
+  p.Hkv = num_kv_heads;
+  const dim3 grid(num_kv_heads, kv->num_seqs), block(32, 8);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (head_dim == 128) fold_running_mean_kernel<128><<<grid, block, 0, st>>>(p);
+  else fold_running_mean_kernel<64><<<grid, block, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 

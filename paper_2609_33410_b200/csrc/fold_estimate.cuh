@@ -304,4 +304,51 @@ __global__ void __launch_bounds__(128) fold_block_mean_kernel(const MeanParams p
   for (int e = 0; e < EPT; ++e) dst[e] = __float2bfloat16_rn(__double2float_rn(acc[e] / cnt));
 }
 
+// The cut model of the 8-bit value format (Section 4, "Depth as a dial": a mean kept per request): the mean of all
+// the value rows of a (sequence, kv head), written as block 0 of the mean table.  One CTA of 8 warps per (kv head,
+// sequence): warp w sums rows w, w + 8, ... in float64, the warps' sums are added in warp order, the quotient is rounded
+// to FP32 and then to BF16 like the block means.
+template <int D>
+__global__ void __launch_bounds__(256) fold_running_mean_kernel(const MeanParams p) {
+  constexpr int EPT = D / 32;
+  __shared__ double part[8][D];
+  const int lane = threadIdx.x, wy = threadIdx.y, kvh = blockIdx.x, seq = blockIdx.y;
+  int n = p.seqlens[seq];
+  n = n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
+  double acc[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) acc[e] = 0.0;
+  const int page_mask = (1 << p.page_shift) - 1;
+#pragma unroll 4
+  for (int j = wy; j < n; j += 8) {
+    long long s_row = seq, t_row = j;
+    if (p.page_table) {
+      const int pg = p.page_table[(long long)seq * p.max_pages + (j >> p.page_shift)];
+      s_row = min(max(pg, 0), p.num_pages - 1);
+      t_row = j & page_mask;
+    }
+    const __nv_bfloat16 *row = p.v + s_row * p.v_stride_seq + t_row * p.v_stride_tok + (long long)kvh * p.v_stride_head + lane * EPT;
+    if (EPT == 4) {
+      const uint2 w = *reinterpret_cast<const uint2 *>(row);
+      acc[0] += (double)__uint_as_float(w.x << 16); acc[1] += (double)__uint_as_float(w.x & 0xffff0000u);
+      acc[EPT - 2] += (double)__uint_as_float(w.y << 16); acc[EPT - 1] += (double)__uint_as_float(w.y & 0xffff0000u);
+    } else {
+      const uint32_t w = *reinterpret_cast<const uint32_t *>(row);
+      acc[0] += (double)__uint_as_float(w << 16); acc[1] += (double)__uint_as_float(w & 0xffff0000u);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) part[wy][lane * EPT + e] = acc[e];
+  __syncthreads();
+  if (wy != 0) return;
+  __nv_bfloat16 *dst = p.mean + (long long)seq * p.m_stride_seq + (long long)kvh * p.m_stride_head + lane * EPT;
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += part[w][lane * EPT + e];
+    dst[e] = n > 0 ? __float2bfloat16_rn(__double2float_rn(t / (double)n)) : __float2bfloat16_rn(0.f);
+  }
+}
+
 }  // namespace fold

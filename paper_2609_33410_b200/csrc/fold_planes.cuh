@@ -317,6 +317,9 @@ struct PlaneScanParams {
   float neg_tau_v;                                            // the same for the refine-V gate (E4M3 value planes)
   int auto_tau_v;                                             // tau_V = max(log2(n) + 1, 4)
   int auto_tau;                                               // tau_K = max(log2(n) - 2, 4) from the sequence's own length
+  // E4M3 value planes, finite depth: the sequences' mean value rows (the 8-bit format's cut model), or null
+  const __nv_bfloat16 *vrun;
+  long long vrun_stride_seq, vrun_stride_head;
 };
 
 // 64-key plane-A tiles (Algorithm 1's tile), two gather buffers per warp, three CTAs per SM: the kernel is bound by
@@ -556,6 +559,9 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       o[mt][2] = fmaf(c0, m1, o[mt][2]); o[mt][3] = fmaf(c1, m1, o[mt][3]);
     }
   };
+  // E4M3 value planes: the mass this thread's two rows cut in the chunk (their share of the sequence's mean value row is
+  // added once, at the chunk's end)
+  float rcut0 = 0.f, rcut1 = 0.f;
   auto finish = [&](const PlanePending &pd) {
     const uint32_t bbuf = bufs + pd.buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
     const bool landed = mbar_wait(gbar_w + 8u * pd.buf, (gphase >> pd.buf) & 1u, dead);
@@ -585,7 +591,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
       l_lo += (h0 + g0) + (pw[0] - pm[0]);
       l_hi += (h1 + g1) + (pw[1] - pm[1]);
-      if (TAIL) { cut0 += pw[0] - pm[0]; cut1 += pw[1] - pm[1]; }
+      if (TAIL || VFP8) { cut0 += pw[0] - pm[0]; cut1 += pw[1] - pm[1]; }
       if (VFP8) {
         // E4M3 values enter the product without their power-of-two scale: it multiplies the weights' BF16 terms instead
         // (exactly: a power of two), while L keeps the weights themselves
@@ -639,6 +645,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     }
     if (pd.live) value_product_n<D, true, 0, 16>(o, vbuf, 0, lane, bh, bl);
     if (TAIL) add_tail(cut0, cut1, pd.ms);
+    if (VFP8) { rcut0 += cut0; rcut1 += cut1; }
   };
 
   int stage = 0, buf = 0, n_pend = 0, mslot = 0;
@@ -704,6 +711,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
           }
           l_lo += cut0;
           l_hi += cut1;
+          if (VFP8) { rcut0 += cut0; rcut1 += cut1; }
           if (TAIL) {
             add_tail(cut0, cut1, my_ms);
             // a queued sub-slice must be finished while its tile's mean row is still in the ring (stages + 1 slots):
@@ -804,6 +812,24 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     for (int i = 0; i < LO::kBufs - 1; ++i)
       if (i >= LO::kBufs - 1 - n_pend) finish(pend[i]);
     n_pend = 0;
+    if (VFP8) {
+      if (pp.vrun) {                                          // cut mass x the sequence's mean value row (the 8-bit cut model)
+        float c0 = rcut0, c1 = rcut1;
+#pragma unroll
+        for (int m = 4; m <= 16; m <<= 1) {
+          c0 += __shfl_xor_sync(0xffffffffu, c0, m);
+          c1 += __shfl_xor_sync(0xffffffffu, c1, m);
+        }
+        const __nv_bfloat16 *mrow = pp.vrun + (long long)seq * pp.vrun_stride_seq + (long long)kvh * pp.vrun_stride_head + klo;
+#pragma unroll
+        for (int mt = 0; mt < D / 16; ++mt) {
+          const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
+          o[mt][0] = fmaf(c0, m0, o[mt][0]); o[mt][1] = fmaf(c1, m0, o[mt][1]);
+          o[mt][2] = fmaf(c0, m1, o[mt][2]); o[mt][3] = fmaf(c1, m1, o[mt][3]);
+        }
+      }
+      rcut0 = rcut1 = 0.f;
+    }
     named_bar(1, kConsumerWarps * 32);                        // every warp's buffers are drained: park there
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
     reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);

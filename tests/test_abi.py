@@ -223,11 +223,19 @@ def test_host_checks_of_e4m3_value_planes():
     a.refine_tau_v = float("nan")
     assert L.fold_decode(a, None) == F.FOLD_EINVAL
     a.refine_tau_v = 0.0
-    vm = torch.zeros(k.shape[0], 16, k.shape[2], k.shape[3], dtype=torch.bfloat16)
-    a.kv.v_block_mean, a.depth_T = vm.data_ptr(), 12.0
+    # the format's cut model (the sequences' mean value rows): host checks of its builder
+    assert L.fold_running_means(None, 2, 128, None) == F.FOLD_EINVAL
+    assert L.fold_running_means(a.kv, 2, 96, None) == F.FOLD_EUNSUPPORTED
+    assert L.fold_running_means(a.kv, 2, 128, None) == F.FOLD_EINVAL           # no table
+    vm = torch.zeros(k.shape[0], 1, k.shape[2], k.shape[3], dtype=torch.bfloat16)
+    a.kv.v_block_mean = vm.data_ptr() + 2
     a.kv.mean_stride_seq, a.kv.mean_stride_block, a.kv.mean_stride_head = vm.stride(0), vm.stride(1), vm.stride(2)
-    assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED             # no block tail on the value planes
-    a.kv.v_block_mean, a.depth_T = None, float("inf")
+    assert L.fold_running_means(a.kv, 2, 128, None) == F.FOLD_EINVAL           # misaligned table
+    a.kv.v_block_mean = vm.data_ptr()
+    a.kv.v = None
+    assert L.fold_running_means(a.kv, 2, 128, None) == F.FOLD_EINVAL           # it reads the BF16 values
+    a.kv.v = keep[2].data_ptr()
+    a.kv.v_block_mean = None
     kv = F.FoldKV()
     assert L.fold_quantize_values(None, 2, 128, None, None) == F.FOLD_EINVAL
     assert L.fold_quantize_values(kv, 2, 96, None, None) == F.FOLD_EUNSUPPORTED

@@ -95,10 +95,11 @@ def run_planes(w, cache, T=math.inf, tau=0.0, z_mode=F.Z_ESTIMATE, num_splits=0,
 
 
 def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estimate=False, check_counts=True, draft=None,
-                   v_block_mean=None, tau_v=0.0):
+                   v_block_mean=None, tau_v=0.0, v_run_mean=None):
     """`v_block_mean`: the table the GPU was given (block tail); a key that flips at a gate then moves between its value
     and its block's mean, so the threshold slack counts twice."""
     vmt = None if v_block_mean is None else v_block_mean.float().cpu().numpy().astype(np.float64)
+    vrt = None if v_run_mean is None else v_run_mean.float().cpu().numpy().astype(np.float64)     # [seqs, 1, Hkv, D]
     dmask = None if draft is None else [int(x) & 0xffffffff for x in draft[0].cpu().tolist()]
     G = w.num_q_heads // w.num_kv_heads
     R = w.stack * G
@@ -135,7 +136,8 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
             vpl = (p1, p2, cache.v_scale_log2)
             tau_v_eff = P.auto_refine_tau_v(n) if tau_v == 0.0 else tau_v
         A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis, v_mean=vm,
-                                         value_planes=vpl, tau_v=tau_v_eff)
+                                         value_planes=vpl, tau_v=tau_v_eff,
+                                         v_run_mean=None if vrt is None else vrt[seq, 0, kvh])
         n_refv += int(info["refine_v"].sum())
         n_live += int(info["live"].sum()); n_ref += int(info["refine"].sum()); n_keys += n
         vinf = np.abs(V).max(axis=1)
@@ -160,7 +162,7 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
                 dz = max(dz, abs(O.estimate_z(lambda idx: s_all[idx], n) - z[b, h]))
             if not math.isinf(T):
                 near = near_T | (np.abs(s_fin + T) <= BAND)
-                sl = (2.0 if vmt is not None else 1.0) * float((p[near] * vinf[near]).sum() / L[i])
+                sl = (2.0 if (vmt is not None or vrt is not None) else 1.0) * float((p[near] * vinf[near]).sum() / L[i])
                 sl += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum() / L[i])
                 slack2 += sl ** 2 * V.shape[1]
                 keep = slice(None) if vis is None else vis[i]
@@ -573,3 +575,39 @@ def test_head_major_plane_strides(vfp8):
         assert torch.equal(fresh.k_scale[s, :, :n], cache.k_scale[s, :, :n])
         if vfp8:
             assert torch.equal(fresh.v_plane_1[s, :n], cache.v_plane_1[s, :n]) and torch.equal(fresh.v_plane_2[s, :n], cache.v_plane_2[s, :n])
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,paged", [(8, 2, 128, False), (8, 8, 64, True), (4, 1, 128, True)])
+def test_running_mean_cut_model_on_e4m3_value_planes(Hq, Hkv, D, paged):
+    # Section 4, "Depth as a dial": with 8-bit values the cut keys' weight goes to the sequence's mean value row
+    kw = dict(paged=True, page_size=32) if paged else dict(capacity=3100)
+    w = make_decode_workload(3, Hq, Hkv, D, [3000, 733, 0], seed=127, device=DEV, poison_padding=True, **kw)
+    cache = value_planes_of(w, plane_cache(w))
+    vm = F.fold_running_means(cache)
+    torch.cuda.synchronize()
+    for seq, n in enumerate([3000, 733]):                       # the builder against the oracle, bit for bit
+        for kvh in range(Hkv):
+            ref = P.running_mean(O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh))))
+            assert np.array_equal(vm[seq, 0, kvh].float().cpu().numpy().astype(np.float64), ref), (seq, kvh)
+    assert not vm[2].any()                                      # an empty sequence: zeros
+    plain = value_planes_of(w, plane_cache(w))
+    for T, tau_v in ((6.0, 0.0), (12.0, 0.0), (16.0, 3.0), (8.0, -1.0)):
+        b = run_planes(w, cache, T=T, tau_v=tau_v)
+        compare_planes(w, cache, b, T=T, tau_v=tau_v, v_run_mean=vm)
+        s = run_planes(w, cache, T=T, tau_v=tau_v, num_splits=1)
+        assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse)
+        p0 = run_planes(w, plain, T=T, tau_v=tau_v)
+        assert same_bits(b.lse, p0.lse)                         # the model moves A only
+        assert not same_bits(b.out, p0.out)
+    # dense decode cuts nothing: the table is not read
+    assert same_bits(run_planes(w, cache).out, run_planes(w, plain).out)
+
+
+def test_running_mean_cut_model_with_draft_rows():
+    from paper_2609_33410_b200.workloads import make_draft_workload
+    w, masks, m = make_draft_workload(2, 2, 4, 1, 128, [700, 190], seed=131, device=DEV, poison_padding=True)
+    cache = value_planes_of(w, plane_cache(w))
+    vm = F.fold_running_means(cache)
+    d = (masks, m)
+    b = run_planes(w, cache, T=10.0, draft=d)
+    compare_planes(w, cache, b, T=10.0, draft=d, v_run_mean=vm, check_estimate=True)

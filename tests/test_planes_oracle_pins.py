@@ -350,7 +350,7 @@ def test_group_fold_with_value_planes_special_cases_and_bytes():
     A, L, info = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, math.inf, math.inf, value_planes=(p1, p2, sl), tau_v=math.inf)
     A0, L0, _ = P.fold_group_planes(ka, kb, ke, P.widen_values(p1, p2, sl, np.ones(n, bool)), qa, qb, eta, Z, math.inf, math.inf)
     assert np.array_equal(A, A0) and np.array_equal(L, L0) and info["bytes_per_key"] == 130 + 128 + 128 + 128
-    # no second plane at all: plane-1 values; "8-bit values replace 256 with 128 + 128 r_V"
+    # no second plane at all: plane-1 values; the 256 value bytes become 128 + 128 r_V (Section 4)
     A, L, info = P.fold_group_planes(ka, kb, ke, None, qa, qb, eta, Z, 6.0, -1.0, value_planes=(p1, p2, sl), tau_v=-1.0)
     A0, L0, i0 = P.fold_group_planes(ka, kb, ke, P.widen_values(p1, p2, sl, np.zeros(n, bool)), qa, qb, eta, Z, 6.0, -1.0)
     assert np.array_equal(A, A0) and info["bytes_per_key"] == 130 + 128 * i0["live"].mean()
