@@ -409,7 +409,7 @@ def test_random_shapes_match_the_oracle(seed):
             kw.update(capacity=max(lens) + rnd.choice([0, 5, 100]))
         tail = (not math.isinf(T)) and rnd.random() < 0.4
         drafts = stack > 1 and rnd.random() < 0.5
-        vfp8 = (not tail) and rnd.random() < 0.4
+        vfp8 = rnd.random() < 0.4                                # (with the tail: the format's own cut model, the mean row)
         tau_v = rnd.choice([0.0, 0.0, -1.0, 5.0, math.inf])
         case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw, tail=tail, drafts=drafts, vfp8=vfp8, tau_v=tau_v)
         draft = None
@@ -422,14 +422,16 @@ def test_random_shapes_match_the_oracle(seed):
         else:
             w = make_decode_workload(nseq * stack, G * Hkv, Hkv, D, lens, seed=seed * 100 + i, stack=stack, **kw)
         cache = plane_cache(w)
-        vm = oracle_block_means(w) if tail else None
-        if tail:
+        vm = oracle_block_means(w) if tail and not vfp8 else None
+        if vm is not None:
             cache = with_means(cache, vm)
         if vfp8:
             value_planes_of(w, cache)
+        vr = F.fold_running_means(cache) if tail and vfp8 else None
         try:
             b = run_planes(w, cache, T=T, tau=tau, draft=draft, tau_v=tau_v)
-            compare_planes(w, cache, b, T=T, tau=tau, check_estimate=True, draft=draft, v_block_mean=vm, tau_v=tau_v)
+            compare_planes(w, cache, b, T=T, tau=tau, check_estimate=True, draft=draft, v_block_mean=vm, tau_v=tau_v,
+                           v_run_mean=vr)
             s = run_planes(w, cache, T=T, tau=tau, num_splits=rnd.choice([1, 2, 5]), draft=draft, tau_v=tau_v)
             assert same_bits(s.out, b.out) and same_bits(s.lse, b.lse), "split count changed a bit"
         except AssertionError as e:
