@@ -181,6 +181,8 @@ class KVCache:
             assert m.dtype == torch.bfloat16 and m.dim() == 4 and m.stride(3) == 1 and m.shape[0] == kv.num_seqs
             # (with E4M3 value planes the table is the sequences' mean rows: one block)
             assert (m.shape[1] * 64 >= kv.max_seqlen or self.v_plane_1 is not None or mean_rows_only) and m.shape[2:] == k.shape[2:]
+            # with value planes only row 0 is read, as the sequence's mean: a table of block means would be misread
+            assert self.v_plane_1 is None or m.shape[1] == 1, "E4M3 value planes take the one-row table of fold_running_means"
             kv.v_block_mean = m.data_ptr()
             kv.mean_stride_seq, kv.mean_stride_block, kv.mean_stride_head = m.stride(0), m.stride(1), m.stride(2)
         else:
