@@ -870,7 +870,7 @@ int fold_running_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim
   p.page_shift = kv->page_table ? ilog2(kv->page_size) : 0;
   p.max_pages = kv->max_pages_per_seq; p.num_pages = kv->num_pages > 0 ? kv->num_pages : 1;
   p.Hkv = num_kv_heads;
-  const dim3 grid(num_kv_heads, kv->num_seqs), block(32, 8);
+  const dim3 grid(num_kv_heads, kv->num_seqs), block(32, kRunMeanWarps);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (head_dim == 128) fold_running_mean_kernel<128><<<grid, block, 0, st>>>(p);
   else fold_running_mean_kernel<64><<<grid, block, 0, st>>>(p);

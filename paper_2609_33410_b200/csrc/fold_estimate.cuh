@@ -305,13 +305,14 @@ __global__ void __launch_bounds__(128) fold_block_mean_kernel(const MeanParams p
 }
 
 // The cut model of the 8-bit value format (Section 4, "Depth as a dial": a mean kept per request): the mean of all
-// the value rows of a (sequence, kv head), written as block 0 of the mean table.  One CTA of 8 warps per (kv head,
-// sequence): warp w sums rows w, w + 8, ... in float64, the warps' sums are added in warp order, the quotient is rounded
+// the value rows of a (sequence, kv head), written as block 0 of the mean table.  One CTA of 32 warps per (kv head,
+// sequence): warp w sums rows w, w + 32, ... in float64, the warps' sums are added in warp order, the quotient is rounded
 // to FP32 and then to BF16 like the block means.
+constexpr int kRunMeanWarps = 32;
 template <int D>
-__global__ void __launch_bounds__(256) fold_running_mean_kernel(const MeanParams p) {
+__global__ void __launch_bounds__(32 * kRunMeanWarps) fold_running_mean_kernel(const MeanParams p) {
   constexpr int EPT = D / 32;
-  __shared__ double part[8][D];
+  __shared__ double part[kRunMeanWarps][D];
   const int lane = threadIdx.x, wy = threadIdx.y, kvh = blockIdx.x, seq = blockIdx.y;
   int n = p.seqlens[seq];
   n = n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
@@ -320,7 +321,7 @@ __global__ void __launch_bounds__(256) fold_running_mean_kernel(const MeanParams
   for (int e = 0; e < EPT; ++e) acc[e] = 0.0;
   const int page_mask = (1 << p.page_shift) - 1;
 #pragma unroll 4
-  for (int j = wy; j < n; j += 8) {
+  for (int j = wy; j < n; j += kRunMeanWarps) {
     long long s_row = seq, t_row = j;
     if (p.page_table) {
       const int pg = p.page_table[(long long)seq * p.max_pages + (j >> p.page_shift)];
@@ -346,7 +347,7 @@ __global__ void __launch_bounds__(256) fold_running_mean_kernel(const MeanParams
   for (int e = 0; e < EPT; ++e) {
     double t = 0.0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) t += part[w][lane * EPT + e];
+    for (int w = 0; w < kRunMeanWarps; ++w) t += part[w][lane * EPT + e];
     dst[e] = n > 0 ? __float2bfloat16_rn(__double2float_rn(t / (double)n)) : __float2bfloat16_rn(0.f);
   }
 }
