@@ -613,3 +613,18 @@ def test_running_mean_cut_model_with_draft_rows():
     d = (masks, m)
     b = run_planes(w, cache, T=10.0, draft=d)
     compare_planes(w, cache, b, T=10.0, draft=d, v_run_mean=vm, check_estimate=True)
+
+
+def test_million_key_sequence_on_planes_and_value_planes():
+    # a thousand canonical chunks per row, plane offsets past 2^31 bytes across the tensor
+    free, _ = torch.cuda.mem_get_info()
+    if free / 2 ** 30 < 6:
+        pytest.skip("not enough free device memory")
+    w = make_decode_workload(1, 8, 4, 128, 1_100_003, seed=9, device=DEV)
+    cache = value_planes_of(w, plane_cache(w))
+    for T in (math.inf, 16.0):
+        b = run_planes(w, cache, T=T)
+        compare_planes(w, cache, b, T=T, units=[(0, 3)], check_estimate=True)
+        assert same_bits(run_planes(w, cache, T=T, num_splits=3).out, b.out)
+    del w, cache
+    torch.cuda.empty_cache()
