@@ -12,6 +12,7 @@
 #include "fold_planes.cuh"
 #include "fold_scan.cuh"
 #include "fold_scan_umma.cuh"
+#include "fold_scan_decode.cuh"
 
 using namespace fold;
 
@@ -422,6 +423,29 @@ int launch_stacked_pair(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+// Row blocks of up to 16 rows at head_dim 128 on tcgen05: a persistent grid of at most one CTA per SM, two workers each.
+int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+    return 148;
+  return n;
+}
+template <bool GATED, int NC>
+int launch_decode_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, int ctas, cudaStream_t st) {
+  static int configured[64] = {0};
+  if (int rc = opt_in_smem(fold_scan_decode_kernel<GATED, NC>, configured)) return rc;
+  if (launch_pdl(fold_scan_decode_kernel<GATED, NC>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p) != cudaSuccess)
+    return FOLD_ECUDA;
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+template <bool GATED>
+int launch_decode(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, int ctas, cudaStream_t st) {
+  if (p.R == 1) return launch_decode_as<GATED, 1>(mk, mv, p, ctas, st);
+  if (p.R <= 4) return launch_decode_as<GATED, 4>(mk, mv, p, ctas, st);
+  if (p.R <= 8) return launch_decode_as<GATED, 8>(mk, mv, p, ctas, st);
+  return launch_decode_as<GATED, 16>(mk, mv, p, ctas, st);
+}
+
 // Narrow row blocks (rows on N): unpadded value slices; three K stages (measured: a fourth buys nothing and costs L1).
 template <int D, bool TAIL, int NT>
 int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, dim3 grid, cudaStream_t st) {
@@ -577,15 +601,30 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   // narrow row blocks walk 16 KB key tiles: 128 keys at D = 64
   // (row blocks of 9..16 rows run the same kernels with two N tiles per warp)
   const bool narrow_tiles = g.R <= row_block_rows();
-  const int tile_keys = (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
-  const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   const bool gated = !isinf(a->depth_T);
+  // head_dim 128, up to 16 rows: the tcgen05 row-block kernel (keys on M, 128-key tiles); it has no block tail yet
+  bool decode_umma = g.D == 128 && g.R <= kDecMaxRows && !(gated && kv.v_block_mean);
+#ifdef FOLD_TUNING
+  {
+    const char *e = getenv("FOLD_TUNE_DEC");                 // (development: off unless asked for, until it wins everywhere)
+    decode_umma = decode_umma && e && atoi(e) != 0;
+  }
+#else
+  decode_umma = false;
+#endif
+  const int tile_keys = decode_umma ? kDecKeys : (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
+  int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
+#ifdef FOLD_TUNING
+  if (const char *e = getenv("FOLD_TUNE_BOXTOK")) if (decode_umma && atoi(e) < box_tok) box_tok = atoi(e);
+#endif
   CUtensorMap mk, mv;
   MapAxes axes;
   if (int rc = make_map(&mk, &axes, kv.k, kv, g.D, g.Hkv, box_tok)) return rc;
   const bool stacked = g.R > row_block_rows();
   // dense and stacked: value tiles like key tiles; gated: a box of one 16-key slice
-  if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, (gated && !stacked) ? 16 : box_tok)) return rc;
+  // (the tcgen05 row-block kernel: groups of 32 keys, or of a page if pages are shorter)
+  const int vbox = decode_umma ? (paged && kv.page_size < 32 ? kv.page_size : 32) : 16;
+  if (int rc = make_map(&mv, &axes, kv.v, kv, g.D, g.Hkv, (gated && !stacked) ? vbox : box_tok)) return rc;
 
   ScanParams p;
   memset(&p, 0, sizeof(p));
@@ -595,6 +634,7 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.seqlens = kv.seqlens;
   p.page_table = kv.page_table;
   p.v = static_cast<const __nv_bfloat16 *>(kv.v);
+  p.k = static_cast<const __nv_bfloat16 *>(kv.k);
   p.v_stride_seq = kv.stride_seq; p.v_stride_tok = kv.stride_tok; p.v_stride_head = kv.stride_head;
   p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
   p.draft_len = a->draft_len;
@@ -605,13 +645,34 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.hdr = static_cast<fold_ws_header *>(a->workspace);
   p.max_slots = g.max_slots; p.max_seqlen = kv.max_seqlen;
   p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G; p.stack = g.stack; p.R = g.R;
+  p.num_seqs = g.num_seqs;
   p.paged = paged; p.page_shift = paged ? ilog2(kv.page_size) : 0;
   p.max_pages = kv.max_pages_per_seq; p.num_pages = kv.num_pages > 0 ? kv.num_pages : 1;
   p.box_tok = box_tok;
   p.pos_tok = axes.pos_tok; p.pos_head = axes.pos_head; p.pos_seq = axes.pos_seq;
-  p.num_splits = choose_splits(a, g, tile_keys);
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
   p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
+  if (decode_umma) {
+    // one CTA per SM at most, two workers each; the split hint only bounds the grid (never a bit of the result)
+    const long long units = (long long)g.num_seqs * g.Hkv;
+    long long ctas = (units * g.max_slots + 1) / 2;
+    if (a->num_splits > 0 && (units * a->num_splits + 1) / 2 < ctas) ctas = (units * a->num_splits + 1) / 2;
+    const int sms = sm_count();
+    if (ctas > sms) ctas = sms;
+    p.vr = vbox;                                             // tokens per value box
+    p.box_min = vbox * 13 / 16;                              // fetch a group whole from this many live rows on
+#ifdef FOLD_TUNING
+    if (const char *e = getenv("FOLD_TUNE_BOXMIN")) p.box_min = atoi(e);
+    if (const char *e = getenv("FOLD_TUNE_CTAS")) ctas = atoi(e);
+#endif
+    p.num_splits = 1;
+    p.stages = 8;                                            // tiles the L2 requests run ahead of the ring
+#ifdef FOLD_TUNING
+    if (const char *e = getenv("FOLD_TUNE_PF")) p.stages = atoi(e);
+#endif
+    return gated ? launch_decode<true>(mk, mv, p, (int)ctas, st) : launch_decode<false>(mk, mv, p, (int)ctas, st);
+  }
+  p.num_splits = choose_splits(a, g, tile_keys);
 
   // row-block kernels: kv heads on x (fastest), splits on y; stacked kernels: (row group, split) on x, heads on y
   p.row_groups = stacked || g.R <= kMaxRows ? 1 : (g.R + kMaxRows - 1) / kMaxRows;
@@ -1111,5 +1172,8 @@ const char *fold_status_string(int status) {
 }
 
 int fold_version(void) { return 100; }
+#ifdef FOLD_PROFILE
+int fold_debug_trace(long long *host_out) { return (int)cudaMemcpyFromSymbol(host_out, fold::g_dec_trace, sizeof(long long) * 64 * 16); }
+#endif
 
 }  // extern "C"

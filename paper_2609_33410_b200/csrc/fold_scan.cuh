@@ -43,6 +43,7 @@ struct ScanParams {
   const int *seqlens;
   const int *page_table;
   const __nv_bfloat16 *v;                         // gated path reads value rows directly
+  const __nv_bfloat16 *k;                         // key rows (same strides as v): L2 prefetches of the tcgen05 row-block kernel
   long long v_stride_seq, v_stride_tok, v_stride_head;
   const uint32_t *draft_mask;                     // drafts: per request, which of the last draft_len keys it uses
   int draft_len;
@@ -52,6 +53,7 @@ struct ScanParams {
   long long slot_stride;
   fold_ws_header *hdr;
   int max_slots, max_seqlen, Hq, Hkv, G, stack, R;
+  int num_seqs;                                   // KV sequences of the launch (persistent kernels walk them all)
   int paged, page_shift, max_pages, num_pages, box_tok;
   int num_splits, stages, vr;
   int pos_tok, pos_head, pos_seq;                 // which tensor-map coordinate (1..3) each axis is

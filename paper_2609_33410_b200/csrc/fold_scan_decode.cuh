@@ -1,0 +1,691 @@
+// Row-block decode scan on the 5th-generation tensor cores (tcgen05 + TMEM), head_dim 128, up to 16 query
+// rows per (sequence, kv head), dense or depth-gated.
+//
+// Algorithm 1 puts the keys on the M side of its score product and the group's rows on N, and reads the
+// verdicts of a tile off the accumulator.  On sm_100a that shape is native: one tcgen05.mma covers 128 keys,
+// the scores S^T[128 keys x 16 rows] land in tensor memory with ONE KEY PER LANE, and a tcgen05.ld hands every
+// thread of the weight warps all the rows' scores of one key.  The verdict "some row keeps this key" is then a
+// thread-local OR, the weights need no shuffles, and the per-key cost in warp instructions is a fraction of the
+// mma.sync form's (no ldmatrix, no movmatrix, no warp-wide reduction per 16 keys).
+//
+//   scores   S^T[128 keys, 16]  = K tile [128 keys, D] (A, shared memory, K-major)  x  Q^T (B, shared memory)
+//   weights  thread-per-key: p = 2^(s - Z) per row, depth gate, two-term BF16 split, L in registers;
+//            P_hi / P_lo written to shared memory as the B operand [16 rows, 128 keys] of the value product
+//   values   A^T[D, 16] += V^T[D, 128 keys] (A, the value tile as it lies in shared memory, MN-major) x P^T
+//            accumulated in tensor memory over the tiles of a canonical chunk, read out once per chunk
+//
+// Depth-gated: only K is streamed ahead by the producer; after the verdicts the weight warps request the value
+// rows some row of the group keeps -- a 16-key group that is mostly live as one tensor-map box, otherwise row by
+// row with 16-byte async copies issued for live rows only.  Rows nobody keeps cost no traffic and no
+// instruction; their weights are exactly zero and the shared-memory rows they would occupy hold zeros or
+// earlier rows of the same cache (finite), so the product is unaffected.
+//
+// Scheduling: a persistent grid.  The canonical chunks of the whole launch form one list, ordered kv head
+// fastest, then chunk, then sequence; a CTA hosts two WORKERS (worker v takes chunks v, v + W, v + 2 W, ...,
+// W = 2 x CTAs), each a set of four weight warps with its own score / weight / accumulator buffers.  The two
+// workers' tiles alternate in the CTA's key ring and on the tensor pipe, so one worker's weight phase hides
+// behind the other's products, and the ring never drains between chunks or (sequence, kv head) units.  A chunk's
+// (A, L) is formed by the same instruction sequence whichever worker runs it: the slot's bits do not depend on
+// the grid, the batch or the split hint.
+#pragma once
+
+#include "fold_scan_umma.cuh"
+
+namespace fold {
+
+#ifdef FOLD_PROFILE
+#define PROF_DECL(n) long long prof[n] = {0}; long long prof_t = clock64();
+#define PROF(i) { const long long now_ = clock64(); prof[i] += now_ - prof_t; prof_t = now_; }
+#define PROF_OUT(base, n) if (blockIdx.x == 0 && lane == 0) { for (int i_ = 0; i_ < n; ++i_) reinterpret_cast<long long *>(p.hdr)[8 + base + i_] = prof[i_]; }
+__device__ long long g_dec_trace[64 * 16];
+#define TRACE(ev, it_) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (it_) >= 2 && (it_) < 66) g_dec_trace[((it_) - 2) * 16 + (ev)] = clock64(); } while (0)
+#else
+#define TRACE(ev, it_) do { } while (0)
+#define PROF_DECL(n)
+#define PROF(i)
+#define PROF_OUT(base, n)
+#endif
+
+constexpr int kDecKeys = 128;                        // keys per tile (MMA M of the score product)
+constexpr int kDecKS = 3, kDecVS = 3;                // key / value ring depths (32 KB stages)
+constexpr int kDecThreads = 12 * 32;                 // key producer, score issuer, value-product issuer, value producer (dense), 2 workers x 4 weight warps
+constexpr int kDecTmemCols = 128;                    // S[worker][2]: 16 columns each from 0;  O[worker]: 32 columns each from 64
+constexpr int kDecMaxRows = 16;
+
+struct DecLayout {                                   // byte offsets from a 1 KB-aligned base
+  static constexpr int kTile = kDecKeys * 256;       // one key or value tile: [2 halves][128 keys][128 B], swizzled
+  static constexpr int kK = 0;
+  static constexpr int kV = kK + kDecKS * kTile;
+  static constexpr int kP = kV + kDecVS * kTile;     // weights, 8 KB per worker: two 4 KB buffers (up to 8 rows) or one of 8 KB
+  static constexpr int kQ = kP + 4 * 4096;           // [worker][parity]: [2 halves][16 rows][128 B] = 4 KB each
+  static constexpr int kLpart = kQ + 4 * 4096;       // [worker][chunk parity][4 warps][16] floats
+  static constexpr int kBar = kLpart + 1024;
+  static constexpr int kTotal = kBar + 512 + 1024;   // + alignment slack
+};
+// barrier indices (8 bytes each, from kBar)
+constexpr int kDecBarKFull = 40, kDecBarKEmpty = 3, kDecBarVFull = 6, kDecBarPvDone = 9, kDecBarSEmpty = 12,
+              kDecBarPFull = 16, kDecBarQFull = 20, kDecBarLFull = 24, kDecBarSFull = 28, kDecBarPFree = 32, kDecBarTmemSlot = 38;
+constexpr int kDecProdPos = 448;                     // byte offset from kBar: the key producer's position in the tile order
+constexpr int kDecLiveFlags = 384;                   // byte offset from kBar: [worker][weight buffer][warp] words: a key of the warp's 32 is live
+
+// D[tmem] (+)= A * B with both operands in shared memory (64-bit matrix descriptors as two words each).
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 ad, bd;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 ad, {%1, %2};\n\t"
+      "mov.b64 bd, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+// Instruction descriptor: FP32 accumulate, BF16 operands, M = 128, N = n; a_mn: the A operand is MN-major.
+__host__ __device__ constexpr uint32_t dec_idesc(int n, int a_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+// N consecutive FP32 columns of this thread's TMEM lane.
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&v)[N]) {
+  static_assert(N == 1 || N == 4 || N == 8 || N == 16 || N == 32, "column counts the decode scan uses");
+  if constexpr (N == 32) {
+    tmem_ld32(taddr, v);
+    return;
+  }
+  uint32_t r[N];
+  if constexpr (N == 1) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r[0]) : "r"(taddr) : "memory");
+  } else if constexpr (N == 4) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
+  } else if constexpr (N == 8) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+  } else {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+  }
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < N; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ------------------------------------------------------------------------------------------------
+// A worker's walk over its canonical chunks: entries g = first, first + step, ... of the launch's chunk list
+// (kv head fastest, then chunk, then sequence); entries past a sequence's own chunk count are skipped.
+struct DecWorker {
+  int g, step, n_entries;        // next list entry to look at
+  int seq, kvh, c, n;            // the current chunk: sequence, kv head, chunk index, the sequence's length
+  int t, t_end;                  // tile cursor: 128-key tiles [t, t_end) of the sequence remain in the chunk
+  int t_first;                   // first tile of the chunk
+};
+__device__ __forceinline__ int dec_seqlen(const ScanParams &p, int seq) {
+  const int n = p.seqlens[seq];
+  return n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
+}
+__device__ __forceinline__ void dec_worker_init(DecWorker &w, const ScanParams &p, int first, int step) {
+  w.g = first; w.step = step;
+  w.n_entries = p.num_seqs * p.max_slots * p.Hkv;
+  w.seq = w.kvh = w.c = w.n = 0;
+  w.t = w.t_end = w.t_first = 0;
+}
+// Move to the worker's next non-empty chunk.  False when its list is exhausted.
+__device__ __forceinline__ bool dec_worker_next_chunk(DecWorker &w, const ScanParams &p) {
+  while (w.g < w.n_entries) {
+    const int g = w.g;
+    w.g += w.step;
+    const int kvh = g % p.Hkv, rest = g / p.Hkv;
+    const int c = rest % p.max_slots, seq = rest / p.max_slots;
+    const int n = dec_seqlen(p, seq);
+    if (c < num_chunks_of(n)) {
+      const int ctiles = chunk_keys_of(n) / kDecKeys;
+      w.seq = seq; w.kvh = kvh; w.c = c; w.n = n;
+      w.t_first = w.t = c * ctiles;
+      w.t_end = min((c + 1) * ctiles, (n + kDecKeys - 1) / kDecKeys);
+      return true;
+    }
+  }
+  return false;
+}
+// Tiles of list entry g (0 for an entry past its sequence's chunks).
+__device__ __forceinline__ int dec_entry_tiles(const ScanParams &p, int g) {
+  const int rest = g / p.Hkv;
+  const int c = rest % p.max_slots, seq = rest / p.max_slots;
+  const int n = dec_seqlen(p, seq);
+  if (c >= num_chunks_of(n)) return 0;
+  const int ctiles = chunk_keys_of(n) / kDecKeys;
+  return min((c + 1) * ctiles, (n + kDecKeys - 1) / kDecKeys) - c * ctiles;
+}
+// Position in the CTA's tile order of the i-th tile of worker `set`, the workers having ta and tb tiles in all:
+// the two alternate (a first) while both have tiles left, then the longer one runs on alone.
+__device__ __forceinline__ int dec_global_index(int set, int i, int ta, int tb) {
+  return set == 0 ? i + min(i, tb) : i + min(i + 1, ta);
+}
+// The CTA's tile order as seen by the roles that serve both workers (producer, MMA issuer): both walks are kept in
+// named registers, never indexed.
+struct DecPairWalk {
+  DecWorker a, b;
+  bool alive_a, alive_b;
+  int cnt_a, cnt_b, ent_a, ent_b;                            // tiles and chunks each worker has been through
+  int s, it;                                                 // whose tile is next; its position in the order
+};
+__device__ __forceinline__ void dec_pair_init(DecPairWalk &x, const ScanParams &p, int cta, int workers) {
+  dec_worker_init(x.a, p, 2 * cta, workers);
+  dec_worker_init(x.b, p, 2 * cta + 1, workers);
+  x.alive_a = dec_worker_next_chunk(x.a, p);
+  x.alive_b = dec_worker_next_chunk(x.b, p);
+  x.cnt_a = x.cnt_b = x.ent_a = x.ent_b = 0;
+  x.it = 0;
+  x.s = x.alive_a ? 0 : 1;
+}
+__device__ __forceinline__ bool dec_pair_valid(const DecPairWalk &x) { return x.alive_a || x.alive_b; }
+__device__ __forceinline__ void dec_pair_next(DecPairWalk &x, const ScanParams &p) {
+  if (x.s == 0) {
+    ++x.cnt_a;
+    if (++x.a.t == x.a.t_end) { x.alive_a = dec_worker_next_chunk(x.a, p); ++x.ent_a; }
+    x.s = x.alive_b ? 1 : 0;
+  } else {
+    ++x.cnt_b;
+    if (++x.b.t == x.b.t_end) { x.alive_b = dec_worker_next_chunk(x.b, p); ++x.ent_b; }
+    x.s = x.alive_a ? 0 : 1;
+  }
+  ++x.it;
+}
+
+// NC: score columns a weight thread reads (query rows, rounded up).  Up to 8 rows the two weight terms share one
+// N = 16 operand (P_hi in rows 0..7, P_lo in rows 8..15: the value tile is read once per tile, not twice) and the
+// weights are double-buffered; 9..16 rows take N = 32 and one buffer.
+template <bool GATED, int NC>
+__global__ void __launch_bounds__(kDecThreads, 1)
+fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                        const ScanParams p) {
+  constexpr int D = 128;
+  constexpr int NPV = NC <= 8 ? 16 : 32;                     // N of the value product; P_lo sits NPV / 2 rows after P_hi
+  constexpr int PB = NC <= 8 ? 2 : 1;                        // weight buffers per worker
+  constexpr int PBYTES = NPV * 256;                          // [2 key halves][NPV rows][128 B]
+  using LO = DecLayout;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t *gen = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = base + LO::kBar;
+  auto bar = [&](int idx) { return bar0 + 8u * idx; };
+
+  if (threadIdx.x == 0) {
+    // "key tile landed": twice as many barriers as stages, so that a barrier only ever serves one worker's tiles (the
+    // workers alternate) and its waiter, who takes them in order, is never more than one phase ahead of it
+    for (int s = 0; s < 2 * kDecKS; ++s) mbar_init(bar(kDecBarKFull + s), 1);
+    for (int s = 0; s < kDecKS; ++s) mbar_init(bar(kDecBarKEmpty + s), 1);
+    for (int s = 0; s < kDecVS; ++s) { mbar_init(bar(kDecBarVFull + s), GATED ? 4 : 1); mbar_init(bar(kDecBarPvDone + s), 1); }
+    for (int s = 0; s < 4; ++s) {                            // one arrival per weight warp of the worker
+      mbar_init(bar(kDecBarSEmpty + s), 4);
+      mbar_init(bar(kDecBarPFull + s), 4);
+      mbar_init(bar(kDecBarQFull + s), 4);
+      mbar_init(bar(kDecBarLFull + s), 4);
+      mbar_init(bar(kDecBarSFull + s), 1);
+      mbar_init(bar(kDecBarPFree + s), 1);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(bar(kDecBarTmemSlot), kDecTmemCols);
+  // value ring, weight buffers and query tiles start as zeros: a row or column nobody writes must hold finite data
+  for (int i = threadIdx.x; i < (LO::kLpart - LO::kV) / 16; i += kDecThreads)
+    *reinterpret_cast<uint4 *>(gen + LO::kV + i * 16) = make_uint4(0, 0, 0, 0);
+  fence_proxy_async_smem();
+  pdl_launch_dependents();
+  tc_fence_before();
+  __syncthreads();                                           // barriers initialised, TMEM allocated, buffers cleared
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(gen + LO::kBar + 8 * kDecBarTmemSlot);
+
+  // the CTA's two workers and how many tiles each will walk (every warp computes both counts, a lane per entry)
+  const int W = 2 * gridDim.x;
+  const int n_entries = p.num_seqs * p.max_slots * p.Hkv;
+  int TA = 0, TB = 0;
+  {
+    int ca = 0, cb = 0;
+    for (int g = 2 * blockIdx.x + lane * W; g < n_entries; g += 32 * W) {
+      ca += dec_entry_tiles(p, g);
+      if (g + 1 < n_entries) cb += dec_entry_tiles(p, g + 1);
+    }
+    TA = __reduce_add_sync(0xffffffffu, ca);
+    TB = __reduce_add_sync(0xffffffffu, cb);
+  }
+  const int page_mask = (1 << p.page_shift) - 1;
+  bool dead = false;
+  // warp-uniform bounded wait: the warp goes on together or gives up together
+  auto wait_u = [&](uint32_t b, uint32_t parity) {
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(b, parity, dead));
+    if (!ok) dead = true;
+    return ok;
+  };
+
+  if (warp == 0 || (!GATED && warp == 3)) {
+    // ------------------------------------------------------------ producers: warp 0 streams the key tiles; dense decode
+    // reads every value row, so there warp 3 streams the value tiles the same way (its ring is freed by the value
+    // products, the key ring by the score products: neither waits for the other)
+    const bool keys = warp == 0;
+    if (lane == 0 && TA + TB > 0) {
+      const CUtensorMap *tm_ = keys ? &tmK : &tmV;
+      tma_prefetch_desc(tm_);
+      const uint64_t pol = policy_evict_first();
+      DecPairWalk x;
+      dec_pair_init(x, p, blockIdx.x, W);
+      const int boxes_per_tile = kDecKeys / p.box_tok;
+      const int full0 = keys ? kDecBarKFull : kDecBarVFull, empty0 = keys ? kDecBarKEmpty : kDecBarPvDone;
+      const int depth = keys ? kDecKS : kDecVS;
+      // One tile of (sequence, kv head, first token): into stage `st` (dst != 0) or into L2 only.  A tile takes
+      // thousands of cycles from request to arrival whatever the load on memory, and the ring holds three: the L2
+      // requests run further ahead, so the ring's own requests find their lines on the chip.
+      auto tile = [&](const DecPairWalk &y, uint32_t dst, uint32_t full) {
+        const int seq = y.s ? y.b.seq : y.a.seq, kvh = y.s ? y.b.kvh : y.a.kvh, n = y.s ? y.b.n : y.a.n;
+        const int tok0 = (y.s ? y.b.t : y.a.t) * kDecKeys;
+        const int nbox = min(boxes_per_tile, (n - tok0 + p.box_tok - 1) / p.box_tok);
+        if (dst) mbar_expect_tx(full, nbox * p.box_tok * D * 2);
+        for (int bx = 0; bx < nbox; ++bx) {
+          const int j0 = tok0 + bx * p.box_tok;
+          int c_seq = seq, c_tok = j0;
+          if (p.paged) {
+            const int pg = p.page_table[(long long)seq * p.max_pages + (j0 >> p.page_shift)];
+            c_seq = min(max(pg, 0), p.num_pages - 1);
+            c_tok = j0 & page_mask;
+          }
+          const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
+          const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
+          const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            if (dst) tma_load_4d(dst + (h * kDecKeys + bx * p.box_tok) * 128, tm_, full, h * 64, c1, c2, c3, pol);
+            else tma_prefetch_l2_4d(tm_, h * 64, c1, c2, c3);
+          }
+        }
+      };
+      for (; dec_pair_valid(x); dec_pair_next(x, p)) {
+        const int it = x.it, st = it % depth;
+        if (it >= depth && !mbar_wait(bar(empty0 + st), (uint32_t)((it / depth - 1) & 1), dead)) break;
+        if (keys) TRACE(0, it);
+        if (keys) *reinterpret_cast<volatile int *>(gen + LO::kBar + kDecProdPos) = it;
+        tile(x, base + (keys ? LO::kK : LO::kV) + st * LO::kTile, bar(keys ? kDecBarKFull + it % (2 * kDecKS) : full0 + st));
+      }
+      if (dead) {
+        // gave up: the copies already requested must still land before the CTA may leave (bounded waits again)
+        atomicOr(&p.hdr->wait_timeouts, 1u);
+        bool d2 = false;
+        for (int back = 1; back <= depth && x.it - back >= 0; ++back) {
+          const int it = x.it - back;
+          if (keys) mbar_wait(bar(kDecBarKFull + it % (2 * kDecKS)), (uint32_t)((it / (2 * kDecKS)) & 1), d2);
+          else mbar_wait(bar(full0 + it % depth), (uint32_t)((it / depth) & 1), d2);
+        }
+      }
+    }
+  } else if (GATED && warp == 3) {
+    // ------------------------------------------------------------ L2 warm-up of the key rows, p.stages tiles ahead of the ring
+    // A request from the ring takes thousands of cycles from issue to arrival once the memory system is loaded, and
+    // shared memory holds only three key tiles: the bytes in flight it allows do not fill the memory pipe on their own.
+    // This warp touches the rows of the tiles further ahead with L2 prefetches (no shared memory, nothing to wait for),
+    // so the ring's own requests mostly find their lines on the chip.
+    if (p.stages > 0 && TA + TB > 0) {
+      DecPairWalk xf;
+      dec_pair_init(xf, p, blockIdx.x, W);
+      const volatile int *pos = reinterpret_cast<const volatile int *>(gen + LO::kBar + kDecProdPos);
+      uint32_t idle = 0;
+      while (dec_pair_valid(xf) && idle < kWaitLimit) {
+        if (xf.it > *pos + p.stages) { ++idle; __nanosleep(200); continue; }
+        idle = 0;
+        if (xf.it >= kDecKS) {                               // the first tiles go straight into the ring
+          const int seq = xf.s ? xf.b.seq : xf.a.seq, kvh = xf.s ? xf.b.kvh : xf.a.kvh, n = xf.s ? xf.b.n : xf.a.n;
+          const int tok0 = (xf.s ? xf.b.t : xf.a.t) * kDecKeys;
+#pragma unroll
+          for (int r = 0; r < kDecKeys / 16; ++r) {          // 16 rows of 256 bytes per warp-wide request
+            const int tok = tok0 + r * 16 + (lane >> 1);
+            if (tok < n) {
+              int c_seq = seq, c_tok = tok;
+              if (p.paged) {
+                const int pg = p.page_table[(long long)seq * p.max_pages + (tok >> p.page_shift)];
+                c_seq = min(max(pg, 0), p.num_pages - 1);
+                c_tok = tok & page_mask;
+              }
+              const __nv_bfloat16 *row = p.k + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
+                                         (long long)kvh * p.v_stride_head + (lane & 1) * 64;
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
+            }
+          }
+        }
+        dec_pair_next(xf, p);
+      }
+    }
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------------------------------------ MMA issuers, one thread per worker
+    // One thread can start a tcgen05.mma about every 72 cycles while the pipe takes an M128 N16 K16 product about every
+    // 40, so each worker has its own issuing thread.  It keeps two walks over the worker's tiles -- value products, and
+    // scores up to two tiles ahead (the worker has two score buffers) -- and issues whichever is ready, value products
+    // first (they free a value stage and a weight buffer), probing the barriers without suspending.  The worker thus
+    // forms the weights of its next tile, and requests that tile's value rows, while those of its current tile travel.
+    const int set = warp - 1;
+    const int my_tiles = set == 0 ? TA : TB;
+    if (lane == 0 && my_tiles > 0) {
+      constexpr uint32_t idesc_qk = dec_idesc(16, 0), idesc_pv = dec_idesc(NPV, 1);
+      constexpr uint32_t desc_hi = umma_desc_hi(1024);
+      DecWorker wq, wp;
+      dec_worker_init(wq, p, 2 * blockIdx.x + set, W);
+      dec_worker_init(wp, p, 2 * blockIdx.x + set, W);
+      bool q_alive = dec_worker_next_chunk(wq, p);
+      bool p_alive = dec_worker_next_chunk(wp, p);
+      int iq = 0, eq = 0;                                    // tiles / chunks the score walk has been through
+      int ip = 0, ep = 0;                                    // the same for the value products
+      uint32_t idle = 0;
+      while (p_alive) {
+        // ---- value product of tile ip, if its weights and value rows are in
+        {
+          const int it = dec_global_index(set, ip, TA, TB), vs = it % kDecVS;
+          const bool pf = mbar_test_wait(bar(kDecBarPFull + 2 * set + (ip % PB)), (uint32_t)((ip / PB) & 1));
+          const bool vf = mbar_test_wait(bar(kDecBarVFull + vs), (uint32_t)((it / kDecVS) & 1));
+          if (pf && vf) {
+            TRACE(10, it);
+            const bool first = wp.t == wp.t_first;
+            bool some = true;                                // depth-gated: a tile nobody keeps a key of adds nothing
+            if (GATED && !first) {                           // (a chunk's first tile always runs: it initialises the accumulator)
+              const volatile uint32_t *f = reinterpret_cast<const volatile uint32_t *>(gen + LO::kBar + kDecLiveFlags) + (set * 2 + (ip % PB)) * 4;
+              some = (f[0] | f[1] | f[2] | f[3]) != 0u;
+            }
+            fence_proxy_async_smem();                        // value rows written by plain async copies, read by the tensor pipe
+            tc_fence_after();
+            // value tile [2 channel halves][128 keys][128 B] as the MN-major A operand: 16 keys = 2048 B per K step,
+            // the halves 16 KB apart (leading-dimension offset); weights [2 key halves][NPV rows][128 B], K-major
+            const uint32_t a_lo = umma_desc_lo(base + LO::kV + vs * LO::kTile, kDecKeys * 128);
+            const uint32_t b_lo = umma_desc_lo(base + LO::kP + set * 8192 + (ip % PB) * PBYTES, 16);
+            const uint32_t d = tmem + 64 + set * 32;
+            if (some) {
+#pragma unroll
+              for (int j = 0; j < kDecKeys / 16; ++j) {
+                const uint32_t bo = ((j >> 2) * (NPV * 128) + (j & 3) * 32) >> 4;
+                if (j == 0) {
+                  if (first) umma_bf16_ss<false>(d, a_lo, desc_hi, b_lo, desc_hi, idesc_pv);
+                  else umma_bf16_ss<true>(d, a_lo, desc_hi, b_lo, desc_hi, idesc_pv);
+                } else {
+                  umma_bf16_ss<true>(d, a_lo + j * (2048 >> 4), desc_hi, b_lo + bo, desc_hi, idesc_pv);
+                }
+              }
+            }
+            tc_commit(bar(kDecBarPvDone + vs));              // the value stage is free
+            tc_commit(bar(kDecBarPFree + 2 * set + (ip % PB)));   // so is the worker's weight buffer (and, at a chunk's end, A is final)
+            TRACE(12, it);
+            ++ip;
+            if (++wp.t == wp.t_end) { p_alive = dec_worker_next_chunk(wp, p); ++ep; }
+            idle = 0;
+            continue;
+          }
+        }
+        // ---- scores of tile iq: at most two tiles ahead of the value products, and at most one chunk ahead (a chunk's
+        // query rows are staged while the worker is on the chunk before)
+        if (q_alive && iq <= ip + 2 && eq <= ep + 1) {
+          const int it = dec_global_index(set, iq, TA, TB), ks = it % kDecKS;
+          const bool first = wq.t == wq.t_first;
+          bool ok = mbar_test_wait(bar(kDecBarKFull + it % (2 * kDecKS)), (uint32_t)((it / (2 * kDecKS)) & 1));
+          if (iq >= 2) ok &= mbar_test_wait(bar(kDecBarSEmpty + 2 * set + (iq & 1)), (uint32_t)(((iq >> 1) - 1) & 1));
+          if (first) ok &= mbar_test_wait(bar(kDecBarQFull + 2 * set + (eq & 1)), (uint32_t)((eq >> 1) & 1));
+          if (ok) {
+            TRACE(3, it);
+            tc_fence_after();
+            const uint32_t a_lo = umma_desc_lo(base + LO::kK + ks * LO::kTile, 16);
+            const uint32_t b_lo = umma_desc_lo(base + LO::kQ + (2 * set + (eq & 1)) * 4096, 16);
+            const uint32_t d = tmem + set * 32 + (iq & 1) * 16;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint32_t ao = ((kk >> 2) * (kDecKeys * 128) + (kk & 3) * 32) >> 4;
+              const uint32_t bo = ((kk >> 2) * 2048 + (kk & 3) * 32) >> 4;
+              if (kk == 0) umma_bf16_ss<false>(d, a_lo + ao, desc_hi, b_lo + bo, desc_hi, idesc_qk);
+              else umma_bf16_ss<true>(d, a_lo + ao, desc_hi, b_lo + bo, desc_hi, idesc_qk);
+            }
+            tc_commit(bar(kDecBarSFull + 2 * set + (iq & 1)));   // the worker's scores are ready
+            tc_commit(bar(kDecBarKEmpty + ks));              // the key stage is free
+            TRACE(4, it);
+            ++iq;
+            if (++wq.t == wq.t_end) { q_alive = dec_worker_next_chunk(wq, p); ++eq; }
+            idle = 0;
+            continue;
+          }
+        }
+        if (++idle > 8u * kWaitLimit) { dead = true; break; }   // bounded: give up, flag, fall through
+      }
+      if (dead) atomicOr(&p.hdr->wait_timeouts, 8u);
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------ weight warps: one key per thread
+    const int set = (warp - 4) >> 2, qd = warp & 3;          // worker; TMEM lane quarter this warp may touch
+    const int my_tiles = set == 0 ? TA : TB;
+    const uint32_t lane_addr = tmem + ((uint32_t)(qd * 32) << 16);
+    const int wtid = (warp - 4 - 4 * set) * 32 + lane;       // 0..127 within the worker
+    const int krow = qd * 32 + lane;                         // this thread's key row within a tile
+    float *lpart = reinterpret_cast<float *>(gen + LO::kLpart) + set * 128;
+    DecWorker cur, nxt;
+    dec_worker_init(nxt, p, 2 * blockIdx.x + set, W);
+    bool have_next = my_tiles > 0 && dec_worker_next_chunk(nxt, p);
+    float z_next[NC];
+    pdl_wait();                                              // z comes from the kernel before
+    // Stage the query rows (and fetch the references) of chunk `w`, the worker's e-th, into query buffer e & 1.
+    auto stage_rows = [&](const DecWorker &w, int e) {
+      uint8_t *qb = gen + LO::kQ + (2 * set + (e & 1)) * 4096;
+      for (int i = wtid; i < p.R * 16; i += 128) {           // 16-byte chunk i % 16 of row i / 16
+        const int r = i >> 4, c16 = i & 15;
+        const int req = w.seq * p.stack + r / p.G, head = w.kvh * p.G + r % p.G;
+        const uint4 v = *reinterpret_cast<const uint4 *>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + c16 * 8);
+        *reinterpret_cast<uint4 *>(qb + (c16 >> 3) * 2048 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = v;
+      }
+#pragma unroll
+      for (int r = 0; r < NC; ++r) {
+        const int req = w.seq * p.stack + r / p.G, head = w.kvh * p.G + r % p.G;
+        z_next[r] = r < p.R ? p.z[(long long)req * p.Hq + head] : INFINITY;   // rows past R: weight 0 by themselves
+      }
+      fence_proxy_async_smem();                              // generic writes, then tensor-core (async proxy) reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kDecBarQFull + 2 * set + (e & 1)));
+    };
+    if (have_next) stage_rows(nxt, 0);
+    unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
+    const uint64_t vpol = policy_evict_first();
+    const int vbox = p.vr;                                   // tokens per value box (16 or 32)
+    const uint32_t gmask = vbox == 32 ? 0xffffffffu : 0xffffu;
+    int i = 0;                                               // tiles this worker has been through
+    PROF_DECL(8)
+    for (int e = 0; have_next && !dead; ++e) {
+      cur = nxt;
+      float z[NC];
+#pragma unroll
+      for (int r = 0; r < NC; ++r) z[r] = z_next[r];
+      have_next = dec_worker_next_chunk(nxt, p);
+      if (have_next) stage_rows(nxt, e + 1);                 // one chunk ahead: the score products never wait for rows
+      const int n = cur.n, dstart = draft_start(p, n);
+      float L[NC];
+#pragma unroll
+      for (int r = 0; r < NC; ++r) L[r] = 0.f;
+      int it = 0;
+      for (; cur.t < cur.t_end; ++cur.t, ++i) {
+        it = dec_global_index(set, i, TA, TB);
+        const int vs = it % kDecVS;
+        const int key = cur.t * kDecKeys + krow;
+        const int tok_w = cur.t * kDecKeys + qd * 32;        // first key of this warp's 32
+        int pg0 = 0, pg1 = 0;                                // pages of the warp's value groups, fetched ahead of their use
+        if (GATED && p.paged) {
+          const int *pt = p.page_table + (long long)cur.seq * p.max_pages;
+          if (tok_w < n) pg0 = pt[tok_w >> p.page_shift];
+          if (tok_w + 16 < n) pg1 = pt[(tok_w + 16) >> p.page_shift];
+        }
+        PROF(0)
+        // the tcgen05 loads are warp-wide: the warp takes them together or not at all
+        if (wtid < 32) TRACE(5, it);
+        if (!wait_u(bar(kDecBarSFull + 2 * set + (i & 1)), (uint32_t)((i >> 1) & 1))) break;
+        if (wtid < 32) TRACE(6, it);
+        PROF(1)
+        tc_fence_after();
+        float s[NC];
+        tmem_ld_cols<NC>(lane_addr + set * 32 + (i & 1) * 16, s);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(kDecBarSEmpty + 2 * set + (i & 1)));   // this score buffer may be rewritten
+        PROF(2)
+        const bool valid = key < n;
+        const bool drafts = p.draft_len > 0 && key >= dstart;
+        uint32_t hi16[NC], lo16[NC];
+        bool any_live = false;
+#pragma unroll
+        for (int r = 0; r < NC; ++r) {
+          float x = valid ? fmaf(s[r], p.scale_log2, -z[r]) : -INFINITY;   // select: rows past n may hold anything
+          if (drafts && r < p.R && !draft_ok(p.draft_mask[cur.seq * p.stack + r / p.G], key, dstart)) x = -INFINITY;
+          const float pw = ex2_approx(x);                    // 2^-inf = 0
+          const bool live = GATED ? (x >= p.neg_T) : true;
+          const float pm = live ? pw : 0.f;
+          const float h = __bfloat162float(__float2bfloat16_rn(pm));
+          const float g = __bfloat162float(__float2bfloat16_rn(pm - h));
+          L[r] += (h + g) + (pw - pm);                       // L sums the weights the products use; cut keys add p
+          hi16[r] = __float_as_uint(h) >> 16;
+          lo16[r] = __float_as_uint(g) >> 16;
+          any_live |= live;
+        }
+        PROF(3)
+        // this tile's value stage is free once the value product of the tile three back in the CTA's order is over (the
+        // other worker's, while the two alternate), its weight buffer once the worker's own product PB tiles back is
+        if (it >= kDecVS && !wait_u(bar(kDecBarPvDone + vs), (uint32_t)((it / kDecVS - 1) & 1))) break;
+        if (i >= PB && !wait_u(bar(kDecBarPFree + 2 * set + (i % PB)), (uint32_t)((i / PB - 1) & 1))) break;
+        PROF(4)
+        if (wtid < 32) TRACE(7, it);
+        const uint32_t vfull = bar(kDecBarVFull + vs);
+        if (GATED) {
+          // requests for the value rows some row keeps, per group of vbox keys: a mostly-live group whole as one
+          // tensor-map box per 64 channels (never past the sequence end), otherwise its live rows one by one
+          const uint32_t fetch = __ballot_sync(0xffffffffu, any_live);
+          if (lane == 0) reinterpret_cast<uint32_t *>(gen + LO::kBar + kDecLiveFlags)[(set * 2 + (i % PB)) * 4 + qd] = fetch;
+          const uint32_t vdst = base + LO::kV + vs * LO::kTile;
+          bool rows = false;
+          for (int gq = 0; gq * vbox < 32; ++gq) {
+            uint32_t m = (fetch >> (gq * vbox)) & gmask;
+            const int tok = tok_w + gq * vbox;
+            const int nvalid = min(vbox, max(0, n - tok));
+            st_total += nvalid;
+            if (m == 0u) { st_skipped += nvalid > 0 ? 1 : 0; continue; }
+            int c_seq = cur.seq, c_tok = tok;
+            if (p.paged) {
+              c_seq = min(max(gq ? pg1 : pg0, 0), p.num_pages - 1);
+              c_tok = tok & page_mask;
+            }
+            const int row0 = qd * 32 + gq * vbox;            // the group's first row within the tile
+            if (__popc(m) >= p.box_min && tok + vbox <= n) {
+              st_fetched += vbox;
+              if (lane == 0) {
+                mbar_expect_tx_only(vfull, vbox * D * 2);
+                const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? cur.kvh : c_seq);
+                const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? cur.kvh : c_seq);
+                const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? cur.kvh : c_seq);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) tma_load_4d(vdst + (h * kDecKeys + row0) * 128, &tmV, vfull, h * 64, c1, c2, c3, vpol);
+              }
+            } else {
+              st_fetched += __popc(m);
+              rows = true;
+              const __nv_bfloat16 *src = p.v + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
+                                         (long long)cur.kvh * p.v_stride_head + (lane & 15) * 8;
+              const uint32_t dst = vdst + ((lane & 15) >> 3) * (kDecKeys * 128);
+              while (m) {                                    // two live rows per warp-wide copy: lanes 0..15, 16..31
+                const int r0 = __ffs(m) - 1;
+                m &= m - 1;
+                const int r1 = m ? __ffs(m) - 1 : -1;
+                m &= m - 1;
+                const int row = lane < 16 ? r0 : r1;
+                if (row >= 0)
+                  cp_async_16(dst + (row0 + row) * 128 + ((((lane & 15) ^ row) & 7) << 4), src + (long long)row * p.v_stride_tok, 16u);
+              }
+            }
+          }
+          if (rows) cp_async_mbar_arrive(vfull);             // this lane's copies hold the phase open
+        } else {
+          st_total += min(32, max(0, n - tok_w));
+          if (cur.t * kDecKeys + kDecKeys > n) {             // ragged tail: value rows past n may hold anything
+            if (!wait_u(vfull, (uint32_t)((it / kDecVS) & 1))) break;
+            if (!valid) {
+#pragma unroll
+              for (int c16 = 0; c16 < 16; ++c16)
+                *reinterpret_cast<uint4 *>(gen + LO::kV + vs * LO::kTile + tile_off(krow, c16, kDecKeys)) = make_uint4(0, 0, 0, 0);
+            }
+          }
+        }
+        PROF(5)
+        // weights: B operand [2 key halves][NPV rows][128 B], K-major, swizzled like a tensor-map box; P_hi of row r in
+        // row r, P_lo in row NPV / 2 + r (the same swizzle phase: NPV / 2 is a multiple of 8)
+        {
+          uint8_t *ph = gen + LO::kP + set * 8192 + (i % PB) * PBYTES + (krow >> 6) * (NPV * 128) + (krow & 7) * 2;
+          const int kc = (krow >> 3) & 7;
+#pragma unroll
+          for (int r = 0; r < NC; ++r) {
+            const int off = r * 128 + ((kc ^ (r & 7)) << 4);
+            *reinterpret_cast<uint16_t *>(ph + off) = (uint16_t)hi16[r];
+            *reinterpret_cast<uint16_t *>(ph + (NPV / 2) * 128 + off) = (uint16_t)lo16[r];
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar(kDecBarPFull + 2 * set + (i % PB)));
+          if (GATED) mbar_arrive(vfull);
+        }
+        if (wtid < 32) TRACE(8, it);
+        PROF(6)
+      }
+      if (dead) break;
+      // chunk end: L over the worker's 128 threads in a fixed order, then the accumulator out of tensor memory.
+      // The four warps hand their sums to the worker's first warp through shared memory and an mbarrier (bounded
+      // wait); the buffer alternates with the chunk's parity, and a warp can only reach the chunk after next once the
+      // first warp has finished this one (every tile's weights need all four warps).
+      float *slot = p.slots + (((long long)cur.seq * p.Hkv + cur.kvh) * p.max_slots + cur.c) * p.slot_stride;
+      float *lp = lpart + (e & 1) * 64;
+#pragma unroll
+      for (int r = 0; r < NC; ++r) {
+#pragma unroll
+        for (int m = 16; m >= 1; m >>= 1) L[r] += __shfl_xor_sync(0xffffffffu, L[r], m);
+        if (lane == 0) lp[qd * 16 + r] = L[r];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(kDecBarLFull + 2 * set + (e & 1)));
+      if (wtid < 32) {                                       // the worker's first warp
+        if (!wait_u(bar(kDecBarLFull + 2 * set + (e & 1)), (uint32_t)((e >> 1) & 1))) break;
+        // in the order of the key rows: lane quarters 0, 1, 2, 3
+        if (lane < p.R) slot[(long long)p.R * D + lane] = ((lp[lane] + lp[16 + lane]) + lp[32 + lane]) + lp[48 + lane];
+      }
+      if (!wait_u(bar(kDecBarPFree + 2 * set + ((i - 1) % PB)), (uint32_t)(((i - 1) / PB) & 1))) break;   // the chunk's last product
+      tc_fence_after();
+      float o[NPV];
+      tmem_ld_cols<NPV>(lane_addr + 64 + set * 32, o);       // this thread's channel: every row's P_hi part, then the P_lo parts
+      tc_fence_before();
+#pragma unroll
+      for (int r = 0; r < NC; ++r)
+        if (r < p.R) slot[(long long)r * D + krow] = o[r] + o[NPV / 2 + r];
+      PROF(7)
+    }
+    if (warp == 4) PROF_OUT(16, 8)
+    if (lane == 0) {
+      if (dead) atomicOr(&p.hdr->wait_timeouts, 16u);
+      if (st_total) {
+        atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), GATED ? st_fetched : st_total);
+        atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
+      }
+      if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
+    }
+  }
+
+  // every warp meets here; the allocating warp returns the tensor memory
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kDecTmemCols);
+  }
+}
+
+}  // namespace fold
