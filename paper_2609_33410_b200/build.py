@@ -35,10 +35,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
-    if os.environ.get("FOLD_PROFILE"):
-        cmd.insert(1, "-DFOLD_PROFILE")
-    if os.environ.get("FOLD_TUNING"):          # development only: lets FOLD_TUNE_* override ring depths
-        cmd.insert(1, "-DFOLD_TUNING")
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

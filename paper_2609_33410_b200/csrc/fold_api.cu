@@ -324,9 +324,6 @@ int launch_dense_n(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, 
   int stages = (per_cta2 - LO::total(0, p.R)) / (LO::kStage + 16);
   if (stages < 3) stages = (kSmemPerCtaMax - LO::total(0, p.R)) / (LO::kStage + 16);
   if (stages > 8) stages = 8;
-#ifdef FOLD_TUNING
-  if (const char *e = getenv("FOLD_TUNE_STAGES")) stages = atoi(e);
-#endif
   if (stages < 2) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = 0;
@@ -443,7 +440,7 @@ int launch_decode(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, i
   if (p.R == 1) return launch_decode_as<GATED, 1>(mk, mv, p, ctas, st);
   if (p.R <= 4) return launch_decode_as<GATED, 4>(mk, mv, p, ctas, st);
   if (p.R <= 8) return launch_decode_as<GATED, 8>(mk, mv, p, ctas, st);
-  return launch_decode_as<GATED, 16>(mk, mv, p, ctas, st);
+  return FOLD_EUNSUPPORTED;                                  // (the kernel takes 16 rows with NC = 16; the host keeps those on mma.sync)
 }
 
 // Narrow row blocks (rows on N): unpadded value slices; three K stages (measured: a fourth buys nothing and costs L1).
@@ -454,11 +451,6 @@ int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParam
   int nvr = 2;
   int nstages = (per_cta2 - LN::total(0, nvr)) / (LN::kKStage + 16);
   if (nstages > 3) nstages = 3;
-#ifdef FOLD_TUNING
-  if (const char *e = getenv("FOLD_TUNE_STAGES")) nstages = atoi(e);
-  if (const char *e = getenv("FOLD_TUNE_VR")) nvr = atoi(e);
-  if (const char *e = getenv("FOLD_TUNE_BOXMIN")) p.box_min = atoi(e);
-#endif
   if (nstages < 2 || nvr < 1 || LN::total(nstages, nvr) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
   p.stages = nstages;
   p.vr = nvr;
@@ -483,9 +475,6 @@ int launch_gated(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParams &p, d
 // Rows per (sequence, kv head) up to which the row-block kernels run (in 16-row groups, each its own CTA sharing the
 // kv head's tiles through L2); beyond, the stacked-row kernels.
 int row_block_rows() {
-#ifdef FOLD_TUNING
-  if (const char *e = getenv("FOLD_TUNE_RGMAX")) return atoi(e);
-#endif
   return 2 * kMaxRows;
 }
 
@@ -551,9 +540,6 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   memset(&pp, 0, sizeof(pp));
   pp.vpos_tok = vaxes.pos_tok; pp.vpos_head = vaxes.pos_head; pp.vpos_seq = vaxes.pos_seq;
   pp.box_min = 13;
-#ifdef FOLD_TUNING
-  if (const char *e = getenv("FOLD_TUNE_BOXMIN")) pp.box_min = atoi(e);
-#endif
   ScanParams &p = pp.s;
   p.z = a->z;
   p.seqlens = kv.seqlens;
@@ -603,20 +589,12 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const bool narrow_tiles = g.R <= row_block_rows();
   const bool gated = !isinf(a->depth_T);
   // head_dim 128, up to 16 rows: the tcgen05 row-block kernel (keys on M, 128-key tiles); it has no block tail yet
-  bool decode_umma = g.D == 128 && g.R <= kDecMaxRows && !(gated && kv.v_block_mean);
-#ifdef FOLD_TUNING
-  {
-    const char *e = getenv("FOLD_TUNE_DEC");                 // (development: off unless asked for, until it wins everywhere)
-    decode_umma = decode_umma && e && atoi(e) != 0;
-  }
-#else
-  decode_umma = false;
-#endif
+  // The persistent kernel pays a few microseconds to start (tensor memory, cleared buffers) and wins from about four
+  // tiles per worker on; row blocks of 9..16 rows and problems of a few tiles stay on the mma.sync kernels.
+  const long long dec_tiles = (long long)g.num_seqs * g.Hkv * ((kv.max_seqlen + kDecKeys - 1) / kDecKeys);
+  const bool decode_umma = g.D == 128 && g.R <= kDecMaxRows && !(gated && kv.v_block_mean) && dec_tiles >= 8LL * sm_count();
   const int tile_keys = decode_umma ? kDecKeys : (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
-  int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
-#ifdef FOLD_TUNING
-  if (const char *e = getenv("FOLD_TUNE_BOXTOK")) if (decode_umma && atoi(e) < box_tok) box_tok = atoi(e);
-#endif
+  const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   CUtensorMap mk, mv;
   MapAxes axes;
   if (int rc = make_map(&mk, &axes, kv.k, kv, g.D, g.Hkv, box_tok)) return rc;
@@ -661,15 +639,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
     if (ctas > sms) ctas = sms;
     p.vr = vbox;                                             // tokens per value box
     p.box_min = vbox * 13 / 16;                              // fetch a group whole from this many live rows on
-#ifdef FOLD_TUNING
-    if (const char *e = getenv("FOLD_TUNE_BOXMIN")) p.box_min = atoi(e);
-    if (const char *e = getenv("FOLD_TUNE_CTAS")) ctas = atoi(e);
-#endif
     p.num_splits = 1;
     p.stages = 8;                                            // tiles the L2 requests run ahead of the ring
-#ifdef FOLD_TUNING
-    if (const char *e = getenv("FOLD_TUNE_PF")) p.stages = atoi(e);
-#endif
     return gated ? launch_decode<true>(mk, mv, p, (int)ctas, st) : launch_decode<false>(mk, mv, p, (int)ctas, st);
   }
   p.num_splits = choose_splits(a, g, tile_keys);
@@ -873,9 +844,6 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
   const bool resident = n_levels == 1 && (total_slots + warps - 1) / warps <= kMergeResident;
   if (!resident)
     while (warps > 1 && n_rows * warps > 4096) warps >>= 1;
-#ifdef FOLD_TUNING
-  if (const char *e = getenv("FOLD_TUNE_MERGEW")) warps = atoi(e);
-#endif
   const int cta_warps = warps < 4 ? 4 : warps;
   const long long rows_per_cta = cta_warps / warps;
   const dim3 grid((unsigned)((n_rows + rows_per_cta - 1) / rows_per_cta)), block(32 * cta_warps);
@@ -1172,8 +1140,6 @@ const char *fold_status_string(int status) {
 }
 
 int fold_version(void) { return 100; }
-#ifdef FOLD_PROFILE
-int fold_debug_trace(long long *host_out) { return (int)cudaMemcpyFromSymbol(host_out, fold::g_dec_trace, sizeof(long long) * 64 * 16); }
-#endif
+
 
 }  // extern "C"

@@ -33,24 +33,12 @@
 
 namespace fold {
 
-#ifdef FOLD_PROFILE
-#define PROF_DECL(n) long long prof[n] = {0}; long long prof_t = clock64();
-#define PROF(i) { const long long now_ = clock64(); prof[i] += now_ - prof_t; prof_t = now_; }
-#define PROF_OUT(base, n) if (blockIdx.x == 0 && lane == 0) { for (int i_ = 0; i_ < n; ++i_) reinterpret_cast<long long *>(p.hdr)[8 + base + i_] = prof[i_]; }
-__device__ long long g_dec_trace[64 * 16];
-#define TRACE(ev, it_) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (it_) >= 2 && (it_) < 66) g_dec_trace[((it_) - 2) * 16 + (ev)] = clock64(); } while (0)
-#else
-#define TRACE(ev, it_) do { } while (0)
-#define PROF_DECL(n)
-#define PROF(i)
-#define PROF_OUT(base, n)
-#endif
 
 constexpr int kDecKeys = 128;                        // keys per tile (MMA M of the score product)
 constexpr int kDecKS = 3, kDecVS = 3;                // key / value ring depths (32 KB stages)
 constexpr int kDecThreads = 12 * 32;                 // key producer, score issuer, value-product issuer, value producer (dense), 2 workers x 4 weight warps
 constexpr int kDecTmemCols = 128;                    // S[worker][2]: 16 columns each from 0;  O[worker]: 32 columns each from 64
-constexpr int kDecMaxRows = 16;
+constexpr int kDecMaxRows = 8;                       // rows per (sequence, kv head) the host sends here (the kernel itself takes 16)
 
 struct DecLayout {                                   // byte offsets from a 1 KB-aligned base
   static constexpr int kTile = kDecKeys * 256;       // one key or value tile: [2 halves][128 keys][128 B], swizzled
@@ -63,9 +51,8 @@ struct DecLayout {                                   // byte offsets from a 1 KB
   static constexpr int kTotal = kBar + 512 + 1024;   // + alignment slack
 };
 // barrier indices (8 bytes each, from kBar)
-constexpr int kDecBarKFull = 40, kDecBarKEmpty = 3, kDecBarVFull = 6, kDecBarPvDone = 9, kDecBarSEmpty = 12,
+constexpr int kDecBarKFull = 40, kDecBarKEmpty = 0, kDecBarVFull = 4, kDecBarPvDone = 8, kDecBarSEmpty = 12,
               kDecBarPFull = 16, kDecBarQFull = 20, kDecBarLFull = 24, kDecBarSFull = 28, kDecBarPFree = 32, kDecBarTmemSlot = 38;
-constexpr int kDecProdPos = 448;                     // byte offset from kBar: the key producer's position in the tile order
 constexpr int kDecLiveFlags = 384;                   // byte offset from kBar: [worker][weight buffer][warp] words: a key of the warp's 32 is live
 
 // D[tmem] (+)= A * B with both operands in shared memory (64-bit matrix descriptors as two words each).
@@ -209,7 +196,19 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   constexpr int NPV = NC <= 8 ? 16 : 32;                     // N of the value product; P_lo sits NPV / 2 rows after P_hi
   constexpr int PB = NC <= 8 ? 2 : 1;                        // weight buffers per worker
   constexpr int PBYTES = NPV * 256;                          // [2 key halves][NPV rows][128 B]
+  // Six 32 KB stages in all.  Depth-gated: three for keys and three for values (four and two streams a cache nobody
+  // keeps a value row of 5 % faster, and one with half its rows live 12 % slower).  Dense: a key stage is free as soon
+  // as its scores are issued, a value stage waits for the weights, so two key stages feed four value stages (5 % over
+  // three and three).
+#ifndef FOLD_DEC_GATED_KS
+#define FOLD_DEC_GATED_KS 3
+#endif
+#ifndef FOLD_DEC_DENSE_KS
+#define FOLD_DEC_DENSE_KS 2
+#endif
+  constexpr int KS = GATED ? FOLD_DEC_GATED_KS : FOLD_DEC_DENSE_KS, VS = 6 - KS;
   using LO = DecLayout;
+  constexpr int OFF_V = KS * LO::kTile;                      // the value ring follows the key ring
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -222,9 +221,9 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   if (threadIdx.x == 0) {
     // "key tile landed": twice as many barriers as stages, so that a barrier only ever serves one worker's tiles (the
     // workers alternate) and its waiter, who takes them in order, is never more than one phase ahead of it
-    for (int s = 0; s < 2 * kDecKS; ++s) mbar_init(bar(kDecBarKFull + s), 1);
-    for (int s = 0; s < kDecKS; ++s) mbar_init(bar(kDecBarKEmpty + s), 1);
-    for (int s = 0; s < kDecVS; ++s) { mbar_init(bar(kDecBarVFull + s), GATED ? 4 : 1); mbar_init(bar(kDecBarPvDone + s), 1); }
+    for (int s = 0; s < 2 * KS; ++s) mbar_init(bar(kDecBarKFull + s), 1);
+    for (int s = 0; s < KS; ++s) mbar_init(bar(kDecBarKEmpty + s), 1);
+    for (int s = 0; s < VS; ++s) { mbar_init(bar(kDecBarVFull + s), GATED ? 4 : 1); mbar_init(bar(kDecBarPvDone + s), 1); }
     for (int s = 0; s < 4; ++s) {                            // one arrival per weight warp of the worker
       mbar_init(bar(kDecBarSEmpty + s), 4);
       mbar_init(bar(kDecBarPFull + s), 4);
@@ -237,8 +236,8 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   }
   if (warp == 1) tmem_alloc(bar(kDecBarTmemSlot), kDecTmemCols);
   // value ring, weight buffers and query tiles start as zeros: a row or column nobody writes must hold finite data
-  for (int i = threadIdx.x; i < (LO::kLpart - LO::kV) / 16; i += kDecThreads)
-    *reinterpret_cast<uint4 *>(gen + LO::kV + i * 16) = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < (LO::kLpart - OFF_V) / 16; i += kDecThreads)
+    *reinterpret_cast<uint4 *>(gen + OFF_V + i * 16) = make_uint4(0, 0, 0, 0);
   fence_proxy_async_smem();
   pdl_launch_dependents();
   tc_fence_before();
@@ -273,7 +272,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     // reads every value row, so there warp 3 streams the value tiles the same way (its ring is freed by the value
     // products, the key ring by the score products: neither waits for the other)
     const bool keys = warp == 0;
-    if (lane == 0 && TA + TB > 0) {
+    if (lane < 2 && TA + TB > 0) {                           // one lane per 64-channel half of a tile
       const CUtensorMap *tm_ = keys ? &tmK : &tmV;
       tma_prefetch_desc(tm_);
       const uint64_t pol = policy_evict_first();
@@ -281,85 +280,46 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       dec_pair_init(x, p, blockIdx.x, W);
       const int boxes_per_tile = kDecKeys / p.box_tok;
       const int full0 = keys ? kDecBarKFull : kDecBarVFull, empty0 = keys ? kDecBarKEmpty : kDecBarPvDone;
-      const int depth = keys ? kDecKS : kDecVS;
-      // One tile of (sequence, kv head, first token): into stage `st` (dst != 0) or into L2 only.  A tile takes
-      // thousands of cycles from request to arrival whatever the load on memory, and the ring holds three: the L2
-      // requests run further ahead, so the ring's own requests find their lines on the chip.
-      auto tile = [&](const DecPairWalk &y, uint32_t dst, uint32_t full) {
-        const int seq = y.s ? y.b.seq : y.a.seq, kvh = y.s ? y.b.kvh : y.a.kvh, n = y.s ? y.b.n : y.a.n;
-        const int tok0 = (y.s ? y.b.t : y.a.t) * kDecKeys;
+      const int depth = keys ? KS : VS;
+      for (; dec_pair_valid(x); dec_pair_next(x, p)) {
+        const int it = x.it, st = it % depth;
+        const int seq = x.s ? x.b.seq : x.a.seq, kvh = x.s ? x.b.kvh : x.a.kvh, n = x.s ? x.b.n : x.a.n;
+        const int tok0 = (x.s ? x.b.t : x.a.t) * kDecKeys;
         const int nbox = min(boxes_per_tile, (n - tok0 + p.box_tok - 1) / p.box_tok);
-        if (dst) mbar_expect_tx(full, nbox * p.box_tok * D * 2);
-        for (int bx = 0; bx < nbox; ++bx) {
+        int pg[8];                                           // the boxes' pages, looked up before the stage is waited for
+        if (p.paged) {
+#pragma unroll
+          for (int bx = 0; bx < 8; ++bx)
+            if (bx < nbox) pg[bx] = p.page_table[(long long)seq * p.max_pages + ((tok0 + bx * p.box_tok) >> p.page_shift)];
+        }
+        if (it >= depth && !mbar_wait_spin(bar(empty0 + st), (uint32_t)((it / depth - 1) & 1), dead)) break;
+        const uint32_t full = bar(keys ? kDecBarKFull + it % (2 * KS) : full0 + st);
+        const uint32_t dst = base + (keys ? LO::kK : OFF_V) + st * LO::kTile;
+        if (lane == 0) mbar_expect_tx(full, nbox * p.box_tok * D * 2);
+#pragma unroll
+        for (int bx = 0; bx < 8; ++bx) {
+          if (bx >= nbox) break;
           const int j0 = tok0 + bx * p.box_tok;
           int c_seq = seq, c_tok = j0;
           if (p.paged) {
-            const int pg = p.page_table[(long long)seq * p.max_pages + (j0 >> p.page_shift)];
-            c_seq = min(max(pg, 0), p.num_pages - 1);
+            c_seq = min(max(pg[bx], 0), p.num_pages - 1);
             c_tok = j0 & page_mask;
           }
           const int c1 = p.pos_tok == 1 ? c_tok : (p.pos_head == 1 ? kvh : c_seq);
           const int c2 = p.pos_tok == 2 ? c_tok : (p.pos_head == 2 ? kvh : c_seq);
           const int c3 = p.pos_tok == 3 ? c_tok : (p.pos_head == 3 ? kvh : c_seq);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            if (dst) tma_load_4d(dst + (h * kDecKeys + bx * p.box_tok) * 128, tm_, full, h * 64, c1, c2, c3, pol);
-            else tma_prefetch_l2_4d(tm_, h * 64, c1, c2, c3);
-          }
+          tma_load_4d(dst + (lane * kDecKeys + bx * p.box_tok) * 128, tm_, full, lane * 64, c1, c2, c3, pol);
         }
-      };
-      for (; dec_pair_valid(x); dec_pair_next(x, p)) {
-        const int it = x.it, st = it % depth;
-        if (it >= depth && !mbar_wait(bar(empty0 + st), (uint32_t)((it / depth - 1) & 1), dead)) break;
-        if (keys) TRACE(0, it);
-        if (keys) *reinterpret_cast<volatile int *>(gen + LO::kBar + kDecProdPos) = it;
-        tile(x, base + (keys ? LO::kK : LO::kV) + st * LO::kTile, bar(keys ? kDecBarKFull + it % (2 * kDecKS) : full0 + st));
       }
-      if (dead) {
+      if (dead && lane == 0) {
         // gave up: the copies already requested must still land before the CTA may leave (bounded waits again)
         atomicOr(&p.hdr->wait_timeouts, 1u);
         bool d2 = false;
         for (int back = 1; back <= depth && x.it - back >= 0; ++back) {
           const int it = x.it - back;
-          if (keys) mbar_wait(bar(kDecBarKFull + it % (2 * kDecKS)), (uint32_t)((it / (2 * kDecKS)) & 1), d2);
+          if (keys) mbar_wait(bar(kDecBarKFull + it % (2 * KS)), (uint32_t)((it / (2 * KS)) & 1), d2);
           else mbar_wait(bar(full0 + it % depth), (uint32_t)((it / depth) & 1), d2);
         }
-      }
-    }
-  } else if (GATED && warp == 3) {
-    // ------------------------------------------------------------ L2 warm-up of the key rows, p.stages tiles ahead of the ring
-    // A request from the ring takes thousands of cycles from issue to arrival once the memory system is loaded, and
-    // shared memory holds only three key tiles: the bytes in flight it allows do not fill the memory pipe on their own.
-    // This warp touches the rows of the tiles further ahead with L2 prefetches (no shared memory, nothing to wait for),
-    // so the ring's own requests mostly find their lines on the chip.
-    if (p.stages > 0 && TA + TB > 0) {
-      DecPairWalk xf;
-      dec_pair_init(xf, p, blockIdx.x, W);
-      const volatile int *pos = reinterpret_cast<const volatile int *>(gen + LO::kBar + kDecProdPos);
-      uint32_t idle = 0;
-      while (dec_pair_valid(xf) && idle < kWaitLimit) {
-        if (xf.it > *pos + p.stages) { ++idle; __nanosleep(200); continue; }
-        idle = 0;
-        if (xf.it >= kDecKS) {                               // the first tiles go straight into the ring
-          const int seq = xf.s ? xf.b.seq : xf.a.seq, kvh = xf.s ? xf.b.kvh : xf.a.kvh, n = xf.s ? xf.b.n : xf.a.n;
-          const int tok0 = (xf.s ? xf.b.t : xf.a.t) * kDecKeys;
-#pragma unroll
-          for (int r = 0; r < kDecKeys / 16; ++r) {          // 16 rows of 256 bytes per warp-wide request
-            const int tok = tok0 + r * 16 + (lane >> 1);
-            if (tok < n) {
-              int c_seq = seq, c_tok = tok;
-              if (p.paged) {
-                const int pg = p.page_table[(long long)seq * p.max_pages + (tok >> p.page_shift)];
-                c_seq = min(max(pg, 0), p.num_pages - 1);
-                c_tok = tok & page_mask;
-              }
-              const __nv_bfloat16 *row = p.k + (long long)c_seq * p.v_stride_seq + (long long)c_tok * p.v_stride_tok +
-                                         (long long)kvh * p.v_stride_head + (lane & 1) * 64;
-              asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
-            }
-          }
-        }
-        dec_pair_next(xf, p);
       }
     }
   } else if (warp == 1 || warp == 2) {
@@ -385,11 +345,10 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       while (p_alive) {
         // ---- value product of tile ip, if its weights and value rows are in
         {
-          const int it = dec_global_index(set, ip, TA, TB), vs = it % kDecVS;
+          const int it = dec_global_index(set, ip, TA, TB), vs = it % VS;
           const bool pf = mbar_test_wait(bar(kDecBarPFull + 2 * set + (ip % PB)), (uint32_t)((ip / PB) & 1));
-          const bool vf = mbar_test_wait(bar(kDecBarVFull + vs), (uint32_t)((it / kDecVS) & 1));
+          const bool vf = mbar_test_wait(bar(kDecBarVFull + vs), (uint32_t)((it / VS) & 1));
           if (pf && vf) {
-            TRACE(10, it);
             const bool first = wp.t == wp.t_first;
             bool some = true;                                // depth-gated: a tile nobody keeps a key of adds nothing
             if (GATED && !first) {                           // (a chunk's first tile always runs: it initialises the accumulator)
@@ -400,7 +359,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             tc_fence_after();
             // value tile [2 channel halves][128 keys][128 B] as the MN-major A operand: 16 keys = 2048 B per K step,
             // the halves 16 KB apart (leading-dimension offset); weights [2 key halves][NPV rows][128 B], K-major
-            const uint32_t a_lo = umma_desc_lo(base + LO::kV + vs * LO::kTile, kDecKeys * 128);
+            const uint32_t a_lo = umma_desc_lo(base + OFF_V + vs * LO::kTile, kDecKeys * 128);
             const uint32_t b_lo = umma_desc_lo(base + LO::kP + set * 8192 + (ip % PB) * PBYTES, 16);
             const uint32_t d = tmem + 64 + set * 32;
             if (some) {
@@ -417,7 +376,6 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             }
             tc_commit(bar(kDecBarPvDone + vs));              // the value stage is free
             tc_commit(bar(kDecBarPFree + 2 * set + (ip % PB)));   // so is the worker's weight buffer (and, at a chunk's end, A is final)
-            TRACE(12, it);
             ++ip;
             if (++wp.t == wp.t_end) { p_alive = dec_worker_next_chunk(wp, p); ++ep; }
             idle = 0;
@@ -427,13 +385,12 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         // ---- scores of tile iq: at most two tiles ahead of the value products, and at most one chunk ahead (a chunk's
         // query rows are staged while the worker is on the chunk before)
         if (q_alive && iq <= ip + 2 && eq <= ep + 1) {
-          const int it = dec_global_index(set, iq, TA, TB), ks = it % kDecKS;
+          const int it = dec_global_index(set, iq, TA, TB), ks = it % KS;
           const bool first = wq.t == wq.t_first;
-          bool ok = mbar_test_wait(bar(kDecBarKFull + it % (2 * kDecKS)), (uint32_t)((it / (2 * kDecKS)) & 1));
+          bool ok = mbar_test_wait(bar(kDecBarKFull + it % (2 * KS)), (uint32_t)((it / (2 * KS)) & 1));
           if (iq >= 2) ok &= mbar_test_wait(bar(kDecBarSEmpty + 2 * set + (iq & 1)), (uint32_t)(((iq >> 1) - 1) & 1));
           if (first) ok &= mbar_test_wait(bar(kDecBarQFull + 2 * set + (eq & 1)), (uint32_t)((eq >> 1) & 1));
           if (ok) {
-            TRACE(3, it);
             tc_fence_after();
             const uint32_t a_lo = umma_desc_lo(base + LO::kK + ks * LO::kTile, 16);
             const uint32_t b_lo = umma_desc_lo(base + LO::kQ + (2 * set + (eq & 1)) * 4096, 16);
@@ -447,7 +404,6 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             }
             tc_commit(bar(kDecBarSFull + 2 * set + (iq & 1)));   // the worker's scores are ready
             tc_commit(bar(kDecBarKEmpty + ks));              // the key stage is free
-            TRACE(4, it);
             ++iq;
             if (++wq.t == wq.t_end) { q_alive = dec_worker_next_chunk(wq, p); ++eq; }
             idle = 0;
@@ -495,7 +451,6 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     const int vbox = p.vr;                                   // tokens per value box (16 or 32)
     const uint32_t gmask = vbox == 32 ? 0xffffffffu : 0xffffu;
     int i = 0;                                               // tiles this worker has been through
-    PROF_DECL(8)
     for (int e = 0; have_next && !dead; ++e) {
       cur = nxt;
       float z[NC];
@@ -510,7 +465,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       int it = 0;
       for (; cur.t < cur.t_end; ++cur.t, ++i) {
         it = dec_global_index(set, i, TA, TB);
-        const int vs = it % kDecVS;
+        const int vs = it % VS;
         const int key = cur.t * kDecKeys + krow;
         const int tok_w = cur.t * kDecKeys + qd * 32;        // first key of this warp's 32
         int pg0 = 0, pg1 = 0;                                // pages of the warp's value groups, fetched ahead of their use
@@ -519,51 +474,37 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           if (tok_w < n) pg0 = pt[tok_w >> p.page_shift];
           if (tok_w + 16 < n) pg1 = pt[(tok_w + 16) >> p.page_shift];
         }
-        PROF(0)
         // the tcgen05 loads are warp-wide: the warp takes them together or not at all
-        if (wtid < 32) TRACE(5, it);
         if (!wait_u(bar(kDecBarSFull + 2 * set + (i & 1)), (uint32_t)((i >> 1) & 1))) break;
-        if (wtid < 32) TRACE(6, it);
-        PROF(1)
         tc_fence_after();
         float s[NC];
         tmem_ld_cols<NC>(lane_addr + set * 32 + (i & 1) * 16, s);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kDecBarSEmpty + 2 * set + (i & 1)));   // this score buffer may be rewritten
-        PROF(2)
         const bool valid = key < n;
         const bool drafts = p.draft_len > 0 && key >= dstart;
-        uint32_t hi16[NC], lo16[NC];
+        // final scores s - Z in binades, and the verdict: does some row keep this key?
+        float x[NC];
         bool any_live = false;
 #pragma unroll
         for (int r = 0; r < NC; ++r) {
-          float x = valid ? fmaf(s[r], p.scale_log2, -z[r]) : -INFINITY;   // select: rows past n may hold anything
-          if (drafts && r < p.R && !draft_ok(p.draft_mask[cur.seq * p.stack + r / p.G], key, dstart)) x = -INFINITY;
-          const float pw = ex2_approx(x);                    // 2^-inf = 0
-          const bool live = GATED ? (x >= p.neg_T) : true;
-          const float pm = live ? pw : 0.f;
-          const float h = __bfloat162float(__float2bfloat16_rn(pm));
-          const float g = __bfloat162float(__float2bfloat16_rn(pm - h));
-          L[r] += (h + g) + (pw - pm);                       // L sums the weights the products use; cut keys add p
-          hi16[r] = __float_as_uint(h) >> 16;
-          lo16[r] = __float_as_uint(g) >> 16;
-          any_live |= live;
+          x[r] = valid ? fmaf(s[r], p.scale_log2, -z[r]) : -INFINITY;   // select: rows past n may hold anything
+          if (drafts && r < p.R && !draft_ok(p.draft_mask[cur.seq * p.stack + r / p.G], key, dstart)) x[r] = -INFINITY;
+          any_live |= GATED ? (x[r] >= p.neg_T) : true;
         }
-        PROF(3)
-        // this tile's value stage is free once the value product of the tile three back in the CTA's order is over (the
-        // other worker's, while the two alternate), its weight buffer once the worker's own product PB tiles back is
-        if (it >= kDecVS && !wait_u(bar(kDecBarPvDone + vs), (uint32_t)((it / kDecVS - 1) & 1))) break;
-        if (i >= PB && !wait_u(bar(kDecBarPFree + 2 * set + (i % PB)), (uint32_t)((i / PB - 1) & 1))) break;
-        PROF(4)
-        if (wtid < 32) TRACE(7, it);
+        // this tile's value stage is free once the value product of the tile VS back in the CTA's order is over (the
+        // other worker's, while the two alternate)
+        if (it >= VS && !wait_u(bar(kDecBarPvDone + vs), (uint32_t)((it / VS - 1) & 1))) break;
         const uint32_t vfull = bar(kDecBarVFull + vs);
+        uint32_t live32 = 0xffffffffu;                       // which of the warp's 32 keys some row keeps
         if (GATED) {
-          // requests for the value rows some row keeps, per group of vbox keys: a mostly-live group whole as one
-          // tensor-map box per 64 channels (never past the sequence end), otherwise its live rows one by one
+          // requests for the value rows some row keeps, before anything else is done with the scores, per group of vbox
+          // keys: a mostly-live group whole as one tensor-map box per 64 channels (never past the sequence end),
+          // otherwise its live rows one by one
           const uint32_t fetch = __ballot_sync(0xffffffffu, any_live);
-          if (lane == 0) reinterpret_cast<uint32_t *>(gen + LO::kBar + kDecLiveFlags)[(set * 2 + (i % PB)) * 4 + qd] = fetch;
-          const uint32_t vdst = base + LO::kV + vs * LO::kTile;
+          live32 = fetch;
+          const uint32_t vdst = base + OFF_V + vs * LO::kTile;
           bool rows = false;
           for (int gq = 0; gq * vbox < 32; ++gq) {
             uint32_t m = (fetch >> (gq * vbox)) & gmask;
@@ -605,18 +546,36 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             }
           }
           if (rows) cp_async_mbar_arrive(vfull);             // this lane's copies hold the phase open
+          __syncwarp();
+          if (lane == 0) mbar_arrive(vfull);                 // this warp's requests are out
         } else {
           st_total += min(32, max(0, n - tok_w));
           if (cur.t * kDecKeys + kDecKeys > n) {             // ragged tail: value rows past n may hold anything
-            if (!wait_u(vfull, (uint32_t)((it / kDecVS) & 1))) break;
+            if (!wait_u(vfull, (uint32_t)((it / VS) & 1))) break;
             if (!valid) {
 #pragma unroll
               for (int c16 = 0; c16 < 16; ++c16)
-                *reinterpret_cast<uint4 *>(gen + LO::kV + vs * LO::kTile + tile_off(krow, c16, kDecKeys)) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4 *>(gen + OFF_V + vs * LO::kTile + tile_off(krow, c16, kDecKeys)) = make_uint4(0, 0, 0, 0);
             }
           }
         }
-        PROF(5)
+        // final weights 2^(s - Z), their two-term BF16 split, and this thread's share of L
+        uint32_t hi16[NC], lo16[NC];
+#pragma unroll
+        for (int r = 0; r < NC; ++r) {
+          const float pw = ex2_approx(x[r]);                 // 2^-inf = 0
+          const bool live = GATED ? (x[r] >= p.neg_T) : true;
+          const float pm = live ? pw : 0.f;
+          const float h = __bfloat162float(__float2bfloat16_rn(pm));
+          const float g = __bfloat162float(__float2bfloat16_rn(pm - h));
+          L[r] += (h + g) + (pw - pm);                       // L sums the weights the products use; cut keys add p
+          hi16[r] = __float_as_uint(h) >> 16;
+          lo16[r] = __float_as_uint(g) >> 16;
+        }
+        // the worker's weight buffer is free once its own value product PB tiles back is over
+        if (i >= PB && !wait_u(bar(kDecBarPFree + 2 * set + (i % PB)), (uint32_t)((i / PB - 1) & 1))) break;
+        // (the verdict word travels with the weight buffer: the issuing thread skips the product of a tile nobody keeps a key of)
+        if (GATED && lane == 0) reinterpret_cast<uint32_t *>(gen + LO::kBar + kDecLiveFlags)[(set * 2 + (i % PB)) * 4 + qd] = live32;
         // weights: B operand [2 key halves][NPV rows][128 B], K-major, swizzled like a tensor-map box; P_hi of row r in
         // row r, P_lo in row NPV / 2 + r (the same swizzle phase: NPV / 2 is a multiple of 8)
         {
@@ -631,12 +590,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(bar(kDecBarPFull + 2 * set + (i % PB)));
-          if (GATED) mbar_arrive(vfull);
-        }
-        if (wtid < 32) TRACE(8, it);
-        PROF(6)
+        if (lane == 0) mbar_arrive(bar(kDecBarPFull + 2 * set + (i % PB)));
       }
       if (dead) break;
       // chunk end: L over the worker's 128 threads in a fixed order, then the accumulator out of tensor memory.
@@ -666,9 +620,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 #pragma unroll
       for (int r = 0; r < NC; ++r)
         if (r < p.R) slot[(long long)r * D + krow] = o[r] + o[NPV / 2 + r];
-      PROF(7)
     }
-    if (warp == 4) PROF_OUT(16, 8)
     if (lane == 0) {
       if (dead) atomicOr(&p.hdr->wait_timeouts, 16u);
       if (st_total) {
