@@ -589,10 +589,9 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   const bool narrow_tiles = g.R <= row_block_rows();
   const bool gated = !isinf(a->depth_T);
   // head_dim 128, up to 16 rows: the tcgen05 row-block kernel (keys on M, 128-key tiles); it has no block tail yet
-  // The persistent kernel pays a few microseconds to start (tensor memory, cleared buffers) and wins from about four
-  // tiles per worker on; row blocks of 9..16 rows and problems of a few tiles stay on the mma.sync kernels.
-  const long long dec_tiles = (long long)g.num_seqs * g.Hkv * ((kv.max_seqlen + kDecKeys - 1) / kDecKeys);
-  const bool decode_umma = g.D == 128 && g.R <= kDecMaxRows && !(gated && kv.v_block_mean) && dec_tiles >= 8LL * sm_count();
+  // Which kernel runs may depend on the head dimension, the rows per (sequence, kv head), the depth being finite and
+  // the block tail only -- never on the batch or on lengths: a slot's bits must not depend on what else is decoded.
+  const bool decode_umma = g.D == 128 && g.R <= kDecMaxRows && !(gated && kv.v_block_mean);
   const int tile_keys = decode_umma ? kDecKeys : (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
   const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   CUtensorMap mk, mv;

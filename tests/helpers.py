@@ -18,9 +18,13 @@ from paper_2609_33410_b200.workloads import DecodeWorkload, bf16_bits
 #                    at the same Z and T  <=  1.5 x the error of a plain BF16 online-softmax
 #                    kernel (emulated) against float64 softmax attention, plus the mass of keys
 #                    within 2^-10 binades of the threshold (fp32 vs fp64 scores may flip them).
+#   every row by itself, finite T:  |out - oracle|_inf <= 1e-2 * max|V| + that row's threshold slack, and
+#                    |out - oracle|_2 <= 3 x (that row's own yardstick error, or 5e-3 |oracle|_2 where no yardstick is
+#                    computed) + sqrt(D) x the row's slack: one wrong row or channel among many cannot hide in a pooled norm.
 DENSE_MAX_ABS = 1e-2
 DENSE_MEAN_REL = 5e-3
 FINITE_T_FACTOR = 1.5
+ROW_FACTOR = 3.0
 Z_TOL = 1e-3
 LSE_TOL = 2e-3
 
@@ -89,6 +93,7 @@ def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False
     max_abs = 0.0
     vmax = 0.0
     rel_rows, slack_sum, dz = [], 0.0, 0.0
+    per_row = []                                             # (b, h, |d|_2, |d|_inf, |ref|_2, slack, max|V| of the row's cache)
     for (b, h) in rows:
         q, K, V = row_inputs(w, b, h)
         n = K.shape[0]
@@ -110,12 +115,17 @@ def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False
         if check_estimate:
             dz = max(dz, abs(O.estimate_z(lambda i: s[i], n) - z[b, h]))
         if not math.isinf(T):
-            slack_sum += ((2.0 if vm is not None else 1.0) * O.cut_report(s, V, z[b, h], T)["slack"]) ** 2 * V.shape[1]
+            row_slack = (2.0 if vm is not None else 1.0) * O.cut_report(s, V, z[b, h], T)["slack"]
+            slack_sum += row_slack ** 2 * V.shape[1]
+            yard_row = None
             if yardstick:
                 o_dense, _ = O.dense_row(s, V)
                 vis = np.isfinite(s)
                 y = O.online_softmax_bf16(q, K[vis], V[vis], w.scale) - o_dense
                 ynum += float(y @ y)
+                yard_row = float(np.linalg.norm(y))
+            per_row.append((b, h, float(np.linalg.norm(d)), float(np.abs(d).max()), float(np.linalg.norm(o_ref)), row_slack,
+                            float(np.abs(V).max()), yard_row))
     res = dict(rel_l2=math.sqrt(num / max(den, 1e-300)), max_abs=max_abs, vmax=vmax,
                mean_rel=float(np.mean(rel_rows)) if rel_rows else 0.0, dz=dz)
     if math.isinf(T):
@@ -126,6 +136,14 @@ def compare(w: DecodeWorkload, bufs, T=math.inf, rows=None, check_estimate=False
         res["slack"] = math.sqrt(slack_sum / max(den, 1e-300))
         # (1e-12: a one-key row is exact on both sides, and 0 <= 1.5 x 0 must not hinge on the oracle's own rounding)
         assert res["rel_l2"] <= FINITE_T_FACTOR * res["yard"] + res["slack"] + 1e-12, res
+    if not math.isinf(T):
+        # row by row, element by element: the pooled norm above cannot see one bad row among dozens
+        D = w.head_dim
+        for (b, h, d2, dinf, r2, row_slack, row_vmax, yard_row) in per_row:
+            tol = yard_row if yard_row is not None else DENSE_MEAN_REL * r2
+            assert dinf <= DENSE_MAX_ABS * row_vmax + row_slack + 1e-30, (b, h, dinf, row_vmax, row_slack)
+            assert d2 <= ROW_FACTOR * tol + math.sqrt(D) * row_slack + 1e-12, (b, h, d2, r2, tol, row_slack)
+        res["max_row_rel"] = max([d2 / max(r2, 1e-300) for (_, _, d2, _, r2, _, _, _) in per_row] + [0.0])
     if check_estimate:
         assert dz <= Z_TOL, res
     return res

@@ -11,7 +11,7 @@ import paper_2609_33410_b200 as F
 from oracle import fold_oracle as O
 from oracle import fold_planes_oracle as P
 from paper_2609_33410_b200.workloads import make_decode_workload, bf16_bits
-from helpers import cache_of, oracle_block_means, same_bits, DENSE_MAX_ABS, DENSE_MEAN_REL, FINITE_T_FACTOR, LSE_TOL, Z_TOL
+from helpers import cache_of, oracle_block_means, same_bits, DENSE_MAX_ABS, DENSE_MEAN_REL, FINITE_T_FACTOR, LSE_TOL, ROW_FACTOR, Z_TOL
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -112,6 +112,7 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
     num = den = ynum = slack2 = 0.0
     max_abs = vmax = dz = 0.0
     rel_rows = []
+    per_row = []                                             # (b, h, |d|_2, |d|_inf, |ref|_2, slack, max|V|): judged row by row below
     n_live = n_ref = n_keys = n_refv = 0
     vfp8 = cache.v_plane_1 is not None
     for (seq, kvh) in units:
@@ -169,6 +170,8 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
                 o_dense = O.dense_row(O.scores(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], w.scale), V[keep])[0]
                 y = O.online_softmax_bf16(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], V[keep], w.scale) - o_dense
                 ynum += float(y @ y)
+                per_row.append((b, h, float(np.linalg.norm(d)), float(np.abs(d).max()), float(np.linalg.norm(o_ref)), sl,
+                                float(vinf.max()), float(np.linalg.norm(y))))
     res = dict(rel_l2=math.sqrt(num / max(den, 1e-300)), max_abs=max_abs, vmax=vmax,
                mean_rel=float(np.mean(rel_rows)) if rel_rows else 0.0, dz=dz,
                live_frac=n_live / max(n_keys, 1), refine_frac=n_ref / max(n_keys, 1))
@@ -178,6 +181,10 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
     else:
         res["yard"] = math.sqrt(ynum / max(den, 1e-300)); res["slack"] = math.sqrt(slack2 / max(den, 1e-300))
         assert res["rel_l2"] <= FINITE_T_FACTOR * res["yard"] + res["slack"] + 1e-12, res
+        # and every row by itself (a pooled norm cannot see one bad row or channel among dozens)
+        for (b, h, d2, dinf, r2, sl, row_vmax, yard_row) in per_row:
+            assert dinf <= DENSE_MAX_ABS * row_vmax + sl + 1e-30, (b, h, dinf, row_vmax, sl)
+            assert d2 <= ROW_FACTOR * yard_row + math.sqrt(w.head_dim) * sl + 1e-12, (b, h, d2, r2, yard_row, sl)
     if check_estimate:
         assert dz <= Z_TOL, res
     if check_counts and len(units) == w.num_seqs * w.num_kv_heads:
