@@ -431,13 +431,16 @@ def main():
     cache_bytes = sum(l.cache_bytes() for l in levels)                    # unique bytes: a shared prefix counts once
     flat_bytes = sum(l.cache_bytes() * l.stack for l in levels)           # what a flat decode of every request reads
 
+    # a cascade's first level may be scanned on a side stream of the caller's (fork / join inside the one C-ABI call)
+    cside = F.CascadeSide(dev) if cascade and args.cascade_streams == 1 else None
+
     def make(depth, z_mode):
         return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
                             num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
                             row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
                             draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau,
-                            refine_tau_v=args.refine_tau_v)
-                for l, c, b in zip(levels, caches, lbufs)]
+                            refine_tau_v=args.refine_tau_v, side=cside if i == 0 else None)
+                for i, (l, c, b) in enumerate(zip(levels, caches, lbufs))]
 
     # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
     # is scanned on a side stream while the suffix level is scanned on the main one (fork / join with events).

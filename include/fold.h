@@ -14,9 +14,17 @@
  * z, lse and depth_T are all in binades; natural-log lse = ln(2) * lse.
  *
  * Pointers.  Unless a comment says HOST, every pointer is a DEVICE pointer owned by the
- * caller.  The library allocates, frees and retains nothing.  Every call enqueues work
- * on `stream` and returns without synchronising the host.  Calls that share a workspace
- * must be ordered by the caller (same stream, or events).
+ * caller.  The library allocates and frees nothing and keeps no device resource (no stream,
+ * no event, no buffer beyond the static scratch array of fold_decode_static); the only state it
+ * holds is, per device, "this kernel has been allowed its shared memory" flags and the address of
+ * that array, both set at a first call and safe against host threads racing on it.  Every call
+ * enqueues work on `stream` and returns without synchronising the host; every call can be captured
+ * in a CUDA graph.  Calls that share a workspace must be ordered by the caller (same stream, or events).
+ *
+ * Values.  Key and value rows of tokens below seqlens[] must be finite.  The depth gate never reads the value row
+ * of a key no row keeps, but a row that IS read under a weight of zero (a cut key inside a group of keys fetched
+ * whole) is multiplied, not skipped: a NaN or infinity stored there would reach the outputs of that (sequence, kv
+ * head).  Rows at or beyond seqlens[] may hold anything.
  *
  * Errors.  Functions return a fold_status.  Only host-detectable conditions are
  * returned (bad arguments, unsupported shapes, workspace too small, a CUDA launch
@@ -53,6 +61,16 @@ typedef enum fold_zmode {
   FOLD_Z_EXACT_MAX = 2, /* test mode: an extra full pass sets z = max_j s_ij; written to z[] */
   FOLD_Z_ZERO = 3       /* z = 0 for every row; written to z[] */
 } fold_zmode;
+
+/* Bits of fold_args.flags. */
+enum {
+  FOLD_INPUTS_SETTLED = 1  /* q, the cache rows, seqlens, page_table and draft_mask were complete before the kernel that
+                              precedes this call on `stream` STARTED (they were not written by it).  The call's first
+                              kernel may then begin, and read them, while that kernel is still draining (programmatic
+                              dependent launch); everything it writes still waits.  Without the flag the first kernel is
+                              launched in plain stream order, which is what a decode loop that appends to the cache or
+                              projects q just before the call needs. */
+};
 
 /* Bits of row_status[b * num_q_heads + h]. */
 enum {
@@ -175,6 +193,10 @@ typedef struct fold_args {
                                           INFINITY = every live key; negative = none (plane A scores only) */
   float refine_tau_v;                  /* E4M3 value planes only: the refine-V gate, binades, like refine_tau.
                                           0 = choose: max(log2(n) + 1, 4); INFINITY = every live key; negative = none */
+  int32_t flags;                       /* FOLD_INPUTS_SETTLED or 0 */
+  fold_stream side_stream;             /* fold_decode_cascade, levels[0] only: a second stream of the caller's and two */
+  void *side_fork_event;               /* cudaEvent_t of the caller's (created with timing disabled, say) on which the */
+  void *side_join_event;               /* first level is scanned; all three NULL: every level on `stream` */
 } fold_args;
 
 /* First 64 bytes of every workspace, zeroed at the start of each scan. */
@@ -253,9 +275,11 @@ int fold_decode(const fold_args *args, fold_stream stream);
  * head_dim, softmax_scale and depth_T; each level has its own kv, stack and workspace.
  * levels[0]->z_mode is FOLD_Z_ESTIMATE (estimate over all levels, written to z) or FOLD_Z_GIVEN;
  * out, lse and row_status are taken from levels[0].
- * With two or more levels the first level is scanned on a stream the library keeps per device (created, with two
- * events, at the first such call on the device: make that call outside stream capture), forked from and joined
- * back into `stream` with events, so to the caller the call is still one ordered piece of work on `stream`. */
+ * With two or more levels and levels[0]->side_stream / side_fork_event / side_join_event set (a stream and two events the
+ * CALLER owns, the stream different from `stream`), the first level is scanned on the side stream, forked from and
+ * joined back into `stream` with the events, so to the caller the call is still one ordered piece of work on `stream`;
+ * the events are recorded by every such call, so calls that share them must not overlap.  Without them every level
+ * is scanned on `stream`. */
 int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_stream stream);
 
 /* Fill kv->v_block_mean (DEVICE memory of the caller, laid out as the fold_kv comment says, at least
@@ -325,10 +349,11 @@ int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_b
  *
  * Limits and rules:
  *  - A call whose fold_workspace_bytes(args) exceeds FOLD_STATIC_SCRATCH_BYTES is refused with
- *    FOLD_ETOOLARGE before anything is enqueued (the default benchmark shape -- 16 requests x 8 kv
- *    heads x 32768 keys, group 4, head_dim 128 -- needs 8.1 MiB).
+ *    FOLD_ETOOLARGE before anything is enqueued (16 requests x 8 kv heads x 32768 keys at group 4,
+ *    head_dim 128, need 8.1 MiB).
  *  - The first call on each device looks up the array's device address (with that device current);
  *    make that first call outside any stream capture.  Later calls on the device reuse the address.
+ *    Host threads that race on that first call look up the same address and store the same value.
  *  - All calls on a device share the one array, and it keeps whatever the previous call left.  The
  *    library re-zeroes the part that must start at zero (the header) at the start of every call and
  *    never reads a slot the same call has not written, so stale contents are harmless -- but two

@@ -21,6 +21,7 @@ FOLD_OK, FOLD_EINVAL, FOLD_EUNSUPPORTED, FOLD_EWORKSPACE, FOLD_ECUDA, FOLD_ETOOL
 STATIC_SCRATCH_BYTES = 16 << 20
 Z_ESTIMATE, Z_GIVEN, Z_EXACT_MAX, Z_ZERO = range(4)
 ROW_RANGE, ROW_NONFINITE, ROW_EMPTY = 1, 2, 4
+INPUTS_SETTLED = 1                               # fold_args.flags
 
 
 class FoldKV(C.Structure):
@@ -47,7 +48,8 @@ class FoldArgs(C.Structure):
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("out", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p),
                 ("draft_mask", C.c_void_p), ("draft_len", C.c_int32), ("refine_tau", C.c_float),
-                ("refine_tau_v", C.c_float)]
+                ("refine_tau_v", C.c_float), ("flags", C.c_int32),
+                ("side_stream", C.c_void_p), ("side_fork_event", C.c_void_p), ("side_join_event", C.c_void_p)]
 
 
 class FoldPartials(C.Structure):
@@ -227,7 +229,8 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
               workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
               lse: Optional[torch.Tensor] = None, row_status: Optional[torch.Tensor] = None,
               draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0,
-              refine_tau_v: float = 0.0) -> FoldArgs:
+              refine_tau_v: float = 0.0, flags: int = 0, side=None) -> FoldArgs:
+    """`side`: a CascadeSide (a second stream and two events of the caller's) for fold_decode_cascade's first level."""
     assert q.dtype == torch.bfloat16 and q.dim() == 3 and q.stride(2) == 1
     B, Hq, D = q.shape
     a = FoldArgs()
@@ -250,7 +253,22 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
     a.draft_mask, a.draft_len = (_ptr(draft_mask), int(draft_len)) if draft_len else (None, 0)
     a.refine_tau = float(refine_tau)
     a.refine_tau_v = float(refine_tau_v)
+    a.flags = int(flags)
+    if side is not None:
+        a.side_stream, a.side_fork_event, a.side_join_event = side.stream.cuda_stream, side.fork.cuda_event, side.join.cuda_event
     return a
+
+
+class CascadeSide:
+    """A side stream and two events owned by the caller, handed to fold_decode_cascade through the first level's
+    arguments (the library keeps no stream or event of its own).  Keep the object alive while calls that use it run."""
+
+    def __init__(self, device=None):
+        self.stream = torch.cuda.Stream(device=device)
+        self.fork, self.join = torch.cuda.Event(), torch.cuda.Event()
+        for e in (self.fork, self.join):                     # torch creates the CUDA event at its first record
+            e.record(self.stream)
+        self.stream.synchronize()
 
 
 def fold_workspace_bytes(args: FoldArgs) -> int:
@@ -389,10 +407,11 @@ def alloc_buffers(q: torch.Tensor, cache: KVCache, stack: int = 1) -> DecodeBuff
 def decode(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, depth_T: float = math.inf,
            z_mode: int = Z_ESTIMATE, num_splits: int = 0, scale: Optional[float] = None, stack: int = 1,
            draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0,
-           refine_tau_v: float = 0.0, stream=None) -> FoldArgs:
+           refine_tau_v: float = 0.0, flags: int = 0, stream=None) -> FoldArgs:
     args = make_args(q, cache, scale=scale, z_mode=z_mode, z=bufs.z, depth_T=depth_T, num_splits=num_splits,
                      stack=stack, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status,
-                     draft_mask=draft_mask, draft_len=draft_len, refine_tau=refine_tau, refine_tau_v=refine_tau_v)
+                     draft_mask=draft_mask, draft_len=draft_len, refine_tau=refine_tau, refine_tau_v=refine_tau_v,
+                     flags=flags)
     fold_decode(args, stream)
     return args
 

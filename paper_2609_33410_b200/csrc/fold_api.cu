@@ -4,7 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-#include <mutex>
+#include <atomic>
 
 #include "fold_common.cuh"
 #include "fold_estimate.cuh"
@@ -39,7 +39,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // bytes after the slots for the split query rows: codes [rows][2][D], then one eta per row
 inline size_t qplane_bytes(long long rows, int D) { return round_up((size_t)rows * 2 * D, 256) + round_up((size_t)rows * 4, 256); }
 
-int check_kv(const fold_kv &kv, int D) {
+int check_kv(const fold_kv &kv, int D, int Hkv) {
   const bool planes = kv.k_plane_a != nullptr, vplanes = kv.v_plane_1 != nullptr;
   if ((!kv.k && !planes) || (!kv.v && !vplanes) || !kv.seqlens) return FOLD_EINVAL;
   if (vplanes) {
@@ -59,6 +59,15 @@ int check_kv(const fold_kv &kv, int D) {
   if (kv.num_seqs < 1 || kv.max_seqlen < 0) return FOLD_EINVAL;
   if (kv.stride_tok < D || kv.stride_head < 0 || kv.stride_seq < 0) return FOLD_EINVAL;
   if (kv.stride_tok % 8 || kv.stride_head % 8 || kv.stride_seq % 8) return FOLD_EINVAL;
+  // an axis with more than one entry needs a stride that spans a row: a broadcast (zero) stride would make the tensor
+  // maps and the plain loads disagree about where rows lie
+  if (Hkv > 1 && kv.stride_head < D) return FOLD_EINVAL;
+  if ((kv.page_table ? kv.num_pages : kv.num_seqs) > 1 && kv.stride_seq < D) return FOLD_EINVAL;
+  if (planes) {
+    if (Hkv > 1 && kv.plane_stride_head < D) return FOLD_EINVAL;
+    if ((kv.page_table ? kv.num_pages : kv.num_seqs) > 1 && kv.plane_stride_seq < D) return FOLD_EINVAL;
+  }
+  if (kv.v_block_mean && Hkv > 1 && kv.mean_stride_head < D) return FOLD_EINVAL;
   if (kv.page_table) {
     if (kv.page_size < 16 || (kv.page_size & (kv.page_size - 1))) return FOLD_EUNSUPPORTED;
     if (kv.num_pages < 1 || kv.max_pages_per_seq < 1) return FOLD_EINVAL;
@@ -83,7 +92,7 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   if (a->batch > 65535) return FOLD_EUNSUPPORTED;           // requests and sequences index a grid's y / z dimension
   if (!a->q || !aligned(a->q, 16) || a->q_stride_b % 8 || a->q_stride_h % 8) return FOLD_EINVAL;
   if (a->q_stride_h < a->head_dim && a->num_q_heads > 1) return FOLD_EINVAL;
-  if (int rc = check_kv(a->kv, a->head_dim)) return rc;
+  if (int rc = check_kv(a->kv, a->head_dim, a->num_kv_heads)) return rc;
   if (!(a->softmax_scale > 0.f) || isinf(a->softmax_scale)) return FOLD_EINVAL;
   if (a->z_mode < FOLD_Z_ESTIMATE || a->z_mode > FOLD_Z_ZERO) return FOLD_EINVAL;
   if (!a->z || !aligned(a->z, 4)) return FOLD_EINVAL;
@@ -201,6 +210,18 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   cfg.attrs = attr; cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
+// The first kernel of a call reads the caller's inputs (q, the newest cache rows, seqlens, the page table) before its
+// dependency wait.  Behind a kernel of the library that is safe; behind the CALLER's kernel it is only safe if those
+// inputs were complete before that kernel started, which the caller says with FOLD_INPUTS_SETTLED.  Otherwise the
+// kernel is launched in plain stream order.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_first(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  if (early) return launch_pdl(kernel, grid, block, smem, st, args...);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 KvLevel kv_level(const fold_kv &kv, int stack) {
   KvLevel L;
@@ -270,8 +291,9 @@ int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st, 
     fold_fill_kernel<<<(rows + 255) / 256, 256, 0, st>>>(a->z, rows, 0.f);
   }
   const dim3 grid(g.Hkv, g.B);
-  const cudaError_t rc = g.D == 128 ? launch_pdl(fold_planes_front_kernel<128>, grid, dim3(kFrontThreads), 0, st, p)
-                                    : launch_pdl(fold_planes_front_kernel<64>, grid, dim3(kFrontThreads), 0, st, p);
+  const bool early = (a->flags & FOLD_INPUTS_SETTLED) != 0;
+  const cudaError_t rc = g.D == 128 ? launch_first(early, fold_planes_front_kernel<128>, grid, dim3(kFrontThreads), 0, st, p)
+                                    : launch_first(early, fold_planes_front_kernel<64>, grid, dim3(kFrontThreads), 0, st, p);
   if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
@@ -293,8 +315,9 @@ int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st, boo
     p.hdr[0] = (zero_header && a->z_mode == FOLD_Z_ESTIMATE) ? static_cast<fold_ws_header *>(a->workspace) : nullptr;
     const dim3 grid(g.Hkv, g.B);
     if (a->z_mode == FOLD_Z_ESTIMATE) {
-      const cudaError_t rc = g.D == 128 ? launch_pdl(fold_estimate_kernel<128>, grid, dim3(kEstSampleThreads), 0, st, p)
-                                        : launch_pdl(fold_estimate_kernel<64>, grid, dim3(kEstSampleThreads), 0, st, p);
+      const bool early = (a->flags & FOLD_INPUTS_SETTLED) != 0;
+      const cudaError_t rc = g.D == 128 ? launch_first(early, fold_estimate_kernel<128>, grid, dim3(kEstSampleThreads), 0, st, p)
+                                        : launch_first(early, fold_estimate_kernel<64>, grid, dim3(kEstSampleThreads), 0, st, p);
       if (rc != cudaSuccess) return FOLD_ECUDA;
     } else {
       if (g.D == 128) fold_exact_max_kernel<128><<<grid, kEstThreads, 0, st>>>(p);
@@ -304,14 +327,18 @@ int launch_reference(const fold_args *a, const Geometry &g, cudaStream_t st, boo
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
+// The opt-in to large dynamic shared memory is a per-device attribute of the kernel: set at the kernel's first launch on
+// a device and remembered in an atomic flag (two host threads racing on a first launch both set it; that is harmless).
+// These flags and the address of the static scratch array are the only state the library keeps: no device resources.
+typedef std::atomic<int> SmemFlags[64];
 template <typename Kernel>
-int opt_in_smem(Kernel k, int *configured) {
+int opt_in_smem(Kernel k, SmemFlags &configured) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return FOLD_ECUDA;
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCtaMax) != cudaSuccess)
       return FOLD_ECUDA;
-    if (dev >= 0 && dev < 64) configured[dev] = 1;
+    if (dev >= 0 && dev < 64) configured[dev].store(1, std::memory_order_release);
   }
   return FOLD_OK;
 }
@@ -327,7 +354,7 @@ int launch_dense_n(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, 
   if (stages < 2) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = 0;
-  static int configured[64] = {0};
+  static SmemFlags configured;
   if (int rc = opt_in_smem(fold_scan_dense_kernel<D>, configured)) return rc;
   if (launch_pdl(fold_scan_dense_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages, p.R), st, mk, mv, p) != cudaSuccess)
     return FOLD_ECUDA;
@@ -344,7 +371,7 @@ int launch_dense_nt2(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p
   if (stages < 2) return FOLD_EUNSUPPORTED;
   p.stages = stages;
   p.vr = 0;
-  static int configured[64] = {0};
+  static SmemFlags configured;
   if (int rc = opt_in_smem(fold_scan_dense_nt2_kernel<D>, configured)) return rc;
   if (launch_pdl(fold_scan_dense_nt2_kernel<D>, grid, dim3(kDenseThreads), LO::total(stages), st, mk, mv, p) != cudaSuccess)
     return FOLD_ECUDA;
@@ -369,7 +396,7 @@ int launch_stacked_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &
   p.stages = stages;
   p.vr = 0;
   grid.x *= (p.R + 63) / 64;
-  static int configured[64] = {0};
+  static SmemFlags configured;
   if (int e = opt_in_smem(fold_scan_stacked_kernel<D, GATED, TAIL>, configured)) return e;
   if (launch_pdl(fold_scan_stacked_kernel<D, GATED, TAIL>, grid, dim3(kDenseThreads),
                  LO::total(stages, 0) + stages * (kStageBytes - LO::kStage), st, mk, mv, p) != cudaSuccess)
@@ -388,7 +415,7 @@ int launch_stacked_umma(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams
   p.stages = kUmmaStages;
   p.vr = 0;
   grid.x *= (p.R + kUmmaRows - 1) / kUmmaRows;
-  static int configured_g[64] = {0}, configured_d[64] = {0};
+  static SmemFlags configured_g, configured_d;
   cudaError_t rc;
   if (gated) {
     if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<true>, configured_g)) return e;
@@ -407,7 +434,7 @@ int launch_stacked_pair(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams
   p.stages = kPairStages;
   p.vr = 0;
   grid.x *= (p.R + kPairRows - 1) / kPairRows;
-  static int configured_g[64] = {0}, configured_d[64] = {0};
+  static SmemFlags configured_g, configured_d;
   cudaError_t rc;
   if (gated) {
     if (int e = opt_in_smem(fold_scan_stacked_pair_kernel<true>, configured_g)) return e;
@@ -429,7 +456,7 @@ int sm_count() {
 }
 template <bool GATED, int NC>
 int launch_decode_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, int ctas, cudaStream_t st) {
-  static int configured[64] = {0};
+  static SmemFlags configured;
   if (int rc = opt_in_smem(fold_scan_decode_kernel<GATED, NC>, configured)) return rc;
   if (launch_pdl(fold_scan_decode_kernel<GATED, NC>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p) != cudaSuccess)
     return FOLD_ECUDA;
@@ -454,7 +481,7 @@ int launch_gated_narrow(const CUtensorMap &mk, const CUtensorMap &mvs, ScanParam
   if (nstages < 2 || nvr < 1 || LN::total(nstages, nvr) > kSmemPerCtaMax) return FOLD_EUNSUPPORTED;
   p.stages = nstages;
   p.vr = nvr;
-  static int configured[64] = {0};
+  static SmemFlags configured;
   if (int rc = opt_in_smem(fold_scan_gated_narrow_kernel<D, TAIL, NT>, configured)) return rc;
   if (launch_pdl(fold_scan_gated_narrow_kernel<D, TAIL, NT>, grid, dim3(kGatedThreads), LN::total(nstages, nvr), st, mk, mvs, p) !=
       cudaSuccess)
@@ -507,7 +534,7 @@ int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanPara
   if (stages > LO::kMaxStages) stages = LO::kMaxStages;
   if (stages < 2) return FOLD_EUNSUPPORTED;
   pp.s.stages = stages;
-  static int configured[64] = {0};
+  static SmemFlags configured;
   if (int rc = opt_in_smem(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8>, configured)) return rc;
   if (launch_pdl(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) !=
       cudaSuccess)
@@ -669,30 +696,6 @@ void fill_partials(const fold_args *a, const Geometry &g, fold_partials *dst) {
   dst->max_seqlen = a->kv.max_seqlen;
 }
 
-// One non-blocking stream and two events per device for fold_decode_cascade's fork / join, created at the first
-// cascade call on the device.  Null if they cannot be created: the cascade then runs on the caller's stream alone.
-struct CascadeSide {
-  std::mutex mu;
-  cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
-  int state = 0;                                             // 0 untried, 1 ready, -1 unavailable
-};
-CascadeSide *cascade_side() {
-  static CascadeSide sides[64];
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  CascadeSide *s = &sides[dev];
-  std::lock_guard<std::mutex> lock(s->mu);
-  if (s->state == 0) {
-    const bool ok = cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) == cudaSuccess &&
-                    cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) == cudaSuccess &&
-                    cudaEventCreateWithFlags(&s->join, cudaEventDisableTiming) == cudaSuccess;
-    if (!ok) (void)cudaGetLastError();
-    s->state = ok ? 1 : -1;
-  }
-  return s->state == 1 ? s : nullptr;
-}
-
 }  // namespace
 
 extern "C" {
@@ -763,7 +766,7 @@ int estimate_levels(const fold_args *const *levels, int n_levels, fold_stream st
     if (!a || a->head_dim != a0->head_dim || a->num_kv_heads != a0->num_kv_heads || a->batch != a0->batch)
       return FOLD_EINVAL;
     if (a->stack < 1 || a->batch % a->stack || a->batch / a->stack != a->kv.num_seqs) return FOLD_EINVAL;
-    if (int rc = check_kv(a->kv, a->head_dim)) return rc;
+    if (int rc = check_kv(a->kv, a->head_dim, a->num_kv_heads)) return rc;
     p.lv[l] = kv_level(a->kv, a->stack);
     if (zero_headers) {
       if (!a->workspace || !aligned(a->workspace, 256)) return FOLD_EINVAL;
@@ -773,8 +776,9 @@ int estimate_levels(const fold_args *const *levels, int n_levels, fold_stream st
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid(g.Hkv, g.B);
-  const cudaError_t rc = g.D == 128 ? launch_pdl(fold_estimate_kernel<128>, grid, dim3(kEstSampleThreads), 0, st, p)
-                                    : launch_pdl(fold_estimate_kernel<64>, grid, dim3(kEstSampleThreads), 0, st, p);
+  const bool early = (a0->flags & FOLD_INPUTS_SETTLED) != 0;
+  const cudaError_t rc = g.D == 128 ? launch_first(early, fold_estimate_kernel<128>, grid, dim3(kEstSampleThreads), 0, st, p)
+                                    : launch_first(early, fold_estimate_kernel<64>, grid, dim3(kEstSampleThreads), 0, st, p);
   if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
@@ -863,7 +867,7 @@ int fold_block_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim, 
   if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
   if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
   if (!kv->v_block_mean) return FOLD_EINVAL;
-  if (int rc = check_kv(*kv, head_dim)) return rc;
+  if (int rc = check_kv(*kv, head_dim, num_kv_heads)) return rc;
   const int max_blocks = (kv->max_seqlen + 63) / 64;
   if (max_blocks == 0) return FOLD_OK;
   MeanParams p;
@@ -887,7 +891,7 @@ int fold_running_means(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim
   if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
   if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
   if (!kv->v_block_mean || !kv->v) return FOLD_EINVAL;
-  if (int rc = check_kv(*kv, head_dim)) return rc;
+  if (int rc = check_kv(*kv, head_dim, num_kv_heads)) return rc;
   MeanParams p;
   p.v = static_cast<const __nv_bfloat16 *>(kv->v);
   p.v_stride_seq = kv->stride_seq; p.v_stride_tok = kv->stride_tok; p.v_stride_head = kv->stride_head;
@@ -910,7 +914,7 @@ int fold_quantize_keys(const fold_kv *kv, int32_t num_kv_heads, int32_t head_dim
   if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
   if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
   if (!kv->k || !kv->k_plane_a) return FOLD_EINVAL;
-  if (int rc = check_kv(*kv, head_dim)) return rc;
+  if (int rc = check_kv(*kv, head_dim, num_kv_heads)) return rc;
   if (kv->max_seqlen == 0) return FOLD_OK;
   QuantParams p;
   memset(&p, 0, sizeof(p));
@@ -931,7 +935,7 @@ int fold_quantize_values(const fold_kv *kv, int32_t num_kv_heads, int32_t head_d
   if (!kv || num_kv_heads < 1) return FOLD_EINVAL;
   if (head_dim != 64 && head_dim != 128) return FOLD_EUNSUPPORTED;
   if (!kv->v || !kv->v_plane_1) return FOLD_EINVAL;
-  if (int rc = check_kv(*kv, head_dim)) return rc;
+  if (int rc = check_kv(*kv, head_dim, num_kv_heads)) return rc;
   if (kv->max_seqlen == 0) return FOLD_OK;
   QuantValueParams p;
   memset(&p, 0, sizeof(p));
@@ -981,20 +985,20 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
   fold_partials parts[kMaxLevels];
   const fold_partials *pp[kMaxLevels];
   for (int l = 0; l < n_levels; ++l) pp[l] = &parts[l];
-  // Once the reference is fixed the levels are independent: the first level (the shared prefix: a tensor-bound
-  // kernel on fewer CTAs than SMs) is scanned on a side stream of the library's while the others are scanned on the
-  // caller's stream, forked and joined with events, so the caller still sees one ordered call on `stream`.
+  // Once the reference is fixed the levels are independent: with a side stream and two events from the caller the first
+  // level (the shared prefix: a tensor-bound kernel on fewer CTAs than SMs) is scanned there while the others are
+  // scanned on `stream`, forked and joined with the events, so the caller still sees one ordered call on `stream`.
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  CascadeSide *side = n_levels >= 2 ? cascade_side() : nullptr;
-  if (side) {
-    std::lock_guard<std::mutex> lock(side->mu);               // the events are shared by every call on the device
-    if (cudaEventRecord(side->fork, st) != cudaSuccess || cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess)
-      return FOLD_ECUDA;
-    int rc = decode_split_impl(&lv[0], &parts[0], side->stream, est);
-    const bool recorded = cudaEventRecord(side->join, side->stream) == cudaSuccess;
+  if (n_levels >= 2 && a0->side_stream && a0->side_fork_event && a0->side_join_event) {
+    cudaStream_t side = static_cast<cudaStream_t>(a0->side_stream);
+    cudaEvent_t fork = static_cast<cudaEvent_t>(a0->side_fork_event), join = static_cast<cudaEvent_t>(a0->side_join_event);
+    if (side == st) return FOLD_EINVAL;
+    if (cudaEventRecord(fork, st) != cudaSuccess || cudaStreamWaitEvent(side, fork, 0) != cudaSuccess) return FOLD_ECUDA;
+    int rc = decode_split_impl(&lv[0], &parts[0], a0->side_stream, est);
+    const bool recorded = cudaEventRecord(join, side) == cudaSuccess;
     for (int l = 1; l < n_levels && rc == FOLD_OK; ++l) rc = decode_split_impl(&lv[l], &parts[l], stream, est);
     // join in every case, so that the side stream never holds work the caller's stream does not wait for
-    if (!recorded || cudaStreamWaitEvent(st, side->join, 0) != cudaSuccess) return FOLD_ECUDA;
+    if (!recorded || cudaStreamWaitEvent(st, join, 0) != cudaSuccess) return FOLD_ECUDA;
     if (rc) return rc;
     return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
   }
@@ -1097,18 +1101,19 @@ int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, f
 static __device__ __align__(256) unsigned char g_fold_static_scratch[FOLD_STATIC_SCRATCH_BYTES];
 
 namespace {
-void *g_static_scratch_addr[64] = {nullptr};   // device address of the array, per device ordinal
+std::atomic<void *> g_static_scratch_addr[64];   // device address of the array, per device ordinal (first call: looked up, stored)
 
 int static_scratch_address(void **out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return FOLD_ECUDA;
   if (dev < 0 || dev >= 64) return FOLD_EUNSUPPORTED;
-  if (!g_static_scratch_addr[dev]) {           // first call on this device: resolve the symbol here, once
-    void *addr = nullptr;
+  void *addr = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!addr) {                                 // first call on this device: resolve the symbol here (threads racing on
+    //                                            it look up the same address and store the same value)
     if (cudaGetSymbolAddress(&addr, g_fold_static_scratch) != cudaSuccess || !addr) return FOLD_ECUDA;
-    g_static_scratch_addr[dev] = addr;
+    g_static_scratch_addr[dev].store(addr, std::memory_order_release);
   }
-  *out = g_static_scratch_addr[dev];
+  *out = addr;
   return FOLD_OK;
 }
 }  // namespace

@@ -45,6 +45,7 @@ int main(void) {
          offsetof(fold_args, depth_T), offsetof(fold_args, row_status));
   printf("%zu %zu %zu\n", offsetof(fold_partials, rows), offsetof(fold_partials, slot_stride),
          offsetof(fold_ws_header, v_rows_total));
+  printf("%zu %zu %zu\n", offsetof(fold_args, flags), offsetof(fold_args, side_stream), offsetof(fold_args, side_join_event));
   return 0;
 }
 """
@@ -58,7 +59,8 @@ int main(void) {
     want = [C.sizeof(F.FoldKV), C.sizeof(F.FoldArgs), C.sizeof(F.FoldPartials), C.sizeof(F.FoldWsHeader),
             F.FoldKV.seqlens.offset, F.FoldKV.max_seqlen.offset, F.FoldArgs.kv.offset, F.FoldArgs.depth_T.offset,
             F.FoldArgs.row_status.offset, F.FoldPartials.rows.offset, F.FoldPartials.slot_stride.offset,
-            F.FoldWsHeader.v_rows_total.offset]
+            F.FoldWsHeader.v_rows_total.offset, F.FoldArgs.flags.offset, F.FoldArgs.side_stream.offset,
+            F.FoldArgs.side_join_event.offset]
     assert got == want
 
 
@@ -116,6 +118,32 @@ def test_host_checks_answer_before_any_cuda_call():
     a.kv.page_table = None
     a.batch, a.kv.num_seqs = 70000, 70000                         # requests index a grid dimension: at most 65535
     assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED
+
+
+def test_broadcast_strides_are_refused():
+    # an axis with more than one entry must have a stride that spans a row: a zero (broadcast) stride would let the
+    # tensor maps and the plain loads disagree about where the rows lie
+    L = F.lib()
+    a, keep = _cpu_args()
+    ws = torch.zeros(F.fold_workspace_bytes(a) + 256, dtype=torch.uint8)
+    a.workspace = ws.data_ptr() + (-ws.data_ptr()) % 256
+    a.workspace_bytes = ws.numel() - 256
+    for field in ("stride_head", "stride_seq"):
+        old = getattr(a.kv, field)
+        setattr(a.kv, field, 0)
+        assert L.fold_decode(a, None) == F.FOLD_EINVAL, field
+        setattr(a.kv, field, old)
+    a1, keep1 = _cpu_args(B=1, Hq=4, Hkv=1)                  # one sequence, one kv head: their strides carry no information
+    a1.kv.stride_head = 0; a1.kv.stride_seq = 0
+    a1.depth_T = -1.0                                        # (a later check must be the one that answers)
+    assert L.fold_decode(a1, None) == F.FOLD_EINVAL
+
+
+def test_new_argument_fields_default_to_plain_behaviour():
+    a, _ = _cpu_args()
+    assert a.flags == 0 and not a.side_stream and not a.side_fork_event and not a.side_join_event
+    b, _ = _cpu_args(flags=F.INPUTS_SETTLED)
+    assert b.flags == 1
 
 
 def test_host_checks_of_draft_masks_and_block_means():

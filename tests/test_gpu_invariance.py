@@ -174,8 +174,10 @@ def test_graph_replay_equals_eager_call(T):
         assert bufs.header().wait_timeouts == 0
 
 
-def test_cascade_call_is_graph_capturable_with_its_side_stream():
-    # the cascade forks its first level onto a stream of the library's and joins it back: still one capturable call
+@pytest.mark.parametrize("with_side", [False, True])
+def test_cascade_call_is_graph_capturable_with_its_side_stream(with_side):
+    # with a side stream and two events of the CALLER's the cascade forks its first level onto that stream and joins it
+    # back: still one capturable call, and the same bits as on one stream
     B, Hq, Hkv, D = 6, 8, 2, 128
     suffixes = [300, 1, 0, 257, 64, 65]
     g = torch.Generator(device=DEV); g.manual_seed(97)
@@ -185,10 +187,16 @@ def test_cascade_call_is_graph_capturable_with_its_side_stream():
     cp, cs = cache_of(pre), cache_of(suf)
     bp, bs = F.alloc_buffers(q, cp, stack=B), F.alloc_buffers(q, cs)
     common = dict(z=bs.z, depth_T=16.0, out=bs.out, lse=bs.lse, row_status=bs.row_status)
-    levels = [F.make_args(q, cp, stack=B, workspace=bp.workspace, **common), F.make_args(q, cs, workspace=bs.workspace, **common)]
-    F.fold_decode_cascade(levels, torch.cuda.current_stream())           # first call outside capture
+    one = [F.make_args(q, cp, stack=B, workspace=bp.workspace, **common), F.make_args(q, cs, workspace=bs.workspace, **common)]
+    F.fold_decode_cascade(one, torch.cuda.current_stream())
     torch.cuda.synchronize()
     o, l = bs.out.clone(), bs.lse.clone()
+    side = F.CascadeSide(DEV) if with_side else None
+    levels = [F.make_args(q, cp, stack=B, workspace=bp.workspace, side=side, **common), F.make_args(q, cs, workspace=bs.workspace, **common)]
+    bs.out.zero_(); bs.lse.zero_()
+    F.fold_decode_cascade(levels, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    assert same_bits(bs.out, o) and same_bits(bs.lse, l)
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         F.fold_decode_cascade(levels, torch.cuda.current_stream())
@@ -198,6 +206,36 @@ def test_cascade_call_is_graph_capturable_with_its_side_stream():
         torch.cuda.synchronize()
         assert same_bits(bs.out, o) and same_bits(bs.lse, l)
         assert bp.header().wait_timeouts == 0 and bs.header().wait_timeouts == 0
+
+
+@pytest.mark.parametrize("flags", [0, F.INPUTS_SETTLED])
+def test_inputs_written_on_the_stream_just_before_a_call_are_seen(flags):
+    # A decode loop appends the newest token's K / V rows, projects q and bumps seqlens with kernels on the stream right
+    # before the call, with no host synchronisation.  Without FOLD_INPUTS_SETTLED the call's first kernel is launched in
+    # plain stream order and must see all of it.  (With the flag the caller promises the inputs were complete earlier; the
+    # writers here are ordinary kernels that end before the call's first kernel may run, so the bits agree there too.)
+    w = make_decode_workload(3, 8, 2, 128, [5000, 777, 8200], seed=73, device=DEV, capacity=8300)
+    cache = cache_of(w)
+    bufs = F.alloc_buffers(w.q, cache)
+    g = torch.Generator(device=DEV); g.manual_seed(74)
+    new_k = torch.randn(3, 2, 128, generator=g, device=DEV).to(torch.bfloat16) * 3
+    new_v = torch.randn(3, 2, 128, generator=g, device=DEV).to(torch.bfloat16)
+    new_q = torch.randn(w.q.shape, generator=g, device=DEV).to(torch.bfloat16)
+    lens = w.seqlens.clone()
+    idx = torch.arange(3, device=DEV)
+    F.decode(w.q, cache, bufs, depth_T=16.0)                     # a step before: the stream is busy with the library's kernels
+    # the append + projection of the next step, then the call, all enqueued without a host synchronisation
+    w.k[idx, lens.long()] = new_k
+    w.v[idx, lens.long()] = new_v
+    w.q.copy_(new_q)
+    w.seqlens.add_(1)
+    F.decode(w.q, cache, bufs, depth_T=16.0, flags=flags)
+    torch.cuda.synchronize()
+    got = (bufs.out.clone(), bufs.lse.clone(), bufs.z.clone())
+    ref = F.alloc_buffers(w.q, cache)                            # the same state decoded after a full synchronisation
+    F.decode(w.q, cache, ref, depth_T=16.0)
+    torch.cuda.synchronize()
+    assert same_bits(got[0], ref.out) and same_bits(got[1], ref.lse) and same_bits(got[2], ref.z)
 
 
 @pytest.mark.parametrize("planes", [False, True])
