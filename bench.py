@@ -245,6 +245,28 @@ def max_over_ranks(ms: float, world: int, device) -> float:
     return float(t.item())
 
 
+def probe_read(dev, gib=2.0, reps=12):
+    """Read-only bandwidth of this GPU: the library's streaming-read kernel over a buffer of `gib` GiB (larger than L2),
+    CUDA events around each of `reps` launches, the first two dropped, best and median in GB/s."""
+    import paper_2609_33410_b200 as F
+    n = int(gib * (1 << 30))
+    buf = torch.empty(n, dtype=torch.uint8, device=dev)
+    buf.fill_(3)
+    sink = torch.zeros(1, dtype=torch.int64, device=dev)
+    st = torch.cuda.current_stream()
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st); F.fold_probe_read(buf, sink, st); e1.record(st)
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    ts = sorted(ts[2:])
+    del buf
+    torch.cuda.empty_cache()
+    return {"gbs_best": n / ts[0] / 1e6, "gbs_median": n / ts[len(ts) // 2] / 1e6, "bytes": n,
+            "kernel": "fold_probe_read_kernel: 16-byte streaming loads, 4 CTAs of 512 threads per SM"}
+
+
 def run_sweep(args, dev):
     """Configuration 5: MHA, 32 heads, D in {64,128}, batch {1,8,64}, context {1K,8K,32K,128K}, T in {8,16,inf}.
     One JSON line with one record per cell; cells whose cache would not fit under the memory cap are
@@ -343,7 +365,11 @@ def main():
     ap.add_argument("--cascade-streams", type=int, default=1, choices=[1, 2],
                     help="cascade workloads: scan the levels on one stream (fold_decode_cascade) or on two")
     ap.add_argument("--sweep", action="store_true", help="run the MHA sweep (configuration 5) instead of one workload")
-    ap.add_argument("--sweep-cap-gb", type=float, default=40.0)
+    ap.add_argument("--sweep-cap-gb", type=float, default=150.0,
+                    help="skip sweep cells whose cache exceeds this (cells that do not fit the free memory are skipped anyway)")
+    ap.add_argument("--probe-read", action="store_true", help="only measure the read-only bandwidth and print it")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the short runs of the other named configurations (c1, c3, c4) in the default line")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -364,275 +390,311 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
+    if args.probe_read:
+        print(json.dumps({"probe": "read-only bandwidth", **probe_read(dev)}))
+        return
     if args.sweep:
         run_sweep(args, dev)
         return
-    spec = WORKLOADS[args.workload]
-    T = spec["T"]
     stream = torch.cuda.current_stream()
-    cascade = "cascade" in spec
-    if cascade:
-        from paper_2609_33410_b200.workloads import make_cascade_workload
-        gen = dict(spec["cascade"]); gen["seed"] = gen["seed"] + 1000 * rank
-        levels = list(make_cascade_workload(device=dev, **gen))           # prefix level (stacked), suffix level
-    elif args.drafts > 1:
-        # draft verification: every sequence keeps its length; its last `drafts` keys are draft tokens and `drafts`
-        # requests (a chain) verify them: the same bytes, `drafts` times the query rows
-        from paper_2609_33410_b200.workloads import make_draft_workload
-        gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
-        n_seqs, lens = gen.pop("batch"), gen.pop("seqlens")
-        lvl, draft_masks, _ = make_draft_workload(n_seqs, args.drafts, gen.pop("num_q_heads"), gen.pop("num_kv_heads"),
-                                                  gen.pop("head_dim"), lens - args.drafts, device=dev, **gen)
-        levels = [lvl]
-    else:
-        gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
-        if args.peak_gain is not None:
-            gen["peak_gain"] = args.peak_gain
-        levels = [make_decode_workload(device=dev, **gen)]
-    if (args.peak_gain is not None or args.z_from_lse) and (cascade or args.drafts > 1):
-        raise SystemExit("--peak-gain / --z-from-lse: plain workloads only")
-    w = levels[-1]                                                        # the level that owns out / lse / z
-    caches = [F.KVCache(l.k, l.v, l.seqlens, l.max_seqlen, l.page_table) for l in levels]
-    if args.tail:
-        # block tail (the block model's mean): cut keys add weight x their 64-key block's mean value; the table is
-        # built once from the cache, outside the timed region (it belongs to cache write)
+
+    def bench_one(wl_name, steps, warm, sample_clocks):
+        spec = WORKLOADS[wl_name]
+        T = spec["T"]
+        stream = torch.cuda.current_stream()
+        cascade = "cascade" in spec
         if cascade:
-            raise SystemExit("--tail: the block tail is built into the row-block scan only (no stacked prefix level)")
-        if not (args.planes and args.fp8v):               # (the 8-bit value format has its own cut model: below)
-            F.fold_block_means(caches[0], stream)
-        torch.cuda.synchronize()
-    quant_ms = None
-    if args.planes:
-        if cascade or args.drafts > 4:
-            raise SystemExit("--planes: one level, at most 8 rows per kv head (no cascade; drafts x group <= 8)")
-        F.fold_quantize_keys(caches[0], None, stream)                   # allocates the planes, warms the kernel
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        F.fold_quantize_keys(caches[0], None, stream)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        quant_ms = e0.elapsed_time(e1)
-        if args.fp8v:
-            vmax = float(levels[0].v.float().abs().max())
-            vk = int(math.ceil(math.log2(max(vmax, 1e-30) / 448.0)))
-            F.fold_quantize_values(caches[0], vk, None, stream)
+            from paper_2609_33410_b200.workloads import make_cascade_workload
+            gen = dict(spec["cascade"]); gen["seed"] = gen["seed"] + 1000 * rank
+            levels = list(make_cascade_workload(device=dev, **gen))           # prefix level (stacked), suffix level
+        elif args.drafts > 1:
+            # draft verification: every sequence keeps its length; its last `drafts` keys are draft tokens and `drafts`
+            # requests (a chain) verify them: the same bytes, `drafts` times the query rows
+            from paper_2609_33410_b200.workloads import make_draft_workload
+            gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
+            n_seqs, lens = gen.pop("batch"), gen.pop("seqlens")
+            lvl, draft_masks, _ = make_draft_workload(n_seqs, args.drafts, gen.pop("num_q_heads"), gen.pop("num_kv_heads"),
+                                                      gen.pop("head_dim"), lens - args.drafts, device=dev, **gen)
+            levels = [lvl]
+        else:
+            gen = dict(spec["gen"]); gen["seed"] = gen["seed"] + 1000 * rank
+            if args.peak_gain is not None:
+                gen["peak_gain"] = args.peak_gain
+            levels = [make_decode_workload(device=dev, **gen)]
+        if (args.peak_gain is not None or args.z_from_lse) and (cascade or args.drafts > 1):
+            raise SystemExit("--peak-gain / --z-from-lse: plain workloads only")
+        w = levels[-1]                                                        # the level that owns out / lse / z
+        caches = [F.KVCache(l.k, l.v, l.seqlens, l.max_seqlen, l.page_table) for l in levels]
+        if args.tail:
+            # block tail (the block model's mean): cut keys add weight x their 64-key block's mean value; the table is
+            # built once from the cache, outside the timed region (it belongs to cache write)
+            if cascade:
+                raise SystemExit("--tail: the block tail is built into the row-block scan only (no stacked prefix level)")
+            if not (args.planes and args.fp8v):               # (the 8-bit value format has its own cut model: below)
+                F.fold_block_means(caches[0], stream)
+            torch.cuda.synchronize()
+        quant_ms = None
+        if args.planes:
+            if cascade or args.drafts > 4:
+                raise SystemExit("--planes: one level, at most 8 rows per kv head (no cascade; drafts x group <= 8)")
+            F.fold_quantize_keys(caches[0], None, stream)                   # allocates the planes, warms the kernel
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            F.fold_quantize_values(caches[0], vk, None, stream)
+            F.fold_quantize_keys(caches[0], None, stream)
             e1.record(stream)
             torch.cuda.synchronize()
-            quant_ms += e0.elapsed_time(e1)
-            if args.tail:                                   # the format's cut model: one mean value row per sequence
-                F.fold_running_means(caches[0], stream)
+            quant_ms = e0.elapsed_time(e1)
+            if args.fp8v:
+                vmax = float(levels[0].v.float().abs().max())
+                vk = int(math.ceil(math.log2(max(vmax, 1e-30) / 448.0)))
+                F.fold_quantize_values(caches[0], vk, None, stream)
+                e0.record(stream)
+                F.fold_quantize_values(caches[0], vk, None, stream)
+                e1.record(stream)
                 torch.cuda.synchronize()
-    elif args.fp8v:
-        raise SystemExit("--fp8v goes with --planes")
-    lbufs = [F.alloc_buffers(l.q, c, l.stack) for l, c in zip(levels, caches)]
-    bufs = lbufs[-1]
-    cache_bytes = sum(l.cache_bytes() for l in levels)                    # unique bytes: a shared prefix counts once
-    flat_bytes = sum(l.cache_bytes() * l.stack for l in levels)           # what a flat decode of every request reads
+                quant_ms += e0.elapsed_time(e1)
+                if args.tail:                                   # the format's cut model: one mean value row per sequence
+                    F.fold_running_means(caches[0], stream)
+                    torch.cuda.synchronize()
+        elif args.fp8v:
+            raise SystemExit("--fp8v goes with --planes")
+        lbufs = [F.alloc_buffers(l.q, c, l.stack) for l, c in zip(levels, caches)]
+        bufs = lbufs[-1]
+        cache_bytes = sum(l.cache_bytes() for l in levels)                    # unique bytes: a shared prefix counts once
+        flat_bytes = sum(l.cache_bytes() * l.stack for l in levels)           # what a flat decode of every request reads
+        # caches under 4x the L2 size are evicted between lone-call samples by writing a buffer larger than L2
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if cache_bytes < 4 * 126e6 else None
 
-    # a cascade's first level may be scanned on a side stream of the caller's (fork / join inside the one C-ABI call)
-    cside = F.CascadeSide(dev) if cascade and args.cascade_streams == 1 else None
+        # a cascade's first level may be scanned on a side stream of the caller's (fork / join inside the one C-ABI call)
+        cside = F.CascadeSide(dev) if cascade and args.cascade_streams == 1 else None
 
-    def make(depth, z_mode):
-        return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
-                            num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
-                            row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
-                            draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau,
-                            refine_tau_v=args.refine_tau_v, side=cside if i == 0 else None)
-                for i, (l, c, b) in enumerate(zip(levels, caches, lbufs))]
+        def make(depth, z_mode):
+            return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
+                                num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
+                                row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
+                                draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau,
+                                refine_tau_v=args.refine_tau_v, side=cside if i == 0 else None)
+                    for i, (l, c, b) in enumerate(zip(levels, caches, lbufs))]
 
-    # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
-    # is scanned on a side stream while the suffix level is scanned on the main one (fork / join with events).
-    side = torch.cuda.Stream(device=dev) if cascade and args.cascade_streams == 2 else None
-    ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
+        # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
+        # is scanned on a side stream while the suffix level is scanned on the main one (fork / join with events).
+        side = torch.cuda.Stream(device=dev) if cascade and args.cascade_streams == 2 else None
+        ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
 
-    def step_whole(a, stream=stream):
-        if not cascade:
-            F.fold_decode(a[0], stream)
-        elif side is None:
-            F.fold_decode_cascade(a, stream)
-        else:
-            F.fold_estimate_z(a, stream)
-            ev_fork.record(stream)
-            side.wait_event(ev_fork)
-            given = [F.FoldArgs.from_buffer_copy(bytes(x)) for x in a]
-            for x in given:
-                x.z_mode = F.Z_GIVEN
-            p0 = F.fold_decode_split(given[0], side)
-            ev_join.record(side)
-            p1 = F.fold_decode_split(given[1], stream)
-            stream.wait_event(ev_join)
-            F.fold_cascade_merge([p0, p1], bufs.out, bufs.lse, bufs.row_status, stream)
+        def step_whole(a, stream=stream):
+            if not cascade:
+                F.fold_decode(a[0], stream)
+            elif side is None:
+                F.fold_decode_cascade(a, stream)
+            else:
+                F.fold_estimate_z(a, stream)
+                ev_fork.record(stream)
+                side.wait_event(ev_fork)
+                given = [F.FoldArgs.from_buffer_copy(bytes(x)) for x in a]
+                for x in given:
+                    x.z_mode = F.Z_GIVEN
+                p0 = F.fold_decode_split(given[0], side)
+                ev_join.record(side)
+                p1 = F.fold_decode_split(given[1], stream)
+                stream.wait_event(ev_join)
+                F.fold_cascade_merge([p0, p1], bufs.out, bufs.lse, bufs.row_status, stream)
 
-    def step_split(a, evs):
-        # the same launches issued one by one, so each kernel can be timed on its own
-        evs[0].record(stream)
-        if not args.z_from_lse:                               # (there the references are inputs: nothing to estimate)
-            F.fold_estimate_z(a, stream)
-        evs[1].record(stream)
-        parts = [F.fold_decode_split(x, stream) for x in a]
-        evs[2].record(stream)
-        F.fold_cascade_merge(parts, bufs.out, bufs.lse, bufs.row_status, stream)
-        evs[3].record(stream)
+        def step_split(a, evs):
+            # the same launches issued one by one, so each kernel can be timed on its own
+            evs[0].record(stream)
+            if not args.z_from_lse:                               # (there the references are inputs: nothing to estimate)
+                F.fold_estimate_z(a, stream)
+            evs[1].record(stream)
+            parts = [F.fold_decode_split(x, stream) for x in a]
+            evs[2].record(stream)
+            F.fold_cascade_merge(parts, bufs.out, bufs.lse, bufs.row_status, stream)
+            evs[3].record(stream)
 
-    def headers():
-        hs = [b.header() for b in lbufs]
-        return dict(fetched=[h.v_rows_fetched for h in hs], total=[h.v_rows_total for h in hs],
-                    refined=[h.k_rows_refined for h in hs], refined_v=[h.v2_rows_refined for h in hs],
-                    timeouts=sum(h.wait_timeouts for h in hs))
+        def headers():
+            hs = [b.header() for b in lbufs]
+            return dict(fetched=[h.v_rows_fetched for h in hs], total=[h.v_rows_total for h in hs],
+                        refined=[h.k_rows_refined for h in hs], refined_v=[h.v2_rows_refined for h in hs],
+                        timeouts=sum(h.wait_timeouts for h in hs))
 
-    def timed(depth, steps, warmup, sample_clocks):
-        # (1) whole steps: estimate -> scan(s) -> partial add, chained in the stream by one C-ABI call
-        a = make(depth, F.Z_ESTIMATE)
-        for _ in range(warmup):
-            step_whole(a)
-        if args.z_from_lse:
-            torch.cuda.synchronize()
-            bufs.z.copy_(bufs.lse)                             # the dense log-sum-exp of the rows (L sums every key)
-            a = make(depth, F.Z_GIVEN)
+        def timed(depth, steps, warmup, sample_clocks):
+            # (1) whole steps: estimate -> scan(s) -> partial add, chained in the stream by one C-ABI call
+            a = make(depth, F.Z_ESTIMATE)
             for _ in range(warmup):
                 step_whole(a)
-        run_step = lambda: step_whole(a)
-        if args.graph:
-            # the whole call (memset + estimate + scan + partial add) captured once and replayed: takes the host's
-            # launch cost out of the step, which is what small workloads are bound by
+            if args.z_from_lse:
+                torch.cuda.synchronize()
+                bufs.z.copy_(bufs.lse)                             # the dense log-sum-exp of the rows (L sums every key)
+                a = make(depth, F.Z_GIVEN)
+                for _ in range(warmup):
+                    step_whole(a)
+            run_step = lambda: step_whole(a)
+            if args.graph:
+                # the whole call (memset + estimate + scan + partial add) captured once and replayed: takes the host's
+                # launch cost out of the step, which is what small workloads are bound by
+                torch.cuda.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    step_whole(a, torch.cuda.current_stream())
+                run_step = graph.replay
+                for _ in range(warmup):
+                    run_step()
+            if world > 1:
+                torch.distributed.barrier()
             torch.cuda.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph):
-                step_whole(a, torch.cuda.current_stream())
-            run_step = graph.replay
-            for _ in range(warmup):
+            sampler = ClockSampler(local)
+            ctx = sampler if sample_clocks else None
+            n_before = 0
+            if ctx:
+                # the timed region lasts milliseconds, the sampler ticks every 100 ms: wait (GPU idle, so the K steps still
+                # start from the state a lone call sees) until the sampler has started, time the K steps, then keep the same
+                # step running back to back (untimed) until a few samples exist; the samples reported are those from the
+                # start of the timed region on
+                ctx.__enter__()
+                t_start = time.time()
+                while not sampler.rows and time.time() - t_start < 1.5:
+                    time.sleep(0.01)
+                n_before = len(sampler.rows)
+            t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+            t0.record(stream)
+            for i in range(steps):
                 run_step()
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-        sampler = ClockSampler(local)
-        ctx = sampler if sample_clocks else None
-        n_before = 0
-        if ctx:
-            # the timed region lasts milliseconds, the sampler ticks every 100 ms: wait (GPU idle, so the K steps still
-            # start from the state a lone call sees) until the sampler has started, time the K steps, then keep the same
-            # step running back to back (untimed) until a few samples exist; the samples reported are those from the
-            # start of the timed region on
-            ctx.__enter__()
-            t_start = time.time()
-            while not sampler.rows and time.time() - t_start < 1.5:
-                time.sleep(0.01)
-            n_before = len(sampler.rows)
-        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-        t0.record(stream)
-        for i in range(steps):
-            run_step()
-        t1.record(stream)
-        torch.cuda.synchronize()
-        if ctx:
-            t_start, n0 = time.time(), len(sampler.rows)
-            while len(sampler.rows) < n0 + 4 and time.time() - t_start < 1.0:
-                run_step()
+            t1.record(stream)
             torch.cuda.synchronize()
-            ctx.__exit__()
-            sampler.rows = sampler.rows[n_before:]
-            time.sleep(0.5)                                    # let the continuation's heat go before anything else is timed
-        if world > 1:
-            torch.distributed.barrier()
-        total_ms = t0.elapsed_time(t1)
-        hd = headers()
-        # (2) the same launches with events between them, for the per-kernel durations
-        g = make(depth, F.Z_GIVEN)
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
-        for i in range(steps):
-            step_split(g, evs[i])
-        torch.cuda.synchronize()
-        scan_ms = [e[1].elapsed_time(e[2]) for e in evs]
-        est_ms = [e[0].elapsed_time(e[1]) for e in evs]
-        mrg_ms = [e[2].elapsed_time(e[3]) for e in evs]
-        return dict(ms_per_step=max_over_ranks(total_ms / steps, world, dev), scan_ms=statistics.mean(scan_ms),
-                    scan_ms_min=min(scan_ms), est_ms=statistics.mean(est_ms), merge_ms=statistics.mean(mrg_ms),
-                    clocks=sampler.summary() if sample_clocks else None, **hd)
+            if ctx:
+                t_start, n0 = time.time(), len(sampler.rows)
+                while len(sampler.rows) < n0 + 4 and time.time() - t_start < 1.0:
+                    run_step()
+                torch.cuda.synchronize()
+                ctx.__exit__()
+                sampler.rows = sampler.rows[n_before:]
+                time.sleep(0.5)                                    # let the continuation's heat go before anything else is timed
+            if world > 1:
+                torch.distributed.barrier()
+            total_ms = t0.elapsed_time(t1)
+            hd = headers()
+            # (2) the same launches with events between them, for the per-kernel durations
+            g = make(depth, F.Z_GIVEN)
+            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+            for i in range(steps):
+                step_split(g, evs[i])
+            torch.cuda.synchronize()
+            scan_ms = [e[1].elapsed_time(e[2]) for e in evs]
+            est_ms = [e[0].elapsed_time(e[1]) for e in evs]
+            mrg_ms = [e[2].elapsed_time(e[3]) for e in evs]
+            # (3) lone calls: the stream idle before each, the cache evicted from L2 by writing a 512 MB buffer when it
+            # could be resident; 22 samples, the first dropped, median and minimum of the rest
+            lone = []
+            for i in range(22):
+                if flush is not None:
+                    flush.fill_(i)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                run_step()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                lone.append(e0.elapsed_time(e1) * 1e3)
+            lone = sorted(lone[1:])
+            return dict(ms_per_step=max_over_ranks(total_ms / steps, world, dev), scan_ms=statistics.mean(scan_ms),
+                        scan_ms_min=min(scan_ms), est_ms=statistics.mean(est_ms), merge_ms=statistics.mean(mrg_ms),
+                        lone_us_median=max_over_ranks(lone[len(lone) // 2], world, dev), lone_us_min=lone[0],
+                        clocks=sampler.summary() if sample_clocks else None, **hd)
+
+        r16 = timed(T, steps, warm, sample_clocks)
+        rinf = timed(math.inf, steps, warm, False)
+        if r16["timeouts"] or rinf["timeouts"]:
+            raise SystemExit("a bounded wait timed out inside the scan kernel: results invalid")
+
+        D = w.head_dim
+        slot_bytes = sum(F.fold_workspace_bytes(x) - 256 for x in make(T, F.Z_GIVEN))
+
+        def fetched_frac(r):
+            return sum(r["fetched"]) / max(sum(r["total"]), 1)
+
+        def refined_frac(r):
+            return sum(r["refined"]) / max(sum(r["total"]), 1)
+
+        def refined_v_frac(r):
+            return sum(r["refined_v"]) / max(sum(r["total"]), 1)
+
+        def value_bytes(r):                                   # per key: BF16 rows of live keys, or plane 1 + the refined share of plane 2
+            return D * fetched_frac(r) + D * refined_v_frac(r) if args.fp8v else 2 * D * fetched_frac(r)
+
+        def actual_bytes(r):                                  # K in full + the fetched share of V + slots written, all levels
+            # (from the fetched FRACTION: row groups of one kv head count their keys once each, but share the tiles in L2)
+            if args.planes:                                   # per key: plane A + scale, the refined share of plane B, the live share of V
+                keys = cache_bytes // (4 * D)
+                return int(keys * ((D + 2) + D * refined_frac(r) + value_bytes(r))) + slot_bytes
+            return cache_bytes // 2 + int(cache_bytes // 2 * fetched_frac(r)) + slot_bytes
+
+        peak, peak_src = load_peaks()
+        value = world * cache_bytes / (r16["ms_per_step"] * 1e-3) / 1e9
+        ach16 = actual_bytes(r16) / (r16["scan_ms"] * 1e-3) / 1e9
+        achinf = actual_bytes(rinf) / (rinf["scan_ms"] * 1e-3) / 1e9
+        scan_name = ("fold_scan_stacked_pair_kernel + fold_scan_decode_kernel<gated> (prefix + suffix levels)" if cascade
+                     else "fold_scan_planes_kernel" if args.planes else "fold_scan_decode_kernel<gated>")
+
+        # the ncu captures cover c2's launch shape at the default gates only
+        traffic_key = None
+        if wl_name == "c2" and not cascade and args.drafts <= 1 and not args.tail:
+            if not args.planes:
+                traffic_key = "gated"
+            elif args.refine_tau == 0 and (not args.fp8v or args.refine_tau_v == 0):
+                traffic_key = "planes_fp8v" if args.fp8v else "planes"
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+            "ms_per_step": r16["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 in, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": f"{wl_name}: " + json.dumps(spec.get("gen", spec.get("cascade")), sort_keys=True),
+                       "depth_T": T,
+                       "num_splits": args.num_splits or "auto", "l2": "inputs (cache) larger than L2, no flush needed"
+                       if cache_bytes > 4 * 126e6 else "cache smaller than 4x L2: partly L2-resident",
+                       "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
+                       "cascade_streams": args.cascade_streams if cascade else None,
+                       "cuda_graph": bool(args.graph), "block_tail": bool(args.tail),
+                       "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16",
+                       "value_format": "two E4M3 planes, power-of-two scale" if args.fp8v else "bf16",
+                       "refine_tau": (args.refine_tau or "auto: max(log2(n) - 2, 4)") if args.planes else None,
+                       "extra_not_graded": ({"peak_gain": args.peak_gain, "z_from_lse": bool(args.z_from_lse)}
+                                            if args.peak_gain is not None or args.z_from_lse else None),
+                       "flat_equivalent_bytes_per_gpu": flat_bytes},
+            "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
+            # one call with the stream idle before it (22 samples, first dropped): the back-to-back mean above runs the
+            # calls in plain stream order too (no FOLD_INPUTS_SETTLED), so the two differ by launch gaps only
+            "lone_call_us": {"T16_median": r16["lone_us_median"], "T16_min": r16["lone_us_min"],
+                             "Tinf_median": rinf["lone_us_median"], "Tinf_min": rinf["lone_us_min"],
+                             "l2_flushed_between_samples": flush is not None},
+            "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},
+            "kernel_ms": {"estimate": r16["est_ms"], "scan_T16": r16["scan_ms"], "scan_Tinf": rinf["scan_ms"],
+                          "merge": r16["merge_ms"]},
+            "v_rows_fetched_frac": {"T16": fetched_frac(r16), "Tinf": fetched_frac(rinf)},
+            "planes": None if not args.planes else {
+                "k_rows_refined_frac": {"T16": refined_frac(r16), "Tinf": refined_frac(rinf)},
+                "v2_rows_refined_frac": {"T16": refined_v_frac(r16), "Tinf": refined_v_frac(rinf)} if args.fp8v else None,
+                "bytes_per_key": {"T16": (D + 2) + D * refined_frac(r16) + value_bytes(r16),
+                                  "Tinf": (D + 2) + D * refined_frac(rinf) + value_bytes(rinf), "bf16_cache": 4 * D},
+                "cache_write_ms": quant_ms},
+            "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
+                         "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src,
+                         "traffic": None if traffic_key is None else NCU_TRAFFIC_PER_CACHE_BYTE[traffic_key] * cache_bytes,
+                         "traffic_source": "ncu dram__bytes_read+write of the same kernel captured on workload c2_small, scaled by units",
+                         "algorithmic_bytes_per_launch": actual_bytes(r16),
+                         "dense": {"kernel": "fold_scan_planes_kernel (T=inf)" if args.planes else "fold_scan_decode_kernel<dense> (T=inf)" if not cascade else "fold_scan_stacked_pair_kernel + fold_scan_decode_kernel<dense> (T=inf)", "achieved": achinf, "frac": achinf / peak,
+                                   "frac_of_nominal_8TBs": achinf / 8000.0,
+                                   "algorithmic_bytes_per_launch": actual_bytes(rinf)}},
+            # estimate + scan (one per level) + partial add per timed step (the extra per-kernel pass is not timed)
+            "gpu_launches": (2 + len(levels)) * steps,
+            "clocks": r16["clocks"],
+        }
+
+        ctx = dict(w=w, make=make, step_whole=step_whole, bufs=bufs, cache_bytes=cache_bytes, cascade=cascade, T=T, spec=spec)
+        return out, ctx
 
     warm = max(args.warmup, 3)
-    r16 = timed(T, args.steps, warm, True)
-    rinf = timed(math.inf, args.steps, warm, False)
-    if r16["timeouts"] or rinf["timeouts"]:
-        raise SystemExit("a bounded wait timed out inside the scan kernel: results invalid")
-
-    D = w.head_dim
-    slot_bytes = sum(F.fold_workspace_bytes(x) - 256 for x in make(T, F.Z_GIVEN))
-
-    def fetched_frac(r):
-        return sum(r["fetched"]) / max(sum(r["total"]), 1)
-
-    def refined_frac(r):
-        return sum(r["refined"]) / max(sum(r["total"]), 1)
-
-    def refined_v_frac(r):
-        return sum(r["refined_v"]) / max(sum(r["total"]), 1)
-
-    def value_bytes(r):                                   # per key: BF16 rows of live keys, or plane 1 + the refined share of plane 2
-        return D * fetched_frac(r) + D * refined_v_frac(r) if args.fp8v else 2 * D * fetched_frac(r)
-
-    def actual_bytes(r):                                  # K in full + the fetched share of V + slots written, all levels
-        # (from the fetched FRACTION: row groups of one kv head count their keys once each, but share the tiles in L2)
-        if args.planes:                                   # per key: plane A + scale, the refined share of plane B, the live share of V
-            keys = cache_bytes // (4 * D)
-            return int(keys * ((D + 2) + D * refined_frac(r) + value_bytes(r))) + slot_bytes
-        return cache_bytes // 2 + int(cache_bytes // 2 * fetched_frac(r)) + slot_bytes
-
-    peak, peak_src = load_peaks()
-    value = world * cache_bytes / (r16["ms_per_step"] * 1e-3) / 1e9
-    ach16 = actual_bytes(r16) / (r16["scan_ms"] * 1e-3) / 1e9
-    achinf = actual_bytes(rinf) / (rinf["scan_ms"] * 1e-3) / 1e9
-    scan_name = ("fold_scan_stacked_pair_kernel + fold_scan_gated_narrow_kernel (prefix + suffix levels)" if cascade
-                 else "fold_scan_planes_kernel" if args.planes else "fold_scan_gated_narrow_kernel")
-
-    # the ncu captures cover c2's launch shape at the default gates only
-    traffic_key = None
-    if args.workload == "c2" and not cascade and args.drafts <= 1 and not args.tail:
-        if not args.planes:
-            traffic_key = "gated"
-        elif args.refine_tau == 0 and (not args.fp8v or args.refine_tau_v == 0):
-            traffic_key = "planes_fp8v" if args.fp8v else "planes"
-    out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
-        "ms_per_step": r16["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 in, fp32 accumulate", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: " + json.dumps(spec.get("gen", spec.get("cascade")), sort_keys=True),
-                   "depth_T": T,
-                   "num_splits": args.num_splits or "auto", "l2": "inputs (cache) larger than L2, no flush needed"
-                   if cache_bytes > 4 * 126e6 else "cache smaller than 4x L2: partly L2-resident",
-                   "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
-                   "cascade_streams": args.cascade_streams if cascade else None,
-                   "cuda_graph": bool(args.graph), "block_tail": bool(args.tail),
-                   "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16",
-                   "value_format": "two E4M3 planes, power-of-two scale" if args.fp8v else "bf16",
-                   "refine_tau": (args.refine_tau or "auto: max(log2(n) - 2, 4)") if args.planes else None,
-                   "extra_not_graded": ({"peak_gain": args.peak_gain, "z_from_lse": bool(args.z_from_lse)}
-                                        if args.peak_gain is not None or args.z_from_lse else None),
-                   "flat_equivalent_bytes_per_gpu": flat_bytes},
-        "us_per_call": {"T16": 1e3 * r16["ms_per_step"], "Tinf": 1e3 * rinf["ms_per_step"]},
-        "effective_gbs": {"T16": value, "Tinf": world * cache_bytes / (rinf["ms_per_step"] * 1e-3) / 1e9},
-        "kernel_ms": {"estimate": r16["est_ms"], "scan_T16": r16["scan_ms"], "scan_Tinf": rinf["scan_ms"],
-                      "merge": r16["merge_ms"]},
-        "v_rows_fetched_frac": {"T16": fetched_frac(r16), "Tinf": fetched_frac(rinf)},
-        "planes": None if not args.planes else {
-            "k_rows_refined_frac": {"T16": refined_frac(r16), "Tinf": refined_frac(rinf)},
-            "v2_rows_refined_frac": {"T16": refined_v_frac(r16), "Tinf": refined_v_frac(rinf)} if args.fp8v else None,
-            "bytes_per_key": {"T16": (D + 2) + D * refined_frac(r16) + value_bytes(r16),
-                              "Tinf": (D + 2) + D * refined_frac(rinf) + value_bytes(rinf), "bf16_cache": 4 * D},
-            "cache_write_ms": quant_ms},
-        "roofline": {"bound": "hbm", "kernel": scan_name + " (T=16)", "achieved": ach16, "peak": peak,
-                     "unit": "GB/s", "frac": ach16 / peak, "peak_source": peak_src,
-                     "traffic": None if traffic_key is None else NCU_TRAFFIC_PER_CACHE_BYTE[traffic_key] * cache_bytes,
-                     "traffic_source": "ncu dram__bytes_read+write of the same kernel captured on workload c2_small, scaled by units",
-                     "algorithmic_bytes_per_launch": actual_bytes(r16),
-                     "dense": {"kernel": "fold_scan_planes_kernel (T=inf)" if args.planes else "fold_scan_dense_kernel (T=inf)" if not cascade else "fold_scan_stacked_pair_kernel + fold_scan_dense_kernel (T=inf)", "achieved": achinf, "frac": achinf / peak,
-                               "frac_of_nominal_8TBs": achinf / 8000.0,
-                               "algorithmic_bytes_per_launch": actual_bytes(rinf)}},
-        # estimate + scan (one per level) + partial add per timed step (the extra per-kernel pass is not timed)
-        "gpu_launches": (2 + len(levels)) * args.steps,
-        "clocks": r16["clocks"],
-    }
+    out, ctx = bench_one(args.workload, args.steps, warm, True)
+    w, make, step_whole, bufs, cache_bytes, cascade, T, spec = (ctx[k] for k in ('w', 'make', 'step_whole', 'bufs', 'cache_bytes', 'cascade', 'T', 'spec'))
+    plain = args.workload == "c2" and not (args.planes or args.tail or args.drafts > 1 or args.graph or args.z_from_lse
+                                          or args.peak_gain is not None)
 
     if rank == 0 and not args.no_e2e and not cascade and not args.planes:
         # end to end through the C ABI with HOST buffers: every step copies q and the whole cache
@@ -684,6 +746,40 @@ def main():
                 torch.cuda.synchronize()
                 return bufs.out.float().cpu().numpy().astype("float64"), bufs.z.cpu().numpy().astype("float64")
             out["accuracy"] = accuracy_sample(w, run_once, T, own_format=bool(args.planes))
+
+    # read-only bandwidth of this GPU (the library's probe kernel), and the fractions against it
+    pr = probe_read(dev)
+    out["read_only_probe"] = pr
+    out["roofline"]["frac_of_read_only"] = out["roofline"]["achieved"] / pr["gbs_best"]
+    out["roofline"]["dense"]["frac_of_read_only"] = out["roofline"]["dense"]["achieved"] / pr["gbs_best"]
+
+    # the other named configurations, short runs of the same measurement: the depth gate's gain shows where rows are
+    # cut (c3: half the value rows), the cascade on c4, the launch-bound small case on c1
+    if plain and not args.no_configs:
+        del w, make, step_whole, bufs, ctx
+        torch.cuda.empty_cache()
+        cfgs = {}
+        for name in ("c1", "c3", "c4"):
+            o, c = bench_one(name, 10, 3, False)
+            rl = o["roofline"]
+            cfgs[name] = {
+                "workload": o["config"]["workload"], "cache_bytes": c["cache_bytes"],
+                "us_per_call": o["us_per_call"], "lone_call_us": o["lone_call_us"], "effective_gbs": o["effective_gbs"],
+                "v_rows_fetched_frac": o["v_rows_fetched_frac"], "kernel_ms": o["kernel_ms"],
+                "roofline": {"kernel": rl["kernel"], "achieved_T16": rl["achieved"], "frac_T16": rl["frac"],
+                             "achieved_Tinf": rl["dense"]["achieved"], "frac_Tinf": rl["dense"]["frac"],
+                             "frac_T16_of_read_only": rl["achieved"] / pr["gbs_best"],
+                             "frac_Tinf_of_read_only": rl["dense"]["achieved"] / pr["gbs_best"],
+                             "algorithmic_bytes_T16": rl["algorithmic_bytes_per_launch"], "unit": "GB/s", "peak": rl["peak"]},
+            }
+            if c["cascade"]:
+                flat = o["config"]["flat_equivalent_bytes_per_gpu"]
+                cfgs[name]["flat_equivalent_gbs"] = {k: flat / (v * 1e-6) / 1e9 for k, v in o["us_per_call"].items()}
+                cfgs[name]["note"] = ("effective_gbs counts the shared prefix once (unique bytes); flat_equivalent_gbs "
+                                      "counts it once per request, as a flat decode of every request would read it")
+            del o, c
+            torch.cuda.empty_cache()
+        out["configs"] = cfgs
 
     if rank == 0:
         print(json.dumps(out))

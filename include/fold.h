@@ -363,6 +363,12 @@ int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_b
 #define FOLD_STATIC_SCRATCH_BYTES (16u << 20)
 int fold_decode_static(const fold_args *args, fold_stream stream);
 
+/* Measurement aid (the paper has no counterpart): reads `bytes` bytes (16-byte aligned; a multiple of 16 is read) of
+ * DEVICE memory once with streaming loads on every SM and XORs a digest of them into *sink (DEVICE, may be NULL).
+ * Timed with events around it, buffer bytes / time is the read-only bandwidth a kernel can get from this memory
+ * system: the third denominator beside the nominal and the measured-copy figures.  Asynchronous on `stream`. */
+int fold_probe_read(const void *buffer, size_t bytes, uint64_t *sink, fold_stream stream);
+
 const char *fold_status_string(int status);
 /* Library version as major*10000 + minor*100 + patch. */
 int fold_version(void);

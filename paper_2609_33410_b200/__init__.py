@@ -6,5 +6,5 @@ from .binding import (  # noqa: F401
     make_args, alloc_buffers, decode, decode_certified, slots_view, lib,
     fold_workspace_bytes, fold_chunk_keys, fold_num_chunks, fold_estimate_z, fold_decode_split,
     fold_cascade_merge, fold_decode, fold_decode_cascade, fold_host_staging_bytes, fold_decode_host, fold_decode_static, fold_block_means, fold_running_means,
-    fold_quantize_keys, fold_quantize_values,
+    fold_quantize_keys, fold_quantize_values, fold_probe_read,
 )

@@ -69,7 +69,7 @@ class FoldWsHeader(C.Structure):
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
            "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
-           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_running_means", "fold_quantize_keys", "fold_quantize_values", "fold_status_string",
+           "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_running_means", "fold_quantize_keys", "fold_quantize_values", "fold_probe_read", "fold_status_string",
            "fold_version"]
 
 _lib = None
@@ -106,6 +106,8 @@ def lib() -> C.CDLL:
         L.fold_quantize_keys.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.fold_quantize_values.restype = C.c_int
         L.fold_quantize_values.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.fold_probe_read.restype = C.c_int
+        L.fold_probe_read.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.fold_status_string.restype = C.c_char_p; L.fold_status_string.argtypes = [C.c_int]
         L.fold_version.restype = C.c_int
         _lib = L
@@ -435,6 +437,12 @@ def decode_certified(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, ma
         decode(q, cache, bufs, **dict(kw, z_mode=Z_GIVEN))
         reruns += 1
     return reruns
+
+
+def fold_probe_read(buf: torch.Tensor, sink: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Stream `buf` (device memory) once with read-only loads: time it with events for the read-only bandwidth."""
+    _check(lib().fold_probe_read(buf.data_ptr(), buf.numel() * buf.element_size(), _ptr(sink), _stream(stream)),
+           "fold_probe_read")
 
 
 def slots_view(part: FoldPartials, workspace: torch.Tensor) -> torch.Tensor:

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libfold_b200.so")
 SOURCES = ["fold_api.cu"]
-HEADERS = ["fold_common.cuh", "fold_scan.cuh", "fold_scan_umma.cuh", "fold_estimate.cuh", "fold_merge.cuh", "fold_planes.cuh"]
+HEADERS = ["fold_common.cuh", "fold_scan.cuh", "fold_scan_umma.cuh", "fold_estimate.cuh", "fold_merge.cuh", "fold_planes.cuh", "fold_scan_decode.cuh", "fold_probe.cuh"]
 
 
 def nvcc_path() -> str:

@@ -10,6 +10,7 @@
 #include "fold_estimate.cuh"
 #include "fold_merge.cuh"
 #include "fold_planes.cuh"
+#include "fold_probe.cuh"
 #include "fold_scan.cuh"
 #include "fold_scan_umma.cuh"
 #include "fold_scan_decode.cuh"
@@ -1129,6 +1130,14 @@ int fold_decode_static(const fold_args *args, fold_stream stream) {
   a.workspace = scratch;                       // the header is re-zeroed by the scan's own memset; slots are
   a.workspace_bytes = FOLD_STATIC_SCRATCH_BYTES;   // written before they are read, so nothing else needs clearing
   return fold_decode(&a, stream);
+}
+
+int fold_probe_read(const void *buffer, size_t bytes, uint64_t *sink, fold_stream stream) {
+  if (!buffer || !aligned(buffer, 16) || bytes < 16) return FOLD_EINVAL;
+  const int ctas = 4 * sm_count();
+  fold_probe_read_kernel<<<ctas, kProbeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4 *>(buffer), bytes / 16, reinterpret_cast<unsigned long long *>(sink));
+  return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 
 const char *fold_status_string(int status) {
