@@ -45,10 +45,10 @@ WORKLOADS = {
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one scan launch from the ncu captures
 # of the c2_small workload (`--workload c2_small`), per byte of cache the launch covers: the c2_small
-# capture (268.4 MB of K+V) moved 272.2 MB (gated, T=16) and 271.8 MB (dense).  Traffic grows in
-# proportion to the (sequence, kv head, key) units, so a launch is scaled by its cache bytes.
+# capture (268.4 MB of K+V) moved 272.8 MB (tcgen05 row-block scan, gated, T=16; the dense variant streams the
+# same tiles).  Traffic grows in proportion to the (sequence, kv head, key) units, so a launch is scaled by its cache bytes.
 # The two-plane scan at its automatic gates moved 218.4 MB (BF16 values) and 219.3 MB (E4M3 value planes) on c2_small.
-NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 272.2 / 268.4, "dense": 271.8 / 268.4, "planes": 218.4 / 268.4, "planes_fp8v": 219.3 / 268.4}
+NCU_TRAFFIC_PER_CACHE_BYTE = {"gated": 272.8 / 268.4, "dense": 272.8 / 268.4, "planes": 218.4 / 268.4, "planes_fp8v": 219.3 / 268.4}
 
 
 def load_peaks():
