@@ -217,6 +217,34 @@ def test_cache_writer_and_query_split_match_the_oracle_bit_for_bit(D, paged):
     assert np.array_equal(eta, (re * scale_log2_f32(w)).astype(np.float32))
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_device_key_codes_against_the_hadamard_matrix_in_float64(D):
+    # The bit-for-bit test above compares two copies of one FP32 procedure.  This one compares the codes the DEVICE
+    # wrote with the DEFINITION, independently of any operation order: H the orthonormal Hadamard matrix (Sylvester's
+    # construction, built here by Kronecker products), y = H k in float64, and the format's claim
+    # |e (a + b / 256) - y| <= one plane-B step e / 256 (half a step of rounding, the +128 clamp, FP32 rotation error),
+    # with plane A never saturated and e the smallest BF16 >= max|y| / 127 up to the FP32 rotation error.
+    w = make_decode_workload(2, 4, 2, D, [900, 257], seed=43, device=DEV)
+    cache = plane_cache(w)
+    H = np.array([[1.0]])
+    while H.shape[0] < D:
+        H = np.kron(H, np.array([[1.0, 1.0], [1.0, -1.0]]))
+    H /= math.sqrt(D)
+    assert np.allclose(H @ H.T, np.eye(D), atol=1e-12)
+    for seq in range(2):
+        for kvh in range(2):
+            a, b, e = logical_planes(w, cache, seq, kvh)
+            K = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh)))
+            Y = K @ H.T                                        # float64, matrix definition
+            e64 = e.astype(np.float64)[:, None]
+            rec = e64 * (a.astype(np.float64) + b.astype(np.float64) / 256.0)
+            ymax = np.abs(Y).max(axis=1, keepdims=True)
+            assert np.all(np.abs(rec - Y) <= e64 / 256.0 + 4e-6 * ymax)
+            assert np.abs(a.astype(np.int32)).max() <= 127
+            # the scale: at least max|y| / 127 (no saturation), and no more than one BF16 step above it
+            assert np.all(e64 >= ymax / 127.0 * (1 - 1e-5)) and np.all(e64 <= ymax / 127.0 * (1 + 2.0 ** -7) + 1e-30)
+
+
 def test_appending_tokens_quantizes_only_the_new_rows():
     w = make_decode_workload(2, 4, 2, 128, [500, 200], seed=43, device=DEV, capacity=640)
     cache = plane_cache(w)
