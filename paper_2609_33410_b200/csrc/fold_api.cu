@@ -455,20 +455,20 @@ int sm_count() {
     return 148;
   return n;
 }
-template <bool GATED, int NC>
+template <bool GATED, int NC, bool TAIL>
 int launch_decode_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, int ctas, cudaStream_t st) {
   static SmemFlags configured;
-  if (int rc = opt_in_smem(fold_scan_decode_kernel<GATED, NC>, configured)) return rc;
-  if (launch_pdl(fold_scan_decode_kernel<GATED, NC>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p) != cudaSuccess)
+  if (int rc = opt_in_smem(fold_scan_decode_kernel<GATED, NC, TAIL>, configured)) return rc;
+  if (launch_pdl(fold_scan_decode_kernel<GATED, NC, TAIL>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p) != cudaSuccess)
     return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
-template <bool GATED>
+template <bool GATED, bool TAIL>
 int launch_decode(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, int ctas, cudaStream_t st) {
-  if (p.R == 1) return launch_decode_as<GATED, 1>(mk, mv, p, ctas, st);
-  if (p.R <= 4) return launch_decode_as<GATED, 4>(mk, mv, p, ctas, st);
-  if (p.R <= 8) return launch_decode_as<GATED, 8>(mk, mv, p, ctas, st);
-  return FOLD_EUNSUPPORTED;                                  // (the kernel takes 16 rows with NC = 16; the host keeps those on mma.sync)
+  if (p.R == 1) return launch_decode_as<GATED, 1, TAIL>(mk, mv, p, ctas, st);
+  if (p.R <= 4) return launch_decode_as<GATED, 4, TAIL>(mk, mv, p, ctas, st);
+  if (p.R <= 8) return launch_decode_as<GATED, 8, TAIL>(mk, mv, p, ctas, st);
+  return FOLD_EUNSUPPORTED;                                  // more rows stay on the mma.sync kernels
 }
 
 // Narrow row blocks (rows on N): unpadded value slices; three K stages (measured: a fourth buys nothing and costs L1).
@@ -616,10 +616,10 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
   // (row blocks of 9..16 rows run the same kernels with two N tiles per warp)
   const bool narrow_tiles = g.R <= row_block_rows();
   const bool gated = !isinf(a->depth_T);
-  // head_dim 128, up to 16 rows: the tcgen05 row-block kernel (keys on M, 128-key tiles); it has no block tail yet
-  // Which kernel runs may depend on the head dimension, the rows per (sequence, kv head), the depth being finite and
-  // the block tail only -- never on the batch or on lengths: a slot's bits must not depend on what else is decoded.
-  const bool decode_umma = g.D == 128 && g.R <= kDecMaxRows && !(gated && kv.v_block_mean);
+  // head_dim 128, up to 8 rows: the tcgen05 row-block kernel (keys on M, 128-key tiles)
+  // Which kernel runs may depend on the head dimension, the rows per (sequence, kv head) and the depth being finite
+  // only -- never on the batch or on lengths: a slot's bits must not depend on what else is decoded.
+  const bool decode_umma = g.D == 128 && g.R <= kDecMaxRows;
   const int tile_keys = decode_umma ? kDecKeys : (narrow_tiles && g.D == 64) ? narrow_tile_keys<64>() : kTileKeys;
   const int box_tok = paged ? (kv.page_size < tile_keys ? kv.page_size : tile_keys) : tile_keys;
   CUtensorMap mk, mv;
@@ -668,7 +668,8 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
     p.box_min = vbox * 13 / 16;                              // fetch a group whole from this many live rows on
     p.num_splits = 1;
     p.stages = 8;                                            // tiles the L2 requests run ahead of the ring
-    return gated ? launch_decode<true>(mk, mv, p, (int)ctas, st) : launch_decode<false>(mk, mv, p, (int)ctas, st);
+    if (!gated) return launch_decode<false, false>(mk, mv, p, (int)ctas, st);
+    return p.vmean ? launch_decode<true, true>(mk, mv, p, (int)ctas, st) : launch_decode<true, false>(mk, mv, p, (int)ctas, st);
   }
   p.num_splits = choose_splits(a, g, tile_keys);
 

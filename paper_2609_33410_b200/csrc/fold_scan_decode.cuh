@@ -45,8 +45,10 @@ struct DecLayout {                                   // byte offsets from a 1 KB
   static constexpr int kK = 0;
   static constexpr int kV = kK + kDecKS * kTile;
   static constexpr int kP = kV + kDecVS * kTile;     // weights, 8 KB per worker: two 4 KB buffers (up to 8 rows) or one of 8 KB
-  static constexpr int kQ = kP + 4 * 4096;           // [worker][parity]: [2 halves][16 rows][128 B] = 4 KB each
-  static constexpr int kLpart = kQ + 4 * 4096;       // [worker][chunk parity][4 warps][16] floats
+  static constexpr int kQ = kP + 4 * 4096;           // query rows [worker][parity]: [2 halves][8 rows][128 B] = 2 KB each
+  static constexpr int kQZero = kQ + 4 * 2048;       // [2 halves][8 rows][128 B] of zeros: rows 8..15 of every query operand
+  static constexpr int kCut = kQZero + 2048;         // block tail: cut mass [worker][chunk parity][8 tiles][4 warps][8 rows] floats
+  static constexpr int kLpart = kCut + 4096;         // [worker][chunk parity][4 warps][16] floats (kQ .. kLpart is 16 KB)
   static constexpr int kBar = kLpart + 1024;
   static constexpr int kTotal = kBar + 512 + 1024;   // + alignment slack
 };
@@ -185,16 +187,22 @@ __device__ __forceinline__ void dec_pair_next(DecPairWalk &x, const ScanParams &
   ++x.it;
 }
 
-// NC: score columns a weight thread reads (query rows, rounded up).  Up to 8 rows the two weight terms share one
-// N = 16 operand (P_hi in rows 0..7, P_lo in rows 8..15: the value tile is read once per tile, not twice) and the
-// weights are double-buffered; 9..16 rows take N = 32 and one buffer.
-template <bool GATED, int NC>
+// NC: score columns a weight thread reads (query rows, rounded up; at most 8).  The two weight terms share one N = 16
+// operand (P_hi in rows 0..7, P_lo in rows 8..15: the value tile is read once per tile, not twice), double-buffered.
+// The score product's B operand needs 16 rows too: rows 8..15 of every query buffer are one shared group of zeros
+// (the descriptor's stride between 8-row groups points there).
+// TAIL (with GATED; Section 4 "Depth as a dial", the block model's mean): a row's cut keys add their summed weight times
+// the mean value row of their 64-key block.  Each weight warp sums its 32 keys' cut weights per row and tile (a tile
+// is two blocks, a block two warps); at the chunk's end every thread -- one channel -- adds cut mass x mean for the
+// chunk's blocks in block order, in FP32.
+template <bool GATED, int NC, bool TAIL = false>
 __global__ void __launch_bounds__(kDecThreads, 1)
 fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                         const ScanParams p) {
   constexpr int D = 128;
-  constexpr int NPV = NC <= 8 ? 16 : 32;                     // N of the value product; P_lo sits NPV / 2 rows after P_hi
-  constexpr int PB = NC <= 8 ? 2 : 1;                        // weight buffers per worker
+  static_assert(NC <= 8 && (!TAIL || GATED), "up to 8 rows; the tail belongs to finite depth");
+  constexpr int NPV = 16;                                    // N of the value product; P_lo sits NPV / 2 rows after P_hi
+  constexpr int PB = 2;                                      // weight buffers per worker
   constexpr int PBYTES = NPV * 256;                          // [2 key halves][NPV rows][128 B]
   // Six 32 KB stages in all.  Depth-gated: three for keys and three for values (four and two streams a cache nobody
   // keeps a value row of 5 % faster, and one with half its rows live 12 % slower).  Dense: a key stage is free as soon
@@ -393,14 +401,18 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           if (ok) {
             tc_fence_after();
             const uint32_t a_lo = umma_desc_lo(base + LO::kK + ks * LO::kTile, 16);
-            const uint32_t b_lo = umma_desc_lo(base + LO::kQ + (2 * set + (eq & 1)) * 4096, 16);
+            // query rows 0..7 of each 64-channel half in the worker's buffer, rows 8..15 in the shared zero group: the
+            // descriptor's stride between 8-row groups is the distance from the one to the other
+            const uint32_t qoff = LO::kQ + (2 * set + (eq & 1)) * 2048;
+            const uint32_t b_lo = umma_desc_lo(base + qoff, 16);
+            const uint32_t b_hi = umma_desc_hi(LO::kQZero - qoff);
             const uint32_t d = tmem + set * 32 + (iq & 1) * 16;
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t ao = ((kk >> 2) * (kDecKeys * 128) + (kk & 3) * 32) >> 4;
-              const uint32_t bo = ((kk >> 2) * 2048 + (kk & 3) * 32) >> 4;
-              if (kk == 0) umma_bf16_ss<false>(d, a_lo + ao, desc_hi, b_lo + bo, desc_hi, idesc_qk);
-              else umma_bf16_ss<true>(d, a_lo + ao, desc_hi, b_lo + bo, desc_hi, idesc_qk);
+              const uint32_t bo = ((kk >> 2) * 1024 + (kk & 3) * 32) >> 4;
+              if (kk == 0) umma_bf16_ss<false>(d, a_lo + ao, desc_hi, b_lo + bo, b_hi, idesc_qk);
+              else umma_bf16_ss<true>(d, a_lo + ao, desc_hi, b_lo + bo, b_hi, idesc_qk);
             }
             tc_commit(bar(kDecBarSFull + 2 * set + (iq & 1)));   // the worker's scores are ready
             tc_commit(bar(kDecBarKEmpty + ks));              // the key stage is free
@@ -422,6 +434,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     const int wtid = (warp - 4 - 4 * set) * 32 + lane;       // 0..127 within the worker
     const int krow = qd * 32 + lane;                         // this thread's key row within a tile
     float *lpart = reinterpret_cast<float *>(gen + LO::kLpart) + set * 128;
+    float *cutp = reinterpret_cast<float *>(gen + LO::kCut) + set * 512;   // [chunk parity][8 tiles][4 warps][8 rows]
     DecWorker cur, nxt;
     dec_worker_init(nxt, p, 2 * blockIdx.x + set, W);
     bool have_next = my_tiles > 0 && dec_worker_next_chunk(nxt, p);
@@ -429,12 +442,12 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     pdl_wait();                                              // z comes from the kernel before
     // Stage the query rows (and fetch the references) of chunk `w`, the worker's e-th, into query buffer e & 1.
     auto stage_rows = [&](const DecWorker &w, int e) {
-      uint8_t *qb = gen + LO::kQ + (2 * set + (e & 1)) * 4096;
+      uint8_t *qb = gen + LO::kQ + (2 * set + (e & 1)) * 2048;
       for (int i = wtid; i < p.R * 16; i += 128) {           // 16-byte chunk i % 16 of row i / 16
         const int r = i >> 4, c16 = i & 15;
         const int req = w.seq * p.stack + r / p.G, head = w.kvh * p.G + r % p.G;
         const uint4 v = *reinterpret_cast<const uint4 *>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + c16 * 8);
-        *reinterpret_cast<uint4 *>(qb + (c16 >> 3) * 2048 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = v;
+        *reinterpret_cast<uint4 *>(qb + (c16 >> 3) * 1024 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = v;
       }
 #pragma unroll
       for (int r = 0; r < NC; ++r) {
@@ -571,6 +584,12 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           L[r] += (h + g) + (pw - pm);                       // L sums the weights the products use; cut keys add p
           hi16[r] = __float_as_uint(h) >> 16;
           lo16[r] = __float_as_uint(g) >> 16;
+          if (TAIL) {                                        // the warp's cut mass of row r in this tile (fixed shuffle order)
+            float c = pw - pm;
+#pragma unroll
+            for (int m = 16; m >= 1; m >>= 1) c += __shfl_xor_sync(0xffffffffu, c, m);
+            if (lane == 0) cutp[(((e & 1) * 8 + (cur.t - cur.t_first)) * 4 + qd) * 8 + r] = c;
+          }
         }
         // the worker's weight buffer is free once its own value product PB tiles back is over
         if (i >= PB && !wait_u(bar(kDecBarPFree + 2 * set + (i % PB)), (uint32_t)((i / PB - 1) & 1))) break;
@@ -607,8 +626,10 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kDecBarLFull + 2 * set + (e & 1)));
-      if (wtid < 32) {                                       // the worker's first warp
+      if (TAIL || wtid < 32) {                               // the worker's first warp (block tail: every warp reads the cut mass)
         if (!wait_u(bar(kDecBarLFull + 2 * set + (e & 1)), (uint32_t)((e >> 1) & 1))) break;
+      }
+      if (wtid < 32) {
         // in the order of the key rows: lane quarters 0, 1, 2, 3
         if (lane < p.R) slot[(long long)p.R * D + lane] = ((lp[lane] + lp[16 + lane]) + lp[32 + lane]) + lp[48 + lane];
       }
@@ -617,9 +638,29 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       float o[NPV];
       tmem_ld_cols<NPV>(lane_addr + 64 + set * 32, o);       // this thread's channel: every row's P_hi part, then the P_lo parts
       tc_fence_before();
+      float tl[NC];
+#pragma unroll
+      for (int r = 0; r < NC; ++r) tl[r] = 0.f;
+      if (TAIL) {
+        // cut mass x block mean, the chunk's blocks in order (a tile is two 64-key blocks, a block two warps' keys)
+        const float *cp = cutp + (e & 1) * 256;
+        const int nblocks = (n + 63) >> 6, ntile = cur.t_end - cur.t_first;
+        const __nv_bfloat16 *mrow = p.vmean + (long long)cur.seq * p.vm_stride_seq + (long long)cur.kvh * p.vm_stride_head + krow;
+        for (int t = 0; t < ntile; ++t) {
+#pragma unroll
+          for (int blk = 0; blk < 2; ++blk) {
+            const int bi = (cur.t_first + t) * 2 + blk;
+            if (bi >= nblocks) break;
+            const float m = __bfloat162float(mrow[(long long)bi * p.vm_stride_block]);
+#pragma unroll
+            for (int r = 0; r < NC; ++r)
+              tl[r] = fmaf(cp[(t * 4 + 2 * blk) * 8 + r] + cp[(t * 4 + 2 * blk + 1) * 8 + r], m, tl[r]);
+          }
+        }
+      }
 #pragma unroll
       for (int r = 0; r < NC; ++r)
-        if (r < p.R) slot[(long long)r * D + krow] = o[r] + o[NPV / 2 + r];
+        if (r < p.R) slot[(long long)r * D + krow] = (o[r] + o[NPV / 2 + r]) + tl[r];
     }
     if (lane == 0) {
       if (dead) atomicOr(&p.hdr->wait_timeouts, 16u);
