@@ -37,7 +37,7 @@ namespace fold {
 constexpr int kDecKeys = 128;                        // keys per tile (MMA M of the score product)
 constexpr int kDecKS = 3, kDecVS = 3;                // key / value ring depths (32 KB stages)
 constexpr int kDecThreads = 12 * 32;                 // key producer, score issuer, value-product issuer, value producer (dense), 2 workers x 4 weight warps
-constexpr int kDecTmemCols = 128;                    // S[worker][2]: 16 columns each from 0;  O[worker]: 32 columns each from 64
+constexpr int kDecTmemCols = 128;                    // S[worker][2]: 16 columns each from 0;  A[worker][chunk parity]: 16 columns each from 64
 constexpr int kDecMaxRows = 8;                       // rows per (sequence, kv head) the host sends here (the kernel itself takes 16)
 
 struct DecLayout {                                   // byte offsets from a 1 KB-aligned base
@@ -110,6 +110,9 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&v)[N]) {
 // (kv head fastest, then chunk, then sequence); entries past a sequence's own chunk count are skipped.
 struct DecWorker {
   int g, step, n_entries;        // next list entry to look at
+  int g_kvh, g_c, g_seq;         // that entry as (kv head, chunk, sequence): kept in step with g, no divisions per chunk
+  int d_kvh, d_c, d_seq;         // the step in the same mixed radix
+  int len_seq, len_n;            // the sequence whose length was read last (entries of a worker mostly stay in one)
   int seq, kvh, c, n;            // the current chunk: sequence, kv head, chunk index, the sequence's length
   int t, t_end;                  // tile cursor: 128-key tiles [t, t_end) of the sequence remain in the chunk
   int t_first;                   // first tile of the chunk
@@ -121,17 +124,24 @@ __device__ __forceinline__ int dec_seqlen(const ScanParams &p, int seq) {
 __device__ __forceinline__ void dec_worker_init(DecWorker &w, const ScanParams &p, int first, int step) {
   w.g = first; w.step = step;
   w.n_entries = p.num_seqs * p.max_slots * p.Hkv;
+  w.g_kvh = first % p.Hkv; w.g_c = (first / p.Hkv) % p.max_slots; w.g_seq = first / p.Hkv / p.max_slots;
+  w.d_kvh = step % p.Hkv; w.d_c = (step / p.Hkv) % p.max_slots; w.d_seq = step / p.Hkv / p.max_slots;
+  w.len_seq = -1; w.len_n = 0;
   w.seq = w.kvh = w.c = w.n = 0;
   w.t = w.t_end = w.t_first = 0;
 }
 // Move to the worker's next non-empty chunk.  False when its list is exhausted.
 __device__ __forceinline__ bool dec_worker_next_chunk(DecWorker &w, const ScanParams &p) {
   while (w.g < w.n_entries) {
-    const int g = w.g;
-    w.g += w.step;
-    const int kvh = g % p.Hkv, rest = g / p.Hkv;
-    const int c = rest % p.max_slots, seq = rest / p.max_slots;
-    const int n = dec_seqlen(p, seq);
+    const int kvh = w.g_kvh, c = w.g_c, seq = w.g_seq;
+    w.g += w.step;                                           // and the same step in (kv head, chunk, sequence), with carries
+    w.g_kvh += w.d_kvh;
+    if (w.g_kvh >= p.Hkv) { w.g_kvh -= p.Hkv; ++w.g_c; }
+    w.g_c += w.d_c;
+    if (w.g_c >= p.max_slots) { w.g_c -= p.max_slots; ++w.g_seq; }
+    w.g_seq += w.d_seq;
+    if (seq != w.len_seq) { w.len_seq = seq; w.len_n = dec_seqlen(p, seq); }
+    const int n = w.len_n;
     if (c < num_chunks_of(n)) {
       const int ctiles = chunk_keys_of(n) / kDecKeys;
       w.seq = seq; w.kvh = kvh; w.c = c; w.n = n;
@@ -369,7 +379,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             // the halves 16 KB apart (leading-dimension offset); weights [2 key halves][NPV rows][128 B], K-major
             const uint32_t a_lo = umma_desc_lo(base + OFF_V + vs * LO::kTile, kDecKeys * 128);
             const uint32_t b_lo = umma_desc_lo(base + LO::kP + set * 8192 + (ip % PB) * PBYTES, 16);
-            const uint32_t d = tmem + 64 + set * 32;
+            const uint32_t d = tmem + 64 + set * 32 + (ep & 1) * 16;   // the accumulators alternate with the chunk's parity
             if (some) {
 #pragma unroll
               for (int j = 0; j < kDecKeys / 16; ++j) {
@@ -440,37 +450,93 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     bool have_next = my_tiles > 0 && dec_worker_next_chunk(nxt, p);
     float z_next[NC];
     pdl_wait();                                              // z comes from the kernel before
-    // Stage the query rows (and fetch the references) of chunk `w`, the worker's e-th, into query buffer e & 1.
-    auto stage_rows = [&](const DecWorker &w, int e) {
-      uint8_t *qb = gen + LO::kQ + (2 * set + (e & 1)) * 2048;
-      for (int i = wtid; i < p.R * 16; i += 128) {           // 16-byte chunk i % 16 of row i / 16
-        const int r = i >> 4, c16 = i & 15;
+    // Staging the query rows (and the references) of chunk `w`, the worker's e-th, into query buffer e & 1, in two
+    // steps so that the global loads are not waited for: stage_load requests them (one 16-byte piece of a row per
+    // thread: at most 8 rows), stage_store puts them into shared memory a tile later.
+    uint4 q_piece = make_uint4(0, 0, 0, 0);
+    auto stage_load = [&](const DecWorker &w) {
+      if (wtid < p.R * 16) {                                 // 16-byte chunk wtid % 16 of row wtid / 16
+        const int r = wtid >> 4, c16 = wtid & 15;
         const int req = w.seq * p.stack + r / p.G, head = w.kvh * p.G + r % p.G;
-        const uint4 v = *reinterpret_cast<const uint4 *>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + c16 * 8);
-        *reinterpret_cast<uint4 *>(qb + (c16 >> 3) * 1024 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = v;
+        q_piece = *reinterpret_cast<const uint4 *>(p.q + (long long)req * p.q_stride_b + (long long)head * p.q_stride_h + c16 * 8);
       }
 #pragma unroll
       for (int r = 0; r < NC; ++r) {
         const int req = w.seq * p.stack + r / p.G, head = w.kvh * p.G + r % p.G;
         z_next[r] = r < p.R ? p.z[(long long)req * p.Hq + head] : INFINITY;   // rows past R: weight 0 by themselves
       }
+    };
+    auto stage_store = [&](int e) {
+      uint8_t *qb = gen + LO::kQ + (2 * set + (e & 1)) * 2048;
+      if (wtid < p.R * 16) {
+        const int r = wtid >> 4, c16 = wtid & 15;
+        *reinterpret_cast<uint4 *>(qb + (c16 >> 3) * 1024 + r * 128 + (((c16 & 7) ^ (r & 7)) << 4)) = q_piece;
+      }
       fence_proxy_async_smem();                              // generic writes, then tensor-core (async proxy) reads
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kDecBarQFull + 2 * set + (e & 1)));
     };
-    if (have_next) stage_rows(nxt, 0);
+    bool stage_open = false;                                 // loads requested, not yet stored
+    if (have_next) { stage_load(nxt); stage_store(0); }
     unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
     const uint64_t vpol = policy_evict_first();
     const int vbox = p.vr;                                   // tokens per value box (16 or 32)
     const uint32_t gmask = vbox == 32 ? 0xffffffffu : 0xffffu;
     int i = 0;                                               // tiles this worker has been through
+    DecWorker pend;                                          // the chunk whose slot is still to be written
+    int pend_e = 0, pend_i = 0;
+    bool pending = false;
+    // Chunk end, second half: the row sums from the four warps, the accumulator out of tensor memory, the block tail,
+    // the slot.  A warp can only reach the chunk after next once every warp has been here (each tile's value product
+    // needs all four warps' weights), so the parity-indexed buffers are free again when they are rewritten.
+    auto flush_chunk = [&]() {
+      pending = false;
+      const int pe = pend_e, par = pe & 1;
+      float *slot = p.slots + (((long long)pend.seq * p.Hkv + pend.kvh) * p.max_slots + pend.c) * p.slot_stride;
+      const float *lp = lpart + par * 64;
+      if (TAIL || wtid < 32) {                               // the worker's first warp (block tail: every warp reads the cut mass)
+        if (!wait_u(bar(kDecBarLFull + 2 * set + par), (uint32_t)((pe >> 1) & 1))) return;
+      }
+      if (wtid < 32) {
+        // in the order of the key rows: lane quarters 0, 1, 2, 3
+        if (lane < p.R) slot[(long long)p.R * D + lane] = ((lp[lane] + lp[16 + lane]) + lp[32 + lane]) + lp[48 + lane];
+      }
+      if (!wait_u(bar(kDecBarPFree + 2 * set + (pend_i % PB)), (uint32_t)((pend_i / PB) & 1))) return;   // the chunk's last product
+      tc_fence_after();
+      float o[NPV];
+      tmem_ld_cols<NPV>(lane_addr + 64 + set * 32 + par * 16, o);   // this thread's channel: every row's P_hi part, then the P_lo parts
+      tc_fence_before();
+      float tl[NC];
+#pragma unroll
+      for (int r = 0; r < NC; ++r) tl[r] = 0.f;
+      if (TAIL) {
+        // cut mass x block mean, the chunk's blocks in order (a tile is two 64-key blocks, a block two warps' keys)
+        const float *cp = cutp + par * 256;
+        const int nblocks = (pend.n + 63) >> 6, ntile = pend.t_end - pend.t_first;
+        const __nv_bfloat16 *mrow = p.vmean + (long long)pend.seq * p.vm_stride_seq + (long long)pend.kvh * p.vm_stride_head + krow;
+        for (int t = 0; t < ntile; ++t) {
+#pragma unroll
+          for (int blk = 0; blk < 2; ++blk) {
+            const int bi = (pend.t_first + t) * 2 + blk;
+            if (bi >= nblocks) break;
+            const float m = __bfloat162float(mrow[(long long)bi * p.vm_stride_block]);
+#pragma unroll
+            for (int r = 0; r < NC; ++r)
+              tl[r] = fmaf(cp[(t * 4 + 2 * blk) * 8 + r] + cp[(t * 4 + 2 * blk + 1) * 8 + r], m, tl[r]);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < NC; ++r)
+        if (r < p.R) slot[(long long)r * D + krow] = (o[r] + o[NPV / 2 + r]) + tl[r];
+    };
     for (int e = 0; have_next && !dead; ++e) {
       cur = nxt;
       float z[NC];
 #pragma unroll
       for (int r = 0; r < NC; ++r) z[r] = z_next[r];
       have_next = dec_worker_next_chunk(nxt, p);
-      if (have_next) stage_rows(nxt, e + 1);                 // one chunk ahead: the score products never wait for rows
+      if (have_next) { stage_load(nxt); stage_open = true; } // one chunk ahead: the score products never wait for rows
       const int n = cur.n, dstart = draft_start(p, n);
       float L[NC];
 #pragma unroll
@@ -610,58 +676,26 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kDecBarPFull + 2 * set + (i % PB)));
+        if (stage_open) { stage_store(e + 1); stage_open = false; }   // the next chunk's rows, requested a tile ago
+        if (pending) flush_chunk();                          // the chunk before: its slot, now that this tile's weights are out
+        if (dead) break;
       }
       if (dead) break;
-      // chunk end: L over the worker's 128 threads in a fixed order, then the accumulator out of tensor memory.
-      // The four warps hand their sums to the worker's first warp through shared memory and an mbarrier (bounded
-      // wait); the buffer alternates with the chunk's parity, and a warp can only reach the chunk after next once the
-      // first warp has finished this one (every tile's weights need all four warps).
-      float *slot = p.slots + (((long long)cur.seq * p.Hkv + cur.kvh) * p.max_slots + cur.c) * p.slot_stride;
-      float *lp = lpart + (e & 1) * 64;
+      // chunk end, first half: L over the warp in a fixed shuffle order, handed to the worker's first warp through shared
+      // memory (the buffer alternates with the chunk's parity).  The rest -- the accumulator out of tensor memory, the
+      // slot -- is put off until the worker has issued the weights of its next tile (flush_chunk): the value product of
+      // the chunk's last tile is then long over, and the next chunk accumulates in the other accumulator meanwhile.
 #pragma unroll
       for (int r = 0; r < NC; ++r) {
 #pragma unroll
         for (int m = 16; m >= 1; m >>= 1) L[r] += __shfl_xor_sync(0xffffffffu, L[r], m);
-        if (lane == 0) lp[qd * 16 + r] = L[r];
+        if (lane == 0) lpart[(e & 1) * 64 + qd * 16 + r] = L[r];
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kDecBarLFull + 2 * set + (e & 1)));
-      if (TAIL || wtid < 32) {                               // the worker's first warp (block tail: every warp reads the cut mass)
-        if (!wait_u(bar(kDecBarLFull + 2 * set + (e & 1)), (uint32_t)((e >> 1) & 1))) break;
-      }
-      if (wtid < 32) {
-        // in the order of the key rows: lane quarters 0, 1, 2, 3
-        if (lane < p.R) slot[(long long)p.R * D + lane] = ((lp[lane] + lp[16 + lane]) + lp[32 + lane]) + lp[48 + lane];
-      }
-      if (!wait_u(bar(kDecBarPFree + 2 * set + ((i - 1) % PB)), (uint32_t)(((i - 1) / PB) & 1))) break;   // the chunk's last product
-      tc_fence_after();
-      float o[NPV];
-      tmem_ld_cols<NPV>(lane_addr + 64 + set * 32, o);       // this thread's channel: every row's P_hi part, then the P_lo parts
-      tc_fence_before();
-      float tl[NC];
-#pragma unroll
-      for (int r = 0; r < NC; ++r) tl[r] = 0.f;
-      if (TAIL) {
-        // cut mass x block mean, the chunk's blocks in order (a tile is two 64-key blocks, a block two warps' keys)
-        const float *cp = cutp + (e & 1) * 256;
-        const int nblocks = (n + 63) >> 6, ntile = cur.t_end - cur.t_first;
-        const __nv_bfloat16 *mrow = p.vmean + (long long)cur.seq * p.vm_stride_seq + (long long)cur.kvh * p.vm_stride_head + krow;
-        for (int t = 0; t < ntile; ++t) {
-#pragma unroll
-          for (int blk = 0; blk < 2; ++blk) {
-            const int bi = (cur.t_first + t) * 2 + blk;
-            if (bi >= nblocks) break;
-            const float m = __bfloat162float(mrow[(long long)bi * p.vm_stride_block]);
-#pragma unroll
-            for (int r = 0; r < NC; ++r)
-              tl[r] = fmaf(cp[(t * 4 + 2 * blk) * 8 + r] + cp[(t * 4 + 2 * blk + 1) * 8 + r], m, tl[r]);
-          }
-        }
-      }
-#pragma unroll
-      for (int r = 0; r < NC; ++r)
-        if (r < p.R) slot[(long long)r * D + krow] = (o[r] + o[NPV / 2 + r]) + tl[r];
+      pend = cur; pend_e = e; pend_i = i - 1; pending = true;
     }
+    if (pending && !dead) flush_chunk();
     if (lane == 0) {
       if (dead) atomicOr(&p.hdr->wait_timeouts, 16u);
       if (st_total) {
