@@ -483,14 +483,12 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     const int vbox = p.vr;                                   // tokens per value box (16 or 32)
     const uint32_t gmask = vbox == 32 ? 0xffffffffu : 0xffffu;
     int i = 0;                                               // tiles this worker has been through
-    DecWorker pend;                                          // the chunk whose slot is still to be written
+    DecWorker pend;                                          // the chunk whose slot is being written
     int pend_e = 0, pend_i = 0;
-    bool pending = false;
     // Chunk end, second half: the row sums from the four warps, the accumulator out of tensor memory, the block tail,
     // the slot.  A warp can only reach the chunk after next once every warp has been here (each tile's value product
     // needs all four warps' weights), so the parity-indexed buffers are free again when they are rewritten.
     auto flush_chunk = [&]() {
-      pending = false;
       const int pe = pend_e, par = pe & 1;
       float *slot = p.slots + (((long long)pend.seq * p.Hkv + pend.kvh) * p.max_slots + pend.c) * p.slot_stride;
       const float *lp = lpart + par * 64;
@@ -501,6 +499,17 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         // in the order of the key rows: lane quarters 0, 1, 2, 3
         if (lane < p.R) slot[(long long)p.R * D + lane] = ((lp[lane] + lp[16 + lane]) + lp[32 + lane]) + lp[48 + lane];
       }
+      // block tail: this channel of the chunk's block means (up to 16 blocks), requested before the waits below
+      float mean[16];
+      if (TAIL) {
+        const int nblocks = (pend.n + 63) >> 6;
+        const __nv_bfloat16 *mrow = p.vmean + (long long)pend.seq * p.vm_stride_seq + (long long)pend.kvh * p.vm_stride_head + krow;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int bi = pend.t_first * 2 + j;
+          mean[j] = (j < 2 * (pend.t_end - pend.t_first) && bi < nblocks) ? __bfloat162float(mrow[(long long)bi * p.vm_stride_block]) : 0.f;
+        }
+      }
       if (!wait_u(bar(kDecBarPFree + 2 * set + (pend_i % PB)), (uint32_t)((pend_i / PB) & 1))) return;   // the chunk's last product
       tc_fence_after();
       float o[NPV];
@@ -510,20 +519,14 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 #pragma unroll
       for (int r = 0; r < NC; ++r) tl[r] = 0.f;
       if (TAIL) {
-        // cut mass x block mean, the chunk's blocks in order (a tile is two 64-key blocks, a block two warps' keys)
+        // cut mass x block mean, the chunk's blocks in order (a tile is two 64-key blocks, a block two warps' keys; tiles
+        // and blocks the chunk does not have carry zero cut mass and a zero mean)
         const float *cp = cutp + par * 256;
-        const int nblocks = (pend.n + 63) >> 6, ntile = pend.t_end - pend.t_first;
-        const __nv_bfloat16 *mrow = p.vmean + (long long)pend.seq * p.vm_stride_seq + (long long)pend.kvh * p.vm_stride_head + krow;
-        for (int t = 0; t < ntile; ++t) {
 #pragma unroll
-          for (int blk = 0; blk < 2; ++blk) {
-            const int bi = (pend.t_first + t) * 2 + blk;
-            if (bi >= nblocks) break;
-            const float m = __bfloat162float(mrow[(long long)bi * p.vm_stride_block]);
+        for (int j = 0; j < 16; ++j) {
 #pragma unroll
-            for (int r = 0; r < NC; ++r)
-              tl[r] = fmaf(cp[(t * 4 + 2 * blk) * 8 + r] + cp[(t * 4 + 2 * blk + 1) * 8 + r], m, tl[r]);
-          }
+          for (int r = 0; r < NC; ++r)
+            tl[r] = fmaf(cp[(j * 2) * 8 + r] + cp[(j * 2 + 1) * 8 + r], mean[j], tl[r]);
         }
       }
 #pragma unroll
@@ -677,14 +680,13 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(kDecBarPFull + 2 * set + (i % PB)));
         if (stage_open) { stage_store(e + 1); stage_open = false; }   // the next chunk's rows, requested a tile ago
-        if (pending) flush_chunk();                          // the chunk before: its slot, now that this tile's weights are out
         if (dead) break;
       }
       if (dead) break;
-      // chunk end, first half: L over the warp in a fixed shuffle order, handed to the worker's first warp through shared
-      // memory (the buffer alternates with the chunk's parity).  The rest -- the accumulator out of tensor memory, the
-      // slot -- is put off until the worker has issued the weights of its next tile (flush_chunk): the value product of
-      // the chunk's last tile is then long over, and the next chunk accumulates in the other accumulator meanwhile.
+      // chunk end: L over the warp in a fixed shuffle order, handed to the worker's first warp through shared memory (the
+      // buffer alternates with the chunk's parity), then the accumulator out of tensor memory and the slot (flush_chunk).
+      // (Putting the second half off behind the next chunk's first tile was measured: no gain on 256-key chunks, 2 % lost
+      // on long ones.)
 #pragma unroll
       for (int r = 0; r < NC; ++r) {
 #pragma unroll
@@ -693,9 +695,9 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(kDecBarLFull + 2 * set + (e & 1)));
-      pend = cur; pend_e = e; pend_i = i - 1; pending = true;
+      pend = cur; pend_e = e; pend_i = i - 1;
+      flush_chunk();
     }
-    if (pending && !dead) flush_chunk();
     if (lane == 0) {
       if (dead) atomicOr(&p.hdr->wait_timeouts, 16u);
       if (st_total) {
