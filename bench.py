@@ -368,6 +368,8 @@ def main():
     ap.add_argument("--sweep-cap-gb", type=float, default=150.0,
                     help="skip sweep cells whose cache exceeds this (cells that do not fit the free memory are skipped anyway)")
     ap.add_argument("--probe-read", action="store_true", help="only measure the read-only bandwidth and print it")
+    ap.add_argument("--launches", default="auto", choices=["auto", "one", "separate"],
+                    help="fold_args.flags: FOLD_ONE_LAUNCH / FOLD_SEPARATE_LAUNCHES (auto: the library's own choice)")
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the short runs of the other named configurations (c1, c3, c4) in the default line")
     args = ap.parse_args()
@@ -473,7 +475,8 @@ def main():
                                 num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
                                 row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
                                 draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau,
-                                refine_tau_v=args.refine_tau_v, side=cside if i == 0 else None)
+                                refine_tau_v=args.refine_tau_v, side=cside if i == 0 else None,
+                                flags={"auto": 0, "one": F.ONE_LAUNCH, "separate": F.SEPARATE_LAUNCHES}[args.launches])
                     for i, (l, c, b) in enumerate(zip(levels, caches, lbufs))]
 
         # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
@@ -683,7 +686,7 @@ def main():
                                    "frac_of_nominal_8TBs": achinf / 8000.0,
                                    "algorithmic_bytes_per_launch": actual_bytes(rinf)}},
             # estimate + scan (one per level) + partial add per timed step (the extra per-kernel pass is not timed)
-            "gpu_launches": (2 + len(levels)) * steps,
+            "gpu_launches": (F.fold_decode_launches(make(T, F.Z_ESTIMATE)[0]) if not cascade else 2 + len(levels)) * steps,
             "clocks": r16["clocks"],
         }
 
@@ -779,6 +782,14 @@ def main():
                                       "counts it once per request, as a flat decode of every request would read it")
             del o, c
             torch.cuda.empty_cache()
+        # the small case once more with reference, scan and partial add inside one cooperative launch (FOLD_ONE_LAUNCH)
+        args.launches = "one"
+        o, c = bench_one("c1", 10, 3, False)
+        cfgs["c1"]["one_launch"] = {"us_per_call": o["us_per_call"], "lone_call_us": o["lone_call_us"],
+                                    "launches_per_call": o["gpu_launches"] // o["steps"]}
+        args.launches = "auto"
+        del o, c
+        torch.cuda.empty_cache()
         out["configs"] = cfgs
 
     if rank == 0:

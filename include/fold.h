@@ -64,12 +64,23 @@ typedef enum fold_zmode {
 
 /* Bits of fold_args.flags. */
 enum {
-  FOLD_INPUTS_SETTLED = 1  /* q, the cache rows, seqlens, page_table and draft_mask were complete before the kernel that
+  FOLD_INPUTS_SETTLED = 1, /* q, the cache rows, seqlens, page_table and draft_mask were complete before the kernel that
                               precedes this call on `stream` STARTED (they were not written by it).  The call's first
                               kernel may then begin, and read them, while that kernel is still draining (programmatic
                               dependent launch); everything it writes still waits.  Without the flag the first kernel is
                               launched in plain stream order, which is what a decode loop that appends to the cache or
                               projects q just before the call needs. */
+  FOLD_SEPARATE_LAUNCHES = 2, /* fold_decode: always run reference, scan and partial add as separate kernels */
+  FOLD_ONE_LAUNCH = 4      /* fold_decode: run them inside ONE cooperative kernel launch wherever the decode is one wave:
+                              head_dim 128, up to 8 rows per (sequence, kv head), stack 1, FOLD_Z_ESTIMATE or
+                              FOLD_Z_GIVEN, no split hint below the chunk count, and at most two canonical chunks per
+                              SM in all (each (sequence, kv head)'s count rounded up to even).  Section 3's three steps
+                              then follow one another on chip; Algorithm 1 is unchanged, and out, lse, z, row_status and
+                              the header are bit for bit those of the separate launches.  With neither flag the library
+                              takes the one launch where it measured faster on a B200 -- FOLD_Z_GIVEN -- and separate
+                              launches for FOLD_Z_ESTIMATE (three short kernels that overlap by programmatic dependent
+                              launch beat one kernel that forms the estimate in every CTA).  Where the one launch does
+                              not apply the flag is ignored. */
 };
 
 /* Bits of row_status[b * num_q_heads + h]. */
@@ -193,7 +204,7 @@ typedef struct fold_args {
                                           INFINITY = every live key; negative = none (plane A scores only) */
   float refine_tau_v;                  /* E4M3 value planes only: the refine-V gate, binades, like refine_tau.
                                           0 = choose: max(log2(n) + 1, 4); INFINITY = every live key; negative = none */
-  int32_t flags;                       /* FOLD_INPUTS_SETTLED or 0 */
+  int32_t flags;                       /* FOLD_INPUTS_SETTLED, FOLD_SEPARATE_LAUNCHES, FOLD_ONE_LAUNCH: ORed, or 0 */
   fold_stream side_stream;             /* fold_decode_cascade, levels[0] only: a second stream of the caller's and two */
   void *side_fork_event;               /* cudaEvent_t of the caller's (created with timing disabled, say) on which the */
   void *side_join_event;               /* first level is scanned; all three NULL: every level on `stream` */
@@ -267,6 +278,11 @@ int fold_cascade_merge(const fold_partials *const *levels, int n_levels, void *o
 /* Whole decode: reference (per z_mode) -> scan -> partial add.  Equivalent to
  * fold_decode_split followed by fold_cascade_merge over its one level. */
 int fold_decode(const fold_args *args, fold_stream stream);
+
+/* How many kernels fold_decode(args) launches: 1 when the decode is one wave and runs in a single launch (see
+ * FOLD_ONE_LAUNCH), else the reference kernel (if the mode has one), the scan and the partial add; 0 for
+ * arguments fold_decode would refuse.  A host-side query: nothing is enqueued.  (No counterpart in the paper.) */
+int32_t fold_decode_launches(const fold_args *args);
 
 /* Shared-prefix cascade in one call (Section 4, "Value product"; Appendix "Cascades and drafts"):
  * one reference estimate over each request's concatenated levels, one scan per level under

@@ -22,6 +22,8 @@ STATIC_SCRATCH_BYTES = 16 << 20
 Z_ESTIMATE, Z_GIVEN, Z_EXACT_MAX, Z_ZERO = range(4)
 ROW_RANGE, ROW_NONFINITE, ROW_EMPTY = 1, 2, 4
 INPUTS_SETTLED = 1                               # fold_args.flags
+SEPARATE_LAUNCHES = 2
+ONE_LAUNCH = 4
 
 
 class FoldKV(C.Structure):
@@ -68,7 +70,7 @@ class FoldWsHeader(C.Structure):
 
 
 EXPORTS = ["fold_chunk_keys", "fold_num_chunks", "fold_workspace_bytes", "fold_estimate_z",
-           "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_cascade", "fold_host_staging_bytes",
+           "fold_decode_split", "fold_cascade_merge", "fold_decode", "fold_decode_launches", "fold_decode_cascade", "fold_host_staging_bytes",
            "fold_decode_host", "fold_decode_static", "fold_block_means", "fold_running_means", "fold_quantize_keys", "fold_quantize_values", "fold_probe_read", "fold_status_string",
            "fold_version"]
 
@@ -98,6 +100,7 @@ def lib() -> C.CDLL:
         L.fold_decode_host.restype = C.c_int
         L.fold_decode_host.argtypes = [C.POINTER(FoldArgs), C.c_void_p, C.c_size_t, C.c_void_p]
         L.fold_decode_static.restype = C.c_int; L.fold_decode_static.argtypes = [C.POINTER(FoldArgs), C.c_void_p]
+        L.fold_decode_launches.restype = C.c_int32; L.fold_decode_launches.argtypes = [C.POINTER(FoldArgs)]
         L.fold_block_means.restype = C.c_int
         L.fold_block_means.argtypes = [C.POINTER(FoldKV), C.c_int32, C.c_int32, C.c_void_p]
         L.fold_running_means.restype = C.c_int
@@ -353,6 +356,10 @@ def fold_quantize_values(cache: KVCache, scale_log2: int, first_token: Optional[
 
 def fold_decode(args: FoldArgs, stream=None) -> None:
     _check(lib().fold_decode(C.byref(args), _stream(stream)), "fold_decode")
+
+
+def fold_decode_launches(args: FoldArgs) -> int:
+    return int(lib().fold_decode_launches(C.byref(args)))
 
 
 def fold_decode_cascade(levels: Sequence[FoldArgs], stream=None) -> None:

@@ -455,19 +455,33 @@ int sm_count() {
     return 148;
   return n;
 }
+// f.mode != 0: the whole decode in this launch, which is then a cooperative one (its CTAs meet at a grid-wide barrier
+// between the scan and the partial add; the grid is one CTA per SM at most, so all of them are resident).
 template <bool GATED, int NC, bool TAIL>
-int launch_decode_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, int ctas, cudaStream_t st) {
+int launch_decode_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, const FusedParams &f, int ctas, cudaStream_t st) {
   static SmemFlags configured;
   if (int rc = opt_in_smem(fold_scan_decode_kernel<GATED, NC, TAIL>, configured)) return rc;
-  if (launch_pdl(fold_scan_decode_kernel<GATED, NC, TAIL>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p) != cudaSuccess)
-    return FOLD_ECUDA;
+  cudaError_t rc;
+  if (f.mode) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(ctas); cfg.blockDim = dim3(kDecThreads); cfg.dynamicSmemBytes = DecLayout::kTotal; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    rc = cudaLaunchKernelEx(&cfg, fold_scan_decode_kernel<GATED, NC, TAIL>, mk, mv, p, f);
+  } else {
+    rc = launch_pdl(fold_scan_decode_kernel<GATED, NC, TAIL>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p, f);
+  }
+  if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
 template <bool GATED, bool TAIL>
-int launch_decode(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, int ctas, cudaStream_t st) {
-  if (p.R == 1) return launch_decode_as<GATED, 1, TAIL>(mk, mv, p, ctas, st);
-  if (p.R <= 4) return launch_decode_as<GATED, 4, TAIL>(mk, mv, p, ctas, st);
-  if (p.R <= 8) return launch_decode_as<GATED, 8, TAIL>(mk, mv, p, ctas, st);
+int launch_decode(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, const FusedParams &f, int ctas, cudaStream_t st) {
+  if (p.R == 1) return launch_decode_as<GATED, 1, TAIL>(mk, mv, p, f, ctas, st);
+  if (p.R <= 4) return launch_decode_as<GATED, 4, TAIL>(mk, mv, p, f, ctas, st);
+  if (p.R <= 8) return launch_decode_as<GATED, 8, TAIL>(mk, mv, p, f, ctas, st);
   return FOLD_EUNSUPPORTED;                                  // more rows stay on the mma.sync kernels
 }
 
@@ -608,7 +622,23 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   return g.D == 128 ? launch_planes_kernel<128>(ma, mv, pp, grid, st) : launch_planes_kernel<64>(ma, mv, pp, grid, st);
 }
 
-int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
+// Does the whole decode fit one launch of the tcgen05 row-block kernel?  Head_dim 128, up to 8 rows per (sequence, kv
+// head), one request per sequence, the reference estimated or given, and one wave: at most one canonical chunk per
+// worker (two workers per CTA, one CTA per SM).  The result's bits are those of the separate launches.
+bool one_launch_decode(const fold_args *a, const Geometry &g) {
+  if (g.planes || g.D != 128 || g.R > kDecMaxRows || g.stack != 1) return false;
+  if (a->flags & FOLD_SEPARATE_LAUNCHES) return false;
+  if (a->z_mode != FOLD_Z_ESTIMATE && a->z_mode != FOLD_Z_GIVEN) return false;
+  // measured on a B200 (8 heads x 4096 keys, calls back to back): given reference 16.5 us in one launch against 18.6 in
+  // two; estimated reference 19.8 against 19.0 in three -- so the estimate keeps its own kernel unless asked
+  if (a->z_mode == FOLD_Z_ESTIMATE && !(a->flags & FOLD_ONE_LAUNCH)) return false;
+  const long long entries = (long long)g.num_seqs * g.Hkv * ((g.max_slots + 1) & ~1);   // chunk-major list, even per unit
+  if (entries > 2LL * sm_count()) return false;
+  if (a->num_splits > 0 && a->num_splits < g.max_slots) return false;   // a split hint that bounds the grid: honour it
+  return true;
+}
+
+int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st, const FusedParams *fused = nullptr) {
   if (g.planes) return launch_scan_planes(a, g, st);
   const fold_kv &kv = a->kv;
   const bool paged = kv.page_table != nullptr;
@@ -668,8 +698,15 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st) {
     p.box_min = vbox * 13 / 16;                              // fetch a group whole from this many live rows on
     p.num_splits = 1;
     p.stages = 8;                                            // tiles the L2 requests run ahead of the ring
-    if (!gated) return launch_decode<false, false>(mk, mv, p, (int)ctas, st);
-    return p.vmean ? launch_decode<true, true>(mk, mv, p, (int)ctas, st) : launch_decode<true, false>(mk, mv, p, (int)ctas, st);
+    FusedParams f;
+    memset(&f, 0, sizeof(f));
+    if (fused) {
+      f = *fused;
+      p.chunk_major = 1;
+      ctas = units * ((g.max_slots + 1) / 2);                // one chunk per worker at most
+    }
+    if (!gated) return launch_decode<false, false>(mk, mv, p, f, (int)ctas, st);
+    return p.vmean ? launch_decode<true, true>(mk, mv, p, f, (int)ctas, st) : launch_decode<true, false>(mk, mv, p, f, (int)ctas, st);
   }
   p.num_splits = choose_splits(a, g, tile_keys);
 
@@ -957,10 +994,40 @@ int fold_quantize_values(const fold_kv *kv, int32_t num_kv_heads, int32_t head_d
 int fold_decode(const fold_args *args, fold_stream stream) {
   Geometry g;
   if (int rc = check_args(args, &g, true)) return rc;
+  if (one_launch_decode(args, g)) {
+    if (!args->workspace || !aligned(args->workspace, 256)) return FOLD_EINVAL;
+    if (args->workspace_bytes < g.ws_bytes) return FOLD_EWORKSPACE;
+    FusedParams f;
+    memset(&f, 0, sizeof(f));
+    f.mode = args->z_mode == FOLD_Z_ESTIMATE ? 1 : 2;
+    f.est = est_params(args, g);
+    f.est.n_levels = 1;
+    f.est.lv[0] = kv_level(args->kv, args->stack);
+    fold_partials part;
+    fill_partials(args, g, &part);
+    MergeLevel &lv = f.mrg.lv[0];
+    lv.slots = part.slots; lv.seqlens = part.seqlens; lv.slot_stride = part.slot_stride;
+    lv.stack = part.stack; lv.max_slots = part.max_slots; lv.rows = part.rows; lv.max_seqlen = part.max_seqlen;
+    f.mrg.z = args->z;
+    f.mrg.out = static_cast<__nv_bfloat16 *>(args->out);
+    f.mrg.lse = args->lse; f.mrg.row_status = args->row_status;
+    f.mrg.n_levels = 1; f.mrg.Hq = g.Hq; f.mrg.Hkv = g.Hkv; f.mrg.G = g.G; f.mrg.D = g.D;
+    return launch_scan(args, g, static_cast<cudaStream_t>(stream), &f);
+  }
   fold_partials part;
   if (int rc = fold_decode_split(args, &part, stream)) return rc;
   const fold_partials *lv[1] = {&part};
   return fold_cascade_merge(lv, 1, args->out, args->lse, args->row_status, stream);
+}
+
+int32_t fold_decode_launches(const fold_args *args) {
+  Geometry g;
+  if (check_args(args, &g, true)) return 0;
+  if (one_launch_decode(args, g)) return 1;
+  int n = 2;                                                 // scan, partial add
+  if (g.planes || args->z_mode != FOLD_Z_GIVEN) ++n;         // reference (or the two-plane front kernel)
+  if (g.planes && args->z_mode == FOLD_Z_ZERO) ++n;
+  return n;
 }
 
 int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_stream stream) {

@@ -113,71 +113,70 @@ __device__ __forceinline__ float est_reduce_row(const float *row, int n, int n_s
   return zval;
 }
 
-// One CTA per (kv head, request), 12 warps.  The 192 x G scores are one small matrix product: warp w
-// takes sampled keys 16w .. 16w+15 on M, the group's query rows on N (mma.sync m16n8k16, BF16 in,
-// FP32 accumulate).  Each lane loads its A fragments straight from the cache rows (all loads issued
-// before the first MMA, so the kernel pays one memory latency); warp g then reduces row g.
+// The 192 x G scores of one (kv head, request) are one small matrix product, formed in blocks of 16 sampled keys: a
+// warp takes block `blk` (samples 16 blk .. 16 blk + 15) on M and the group's query rows on N (mma.sync m16n8k16,
+// BF16 in, FP32 accumulate) and writes the scaled scores to sc[row][sample].  Each lane loads its A fragments
+// straight from the cache rows (all loads issued before the first MMA, so a block pays one memory latency).
+// n = the request's key count over all levels, lens[] per level.  A score's bits do not depend on which warp of
+// which kernel forms it.
 constexpr int kEstWarps = kEstSamples / 16;              // 12
 constexpr int kEstSampleThreads = kEstWarps * 32;        // 384
 
-template <int D>
-__global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const EstParams p) {
+// NB blocks at once (blk0, blk0 + blk_step, ...): all their cache rows are requested before the first product, so
+// the warp pays one memory latency for the lot.
+template <int D, int NB>
+__device__ __forceinline__ void est_score_blocks(const EstParams &p, int req, int kvh, int blk0, int blk_step, int lane,
+                                                 int n, const int (&lens)[kMaxLevels], float (*sc)[kEstSamples]) {
   constexpr int KS = D / 16;
-  __shared__ float sc[kMaxRows][kEstSamples];
-  const int kvh = blockIdx.x, req = blockIdx.y;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.G;
-  pdl_launch_dependents();                           // the scan may set up while the estimate runs
-
-  int lens[kMaxLevels];
-  int n = 0;
-  for (int l = 0; l < p.n_levels; ++l) {
-    lens[l] = level_len(p.lv[l], req);
-    n += lens[l];
-  }
   const int n_samples = n < kEstSamples ? n : kEstSamples;
   const int qcol = (lane & 3) * 2;
   const int qcol4 = (lane & 3) * 8;                          // this lane's 8 consecutive channels of every 32
-
-  if (warp * 16 < n_samples) {
-    // the two sampled key rows this lane reads fragments of
-    const __nv_bfloat16 *rowp[2];
+  // A dot product does not care in which order its terms meet: the k slots of each pair of MMAs are assigned so
+  // that a lane's fragments of 32 channels are 8 CONSECUTIVE channels of its row (one 16-byte load) -- MMA 2j takes
+  // channels 32j + 8t + {0,1 | 2,3} in its slots {2t,2t+1 | 2t+8,2t+9}, MMA 2j+1 takes 32j + 8t + {4,5 | 6,7} -- and
+  // the query fragments below follow the same assignment.
+  uint4 ka[NB][2][KS / 2];                                   // [block][row lane/4, row lane/4 + 8][32-channel group]
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    const int blk = blk0 + b * blk_step;
 #pragma unroll
     for (int hlf = 0; hlf < 2; ++hlf) {
-      const int i = warp * 16 + (lane >> 2) + hlf * 8;
-      rowp[hlf] = nullptr;
-      if (i < n_samples) {
+      // the two sampled key rows this lane reads fragments of
+      const int i = blk * 16 + (lane >> 2) + hlf * 8;
+      const __nv_bfloat16 *rowp = nullptr;
+      if (blk < kEstWarps && i < n_samples) {
         int j = est_sample_key(i, n), l = 0;
         while (l < p.n_levels - 1 && j >= lens[l]) { j -= lens[l]; ++l; }
-        rowp[hlf] = key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + qcol4;
+        rowp = key_row(p.lv[l], req / p.lv[l].stack, j, kvh) + qcol4;
       }
-    }
-    // A dot product does not care in which order its terms meet: the k slots of each pair of MMAs are assigned so
-    // that a lane's fragments of 32 channels are 8 CONSECUTIVE channels of its row (one 16-byte load) -- MMA 2j takes
-    // channels 32j + 8t + {0,1 | 2,3} in its slots {2t,2t+1 | 2t+8,2t+9}, MMA 2j+1 takes 32j + 8t + {4,5 | 6,7} -- and
-    // the query fragments below follow the same assignment.
-    uint32_t a[KS][4];
 #pragma unroll
-    for (int j = 0; j < KS / 2; ++j) {
-      const uint4 r0 = rowp[0] ? *reinterpret_cast<const uint4 *>(rowp[0] + j * 32) : make_uint4(0, 0, 0, 0);
-      const uint4 r1 = rowp[1] ? *reinterpret_cast<const uint4 *>(rowp[1] + j * 32) : make_uint4(0, 0, 0, 0);
-      a[2 * j][0] = r0.x; a[2 * j][1] = r1.x; a[2 * j][2] = r0.y; a[2 * j][3] = r1.y;
-      a[2 * j + 1][0] = r0.z; a[2 * j + 1][1] = r1.z; a[2 * j + 1][2] = r0.w; a[2 * j + 1][3] = r1.w;
+      for (int j = 0; j < KS / 2; ++j)
+        ka[b][hlf][j] = rowp ? *reinterpret_cast<const uint4 *>(rowp + j * 32) : make_uint4(0, 0, 0, 0);
     }
-    // query rows of the group as B fragments (n = lane / 4), eight rows per n-tile
+  }
+  // query rows of the group as B fragments (n = lane / 4), eight rows per n-tile
 #pragma unroll 1
-    for (int nt = 0; nt * 8 < G; ++nt) {
-      const int g = nt * 8 + (lane >> 2);
-      const __nv_bfloat16 *qrow = p.q + (long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + qcol4;
+  for (int nt = 0; nt * 8 < G; ++nt) {
+    const int g = nt * 8 + (lane >> 2);
+    const __nv_bfloat16 *qrow = p.q + (long long)req * p.q_stride_b + (long long)(kvh * G + g) * p.q_stride_h + qcol4;
+    uint4 qb[KS / 2];
+#pragma unroll
+    for (int j = 0; j < KS / 2; ++j) qb[j] = g < G ? *reinterpret_cast<const uint4 *>(qrow + j * 32) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      const int blk = blk0 + b * blk_step;
+      if (blk >= kEstWarps || blk * 16 >= n_samples) continue;
       float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int j = 0; j < KS / 2; ++j) {
-        const uint4 b = g < G ? *reinterpret_cast<const uint4 *>(qrow + j * 32) : make_uint4(0, 0, 0, 0);
-        mma_bf16(c, a[2 * j], b.x, b.y);
-        mma_bf16(c, a[2 * j + 1], b.z, b.w);
+        const uint4 r0 = ka[b][0][j], r1 = ka[b][1][j];
+        const uint32_t a0[4] = {r0.x, r1.x, r0.y, r1.y}, a1[4] = {r0.z, r1.z, r0.w, r1.w};
+        mma_bf16(c, a0, qb[j].x, qb[j].y);
+        mma_bf16(c, a1, qb[j].z, qb[j].w);
       }
       // c0, c1: key lane/4, rows 2*(lane%4) + {0,1};  c2, c3: key lane/4 + 8
-      const int i0 = warp * 16 + (lane >> 2), g0 = nt * 8 + qcol;
+      const int i0 = blk * 16 + (lane >> 2), g0 = nt * 8 + qcol;
       if (p.draft_len) {                                     // a draft key the request does not use weighs nothing
         const uint32_t dm = p.draft_mask[req];
         const int dstart = n - p.draft_len;
@@ -192,6 +191,26 @@ __global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const 
       if (g0 + 1 < G) { sc[g0 + 1][i0] = c[1] * p.scale_log2; sc[g0 + 1][i0 + 8] = c[3] * p.scale_log2; }
     }
   }
+}
+
+// One CTA per (kv head, request), 12 warps, a block of 16 samples each; warp g then reduces row g.
+template <int D>
+__global__ void __launch_bounds__(kEstSampleThreads) fold_estimate_kernel(const EstParams p) {
+  __shared__ float sc[kMaxRows][kEstSamples];
+  const int kvh = blockIdx.x, req = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = p.G;
+  pdl_launch_dependents();                           // the scan may set up while the estimate runs
+
+  int lens[kMaxLevels];
+  int n = 0;
+#pragma unroll
+  for (int l = 0; l < kMaxLevels; ++l) {
+    lens[l] = l < p.n_levels ? level_len(p.lv[l], req) : 0;
+    n += lens[l];
+  }
+  const int n_samples = n < kEstSamples ? n : kEstSamples;
+  est_score_blocks<D, 1>(p, req, kvh, warp, 1, lane, n, lens, sc);
   __syncthreads();
   // Everything above reads only the caller's inputs.  What follows writes: z, which the partial add of a call before
   // this one may still be reading, and the workspace headers -- so it waits for the kernels before (a no-op unless this

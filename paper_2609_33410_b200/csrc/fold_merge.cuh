@@ -46,29 +46,24 @@ __device__ __forceinline__ double pow2_double(int e) {       // 2^e, e in the no
 // nearest even; |result| < 2^61 / C.
 __device__ __forceinline__ long long to_grid(float g, double alpha) { return __double2ll_rn((double)g * alpha); }
 
-// One CTA of blockDim.x / 32 warps (at most kMergeMaxWarps) covers that many / W rows (a row = one (request, q head));
-// W in {1, 2, 4, 8, 16} warps share a row's slots (warp `sub` takes slots sub, sub + W, ... of every level).  Lane x owns EPT = D / 32
+// One row (a row = one (request, q head)) summed by W in {1, 2, 4, 8, 16} warps that share its slots (warp `sub`
+// takes slots sub, sub + W, ... of every level); wi = this warp's index among the warps that meet at `sync` (its row
+// of the staging arrays), the row's first warp being wi - sub.  Lane x owns EPT = D / 32
 // consecutive elements of A (one vector load per slot); lane 0 also carries L.  Two passes over the slots (the
 // second hits L1): the order-free maximum, then the integer sum.  The W warps of a row combine through staged
 // partials in shared memory: maxima by max, integer sums by integer addition, both exact, so neither the warp
-// count nor the slot order can change a bit.
+// count nor the slot order can change a bit.  Every warp that shares the staging arrays calls this together (sync
+// is their barrier; it is crossed twice when W > 1), active or not.
 // RESIDENT (one level, at most kMergeResident slots per warp): the slots are loaded once and stay in registers for
 // the second pass.
 constexpr int kMergeResident = 8;
-template <int EPT, bool RESIDENT>
-__global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const MergeParams p, const int W,
-                                                                         const long long n_rows) {
+template <int EPT, bool RESIDENT, typename Sync>
+__device__ __forceinline__ void merge_row(const MergeParams &p, const int W, const long long row, const bool active,
+                                          const int sub, const int wi, const int x, unsigned (*s_max)[32 * EPT + 1],
+                                          long long (*s_sum)[32 * EPT + 1], Sync sync) {
   constexpr int D = 32 * EPT;
-  __shared__ unsigned s_max[kMergeMaxWarps][D + 1];
-  __shared__ long long s_sum[kMergeMaxWarps][D + 1];
-  const int x = threadIdx.x & 31, wi = threadIdx.x >> 5;
-  const int sub = wi % W;
-  const long long row = (long long)blockIdx.x * ((blockDim.x >> 5) / W) + wi / W;
-  const bool active = row < n_rows;
   const int b = active ? (int)(row / p.Hq) : 0, h = active ? (int)(row % p.Hq) : 0;
   const int G = p.G, kvh = h / G, hg = h % G;
-  pdl_launch_dependents();                           // the next call's reference kernel may set up and load meanwhile
-  pdl_wait();                                        // slots and z come from the kernels before
   const float zrow = active ? p.z[row] : 0.f;        // requested early: only needed at the very end
 
   auto load_vec = [](const float *a, float (&v)[EPT]) {
@@ -136,7 +131,7 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
 #pragma unroll
     for (int e = 0; e < EPT; ++e) s_max[wi][e * 32 + x] = mx[e];
     if (x == 0) s_max[wi][D] = mxl;
-    __syncthreads();
+    sync();
     const int w0 = wi - sub;
     for (int o = 0; o < W; ++o) {
 #pragma unroll
@@ -184,7 +179,7 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
 #pragma unroll
     for (int e = 0; e < EPT; ++e) s_sum[wi][e * 32 + x] = acc[e];
     if (x == 0) s_sum[wi][D] = accl;
-    __syncthreads();
+    sync();
     if (sub != 0) return;
     for (int o = 1; o < W; ++o) {
 #pragma unroll
@@ -224,6 +219,20 @@ __global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const M
     if (p.lse) p.lse[row] = lse;
     if (p.row_status) p.row_status[row] = flags;
   }
+}
+
+// One CTA of blockDim.x / 32 warps (at most kMergeMaxWarps) covers that many / W rows.
+template <int EPT, bool RESIDENT>
+__global__ void __launch_bounds__(32 * kMergeMaxWarps) fold_merge_kernel(const MergeParams p, const int W,
+                                                                         const long long n_rows) {
+  constexpr int D = 32 * EPT;
+  __shared__ unsigned s_max[kMergeMaxWarps][D + 1];
+  __shared__ long long s_sum[kMergeMaxWarps][D + 1];
+  const int x = threadIdx.x & 31, wi = threadIdx.x >> 5;
+  const long long row = (long long)blockIdx.x * ((blockDim.x >> 5) / W) + wi / W;
+  pdl_launch_dependents();                           // the next call's reference kernel may set up and load meanwhile
+  pdl_wait();                                        // slots and z come from the kernels before
+  merge_row<EPT, RESIDENT>(p, W, row, row < n_rows, wi % W, wi, x, s_max, s_sum, [] { __syncthreads(); });
 }
 
 }  // namespace fold

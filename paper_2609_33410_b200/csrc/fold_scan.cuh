@@ -54,6 +54,7 @@ struct ScanParams {
   fold_ws_header *hdr;
   int max_slots, max_seqlen, Hq, Hkv, G, stack, R;
   int num_seqs;                                   // KV sequences of the launch (persistent kernels walk them all)
+  int chunk_major;                                // tcgen05 row-block kernel: the chunk list's order (1: chunk fastest)
   int paged, page_shift, max_pages, num_pages, box_tok;
   int num_splits, stages, vr;
   int pos_tok, pos_head, pos_seq;                 // which tensor-map coordinate (1..3) each axis is

@@ -29,6 +29,10 @@
 // the grid, the batch or the split hint.
 #pragma once
 
+#include <cooperative_groups.h>
+
+#include "fold_estimate.cuh"
+#include "fold_merge.cuh"
 #include "fold_scan_umma.cuh"
 
 namespace fold {
@@ -56,6 +60,19 @@ struct DecLayout {                                   // byte offsets from a 1 KB
 constexpr int kDecBarKFull = 40, kDecBarKEmpty = 0, kDecBarVFull = 4, kDecBarPvDone = 8, kDecBarSEmpty = 12,
               kDecBarPFull = 16, kDecBarQFull = 20, kDecBarLFull = 24, kDecBarSFull = 28, kDecBarPFree = 32, kDecBarTmemSlot = 38;
 constexpr int kDecLiveFlags = 384;                   // byte offset from kBar: [worker][weight buffer][warp] words: a key of the warp's 32 is live
+constexpr int kDecTimeouts = 448;                    // byte offset from kBar: which roles of this CTA gave up a wait (one word)
+constexpr int kDecStats = 456;                       // byte offset from kBar: value rows fetched, value rows in all, groups skipped (64-bit each)
+
+// A problem of one wave -- every worker has at most one canonical chunk -- runs the whole decode in ONE cooperative
+// launch of the scan kernel: the weight warps form their (sequence, kv head)'s reference from the 192 sampled keys
+// themselves while the key tiles travel (mode 1; mode 2 reads a given z), the chunks are scanned, and after a grid-wide
+// barrier the CTAs share out the rows of the order-free partial add.  Every step is the separate kernels' own device
+// code, so the three-launch path and this one agree bit for bit.
+struct FusedParams {
+  int mode;                                          // 0: the scan alone
+  EstParams est;
+  MergeParams mrg;
+};
 
 // D[tmem] (+)= A * B with both operands in shared memory (64-bit matrix descriptors as two words each).
 template <bool ACC>
@@ -105,13 +122,19 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&v)[N]) {
   for (int i = 0; i < N; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Barrier `id` (1..15) among `threads` threads of the CTA (whole warps); barrier 0 is __syncthreads'.
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // ------------------------------------------------------------------------------------------------
 // A worker's walk over its canonical chunks: entries g = first, first + step, ... of the launch's chunk list
 // (kv head fastest, then chunk, then sequence); entries past a sequence's own chunk count are skipped.
 struct DecWorker {
   int g, step, n_entries;        // next list entry to look at
-  int g_kvh, g_c, g_seq;         // that entry as (kv head, chunk, sequence): kept in step with g, no divisions per chunk
-  int d_kvh, d_c, d_seq;         // the step in the same mixed radix
+  int g_a, g_b, g_seq;           // that entry in the list's mixed radix (fastest digit first): kept in step with g, no divisions per chunk
+  int d_a, d_b, d_seq;           // the step in the same mixed radix
+  int ra, rb;                    // the radices: (kv heads, slots), or chunk-major (slots rounded up to even, kv heads)
   int len_seq, len_n;            // the sequence whose length was read last (entries of a worker mostly stay in one)
   int seq, kvh, c, n;            // the current chunk: sequence, kv head, chunk index, the sequence's length
   int t, t_end;                  // tile cursor: 128-key tiles [t, t_end) of the sequence remain in the chunk
@@ -121,11 +144,17 @@ __device__ __forceinline__ int dec_seqlen(const ScanParams &p, int seq) {
   const int n = p.seqlens[seq];
   return n < 0 ? 0 : (n > p.max_seqlen ? p.max_seqlen : n);
 }
+// The list's two orders.  Ordinarily kv head fastest, then chunk, then sequence.  Chunk-major (a decode that runs in one
+// launch, every worker with one chunk at most): chunk fastest, a (sequence, kv head)'s chunks padded to an even count,
+// so that the two workers of a CTA always scan chunks of the same (sequence, kv head) and share its reference.
+__device__ __forceinline__ int dec_radix_a(const ScanParams &p) { return p.chunk_major ? ((p.max_slots + 1) & ~1) : p.Hkv; }
+__device__ __forceinline__ int dec_radix_b(const ScanParams &p) { return p.chunk_major ? p.Hkv : p.max_slots; }
 __device__ __forceinline__ void dec_worker_init(DecWorker &w, const ScanParams &p, int first, int step) {
   w.g = first; w.step = step;
-  w.n_entries = p.num_seqs * p.max_slots * p.Hkv;
-  w.g_kvh = first % p.Hkv; w.g_c = (first / p.Hkv) % p.max_slots; w.g_seq = first / p.Hkv / p.max_slots;
-  w.d_kvh = step % p.Hkv; w.d_c = (step / p.Hkv) % p.max_slots; w.d_seq = step / p.Hkv / p.max_slots;
+  w.ra = dec_radix_a(p); w.rb = dec_radix_b(p);
+  w.n_entries = p.num_seqs * w.ra * w.rb;
+  w.g_a = first % w.ra; w.g_b = (first / w.ra) % w.rb; w.g_seq = first / w.ra / w.rb;
+  w.d_a = step % w.ra; w.d_b = (step / w.ra) % w.rb; w.d_seq = step / w.ra / w.rb;
   w.len_seq = -1; w.len_n = 0;
   w.seq = w.kvh = w.c = w.n = 0;
   w.t = w.t_end = w.t_first = 0;
@@ -133,12 +162,12 @@ __device__ __forceinline__ void dec_worker_init(DecWorker &w, const ScanParams &
 // Move to the worker's next non-empty chunk.  False when its list is exhausted.
 __device__ __forceinline__ bool dec_worker_next_chunk(DecWorker &w, const ScanParams &p) {
   while (w.g < w.n_entries) {
-    const int kvh = w.g_kvh, c = w.g_c, seq = w.g_seq;
-    w.g += w.step;                                           // and the same step in (kv head, chunk, sequence), with carries
-    w.g_kvh += w.d_kvh;
-    if (w.g_kvh >= p.Hkv) { w.g_kvh -= p.Hkv; ++w.g_c; }
-    w.g_c += w.d_c;
-    if (w.g_c >= p.max_slots) { w.g_c -= p.max_slots; ++w.g_seq; }
+    const int kvh = p.chunk_major ? w.g_b : w.g_a, c = p.chunk_major ? w.g_a : w.g_b, seq = w.g_seq;
+    w.g += w.step;                                           // and the same step in the mixed radix, with carries
+    w.g_a += w.d_a;
+    if (w.g_a >= w.ra) { w.g_a -= w.ra; ++w.g_b; }
+    w.g_b += w.d_b;
+    if (w.g_b >= w.rb) { w.g_b -= w.rb; ++w.g_seq; }
     w.g_seq += w.d_seq;
     if (seq != w.len_seq) { w.len_seq = seq; w.len_n = dec_seqlen(p, seq); }
     const int n = w.len_n;
@@ -154,8 +183,8 @@ __device__ __forceinline__ bool dec_worker_next_chunk(DecWorker &w, const ScanPa
 }
 // Tiles of list entry g (0 for an entry past its sequence's chunks).
 __device__ __forceinline__ int dec_entry_tiles(const ScanParams &p, int g) {
-  const int rest = g / p.Hkv;
-  const int c = rest % p.max_slots, seq = rest / p.max_slots;
+  const int ra = dec_radix_a(p), rb = dec_radix_b(p);
+  const int c = p.chunk_major ? g % ra : (g / ra) % rb, seq = g / ra / rb;
   const int n = dec_seqlen(p, seq);
   if (c >= num_chunks_of(n)) return 0;
   const int ctiles = chunk_keys_of(n) / kDecKeys;
@@ -208,7 +237,7 @@ __device__ __forceinline__ void dec_pair_next(DecPairWalk &x, const ScanParams &
 template <bool GATED, int NC, bool TAIL = false>
 __global__ void __launch_bounds__(kDecThreads, 1)
 fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                        const ScanParams p) {
+                        const ScanParams p, const FusedParams f) {
   constexpr int D = 128;
   static_assert(NC <= 8 && (!TAIL || GATED), "up to 8 rows; the tail belongs to finite depth");
   constexpr int NPV = 16;                                    // N of the value product; P_lo sits NPV / 2 rows after P_hi
@@ -251,7 +280,10 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       mbar_init(bar(kDecBarPFree + s), 1);
     }
     mbar_fence_init();
+    for (int i = 0; i < 8; ++i) reinterpret_cast<uint32_t *>(gen + LO::kBar + kDecTimeouts)[i] = 0u;   // timeouts, statistics
   }
+  // one launch for the whole decode: nothing before this kernel has cleared the workspace header
+  if (f.mode && blockIdx.x == 0 && threadIdx.x >= 32 && threadIdx.x < 48) reinterpret_cast<uint32_t *>(p.hdr)[threadIdx.x - 32] = 0u;
   if (warp == 1) tmem_alloc(bar(kDecBarTmemSlot), kDecTmemCols);
   // value ring, weight buffers and query tiles start as zeros: a row or column nobody writes must hold finite data
   for (int i = threadIdx.x; i < (LO::kLpart - OFF_V) / 16; i += kDecThreads)
@@ -265,7 +297,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 
   // the CTA's two workers and how many tiles each will walk (every warp computes both counts, a lane per entry)
   const int W = 2 * gridDim.x;
-  const int n_entries = p.num_seqs * p.max_slots * p.Hkv;
+  const int n_entries = p.num_seqs * dec_radix_a(p) * dec_radix_b(p);
   int TA = 0, TB = 0;
   {
     int ca = 0, cb = 0;
@@ -277,6 +309,8 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     TB = __reduce_add_sync(0xffffffffu, cb);
   }
   const int page_mask = (1 << p.page_shift) - 1;
+  uint32_t *s_timeouts = reinterpret_cast<uint32_t *>(gen + LO::kBar + kDecTimeouts);
+  unsigned long long *s_stats = reinterpret_cast<unsigned long long *>(gen + LO::kBar + kDecStats);
   bool dead = false;
   // warp-uniform bounded wait: the warp goes on together or gives up together
   auto wait_u = [&](uint32_t b, uint32_t parity) {
@@ -331,7 +365,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       }
       if (dead && lane == 0) {
         // gave up: the copies already requested must still land before the CTA may leave (bounded waits again)
-        atomicOr(&p.hdr->wait_timeouts, 1u);
+        atomicOr(s_timeouts, 1u);
         bool d2 = false;
         for (int back = 1; back <= depth && x.it - back >= 0; ++back) {
           const int it = x.it - back;
@@ -434,7 +468,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         }
         if (++idle > 8u * kWaitLimit) { dead = true; break; }   // bounded: give up, flag, fall through
       }
-      if (dead) atomicOr(&p.hdr->wait_timeouts, 8u);
+      if (dead) atomicOr(s_timeouts, 8u);
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------ weight warps: one key per thread
@@ -448,7 +482,10 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     DecWorker cur, nxt;
     dec_worker_init(nxt, p, 2 * blockIdx.x + set, W);
     bool have_next = my_tiles > 0 && dec_worker_next_chunk(nxt, p);
-    float z_next[NC];
+    float z_next[NC], z_own[NC];                             // z_own: references this worker formed itself (one launch for the whole decode)
+#pragma unroll
+    for (int r = 0; r < NC; ++r) z_own[r] = 0.f;
+    const bool own_z = f.mode == 1;
     pdl_wait();                                              // z comes from the kernel before
     // Staging the query rows (and the references) of chunk `w`, the worker's e-th, into query buffer e & 1, in two
     // steps so that the global loads are not waited for: stage_load requests them (one 16-byte piece of a row per
@@ -463,7 +500,7 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 #pragma unroll
       for (int r = 0; r < NC; ++r) {
         const int req = w.seq * p.stack + r / p.G, head = w.kvh * p.G + r % p.G;
-        z_next[r] = r < p.R ? p.z[(long long)req * p.Hq + head] : INFINITY;   // rows past R: weight 0 by themselves
+        z_next[r] = own_z ? z_own[r] : (r < p.R ? p.z[(long long)req * p.Hq + head] : INFINITY);   // rows past R: weight 0 by themselves
       }
     };
     auto stage_store = [&](int e) {
@@ -478,6 +515,40 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     };
     bool stage_open = false;                                 // loads requested, not yet stored
     if (have_next) { stage_load(nxt); stage_store(0); }
+    if (own_z) {
+      // The reference of the CTA's (sequence, kv head) -- in this mode both workers scan chunks of the same one --
+      // formed here while the key tiles travel: the 192 sampled keys' scores in blocks of 16 over the eight weight
+      // warps, then a warp per row.  The scores sit in the first worker's weight buffers, which nothing else touches
+      // before the first weights are handed over, and which are cleared again afterwards (a weight row nobody writes
+      // must read as zero).
+      const int ra = dec_radix_a(p), first = 2 * blockIdx.x;
+      const int e_c = first % ra, e_kvh = (first / ra) % p.Hkv, e_seq = first / ra / p.Hkv;
+      const int e_n = e_seq < p.num_seqs ? dec_seqlen(p, e_seq) : 0;
+      if (e_c < num_chunks_of(e_n)) {                        // the CTA has a chunk (the same test in all eight warps)
+        float (*sc)[kEstSamples] = reinterpret_cast<float (*)[kEstSamples]>(gen + LO::kP);
+        float *zs = reinterpret_cast<float *>(gen + LO::kP + kMaxRows / 2 * kEstSamples * 4);
+        const int ew = warp - 4;                             // 0..7
+        const int lens[kMaxLevels] = {e_n, 0, 0, 0};
+        const int n_samples = e_n < kEstSamples ? e_n : kEstSamples;
+        est_score_blocks<D, 2>(f.est, e_seq, e_kvh, ew, 8, lane, e_n, lens, sc);   // one request per sequence in this mode
+        named_bar_sync(1, 256);
+        for (int g = ew; g < p.G; g += 8) {
+          const float zval = est_reduce_row(sc[g], e_n, n_samples, lane);
+          if (lane == 0) {
+            zs[g] = zval;
+            if (e_c == 0) f.est.z[(long long)e_seq * p.Hq + e_kvh * p.G + g] = zval;   // the first chunk's CTA publishes it
+          }
+        }
+        named_bar_sync(1, 256);
+#pragma unroll
+        for (int r = 0; r < NC; ++r) z_next[r] = z_own[r] = r < p.R ? zs[r] : INFINITY;
+        named_bar_sync(1, 256);                              // everybody has read the references
+        *reinterpret_cast<uint4 *>(gen + LO::kP + (threadIdx.x - 128) * 32) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4 *>(gen + LO::kP + (threadIdx.x - 128) * 32 + 16) = make_uint4(0, 0, 0, 0);
+        fence_proxy_async_smem();
+        named_bar_sync(1, 256);                              // cleared before the first weights are written
+      }
+    }
     unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
     const uint64_t vpol = policy_evict_first();
     const int vbox = p.vr;                                   // tokens per value box (16 or 32)
@@ -699,12 +770,12 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       flush_chunk();
     }
     if (lane == 0) {
-      if (dead) atomicOr(&p.hdr->wait_timeouts, 16u);
+      if (dead) atomicOr(s_timeouts, 16u);
       if (st_total) {
-        atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), GATED ? st_fetched : st_total);
-        atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), st_total);
+        atomicAdd(s_stats, GATED ? st_fetched : st_total);
+        atomicAdd(s_stats + 1, st_total);
       }
-      if (st_skipped) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), st_skipped);
+      if (st_skipped) atomicAdd(s_stats + 2, st_skipped);
     }
   }
 
@@ -714,6 +785,36 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, kDecTmemCols);
+  }
+  if (f.mode) {
+    // the whole decode in this launch: every CTA's slots (and the cleared header) are out before any row is added
+    __threadfence();
+    cooperative_groups::this_grid().sync();
+  }
+  if (threadIdx.x == 0) {
+    // what the roles of this CTA recorded, into the workspace header (cleared by the kernel before, or above)
+    pdl_wait();
+    if (*s_timeouts) atomicOr(&p.hdr->wait_timeouts, *s_timeouts);
+    if (s_stats[1]) {
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_fetched), s_stats[0]);
+      atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_rows_total), s_stats[1]);
+    }
+    if (s_stats[2]) atomicAdd(reinterpret_cast<unsigned long long *>(&p.hdr->v_slices_skipped), s_stats[2]);
+  }
+  if (f.mode && warp < 8) {
+    // the order-free partial add, a row at a time per CTA: eight warps share the row's slots (the key ring is free now)
+    unsigned (*s_max)[D + 1] = reinterpret_cast<unsigned (*)[D + 1]>(gen);
+    long long (*s_sum)[D + 1] = reinterpret_cast<long long (*)[D + 1]>(gen + 8 * (D + 1) * 4 + 8);
+    const long long n_rows = (long long)p.num_seqs * p.Hq;
+    for (long long row = blockIdx.x; row < n_rows; row += gridDim.x) {
+      // a sequence without keys has no worker: its rows' references are written here (the estimate of no key is 0)
+      if (f.mode == 1 && threadIdx.x == 0 && dec_seqlen(p, (int)(row / p.Hq)) == 0) f.est.z[row] = 0.f;
+      if (p.max_slots <= 8 * kMergeResident)                 // a warp's share of the slots stays in registers
+        merge_row<D / 32, true>(f.mrg, 8, row, true, warp, warp, lane, s_max, s_sum, [] { named_bar_sync(3, 256); });
+      else
+        merge_row<D / 32, false>(f.mrg, 8, row, true, warp, warp, lane, s_max, s_sum, [] { named_bar_sync(3, 256); });
+      named_bar_sync(3, 256);                                // the staging arrays are reused by the next row
+    }
   }
 }
 
