@@ -430,10 +430,9 @@ def main():
         if args.tail:
             # block tail (the block model's mean): cut keys add weight x their 64-key block's mean value; the table is
             # built once from the cache, outside the timed region (it belongs to cache write)
-            if cascade:
-                raise SystemExit("--tail: the block tail is built into the row-block scan only (no stacked prefix level)")
             if not (args.planes and args.fp8v):               # (the 8-bit value format has its own cut model: below)
-                F.fold_block_means(caches[0], stream)
+                for c in caches:                                # a cascade: every level has its own table
+                    F.fold_block_means(c, stream)
             torch.cuda.synchronize()
         quant_ms = None
         if args.planes:

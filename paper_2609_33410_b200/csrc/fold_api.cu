@@ -411,19 +411,22 @@ int launch_stacked(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, 
 }
 
 // Stacked rows on tcgen05 (head_dim 128, at least 64 stacked rows): one CTA per (split, 128-row tile).
-int launch_stacked_umma(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, bool gated,
+int launch_stacked_umma(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, dim3 grid, bool gated, bool tail,
                         cudaStream_t st) {
   p.stages = kUmmaStages;
   p.vr = 0;
   grid.x *= (p.R + kUmmaRows - 1) / kUmmaRows;
-  static SmemFlags configured_g, configured_d;
+  static SmemFlags configured_g, configured_d, configured_t;
   cudaError_t rc;
-  if (gated) {
-    if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<true>, configured_g)) return e;
-    rc = launch_pdl(fold_scan_stacked_umma_kernel<true>, grid, dim3(kUmmaThreads), UmmaLayout::kTotal, st, mk, mv, p);
+  if (gated && tail) {
+    if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<true, true>, configured_t)) return e;
+    rc = launch_pdl(fold_scan_stacked_umma_kernel<true, true>, grid, dim3(kUmmaThreads), UmmaLayout::kTotal, st, mk, mv, p);
+  } else if (gated) {
+    if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<true, false>, configured_g)) return e;
+    rc = launch_pdl(fold_scan_stacked_umma_kernel<true, false>, grid, dim3(kUmmaThreads), UmmaLayout::kTotal, st, mk, mv, p);
   } else {
-    if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<false>, configured_d)) return e;
-    rc = launch_pdl(fold_scan_stacked_umma_kernel<false>, grid, dim3(kUmmaThreads), UmmaLayout::kTotal, st, mk, mv, p);
+    if (int e = opt_in_smem(fold_scan_stacked_umma_kernel<false, false>, configured_d)) return e;
+    rc = launch_pdl(fold_scan_stacked_umma_kernel<false, false>, grid, dim3(kUmmaThreads), UmmaLayout::kTotal, st, mk, mv, p);
   }
   if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
@@ -715,10 +718,11 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st, const Fu
   const dim3 grid = stacked ? dim3(p.num_splits, g.Hkv, g.num_seqs) : dim3(g.Hkv * p.row_groups, p.num_splits, g.num_seqs);
   p.box_min = 13;
   if (stacked) {
-    // the tcgen05 kernels have no block tail yet: a gated stacked level with a mean table runs on mma.sync
+    // with a table of block means the single-tile tcgen05 kernel serves every row count from 64 up (a CTA per 128 rows:
+    // the pair kernel's tensor memory has no room for the cut-mass operand)
     const bool tail = gated && p.vmean != nullptr;
     if (g.D == 128 && g.R > kUmmaRows && !tail) return launch_stacked_pair(mk, mv, p, grid, gated, st);
-    if (g.D == 128 && g.R >= 64 && !tail) return launch_stacked_umma(mk, mv, p, grid, gated, st);
+    if (g.D == 128 && g.R >= 64) return launch_stacked_umma(mk, mv, p, grid, gated, tail, st);
     return g.D == 128 ? launch_stacked<128>(mk, mv, p, grid, gated, st) : launch_stacked<64>(mk, mv, p, grid, gated, st);
   }
   if (g.D == 128) return gated ? launch_gated<128>(mk, mv, p, grid, st) : launch_dense<128>(mk, mv, p, grid, st);

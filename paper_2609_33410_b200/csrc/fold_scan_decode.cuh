@@ -530,7 +530,9 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const int ew = warp - 4;                             // 0..7
         const int lens[kMaxLevels] = {e_n, 0, 0, 0};
         const int n_samples = e_n < kEstSamples ? e_n : kEstSamples;
-        est_score_blocks<D, 2>(f.est, e_seq, e_kvh, ew, 8, lane, e_n, lens, sc);   // one request per sequence in this mode
+#pragma unroll 1
+        for (int blk = ew; blk < kEstWarps; blk += 8)        // (one block at a time: two at once cost the whole kernel registers)
+          est_score_blocks<D, 1>(f.est, e_seq, e_kvh, blk, 1, lane, e_n, lens, sc);   // one request per sequence in this mode
         named_bar_sync(1, 256);
         for (int g = ew; g < p.G; g += 8) {
           const float zval = est_reduce_row(sc[g], e_n, n_samples, lane);

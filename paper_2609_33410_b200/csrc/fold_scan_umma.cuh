@@ -31,15 +31,16 @@ constexpr int kUmmaThreads = 10 * 32;                // producer, MMA, 8 weight 
 constexpr int kUmmaWeightThreads = 8 * 32;
 constexpr int kUmmaRows = 128;                       // query rows per CTA (MMA M)
 constexpr int kUmmaStages = 6;
-constexpr int kUmmaTmemCols = 512;                   // S0 [0,64)  S1 [64,128)  O [128,256)  Q [256,320)  P_hi [320,352)  P_lo [352,384)
-constexpr int kUmmaColQ = 256, kUmmaColPhi = 320, kUmmaColPlo = 352;
+constexpr int kUmmaTmemCols = 512;                   // S0 [0,64)  S1 [64,128)  O [128,256)  Q [256,320)  P_hi [320,352)  P_lo [352,384)  cut mass hi [384,400) lo [400,416)
+constexpr int kUmmaColQ = 256, kUmmaColPhi = 320, kUmmaColPlo = 352, kUmmaColCutHi = 384, kUmmaColCutLo = 400;
 
 struct UmmaLayout {                                  // byte offsets from a 1 KB-aligned base
   static constexpr int kRing = 0;                                // stages x (K tile 16 KB + V tile 16 KB)
   static constexpr int kStage = 32768;
   static constexpr int kBar = kRing + kUmmaStages * kStage;
   static constexpr int kLbuf = kBar + 256;                       // 128 floats: the second half-row's share of L
-  static constexpr int kTotal = kLbuf + 512 + 1024;              // + alignment slack
+  static constexpr int kMean = kBar + 1024;                      // block tail: the chunk's block means [2 halves][16 blocks][128 B], swizzled
+  static constexpr int kTotal = kMean + 4096 + 1024;             // + alignment slack
 };
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -89,6 +90,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // 32 consecutive FP32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
@@ -114,7 +120,13 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major) {
          ((uint32_t)(kUmmaRows >> 4) << 24);
 }
 
-template <bool GATED>
+// TAIL (with GATED; Section 4 "Depth as a dial", the block model's mean): a row's cut keys add their summed weight
+// times the mean value row of their 64-key block -- a tile here.  Each thread keeps the cut mass of its 32 keys per tile
+// of the chunk; with the chunk's last weights it writes them, split into two BF16 terms like the weights, to 16 more
+// columns of its lane (the two threads of a row own 16 K slots each: slot 16 half + block), the chunk's block means
+// go to shared memory as a [16 blocks x 128 channels] MN-major tile, and four more products
+// O += cut_hi M + cut_lo M (K = 16 each, the same tile for both halves' slots) follow the chunk's last value product.
+template <bool GATED, bool TAIL = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                               const ScanParams p) {
@@ -251,6 +263,14 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
             umma_bf16_ta<true>(tm + 128, tm + (term ? kUmmaColPlo : kUmmaColPhi) + j * 8, v_lo + j * (2048 >> 4),
                                umma_desc_hi(1024), idesc_pv);
           }
+          if (TAIL && chunk_ends) {
+            // the chunk's tail: cut mass [128 rows, 2 x 16 slots] x block means [16, 128], the means for both slot groups
+            const uint32_t m_lo = umma_desc_lo(base + LO::kMean, 2048);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              umma_bf16_ta<true>(tm + 128, tm + ((i & 2) ? kUmmaColCutLo : kUmmaColCutHi) + (i & 1) * 8, m_lo,
+                                 umma_desc_hi(1024), idesc_pv);
+          }
           tc_commit(pv_done + 8u * stage);
         }
         __syncwarp();
@@ -265,10 +285,23 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
     // ------------------------------------------------------------ weight warps: one query row per thread
     const bool valid_row = r_glob < R;
     float l_row = 0.f;
+    float cut[TAIL ? 16 : 1];                                // this thread's cut mass per tile (= 64-key block) of the chunk
+#pragma unroll
+    for (int i = 0; i < (TAIL ? 16 : 1); ++i) cut[i] = 0.f;
     int it = 0, chunk_i = 0;
     for (TileCursor k = cursor_begin(w, split); cursor_valid(k, w); ++it) {
       const int b = it & 1, stage = it % kUmmaStages;
       const int key_base = k.t * kTileKeys;
+      TileCursor k_after = k;
+      const bool last_of_chunk = cursor_next(k_after, w, p.num_splits);
+      uint4 mean_piece = make_uint4(0, 0, 0, 0);             // block tail: this thread's 16 bytes of the chunk's means, requested early
+      if (TAIL && last_of_chunk) {
+        const int tw = threadIdx.x - 64, blk = k.c * w.ctiles + (tw >> 4);
+        if ((tw >> 4) < w.ctiles && blk * 64 < n)
+          mean_piece = *reinterpret_cast<const uint4 *>(p.vmean + (long long)seq * p.vm_stride_seq + (long long)blk * p.vm_stride_block +
+                                                        (long long)kvh * p.vm_stride_head + (tw & 15) * 8);
+      }
+      float cm = 0.f;
       uint32_t ph[16], pl[16];                               // this thread's 32 weights, BF16 pairs: hi and lo terms
       // the tcgen05 loads and stores below are warp-wide: the warp takes them together or not at all
       const bool have_s = __all_sync(0xffffffffu, mbar_wait(s_full + 8u * b, (uint32_t)((it >> 1) & 1), dead));
@@ -299,6 +332,7 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
             const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
             const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
             l_row += ((h0 + g0) + (pw[0] - pm[0])) + ((h1 + g1) + (pw[1] - pm[1]));
+            if (TAIL) cm += (pw[0] - pm[0]) + (pw[1] - pm[1]);
             ph[j / 2] = hi2;
             pl[j / 2] = lo2;
           }
@@ -313,6 +347,25 @@ fold_scan_stacked_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __g
                                                         (uint32_t)(((it - 1) / kUmmaStages) & 1), dead))) {
         tmem_st16(lane_addr + kUmmaColPhi + ch * 16, ph);    // this thread's 32 keys = 16 columns of its lane
         tmem_st16(lane_addr + kUmmaColPlo + ch * 16, pl);
+        if (TAIL) {
+          cut[k.t - k.c * w.ctiles] = cm;
+          if (last_of_chunk) {
+            // the chunk's cut mass in two BF16 terms, this thread's 16 slots = 8 columns of each term; and the means
+            uint32_t chi[8], clo[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float c0 = cut[2 * i], c1 = cut[2 * i + 1];
+              chi[i] = pack_bf16(c0, c1);
+              clo[i] = pack_bf16(c0 - __uint_as_float(chi[i] << 16), c1 - __uint_as_float(chi[i] & 0xffff0000u));
+              cut[2 * i] = cut[2 * i + 1] = 0.f;
+            }
+            tmem_st8(lane_addr + kUmmaColCutHi + ch * 8, chi);
+            tmem_st8(lane_addr + kUmmaColCutLo + ch * 8, clo);
+            const int tw = threadIdx.x - 64;
+            *reinterpret_cast<uint4 *>(gen + LO::kMean + tile_off(tw >> 4, tw & 15, 16)) = mean_piece;
+            fence_proxy_async_smem();                        // generic writes, then tensor-core (async proxy) reads
+          }
+        }
         tmem_st_wait();
         if (key_base + kTileKeys > n) {                      // ragged tail: value rows past n may hold anything
           const int tw = threadIdx.x - 64;

@@ -79,9 +79,10 @@ def test_block_tail_is_exact_for_values_constant_within_blocks():
 
 
 @pytest.mark.parametrize("Hq,Hkv,stack,D", [(16, 1, 1, 128), (12, 1, 1, 64), (8, 2, 4, 128), (8, 2, 5, 128), (4, 4, 33, 64),
-                                            (8, 2, 40, 128)])
+                                            (8, 2, 16, 128), (8, 2, 40, 128), (8, 2, 75, 128)])
 def test_block_tail_with_wider_row_blocks_and_stacked_rows(Hq, Hkv, stack, D):
-    # 9..16 rows per (sequence, kv head): the rows-on-M gated kernel; more: the stacked-row kernel
+    # 9..16 rows per (sequence, kv head): the rows-on-M gated kernel; more: the stacked-row kernels (from 64 rows at
+    # head_dim 128 on tcgen05: 64, 160 and 300 rows here, i.e. one, two and three row tiles)
     w = make_decode_workload(2 * stack, Hq, Hkv, D, [1500, 333], seed=91, device=DEV, stack=stack,
                              poison_padding=True, capacity=1600)
     vm = oracle_block_means(w)
