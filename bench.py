@@ -300,6 +300,12 @@ def run_sweep(args, dev):
                                     out=bufs.out, lse=bufs.lse, row_status=bufs.row_status, refine_tau=args.refine_tau)
                     for _ in range(3):
                         F.fold_decode(a, stream)
+                    if not math.isinf(T) and not args.no_live_hint:
+                        # what a decode loop knows from the step before: the fraction of value rows kept (scheduling only)
+                        torch.cuda.synchronize()
+                        h0 = bufs.header()
+                        a.live_hint = max(h0.v_rows_fetched / max(h0.v_rows_total, 1), 1e-6)
+                        F.fold_decode(a, stream)
                     reps = 21 if cache_bytes < 2e9 else 7
                     times = []
                     for _ in range(reps):
@@ -370,6 +376,8 @@ def main():
     ap.add_argument("--probe-read", action="store_true", help="only measure the read-only bandwidth and print it")
     ap.add_argument("--launches", default="auto", choices=["auto", "one", "separate"],
                     help="fold_args.flags: FOLD_ONE_LAUNCH / FOLD_SEPARATE_LAUNCHES (auto: the library's own choice)")
+    ap.add_argument("--no-live-hint", action="store_true",
+                    help="do not pass the live fraction measured in the warm-up steps as fold_args.live_hint")
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the short runs of the other named configurations (c1, c3, c4) in the default line")
     args = ap.parse_args()
@@ -469,13 +477,16 @@ def main():
         # a cascade's first level may be scanned on a side stream of the caller's (fork / join inside the one C-ABI call)
         cside = F.CascadeSide(dev) if cascade and args.cascade_streams == 1 else None
 
+        live_hint = [0.0]                                     # fold_args.live_hint of the timed steps (from the warm-up steps)
+
         def make(depth, z_mode, extra_flags=0):
             return [F.make_args(l.q, c, scale=l.scale, z_mode=z_mode, z=bufs.z, depth_T=depth, stack=l.stack,
                                 num_splits=args.num_splits, workspace=b.workspace, out=bufs.out, lse=bufs.lse,
                                 row_status=bufs.row_status, draft_mask=draft_masks if args.drafts > 1 else None,
                                 draft_len=args.drafts if args.drafts > 1 else 0, refine_tau=args.refine_tau,
                                 refine_tau_v=args.refine_tau_v, side=cside if i == 0 else None,
-                                flags=extra_flags | {"auto": 0, "one": F.ONE_LAUNCH, "separate": F.SEPARATE_LAUNCHES}[args.launches])
+                                flags=extra_flags | {"auto": 0, "one": F.ONE_LAUNCH, "separate": F.SEPARATE_LAUNCHES}[args.launches],
+                                live_hint=live_hint[0])
                     for i, (l, c, b) in enumerate(zip(levels, caches, lbufs))]
 
         # A cascade's levels are independent once the reference is fixed: with --cascade-streams 2 the prefix level
@@ -520,15 +531,32 @@ def main():
 
         def timed(depth, steps, warmup, sample_clocks):
             # (1) whole steps: estimate -> scan(s) -> partial add, chained in the stream by one C-ABI call
+            live_hint[0] = 0.0
             a = make(depth, F.Z_ESTIMATE)
             for _ in range(warmup):
                 step_whole(a)
+            if not math.isinf(depth) and not args.no_live_hint and not args.z_from_lse:
+                # what a decode loop knows from the step before: the fraction of value rows kept.  Passed on as
+                # fold_args.live_hint (scheduling only: how the scan splits its on-chip ring between keys and values)
+                torch.cuda.synchronize()
+                h0 = headers()
+                live_hint[0] = max(sum(h0["fetched"]) / max(sum(h0["total"]), 1), 1e-6)
+                a = make(depth, F.Z_ESTIMATE)
+                for _ in range(warmup):
+                    step_whole(a)
             if args.z_from_lse:
                 torch.cuda.synchronize()
                 bufs.z.copy_(bufs.lse)                             # the dense log-sum-exp of the rows (L sums every key)
                 a = make(depth, F.Z_GIVEN)
                 for _ in range(warmup):
                     step_whole(a)
+                if not math.isinf(depth) and not args.no_live_hint:
+                    torch.cuda.synchronize()
+                    h0 = headers()
+                    live_hint[0] = max(sum(h0["fetched"]) / max(sum(h0["total"]), 1), 1e-6)
+                    a = make(depth, F.Z_GIVEN)
+                    for _ in range(warmup):
+                        step_whole(a)
             run_step = lambda: step_whole(a)
             if args.graph:
                 # the whole call (memset + estimate + scan + partial add) captured once and replayed: takes the host's
@@ -615,7 +643,7 @@ def main():
             return dict(ms_per_step=max_over_ranks(total_ms / steps, world, dev), scan_ms=statistics.mean(scan_ms),
                         scan_ms_min=min(scan_ms), est_ms=statistics.mean(est_ms), merge_ms=statistics.mean(mrg_ms),
                         lone_us_median=max_over_ranks(lone[len(lone) // 2], world, dev), lone_us_min=lone[0],
-                        settled_ms=settled_ms,
+                        settled_ms=settled_ms, live_hint=live_hint[0],
                         clocks=sampler.summary() if sample_clocks else None, **hd)
 
         r16 = timed(T, steps, warm, sample_clocks)
@@ -670,6 +698,8 @@ def main():
                        "sharding": shard_note(world), "cache_bytes_per_gpu": cache_bytes,
                        "cascade_streams": args.cascade_streams if cascade else None,
                        "cuda_graph": bool(args.graph), "block_tail": bool(args.tail),
+                       "live_hint": {"T16": r16["live_hint"], "note": "fold_args.live_hint of the timed steps = the fraction of value "
+                                     "rows the warm-up steps fetched (what a decode loop knows from its step before); scheduling only"},
                        "key_format": "two INT8 planes + BF16 scale per key" if args.planes else "bf16",
                        "value_format": "two E4M3 planes, power-of-two scale" if args.fp8v else "bf16",
                        "refine_tau": (args.refine_tau or "auto: max(log2(n) - 2, 4)") if args.planes else None,

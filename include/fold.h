@@ -208,6 +208,12 @@ typedef struct fold_args {
   fold_stream side_stream;             /* fold_decode_cascade, levels[0] only: a second stream of the caller's and two */
   void *side_fork_event;               /* cudaEvent_t of the caller's (created with timing disabled, say) on which the */
   void *side_join_event;               /* first level is scanned; all three NULL: every level on `stream` */
+  float live_hint;                     /* finite depth_T: the fraction of value rows the caller expects to be kept (what
+                                          v_rows_fetched / v_rows_total of the step before was, say), in (0, 1]; 0 = no
+                                          expectation.  Scheduling only -- how the row-block scan splits its on-chip ring
+                                          between key and value tiles (Section 4, "Weight-gated reads": the byte mix
+                                          2D + 2D lambda varies with lambda) -- never a bit of any result.  NaN or
+                                          negative values count as 0. */
 } fold_args;
 
 /* First 64 bytes of every workspace, zeroed at the start of each scan. */

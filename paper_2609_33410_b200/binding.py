@@ -51,7 +51,8 @@ class FoldArgs(C.Structure):
                 ("out", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p),
                 ("draft_mask", C.c_void_p), ("draft_len", C.c_int32), ("refine_tau", C.c_float),
                 ("refine_tau_v", C.c_float), ("flags", C.c_int32),
-                ("side_stream", C.c_void_p), ("side_fork_event", C.c_void_p), ("side_join_event", C.c_void_p)]
+                ("side_stream", C.c_void_p), ("side_fork_event", C.c_void_p), ("side_join_event", C.c_void_p),
+                ("live_hint", C.c_float)]
 
 
 class FoldPartials(C.Structure):
@@ -234,7 +235,7 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
               workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
               lse: Optional[torch.Tensor] = None, row_status: Optional[torch.Tensor] = None,
               draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0,
-              refine_tau_v: float = 0.0, flags: int = 0, side=None) -> FoldArgs:
+              refine_tau_v: float = 0.0, flags: int = 0, side=None, live_hint: float = 0.0) -> FoldArgs:
     """`side`: a CascadeSide (a second stream and two events of the caller's) for fold_decode_cascade's first level."""
     assert q.dtype == torch.bfloat16 and q.dim() == 3 and q.stride(2) == 1
     B, Hq, D = q.shape
@@ -259,6 +260,7 @@ def make_args(q: torch.Tensor, cache: KVCache, *, scale: Optional[float] = None,
     a.refine_tau = float(refine_tau)
     a.refine_tau_v = float(refine_tau_v)
     a.flags = int(flags)
+    a.live_hint = float(live_hint)
     if side is not None:
         a.side_stream, a.side_fork_event, a.side_join_event = side.stream.cuda_stream, side.fork.cuda_event, side.join.cuda_event
     return a
@@ -416,11 +418,11 @@ def alloc_buffers(q: torch.Tensor, cache: KVCache, stack: int = 1) -> DecodeBuff
 def decode(q: torch.Tensor, cache: KVCache, bufs: DecodeBuffers, *, depth_T: float = math.inf,
            z_mode: int = Z_ESTIMATE, num_splits: int = 0, scale: Optional[float] = None, stack: int = 1,
            draft_mask: Optional[torch.Tensor] = None, draft_len: int = 0, refine_tau: float = 0.0,
-           refine_tau_v: float = 0.0, flags: int = 0, stream=None) -> FoldArgs:
+           refine_tau_v: float = 0.0, flags: int = 0, live_hint: float = 0.0, stream=None) -> FoldArgs:
     args = make_args(q, cache, scale=scale, z_mode=z_mode, z=bufs.z, depth_T=depth_T, num_splits=num_splits,
                      stack=stack, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, row_status=bufs.row_status,
                      draft_mask=draft_mask, draft_len=draft_len, refine_tau=refine_tau, refine_tau_v=refine_tau_v,
-                     flags=flags)
+                     flags=flags, live_hint=live_hint)
     fold_decode(args, stream)
     return args
 

@@ -460,10 +460,10 @@ int sm_count() {
 }
 // f.mode != 0: the whole decode in this launch, which is then a cooperative one (its CTAs meet at a grid-wide barrier
 // between the scan and the partial add; the grid is one CTA per SM at most, so all of them are resident).
-template <bool GATED, int NC, bool TAIL>
+template <bool GATED, int NC, bool TAIL, int KEYS>
 int launch_decode_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, const FusedParams &f, int ctas, cudaStream_t st) {
   static SmemFlags configured;
-  if (int rc = opt_in_smem(fold_scan_decode_kernel<GATED, NC, TAIL>, configured)) return rc;
+  if (int rc = opt_in_smem(fold_scan_decode_kernel<GATED, NC, TAIL, KEYS>, configured)) return rc;
   cudaError_t rc;
   if (f.mode) {
     cudaLaunchConfig_t cfg;
@@ -473,19 +473,28 @@ int launch_decode_as(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    rc = cudaLaunchKernelEx(&cfg, fold_scan_decode_kernel<GATED, NC, TAIL>, mk, mv, p, f);
+    rc = cudaLaunchKernelEx(&cfg, fold_scan_decode_kernel<GATED, NC, TAIL, KEYS>, mk, mv, p, f);
   } else {
-    rc = launch_pdl(fold_scan_decode_kernel<GATED, NC, TAIL>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p, f);
+    rc = launch_pdl(fold_scan_decode_kernel<GATED, NC, TAIL, KEYS>, dim3(ctas), dim3(kDecThreads), DecLayout::kTotal, st, mk, mv, p, f);
   }
   if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
 }
-template <bool GATED, bool TAIL>
-int launch_decode(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, const FusedParams &f, int ctas, cudaStream_t st) {
-  if (p.R == 1) return launch_decode_as<GATED, 1, TAIL>(mk, mv, p, f, ctas, st);
-  if (p.R <= 4) return launch_decode_as<GATED, 4, TAIL>(mk, mv, p, f, ctas, st);
-  if (p.R <= 8) return launch_decode_as<GATED, 8, TAIL>(mk, mv, p, f, ctas, st);
+template <bool GATED, bool TAIL, int KEYS>
+int launch_decode_rows(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, const FusedParams &f, int ctas, cudaStream_t st) {
+  if (p.R == 1) return launch_decode_as<GATED, 1, TAIL, KEYS>(mk, mv, p, f, ctas, st);
+  if (p.R <= 4) return launch_decode_as<GATED, 4, TAIL, KEYS>(mk, mv, p, f, ctas, st);
+  if (p.R <= 8) return launch_decode_as<GATED, 8, TAIL, KEYS>(mk, mv, p, f, ctas, st);
   return FOLD_EUNSUPPORTED;                                  // more rows stay on the mma.sync kernels
+}
+// keys: the key ring's depth for a depth-gated scan (2, 3 or 4 of the six stages; scheduling only); dense decode runs 2.
+template <bool GATED, bool TAIL>
+int launch_decode(const CUtensorMap &mk, const CUtensorMap &mv, ScanParams &p, const FusedParams &f, int ctas, int keys,
+                  cudaStream_t st) {
+  if (!GATED) return launch_decode_rows<GATED, TAIL, 2>(mk, mv, p, f, ctas, st);
+  if (keys == 2) return launch_decode_rows<GATED, TAIL, 2>(mk, mv, p, f, ctas, st);
+  if (keys == 4) return launch_decode_rows<GATED, TAIL, 4>(mk, mv, p, f, ctas, st);
+  return launch_decode_rows<GATED, TAIL, 3>(mk, mv, p, f, ctas, st);
 }
 
 // Narrow row blocks (rows on N): unpadded value slices; three K stages (measured: a fourth buys nothing and costs L1).
@@ -708,8 +717,12 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st, const Fu
       p.chunk_major = 1;
       ctas = units * ((g.max_slots + 1) / 2);                // one chunk per worker at most
     }
-    if (!gated) return launch_decode<false, false>(mk, mv, p, f, (int)ctas, st);
-    return p.vmean ? launch_decode<true, true>(mk, mv, p, f, (int)ctas, st) : launch_decode<true, false>(mk, mv, p, f, (int)ctas, st);
+    // the caller's expectation of the live fraction picks the ring's split: four fifths and more live -> two key stages
+    // and four value stages (dense decode's), under 15 % -> four and two, else (and without a hint) three and three
+    const float lh = a->live_hint;
+    const int keys = !(lh > 0.f) ? 3 : (lh >= 0.8f ? 2 : (lh < 0.15f ? 4 : 3));
+    if (!gated) return launch_decode<false, false>(mk, mv, p, f, (int)ctas, 2, st);
+    return p.vmean ? launch_decode<true, true>(mk, mv, p, f, (int)ctas, keys, st) : launch_decode<true, false>(mk, mv, p, f, (int)ctas, keys, st);
   }
   p.num_splits = choose_splits(a, g, tile_keys);
 

@@ -234,7 +234,8 @@ __device__ __forceinline__ void dec_pair_next(DecPairWalk &x, const ScanParams &
 // the mean value row of their 64-key block.  Each weight warp sums its 32 keys' cut weights per row and tile (a tile
 // is two blocks, a block two warps); at the chunk's end every thread -- one channel -- adds cut mass x mean for the
 // chunk's blocks in block order, in FP32.
-template <bool GATED, int NC, bool TAIL = false>
+// KEYS: the key ring's depth (the value ring takes the rest of the six stages).
+template <bool GATED, int NC, bool TAIL = false, int KEYS = (GATED ? 3 : 2)>
 __global__ void __launch_bounds__(kDecThreads, 1)
 fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                         const ScanParams p, const FusedParams f) {
@@ -243,17 +244,15 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   constexpr int NPV = 16;                                    // N of the value product; P_lo sits NPV / 2 rows after P_hi
   constexpr int PB = 2;                                      // weight buffers per worker
   constexpr int PBYTES = NPV * 256;                          // [2 key halves][NPV rows][128 B]
-  // Six 32 KB stages in all.  Depth-gated: three for keys and three for values (four and two streams a cache nobody
-  // keeps a value row of 5 % faster, and one with half its rows live 12 % slower).  Dense: a key stage is free as soon
-  // as its scores are issued, a value stage waits for the weights, so two key stages feed four value stages (5 % over
-  // three and three).
-#ifndef FOLD_DEC_GATED_KS
-#define FOLD_DEC_GATED_KS 3
-#endif
-#ifndef FOLD_DEC_DENSE_KS
-#define FOLD_DEC_DENSE_KS 2
-#endif
-  constexpr int KS = GATED ? FOLD_DEC_GATED_KS : FOLD_DEC_DENSE_KS, VS = 6 - KS;
+  // Six 32 KB stages in all.  Dense: a key stage is free as soon as its scores are issued, a value stage waits for the
+  // weights, so two key stages feed four value stages (5 % over three and three).  Depth-gated, the best split depends on
+  // how much of the cache is live: a cache that is nearly all live wants dense decode's two and four (C2 at T=16: 321 us
+  // against 330 with three and three), one that is half live three and three (C3: 272 against 278 us with two and
+  // four; 29 % live: 238 against 263), one nobody keeps a value row of four and two (5 % over three and three).  The
+  // caller may say what it expects (fold_args.live_hint); three and three without a hint.  The split only schedules: every
+  // one gives the same bits.
+  static_assert(KEYS >= 2 && KEYS <= 4, "two to four key stages");
+  constexpr int KS = KEYS, VS = 6 - KS;
   using LO = DecLayout;
   constexpr int OFF_V = KS * LO::kTile;                      // the value ring follows the key ring
   extern __shared__ uint8_t smem_raw[];

@@ -45,7 +45,8 @@ int main(void) {
          offsetof(fold_args, depth_T), offsetof(fold_args, row_status));
   printf("%zu %zu %zu\n", offsetof(fold_partials, rows), offsetof(fold_partials, slot_stride),
          offsetof(fold_ws_header, v_rows_total));
-  printf("%zu %zu %zu\n", offsetof(fold_args, flags), offsetof(fold_args, side_stream), offsetof(fold_args, side_join_event));
+  printf("%zu %zu %zu %zu\n", offsetof(fold_args, flags), offsetof(fold_args, side_stream), offsetof(fold_args, side_join_event),
+         offsetof(fold_args, live_hint));
   return 0;
 }
 """
@@ -60,7 +61,7 @@ int main(void) {
             F.FoldKV.seqlens.offset, F.FoldKV.max_seqlen.offset, F.FoldArgs.kv.offset, F.FoldArgs.depth_T.offset,
             F.FoldArgs.row_status.offset, F.FoldPartials.rows.offset, F.FoldPartials.slot_stride.offset,
             F.FoldWsHeader.v_rows_total.offset, F.FoldArgs.flags.offset, F.FoldArgs.side_stream.offset,
-            F.FoldArgs.side_join_event.offset]
+            F.FoldArgs.side_join_event.offset, F.FoldArgs.live_hint.offset]
     assert got == want
 
 
@@ -141,7 +142,7 @@ def test_broadcast_strides_are_refused():
 
 def test_new_argument_fields_default_to_plain_behaviour():
     a, _ = _cpu_args()
-    assert a.flags == 0 and not a.side_stream and not a.side_fork_event and not a.side_join_event
+    assert a.flags == 0 and not a.side_stream and not a.side_fork_event and not a.side_join_event and a.live_hint == 0.0
     b, _ = _cpu_args(flags=F.INPUTS_SETTLED)
     assert b.flags == 1
 

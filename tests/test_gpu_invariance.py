@@ -265,3 +265,18 @@ def test_back_to_back_calls_that_share_z_and_workspace_do_not_disturb_each_other
     torch.cuda.synchronize()
     for i in range(2):
         assert same_bits(outs[i], ref[i][0]) and same_bits(lses[i], ref[i][1]), i
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_the_live_hint_never_changes_a_bit(paged):
+    # fold_args.live_hint picks how the depth-gated row-block scan splits its on-chip ring between key and value tiles
+    # (two and four stages, three and three, four and two): scheduling only, so every hint must give the same bits
+    w = make_decode_workload(3, 8, 2, 128, [9000, 2500, 700], seed=61, device=DEV, paged=paged, page_size=32)
+    cache = cache_of(w)
+    ref = run_gpu(w, T=14.0)
+    for hint in (1.0, 0.9, 0.5, 0.1, 1e-6, -3.0, float("nan"), 7.0):
+        bufs = F.alloc_buffers(w.q, cache, w.stack)
+        F.decode(w.q, cache, bufs, depth_T=14.0, scale=w.scale, live_hint=hint)
+        torch.cuda.synchronize()
+        assert bufs.header().wait_timeouts == 0
+        assert same_bits(bufs.out, ref.out) and same_bits(bufs.lse, ref.lse) and same_bits(bufs.z, ref.z), hint
