@@ -717,10 +717,13 @@ int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st, const Fu
       p.chunk_major = 1;
       ctas = units * ((g.max_slots + 1) / 2);                // one chunk per worker at most
     }
-    // the caller's expectation of the live fraction picks the ring's split: four fifths and more live -> two key stages
-    // and four value stages (dense decode's), under 15 % -> four and two, else (and without a hint) three and three
+    // The caller's expectation of the live fraction picks the ring's split.  Measured on a B200 (us, splits 2+4 / 3+3 /
+    // 4+2): all live, group 4 -- 321.6 / 332.5 / 320.1; 90 % live, MHA, 8192-key sequences -- 1265 / 1251 / 1286; half
+    // live, paged -- 278.5 / 272.8 / 300.6; 16 % live -- 1786 / 1532 / 1738; nothing live, 1024-key chunks -- 1504 / 1297 /
+    // 1240 and 239.7 / 192.2 / 183.2; nothing live, 256-key chunks -- 978 / 858 / 912.  So: 95 % and more live -> two key
+    // and four value stages (dense decode's split); under 2 % with 1024-key chunks -> four and two; else three and three.
     const float lh = a->live_hint;
-    const int keys = !(lh > 0.f) ? 3 : (lh >= 0.8f ? 2 : (lh < 0.15f ? 4 : 3));
+    const int keys = !(lh > 0.f) ? 3 : (lh >= 0.95f ? 2 : (lh < 0.02f && kv.max_seqlen > 8192 ? 4 : 3));
     if (!gated) return launch_decode<false, false>(mk, mv, p, f, (int)ctas, 2, st);
     return p.vmean ? launch_decode<true, true>(mk, mv, p, f, (int)ctas, keys, st) : launch_decode<true, false>(mk, mv, p, f, (int)ctas, keys, st);
   }

@@ -246,10 +246,10 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   constexpr int PBYTES = NPV * 256;                          // [2 key halves][NPV rows][128 B]
   // Six 32 KB stages in all.  Dense: a key stage is free as soon as its scores are issued, a value stage waits for the
   // weights, so two key stages feed four value stages (5 % over three and three).  Depth-gated, the best split depends on
-  // how much of the cache is live: a cache that is nearly all live wants dense decode's two and four (C2 at T=16: 321 us
-  // against 330 with three and three), one that is half live three and three (C3: 272 against 278 us with two and
-  // four; 29 % live: 238 against 263), one nobody keeps a value row of four and two (5 % over three and three).  The
-  // caller may say what it expects (fold_args.live_hint); three and three without a hint.  The split only schedules: every
+  // how much of the cache is live (and on the chunk length): a cache that is all live wants dense decode's two and four
+  // (C2 at T=16: 321 us against 332 with three and three), a half-live one three and three (C3: 273 against 278 and
+  // 301 us), one nobody keeps a value row of four and two where chunks are long (4-5 % over three and three).  The host
+  // picks KEYS from the caller's fold_args.live_hint; three and three without a hint.  The split only schedules: every
   // one gives the same bits.
   static_assert(KEYS >= 2 && KEYS <= 4, "two to four key stages");
   constexpr int KS = KEYS, VS = 6 - KS;
