@@ -458,6 +458,10 @@ int sm_count() {
     return 148;
   return n;
 }
+bool cooperative_launch_supported() {
+  int dev = 0, v = 0;
+  return cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v != 0;
+}
 // f.mode != 0: the whole decode in this launch, which is then a cooperative one (its CTAs meet at a grid-wide barrier
 // between the scan and the partial add; the grid is one CTA per SM at most, so all of them are resident).
 template <bool GATED, int NC, bool TAIL, int KEYS>
@@ -647,7 +651,7 @@ bool one_launch_decode(const fold_args *a, const Geometry &g) {
   const long long entries = (long long)g.num_seqs * g.Hkv * ((g.max_slots + 1) & ~1);   // chunk-major list, even per unit
   if (entries > 2LL * sm_count()) return false;
   if (a->num_splits > 0 && a->num_splits < g.max_slots) return false;   // a split hint that bounds the grid: honour it
-  return true;
+  return cooperative_launch_supported();
 }
 
 int launch_scan(const fold_args *a, const Geometry &g, cudaStream_t st, const FusedParams *fused = nullptr) {
