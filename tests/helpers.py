@@ -48,7 +48,7 @@ def oracle_block_means(w: DecodeWorkload) -> torch.Tensor:
 
 
 def run_gpu(w: DecodeWorkload, T=math.inf, z_mode=F.Z_ESTIMATE, num_splits=0, z=None, bufs=None, v_block_mean=None,
-            draft=None):
+            draft=None, live_hint=0.0):
     """`draft` = (masks int32 [batch], draft_len): draft / tree-verification rows."""
     cache = cache_of(w, v_block_mean)
     if bufs is None:
@@ -56,7 +56,8 @@ def run_gpu(w: DecodeWorkload, T=math.inf, z_mode=F.Z_ESTIMATE, num_splits=0, z=
     if z is not None:
         bufs.z.copy_(z)
     F.decode(w.q, cache, bufs, depth_T=T, z_mode=z_mode, num_splits=num_splits, stack=w.stack, scale=w.scale,
-             draft_mask=None if draft is None else draft[0], draft_len=0 if draft is None else draft[1])
+             draft_mask=None if draft is None else draft[0], draft_len=0 if draft is None else draft[1],
+             live_hint=live_hint)
     torch.cuda.synchronize()
     assert bufs.header().wait_timeouts == 0
     return bufs
