@@ -551,6 +551,8 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       }
     }
     unsigned long long st_fetched = 0, st_total = 0, st_skipped = 0;
+    const int cut_exp = 24 + min(max((int)floorf(-p.neg_T), 0), 96);   // block tail: the cut mass's integer grid
+    const float cut_scale = __int_as_float((127 + cut_exp) << 23), cut_unscale = __int_as_float((127 - cut_exp) << 23);
     const uint64_t vpol = policy_evict_first();
     const int vbox = p.vr;                                   // tokens per value box (16 or 32)
     const uint32_t gmask = vbox == 32 ? 0xffffffffu : 0xffffu;
@@ -571,16 +573,16 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         // in the order of the key rows: lane quarters 0, 1, 2, 3
         if (lane < p.R) slot[(long long)p.R * D + lane] = ((lp[lane] + lp[16 + lane]) + lp[32 + lane]) + lp[48 + lane];
       }
-      // block tail: this channel of the chunk's block means (up to 16 blocks), requested before the waits below
-      float mean[16];
+      // block tail: this channel of the chunk's block means (up to 16 blocks), requested before the waits below -- as raw
+      // bits from clamped block indices, converted and masked only where they are used: a select or a conversion right
+      // behind each load would wait for it, sixteen memory latencies in a row
+      unsigned short mraw[16];
+      const int nblocks = TAIL ? (pend.n + 63) >> 6 : 1;
       if (TAIL) {
-        const int nblocks = (pend.n + 63) >> 6;
-        const __nv_bfloat16 *mrow = p.vmean + (long long)pend.seq * p.vm_stride_seq + (long long)pend.kvh * p.vm_stride_head + krow;
+        const unsigned short *mrow = reinterpret_cast<const unsigned short *>(p.vmean) + (long long)pend.seq * p.vm_stride_seq +
+                                     (long long)pend.kvh * p.vm_stride_head + krow;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int bi = pend.t_first * 2 + j;
-          mean[j] = (j < 2 * (pend.t_end - pend.t_first) && bi < nblocks) ? __bfloat162float(mrow[(long long)bi * p.vm_stride_block]) : 0.f;
-        }
+        for (int j = 0; j < 16; ++j) mraw[j] = mrow[(long long)min(pend.t_first * 2 + j, nblocks - 1) * p.vm_stride_block];
       }
       if (!wait_u(bar(kDecBarPFree + 2 * set + (pend_i % PB)), (uint32_t)((pend_i / PB) & 1))) return;   // the chunk's last product
       tc_fence_after();
@@ -596,9 +598,11 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const float *cp = cutp + par * 256;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
+          const bool there = j < 2 * (pend.t_end - pend.t_first) && pend.t_first * 2 + j < nblocks;
+          const float mean = there ? __uint_as_float((uint32_t)mraw[j] << 16) : 0.f;
 #pragma unroll
           for (int r = 0; r < NC; ++r)
-            tl[r] = fmaf(cp[(j * 2) * 8 + r] + cp[(j * 2 + 1) * 8 + r], mean[j], tl[r]);
+            tl[r] = fmaf(cp[(j * 2) * 8 + r] + cp[(j * 2 + 1) * 8 + r], mean, tl[r]);
         }
       }
 #pragma unroll
@@ -725,11 +729,12 @@ fold_scan_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           L[r] += (h + g) + (pw - pm);                       // L sums the weights the products use; cut keys add p
           hi16[r] = __float_as_uint(h) >> 16;
           lo16[r] = __float_as_uint(g) >> 16;
-          if (TAIL) {                                        // the warp's cut mass of row r in this tile (fixed shuffle order)
-            float c = pw - pm;
-#pragma unroll
-            for (int m = 16; m >= 1; m >>= 1) c += __shfl_xor_sync(0xffffffffu, c, m);
-            if (lane == 0) cutp[(((e & 1) * 8 + (cur.t - cur.t_first)) * 4 + qd) * 8 + r] = c;
+          if (TAIL) {
+            // the warp's cut mass of row r in this tile: a cut weight is below 2^-T, so on the grid 2^-(24 + floor T) it is
+            // an integer under 2^24 and the warp's 32 add up in ONE order-free integer reduction (five dependent shuffles
+            // per row and tile sat on the weight warps' critical chain); weights under half a grid step count as zero
+            const int ci = __reduce_add_sync(0xffffffffu, __float2int_rn((pw - pm) * cut_scale));
+            if (lane == 0) cutp[(((e & 1) * 8 + (cur.t - cur.t_first)) * 4 + qd) * 8 + r] = (float)ci * cut_unscale;
           }
         }
         // the worker's weight buffer is free once its own value product PB tiles back is over
