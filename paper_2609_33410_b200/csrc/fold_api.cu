@@ -1244,7 +1244,7 @@ const char *fold_status_string(int status) {
   }
 }
 
-int fold_version(void) { return 100; }
+int fold_version(void) { return 102; }   // 101: flags, side stream, fold_probe_read; 102: fold_decode_launches, live_hint
 
 
 }  // extern "C"
