@@ -444,8 +444,8 @@ def main():
             torch.cuda.synchronize()
         quant_ms = None
         if args.planes:
-            if cascade or args.drafts > 4:
-                raise SystemExit("--planes: one level, at most 8 rows per kv head (no cascade; drafts x group <= 8)")
+            if cascade or levels[0].stack * (levels[0].num_q_heads // levels[0].num_kv_heads) > 16:
+                raise SystemExit("--planes: one level, at most 16 rows per kv head (no cascade; drafts x group <= 16)")
             F.fold_quantize_keys(caches[0], None, stream)                   # allocates the planes, warms the kernel
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)

@@ -127,8 +127,8 @@ enum {
  * capacity (page_size).  With planes, k may be NULL for the decode calls; v stays BF16.  Each scan scores every
  * key against plane A alone (head_dim + 2 bytes per key), ORs the verdicts over the rows that share the kv head,
  * and only then requests plane B rows (refined keys) and value rows (live keys).  This path takes row blocks of
- * at most 8 rows (stack * group <= 8, draft rows included) and one level (no cascade), with or without the block
- * tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED.
+ * at most 16 rows (stack * group <= 16, draft rows included; the verdicts are ORed over all of them) and one level
+ * (no cascade), with or without the block tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED.
  *
  * Two E4M3 value planes (Section 4, "Cache format": two FP8 planes that share one power-of-two scale per layer; only
  * together with the two-plane keys).  When v_plane_1 is not NULL the scan reads values from

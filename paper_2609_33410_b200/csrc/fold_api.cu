@@ -116,8 +116,8 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   g->ws_bytes = g->planes ? g->q_off + qplane_bytes((long long)g->B * g->Hq, g->D) : kHeaderBytes + g->slot_bytes;
   if (g->planes) {
     if (isnan(a->refine_tau)) return FOLD_EINVAL;
-    // the two-plane scan: one 8-row block, no exact-maximum pass
-    if (R > kNarrowRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
+    // the two-plane scan: one block of up to 16 rows (its verdicts are the group's), no exact-maximum pass
+    if (R > kMaxRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
     if (a->kv.v_plane_1 && isnan(a->refine_tau_v)) return FOLD_EINVAL;
   }
   return FOLD_OK;
@@ -557,8 +557,8 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
 }
 
 // As many plane-A stages as fit beside the gather buffers with kPlaneCtasPerSm CTAs on an SM.
-template <int D, bool DRAFTS, bool TAIL, bool VFP8 = false>
-int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
+template <int D, bool DRAFTS, bool TAIL, bool VFP8, int NT>
+int launch_planes_nt(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
   using LO = PlaneLayout<D, TAIL>;
   const int per_cta = kSmemPerSm / kPlaneCtasPerSm - kSmemCtaReserve;
   int stages = (per_cta - LO::total(0)) / (LO::kStage + 16);
@@ -566,11 +566,17 @@ int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanPara
   if (stages < 2) return FOLD_EUNSUPPORTED;
   pp.s.stages = stages;
   static SmemFlags configured;
-  if (int rc = opt_in_smem(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8>, configured)) return rc;
-  if (launch_pdl(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) !=
+  if (int rc = opt_in_smem(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8, NT>, configured)) return rc;
+  if (launch_pdl(fold_scan_planes_kernel<D, DRAFTS, TAIL, VFP8, NT>, grid, dim3(kDenseThreads), LO::total(stages), st, ma, mv, pp) !=
       cudaSuccess)
     return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+// up to 8 rows per (sequence, kv head): one 8-row tile; 9 to 16: two
+template <int D, bool DRAFTS, bool TAIL, bool VFP8 = false>
+int launch_planes_as(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {
+  return pp.s.R <= kNarrowRows ? launch_planes_nt<D, DRAFTS, TAIL, VFP8, 1>(ma, mv, pp, grid, st)
+                               : launch_planes_nt<D, DRAFTS, TAIL, VFP8, 2>(ma, mv, pp, grid, st);
 }
 template <int D>
 int launch_planes_kernel(const CUtensorMap &ma, const CUtensorMap &mv, PlaneScanParams &pp, dim3 grid, cudaStream_t st) {

@@ -368,22 +368,29 @@ __device__ __forceinline__ void mma_s8(int (&c)[4], const uint32_t (&a)[4], uint
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// c^xa, c^xb [16 keys, 8 rows] = plane X of 16 keys (rows key0.. of the tile at `tile`) times [Q^a; Q^b]^T.
+// c^xa, c^xb [16 keys, 8 rows] (per row tile) = plane X of 16 keys (rows key0.. of the tile at `tile`) times [Q^a; Q^b]^T.
 // c[0], c[1]: key lane/4, rows (lane%4)*2 + {0,1};  c[2], c[3]: key lane/4 + 8.
-template <int D>
-__device__ __forceinline__ void plane_products(uint32_t tile, int key0, int lane, const uint32_t (&qa)[D / 32][2],
-                                               const uint32_t (&qb)[D / 32][2], int (&ca)[4], int (&cb)[4]) {
+// NT 8-row tiles of query rows (rows 8 q + ...): one ldmatrix of the key slice feeds every tile's products.
+template <int D, int NT>
+__device__ __forceinline__ void plane_products(uint32_t tile, int key0, int lane, const uint32_t (&qa)[NT][D / 32][2],
+                                               const uint32_t (&qb)[NT][D / 32][2], int (&ca)[NT][4], int (&cb)[NT][4]) {
   // ldmatrix matrix i = lane/8: keys (i&1)*8 + lane%8, 16-byte chunk 2*kk + (i>>1)
   const int key = key0 + (((lane >> 3) & 1) << 3) + (lane & 7);
-  ca[0] = ca[1] = ca[2] = ca[3] = 0;
-  cb[0] = cb[1] = cb[2] = cb[3] = 0;
+#pragma unroll
+  for (int q = 0; q < NT; ++q) {
+    ca[q][0] = ca[q][1] = ca[q][2] = ca[q][3] = 0;
+    cb[q][0] = cb[q][1] = cb[q][2] = cb[q][3] = 0;
+  }
 #pragma unroll
   for (int kk = 0; kk < D / 32; ++kk) {
     uint32_t a[4];
     const int ch = 2 * kk + (lane >> 4);
     ldsm_x4(tile + plane_off<D>(key, ch), a[0], a[1], a[2], a[3]);
-    mma_s8(ca, a, qa[kk][0], qa[kk][1]);
-    mma_s8(cb, a, qb[kk][0], qb[kk][1]);
+#pragma unroll
+    for (int q = 0; q < NT; ++q) {
+      mma_s8(ca[q], a, qa[q][kk][0], qa[q][kk][1]);
+      mma_s8(cb[q], a, qb[q][kk][0], qb[q][kk][1]);
+    }
   }
 }
 
@@ -438,8 +445,9 @@ __device__ __forceinline__ void produce_plane_tiles(const CUtensorMap *tmA, cons
 }
 
 // One sub-slice (16 keys) between its coarse pass and its second pass.
+template <int NT>
 struct PlanePending {
-  float x[4];            // coarse score minus reference: key lane/4 (+8), rows (lane%4)*2 + {0,1}; -inf if unused
+  float x[NT][4];        // coarse score minus reference: key lane/4 (+8), rows 8 q + (lane%4)*2 + {0,1}; -inf if unused
   float e[2];            // the two keys' scales
   uint32_t live, refine; // verdict bits of the 16 keys, ORed over the rows
   uint32_t refv;         // E4M3 value planes: keys whose second value plane is read
@@ -450,8 +458,10 @@ struct PlanePending {
 // DRAFTS: the rows carry draft masks (a separate instantiation: the plain one is at its register limit).
 // TAIL: cut keys add weight x the mean value row of their 64-key block (Section 4, "Depth as a dial").
 // VFP8: values come from two E4M3 planes (plane 1 for live keys, plane 2 for refine-V keys), widened to BF16 in place.
-template <int D, bool DRAFTS, bool TAIL, bool VFP8 = false>
-__global__ void __launch_bounds__(kDenseThreads, kPlaneCtasPerSm)
+// NT = 2: 9 to 16 rows per (sequence, kv head) as two 8-row tiles (one ldmatrix feeds both tiles' products; the verdicts
+// are ORed over all the rows, as Algorithm 1 takes them over the group); the accumulators double, two CTAs per SM.
+template <int D, bool DRAFTS, bool TAIL, bool VFP8 = false, int NT = 1>
+__global__ void __launch_bounds__(kDenseThreads, NT == 1 ? kPlaneCtasPerSm : 2)
 fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmV,
                         const PlaneScanParams pp) {
   using LO = PlaneLayout<D, TAIL>;
@@ -489,42 +499,49 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   pdl_wait();                                                // z and the split query rows come from the kernel before
 
   // query rows: B fragments of the INT8 products (row lane/4), scales and references of the score rows
-  uint32_t qa[D / 32][2], qb[D / 32][2];
-  {
-    const int r = lane >> 2;
+  uint32_t qa[NT][D / 32][2], qb[NT][D / 32][2];
+#pragma unroll
+  for (int q = 0; q < NT; ++q) {
+    const int r = 8 * q + (lane >> 2);
     const bool ok = r < R;
     const int req = seq * p.stack + r / p.G, head = kvh * p.G + r % p.G;
     const int8_t *qp = pp.qplanes + ((long long)req * p.Hq + head) * (2 * D) + (lane & 3) * 4;
 #pragma unroll
     for (int kk = 0; kk < D / 32; ++kk) {
-      qa[kk][0] = ok ? *reinterpret_cast<const uint32_t *>(qp + kk * 32) : 0u;
-      qa[kk][1] = ok ? *reinterpret_cast<const uint32_t *>(qp + kk * 32 + 16) : 0u;
-      qb[kk][0] = ok ? *reinterpret_cast<const uint32_t *>(qp + D + kk * 32) : 0u;
-      qb[kk][1] = ok ? *reinterpret_cast<const uint32_t *>(qp + D + kk * 32 + 16) : 0u;
+      qa[q][kk][0] = ok ? *reinterpret_cast<const uint32_t *>(qp + kk * 32) : 0u;
+      qa[q][kk][1] = ok ? *reinterpret_cast<const uint32_t *>(qp + kk * 32 + 16) : 0u;
+      qb[q][kk][0] = ok ? *reinterpret_cast<const uint32_t *>(qp + D + kk * 32) : 0u;
+      qb[q][kk][1] = ok ? *reinterpret_cast<const uint32_t *>(qp + D + kk * 32 + 16) : 0u;
     }
   }
-  float eta[2], zr[2];
-  uint32_t dm[2];                                            // the rows' requests' draft masks (all ones without drafts)
-  bool rv[2];
+  float eta[NT][2], zr[NT][2];
+  uint32_t dm[NT][2];                                        // the rows' requests' draft masks (all ones without drafts)
+  bool rv[NT][2];
 #pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    const int r = (lane & 3) * 2 + e;
-    rv[e] = r < R;
-    const int req = seq * p.stack + r / p.G;
-    const long long row = (long long)req * p.Hq + kvh * p.G + r % p.G;
-    eta[e] = rv[e] ? pp.qeta[row] : 0.f;
-    zr[e] = rv[e] ? p.z[row] : 0.f;
-    dm[e] = (DRAFTS && rv[e]) ? p.draft_mask[req] : 0xffffffffu;
-  }
+  for (int q = 0; q < NT; ++q)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int r = 8 * q + (lane & 3) * 2 + e;
+      rv[q][e] = r < R;
+      const int req = seq * p.stack + r / p.G;
+      const long long row = (long long)req * p.Hq + kvh * p.G + r % p.G;
+      eta[q][e] = rv[q][e] ? pp.qeta[row] : 0.f;
+      zr[q][e] = rv[q][e] ? p.z[row] : 0.f;
+      dm[q][e] = (DRAFTS && rv[q][e]) ? p.draft_mask[req] : 0xffffffffu;
+    }
   const int dstart = DRAFTS ? draft_start(p, n) : n;         // keys from here on are per-request drafts
   const float neg_T = p.neg_T;
   const float neg_tau = pp.auto_tau ? -fmaxf(log2f((float)max(n, 1)) - 2.f, 4.f) : pp.neg_tau;
   const float neg_tau_v = pp.auto_tau_v ? -fmaxf(log2f((float)max(n, 1)) + 1.f, 4.f) : pp.neg_tau_v;
 
-  float o[D / 16][4];
+  float o[NT][D / 16][4];
+  float l_lo[NT], l_hi[NT];
 #pragma unroll
-  for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-  float l_lo = 0.f, l_hi = 0.f;
+  for (int q = 0; q < NT; ++q) {
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) o[q][i][0] = o[q][i][1] = o[q][i][2] = o[q][i][3] = 0.f;
+    l_lo[q] = l_hi[q] = 0.f;
+  }
   const uint32_t bufs = base + LO::off_bufs(stages) + warp * LO::kWarpBufs;
   float *red = reinterpret_cast<float *>(gen + LO::off_bufs(stages));
   float *redl = reinterpret_cast<float *>(gen + LO::off_redl(stages));
@@ -545,62 +562,77 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   // Block tail: c0 / c1 = this thread's share of the mass rows (lane%4)*2 + {0,1} cut in the sub-slice; the eight lanes that
   // scored the rows' keys are summed, then every channel this thread accumulates takes cut mass x the block's mean value.
   const __nv_bfloat16 *means = reinterpret_cast<const __nv_bfloat16 *>(gen + LO::off_means(stages));
-  auto add_tail = [&](float c0, float c1, int ms) {
+  auto add_tail = [&](float (&c0)[NT], float (&c1)[NT], int ms) {
 #pragma unroll
-    for (int m = 4; m <= 16; m <<= 1) {
-      c0 += __shfl_xor_sync(0xffffffffu, c0, m);
-      c1 += __shfl_xor_sync(0xffffffffu, c1, m);
-    }
+    for (int q = 0; q < NT; ++q)
+#pragma unroll
+      for (int m = 4; m <= 16; m <<= 1) {
+        c0[q] += __shfl_xor_sync(0xffffffffu, c0[q], m);
+        c1[q] += __shfl_xor_sync(0xffffffffu, c1[q], m);
+      }
     const __nv_bfloat16 *mrow = means + ms * D + klo;
 #pragma unroll
     for (int mt = 0; mt < D / 16; ++mt) {
       const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
-      o[mt][0] = fmaf(c0, m0, o[mt][0]); o[mt][1] = fmaf(c1, m0, o[mt][1]);
-      o[mt][2] = fmaf(c0, m1, o[mt][2]); o[mt][3] = fmaf(c1, m1, o[mt][3]);
+#pragma unroll
+      for (int q = 0; q < NT; ++q) {
+        o[q][mt][0] = fmaf(c0[q], m0, o[q][mt][0]); o[q][mt][1] = fmaf(c1[q], m0, o[q][mt][1]);
+        o[q][mt][2] = fmaf(c0[q], m1, o[q][mt][2]); o[q][mt][3] = fmaf(c1[q], m1, o[q][mt][3]);
+      }
     }
   };
   // E4M3 value planes: the mass this thread's two rows cut in the chunk (their share of the sequence's mean value row is
   // added once, at the chunk's end)
-  float rcut0 = 0.f, rcut1 = 0.f;
-  auto finish = [&](const PlanePending &pd) {
+  float rcut0[NT], rcut1[NT];
+#pragma unroll
+  for (int q = 0; q < NT; ++q) rcut0[q] = rcut1[q] = 0.f;
+  auto finish = [&](const PlanePending<NT> &pd) {
     const uint32_t bbuf = bufs + pd.buf * (LO::kBBuf + LO::kVBuf), vbuf = bbuf + LO::kBBuf;
     const bool landed = mbar_wait(gbar_w + 8u * pd.buf, (gphase >> pd.buf) & 1u, dead);
     gphase ^= 1u << pd.buf;
     if (!landed) return;
-    int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
-    if (pd.refine) plane_products<D>(bbuf, 0, lane, qa, qb, ca, cb);
-    uint32_t bh[2], bl[2];
-    float cut0 = 0.f, cut1 = 0.f;
+    int ca[NT][4], cb[NT][4];
 #pragma unroll
-    for (int kh = 0; kh < 2; ++kh) {
-      const bool klive = (pd.live >> (klo + 8 * kh)) & 1u;
-      const bool kref = (pd.refine >> (klo + 8 * kh)) & 1u;   // an unrefined key's buffer row is stale: no correction
-      float pw[2], pm[2];
+    for (int q = 0; q < NT; ++q)
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int i = 2 * kh + e;
-        const float corr = kref ? ((float)ca[i] + (float)cb[i] * 0.00390625f) * 0.00390625f : 0.f;
-        const float x = fmaf(corr, eta[e] * pd.e[kh], pd.x[i]);
-        const bool live = klive && (x >= neg_T);
-        pw[e] = ex2_approx(x);
-        pm[e] = live ? pw[e] : 0.f;
-      }
-      const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
-      const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
-      const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
-      const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
-      l_lo += (h0 + g0) + (pw[0] - pm[0]);
-      l_hi += (h1 + g1) + (pw[1] - pm[1]);
-      if (TAIL || VFP8) { cut0 += pw[0] - pm[0]; cut1 += pw[1] - pm[1]; }
-      if (VFP8) {
-        // E4M3 values enter the product without their power-of-two scale: it multiplies the weights' BF16 terms instead
-        // (exactly: a power of two), while L keeps the weights themselves
-        const float vs = pp.kv.v_scale;
-        bh[kh] = movmatrix_trans(pack_bf16(h0 * vs, h1 * vs));
-        bl[kh] = movmatrix_trans(pack_bf16(g0 * vs, g1 * vs));
-      } else {
-        bh[kh] = movmatrix_trans(hi2);
-        bl[kh] = movmatrix_trans(lo2);
+      for (int i = 0; i < 4; ++i) ca[q][i] = cb[q][i] = 0;
+    if (pd.refine) plane_products<D, NT>(bbuf, 0, lane, qa, qb, ca, cb);
+    uint32_t bh[NT][2], bl[NT][2];
+    float cut0[NT], cut1[NT];
+#pragma unroll
+    for (int q = 0; q < NT; ++q) {
+      cut0[q] = cut1[q] = 0.f;
+#pragma unroll
+      for (int kh = 0; kh < 2; ++kh) {
+        const bool klive = (pd.live >> (klo + 8 * kh)) & 1u;
+        const bool kref = (pd.refine >> (klo + 8 * kh)) & 1u;   // an unrefined key's buffer row is stale: no correction
+        float pw[2], pm[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int i = 2 * kh + e;
+          const float corr = kref ? ((float)ca[q][i] + (float)cb[q][i] * 0.00390625f) * 0.00390625f : 0.f;
+          const float x = fmaf(corr, eta[q][e] * pd.e[kh], pd.x[q][i]);
+          const bool live = klive && (x >= neg_T);
+          pw[e] = ex2_approx(x);
+          pm[e] = live ? pw[e] : 0.f;
+        }
+        const uint32_t hi2 = pack_bf16(pm[0], pm[1]);
+        const float h0 = __uint_as_float(hi2 << 16), h1 = __uint_as_float(hi2 & 0xffff0000u);
+        const uint32_t lo2 = pack_bf16(pm[0] - h0, pm[1] - h1);
+        const float g0 = __uint_as_float(lo2 << 16), g1 = __uint_as_float(lo2 & 0xffff0000u);
+        l_lo[q] += (h0 + g0) + (pw[0] - pm[0]);
+        l_hi[q] += (h1 + g1) + (pw[1] - pm[1]);
+        if (TAIL || VFP8) { cut0[q] += pw[0] - pm[0]; cut1[q] += pw[1] - pm[1]; }
+        if (VFP8) {
+          // E4M3 values enter the product without their power-of-two scale: it multiplies the weights' BF16 terms instead
+          // (exactly: a power of two), while L keeps the weights themselves
+          const float vs = pp.kv.v_scale;
+          bh[q][kh] = movmatrix_trans(pack_bf16(h0 * vs, h1 * vs));
+          bl[q][kh] = movmatrix_trans(pack_bf16(g0 * vs, g1 * vs));
+        } else {
+          bh[q][kh] = movmatrix_trans(hi2);
+          bl[q][kh] = movmatrix_trans(lo2);
+        }
       }
     }
     if (VFP8 && pd.live) {
@@ -643,15 +675,21 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
       }
       __syncwarp();
     }
-    if (pd.live) value_product_n<D, true, 0, 16>(o, vbuf, 0, lane, bh, bl);
-    if (TAIL) add_tail(cut0, cut1, pd.ms);
-    if (VFP8) { rcut0 += cut0; rcut1 += cut1; }
+    if (pd.live) {
+      if constexpr (NT == 1) value_product_n<D, true, 0, 16>(o[0], vbuf, 0, lane, bh[0], bl[0]);
+      else value_product_nt<D, 16, NT>(o, vbuf, 0, lane, bh, bl, 0u);
+    }
+    if (VFP8) {
+#pragma unroll
+      for (int q = 0; q < NT; ++q) { rcut0[q] += cut0[q]; rcut1[q] += cut1[q]; }
+    }
+    if (TAIL) add_tail(cut0, cut1, pd.ms);                   // (sums the cut mass over the lanes in place)
   };
 
   int stage = 0, buf = 0, n_pend = 0, mslot = 0;
   uint32_t phase = 0;
   unsigned long long st_total = 0, st_live = 0, st_ref = 0, st_refv = 0;
-  PlanePending pend[LO::kBufs - 1];
+  PlanePending<NT> pend[LO::kBufs - 1];
   const int page_mask = (1 << p.page_shift) - 1;
   const uint64_t vpol = policy_evict_first();
 
@@ -672,25 +710,27 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         if (key0 >= n) continue;                              // warp-uniform
         st_total += min(16, n - key0);
         // coarse pass: plane A against both query planes
-        PlanePending cur;
-        int ca[4], cb[4];
-        plane_products<D>(at, sub * 16, lane, qa, qb, ca, cb);
+        PlanePending<NT> cur;
+        int ca[NT][4], cb[NT][4];
+        plane_products<D, NT>(at, sub * 16, lane, qa, qb, ca, cb);
         uint32_t lm = 0, rm = 0, vm = 0;
 #pragma unroll
         for (int kh = 0; kh < 2; ++kh) {
           const int key = key0 + klo + 8 * kh;
           cur.e[kh] = key < n ? __bfloat162float(scales[sub * 16 + klo + 8 * kh]) : 0.f;
 #pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int i = 2 * kh + e;
-            const bool ok = key < n && rv[e] && (!DRAFTS || draft_ok(dm[e], key, dstart));   // an unused draft key: -inf
-            const float f = (float)ca[i] + (float)cb[i] * 0.00390625f;
-            const float x = ok ? fmaf(f, eta[e] * cur.e[kh], -zr[e]) : -INFINITY;
-            cur.x[i] = x;
-            if (ok && x >= neg_T) lm |= 1u << (klo + 8 * kh);
-            if (ok && x >= neg_tau) rm |= 1u << (klo + 8 * kh);
-            if (VFP8 && ok && x >= neg_tau_v) vm |= 1u << (klo + 8 * kh);
-          }
+          for (int q = 0; q < NT; ++q)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int i = 2 * kh + e;
+              const bool ok = key < n && rv[q][e] && (!DRAFTS || draft_ok(dm[q][e], key, dstart));   // an unused draft key: -inf
+              const float f = (float)ca[q][i] + (float)cb[q][i] * 0.00390625f;
+              const float x = ok ? fmaf(f, eta[q][e] * cur.e[kh], -zr[q][e]) : -INFINITY;
+              cur.x[q][i] = x;
+              if (ok && x >= neg_T) lm |= 1u << (klo + 8 * kh);
+              if (ok && x >= neg_tau) rm |= 1u << (klo + 8 * kh);
+              if (VFP8 && ok && x >= neg_tau_v) vm |= 1u << (klo + 8 * kh);
+            }
         }
         cur.live = __reduce_or_sync(0xffffffffu, lm);
         cur.refine = __reduce_or_sync(0xffffffffu, rm) & cur.live;
@@ -703,15 +743,19 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         if (cur.live == 0u) {
           // every key of the sub-slice is cut for every row: no bytes are asked for, nothing is queued, and the weights
           // (the coarse scores are all this scan will ever have for these keys) only add to L
-          float cut0 = 0.f, cut1 = 0.f;
+          float cut0[NT], cut1[NT];
 #pragma unroll
-          for (int kh = 0; kh < 2; ++kh) {
-            cut0 += ex2_approx(cur.x[2 * kh]);
-            cut1 += ex2_approx(cur.x[2 * kh + 1]);
+          for (int q = 0; q < NT; ++q) {
+            cut0[q] = cut1[q] = 0.f;
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+              cut0[q] += ex2_approx(cur.x[q][2 * kh]);
+              cut1[q] += ex2_approx(cur.x[q][2 * kh + 1]);
+            }
+            l_lo[q] += cut0[q];
+            l_hi[q] += cut1[q];
+            if (VFP8) { rcut0[q] += cut0[q]; rcut1[q] += cut1[q]; }
           }
-          l_lo += cut0;
-          l_hi += cut1;
-          if (VFP8) { rcut0 += cut0; rcut1 += cut1; }
           if (TAIL) {
             add_tail(cut0, cut1, my_ms);
             // a queued sub-slice must be finished while its tile's mean row is still in the ring (stages + 1 slots):
@@ -814,26 +858,34 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     n_pend = 0;
     if (VFP8) {
       if (pp.vrun) {                                          // cut mass x the sequence's mean value row (the 8-bit cut model)
-        float c0 = rcut0, c1 = rcut1;
-#pragma unroll
-        for (int m = 4; m <= 16; m <<= 1) {
-          c0 += __shfl_xor_sync(0xffffffffu, c0, m);
-          c1 += __shfl_xor_sync(0xffffffffu, c1, m);
-        }
         const __nv_bfloat16 *mrow = pp.vrun + (long long)seq * pp.vrun_stride_seq + (long long)kvh * pp.vrun_stride_head + klo;
 #pragma unroll
-        for (int mt = 0; mt < D / 16; ++mt) {
-          const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
-          o[mt][0] = fmaf(c0, m0, o[mt][0]); o[mt][1] = fmaf(c1, m0, o[mt][1]);
-          o[mt][2] = fmaf(c0, m1, o[mt][2]); o[mt][3] = fmaf(c1, m1, o[mt][3]);
+        for (int q = 0; q < NT; ++q) {
+          float c0 = rcut0[q], c1 = rcut1[q];
+#pragma unroll
+          for (int m = 4; m <= 16; m <<= 1) {
+            c0 += __shfl_xor_sync(0xffffffffu, c0, m);
+            c1 += __shfl_xor_sync(0xffffffffu, c1, m);
+          }
+#pragma unroll
+          for (int mt = 0; mt < D / 16; ++mt) {
+            const float m0 = __bfloat162float(mrow[mt * 16]), m1 = __bfloat162float(mrow[mt * 16 + 8]);
+            o[q][mt][0] = fmaf(c0, m0, o[q][mt][0]); o[q][mt][1] = fmaf(c1, m0, o[q][mt][1]);
+            o[q][mt][2] = fmaf(c0, m1, o[q][mt][2]); o[q][mt][3] = fmaf(c1, m1, o[q][mt][3]);
+          }
         }
       }
-      rcut0 = rcut1 = 0.f;
+#pragma unroll
+      for (int q = 0; q < NT; ++q) rcut0[q] = rcut1[q] = 0.f;
     }
     named_bar(1, kConsumerWarps * 32);                        // every warp's buffers are drained: park there
     float *slot = p.slots + (((long long)seq * p.Hkv + kvh) * p.max_slots + c) * p.slot_stride;
-    reduce_store_L_n<kConsumerWarps>(l_lo, l_hi, redl, slot + R * D, R, warp, lane, threadIdx.x, 1);
-    reduce_store_A_n<D, kConsumerWarps>(o, red, slot, R, warp, lane, threadIdx.x, 1);
+#pragma unroll
+    for (int q = 0; q < NT; ++q) {                            // a tile's rows: 8 q .. 8 q + 7, as many as the block has
+      const int Rq = min(8, R - 8 * q);
+      reduce_store_L_n<kConsumerWarps>(l_lo[q], l_hi[q], redl, slot + R * D + 8 * q, Rq, warp, lane, threadIdx.x, 1);
+      reduce_store_A_n<D, kConsumerWarps>(o[q], red, slot + 8 * q * D, Rq, warp, lane, threadIdx.x, 1);
+    }
     if (c + p.num_splits < w.n_chunks) clear_bufs();
   }
 

@@ -276,7 +276,9 @@ def test_edge_lengths(D, n):
     compare_planes(w, cache, run_planes(w, cache, T=4.0, tau=2.0), T=4.0, tau=2.0)
 
 
-@pytest.mark.parametrize("Hq,Hkv,stack", [(1, 1, 1), (8, 8, 1), (4, 2, 1), (8, 1, 1), (8, 2, 2), (2, 2, 4), (3, 1, 2)])
+@pytest.mark.parametrize("Hq,Hkv,stack", [(1, 1, 1), (8, 8, 1), (4, 2, 1), (8, 1, 1), (8, 2, 2), (2, 2, 4), (3, 1, 2),
+                                          # 9 to 16 rows per (sequence, kv head): two 8-row tiles, verdicts over all of them
+                                          (16, 1, 1), (9, 1, 1), (24, 2, 1), (8, 2, 4), (3, 1, 5), (4, 2, 7), (13, 1, 1)])
 def test_group_and_stack_shapes(Hq, Hkv, stack):
     w = make_decode_workload(2 * stack, Hq, Hkv, 128, [700, 300], seed=47, device=DEV, stack=stack)
     cache = plane_cache(w)
@@ -344,10 +346,10 @@ def test_empty_sequences_and_unsupported_shapes():
     cache = plane_cache(w)
     compare_planes(w, cache, run_planes(w, cache))
     compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0)
-    wide = make_decode_workload(1, 16, 1, 128, [300], seed=73, device=DEV)              # 16 rows: beyond the two-plane scan
+    wide = make_decode_workload(5, 4, 1, 128, [300], seed=73, device=DEV, stack=5)      # 20 rows: beyond the two-plane scan
     c2 = plane_cache(wide)
-    bufs = F.alloc_buffers(wide.q, cache_of(wide))
-    a = F.make_args(wide.q, c2, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse)
+    bufs = F.alloc_buffers(wide.q, cache_of(wide), 5)
+    a = F.make_args(wide.q, c2, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, stack=5)
     assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
     a = F.make_args(w.q, cache, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, z_mode=F.Z_EXACT_MAX)
     assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
@@ -423,13 +425,14 @@ PLANE_LENGTHS = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255
 
 @pytest.mark.parametrize("seed", range(5))
 def test_random_shapes_match_the_oracle(seed):
-    """Seeded random shapes of the two-plane path: head dimension, rows per kv head (1..8), lengths around every tile /
+    """Seeded random shapes of the two-plane path: head dimension, rows per kv head (1..16), lengths around every tile /
     chunk / estimator boundary, paged or contiguous, depth, refine gates, block tail, draft masks and E4M3 value planes drawn together."""
     import random
     rnd = random.Random(7300 + seed)
     for i in range(8):
         D = rnd.choice([64, 128])
-        G, stack = rnd.choice([(1, 1), (2, 1), (3, 1), (4, 1), (8, 1), (5, 1), (1, 3), (2, 4), (4, 2), (1, 8), (2, 2)])
+        G, stack = rnd.choice([(1, 1), (2, 1), (3, 1), (4, 1), (8, 1), (5, 1), (1, 3), (2, 4), (4, 2), (1, 8), (2, 2),
+                               (16, 1), (9, 1), (4, 4), (2, 7), (3, 5), (1, 13), (12, 1)])
         Hkv = rnd.choice([1, 2, 3])
         nseq = rnd.choice([1, 2, 3])
         lens = [rnd.choice(PLANE_LENGTHS) for _ in range(nseq)]
@@ -485,7 +488,8 @@ def test_static_scratch_entry_point_takes_two_plane_keys():
     assert same_bits(out, ref.out) and same_bits(lse, ref.lse) and same_bits(z, ref.z) and not st.any()
 
 
-@pytest.mark.parametrize("Hq,Hkv,m,tree", [(8, 2, 2, False), (4, 2, 4, True), (2, 2, 8, False), (3, 1, 2, True)])
+@pytest.mark.parametrize("Hq,Hkv,m,tree", [(8, 2, 2, False), (4, 2, 4, True), (2, 2, 8, False), (3, 1, 2, True),
+                                           (8, 2, 4, True), (2, 1, 7, False)])          # 16 and 14 rows: two row tiles
 def test_draft_rows_on_two_plane_keys(Hq, Hkv, m, tree):
     from paper_2609_33410_b200.workloads import make_draft_workload
     w, masks, m = make_draft_workload(2, m, Hq, Hkv, 128, [700, 190], seed=97, device=DEV, tree=tree, poison_padding=True)
