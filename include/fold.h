@@ -127,8 +127,11 @@ enum {
  * capacity (page_size).  With planes, k may be NULL for the decode calls; v stays BF16.  Each scan scores every
  * key against plane A alone (head_dim + 2 bytes per key), ORs the verdicts over the rows that share the kv head,
  * and only then requests plane B rows (refined keys) and value rows (live keys).  This path takes row blocks of
- * at most 16 rows (stack * group <= 16, draft rows included; the verdicts are ORed over all of them) and one level
- * (no cascade), with or without the block tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED.
+ * at most 16 rows (stack * group <= 16, draft rows included; the verdicts are ORed over all of them), with or
+ * without the block tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED.  A cascade may run on
+ * two-plane keys when every level has them and no level stacks more than 16 rows per kv head (see
+ * fold_decode_cascade): each level is Algorithm 1 over its own rows -- the shared level's verdicts are ORed over the
+ * rows of every request that holds it --, and a level's automatic refine gate follows that level's own length.
  *
  * Two E4M3 value planes (Section 4, "Cache format": two FP8 planes that share one power-of-two scale per layer; only
  * together with the two-plane keys).  When v_plane_1 is not NULL the scan reads values from
@@ -263,7 +266,9 @@ size_t fold_workspace_bytes(const fold_args *args);
  * levels[0], levels[1], ... (a cascade's prefix then suffix; Appendix "Cascades and
  * drafts": the cascade takes its references from the flat estimate).  q, z and the head
  * counts are taken from levels[0]; each level contributes its kv and stack.  n_levels
- * in 1..4.  `levels` is a HOST array of HOST pointers. */
+ * in 1..4.  `levels` is a HOST array of HOST pointers.  The levels keep to one key format; with two-plane keys the
+ * sampled keys are scored with both planes, and every level's workspace (required, as for fold_decode_split)
+ * receives the split query rows. */
 int fold_estimate_z(const fold_args *const *levels, int n_levels, fold_stream stream);
 
 /* Scan only (Algorithm 1 with a BF16 cache): obtains z per args->z_mode, scores every key
@@ -296,7 +301,8 @@ int32_t fold_decode_launches(const fold_args *args);
  * pointers, n_levels in 1..4) describe the same requests: the same q, z, batch, head counts,
  * head_dim, softmax_scale and depth_T; each level has its own kv, stack and workspace.
  * levels[0]->z_mode is FOLD_Z_ESTIMATE (estimate over all levels, written to z) or FOLD_Z_GIVEN;
- * out, lse and row_status are taken from levels[0].
+ * out, lse and row_status are taken from levels[0].  The levels' keys are all BF16 or all two-plane
+ * (FOLD_EUNSUPPORTED otherwise); with two-plane keys one front kernel splits the query rows for every level.
  * With two or more levels and levels[0]->side_stream / side_fork_event / side_join_event set (a stream and two events the
  * CALLER owns, the stream different from `stream`), the first level is scanned on the side stream, forked from and
  * joined back into `stream` with the events, so to the caller the call is still one ordered piece of work on `stream`;

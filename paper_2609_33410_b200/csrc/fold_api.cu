@@ -271,22 +271,35 @@ PlaneView plane_view(const fold_kv &kv) {
 
 // Two-plane keys: the front kernel splits the query rows into the workspace whatever the reference mode, and
 // forms the estimate when asked to.
-int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st, bool zero_header = false) {
+// The two-plane front kernel over the levels of a cascade (one level: a plain decode).  Every level's workspace gets
+// the split query rows; the reference is estimated over the levels' keys in order when levels[0] asks for it.  The
+// levels share q, z, batch and head counts (checked by the callers); gs[l] is level l's geometry.
+int launch_planes_front_levels(const fold_args *const *levels, const Geometry *gs, int n_levels, cudaStream_t st,
+                               bool zero_header) {
+  const fold_args *a = levels[0];
+  const Geometry &g = gs[0];
   FrontParams p;
   memset(&p, 0, sizeof(p));
   p.q = static_cast<const __nv_bfloat16 *>(a->q);
   p.q_stride_b = a->q_stride_b; p.q_stride_h = a->q_stride_h;
-  uint8_t *ws = static_cast<uint8_t *>(a->workspace);
-  p.qplanes = reinterpret_cast<int8_t *>(ws + g.q_off);
-  p.qeta = reinterpret_cast<float *>(ws + g.q_off + round_up((size_t)g.B * g.Hq * 2 * g.D, 256));
+  p.n_levels = n_levels;
+  for (int l = 0; l < n_levels; ++l) {
+    uint8_t *ws = static_cast<uint8_t *>(levels[l]->workspace);
+    p.lv[l].qplanes = reinterpret_cast<int8_t *>(ws + gs[l].q_off);
+    p.lv[l].qeta = reinterpret_cast<float *>(ws + gs[l].q_off + round_up((size_t)g.B * g.Hq * 2 * g.D, 256));
+    p.lv[l].kv = plane_view(levels[l]->kv);
+    p.lv[l].stack = gs[l].stack;
+    p.lv[l].hdr = zero_header ? static_cast<fold_ws_header *>(levels[l]->workspace) : nullptr;
+  }
   p.z = a->z;
-  p.kv = plane_view(a->kv);
   p.write_z = a->z_mode == FOLD_Z_ESTIMATE;
-  p.stack = g.stack; p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
+  p.Hq = g.Hq; p.Hkv = g.Hkv; p.G = g.G;
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
-  p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
-  p.draft_len = a->draft_len;
-  p.hdr = zero_header ? static_cast<fold_ws_header *>(a->workspace) : nullptr;
+  {                                                          // drafts sit at the end of the last level
+    const fold_args *al = levels[n_levels - 1];
+    p.draft_mask = al->draft_len > 0 ? al->draft_mask : nullptr;
+    p.draft_len = al->draft_len;
+  }
   if (a->z_mode == FOLD_Z_ZERO) {
     const int rows = g.B * g.Hq;
     fold_fill_kernel<<<(rows + 255) / 256, 256, 0, st>>>(a->z, rows, 0.f);
@@ -297,6 +310,10 @@ int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st, 
                                     : launch_first(early, fold_planes_front_kernel<64>, grid, dim3(kFrontThreads), 0, st, p);
   if (rc != cudaSuccess) return FOLD_ECUDA;
   return cudaGetLastError() == cudaSuccess ? FOLD_OK : FOLD_ECUDA;
+}
+
+int launch_planes_front(const fold_args *a, const Geometry &g, cudaStream_t st, bool zero_header = false) {
+  return launch_planes_front_levels(&a, &g, 1, st, zero_header);
 }
 
 // zero_header: the kernel launched here also zeroes the first 64 bytes of a->workspace; header_zeroed_by_reference()
@@ -800,17 +817,26 @@ int estimate_levels(const fold_args *const *levels, int n_levels, fold_stream st
   if (!levels || n_levels < 1 || n_levels > kMaxLevels) return FOLD_EINVAL;
   const fold_args *a0 = levels[0];
   if (!a0) return FOLD_EINVAL;
-  for (int l = 1; l < n_levels; ++l)
-    if (levels[l] && levels[l]->kv.k_plane_a) return FOLD_EUNSUPPORTED;
-  if (a0->kv.k_plane_a) {                                    // two-plane keys: one level; the split rows go to its workspace
-    if (n_levels != 1) return FOLD_EUNSUPPORTED;
-    Geometry g;
-    fold_args tmp = *a0;
-    tmp.z_mode = FOLD_Z_ESTIMATE;
-    if (int rc = check_args(&tmp, &g, false)) return rc;
-    if (!tmp.workspace || !aligned(tmp.workspace, 256)) return FOLD_EINVAL;
-    if (tmp.workspace_bytes < g.ws_bytes) return FOLD_EWORKSPACE;
-    return launch_planes_front(&tmp, g, static_cast<cudaStream_t>(stream));
+  for (int l = 1; l < n_levels; ++l)                         // a cascade keeps to one key format
+    if (!levels[l] || (levels[l]->kv.k_plane_a != nullptr) != (a0->kv.k_plane_a != nullptr)) return FOLD_EUNSUPPORTED;
+  if (a0->kv.k_plane_a) {                                    // two-plane keys: the split rows go to every level's workspace
+    Geometry gs[kMaxLevels];
+    fold_args tmp[kMaxLevels];
+    const fold_args *tp[kMaxLevels];
+    for (int l = 0; l < n_levels; ++l) {
+      const fold_args *a = levels[l];
+      if (a->q != a0->q || a->z != a0->z || a->batch != a0->batch || a->num_q_heads != a0->num_q_heads ||
+          a->num_kv_heads != a0->num_kv_heads || a->head_dim != a0->head_dim || a->softmax_scale != a0->softmax_scale)
+        return FOLD_EINVAL;
+      tmp[l] = *a;
+      tmp[l].z_mode = FOLD_Z_ESTIMATE;
+      tp[l] = &tmp[l];
+      if (int rc = check_args(&tmp[l], &gs[l], false)) return rc;
+      if (l + 1 < n_levels && tmp[l].draft_len > 0) return FOLD_EINVAL;      // drafts end the last level
+      if (!tmp[l].workspace || !aligned(tmp[l].workspace, 256)) return FOLD_EINVAL;
+      if (tmp[l].workspace_bytes < gs[l].ws_bytes) return FOLD_EWORKSPACE;
+    }
+    return launch_planes_front_levels(tp, gs, n_levels, static_cast<cudaStream_t>(stream), zero_headers);
   }
   if (a0->head_dim != 64 && a0->head_dim != 128) return FOLD_EUNSUPPORTED;
   if (a0->batch < 1 || a0->num_q_heads < 1 || a0->num_kv_heads < 1 || a0->num_q_heads % a0->num_kv_heads)
@@ -853,7 +879,9 @@ int estimate_levels(const fold_args *const *levels, int n_levels, fold_stream st
 }
 
 // header_done: the workspace header has been zeroed by a kernel already in the stream
-int decode_split_impl(const fold_args *args, fold_partials *dst, fold_stream stream, bool header_done) {
+// reference_done: the level's reference kernel (a cascade's two-plane front kernel over all levels) is already in the stream
+int decode_split_impl(const fold_args *args, fold_partials *dst, fold_stream stream, bool header_done,
+                      bool reference_done = false) {
   Geometry g;
   if (int rc = check_args(args, &g, false)) return rc;
   if (!dst) return FOLD_EINVAL;
@@ -862,9 +890,10 @@ int decode_split_impl(const fold_args *args, fold_partials *dst, fold_stream str
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the header is zeroed by the reference kernel where one runs (estimate, or the two-plane front kernel), else by a
   // memset issued first, so that reference -> scan -> partial add stay adjacent kernels in the stream
-  const bool by_kernel = header_zeroed_by_reference(args, g);
+  const bool by_kernel = !reference_done && header_zeroed_by_reference(args, g);
   if (!by_kernel && !header_done && cudaMemsetAsync(args->workspace, 0, 64, st) != cudaSuccess) return FOLD_ECUDA;
-  if (int rc = launch_reference(args, g, st, by_kernel)) return rc;
+  if (!reference_done)
+    if (int rc = launch_reference(args, g, st, by_kernel)) return rc;
   if (int rc = launch_scan(args, g, st)) return rc;
   fill_partials(args, g, dst);
   return FOLD_OK;
@@ -1064,8 +1093,9 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
   if (!levels || n_levels < 1 || n_levels > kMaxLevels || !levels[0]) return FOLD_EINVAL;
   const fold_args *a0 = levels[0];
   if (a0->z_mode != FOLD_Z_ESTIMATE && a0->z_mode != FOLD_Z_GIVEN) return FOLD_EINVAL;
+  const bool planes = a0->kv.k_plane_a != nullptr;           // two-plane keys: every level, or none
   for (int l = 0; l < n_levels; ++l)
-    if (levels[l] && levels[l]->kv.k_plane_a) return FOLD_EUNSUPPORTED;   // two-plane keys: fold_decode only
+    if (levels[l] && (levels[l]->kv.k_plane_a != nullptr) != planes) return FOLD_EUNSUPPORTED;
   fold_args lv[kMaxLevels];
   for (int l = 0; l < n_levels; ++l) {
     const fold_args *a = levels[l];
@@ -1079,8 +1109,26 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
     if (int rc = check_args(&lv[l], &g, l == 0)) return rc;
   }
   const bool est = a0->z_mode == FOLD_Z_ESTIMATE;            // the estimate kernel then zeroes every level's header too
-  if (est)
+  if (planes) {
+    // one front kernel for the whole cascade: the split query rows into every level's workspace, the headers cleared,
+    // the reference over the levels' keys in order if it is to be estimated
+    if (est) {
+      if (int rc = estimate_levels(levels, n_levels, stream, true)) return rc;
+    } else {
+      Geometry gs[kMaxLevels];
+      const fold_args *tp[kMaxLevels];
+      for (int l = 0; l < n_levels; ++l) {
+        tp[l] = &lv[l];
+        if (int rc = check_args(&lv[l], &gs[l], false)) return rc;
+        if (!lv[l].workspace || !aligned(lv[l].workspace, 256)) return FOLD_EINVAL;
+        if (lv[l].workspace_bytes < gs[l].ws_bytes) return FOLD_EWORKSPACE;
+      }
+      if (int rc = launch_planes_front_levels(tp, gs, n_levels, static_cast<cudaStream_t>(stream), true)) return rc;
+    }
+  } else if (est) {
     if (int rc = estimate_levels(levels, n_levels, stream, true)) return rc;
+  }
+  const bool hdr_done = est || planes;
   fold_partials parts[kMaxLevels];
   const fold_partials *pp[kMaxLevels];
   for (int l = 0; l < n_levels; ++l) pp[l] = &parts[l];
@@ -1093,16 +1141,16 @@ int fold_decode_cascade(const fold_args *const *levels, int n_levels, fold_strea
     cudaEvent_t fork = static_cast<cudaEvent_t>(a0->side_fork_event), join = static_cast<cudaEvent_t>(a0->side_join_event);
     if (side == st) return FOLD_EINVAL;
     if (cudaEventRecord(fork, st) != cudaSuccess || cudaStreamWaitEvent(side, fork, 0) != cudaSuccess) return FOLD_ECUDA;
-    int rc = decode_split_impl(&lv[0], &parts[0], a0->side_stream, est);
+    int rc = decode_split_impl(&lv[0], &parts[0], a0->side_stream, hdr_done, planes);
     const bool recorded = cudaEventRecord(join, side) == cudaSuccess;
-    for (int l = 1; l < n_levels && rc == FOLD_OK; ++l) rc = decode_split_impl(&lv[l], &parts[l], stream, est);
+    for (int l = 1; l < n_levels && rc == FOLD_OK; ++l) rc = decode_split_impl(&lv[l], &parts[l], stream, hdr_done, planes);
     // join in every case, so that the side stream never holds work the caller's stream does not wait for
     if (!recorded || cudaStreamWaitEvent(st, join, 0) != cudaSuccess) return FOLD_ECUDA;
     if (rc) return rc;
     return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
   }
   for (int l = 0; l < n_levels; ++l)
-    if (int rc = decode_split_impl(&lv[l], &parts[l], stream, est)) return rc;
+    if (int rc = decode_split_impl(&lv[l], &parts[l], stream, hdr_done, planes)) return rc;
   return fold_cascade_merge(pp, n_levels, a0->out, a0->lse, a0->row_status, stream);
 }
 

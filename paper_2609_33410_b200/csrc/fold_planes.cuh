@@ -209,19 +209,25 @@ __global__ void __launch_bounds__(32 * kQuantWarps) fold_quantize_values_kernel(
 // Front kernel: one CTA per (kv head, request).  Splits the group's query rows (rows of the workspace:
 // [request * Hq + head][2][D] codes and one eta = e_q * scale_log2 per row), then, if the reference is to be
 // estimated, thread i scores sampled key i with both planes (exact integer dot products) and warp g
-// reduces row g.
+// reduces row g.  A cascade's levels are one logical sequence, level after level: the samples are taken over the
+// concatenation, and every level's workspace gets the split rows (and a cleared header).
+struct FrontLevel {
+  PlaneView kv;
+  int stack;                                                   // requests per sequence of this level
+  int8_t *qplanes;
+  float *qeta;
+  fold_ws_header *hdr;                                         // not null: also zero this level's workspace header
+};
 struct FrontParams {
   const __nv_bfloat16 *q;
   long long q_stride_b, q_stride_h;
-  int8_t *qplanes;
-  float *qeta;
   float *z;
-  PlaneView kv;
-  int write_z, stack, Hq, Hkv, G;
+  FrontLevel lv[kMaxLevels];
+  int n_levels;
+  int write_z, Hq, Hkv, G;
   float scale_log2;
   const uint32_t *draft_mask;                                  // drafts: the last draft_len keys are used by request req only
   int draft_len;                                               // where its mask has the bit
-  fold_ws_header *hdr;                                         // not null: also zero the scan's workspace header
 };
 constexpr int kFrontThreads = kEstSamples;                    // 192
 
@@ -252,32 +258,59 @@ __global__ void __launch_bounds__(kFrontThreads) fold_planes_front_kernel(const 
   // the workspace (split rows, header) may still be read by the scan of a call before this one, z by its partial add
   auto publish = [&]() {
     pdl_wait();
-    if (p.hdr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16) reinterpret_cast<uint32_t *>(p.hdr)[threadIdx.x] = 0u;
-    for (int i = threadIdx.x; i < G * 2 * W; i += kFrontThreads) {          // rows kvh * G .. + G - 1 are contiguous
-      const int g = i / (2 * W), w = i % (2 * W);
-      reinterpret_cast<uint32_t *>(p.qplanes + ((long long)req * p.Hq + kvh * G + g) * (2 * D))[w] = sq[g][w / W][w % W];
+#pragma unroll
+    for (int l = 0; l < kMaxLevels; ++l) {                     // (constant indices: the parameter block stays where it is)
+      if (l >= p.n_levels) break;
+      const FrontLevel &lv = p.lv[l];
+      if (lv.hdr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 16) reinterpret_cast<uint32_t *>(lv.hdr)[threadIdx.x] = 0u;
+      for (int i = threadIdx.x; i < G * 2 * W; i += kFrontThreads) {          // rows kvh * G .. + G - 1 are contiguous
+        const int g = i / (2 * W), w = i % (2 * W);
+        reinterpret_cast<uint32_t *>(lv.qplanes + ((long long)req * p.Hq + kvh * G + g) * (2 * D))[w] = sq[g][w / W][w % W];
+      }
+      if (threadIdx.x < G) lv.qeta[(long long)req * p.Hq + kvh * G + threadIdx.x] = seta[threadIdx.x];
     }
-    if (threadIdx.x < G) p.qeta[(long long)req * p.Hq + kvh * G + threadIdx.x] = seta[threadIdx.x];
   };
   if (!p.write_z) { publish(); return; }
 
-  const int seq = req / p.stack;
-  int n = p.kv.seqlens[seq];
-  n = n < 0 ? 0 : (n > p.kv.max_seqlen ? p.kv.max_seqlen : n);
+  // the request's keys: its sequence of every level, one after the other
+  int nl[kMaxLevels], n = 0;
+#pragma unroll
+  for (int l = 0; l < kMaxLevels; ++l) {
+    nl[l] = 0;
+    if (l < p.n_levels) {
+      const int v = p.lv[l].kv.seqlens[req / p.lv[l].stack];
+      nl[l] = v < 0 ? 0 : (v > p.lv[l].kv.max_seqlen ? p.lv[l].kv.max_seqlen : v);
+    }
+    n += nl[l];
+  }
   const int n_samples = n < kEstSamples ? n : kEstSamples;
   const int i = threadIdx.x;
   if (i < n_samples) {
-    long long s, t;
-    plane_locate(p.kv, seq, est_sample_key(i, n), s, t);
-    const long long off = s * p.kv.stride_seq + t * p.kv.stride_tok + (long long)kvh * p.kv.stride_head;
-    const float e = __bfloat162float(p.kv.scale[s * p.kv.sc_stride_seq + (long long)kvh * p.kv.sc_stride_head + t]);
+    int j = est_sample_key(i, n);
+    float e = 0.f;
     uint32_t ka[W], kb[W];
+    bool found = false;
 #pragma unroll
-    for (int w4 = 0; w4 < W / 4; ++w4) {
-      const uint4 va = *reinterpret_cast<const uint4 *>(p.kv.a + off + w4 * 16);
-      const uint4 vb = *reinterpret_cast<const uint4 *>(p.kv.b + off + w4 * 16);
-      ka[4 * w4] = va.x; ka[4 * w4 + 1] = va.y; ka[4 * w4 + 2] = va.z; ka[4 * w4 + 3] = va.w;
-      kb[4 * w4] = vb.x; kb[4 * w4 + 1] = vb.y; kb[4 * w4 + 2] = vb.z; kb[4 * w4 + 3] = vb.w;
+    for (int l = 0; l < kMaxLevels; ++l) {
+      if (l >= p.n_levels || found) continue;
+      if (j >= nl[l]) { j -= nl[l]; continue; }
+      found = true;
+      const PlaneView &kv = p.lv[l].kv;
+      long long s, t;
+      plane_locate(kv, req / p.lv[l].stack, j, s, t);
+      const long long off = s * kv.stride_seq + t * kv.stride_tok + (long long)kvh * kv.stride_head;
+      e = __bfloat162float(kv.scale[s * kv.sc_stride_seq + (long long)kvh * kv.sc_stride_head + t]);
+#pragma unroll
+      for (int w4 = 0; w4 < W / 4; ++w4) {
+        const uint4 va = *reinterpret_cast<const uint4 *>(kv.a + off + w4 * 16);
+        const uint4 vb = *reinterpret_cast<const uint4 *>(kv.b + off + w4 * 16);
+        ka[4 * w4] = va.x; ka[4 * w4 + 1] = va.y; ka[4 * w4 + 2] = va.z; ka[4 * w4 + 3] = va.w;
+        kb[4 * w4] = vb.x; kb[4 * w4 + 1] = vb.y; kb[4 * w4 + 2] = vb.z; kb[4 * w4 + 3] = vb.w;
+      }
+    }
+    if (!found) {                                              // (cannot happen: the sample index is below n)
+#pragma unroll
+      for (int w = 0; w < W; ++w) ka[w] = kb[w] = 0u;
     }
     for (int g = 0; g < G; ++g) {
       int caa = 0, cab = 0, cba = 0, cbb = 0;

@@ -213,15 +213,17 @@ def test_host_checks_of_two_plane_keys():
     for field, value in [("z_mode", F.Z_EXACT_MAX), ("stack", 2)]:
         old = getattr(a, field)
         setattr(a, field, value)
-        if field == "stack":                                        # 2 requests x group 4 on one sequence: 8 rows is the limit,
-            a.num_q_heads, a.num_kv_heads = 8, 1                    # 16 is beyond it
+        if field == "stack":                                        # 2 requests x group 12 on one sequence: 16 rows is the
+            a.num_q_heads, a.num_kv_heads = 12, 1                   # limit, 24 are beyond it
             a.kv.num_seqs = 1
         assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED, field
         setattr(a, field, old)
         a.num_q_heads, a.num_kv_heads = 8, 2; a.kv.num_seqs = 2
     args2 = (F.FoldArgs * 2)(a, a)
+    args2[1].kv.k_plane_a = None
     ptrs = (C.POINTER(F.FoldArgs) * 2)(C.pointer(args2[0]), C.pointer(args2[1]))
-    assert L.fold_decode_cascade(ptrs, 2, None) == F.FOLD_EUNSUPPORTED     # two-plane keys: one level only
+    assert L.fold_decode_cascade(ptrs, 2, None) == F.FOLD_EUNSUPPORTED     # a cascade keeps to one key format
+    assert L.fold_estimate_z(ptrs, 2, None) == F.FOLD_EUNSUPPORTED
     assert L.fold_quantize_keys(None, 2, 128, None, None) == F.FOLD_EINVAL
     kv = F.FoldKV()
     assert L.fold_quantize_keys(kv, 2, 96, None, None) == F.FOLD_EUNSUPPORTED

@@ -667,3 +667,140 @@ def test_million_key_sequence_on_planes_and_value_planes():
         assert same_bits(run_planes(w, cache, T=T, num_splits=3).out, b.out)
     del w, cache
     torch.cuda.empty_cache()
+
+
+# ------------------------------------------------------------------ shared-prefix cascades on two-plane keys
+def _planes_cascade(B, Hq, Hkv, D, n_prefix, suffixes, seed, T, tau, z_mode=F.Z_ESTIMATE, z=None, paged=False, side=None,
+                    separate_calls=False):
+    from paper_2609_33410_b200.workloads import make_cascade_workload
+    kw = dict(paged=True, page_size=32) if paged else {}
+    pre, suf = make_cascade_workload(B, Hq, Hkv, D, n_prefix, suffixes, seed=seed, device=DEV, poison_padding=True, **kw)
+    cp, cs = plane_cache(pre), plane_cache(suf)
+    bp, bs = F.alloc_buffers(pre.q, cp, stack=B), F.alloc_buffers(pre.q, cs)
+    if z is not None:
+        bs.z.copy_(z)
+    common = dict(z=bs.z, depth_T=T, out=bs.out, lse=bs.lse, row_status=bs.row_status, refine_tau=tau, z_mode=z_mode)
+    levels = [F.make_args(pre.q, cp, stack=B, workspace=bp.workspace, side=side, **common),
+              F.make_args(pre.q, cs, workspace=bs.workspace, **common)]
+    if separate_calls:                                         # the cascade spelled out: estimate, two scans, one add
+        if z_mode == F.Z_ESTIMATE:
+            F.fold_estimate_z(levels)
+        given = [F.make_args(pre.q, cp, stack=B, workspace=bp.workspace, **{**common, "z_mode": F.Z_GIVEN}),
+                 F.make_args(pre.q, cs, workspace=bs.workspace, **{**common, "z_mode": F.Z_GIVEN})]
+        parts = [F.fold_decode_split(a) for a in given]
+        F.fold_cascade_merge(parts, bs.out, bs.lse, bs.row_status)
+    else:
+        F.fold_decode_cascade(levels, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    assert bp.header().wait_timeouts == 0 and bs.header().wait_timeouts == 0
+    return pre, suf, cp, cs, bp, bs
+
+
+def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
+    """Each level is Algorithm 1 over its own rows -- the prefix level's verdicts are ORed over every request that
+    holds it, the suffix level's over the request's group --; the levels' (A, L) add (Eq. 3)."""
+    B, Hq, D = pre.q.shape
+    Hkv = pre.num_kv_heads
+    G = Hq // Hkv
+    out = bs.out.float().cpu().numpy().astype(np.float64)
+    lse = bs.lse.cpu().numpy().astype(np.float64)
+    z = bs.z.cpu().numpy().astype(np.float64)
+    qa, qb, eta = split_queries(suf, bs)
+    qa2, qb2, eta2 = split_queries(pre, bp)                    # every level's workspace holds the same split rows
+    assert np.array_equal(qa, qa2) and np.array_equal(qb, qb2) and np.array_equal(eta, eta2)
+    dz = 0.0
+    rels = []
+    for kvh in range(Hkv):
+        A = np.zeros((B, G, D)); L = np.zeros((B, G)); slack = np.zeros((B, G)); vmax = np.zeros((B, G))
+        s_all = [[[] for _ in range(G)] for _ in range(B)]
+
+        def level(w, cache, seq, rows):
+            n = int(w.seqlens[seq])
+            if n == 0:
+                return
+            ka, kb, ke = logical_planes(w, cache, seq, kvh)
+            V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
+            rqa = np.stack([qa[b, h] for (b, h) in rows]); rqb = np.stack([qb[b, h] for (b, h) in rows])
+            reta = np.array([eta[b, h] for (b, h) in rows], dtype=np.float64)
+            rz = np.array([z[b, h] for (b, h) in rows])
+            tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau       # the level's own length sets its automatic gate
+            a, l, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff)
+            vinf = np.abs(V).max(axis=1)
+            near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
+            near_tau = (np.abs(info["coarse"] + tau_eff) <= BAND).any(axis=0) if 0 <= tau_eff < math.inf else np.zeros(n, bool)
+            for i, (b, h) in enumerate(rows):
+                g = h - kvh * G
+                A[b, g] += a[i]; L[b, g] += l[i]; vmax[b, g] = max(vmax[b, g], float(vinf.max()))
+                corr = P.refine_terms(kb, ke, rqa[i], rqb[i], reta[i])
+                s_fin = info["coarse"][i] + np.where(info["refine"], corr, 0.0)
+                p = np.exp2(s_fin)
+                near = near_T if math.isinf(T) else (near_T | (np.abs(s_fin + T) <= BAND))
+                slack[b, g] += float((p[near] * vinf[near]).sum())
+                slack[b, g] += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum())
+                s_all[b][g].append(P.refined_scores(ka, kb, ke, rqa[i], rqb[i], reta[i]))
+
+        level(pre, cp, 0, [(b, kvh * G + g) for b in range(B) for g in range(G)])
+        for b in range(B):
+            level(suf, cs, b, [(b, kvh * G + g) for g in range(G)])
+        for b in range(B):
+            for g in range(G):
+                h = kvh * G + g
+                o_ref = A[b, g] / L[b, g]
+                d = out[b, h] - o_ref
+                assert np.abs(d).max() <= DENSE_MAX_ABS * vmax[b, g] + slack[b, g] / L[b, g] + 1e-30, (b, h, np.abs(d).max())
+                rels.append(np.linalg.norm(d) / max(np.linalg.norm(o_ref), 1e-300))
+                assert abs(lse[b, h] - (z[b, h] + math.log2(L[b, g]))) <= LSE_TOL, (b, h)
+                if check_estimate:
+                    s_cat = np.concatenate(s_all[b][g])
+                    dz = max(dz, abs(O.estimate_z(lambda idx: s_cat[idx], len(s_cat)) - z[b, h]))
+    if math.isinf(T):
+        assert float(np.mean(rels)) <= DENSE_MEAN_REL, np.mean(rels)
+    if check_estimate:
+        assert dz <= Z_TOL, dz
+    return dict(mean_rel=float(np.mean(rels)), dz=dz)
+
+
+@pytest.mark.parametrize("T,tau", [(math.inf, 0.0), (16.0, 0.0), (12.0, 6.0), (math.inf, math.inf)])
+@pytest.mark.parametrize("B,Hq,Hkv,paged", [(4, 8, 2, False), (3, 4, 1, True), (16, 2, 2, False), (2, 8, 1, False)])
+def test_shared_prefix_cascade_on_two_plane_keys(T, tau, B, Hq, Hkv, paged):
+    # the prefix level stacks every request's rows (up to 16 per kv head) on the shared keys; suffixes ragged, one empty
+    suffixes = ([500, 1, 0, 257] * 4)[:B]
+    lv = _planes_cascade(B, Hq, Hkv, 128, 3000, suffixes, seed=131, T=T, tau=tau, paged=paged)
+    _compare_planes_cascade(*lv, T=T, tau=tau, check_estimate=True)
+    # the call is its parts: estimate over both levels, two scans, one order-free add -- bit for bit
+    sp = _planes_cascade(B, Hq, Hkv, 128, 3000, suffixes, seed=131, T=T, tau=tau, paged=paged, separate_calls=True)
+    assert same_bits(sp[5].out, lv[5].out) and same_bits(sp[5].lse, lv[5].lse) and same_bits(sp[5].z, lv[5].z)
+    # a given reference, and the first level on the caller's side stream: the same bits again
+    gv = _planes_cascade(B, Hq, Hkv, 128, 3000, suffixes, seed=131, T=T, tau=tau, paged=paged, z_mode=F.Z_GIVEN,
+                         z=lv[5].z.clone(), side=F.CascadeSide(DEV))
+    assert same_bits(gv[5].out, lv[5].out) and same_bits(gv[5].lse, lv[5].lse)
+
+
+def test_cascade_on_two_plane_keys_head_dim_64_and_graph_replay():
+    lv = _planes_cascade(4, 8, 2, 64, 1000, [100, 0, 64, 33], seed=137, T=16.0, tau=0.0)
+    _compare_planes_cascade(*lv, T=16.0, tau=0.0, check_estimate=True)
+    pre, suf, cp, cs, bp, bs = lv
+    o, l = bs.out.clone(), bs.lse.clone()
+    common = dict(z=bs.z, depth_T=16.0, out=bs.out, lse=bs.lse, row_status=bs.row_status)
+    levels = [F.make_args(pre.q, cp, stack=4, workspace=bp.workspace, **common), F.make_args(pre.q, cs, workspace=bs.workspace, **common)]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        F.fold_decode_cascade(levels, torch.cuda.current_stream())
+    for _ in range(2):
+        bs.out.zero_(); bs.lse.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert same_bits(bs.out, o) and same_bits(bs.lse, l)
+    # a level of more than 16 stacked rows, or levels of two key formats, are refused
+    from paper_2609_33410_b200.workloads import make_cascade_workload
+    p5, s5 = make_cascade_workload(5, 8, 2, 128, 500, [10] * 5, seed=139, device=DEV)
+    c5p, c5s = plane_cache(p5), plane_cache(s5)
+    b5p, b5s = F.alloc_buffers(p5.q, cache_of(p5), stack=5), F.alloc_buffers(p5.q, c5s)
+    arr = [F.make_args(p5.q, c5p, stack=5, workspace=b5p.workspace, z=b5s.z, out=b5s.out, lse=b5s.lse),
+           F.make_args(p5.q, c5s, workspace=b5s.workspace, z=b5s.z, out=b5s.out, lse=b5s.lse)]
+    with pytest.raises(F.FoldError):
+        F.fold_decode_cascade(arr)
+    mixed = [F.make_args(pre.q, cache_of(pre), stack=4, workspace=bp.workspace, **common), levels[1]]
+    with pytest.raises(F.FoldError):
+        F.fold_decode_cascade(mixed)
+    torch.cuda.synchronize()
