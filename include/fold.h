@@ -126,12 +126,12 @@ enum {
  * and every (sequence-or-page, head) scale row must be readable up to the next multiple of 8 tokens past
  * capacity (page_size).  With planes, k may be NULL for the decode calls; v stays BF16.  Each scan scores every
  * key against plane A alone (head_dim + 2 bytes per key), ORs the verdicts over the rows that share the kv head,
- * and only then requests plane B rows (refined keys) and value rows (live keys).  This path takes row blocks of
- * at most 16 rows (stack * group <= 16, draft rows included; the verdicts are ORed over all of them), with or
- * without the block tail, and no FOLD_Z_EXACT_MAX; anything else returns FOLD_EUNSUPPORTED.  A cascade may run on
- * two-plane keys when every level has them and no level stacks more than 16 rows per kv head (see
- * fold_decode_cascade): each level is Algorithm 1 over its own rows -- the shared level's verdicts are ORed over the
- * rows of every request that holds it --, and a level's automatic refine gate follows that level's own length.
+ * and only then requests plane B rows (refined keys) and value rows (live keys).  Up to 16 rows per
+ * (sequence, kv head) (stack * group, draft rows included) form one block whose verdicts are ORed over all of them;
+ * more stacked rows (a cascade's shared level) are cut into blocks of 16 rows in row order, each block scanned as
+ * Algorithm 1 over its own rows with its own verdicts.  With or without the block tail; no FOLD_Z_EXACT_MAX, and
+ * draft rows only within one block (FOLD_EUNSUPPORTED otherwise).  A cascade may run on two-plane keys when every
+ * level has them (see fold_decode_cascade); a level's automatic refine gate follows that level's own length.
  *
  * Two E4M3 value planes (Section 4, "Cache format": two FP8 planes that share one power-of-two scale per layer; only
  * together with the two-plane keys).  When v_plane_1 is not NULL the scan reads values from

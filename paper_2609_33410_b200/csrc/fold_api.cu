@@ -116,8 +116,9 @@ int check_args(const fold_args *a, Geometry *g, bool need_out) {
   g->ws_bytes = g->planes ? g->q_off + qplane_bytes((long long)g->B * g->Hq, g->D) : kHeaderBytes + g->slot_bytes;
   if (g->planes) {
     if (isnan(a->refine_tau)) return FOLD_EINVAL;
-    // the two-plane scan: one block of up to 16 rows (its verdicts are the group's), no exact-maximum pass
-    if (R > kMaxRows || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
+    // the two-plane scan: blocks of up to 16 rows (a block's verdicts are ORed over its rows), no exact-maximum pass;
+    // draft rows share their sequence's verdicts, so they stay within one block
+    if ((R > kMaxRows && a->draft_len > 0) || a->z_mode == FOLD_Z_EXACT_MAX) return FOLD_EUNSUPPORTED;
     if (a->kv.v_plane_1 && isnan(a->refine_tau_v)) return FOLD_EINVAL;
   }
   return FOLD_OK;
@@ -562,7 +563,8 @@ int choose_splits(const fold_args *a, const Geometry &g, int tile_keys) {
   if (max_chunks > 65535) max_chunks = 65535;               // splits index a grid dimension (a split walks several chunks)
   if (a->num_splits > 0) return a->num_splits < max_chunks ? a->num_splits : max_chunks;
   const long long units = (long long)g.num_seqs * g.Hkv *
-                          (g.R > 128 ? (g.R + 255) / 256 : (g.R <= row_block_rows() ? (g.R + kMaxRows - 1) / kMaxRows : 1));   // CTAs per split
+                          (g.planes ? (g.R + kMaxRows - 1) / kMaxRows :
+                           g.R > 128 ? (g.R + 255) / 256 : (g.R <= row_block_rows() ? (g.R + kMaxRows - 1) / kMaxRows : 1));   // CTAs per split
   const int tiles_unit = max_chunks * (chunk_keys_of(n) / tile_keys);
   int s = tiles_unit / 32;
   s = s < 1 ? 1 : (s > max_chunks ? max_chunks : s);
@@ -639,7 +641,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   p.num_splits = choose_splits(a, g, tile_keys);
   p.scale_log2 = (float)((double)a->softmax_scale * 1.4426950408889634);
   p.neg_T = isinf(a->depth_T) ? -INFINITY : -a->depth_T;
-  p.row_groups = 1;
+  p.row_groups = (g.R + kMaxRows - 1) / kMaxRows;            // blocks of 16 rows, each its own CTA (a cascade's shared level)
   p.draft_mask = a->draft_len > 0 ? a->draft_mask : nullptr;
   p.draft_len = a->draft_len;
   if (!isinf(a->depth_T) && kv.v_plane_1) {                  // 8-bit values: the table holds the sequences' mean rows (block 0)
@@ -657,7 +659,7 @@ int launch_scan_planes(const fold_args *a, const Geometry &g, cudaStream_t st) {
   pp.neg_tau_v = a->refine_tau_v < 0.f ? INFINITY : -a->refine_tau_v;
   pp.auto_tau = a->refine_tau == 0.f;
   pp.neg_tau = a->refine_tau < 0.f ? INFINITY : -a->refine_tau;      // tau = inf -> -inf: every live key
-  const dim3 grid(g.Hkv, p.num_splits, g.num_seqs);
+  const dim3 grid(g.Hkv * p.row_groups, p.num_splits, g.num_seqs);
   return g.D == 128 ? launch_planes_kernel<128>(ma, mv, pp, grid, st) : launch_planes_kernel<64>(ma, mv, pp, grid, st);
 }
 

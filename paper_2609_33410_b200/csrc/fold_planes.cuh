@@ -508,10 +508,14 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   uint8_t *gen = smem_raw + (base - raw);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kvh = blockIdx.x, split = blockIdx.y, seq = blockIdx.z;
+  // x = row group + row_groups * kv head: more than 16 stacked rows (a cascade's shared level) are cut into blocks of
+  // 16 rows in row order, each block a CTA of its own that runs Algorithm 1 over its rows (its verdicts are ORed over
+  // the block); the blocks of a kv head sit side by side and share its tiles in L2
+  const int rg = blockIdx.x % p.row_groups, kvh = blockIdx.x / p.row_groups, split = blockIdx.y, seq = blockIdx.z;
   const SeqWork w = seq_work<TK>(p, seq);
   if (split >= w.n_chunks) return;
-  const int stages = p.stages, R = p.R, n = w.n;
+  const int rbase = rg * kMaxRows;                            // the block's first row among the (sequence, kv head)'s rows
+  const int stages = p.stages, R = min(p.R - rbase, 8 * NT), n = w.n;
   const uint32_t full0 = base + LO::off_bar(stages), empty0 = full0 + 8u * stages;
   const uint32_t gbar0 = empty0 + 8u * stages;               // one barrier per (warp, gather buffer)
 
@@ -537,7 +541,7 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
   for (int q = 0; q < NT; ++q) {
     const int r = 8 * q + (lane >> 2);
     const bool ok = r < R;
-    const int req = seq * p.stack + r / p.G, head = kvh * p.G + r % p.G;
+    const int req = seq * p.stack + (rbase + r) / p.G, head = kvh * p.G + (rbase + r) % p.G;
     const int8_t *qp = pp.qplanes + ((long long)req * p.Hq + head) * (2 * D) + (lane & 3) * 4;
 #pragma unroll
     for (int kk = 0; kk < D / 32; ++kk) {
@@ -556,8 +560,8 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     for (int e = 0; e < 2; ++e) {
       const int r = 8 * q + (lane & 3) * 2 + e;
       rv[q][e] = r < R;
-      const int req = seq * p.stack + r / p.G;
-      const long long row = (long long)req * p.Hq + kvh * p.G + r % p.G;
+      const int req = seq * p.stack + (rbase + r) / p.G;
+      const long long row = (long long)req * p.Hq + kvh * p.G + (rbase + r) % p.G;
       eta[q][e] = rv[q][e] ? pp.qeta[row] : 0.f;
       zr[q][e] = rv[q][e] ? p.z[row] : 0.f;
       dm[q][e] = (DRAFTS && rv[q][e]) ? p.draft_mask[req] : 0xffffffffu;
@@ -916,8 +920,8 @@ fold_scan_planes_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
     for (int q = 0; q < NT; ++q) {                            // a tile's rows: 8 q .. 8 q + 7, as many as the block has
       const int Rq = min(8, R - 8 * q);
-      reduce_store_L_n<kConsumerWarps>(l_lo[q], l_hi[q], redl, slot + R * D + 8 * q, Rq, warp, lane, threadIdx.x, 1);
-      reduce_store_A_n<D, kConsumerWarps>(o[q], red, slot + 8 * q * D, Rq, warp, lane, threadIdx.x, 1);
+      reduce_store_L_n<kConsumerWarps>(l_lo[q], l_hi[q], redl, slot + p.R * D + rbase + 8 * q, Rq, warp, lane, threadIdx.x, 1);
+      reduce_store_A_n<D, kConsumerWarps>(o[q], red, slot + (rbase + 8 * q) * D, Rq, warp, lane, threadIdx.x, 1);
     }
     if (c + p.num_splits < w.n_chunks) clear_bufs();
   }

@@ -125,53 +125,57 @@ def compare_planes(w, cache, bufs, T=math.inf, tau=0.0, units=None, check_estima
         ka, kb, ke = logical_planes(w, cache, seq, kvh)
         V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
         Kx = O.widen_bf16(bf16_bits(w.logical_rows("k", seq, kvh)))
-        rqa = np.stack([qa[b, h] for (b, h) in rows]); rqb = np.stack([qb[b, h] for (b, h) in rows])
-        reta = np.array([eta[b, h] for (b, h) in rows], dtype=np.float64)
-        rz = np.array([z[b, h] for (b, h) in rows])
-        tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
-        vis = None if draft is None else np.stack([O.draft_visible(n, draft[1], dmask[b]) for (b, h) in rows])
-        vm = None if vmt is None else vmt[seq, :(n + 63) // 64, kvh]
-        vpl, tau_v_eff = None, None
-        if vfp8:
-            p1, p2 = logical_value_planes(w, cache, seq, kvh)
-            vpl = (p1, p2, cache.v_scale_log2)
-            tau_v_eff = P.auto_refine_tau_v(n) if tau_v == 0.0 else tau_v
-        A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis, v_mean=vm,
-                                         value_planes=vpl, tau_v=tau_v_eff,
-                                         v_run_mean=None if vrt is None else vrt[seq, 0, kvh])
-        n_refv += int(info["refine_v"].sum())
-        n_live += int(info["live"].sum()); n_ref += int(info["refine"].sum()); n_keys += n
-        vinf = np.abs(V).max(axis=1)
-        near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
-        near_tau = (np.abs(info["coarse"] + tau_eff) <= BAND).any(axis=0) if 0 <= tau_eff < math.inf else np.zeros(n, bool)
-        for i, (b, h) in enumerate(rows):
-            o_ref = A[i] / L[i]
-            d = out[b, h] - o_ref
-            num += float(d @ d); den += float(o_ref @ o_ref)
-            max_abs = max(max_abs, float(np.abs(d).max())); vmax = max(vmax, float(vinf.max()))
-            rel_rows.append(np.linalg.norm(d) / max(np.linalg.norm(o_ref), 1e-300))
-            assert abs(lse[b, h] - (rz[i] + math.log2(L[i]))) <= LSE_TOL, (b, h)
-            if 0.5 <= L[i] <= 2.0 ** 100:
-                assert status[b, h] == 0, (b, h, status[b, h], L[i])
-            corr = P.refine_terms(kb, ke, rqa[i], rqb[i], reta[i])
-            s_fin = info["coarse"][i] + np.where(info["refine"], corr, 0.0)
-            p = np.exp2(s_fin)
-            if check_estimate:
-                s_all = P.refined_scores(ka, kb, ke, rqa[i], rqb[i], reta[i])
-                if vis is not None:
-                    s_all = np.where(vis[i], s_all, -np.inf)
-                dz = max(dz, abs(O.estimate_z(lambda idx: s_all[idx], n) - z[b, h]))
-            if not math.isinf(T):
-                near = near_T | (np.abs(s_fin + T) <= BAND)
-                sl = (2.0 if (vmt is not None or vrt is not None) else 1.0) * float((p[near] * vinf[near]).sum() / L[i])
-                sl += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum() / L[i])
-                slack2 += sl ** 2 * V.shape[1]
-                keep = slice(None) if vis is None else vis[i]
-                o_dense = O.dense_row(O.scores(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], w.scale), V[keep])[0]
-                y = O.online_softmax_bf16(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], V[keep], w.scale) - o_dense
-                ynum += float(y @ y)
-                per_row.append((b, h, float(np.linalg.norm(d)), float(np.abs(d).max()), float(np.linalg.norm(o_ref)), sl,
-                                float(vinf.max()), float(np.linalg.norm(y))))
+        # more than 16 rows per (sequence, kv head): blocks of 16 rows in row order, each Algorithm 1 over its own rows
+        all_rows = rows
+        for blk0 in range(0, R, 16):
+            rows_blk = all_rows[blk0:blk0 + 16]
+            rqa = np.stack([qa[b, h] for (b, h) in rows_blk]); rqb = np.stack([qb[b, h] for (b, h) in rows_blk])
+            reta = np.array([eta[b, h] for (b, h) in rows_blk], dtype=np.float64)
+            rz = np.array([z[b, h] for (b, h) in rows_blk])
+            tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
+            vis = None if draft is None else np.stack([O.draft_visible(n, draft[1], dmask[b]) for (b, h) in rows_blk])
+            vm = None if vmt is None else vmt[seq, :(n + 63) // 64, kvh]
+            vpl, tau_v_eff = None, None
+            if vfp8:
+                p1, p2 = logical_value_planes(w, cache, seq, kvh)
+                vpl = (p1, p2, cache.v_scale_log2)
+                tau_v_eff = P.auto_refine_tau_v(n) if tau_v == 0.0 else tau_v
+            A, L, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff, visible=vis, v_mean=vm,
+                                             value_planes=vpl, tau_v=tau_v_eff,
+                                             v_run_mean=None if vrt is None else vrt[seq, 0, kvh])
+            n_refv += int(info["refine_v"].sum())
+            n_live += int(info["live"].sum()); n_ref += int(info["refine"].sum()); n_keys += n
+            vinf = np.abs(V).max(axis=1)
+            near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
+            near_tau = (np.abs(info["coarse"] + tau_eff) <= BAND).any(axis=0) if 0 <= tau_eff < math.inf else np.zeros(n, bool)
+            for i, (b, h) in enumerate(rows_blk):
+                o_ref = A[i] / L[i]
+                d = out[b, h] - o_ref
+                num += float(d @ d); den += float(o_ref @ o_ref)
+                max_abs = max(max_abs, float(np.abs(d).max())); vmax = max(vmax, float(vinf.max()))
+                rel_rows.append(np.linalg.norm(d) / max(np.linalg.norm(o_ref), 1e-300))
+                assert abs(lse[b, h] - (rz[i] + math.log2(L[i]))) <= LSE_TOL, (b, h)
+                if 0.5 <= L[i] <= 2.0 ** 100:
+                    assert status[b, h] == 0, (b, h, status[b, h], L[i])
+                corr = P.refine_terms(kb, ke, rqa[i], rqb[i], reta[i])
+                s_fin = info["coarse"][i] + np.where(info["refine"], corr, 0.0)
+                p = np.exp2(s_fin)
+                if check_estimate:
+                    s_all = P.refined_scores(ka, kb, ke, rqa[i], rqb[i], reta[i])
+                    if vis is not None:
+                        s_all = np.where(vis[i], s_all, -np.inf)
+                    dz = max(dz, abs(O.estimate_z(lambda idx: s_all[idx], n) - z[b, h]))
+                if not math.isinf(T):
+                    near = near_T | (np.abs(s_fin + T) <= BAND)
+                    sl = (2.0 if (vmt is not None or vrt is not None) else 1.0) * float((p[near] * vinf[near]).sum() / L[i])
+                    sl += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum() / L[i])
+                    slack2 += sl ** 2 * V.shape[1]
+                    keep = slice(None) if vis is None else vis[i]
+                    o_dense = O.dense_row(O.scores(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], w.scale), V[keep])[0]
+                    y = O.online_softmax_bf16(O.widen_bf16(bf16_bits(w.q[b, h])), Kx[keep], V[keep], w.scale) - o_dense
+                    ynum += float(y @ y)
+                    per_row.append((b, h, float(np.linalg.norm(d)), float(np.abs(d).max()), float(np.linalg.norm(o_ref)), sl,
+                                    float(vinf.max()), float(np.linalg.norm(y))))
     res = dict(rel_l2=math.sqrt(num / max(den, 1e-300)), max_abs=max_abs, vmax=vmax,
                mean_rel=float(np.mean(rel_rows)) if rel_rows else 0.0, dz=dz,
                live_frac=n_live / max(n_keys, 1), refine_frac=n_ref / max(n_keys, 1))
@@ -278,12 +282,20 @@ def test_edge_lengths(D, n):
 
 @pytest.mark.parametrize("Hq,Hkv,stack", [(1, 1, 1), (8, 8, 1), (4, 2, 1), (8, 1, 1), (8, 2, 2), (2, 2, 4), (3, 1, 2),
                                           # 9 to 16 rows per (sequence, kv head): two 8-row tiles, verdicts over all of them
-                                          (16, 1, 1), (9, 1, 1), (24, 2, 1), (8, 2, 4), (3, 1, 5), (4, 2, 7), (13, 1, 1)])
+                                          (16, 1, 1), (9, 1, 1), (24, 2, 1), (8, 2, 4), (3, 1, 5), (4, 2, 7), (13, 1, 1),
+                                          # more than 16 stacked rows: blocks of 16 rows, each with its own verdicts
+                                          (8, 2, 5), (4, 1, 20), (16, 2, 3), (3, 1, 11)])
 def test_group_and_stack_shapes(Hq, Hkv, stack):
     w = make_decode_workload(2 * stack, Hq, Hkv, 128, [700, 300], seed=47, device=DEV, stack=stack)
     cache = plane_cache(w)
     compare_planes(w, cache, run_planes(w, cache))
     compare_planes(w, cache, run_planes(w, cache, T=12.0), T=12.0)
+    if stack * (Hq // Hkv) > 16:                                # the wide forms with the block tail and with E4M3 values too
+        vm = oracle_block_means(w)
+        ct = with_means(cache, vm)
+        compare_planes(w, ct, run_planes(w, ct, T=10.0), T=10.0, v_block_mean=vm)
+        value_planes_of(w, cache)
+        compare_planes(w, cache, run_planes(w, cache, T=12.0), T=12.0)
 
 
 @pytest.mark.parametrize("page_size", [16, 32, 64, 128, 256])
@@ -346,10 +358,11 @@ def test_empty_sequences_and_unsupported_shapes():
     cache = plane_cache(w)
     compare_planes(w, cache, run_planes(w, cache))
     compare_planes(w, cache, run_planes(w, cache, T=16.0), T=16.0)
-    wide = make_decode_workload(5, 4, 1, 128, [300], seed=73, device=DEV, stack=5)      # 20 rows: beyond the two-plane scan
-    c2 = plane_cache(wide)
-    bufs = F.alloc_buffers(wide.q, cache_of(wide), 5)
-    a = F.make_args(wide.q, c2, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, stack=5)
+    wide = make_decode_workload(5, 4, 1, 128, [300], seed=73, device=DEV, stack=5)      # 20 rows: two blocks -- not with draft rows,
+    c2 = plane_cache(wide)                                                              # which share their sequence's verdicts
+    bufs = F.alloc_buffers(wide.q, c2, 5)
+    masks = torch.full((5,), 1, dtype=torch.int32, device=DEV)
+    a = F.make_args(wide.q, c2, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, stack=5, draft_mask=masks, draft_len=5)
     assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
     a = F.make_args(w.q, cache, z=bufs.z, workspace=bufs.workspace, out=bufs.out, lse=bufs.lse, z_mode=F.Z_EXACT_MAX)
     assert F.lib().fold_decode(a, None) == F.FOLD_EUNSUPPORTED
@@ -739,7 +752,9 @@ def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
                 slack[b, g] += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum())
                 s_all[b][g].append(P.refined_scores(ka, kb, ke, rqa[i], rqb[i], reta[i]))
 
-        level(pre, cp, 0, [(b, kvh * G + g) for b in range(B) for g in range(G)])
+        stacked = [(b, kvh * G + g) for b in range(B) for g in range(G)]
+        for blk0 in range(0, len(stacked), 16):                # a level of more than 16 stacked rows: blocks of 16, in row order
+            level(pre, cp, 0, stacked[blk0:blk0 + 16])
         for b in range(B):
             level(suf, cs, b, [(b, kvh * G + g) for g in range(G)])
         for b in range(B):
@@ -761,10 +776,11 @@ def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
 
 
 @pytest.mark.parametrize("T,tau", [(math.inf, 0.0), (16.0, 0.0), (12.0, 6.0), (math.inf, math.inf)])
-@pytest.mark.parametrize("B,Hq,Hkv,paged", [(4, 8, 2, False), (3, 4, 1, True), (16, 2, 2, False), (2, 8, 1, False)])
+@pytest.mark.parametrize("B,Hq,Hkv,paged", [(4, 8, 2, False), (3, 4, 1, True), (16, 2, 2, False), (2, 8, 1, False),
+                                            (20, 8, 2, False), (7, 8, 1, True)])          # 80 and 56 stacked rows: blocks of 16
 def test_shared_prefix_cascade_on_two_plane_keys(T, tau, B, Hq, Hkv, paged):
     # the prefix level stacks every request's rows (up to 16 per kv head) on the shared keys; suffixes ragged, one empty
-    suffixes = ([500, 1, 0, 257] * 4)[:B]
+    suffixes = ([500, 1, 0, 257] * 5)[:B]
     lv = _planes_cascade(B, Hq, Hkv, 128, 3000, suffixes, seed=131, T=T, tau=tau, paged=paged)
     _compare_planes_cascade(*lv, T=T, tau=tau, check_estimate=True)
     # the call is its parts: estimate over both levels, two scans, one order-free add -- bit for bit
@@ -791,15 +807,7 @@ def test_cascade_on_two_plane_keys_head_dim_64_and_graph_replay():
         graph.replay()
         torch.cuda.synchronize()
         assert same_bits(bs.out, o) and same_bits(bs.lse, l)
-    # a level of more than 16 stacked rows, or levels of two key formats, are refused
-    from paper_2609_33410_b200.workloads import make_cascade_workload
-    p5, s5 = make_cascade_workload(5, 8, 2, 128, 500, [10] * 5, seed=139, device=DEV)
-    c5p, c5s = plane_cache(p5), plane_cache(s5)
-    b5p, b5s = F.alloc_buffers(p5.q, cache_of(p5), stack=5), F.alloc_buffers(p5.q, c5s)
-    arr = [F.make_args(p5.q, c5p, stack=5, workspace=b5p.workspace, z=b5s.z, out=b5s.out, lse=b5s.lse),
-           F.make_args(p5.q, c5s, workspace=b5s.workspace, z=b5s.z, out=b5s.out, lse=b5s.lse)]
-    with pytest.raises(F.FoldError):
-        F.fold_decode_cascade(arr)
+    # levels of two key formats are refused
     mixed = [F.make_args(pre.q, cache_of(pre), stack=4, workspace=bp.workspace, **common), levels[1]]
     with pytest.raises(F.FoldError):
         F.fold_decode_cascade(mixed)
