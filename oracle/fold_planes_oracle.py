@@ -30,6 +30,9 @@ What is here, with the passage each function restates (Section 4, "Cache format"
   fold_group_planes   Algorithm 1 for one (sequence, kv head): verdict bits ORed over the
                       group's rows, final weights, (A, L) per row; also counts the bytes the
                       gates ask for (130 + 128 r_K + 256 lambda per key at D = 128)
+  fold_levels_planes  a cascade over two-plane levels for one kv head (Appendix "Cascades and drafts";
+                      Prop. 1(i)): every level's sequence is Algorithm 1 over the rows of the requests
+                      stacked on it, in blocks of 16 rows with their own verdicts; the levels' (A, L) add
 """
 from __future__ import annotations
 
@@ -266,6 +269,39 @@ def fold_group_planes(ka, kb, ke, V, qa, qb, eta, Z, T: float = math.inf, tau: O
     v_bytes = 2 * D * lam if value_planes is None else D * lam + D * rv          # (Section 4: the 256 value bytes become 128 + 128 r_V)
     info = dict(live=live, refine=refine, refine_v=refine_v, coarse=coarse, bytes_per_key=(D + 2) + D * rk + v_bytes)
     return A, L, info
+
+
+def fold_levels_planes(levels, qa, qb, eta, Z, T: float = math.inf, tau: Optional[float] = None, block_rows: int = 16):
+    """A cascade on two-plane keys, one kv head.  `levels` = [(stack, [(ka, kb, ke, V), ...]), ...]: level l holds one
+    key sequence per `stack` consecutive requests (request b reads sequence b // stack; a shared prefix is stack =
+    all requests, a private suffix stack = 1).  qa, qb [B, G, D] int8; eta, Z [B, G].
+    Readings (the paper states Algorithm 1 for one group and says a cascade level stacks the rows of the requests
+    that hold it): a sequence's rows -- request-major, the group's rows within a request -- are cut into blocks of
+    `block_rows`, each block is `fold_group_planes` over its own rows (its verdicts ORed over the block), and
+    tau = None takes `auto_refine_tau` of the LEVEL's own sequence length.  Partials of one row under one reference
+    add (Prop. 1(i)).  Returns (A [B, G, D], L [B, G], infos) with infos = [(level, sequence, rows of the block as
+    (b, g) pairs, info of fold_group_planes)]."""
+    qa = np.asarray(qa); qb = np.asarray(qb)
+    B, G, D = qa.shape
+    A = np.zeros((B, G, D)); L = np.zeros((B, G))
+    infos = []
+    for li, (stack, seqs) in enumerate(levels):
+        assert B % stack == 0 and len(seqs) == B // stack
+        for j, (ka, kb, ke, V) in enumerate(seqs):
+            n = np.asarray(ka).shape[0]
+            if n == 0:
+                continue
+            rows = [(b, g) for b in range(j * stack, (j + 1) * stack) for g in range(G)]
+            for r0 in range(0, len(rows), block_rows):
+                blk = rows[r0:r0 + block_rows]
+                a, l, info = fold_group_planes(ka, kb, ke, V, np.stack([qa[b, g] for b, g in blk]), np.stack([qb[b, g] for b, g in blk]),
+                                               np.array([eta[b][g] for b, g in blk], dtype=np.float64),
+                                               np.array([Z[b][g] for b, g in blk], dtype=np.float64), T,
+                                               auto_refine_tau(n) if tau is None else tau)
+                for i, (b, g) in enumerate(blk):
+                    A[b, g] += a[i]; L[b, g] += l[i]
+                infos.append((li, j, blk, info))
+    return A, L, infos
 
 
 def estimate_z_planes(ka, kb, ke, qa, qb, eta: float) -> float:

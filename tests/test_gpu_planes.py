@@ -710,8 +710,8 @@ def _planes_cascade(B, Hq, Hkv, D, n_prefix, suffixes, seed, T, tau, z_mode=F.Z_
 
 
 def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
-    """Each level is Algorithm 1 over its own rows -- the prefix level's verdicts are ORed over every request that
-    holds it, the suffix level's over the request's group --; the levels' (A, L) add (Eq. 3)."""
+    """The oracle's cascade (`fold_levels_planes`: each level Algorithm 1 over its own rows in blocks of 16, the levels'
+    (A, L) added, Eq. 3) at the GPU's own references and split query rows."""
     B, Hq, D = pre.q.shape
     Hkv = pre.num_kv_heads
     G = Hq // Hkv
@@ -724,39 +724,36 @@ def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
     dz = 0.0
     rels = []
     for kvh in range(Hkv):
-        A = np.zeros((B, G, D)); L = np.zeros((B, G)); slack = np.zeros((B, G)); vmax = np.zeros((B, G))
-        s_all = [[[] for _ in range(G)] for _ in range(B)]
+        hs = slice(kvh * G, (kvh + 1) * G)
 
-        def level(w, cache, seq, rows):
+        def seq_of(w, cache, seq):
             n = int(w.seqlens[seq])
             if n == 0:
-                return
-            ka, kb, ke = logical_planes(w, cache, seq, kvh)
-            V = O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh)))
-            rqa = np.stack([qa[b, h] for (b, h) in rows]); rqb = np.stack([qb[b, h] for (b, h) in rows])
-            reta = np.array([eta[b, h] for (b, h) in rows], dtype=np.float64)
-            rz = np.array([z[b, h] for (b, h) in rows])
-            tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau       # the level's own length sets its automatic gate
-            a, l, info = P.fold_group_planes(ka, kb, ke, V, rqa, rqb, reta, rz, T, tau_eff)
+                return (np.zeros((0, D), np.int8), np.zeros((0, D), np.int8), np.zeros(0), np.zeros((0, D)))
+            return logical_planes(w, cache, seq, kvh) + (O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh))),)
+
+        levels = [(B, [seq_of(pre, cp, 0)]), (1, [seq_of(suf, cs, b) for b in range(B)])]
+        A, L, infos = P.fold_levels_planes(levels, qa[:, hs], qb[:, hs], eta[:, hs].astype(np.float64), z[:, hs], T,
+                                           None if tau == 0.0 else tau)
+        # what a key next to a gate may cost (fp32 against fp64 decisions), and the rows' full two-plane scores
+        slack = np.zeros((B, G)); vmax = np.zeros((B, G))
+        s_all = [[[] for _ in range(G)] for _ in range(B)]
+        for (li, j, blk, info) in infos:
+            ka, kb, ke, V = levels[li][1][j]
+            n = ka.shape[0]
+            tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
             vinf = np.abs(V).max(axis=1)
             near_T = np.zeros(n, bool) if math.isinf(T) else (np.abs(info["coarse"] + T) <= BAND).any(axis=0)
             near_tau = (np.abs(info["coarse"] + tau_eff) <= BAND).any(axis=0) if 0 <= tau_eff < math.inf else np.zeros(n, bool)
-            for i, (b, h) in enumerate(rows):
-                g = h - kvh * G
-                A[b, g] += a[i]; L[b, g] += l[i]; vmax[b, g] = max(vmax[b, g], float(vinf.max()))
-                corr = P.refine_terms(kb, ke, rqa[i], rqb[i], reta[i])
+            for i, (b, g) in enumerate(blk):
+                vmax[b, g] = max(vmax[b, g], float(vinf.max()))
+                corr = P.refine_terms(kb, ke, qa[b, kvh * G + g], qb[b, kvh * G + g], eta[b, kvh * G + g])
                 s_fin = info["coarse"][i] + np.where(info["refine"], corr, 0.0)
                 p = np.exp2(s_fin)
                 near = near_T if math.isinf(T) else (near_T | (np.abs(s_fin + T) <= BAND))
                 slack[b, g] += float((p[near] * vinf[near]).sum())
                 slack[b, g] += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum())
-                s_all[b][g].append(P.refined_scores(ka, kb, ke, rqa[i], rqb[i], reta[i]))
-
-        stacked = [(b, kvh * G + g) for b in range(B) for g in range(G)]
-        for blk0 in range(0, len(stacked), 16):                # a level of more than 16 stacked rows: blocks of 16, in row order
-            level(pre, cp, 0, stacked[blk0:blk0 + 16])
-        for b in range(B):
-            level(suf, cs, b, [(b, kvh * G + g) for g in range(G)])
+                s_all[b][g].append(P.refined_scores(ka, kb, ke, qa[b, kvh * G + g], qb[b, kvh * G + g], eta[b, kvh * G + g]))
         for b in range(B):
             for g in range(G):
                 h = kvh * G + g

@@ -403,3 +403,70 @@ def test_running_mean_cut_model_of_the_value_planes():
     Ar, Lr, _ = P.fold_group_planes(a2, b2, e2, None, qa, qb, eta, Z2, 3.0, 1.0, value_planes=vs, tau_v=2.0, v_run_mean=P.running_mean(Vs))
     Ab, Lb, _ = P.fold_group_planes(a2, b2, e2, None, qa, qb, eta, Z2, 3.0, 1.0, value_planes=vs, tau_v=2.0, v_mean=O.block_means(Vs))
     assert np.allclose(Ar, Ab, rtol=1e-12) and np.array_equal(Lr, Lb)
+
+
+# --------------------------------------------------------------------------- cascades on two-plane keys
+def _cascade_inputs(B=6, G=2, D=64, n_prefix=150, suffixes=(40, 0, 7, 64, 1, 90)):
+    q = rng_rows(31, B * G, D).reshape(B, G, D)
+    qa, qb, qe = P.quantize_rows(q.reshape(B * G, D))
+    qa = qa.reshape(B, G, D); qb = qb.reshape(B, G, D)
+    eta = qe.reshape(B, G).astype(np.float64) * (O.LOG2E / math.sqrt(D))
+    kp = rng_rows(32, n_prefix, D); vp = rng_rows(33, n_prefix, D)
+    pre = P.quantize_rows(kp) + (vp,)
+    sufs = []
+    for b, n in enumerate(suffixes):
+        ks = rng_rows(40 + b, n, D) if n else np.zeros((0, D)); vs = rng_rows(60 + b, n, D) if n else np.zeros((0, D))
+        sufs.append((P.quantize_rows(ks) + (vs,)) if n else (np.zeros((0, D), np.int8), np.zeros((0, D), np.int8), np.zeros(0), vs))
+    return qa, qb, eta, pre, sufs
+
+
+def test_cascade_levels_add_up_to_the_flat_decode_when_no_gate_couples_the_rows():
+    """Prop. 1(i): partials of one row under one reference add.  Without refinement (tau < 0) no verdict couples a row's
+    scores to the other rows of its block, so the cascade -- any block size -- equals each request's flat decode over
+    prefix ++ suffix, at any depth."""
+    qa, qb, eta, pre, sufs = _cascade_inputs()
+    B, G, D = qa.shape
+    Z = np.array([[5.0 + 0.25 * b - 0.5 * g for g in range(G)] for b in range(B)])
+    for T in (math.inf, 6.0):
+        for block_rows in (16, 4, 1):
+            A, L, infos = P.fold_levels_planes([(B, [pre]), (1, sufs)], qa, qb, eta, Z, T, -1.0, block_rows)
+            for b in range(B):
+                ka = np.concatenate([pre[0], sufs[b][0]]); kb = np.concatenate([pre[1], sufs[b][1]])
+                ke = np.concatenate([pre[2], sufs[b][2]]); V = np.concatenate([pre[3], sufs[b][3]])
+                A1, L1, _ = P.fold_group_planes(ka, kb, ke, V, qa[b], qb[b], eta[b], Z[b], T, -1.0)
+                # (two orders of one sum: equal to rounding, measured against the row's largest entry)
+                assert np.abs(A[b] - A1).max() <= 1e-12 * np.abs(A1).max() and np.allclose(L[b], L1, rtol=1e-12)
+    # and with one level, one request per sequence, it IS fold_group_planes (any gate)
+    A, L, infos = P.fold_levels_planes([(1, sufs)], qa, qb, eta, Z, 5.0, 3.0)
+    for b in range(B):
+        if sufs[b][0].shape[0]:
+            A1, L1, _ = P.fold_group_planes(sufs[b][0], sufs[b][1], sufs[b][2], sufs[b][3], qa[b], qb[b], eta[b], Z[b], 5.0, 3.0)
+            assert np.array_equal(A[b], A1) and np.array_equal(L[b], L1)
+        else:
+            assert not A[b].any() and not L[b].any()
+
+
+def test_cascade_blocks_keep_their_verdicts_to_themselves_and_levels_take_their_own_gate():
+    qa, qb, eta, pre, sufs = _cascade_inputs(B=5, G=4, suffixes=(40, 0, 7, 64, 90))   # 20 stacked rows on the prefix: blocks of 16 and 4
+    B, G, D = qa.shape
+    Z = np.zeros((B, G))
+    for b in range(B):
+        for g in range(G):
+            Z[b, g] = P.coarse_scores(pre[0], pre[2], qa[b, g], qb[b, g], eta[b, g]).max() - 1.0
+    A, L, infos = P.fold_levels_planes([(B, [pre])], qa, qb, eta, Z, 6.0, 2.0)
+    assert [len(blk) for (_, _, blk, _) in infos] == [16, 4]
+    rows = [(b, g) for b in range(B) for g in range(G)]
+    assert infos[0][2] == rows[:16] and infos[1][2] == rows[16:]
+    # a block's refine verdicts are the OR over ITS rows only: recompute them from the coarse scores it reports
+    differ = False
+    for (_, _, blk, info) in infos:
+        own = (info["coarse"] >= -2.0).any(axis=0) & (info["coarse"] >= -6.0).any(axis=0)
+        assert np.array_equal(info["refine"], own)
+    differ = not np.array_equal(infos[0][3]["refine"], infos[1][3]["refine"])
+    assert differ                                               # the case tells blocks apart
+    # the automatic gate is the level's own: a 150-key prefix and a 90-key suffix both take max(log2 n - 2, 4) = 4 ... 5.2
+    A2, L2, infos2 = P.fold_levels_planes([(B, [pre]), (1, sufs)], qa, qb, eta, Z, math.inf, None)
+    for (li, j, blk, info) in infos2:
+        n = pre[0].shape[0] if li == 0 else sufs[j][0].shape[0]
+        tau = P.auto_refine_tau(n)
+        assert np.array_equal(info["refine"], (info["coarse"] >= -tau).any(axis=0) & info["live"])
