@@ -213,12 +213,15 @@ def test_host_checks_of_two_plane_keys():
     for field, value in [("z_mode", F.Z_EXACT_MAX), ("stack", 2)]:
         old = getattr(a, field)
         setattr(a, field, value)
-        if field == "stack":                                        # 2 requests x group 12 on one sequence: 16 rows is the
-            a.num_q_heads, a.num_kv_heads = 12, 1                   # limit, 24 are beyond it
+        if field == "stack":                                        # 2 requests x group 12 on one sequence: 24 rows are two
+            a.num_q_heads, a.num_kv_heads = 12, 1                   # 16-row blocks, and draft rows must stay within one
             a.kv.num_seqs = 1
+            masks = torch.ones(2, dtype=torch.int32)
+            a.draft_mask, a.draft_len = masks.data_ptr(), 2
         assert L.fold_decode(a, None) == F.FOLD_EUNSUPPORTED, field
         setattr(a, field, old)
         a.num_q_heads, a.num_kv_heads = 8, 2; a.kv.num_seqs = 2
+        a.draft_mask, a.draft_len = None, 0
     args2 = (F.FoldArgs * 2)(a, a)
     args2[1].kv.k_plane_a = None
     ptrs = (C.POINTER(F.FoldArgs) * 2)(C.pointer(args2[0]), C.pointer(args2[1]))
