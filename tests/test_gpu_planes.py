@@ -438,14 +438,14 @@ PLANE_LENGTHS = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255
 
 @pytest.mark.parametrize("seed", range(5))
 def test_random_shapes_match_the_oracle(seed):
-    """Seeded random shapes of the two-plane path: head dimension, rows per kv head (1..16), lengths around every tile /
+    """Seeded random shapes of the two-plane path: head dimension, rows per kv head (1..33: up to three 16-row blocks), lengths around every tile /
     chunk / estimator boundary, paged or contiguous, depth, refine gates, block tail, draft masks and E4M3 value planes drawn together."""
     import random
     rnd = random.Random(7300 + seed)
     for i in range(8):
         D = rnd.choice([64, 128])
         G, stack = rnd.choice([(1, 1), (2, 1), (3, 1), (4, 1), (8, 1), (5, 1), (1, 3), (2, 4), (4, 2), (1, 8), (2, 2),
-                               (16, 1), (9, 1), (4, 4), (2, 7), (3, 5), (1, 13), (12, 1)])
+                               (16, 1), (9, 1), (4, 4), (2, 7), (3, 5), (1, 13), (12, 1), (4, 5), (2, 12), (8, 3), (1, 33)])
         Hkv = rnd.choice([1, 2, 3])
         nseq = rnd.choice([1, 2, 3])
         lens = [rnd.choice(PLANE_LENGTHS) for _ in range(nseq)]
@@ -459,7 +459,7 @@ def test_random_shapes_match_the_oracle(seed):
         else:
             kw.update(capacity=max(lens) + rnd.choice([0, 5, 100]))
         tail = (not math.isinf(T)) and rnd.random() < 0.4
-        drafts = stack > 1 and rnd.random() < 0.5
+        drafts = stack > 1 and G * stack <= 16 and rnd.random() < 0.5        # (draft rows stay within one 16-row block)
         vfp8 = rnd.random() < 0.4                                # (with the tail: the format's own cut model, the mean row)
         tau_v = rnd.choice([0.0, 0.0, -1.0, 5.0, math.inf])
         case = dict(D=D, G=G, stack=stack, Hkv=Hkv, lens=lens, T=T, tau=tau, kw=kw, tail=tail, drafts=drafts, vfp8=vfp8, tau_v=tau_v)
