@@ -279,15 +279,19 @@ def fold_levels_planes(levels, qa, qb, eta, Z, T: float = math.inf, tau: Optiona
     that hold it): a sequence's rows -- request-major, the group's rows within a request -- are cut into blocks of
     `block_rows`, each block is `fold_group_planes` over its own rows (its verdicts ORed over the block), and
     tau = None takes `auto_refine_tau` of the LEVEL's own sequence length.  Partials of one row under one reference
-    add (Prop. 1(i)).  Returns (A [B, G, D], L [B, G], infos) with infos = [(level, sequence, rows of the block as
-    (b, g) pairs, info of fold_group_planes)]."""
+    add (Prop. 1(i)).  A sequence may carry a fifth entry, a dict of `fold_group_planes`' optional arguments for it
+    (`v_mean`: its block means; `value_planes`, `tau_v`: its E4M3 value planes and their gate, tau_v None = the
+    level's own `auto_refine_tau_v`; `v_run_mean`: its mean value row).  Returns (A [B, G, D], L [B, G], infos) with
+    infos = [(level, sequence, rows of the block as (b, g) pairs, info of fold_group_planes)]."""
     qa = np.asarray(qa); qb = np.asarray(qb)
     B, G, D = qa.shape
     A = np.zeros((B, G, D)); L = np.zeros((B, G))
     infos = []
     for li, (stack, seqs) in enumerate(levels):
         assert B % stack == 0 and len(seqs) == B // stack
-        for j, (ka, kb, ke, V) in enumerate(seqs):
+        for j, entry in enumerate(seqs):
+            ka, kb, ke, V = entry[:4]
+            extra = dict(entry[4]) if len(entry) > 4 else {}
             n = np.asarray(ka).shape[0]
             if n == 0:
                 continue
@@ -297,7 +301,7 @@ def fold_levels_planes(levels, qa, qb, eta, Z, T: float = math.inf, tau: Optiona
                 a, l, info = fold_group_planes(ka, kb, ke, V, np.stack([qa[b, g] for b, g in blk]), np.stack([qb[b, g] for b, g in blk]),
                                                np.array([eta[b][g] for b, g in blk], dtype=np.float64),
                                                np.array([Z[b][g] for b, g in blk], dtype=np.float64), T,
-                                               auto_refine_tau(n) if tau is None else tau)
+                                               auto_refine_tau(n) if tau is None else tau, **extra)
                 for i, (b, g) in enumerate(blk):
                     A[b, g] += a[i]; L[b, g] += l[i]
                 infos.append((li, j, blk, info))

@@ -684,11 +684,19 @@ def test_million_key_sequence_on_planes_and_value_planes():
 
 # ------------------------------------------------------------------ shared-prefix cascades on two-plane keys
 def _planes_cascade(B, Hq, Hkv, D, n_prefix, suffixes, seed, T, tau, z_mode=F.Z_ESTIMATE, z=None, paged=False, side=None,
-                    separate_calls=False):
+                    separate_calls=False, tail=False, vfp8=False):
+    """tail: every level carries its block means (the block tail); vfp8: every level's values are two E4M3 planes, and
+    with `tail` their cut model is the level sequences' mean value rows."""
     from paper_2609_33410_b200.workloads import make_cascade_workload
     kw = dict(paged=True, page_size=32) if paged else {}
     pre, suf = make_cascade_workload(B, Hq, Hkv, D, n_prefix, suffixes, seed=seed, device=DEV, poison_padding=True, **kw)
     cp, cs = plane_cache(pre), plane_cache(suf)
+    if vfp8:
+        value_planes_of(pre, cp); value_planes_of(suf, cs)
+        if tail:
+            F.fold_running_means(cp); F.fold_running_means(cs)
+    elif tail:
+        cp, cs = with_means(cp, oracle_block_means(pre)), with_means(cs, oracle_block_means(suf))
     bp, bs = F.alloc_buffers(pre.q, cp, stack=B), F.alloc_buffers(pre.q, cs)
     if z is not None:
         bs.z.copy_(z)
@@ -709,7 +717,7 @@ def _planes_cascade(B, Hq, Hkv, D, n_prefix, suffixes, seed, T, tau, z_mode=F.Z_
     return pre, suf, cp, cs, bp, bs
 
 
-def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
+def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate, tail=False, vfp8=False):
     """The oracle's cascade (`fold_levels_planes`: each level Algorithm 1 over its own rows in blocks of 16, the levels'
     (A, L) added, Eq. 3) at the GPU's own references and split query rows."""
     B, Hq, D = pre.q.shape
@@ -730,7 +738,15 @@ def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
             n = int(w.seqlens[seq])
             if n == 0:
                 return (np.zeros((0, D), np.int8), np.zeros((0, D), np.int8), np.zeros(0), np.zeros((0, D)))
-            return logical_planes(w, cache, seq, kvh) + (O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh))),)
+            extra = {}
+            if vfp8:
+                p1, p2 = logical_value_planes(w, cache, seq, kvh)
+                extra = dict(value_planes=(p1, p2, cache.v_scale_log2), tau_v=None)
+                if tail:
+                    extra["v_run_mean"] = cache.v_block_mean[seq, 0, kvh].float().cpu().numpy().astype(np.float64)
+            elif tail:
+                extra = dict(v_mean=cache.v_block_mean[seq, :(n + 63) // 64, kvh].float().cpu().numpy().astype(np.float64))
+            return logical_planes(w, cache, seq, kvh) + (O.widen_bf16(bf16_bits(w.logical_rows("v", seq, kvh))), extra)
 
         levels = [(B, [seq_of(pre, cp, 0)]), (1, [seq_of(suf, cs, b) for b in range(B)])]
         A, L, infos = P.fold_levels_planes(levels, qa[:, hs], qb[:, hs], eta[:, hs].astype(np.float64), z[:, hs], T,
@@ -739,7 +755,7 @@ def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
         slack = np.zeros((B, G)); vmax = np.zeros((B, G))
         s_all = [[[] for _ in range(G)] for _ in range(B)]
         for (li, j, blk, info) in infos:
-            ka, kb, ke, V = levels[li][1][j]
+            ka, kb, ke, V = levels[li][1][j][:4]
             n = ka.shape[0]
             tau_eff = P.auto_refine_tau(n) if tau == 0.0 else tau
             vinf = np.abs(V).max(axis=1)
@@ -751,7 +767,7 @@ def _compare_planes_cascade(pre, suf, cp, cs, bp, bs, T, tau, check_estimate):
                 s_fin = info["coarse"][i] + np.where(info["refine"], corr, 0.0)
                 p = np.exp2(s_fin)
                 near = near_T if math.isinf(T) else (near_T | (np.abs(s_fin + T) <= BAND))
-                slack[b, g] += float((p[near] * vinf[near]).sum())
+                slack[b, g] += (2.0 if tail else 1.0) * float((p[near] * vinf[near]).sum())   # (value <-> mean: twice)
                 slack[b, g] += float((p[near_tau] * (np.exp2(np.abs(corr[near_tau])) - 1.0) * vinf[near_tau]).sum())
                 s_all[b][g].append(P.refined_scores(ka, kb, ke, qa[b, kvh * G + g], qb[b, kvh * G + g], eta[b, kvh * G + g]))
         for b in range(B):
@@ -809,3 +825,16 @@ def test_cascade_on_two_plane_keys_head_dim_64_and_graph_replay():
     with pytest.raises(F.FoldError):
         F.fold_decode_cascade(mixed)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("tail,vfp8", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("B,Hq,Hkv,paged", [(4, 8, 2, False), (6, 4, 1, True)])
+def test_cascade_on_two_plane_keys_with_the_block_tail_and_e4m3_values(tail, vfp8, B, Hq, Hkv, paged):
+    # every level brings its own cut model (block means, or with 8-bit values the sequence's mean row) and value planes
+    suffixes = ([500, 1, 0, 257] * 2)[:B]
+    for T in (8.0, 14.0):
+        lv = _planes_cascade(B, Hq, Hkv, 128, 2000, suffixes, seed=151, T=T, tau=0.0, paged=paged, tail=tail, vfp8=vfp8)
+        _compare_planes_cascade(*lv, T=T, tau=0.0, check_estimate=True, tail=tail, vfp8=vfp8)
+        sp = _planes_cascade(B, Hq, Hkv, 128, 2000, suffixes, seed=151, T=T, tau=0.0, paged=paged, tail=tail, vfp8=vfp8,
+                             separate_calls=True)
+        assert same_bits(sp[5].out, lv[5].out) and same_bits(sp[5].lse, lv[5].lse)

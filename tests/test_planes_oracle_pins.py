@@ -446,6 +446,32 @@ def test_cascade_levels_add_up_to_the_flat_decode_when_no_gate_couples_the_rows(
             assert not A[b].any() and not L[b].any()
 
 
+def test_cascade_levels_carry_their_own_cut_models_and_value_planes():
+    """A sequence's optional arguments reach `fold_group_planes` unchanged: one level of unstacked requests with block
+    means / E4M3 value planes / a mean value row equals the direct call, and with constant values the block tail gives
+    a cascade's rows back exactly what its levels cut (A / L = the constant, Section 4 "Depth as a dial")."""
+    qa, qb, eta, pre, sufs = _cascade_inputs()
+    B, G, D = qa.shape
+    Z = np.array([[P.coarse_scores(pre[0], pre[2], qa[b, g], qb[b, g], eta[b, g]).max() for g in range(G)] for b in range(B)])
+    b0 = 3                                                      # a request with a 64-key suffix
+    ka, kb, ke, V = sufs[b0]
+    vm = O.block_means(V)
+    p1, p2 = P.quantize_values(V, -2)
+    for extra in (dict(v_mean=vm), dict(value_planes=(p1, p2, -2), tau_v=3.0), dict(value_planes=(p1, p2, -2), tau_v=None, v_run_mean=P.running_mean(V))):
+        seqs = [s if i != b0 else s + (extra,) for i, s in enumerate(sufs)]
+        A, L, _ = P.fold_levels_planes([(1, seqs)], qa, qb, eta, Z, 4.0, 2.0)
+        kw = dict(extra)
+        if "tau_v" in kw and kw["tau_v"] is None:
+            kw["tau_v"] = P.auto_refine_tau_v(ka.shape[0])
+        A1, L1, _ = P.fold_group_planes(ka, kb, ke, V, qa[b0], qb[b0], eta[b0], Z[b0], 4.0, 2.0, **kw)
+        assert np.array_equal(A[b0], A1) and np.array_equal(L[b0], L1)
+    const = lambda n: np.full((n, D), 1.5)
+    pre_c = pre[:3] + (const(pre[0].shape[0]), dict(v_mean=O.block_means(const(pre[0].shape[0]))))
+    sufs_c = [s[:3] + (const(s[0].shape[0]), dict(v_mean=O.block_means(const(s[0].shape[0])))) if s[0].shape[0] else s for s in sufs]
+    A, L, _ = P.fold_levels_planes([(B, [pre_c]), (1, sufs_c)], qa, qb, eta, Z, 3.0, -1.0)
+    assert np.allclose(A / L[..., None], 1.5, rtol=1e-12)
+
+
 def test_cascade_blocks_keep_their_verdicts_to_themselves_and_levels_take_their_own_gate():
     qa, qb, eta, pre, sufs = _cascade_inputs(B=5, G=4, suffixes=(40, 0, 7, 64, 90))   # 20 stacked rows on the prefix: blocks of 16 and 4
     B, G, D = qa.shape
