@@ -353,9 +353,11 @@ int fold_quantize_values(const fold_kv *kv, int32_t num_kv_heads, int32_t head_d
  * copied as the single span its strides cover).  `staging` is DEVICE memory of at least
  * fold_host_staging_bytes(host_args) bytes, 256-byte aligned, which receives the copies,
  * the workspace and the results before they are copied back.  Everything is enqueued on
- * `stream`; the host buffers are valid after the caller synchronises the stream.  The block tail is
- * not offered here: kv.v_block_mean must be NULL (FOLD_EUNSUPPORTED otherwise); nor are draft masks
- * (draft_len must be 0) or two-plane keys (kv.k_plane_a must be NULL). */
+ * `stream`; the host buffers are valid after the caller synchronises the stream.  With two-plane keys (and
+ * E4M3 value planes) kv.k_plane_a / k_plane_b / k_scale (v_plane_1 / v_plane_2) are HOST pointers too and are copied
+ * as the spans their strides cover (a scale row up to the next multiple of 8 tokens); kv.k (kv.v) may then be NULL.
+ * The block tail is not offered here: kv.v_block_mean must be NULL (FOLD_EUNSUPPORTED otherwise); nor are draft
+ * masks (draft_len must be 0). */
 size_t fold_host_staging_bytes(const fold_args *host_args);
 int fold_decode_host(const fold_args *host_args, void *staging, size_t staging_bytes, fold_stream stream);
 

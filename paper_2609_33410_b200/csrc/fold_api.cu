@@ -1161,6 +1161,8 @@ namespace {
 struct HostPlan {
   size_t q, k, v, table, lens, z, out, lse, status, ws, total;
   size_t q_bytes, kv_bytes, table_bytes, lens_bytes, rows;
+  // two-plane keys (and E4M3 value planes): the planes' spans and the scales' span
+  size_t pa, pb, sc, v1, v2, plane_bytes, scale_bytes;
 };
 size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 bool plan_host(const fold_args *a, HostPlan *h) {
@@ -1176,10 +1178,22 @@ bool plan_host(const fold_args *a, HostPlan *h) {
   h->kv_bytes = (size_t)span * 2;
   h->table_bytes = paged ? (size_t)kv.num_seqs * kv.max_pages_per_seq * 4 : 0;
   h->lens_bytes = (size_t)kv.num_seqs * 4;
+  h->plane_bytes = h->scale_bytes = 0;
+  if (kv.k_plane_a) {                                        // one byte per code; a scale row is readable up to the next 8 tokens
+    h->plane_bytes = (size_t)((outer - 1) * kv.plane_stride_seq + (toks - 1) * kv.plane_stride_tok +
+                              (long long)(a->num_kv_heads - 1) * kv.plane_stride_head + a->head_dim);
+    h->scale_bytes = (size_t)((outer - 1) * kv.scale_stride_seq + (long long)(a->num_kv_heads - 1) * kv.scale_stride_head +
+                              ((toks + 7) & ~7LL)) * 2;
+  }
   size_t o = 0;
   h->q = o; o += up256(h->q_bytes);
-  h->k = o; o += up256(h->kv_bytes);
-  h->v = o; o += up256(h->kv_bytes);
+  h->k = o; o += kv.k ? up256(h->kv_bytes) : 0;              // (with two-plane keys the BF16 keys may be absent,
+  h->v = o; o += kv.v ? up256(h->kv_bytes) : 0;              //  with E4M3 value planes the BF16 values)
+  h->pa = o; o += up256(h->plane_bytes);
+  h->pb = o; o += up256(h->plane_bytes);
+  h->sc = o; o += up256(h->scale_bytes);
+  h->v1 = o; o += kv.v_plane_1 ? up256(h->plane_bytes) : 0;
+  h->v2 = o; o += kv.v_plane_1 ? up256(h->plane_bytes) : 0;
   h->table = o; o += up256(h->table_bytes);
   h->lens = o; o += up256(h->lens_bytes);
   h->z = o; o += up256(h->rows * 4);
@@ -1200,18 +1214,29 @@ size_t fold_host_staging_bytes(const fold_args *host_args) {
 
 int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, fold_stream stream) {
   if (!ha || !staging || !aligned(staging, 256)) return FOLD_EINVAL;
-  if (!ha->q || !ha->kv.k || !ha->kv.v || !ha->kv.seqlens || !ha->out) return FOLD_EINVAL;
+  const bool planes = ha->kv.k_plane_a != nullptr, vplanes = ha->kv.v_plane_1 != nullptr;
+  if (!ha->q || !ha->kv.seqlens || !ha->out) return FOLD_EINVAL;
+  if ((!ha->kv.k && !planes) || (!ha->kv.v && !vplanes)) return FOLD_EINVAL;
+  if (planes && (!ha->kv.k_plane_b || !ha->kv.k_scale)) return FOLD_EINVAL;
+  if (vplanes && (!planes || !ha->kv.v_plane_2)) return planes ? FOLD_EINVAL : FOLD_EUNSUPPORTED;
   if (ha->z_mode == FOLD_Z_GIVEN && !ha->z) return FOLD_EINVAL;
   if (ha->kv.v_block_mean) return FOLD_EUNSUPPORTED;        // the block tail is not offered for host buffers
   if (ha->draft_len != 0) return FOLD_EUNSUPPORTED;         // nor are draft masks
-  if (ha->kv.k_plane_a) return FOLD_EUNSUPPORTED;           // nor two-plane keys
   HostPlan h;
   if (fold_workspace_bytes(ha) == 0 || !plan_host(ha, &h)) return FOLD_EINVAL;
   if (staging_bytes < h.total) return FOLD_EWORKSPACE;
   uint8_t *d = static_cast<uint8_t *>(staging);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   fold_args da = *ha;
-  da.q = d + h.q; da.kv.k = d + h.k; da.kv.v = d + h.v;
+  da.q = d + h.q;
+  da.kv.k = ha->kv.k ? d + h.k : nullptr;
+  da.kv.v = ha->kv.v ? d + h.v : nullptr;
+  if (planes) {
+    da.kv.k_plane_a = reinterpret_cast<const int8_t *>(d + h.pa);
+    da.kv.k_plane_b = reinterpret_cast<const int8_t *>(d + h.pb);
+    da.kv.k_scale = d + h.sc;
+  }
+  if (vplanes) { da.kv.v_plane_1 = d + h.v1; da.kv.v_plane_2 = d + h.v2; }
   da.kv.page_table = ha->kv.page_table ? reinterpret_cast<const int32_t *>(d + h.table) : nullptr;
   da.kv.seqlens = reinterpret_cast<const int32_t *>(d + h.lens);
   da.z = reinterpret_cast<float *>(d + h.z);
@@ -1224,8 +1249,17 @@ int fold_decode_host(const fold_args *ha, void *staging, size_t staging_bytes, f
   if (int rc = check_args(&da, &g, true)) return rc;
   bool ok = true;
   ok &= cudaMemcpyAsync(d + h.q, ha->q, h.q_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d + h.k, ha->kv.k, h.kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d + h.v, ha->kv.v, h.kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (ha->kv.k) ok &= cudaMemcpyAsync(d + h.k, ha->kv.k, h.kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (ha->kv.v) ok &= cudaMemcpyAsync(d + h.v, ha->kv.v, h.kv_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (planes) {
+    ok &= cudaMemcpyAsync(d + h.pa, ha->kv.k_plane_a, h.plane_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + h.pb, ha->kv.k_plane_b, h.plane_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + h.sc, ha->kv.k_scale, h.scale_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  if (vplanes) {
+    ok &= cudaMemcpyAsync(d + h.v1, ha->kv.v_plane_1, h.plane_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + h.v2, ha->kv.v_plane_2, h.plane_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
   if (h.table_bytes)
     ok &= cudaMemcpyAsync(d + h.table, ha->kv.page_table, h.table_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
   ok &= cudaMemcpyAsync(d + h.lens, ha->kv.seqlens, h.lens_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;

@@ -838,3 +838,30 @@ def test_cascade_on_two_plane_keys_with_the_block_tail_and_e4m3_values(tail, vfp
         sp = _planes_cascade(B, Hq, Hkv, 128, 2000, suffixes, seed=151, T=T, tau=0.0, paged=paged, tail=tail, vfp8=vfp8,
                              separate_calls=True)
         assert same_bits(sp[5].out, lv[5].out) and same_bits(sp[5].lse, lv[5].lse)
+
+
+@pytest.mark.parametrize("vfp8", [False, True])
+@pytest.mark.parametrize("paged", [False, True])
+def test_host_buffer_entry_point_takes_the_two_plane_format(vfp8, paged):
+    # the planes, scales (and value planes) are copied from pinned host memory like the BF16 tensors: same bits as the
+    # device path on the same codes
+    kw = dict(paged=True, page_size=64) if paged else dict(capacity=2600)
+    w = make_decode_workload(2, 8, 2, 128, [2500, 700], seed=163, device=DEV, **kw)
+    cache = plane_cache(w)
+    if vfp8:
+        value_planes_of(w, cache)
+    ref = run_planes(w, cache, T=16.0)
+    pin = lambda t: None if t is None else t.cpu().pin_memory()
+    hcache = F.KVCache(pin(w.k), pin(w.v), pin(w.seqlens), w.max_seqlen, pin(w.page_table), None, pin(cache.k_plane_a),
+                       pin(cache.k_plane_b), pin(cache.k_scale), pin(cache.v_plane_1), pin(cache.v_plane_2), cache.v_scale_log2)
+    hq = w.q.cpu().pin_memory()
+    hout = torch.empty(2, 8, 128, dtype=torch.bfloat16).pin_memory()
+    hlse = torch.empty(2, 8, dtype=torch.float32).pin_memory()
+    hz = torch.empty(2, 8, dtype=torch.float32).pin_memory()
+    hst = torch.empty(2, 8, dtype=torch.int32).pin_memory()
+    args = F.make_args(hq, hcache, scale=w.scale, depth_T=16.0, z=hz, out=hout, lse=hlse, row_status=hst)
+    staging = torch.empty(F.fold_host_staging_bytes(args), dtype=torch.uint8, device=DEV)
+    F.fold_decode_host(args, staging)
+    torch.cuda.synchronize()
+    assert same_bits(hout, ref.out.cpu()) and same_bits(hlse, ref.lse.cpu()) and same_bits(hz, ref.z.cpu())
+    assert not hst.any()
